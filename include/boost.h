@@ -1,0 +1,295 @@
+/*
+ * boost.h - C ABI of the tiered decode hot path (BOOST, arxiv 2609.13592) for NVIDIA B200.
+ *
+ * Every buffer is cut into 2 MiB pages that live in one of two tiers: HBM, or
+ * pinned host memory that the GPU reads with ordinary loads over the CPU-GPU
+ * link.  Pages are placed so that every wave of threadblocks reads both tiers
+ * at once and in proportion to their bandwidths; each threadblock stays on one
+ * tier for a whole work item.
+ *
+ * Conventions
+ *   - plain C; every call returns BOOST_OK (0) or a negative BOOST_ERR_* code;
+ *     no exception crosses the boundary;
+ *   - the library never allocates or frees device or pinned memory: callers
+ *     pass pointers and sizes.  "host" / "device" beside an argument says in
+ *     which address space the pointer must be valid for the library's own
+ *     reads and writes (host = dereferenced on the CPU inside the call;
+ *     device = dereferenced by kernels);
+ *   - kernel launches are asynchronous on the given stream (a cudaStream_t
+ *     passed as void*; NULL is the default stream);
+ *   - `workspace` arguments are scratch in device memory owned by the caller.
+ *     A workspace must be zero-filled once before its first use; kernels leave
+ *     the counters in it at zero when they finish, so the same workspace can be
+ *     reused by later calls on the same stream.  Calls that may overlap on the
+ *     GPU need separate workspaces;
+ *   - handles (boost_kv_pool_t) are not thread safe.
+ */
+#ifndef BOOST_H_
+#define BOOST_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define BOOST_PAGE_BYTES 2097152u /* 2 MiB pages (Sec. 1, Sec. 2.6) */
+#define BOOST_KV_BLOCK_TOKENS 16u /* tokens per KV block (Sec. 4.3) */
+
+enum {
+  BOOST_OK = 0,
+  BOOST_ERR_INVALID = -1,  /* bad argument, unknown request, double free */
+  BOOST_ERR_NOMEM = -2,    /* KV pool exhausted: the scheduler must decide (Sec. 4.3) */
+  BOOST_ERR_ALIGN = -3,    /* pointer or size not aligned as documented */
+  BOOST_ERR_CUDA = -4,     /* a CUDA runtime call failed; see boost_last_cuda_error() */
+  BOOST_ERR_CAPACITY = -5, /* an output or workspace buffer is too small */
+  BOOST_ERR_UNSUPPORTED = -6
+};
+
+enum { BOOST_TIER_HBM = 0, BOOST_TIER_HOST = 1 };
+
+enum {
+  BOOST_POLICY_MODULO = 0,     /* K pages HBM, then one page host, repeating (Sec. 3.1) */
+  BOOST_POLICY_CONTIGUOUS = 1, /* head of the range HBM, tail host (Sec. 4.2, Sec. 5.7) */
+  BOOST_POLICY_RANDOM = 2      /* every page host with the target probability (Sec. 2.6) */
+};
+
+/* boost_place_pages flag: a wave of `wave_size` pages is shorter than one period, so
+ * not every wave can contain a host page (the precondition of Sec. 3.1 fails). */
+#define BOOST_FLAG_WAVE_SHORTER_THAN_PERIOD 1u
+
+/* CUDA error code (cudaError_t as int) of the most recent BOOST_ERR_CUDA on this thread. */
+int boost_last_cuda_error(void);
+
+/* ------------------------------------------------------------------ placement */
+
+/* Period M of the modulo rule for a host share of all pages `host_ratio` (= 1/M):
+ * the smallest M with 1/M <= host_ratio * (1 + 2^-40), so the host share never
+ * exceeds the request (rounding rule of Sec. 4.4).  host_ratio = 0 gives M = 0
+ * (no host pages).  host_ratio must be 0 or lie in [2^-30, 1/2]. */
+int boost_modulus_from_ratio(double host_ratio, uint32_t* modulus_out /*host*/);
+
+/* M = ceil(hbm_bw / link_bw) + 1: K = ceil(1/alpha) pages of HBM, then one host page
+ * (Sec. 3.1, Sec. 4.4).  Any unit, both > 0. */
+int boost_modulus_from_bandwidths(double hbm_bw, double link_bw, uint32_t* modulus_out /*host*/);
+
+/* Page-to-tier table of one tensor under modulo placement (Sec. 3.1).
+ *   buffer      only checked for 2 MiB alignment (may be NULL to skip the check);
+ *   bytes       size of the tensor; P = ceil(bytes / 2 MiB) pages;
+ *   host_ratio  share of all pages that go to the host tier (see above);
+ *   wave_size   pages one wave of threadblocks covers; does not change the table,
+ *               only sets BOOST_FLAG_WAVE_SHORTER_THAN_PERIOD (0 = unknown);
+ *   tier_out    host array of tier_cap bytes; entry i = BOOST_TIER_* of page i;
+ *   n_pages_out receives P.
+ * Page i is a host page iff (i mod M) == M-1.  The function keeps no state, so the
+ * pattern restarts for every tensor (Sec. 3.1).
+ * Errors: INVALID (null outputs, bad ratio), ALIGN, CAPACITY (tier_cap < P). */
+int boost_place_pages(const void* buffer, size_t bytes, double host_ratio, uint32_t wave_size,
+                      uint8_t* tier_out /*host*/, size_t tier_cap, size_t* n_pages_out /*host*/);
+
+/* As boost_place_pages with the comparison policies and superpages.
+ *   policy           BOOST_POLICY_*;
+ *   seed             used by RANDOM only: page i is host iff
+ *                    mix(seed + (i+1)*0x9E3779B97F4A7C15) < floor(2^64 / M), mix being the
+ *                    SplitMix64 output function;
+ *   superpage_pages  S >= 1: groups of S consecutive pages share a tier and the modulo
+ *                    rule runs over groups (Sec. 3.2, Sec. 4.4); MODULO only;
+ *   flags_out        may be NULL.
+ * CONTIGUOUS puts floor(P/M) pages, the last ones, on the host. */
+int boost_place_pages_ex(const void* buffer, size_t bytes, double host_ratio, uint32_t wave_size,
+                         int policy, uint64_t seed, uint32_t superpage_pages,
+                         uint8_t* tier_out /*host*/, size_t tier_cap, size_t* n_pages_out /*host*/,
+                         uint32_t* flags_out /*host*/);
+
+/* Host share of every wave when tiles are handed out in address order (Sec. 2.2, Sec. 2.6). */
+typedef struct {
+  uint64_t n_waves;
+  uint64_t n_host_pages;
+  uint64_t n_zero_waves; /* waves that touch no host tile */
+  uint64_t n_over_waves; /* waves whose host share exceeds host_ratio */
+  double mean, var, min, max; /* of the per-wave host share; var is the population variance */
+} boost_wave_stats_t;
+
+/* tile_bytes must divide 2 MiB; wave w holds tiles [w*G, (w+1)*G), G = ctas_per_wave; the
+ * last wave may be short (Sec. 4.4). */
+int boost_wave_stats(const uint8_t* tier /*host*/, size_t n_pages, size_t tile_bytes,
+                     uint32_t ctas_per_wave, double host_ratio, boost_wave_stats_t* out /*host*/);
+
+/* Visit order for tier-specialised kernels: host pages first (ascending), then HBM pages
+ * (ascending).  Each threadblock works on one tier at a time (Sec. 3.2); handing out the
+ * slow tier's pages first keeps both tiers busy for the whole kernel.
+ * order_out: host array of n_pages entries; n_host_out receives the number of host pages. */
+int boost_tier_order(const uint8_t* tier /*host*/, size_t n_pages, uint32_t* order_out /*host*/,
+                     size_t* n_host_out /*host*/);
+
+/* ------------------------------------------------------------ materialisation */
+
+/* Device-visible address of a pinned (page-locked) host allocation; INVALID when the
+ * pointer is not pinned host memory that the current device can address. */
+int boost_host_device_pointer(void* pinned_host, void** device_ptr_out /*host*/);
+
+/* Page base addresses for a placed tensor (the analogue of binding each 2 MiB region to a
+ * memory node, Sec. 4.4).  HBM pages take consecutive 2 MiB slots of hbm_slab, host pages
+ * consecutive slots of host_slab, both in page order.
+ *   hbm_slab / host_slab  device-visible base addresses, 2 MiB aligned; a slab may be NULL
+ *                         when its tier holds no page; *_slab_bytes are their capacities;
+ *   page_ptr_out          host array of n_pages pointers. */
+int boost_page_table(const uint8_t* tier /*host*/, size_t n_pages, void* hbm_slab,
+                     size_t hbm_slab_bytes, void* host_slab, size_t host_slab_bytes,
+                     void** page_ptr_out /*host*/);
+
+/* Copy a contiguous device buffer of `bytes` into its pages (page i receives bytes
+ * [i*2MiB, (i+1)*2MiB)), or back.  src/dst device; page_ptr device array. bytes % 16 == 0. */
+int boost_scatter_pages(const void* src /*device*/, size_t bytes,
+                        const void* const* page_ptr /*device*/, size_t n_pages, void* stream);
+int boost_gather_pages(void* dst /*device*/, size_t bytes, const void* const* page_ptr /*device*/,
+                       size_t n_pages, void* stream);
+
+/* ------------------------------------------------------------------- KV pool */
+
+typedef struct boost_kv_pool boost_kv_pool_t;
+
+typedef struct {
+  uint32_t n_blocks, n_kv_heads, host_modulus, chunk_bytes;
+  uint32_t n_pages;          /* pages of one K (or V) tensor of one layer */
+  uint32_t n_host_pages;     /* the last n_host_pages pages are host pages (Sec. 4.2) */
+  uint32_t host_heads_lo;    /* host heads of a "lo" block; a "hi" block has one more */
+  uint32_t first_hi_block;   /* blocks >= this index are "hi" blocks */
+  uint32_t free_lo, free_hi; /* free blocks of each kind */
+  uint32_t live_blocks, n_requests;
+  uint64_t live_host_chunks, live_chunks; /* (head, block) chunks of live blocks */
+} boost_kv_pool_info_t;
+
+/* Wave-aware pool of KV blocks (Sec. 4.3, Sec. 4.5).
+ * Geometry: per layer and per K/V the cache is [n_kv_heads][n_blocks][16 tokens][D] with
+ * heads outermost; chunk (h, b) is chunk_bytes long at byte offset (h*n_blocks + b) *
+ * chunk_bytes.  n_blocks*chunk_bytes must be a multiple of 2 MiB so heads never share a
+ * page.  The tensor is placed linearly: its last floor(P/host_modulus) pages are host
+ * pages (host_modulus 0 = none; 1 is rejected).  A block therefore has host_heads_lo or
+ * host_heads_lo+1 of its heads on the host ("lo" and "hi" blocks).
+ * Policy: one FIFO free list per kind, ascending at start.  A request's first allocation
+ * fixes its kind: "hi" iff free_hi / (free_lo+free_hi) exceeds the target share of hi
+ * blocks (n_kv_heads - host_heads_lo*host_modulus) / host_modulus, else "lo".  Blocks
+ * come from the list of the request's kind; when that list is empty the block comes from
+ * the other list and the request keeps that kind from then on. */
+int boost_kv_pool_create(uint32_t n_blocks, uint32_t n_kv_heads, uint32_t host_modulus,
+                         uint32_t chunk_bytes, boost_kv_pool_t** pool_out /*host*/);
+
+/* Give `n` (>= 1) blocks to `request_id`, creating the request on first use.
+ * block_ids_out: host array of n entries.  NOMEM when fewer than n blocks are free in
+ * total; the pool is then unchanged. */
+int boost_kv_pool_alloc(boost_kv_pool_t* pool, uint64_t request_id, uint32_t n,
+                        int32_t* block_ids_out /*host*/);
+
+/* Return all blocks of a request to the tail of their lists, in the order they were
+ * handed out.  INVALID for an unknown (or already freed) request. */
+int boost_kv_pool_free(boost_kv_pool_t* pool, uint64_t request_id);
+
+int boost_kv_pool_query(const boost_kv_pool_t* pool, boost_kv_pool_info_t* info_out /*host*/);
+
+/* Kind (0 = lo, 1 = hi) a live request currently draws from. */
+int boost_kv_pool_request_kind(const boost_kv_pool_t* pool, uint64_t request_id,
+                               int* kind_out /*host*/);
+
+/* Tier of every page of one K (or V) tensor of one layer. */
+int boost_kv_pool_page_tiers(const boost_kv_pool_t* pool, uint8_t* tier_out /*host*/,
+                             size_t tier_cap, size_t* n_pages_out /*host*/);
+
+int boost_kv_pool_destroy(boost_kv_pool_t* pool);
+
+/* ------------------------------------------------------------------- kernels */
+
+/* Streaming read of a paged bf16 buffer: per_page_sum[i] = sum of the 1 Mi bf16 values of
+ * page i, accumulated in fp32 (the "add" micro-benchmark of Sec. 2.6 with a sum as its
+ * trivial compute).  Threadblocks take 128 KiB tiles of pages in `order`; a fixed share of
+ * the blocks starts on the host pages (Sec. 3.2) and all tiles of a page are combined in
+ * a fixed order, so results do not depend on scheduling.
+ *   page_ptr      device array of n_pages page addresses;
+ *   order         device array from boost_tier_order (host pages first);
+ *   per_page_sum  device array of n_pages floats;
+ *   workspace     device, >= boost_stream_reduce_workspace_bytes(n_pages). */
+size_t boost_stream_reduce_workspace_bytes(size_t n_pages);
+int boost_stream_reduce_tiered(const void* const* page_ptr /*device*/,
+                               const uint32_t* order /*device*/, size_t n_pages,
+                               size_t n_host_pages, float* per_page_sum /*device*/,
+                               void* workspace /*device*/, size_t workspace_bytes, void* stream);
+
+/* Weight tensors are stored in pages as a stream of 16 KiB blocks.  Block (t, kb) holds
+ * rows [128 t, 128 t + 128) and columns [64 kb, 64 kb + 64) of the row-major [N, K] bf16
+ * matrix W (zero padded), at byte offset (t * ceil(K/64) + kb) * 16 KiB of the tensor; row
+ * r of the block occupies 128 bytes at r*128 and its 16-byte chunk c sits at position
+ * c ^ (r & 7) (the 128-byte shared-memory swizzle), so one bulk copy brings a block into
+ * shared memory ready for the tensor cores.  A threadblock streams a run of blocks of one
+ * row tile from one page, i.e. a contiguous region of one tier (Sec. 3.1, Sec. 3.2). */
+typedef struct {
+  uint32_t n_row_tiles;     /* ceil(N / 128) */
+  uint32_t k_blocks;        /* ceil(K / 64) */
+  uint32_t blocks_per_item; /* run length L: divides 128 and k_blocks */
+  uint32_t splits;          /* k_blocks / L partial sums per row tile */
+  uint64_t bytes;           /* n_row_tiles * k_blocks * 16 KiB */
+  uint64_t n_pages;
+} boost_weight_layout_t;
+
+int boost_weight_layout(uint32_t N, uint32_t K, boost_weight_layout_t* out /*host*/);
+
+/* Write the packed form of row-major W [N, K] (device, bf16) into its pages. */
+int boost_pack_weights(const void* w_row_major /*device*/, uint32_t N, uint32_t K,
+                       const void* const* w_page_ptr /*device*/, size_t n_pages, void* stream);
+
+/* y[m, n] = sum_k x[m, k] * W[n, k] (+ residual[m, n]), fp32 accumulation: the
+ * weight-streaming product that dominates decode (Sec. 2.1, Sec. 3.1; the two-pointer
+ * handwritten matmul of Sec. 3.1 is the closest thing the paper describes).
+ *   w_page_ptr, w_order  device arrays for the packed weight (n_pages entries; order from
+ *                        boost_tier_order, host pages first);
+ *   x          device, bf16 row-major [M_b, K];  1 <= M_b <= 128;
+ *   y          device, row-major [M_b, N]; y_dtype 0 = fp32, 1 = bf16;
+ *   residual   device bf16 [M_b, N] added before the final rounding, or NULL;
+ *   workspace  device, >= boost_gemv_workspace_bytes(N, K, M_b).
+ * M_b <= 8 runs on CUDA cores with warp-shuffle reductions; larger batches use the tensor
+ * cores.  Split-K partial sums are combined in a fixed order by the last threadblock to
+ * finish a row tile, so the result is deterministic. */
+size_t boost_gemv_workspace_bytes(uint32_t N, uint32_t K, uint32_t M_b);
+int boost_gemv_tiered(const void* const* w_page_ptr /*device*/, const uint32_t* w_order /*device*/,
+                      size_t n_pages, size_t n_host_pages, uint32_t N, uint32_t K,
+                      const void* x /*device*/, uint32_t M_b, void* y /*device*/, int y_dtype,
+                      const void* residual /*device*/, void* workspace /*device*/,
+                      size_t workspace_bytes, void* stream);
+
+/* Copy a logical KV cache [n_kv_heads][n_pool_blocks][16][D] (contiguous device buffer,
+ * bf16) into the pages of a K or V tensor, or back.  Chunk (h, b) lands at byte offset
+ * (h*n_pool_blocks + b) * 4 KiB of the tensor; inside a chunk token t occupies 256 bytes at
+ * t*256 and its 16-byte piece c (8 values of d) sits at position c ^ (t & 7), which keeps
+ * tensor-core loads of 8 consecutive tokens on distinct shared-memory banks.  D = 128. */
+int boost_kv_scatter(const void* src /*device*/, uint32_t n_kv_heads, uint32_t n_pool_blocks,
+                     uint32_t D, const void* const* page_ptr /*device*/, size_t n_pages, void* stream);
+int boost_kv_gather(void* dst /*device*/, uint32_t n_kv_heads, uint32_t n_pool_blocks, uint32_t D,
+                    const void* const* page_ptr /*device*/, size_t n_pages, void* stream);
+
+/* One decode step of softmax attention over the paged KV cache of a boost_kv_pool
+ * (Sec. 3.3: threadblocks work on KV head chunks; chunks of host-resident heads are
+ * started first).
+ *   q            device bf16 [B, Hq, D];  D = 128;  Hq/Hkv in 1..16;
+ *   k_page_ptr, v_page_ptr  device arrays of page addresses of the K and V tensors, each
+ *                laid out [Hkv][n_pool_blocks][16][D] (chunk (h, b) at (h*n_pool_blocks+b)*4 KiB,
+ *                chunk-internal layout as written by boost_kv_scatter);
+ *   kv_tier      host array, tier of each of the n_kv_pages pages, or NULL (all HBM); must be
+ *                a linear placement (HBM pages, then host pages), else UNSUPPORTED;
+ *   block_table  device int32 [B, max_blocks]; ctx_lens device int32 [B] (tokens cached,
+ *                the current one included); query head j reads KV head j / (Hq/Hkv);
+ *   out          device bf16 [B, Hq, D];
+ *   workspace    device, >= boost_paged_attn_workspace_bytes(B, Hq, D, max_blocks). */
+size_t boost_paged_attn_workspace_bytes(uint32_t B, uint32_t Hq, uint32_t D, uint32_t max_blocks);
+int boost_paged_attn_decode_tiered(const void* q /*device*/, const void* const* k_page_ptr /*device*/,
+                                   const void* const* v_page_ptr /*device*/,
+                                   const uint8_t* kv_tier /*host*/, size_t n_kv_pages,
+                                   uint32_t n_pool_blocks, const int32_t* block_table /*device*/,
+                                   uint32_t max_blocks, const int32_t* ctx_lens /*device*/,
+                                   uint32_t B, uint32_t Hq, uint32_t Hkv, uint32_t D, float scale,
+                                   void* workspace /*device*/, size_t workspace_bytes,
+                                   void* out /*device*/, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* BOOST_H_ */

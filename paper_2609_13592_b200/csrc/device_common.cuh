@@ -1,0 +1,175 @@
+// Device-side building blocks shared by the kernels: mbarrier / bulk-copy / cp.async
+// wrappers (inline PTX for sm_100a), bounded waits, bf16 unpacking, work queues.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/boost.h"
+
+namespace boostk {
+
+constexpr uint32_t kPageBytes = BOOST_PAGE_BYTES;
+
+// Words at the start of every kernel workspace.
+enum : uint32_t {
+  kWsStatus = 0,    // sticky error bits, see kErr*
+  kWsHostNext = 1,  // next item of the host-tier queue
+  kWsHbmNext = 2,   // next item of the HBM queue
+  kWsDone = 3,      // threadblocks that have finished (self-reset of the words above)
+  kWsHeaderWords = 16
+};
+enum : uint32_t { kErrWaitTimeout = 1u, kErrBadIndex = 2u };
+
+// A wait that cannot hang the GPU: give up after about a second and record it.
+constexpr long long kWaitLimitCycles = 2000000000LL;
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return (uint32_t)__cvta_generic_to_shared(p);
+}
+
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void fence_barrier_init() {
+  asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes)
+               : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait on an mbarrier phase.  On a timeout the error is recorded in *status and the
+// caller simply carries on (its data is wrong, the host sees the status word), so that no
+// thread is left behind waiting for an arrival that never comes.
+__device__ __forceinline__ void mbar_wait(uint64_t* bar, uint32_t parity, uint32_t* status) {
+  if (mbar_try_wait(bar, parity)) return;
+  const long long t0 = clock64();
+  while (!mbar_try_wait(bar, parity)) {
+    if (clock64() - t0 > kWaitLimitCycles) {
+      atomicOr(status, kErrWaitTimeout);
+      return;
+    }
+  }
+}
+
+// Bulk asynchronous copy global -> shared through the TMA unit; completion is counted in
+// bytes on `bar`.  All three addresses 16-byte aligned, bytes a multiple of 16.
+__device__ __forceinline__ void bulk_copy_g2s(void* dst_smem, const void* src, uint32_t bytes,
+                                              uint64_t* bar) {
+  asm volatile(
+      "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+          smem_u32(dst_smem)),
+      "l"(src), "r"(bytes), "r"(smem_u32(bar))
+      : "memory");
+}
+
+// 16-byte asynchronous copy through the load/store path (works on any mapped address,
+// host-pinned pages included); src_bytes = 0 writes zeros.
+__device__ __forceinline__ void cp_async_16(void* dst_smem, const void* src, uint32_t src_bytes) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(smem_u32(dst_smem)), "l"(src),
+               "r"(src_bytes)
+               : "memory");
+}
+// Arrive on `bar` once all cp.async issued so far by this thread have landed (the arrival
+// is one of the barrier's expected arrivals).
+__device__ __forceinline__ void cp_async_arrive_noinc(uint64_t* bar) {
+  asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
+
+__device__ __forceinline__ void named_barrier_sync(uint32_t id, uint32_t n_threads) {
+  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(n_threads) : "memory");
+}
+
+__device__ __forceinline__ uint4 ld_stream_16(const void* p) {
+  uint4 v;
+  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+               : "l"(p));
+  return v;
+}
+
+// Two bf16 packed in a 32-bit word -> two floats (bf16 is the top half of an fp32).
+__device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xFFFF0000u); }
+
+__device__ __forceinline__ void ldmatrix_x4(uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3,
+                                            uint32_t smem_addr) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
+               : "r"(smem_addr));
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t& r0, uint32_t& r1, uint32_t& r2,
+                                                  uint32_t& r3, uint32_t smem_addr) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
+               : "r"(smem_addr));
+}
+// D (16x8, fp32) += A (16x16, bf16, row) * B (16x8, bf16, col)
+__device__ __forceinline__ void mma_bf16_16816(float (&d)[4], const uint32_t (&a)[4], uint32_t b0,
+                                               uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
+      "{%0,%1,%2,%3};"
+      : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+
+// Two work queues in the workspace header: threadblocks with `host_first` take items of the
+// host-tier queue [0, n_host_items) until it is empty and then help with the HBM queue
+// [n_host_items, n_items); the others do the reverse.  Returns the queue position or
+// 0xFFFFFFFF when both queues are empty.  Called by one thread per threadblock.
+struct TierQueues {
+  uint32_t* ws;
+  uint32_t n_host_items, n_items;
+  bool host_first;
+  bool host_open, hbm_open;
+  __device__ __forceinline__ void init(uint32_t* workspace, uint32_t n_host, uint32_t n_all, bool hf) {
+    ws = workspace; n_host_items = n_host; n_items = n_all; host_first = hf;
+    host_open = n_host > 0; hbm_open = n_all > n_host;
+  }
+  __device__ __forceinline__ uint32_t take_host() {
+    if (!host_open) return 0xFFFFFFFFu;
+    const uint32_t i = atomicAdd(ws + kWsHostNext, 1u);
+    if (i < n_host_items) return i;
+    host_open = false;
+    return 0xFFFFFFFFu;
+  }
+  __device__ __forceinline__ uint32_t take_hbm() {
+    if (!hbm_open) return 0xFFFFFFFFu;
+    const uint32_t i = atomicAdd(ws + kWsHbmNext, 1u);
+    if (i < n_items - n_host_items) return n_host_items + i;
+    hbm_open = false;
+    return 0xFFFFFFFFu;
+  }
+  __device__ __forceinline__ uint32_t next() {
+    uint32_t q = host_first ? take_host() : take_hbm();
+    if (q == 0xFFFFFFFFu) q = host_first ? take_hbm() : take_host();
+    return q;
+  }
+  // Last threadblock out puts the queue words back to zero for the next launch.
+  __device__ __forceinline__ void finish(uint32_t n_ctas) {
+    __threadfence();
+    const uint32_t d = atomicAdd(ws + kWsDone, 1u);
+    if (d == n_ctas - 1) {
+      ws[kWsHostNext] = 0; ws[kWsHbmNext] = 0; ws[kWsDone] = 0;
+      __threadfence();
+    }
+  }
+};
+
+}  // namespace boostk

@@ -1,0 +1,454 @@
+// Tiered weight-streaming product y = x W^T (GEMV at batch 1, skinny GEMM above) and the
+// kernel that packs a row-major weight into its paged 16 KiB-block form.
+//
+// One persistent threadblock per SM.  A producer warp walks the work queue (host-tier items
+// first, Sec. 3.2) and fills a ring of shared-memory stages: a 16 KiB weight block arrives
+// by one bulk copy through the TMA unit when its page is in HBM, or by a deep fan of
+// 16-byte cp.async loads when the page is host memory behind the CPU-GPU link; the matching
+// 64-column slice of x rides along by cp.async.  Eight consumer warps multiply from shared
+// memory: on CUDA cores with warp-shuffle reductions for batches up to 8, with bf16
+// tensor-core MMAs above.  A work item is a run of blocks of one row tile inside one page,
+// so a threadblock reads one tier at a time.
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include "device_common.cuh"
+#include "host_common.h"
+
+namespace {
+
+using namespace boostk;
+
+constexpr uint32_t kBlockRows = 128;
+constexpr uint32_t kBlockK = 64;
+constexpr uint32_t kBlockBytes = kBlockRows * kBlockK * 2;      // 16 KiB
+constexpr uint32_t kBlocksPerPage = kPageBytes / kBlockBytes;   // 128
+constexpr uint32_t kConsumerWarps = 8;
+constexpr uint32_t kConsumerThreads = kConsumerWarps * 32;
+constexpr uint32_t kGemvThreads = kConsumerThreads + 32;
+constexpr uint32_t kMaxStages = 8;
+constexpr uint32_t kSmemBudget = 200u * 1024u;
+
+enum : uint32_t { kFlagFirst = 1u, kFlagLast = 2u, kFlagStop = 4u };
+
+struct GemvParams {
+  const void* const* w_page_ptr;
+  const uint32_t* w_order;
+  uint32_t n_pages, n_host_pages;
+  uint32_t N, K, n_row_tiles, k_blocks, run, splits, items_per_page, n_items;
+  const __nv_bfloat16* x;
+  uint32_t M_b;
+  void* y;
+  int y_dtype;
+  const __nv_bfloat16* residual;
+  uint32_t* ws;        // header, then one counter per row tile
+  float* partials;     // [row_tile][split][x_rows][128]
+  uint32_t n_host_ctas;
+  uint32_t n_stages;
+};
+
+__host__ __device__ constexpr uint32_t x_rows_of(int NT, int MB) { return NT > 0 ? NT * 8 : MB; }
+__host__ __device__ constexpr uint32_t stage_bytes_of(int NT, int MB) {
+  return kBlockBytes + ((x_rows_of(NT, MB) * 128u + 1023u) / 1024u) * 1024u;
+}
+
+__device__ __forceinline__ void store_out(const GemvParams& p, uint32_t m, uint32_t n, float v) {
+  const size_t idx = (size_t)m * p.N + n;
+  if (p.residual) v += __bfloat162float(p.residual[idx]);
+  if (p.y_dtype == 0) static_cast<float*>(p.y)[idx] = v;
+  else static_cast<__nv_bfloat16*>(p.y)[idx] = __float2bfloat16_rn(v);
+}
+
+// NT > 0: tensor-core path with NT batch tiles of 8; NT == 0: CUDA-core path for MB rows.
+template <int NT, int MB>
+__global__ void __launch_bounds__(kGemvThreads, 1) gemv_tiered_kernel(const GemvParams p) {
+  constexpr uint32_t kXRows = x_rows_of(NT, MB);
+  constexpr uint32_t kStageBytes = stage_bytes_of(NT, MB);
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  __shared__ uint64_t full_bar[kMaxStages];
+  __shared__ uint64_t empty_bar[kMaxStages];
+  __shared__ uint4 meta[kMaxStages];
+  __shared__ uint32_t s_old;
+
+  const uint32_t tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const uint32_t n_stages = p.n_stages;
+  uint32_t* status = p.ws + kWsStatus;
+
+  if (tid == 0) {
+    for (uint32_t s = 0; s < n_stages; ++s) {
+      mbar_init(&full_bar[s], 33);              // 32 cp.async arrivals + the lane-0 arrive
+      mbar_init(&empty_bar[s], kConsumerWarps);
+    }
+    fence_barrier_init();
+  }
+  __syncthreads();
+
+  if (warp == kConsumerWarps) {
+    // ------------------------------------------------------------------ producer warp
+    TierQueues q;
+    q.init(p.ws, p.n_host_pages * p.items_per_page, p.n_pages * p.items_per_page,
+           blockIdx.x < p.n_host_ctas);
+    uint32_t stage = 0, phase = 0;
+    for (;;) {
+      uint32_t qi = 0;
+      if (lane == 0) qi = q.next();
+      qi = __shfl_sync(0xFFFFFFFFu, qi, 0);
+      if (qi == 0xFFFFFFFFu) break;
+      const uint32_t page = p.w_order[qi / p.items_per_page];
+      const uint32_t item = page * p.items_per_page + qi % p.items_per_page;
+      if (item >= p.n_items) continue;  // unused tail of the last page
+      const uint32_t first_blk = item * p.run;
+      const uint32_t row_tile = first_blk / p.k_blocks;
+      const uint32_t kb0 = first_blk % p.k_blocks;
+      const bool from_host = qi < p.n_host_pages * p.items_per_page;
+      const uint8_t* src = static_cast<const uint8_t*>(p.w_page_ptr[page]) +
+                           (size_t)(first_blk % kBlocksPerPage) * kBlockBytes;
+      for (uint32_t j = 0; j < p.run; ++j) {
+        mbar_wait(&empty_bar[stage], phase ^ 1u, status);
+        uint8_t* wdst = smem + (size_t)stage * kStageBytes;
+        uint8_t* xdst = wdst + kBlockBytes;
+        if (lane == 0)
+          meta[stage] = make_uint4(row_tile, kb0 / p.run,
+                                   (j == 0 ? kFlagFirst : 0u) | (j + 1 == p.run ? kFlagLast : 0u), 0u);
+        const uint32_t k_base = (kb0 + j) * kBlockK;
+        for (uint32_t idx = lane; idx < kXRows * 8; idx += 32) {
+          const uint32_t m = idx >> 3, c = idx & 7;
+          const uint32_t k = k_base + c * 8;
+          const bool valid = (m < p.M_b) && (k < p.K);
+          const __nv_bfloat16* xs = valid ? p.x + (size_t)m * p.K + k : p.x;
+          cp_async_16(xdst + m * 128 + ((c ^ (m & 7)) << 4), xs, valid ? 16u : 0u);
+        }
+        if (from_host) {
+          const uint8_t* s = src + (size_t)j * kBlockBytes;
+#pragma unroll 8
+          for (uint32_t idx = lane; idx < kBlockBytes / 16; idx += 32)
+            cp_async_16(wdst + idx * 16, s + idx * 16, 16u);
+        }
+        cp_async_arrive_noinc(&full_bar[stage]);
+        if (lane == 0) {
+          if (from_host) {
+            mbar_arrive(&full_bar[stage]);
+          } else {
+            mbar_arrive_expect_tx(&full_bar[stage], kBlockBytes);
+            bulk_copy_g2s(wdst, src + (size_t)j * kBlockBytes, kBlockBytes, &full_bar[stage]);
+          }
+        }
+        if (++stage == n_stages) { stage = 0; phase ^= 1u; }
+      }
+    }
+    // tell the consumers to stop
+    mbar_wait(&empty_bar[stage], phase ^ 1u, status);
+    if (lane == 0) meta[stage] = make_uint4(0u, 0u, kFlagStop, 0u);
+    cp_async_arrive_noinc(&full_bar[stage]);
+    if (lane == 0) {
+      mbar_arrive(&full_bar[stage]);
+      q.finish(gridDim.x);
+    }
+    return;
+  }
+
+  // -------------------------------------------------------------------- consumer warps
+  constexpr int kAccN = NT > 0 ? NT : 4;
+  constexpr int kAccM = NT > 0 ? 4 : MB;
+  float acc[kAccN][kAccM];
+#pragma unroll
+  for (int i = 0; i < kAccN; ++i)
+#pragma unroll
+    for (int j = 0; j < kAccM; ++j) acc[i][j] = 0.f;
+
+  uint32_t* tile_cnt = p.ws + kWsHeaderWords;
+  uint32_t stage = 0, phase = 0;
+  for (;;) {
+    mbar_wait(&full_bar[stage], phase, status);
+    const uint4 mt = meta[stage];
+    if (mt.z & kFlagStop) break;
+    if (mt.z & kFlagFirst) {
+#pragma unroll
+      for (int i = 0; i < kAccN; ++i)
+#pragma unroll
+        for (int j = 0; j < kAccM; ++j) acc[i][j] = 0.f;
+    }
+    const uint8_t* wsm = smem + (size_t)stage * kStageBytes;
+    const uint8_t* xsm = wsm + kBlockBytes;
+    if constexpr (NT > 0) {
+      const uint32_t wbase = smem_u32(wsm), xbase = smem_u32(xsm);
+      const uint32_t a_row = warp * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
+      const uint32_t b_row0 = ((lane >> 4) << 3) + (lane & 7);
+#pragma unroll
+      for (uint32_t ks = 0; ks < 4; ++ks) {
+        uint32_t a[4];
+        const uint32_t a_chunk = ks * 2 + (lane >> 4);
+        ldmatrix_x4(a[0], a[1], a[2], a[3], wbase + a_row * 128 + ((a_chunk ^ (a_row & 7)) << 4));
+        const uint32_t b_chunk = ks * 2 + ((lane >> 3) & 1);
+#pragma unroll
+        for (int n2 = 0; n2 < NT / 2; ++n2) {
+          const uint32_t b_row = n2 * 16 + b_row0;
+          uint32_t b0, b1, b2, b3;
+          ldmatrix_x4(b0, b1, b2, b3, xbase + b_row * 128 + ((b_chunk ^ (b_row & 7)) << 4));
+          mma_bf16_16816(acc[2 * n2], a, b0, b1);
+          mma_bf16_16816(acc[2 * n2 + 1], a, b2, b3);
+        }
+      }
+    } else {
+      // lanes 8g..8g+7 share weight row (warp*16 + 4j + g) and split its 64 columns
+      const uint32_t c = lane & 7, g = lane >> 3;
+      float wf[4][8];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const uint32_t row = warp * 16 + 4 * j + g;
+        const uint4 w = *reinterpret_cast<const uint4*>(wsm + row * 128 + ((c ^ (row & 7)) << 4));
+        wf[j][0] = bf16_lo(w.x); wf[j][1] = bf16_hi(w.x); wf[j][2] = bf16_lo(w.y); wf[j][3] = bf16_hi(w.y);
+        wf[j][4] = bf16_lo(w.z); wf[j][5] = bf16_hi(w.z); wf[j][6] = bf16_lo(w.w); wf[j][7] = bf16_hi(w.w);
+      }
+#pragma unroll
+      for (int m = 0; m < MB; ++m) {
+        const uint4 xv = *reinterpret_cast<const uint4*>(xsm + m * 128 + ((c ^ (m & 7)) << 4));
+        const float xf[8] = {bf16_lo(xv.x), bf16_hi(xv.x), bf16_lo(xv.y), bf16_hi(xv.y),
+                             bf16_lo(xv.z), bf16_hi(xv.z), bf16_lo(xv.w), bf16_hi(xv.w)};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          float s = acc[j][m];
+#pragma unroll
+          for (int e = 0; e < 8; ++e) s = fmaf(wf[j][e], xf[e], s);
+          acc[j][m] = s;
+        }
+      }
+    }
+    __syncwarp();
+    if (lane == 0) mbar_arrive(&empty_bar[stage]);
+    if (++stage == n_stages) { stage = 0; phase ^= 1u; }
+
+    if (mt.z & kFlagLast) {
+      const uint32_t row_tile = mt.x, split = mt.y;
+      if constexpr (NT == 0) {
+        // finish the dot products: sum over the 8 lanes that share a row
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+#pragma unroll
+          for (int m = 0; m < MB; ++m) {
+            float s = acc[j][m];
+            s += __shfl_xor_sync(0xFFFFFFFFu, s, 1);
+            s += __shfl_xor_sync(0xFFFFFFFFu, s, 2);
+            s += __shfl_xor_sync(0xFFFFFFFFu, s, 4);
+            acc[j][m] = s;
+          }
+      }
+      const bool direct = (p.splits == 1);
+      float* part = p.partials + ((size_t)row_tile * p.splits + split) * kXRows * kBlockRows;
+      if constexpr (NT > 0) {
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+          for (int r = 0; r < 4; ++r) {
+            const uint32_t m = nt * 8 + (lane & 3) * 2 + (r & 1);
+            const uint32_t nl = warp * 16 + (lane >> 2) + (r >> 1) * 8;
+            if (direct) {
+              const uint32_t n = row_tile * kBlockRows + nl;
+              if (m < p.M_b && n < p.N) store_out(p, m, n, acc[nt][r]);
+            } else {
+              __stcg(part + m * kBlockRows + nl, acc[nt][r]);
+            }
+          }
+      } else {
+        if ((lane & 7) == 0) {
+#pragma unroll
+          for (int j = 0; j < 4; ++j)
+#pragma unroll
+            for (int m = 0; m < MB; ++m) {
+              const uint32_t nl = warp * 16 + 4 * j + (lane >> 3);
+              if (direct) {
+                const uint32_t n = row_tile * kBlockRows + nl;
+                if ((uint32_t)m < p.M_b && n < p.N) store_out(p, m, n, acc[j][m]);
+              } else {
+                __stcg(part + m * kBlockRows + nl, acc[j][m]);
+              }
+            }
+        }
+      }
+      if (!direct) {
+        // the threadblock that delivers the last partial sum of a row tile adds them up in
+        // split order (fixed order: deterministic) and writes the output
+        __threadfence();
+        named_barrier_sync(1, kConsumerThreads);
+        if (tid == 0) s_old = atomicAdd(tile_cnt + row_tile, 1u);
+        named_barrier_sync(1, kConsumerThreads);
+        if (s_old == p.splits - 1) {
+          __threadfence();
+          const float* base = p.partials + (size_t)row_tile * p.splits * kXRows * kBlockRows;
+          for (uint32_t idx = tid; idx < p.M_b * kBlockRows; idx += kConsumerThreads) {
+            const uint32_t m = idx / kBlockRows, nl = idx % kBlockRows;
+            float s = 0.f;
+            for (uint32_t sp = 0; sp < p.splits; ++sp)
+              s += __ldcg(base + ((size_t)sp * kXRows + m) * kBlockRows + nl);
+            const uint32_t n = row_tile * kBlockRows + nl;
+            if (n < p.N) store_out(p, m, n, s);
+          }
+          if (tid == 0) tile_cnt[row_tile] = 0;
+        }
+        named_barrier_sync(1, kConsumerThreads);
+      }
+    }
+  }
+}
+
+// Packed form: 16-byte chunk `pos` of row r of block (t, kb) holds columns
+// [64 kb + 8 c, +8) of weight row 128 t + r with c = pos ^ (r & 7).
+__global__ void __launch_bounds__(256)
+pack_weights_kernel(const uint4* __restrict__ w, uint32_t N, uint32_t K, uint32_t k_blocks,
+                    size_t n_chunks, const void* const* __restrict__ page_ptr) {
+  const size_t stride = (size_t)gridDim.x * blockDim.x;
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n_chunks; i += stride) {
+    const size_t blk = i / (kBlockBytes / 16);
+    const uint32_t in_blk = (uint32_t)(i % (kBlockBytes / 16));
+    const uint32_t r = in_blk >> 3, pos = in_blk & 7, c = pos ^ (r & 7);
+    const uint32_t t = (uint32_t)(blk / k_blocks), kb = (uint32_t)(blk % k_blocks);
+    const uint32_t row = t * kBlockRows + r, k = kb * kBlockK + c * 8;
+    uint4 v = make_uint4(0u, 0u, 0u, 0u);
+    if (row < N && k < K) v = w[((size_t)row * K + k) / 8];
+    const size_t off = i * 16;
+    uint4* dst = reinterpret_cast<uint4*>(static_cast<uint8_t*>(const_cast<void*>(page_ptr[off / kPageBytes])) +
+                                          off % kPageBytes);
+    *dst = v;
+  }
+}
+
+uint32_t pick_run(uint32_t n_row_tiles, uint32_t k_blocks) {
+  // Run length of a work item in blocks: a power of two that divides the row tile's
+  // k_blocks (and so the 128 blocks of a page).  Longer runs mean fewer split-K partial
+  // sums; shorter runs mean more items to balance over the SMs.  Take the longest run that
+  // leaves about three items per SM, else the longest that leaves one per SM, else 1.
+  const uint64_t total = (uint64_t)n_row_tiles * k_blocks;
+  const uint64_t wanted[2] = {444, 148};
+  for (int pass = 0; pass < 2; ++pass)
+    for (uint32_t run = 32; run >= 1; run >>= 1)
+      if (k_blocks % run == 0 && total / run >= wanted[pass]) return run;
+  return 1;
+}
+
+template <int NT, int MB>
+int launch_gemv(const GemvParams& p, int sms, cudaStream_t stream) {
+  constexpr uint32_t kStage = stage_bytes_of(NT, MB);
+  GemvParams q = p;
+  uint32_t n_stages = kSmemBudget / kStage;
+  if (n_stages > kMaxStages) n_stages = kMaxStages;
+  q.n_stages = n_stages;
+  const size_t smem = (size_t)n_stages * kStage + 1024;
+  static bool configured = false;
+  if (!configured) {
+    const int rc = boosth::check(cudaFuncSetAttribute(gemv_tiered_kernel<NT, MB>,
+                                                      cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(kSmemBudget + 1024)));
+    if (rc != BOOST_OK) return rc;
+    configured = true;
+  }
+  uint32_t grid = (uint32_t)sms;
+  const uint32_t queue_len = q.n_pages * q.items_per_page;
+  if (grid > queue_len) grid = queue_len;
+  uint32_t n_host_ctas = 0;
+  if (q.n_host_pages) {
+    n_host_ctas = 8;
+    if (n_host_ctas > q.n_host_pages * q.items_per_page) n_host_ctas = q.n_host_pages * q.items_per_page;
+    if (n_host_ctas > grid) n_host_ctas = grid;
+  }
+  q.n_host_ctas = n_host_ctas;
+  gemv_tiered_kernel<NT, MB><<<grid, kGemvThreads, smem, stream>>>(q);
+  return boosth::check_launch();
+}
+
+}  // namespace
+
+extern "C" int boost_weight_layout(uint32_t N, uint32_t K, boost_weight_layout_t* out) {
+  if (!out || N == 0 || K == 0) return BOOST_ERR_INVALID;
+  out->n_row_tiles = (N + kBlockRows - 1) / kBlockRows;
+  out->k_blocks = (K + kBlockK - 1) / kBlockK;
+  out->blocks_per_item = pick_run(out->n_row_tiles, out->k_blocks);
+  out->splits = out->k_blocks / out->blocks_per_item;
+  out->bytes = (uint64_t)out->n_row_tiles * out->k_blocks * kBlockBytes;
+  out->n_pages = (out->bytes + kPageBytes - 1) / kPageBytes;
+  return BOOST_OK;
+}
+
+extern "C" int boost_pack_weights(const void* w_row_major, uint32_t N, uint32_t K,
+                                  const void* const* w_page_ptr, size_t n_pages, void* stream) {
+  boost_weight_layout_t lay;
+  const int rc = boost_weight_layout(N, K, &lay);
+  if (rc != BOOST_OK) return rc;
+  if (!w_row_major || !w_page_ptr) return BOOST_ERR_INVALID;
+  if (K % 8 != 0 || ((uintptr_t)w_row_major % 16) != 0) return BOOST_ERR_ALIGN;
+  if (n_pages < lay.n_pages) return BOOST_ERR_CAPACITY;
+  const size_t n_chunks = lay.bytes / 16;
+  size_t blocks = (n_chunks + 255) / 256;
+  const size_t cap = (size_t)(boosth::sm_count() > 0 ? boosth::sm_count() : 148) * 16;
+  if (blocks > cap) blocks = cap;
+  pack_weights_kernel<<<(unsigned)blocks, 256, 0, (cudaStream_t)stream>>>(
+      static_cast<const uint4*>(w_row_major), N, K, lay.k_blocks, n_chunks, w_page_ptr);
+  return boosth::check_launch();
+}
+
+static uint32_t gemv_x_rows(uint32_t M_b) {
+  if (M_b <= 1) return 1;
+  if (M_b <= 2) return 2;
+  if (M_b <= 4) return 4;
+  if (M_b <= 8) return 8;
+  if (M_b <= 16) return 16;
+  if (M_b <= 32) return 32;
+  if (M_b <= 64) return 64;
+  return 128;
+}
+
+extern "C" size_t boost_gemv_workspace_bytes(uint32_t N, uint32_t K, uint32_t M_b) {
+  boost_weight_layout_t lay;
+  if (boost_weight_layout(N, K, &lay) != BOOST_OK || M_b == 0 || M_b > 128) return 0;
+  size_t header = ((size_t)(kWsHeaderWords + lay.n_row_tiles) * 4 + 255) / 256 * 256;
+  size_t partials = lay.splits > 1 ? (size_t)lay.n_row_tiles * lay.splits * gemv_x_rows(M_b) * kBlockRows * 4 : 0;
+  return header + partials;
+}
+
+extern "C" int boost_gemv_tiered(const void* const* w_page_ptr, const uint32_t* w_order,
+                                 size_t n_pages, size_t n_host_pages, uint32_t N, uint32_t K,
+                                 const void* x, uint32_t M_b, void* y, int y_dtype,
+                                 const void* residual, void* workspace, size_t workspace_bytes,
+                                 void* stream) {
+  if (!w_page_ptr || !w_order || !x || !y || !workspace) return BOOST_ERR_INVALID;
+  if (M_b == 0 || M_b > 128 || (y_dtype != 0 && y_dtype != 1)) return BOOST_ERR_INVALID;
+  boost_weight_layout_t lay;
+  const int rc = boost_weight_layout(N, K, &lay);
+  if (rc != BOOST_OK) return rc;
+  if (n_pages != lay.n_pages || n_host_pages > n_pages) return BOOST_ERR_INVALID;
+  if (K % 8 != 0 || ((uintptr_t)x % 16) != 0 || ((uintptr_t)workspace % 256) != 0) return BOOST_ERR_ALIGN;
+  if (workspace_bytes < boost_gemv_workspace_bytes(N, K, M_b)) return BOOST_ERR_CAPACITY;
+  const int sms = boosth::sm_count();
+  if (sms <= 0) return BOOST_ERR_CUDA;
+
+  GemvParams p;
+  p.w_page_ptr = w_page_ptr;
+  p.w_order = w_order;
+  p.n_pages = (uint32_t)n_pages;
+  p.n_host_pages = (uint32_t)n_host_pages;
+  p.N = N; p.K = K;
+  p.n_row_tiles = lay.n_row_tiles;
+  p.k_blocks = lay.k_blocks;
+  p.run = lay.blocks_per_item;
+  p.splits = lay.splits;
+  p.items_per_page = kBlocksPerPage / lay.blocks_per_item;
+  p.n_items = (uint32_t)((uint64_t)lay.n_row_tiles * lay.k_blocks / lay.blocks_per_item);
+  p.x = static_cast<const __nv_bfloat16*>(x);
+  p.M_b = M_b;
+  p.y = y; p.y_dtype = y_dtype;
+  p.residual = static_cast<const __nv_bfloat16*>(residual);
+  p.ws = static_cast<uint32_t*>(workspace);
+  const size_t header = ((size_t)(kWsHeaderWords + lay.n_row_tiles) * 4 + 255) / 256 * 256;
+  p.partials = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + header);
+  p.n_host_ctas = 0; p.n_stages = 0;
+  cudaStream_t st = (cudaStream_t)stream;
+  switch (gemv_x_rows(M_b)) {
+    case 1: return launch_gemv<0, 1>(p, sms, st);
+    case 2: return launch_gemv<0, 2>(p, sms, st);
+    case 4: return launch_gemv<0, 4>(p, sms, st);
+    case 8: return launch_gemv<0, 8>(p, sms, st);
+    case 16: return launch_gemv<2, 0>(p, sms, st);
+    case 32: return launch_gemv<4, 0>(p, sms, st);
+    case 64: return launch_gemv<8, 0>(p, sms, st);
+    default: return launch_gemv<16, 0>(p, sms, st);
+  }
+}

@@ -1,0 +1,140 @@
+"""Device-memory plumbing for tiered buffers: slabs, page tables, visit order.
+
+PyTorch allocates the HBM slab and the pinned host slab; the library decides
+the placement (boost_place_pages*), assigns page addresses (boost_page_table)
+and orders the pages for the kernels (boost_tier_order).  No arithmetic of the
+method lives here.
+"""
+import numpy as np
+import torch
+
+from . import binding as B
+
+PAGE = B.PAGE_BYTES
+
+
+def _aligned(t, align=PAGE):
+    """Address inside the uint8 tensor t aligned up to `align`."""
+    p = t.data_ptr()
+    return (p + align - 1) // align * align
+
+
+class TieredBuffer:
+    """A buffer of n_bytes cut into 2 MiB pages placed over HBM and pinned host memory."""
+
+    def __init__(self, n_bytes, host_ratio=0.0, policy=B.POLICY_MODULO, seed=0, superpage_pages=1,
+                 device="cuda", tier=None, wave_size=0):
+        self.n_bytes = int(n_bytes)
+        self.device = torch.device(device)
+        if tier is None:
+            tier, self.flags = B.boost_place_pages_ex(None, self.n_bytes, host_ratio, wave_size, policy,
+                                                      seed, superpage_pages)
+        else:
+            tier, self.flags = np.ascontiguousarray(tier, dtype=np.uint8), 0
+        self.tier = tier
+        self.n_pages = int(tier.size)
+        self.n_host = int((tier == B.TIER_HOST).sum())
+        self.n_hbm = self.n_pages - self.n_host
+        self._hbm = torch.empty(self.n_hbm * PAGE + PAGE, dtype=torch.uint8, device=self.device)
+        self.hbm_base = _aligned(self._hbm)
+        if self.n_host:
+            self._host = torch.empty(self.n_host * PAGE + PAGE, dtype=torch.uint8, pin_memory=True)
+            self.host_base_cpu = _aligned(self._host)
+            self.host_base = B.boost_host_device_pointer(self.host_base_cpu)
+        else:
+            self._host, self.host_base_cpu, self.host_base = None, 0, 0
+        table = B.boost_page_table(tier, self.hbm_base, self.n_hbm * PAGE,
+                                   self.host_base or None, self.n_host * PAGE)
+        self.page_table_host = table
+        self.page_ptr = torch.from_numpy(table.view(np.int64).copy()).to(self.device)
+        order, n_host = B.boost_tier_order(tier)
+        assert n_host == self.n_host
+        self.order_host = order
+        self.order = torch.from_numpy(order.view(np.int32).copy()).to(self.device)
+
+    def scatter_from(self, flat, stream=None):
+        """Copy a contiguous device tensor (any dtype) of n_bytes into the pages."""
+        assert flat.is_cuda and flat.is_contiguous() and flat.numel() * flat.element_size() == self.n_bytes
+        B.boost_scatter_pages(flat, self.n_bytes, self.page_ptr, self.n_pages, stream)
+
+    def gather_to(self, flat, stream=None):
+        assert flat.is_cuda and flat.is_contiguous() and flat.numel() * flat.element_size() == self.n_bytes
+        B.boost_gather_pages(flat, self.n_bytes, self.page_ptr, self.n_pages, stream)
+
+
+class TieredWeight:
+    """A row-major bf16 weight [N, K] packed into tiered pages for boost_gemv_tiered."""
+
+    def __init__(self, w, host_ratio=0.0, policy=B.POLICY_MODULO, seed=0, device="cuda", tier=None,
+                 superpage_pages=1):
+        assert w.dtype == torch.bfloat16 and w.dim() == 2 and w.is_cuda and w.is_contiguous()
+        self.N, self.K = int(w.shape[0]), int(w.shape[1])
+        self.layout = B.boost_weight_layout(self.N, self.K)
+        self.buf = TieredBuffer(self.layout["bytes"], host_ratio, policy, seed, superpage_pages, device, tier)
+        B.boost_pack_weights(w, self.N, self.K, self.buf.page_ptr, self.buf.n_pages)
+        torch.cuda.current_stream().synchronize()
+        self._ws = {}
+
+    def workspace(self, m_b):
+        n = B.boost_gemv_workspace_bytes(self.N, self.K, m_b)
+        ws = self._ws.get(n)
+        if ws is None:
+            ws = torch.zeros(n + 256, dtype=torch.uint8, device=self.buf.device)
+            self._ws[n] = ws
+        off = (-ws.data_ptr()) % 256
+        return ws.data_ptr() + off, n
+
+    def status_words(self):
+        """Status word (sticky error bits) of every workspace this weight has used."""
+        out = []
+        for ws in self._ws.values():
+            off = (-ws.data_ptr()) % 256
+            out.append(int(ws[off:off + 4].cpu().numpy().view(np.uint32)[0]))
+        return out
+
+    def gemv(self, x, y=None, y_dtype=torch.float32, residual=None, workspace=None, stream=None):
+        """y = x @ W^T (+ residual); x bf16 [M_b, K] (or [K])."""
+        x2 = x.reshape(-1, self.K)
+        m_b = x2.shape[0]
+        if y is None:
+            y = torch.empty(m_b, self.N, dtype=y_dtype, device=x.device)
+        ws_ptr, ws_bytes = workspace if workspace is not None else self.workspace(m_b)
+        B.boost_gemv_tiered(self.buf.page_ptr, self.buf.order, self.buf.n_pages, self.buf.n_host,
+                            self.N, self.K, x2, m_b, y, 0 if y.dtype == torch.float32 else 1, residual,
+                            ws_ptr, ws_bytes, stream)
+        return y
+
+
+class TieredKVCache:
+    """K and V tensors of one layer, [Hkv][n_blocks][16][128] bf16, placed linearly by a KV pool."""
+
+    def __init__(self, pool, n_kv_heads, n_blocks, head_dim=128, device="cuda"):
+        self.pool = pool
+        self.n_kv_heads, self.n_blocks, self.head_dim = n_kv_heads, n_blocks, head_dim
+        self.tier = pool.page_tiers()
+        n_bytes = n_kv_heads * n_blocks * 16 * head_dim * 2
+        assert n_bytes == self.tier.size * PAGE
+        self.k = TieredBuffer(n_bytes, device=device, tier=self.tier)
+        self.v = TieredBuffer(n_bytes, device=device, tier=self.tier)
+        self.n_pages = self.k.n_pages
+
+    def load(self, k_logical, v_logical):
+        """Fill from logical [Hkv, n_blocks, 16, D] bf16 device tensors."""
+        for buf, t in ((self.k, k_logical), (self.v, v_logical)):
+            assert t.is_cuda and t.is_contiguous() and t.dtype == torch.bfloat16
+            B.boost_kv_scatter(t, self.n_kv_heads, self.n_blocks, self.head_dim, buf.page_ptr, buf.n_pages)
+
+    def dump(self):
+        out = []
+        for buf in (self.k, self.v):
+            t = torch.empty(self.n_kv_heads, self.n_blocks, 16, self.head_dim, dtype=torch.bfloat16,
+                            device=buf.device)
+            B.boost_kv_gather(t, self.n_kv_heads, self.n_blocks, self.head_dim, buf.page_ptr, buf.n_pages)
+            out.append(t)
+        return out
+
+
+def aligned_workspace(n_bytes, device):
+    """Zero-filled device scratch of n_bytes whose address is 256-byte aligned -> (tensor, ptr)."""
+    t = torch.zeros(n_bytes + 256, dtype=torch.uint8, device=device)
+    return t, t.data_ptr() + (-t.data_ptr()) % 256

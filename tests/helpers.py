@@ -12,3 +12,28 @@ def load_paper_values():
             key, val = (s.strip() for s in line.split("=", 1))
             out[key] = float(val)
     return out
+
+
+ABS_TOL = 2e-2   # max abs error against fp64 (spec tolerance)
+REL_TOL = 1e-2   # max rel error against fp64
+
+
+def assert_close_to_oracle(got, ref, what=""):
+    """bf16-in / fp32-accumulate outputs against the fp64 oracle: max abs error <= 2e-2 and
+    max rel error <= 1e-2.  The relative error of an element whose reference is (nearly)
+    zero is taken against max(|ref|, 1e-3 * rms(ref)); how many elements needed that floor
+    is returned so callers can report it."""
+    import numpy as np
+    got = np.asarray(got, dtype=np.float64)
+    ref = np.asarray(ref, dtype=np.float64)
+    assert got.shape == ref.shape, (got.shape, ref.shape)
+    assert np.isfinite(got).all(), f"{what}: non-finite output"
+    err = np.abs(got - ref)
+    rms = float(np.sqrt((ref * ref).mean())) if ref.size else 0.0
+    floor = 1e-3 * rms
+    denom = np.maximum(np.abs(ref), floor)
+    denom[denom == 0] = 1.0
+    rel = err / denom
+    assert err.max(initial=0.0) <= ABS_TOL, f"{what}: max abs err {err.max():.3e}"
+    assert rel.max(initial=0.0) <= REL_TOL, f"{what}: max rel err {rel.max():.3e}"
+    return int((np.abs(ref) < floor).sum())

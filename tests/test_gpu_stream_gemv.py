@@ -1,0 +1,193 @@
+"""GPU parity: page copies, tiered stream-reduce and tiered GEMV / skinny GEMM against the
+CPU oracle, through the C ABI."""
+import numpy as np
+import pytest
+
+from oracle import linalg as ol
+from oracle import placement as op
+from paper_2609_13592_b200 import binding as B
+from paper_2609_13592_b200 import synth
+from tests.helpers import assert_close_to_oracle
+
+torch = pytest.importorskip("torch")
+pytestmark = pytest.mark.gpu
+
+PAGE = B.PAGE_BYTES
+PAGE_ELEMS = PAGE // 2
+
+
+@pytest.fixture(scope="module")
+def dev():
+    if not torch.cuda.is_available():
+        pytest.skip("needs a CUDA device")
+    from paper_2609_13592_b200 import build
+    build.build_library()
+    B.lib()
+    return torch.device("cuda:0")
+
+
+def bf16_tensor(bits, dev):
+    return torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).to(dev).view(torch.bfloat16)
+
+
+def status_word(ws_ptr_tensor):
+    return int(ws_ptr_tensor[:4].cpu().numpy().view(np.uint32)[0])
+
+
+def test_scatter_gather_roundtrip(dev):
+    from paper_2609_13592_b200.tiers import TieredBuffer
+    n_bytes = 5 * PAGE + 4096
+    buf = TieredBuffer(n_bytes, 1 / 3, B.POLICY_MODULO, device=dev)
+    assert buf.tier.tolist() == op.place_pages(n_bytes, 1 / 3)
+    src = torch.randint(0, 255, (n_bytes,), dtype=torch.uint8, device=dev)
+    buf.scatter_from(src)
+    back = torch.zeros_like(src)
+    buf.gather_to(back)
+    torch.cuda.synchronize()
+    assert torch.equal(src, back)
+    # the host pages really are in host memory: read them on the CPU
+    host_pages = [i for i, t in enumerate(buf.tier) if t == 1]
+    first = host_pages[0]
+    cpu_view = buf._host[buf.host_base_cpu - buf._host.data_ptr():][:PAGE]
+    assert torch.equal(cpu_view, src[first * PAGE:(first + 1) * PAGE].cpu())
+
+
+@pytest.mark.parametrize("n_pages,ratio,policy", [
+    (37, 1 / 8, B.POLICY_MODULO), (37, 1 / 8, B.POLICY_RANDOM), (37, 1 / 8, B.POLICY_CONTIGUOUS),
+    (3, 0.0, B.POLICY_MODULO), (2, 0.5, B.POLICY_MODULO), (1, 0.0, B.POLICY_MODULO),
+    (80, 1 / 16, B.POLICY_MODULO)])
+def test_stream_reduce_bit_exact(dev, n_pages, ratio, policy):
+    from paper_2609_13592_b200.tiers import TieredBuffer
+    n_elems = n_pages * PAGE_ELEMS
+    buf = TieredBuffer(n_elems * 2, ratio, policy, seed=7, device=dev)
+    assert buf.tier.tolist() == op.place_pages(n_elems * 2, ratio, policy, 7)
+    data = synth.small_int_bf16_torch(0, n_elems, dev)
+    buf.scatter_from(data)
+    ws_bytes = B.boost_stream_reduce_workspace_bytes(n_pages)
+    ws = torch.zeros(ws_bytes, dtype=torch.uint8, device=dev)
+    sums = torch.full((n_pages,), -1.0, dtype=torch.float32, device=dev)
+    for rep in range(2):   # the second run reuses the workspace as the first left it
+        sums.fill_(-1.0)
+        B.boost_stream_reduce_tiered(buf.page_ptr, buf.order, n_pages, buf.n_host, sums, ws, ws_bytes)
+        torch.cuda.synchronize()
+        want, total = ol.stream_sum(synth.small_int_bf16(0, n_elems), PAGE_ELEMS)
+        got = sums.cpu().numpy().astype(np.float64)
+        assert np.array_equal(got, want), rep
+        assert int(got.sum()) == int(total)
+        assert status_word(ws) == 0
+        # queue words and per-page counters are back at zero for the next launch
+        assert not ws[:(16 + n_pages) * 4].cpu().numpy().any()
+
+
+def test_stream_reduce_all_host(dev):
+    from paper_2609_13592_b200.tiers import TieredBuffer
+    n_pages = 4
+    tier = np.ones(n_pages, np.uint8)
+    buf = TieredBuffer(n_pages * PAGE, device=dev, tier=tier)
+    data = synth.small_int_bf16_torch(100, n_pages * PAGE_ELEMS, dev)
+    buf.scatter_from(data)
+    ws_bytes = B.boost_stream_reduce_workspace_bytes(n_pages)
+    ws = torch.zeros(ws_bytes, dtype=torch.uint8, device=dev)
+    sums = torch.zeros(n_pages, dtype=torch.float32, device=dev)
+    B.boost_stream_reduce_tiered(buf.page_ptr, buf.order, n_pages, buf.n_host, sums, ws, ws_bytes)
+    torch.cuda.synchronize()
+    want, _ = ol.stream_sum(synth.small_int_bf16(100, n_pages * PAGE_ELEMS), PAGE_ELEMS)
+    assert np.array_equal(sums.cpu().numpy().astype(np.float64), want)
+
+
+def run_gemv(dev, n, k, m_b, ratio, seed, y_dtype=None, residual=False, policy=B.POLICY_MODULO,
+             tier=None, std_w=0.02):
+    from paper_2609_13592_b200.tiers import TieredWeight
+    y_dtype = y_dtype or torch.float32
+    w_bits = synth.normal_bf16((n, k), std_w, seed)
+    x_bits = synth.normal_bf16((m_b, k), 1.0, seed + 1)
+    w = TieredWeight(bf16_tensor(w_bits, dev), ratio, policy, seed=seed, device=dev, tier=tier)
+    x = bf16_tensor(x_bits, dev)
+    res_bits = synth.normal_bf16((m_b, n), 1.0, seed + 2) if residual else None
+    res = bf16_tensor(res_bits, dev) if residual else None
+    y = w.gemv(x, y_dtype=y_dtype, residual=res)
+    torch.cuda.synchronize()
+    ref = ol.gemm(x_bits, w_bits)
+    if residual:
+        ref = ref + ol.bf16_bits_to_f64(res_bits)
+    return w, y.float().cpu().numpy(), ref, (x, res)
+
+
+def test_gemv_config1(dev):
+    # 4096 x 4096 bf16 weights N(0, 0.02^2), x N(0, 1), modulo placement with host_ratio 1/16
+    w, y, ref, _ = run_gemv(dev, 4096, 4096, 1, 1 / 16, seed=1)
+    assert w.buf.n_pages == 16 and w.buf.tier.tolist() == [0] * 15 + [1]
+    assert w.buf.tier.tolist() == op.place_pages(4096 * 4096 * 2, 1 / 16)
+    n_floor = assert_close_to_oracle(y[0], ref[0], "config 1 y")
+    assert n_floor <= 16
+    assert w.status_words() == [0]   # no bounded wait gave up
+
+
+@pytest.mark.parametrize("m_b", [1, 2, 3, 4, 5, 8, 9, 16, 17, 32, 33, 64, 100, 128])
+def test_gemv_batches(dev, m_b):
+    # several row tiles with a ragged last one, ragged K (5 k-blocks of 64, last one partial)
+    _, y, ref, _ = run_gemv(dev, 328, 296, m_b, 0.5, seed=10 + m_b)
+    assert_close_to_oracle(y, ref, f"gemv m_b={m_b}")
+
+
+@pytest.mark.parametrize("n,k,m_b,ratio", [
+    (1024, 4096, 32, 1 / 4),      # 2 splits per row tile and several pages
+    (4096, 14336, 32, 1 / 8),     # down-projection shape: rows of 28 KiB, 57344-byte ... 1.75 pages per row tile
+    (6144, 4096, 7, 1 / 3),
+    (256, 512, 128, 0.0),
+])
+def test_gemv_shapes(dev, n, k, m_b, ratio):
+    w, y, ref, _ = run_gemv(dev, n, k, m_b, ratio, seed=n + k + m_b)
+    assert_close_to_oracle(y, ref, f"gemv {n}x{k} m_b={m_b}")
+    assert w.buf.tier.tolist() == op.place_pages(w.layout["bytes"], ratio)
+
+
+def test_gemv_bf16_output_with_residual(dev):
+    _, y, ref, _ = run_gemv(dev, 640, 1024, 32, 1 / 2, seed=5, y_dtype=torch.bfloat16, residual=True)
+    assert_close_to_oracle(y, ref, "bf16 out + residual")
+    _, y, ref, _ = run_gemv(dev, 640, 1024, 4, 1 / 2, seed=6, y_dtype=torch.bfloat16, residual=True)
+    assert_close_to_oracle(y, ref, "bf16 out + residual, small batch")
+
+
+@pytest.mark.parametrize("m_b", [1, 32])
+def test_gemv_integer_inputs_are_exact_and_deterministic(dev, m_b):
+    from paper_2609_13592_b200.tiers import TieredWeight
+    n, k = 512, 2048
+    w_int = (synth.small_int_values(0, n * k).reshape(n, k)).astype(np.float32)
+    x_int = (synth.small_int_values(12345, m_b * k).reshape(m_b, k)).astype(np.float32)
+    w_bits, x_bits = synth.f32_to_bf16_bits(w_int), synth.f32_to_bf16_bits(x_int)
+    w = TieredWeight(bf16_tensor(w_bits, dev), 1 / 4, device=dev)
+    x = bf16_tensor(x_bits, dev)
+    y1 = w.gemv(x).clone()
+    y2 = w.gemv(x).clone()
+    torch.cuda.synchronize()
+    ref = ol.gemm(x_bits, w_bits)
+    assert np.array_equal(y1.cpu().numpy().astype(np.float64), ref)   # integers: exact in fp32
+    assert torch.equal(y1, y2)
+
+
+def test_gemv_result_independent_of_placement(dev):
+    outs = []
+    for ratio, policy in ((0.0, B.POLICY_MODULO), (1 / 4, B.POLICY_MODULO), (1 / 4, B.POLICY_RANDOM),
+                          (1 / 4, B.POLICY_CONTIGUOUS)):
+        _, y, ref, _ = run_gemv(dev, 1024, 2048, 16, ratio, seed=3, policy=policy)
+        outs.append(y)
+    for y in outs[1:]:
+        assert np.array_equal(outs[0], y)
+
+
+def test_gemv_argument_errors(dev):
+    from paper_2609_13592_b200.tiers import TieredWeight
+    w = TieredWeight(bf16_tensor(synth.normal_bf16((128, 64), 0.02, 1), dev), device=dev)
+    x = bf16_tensor(synth.normal_bf16((1, 64), 1.0, 2), dev)
+    y = torch.zeros(1, 128, device=dev)
+    ws_ptr, ws_bytes = w.workspace(1)
+    with pytest.raises(B.BoostError) as e:
+        B.boost_gemv_tiered(w.buf.page_ptr, w.buf.order, 1, 0, 128, 64, x, 0, y, 0, None, ws_ptr, ws_bytes)
+    assert e.value.code == B.ERR_INVALID
+    with pytest.raises(B.BoostError) as e:
+        B.boost_gemv_tiered(w.buf.page_ptr, w.buf.order, 1, 0, 128, 64, x, 1, y, 0, None, ws_ptr, 16)
+    assert e.value.code == B.ERR_CAPACITY
+    with pytest.raises(B.BoostError) as e:
+        B.boost_gemv_tiered(w.buf.page_ptr, w.buf.order, 1, 0, 128, 64, x, 200, y, 0, None, ws_ptr, ws_bytes)
+    assert e.value.code == B.ERR_INVALID

@@ -1,0 +1,216 @@
+"""Host-side library (placement, statistics, page tables, KV pool) against the oracle,
+bit for bit, plus loading of the shared library and its exported symbols.  No GPU."""
+import os
+import random
+import re
+
+import numpy as np
+import pytest
+
+from oracle import kv_pool as okp
+from oracle import placement as op
+from paper_2609_13592_b200 import binding as B
+from paper_2609_13592_b200 import build as libbuild
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module", autouse=True)
+def built():
+    libbuild.build_library()
+    return B.lib()
+
+
+def test_every_declared_symbol_is_exported(built):
+    header = open(os.path.join(ROOT, "include", "boost.h")).read()
+    header = re.sub(r"/\*.*?\*/", "", header, flags=re.S)
+    declared = set(re.findall(r"\b(boost_[a-z0-9_]+)\s*\(", header))
+    assert len(declared) >= 25
+    missing = [n for n in sorted(declared) if not hasattr(built, n)]
+    assert not missing, missing
+    # the binding declares a signature for each of them and nothing else
+    assert set(B.SIGNATURES) == declared
+
+
+def test_modulus_matches_oracle():
+    for m in range(2, 4097):
+        assert B.boost_modulus_from_ratio(1.0 / m) == m
+    rng = random.Random(5)
+    for _ in range(3000):
+        r = rng.uniform(2.0 ** -20, 0.5)
+        assert B.boost_modulus_from_ratio(r) == op.modulus_from_ratio(r)
+    assert B.boost_modulus_from_ratio(0.0) == 0
+    for bad in (-1.0, 0.51, 1e-12, float("nan")):
+        with pytest.raises(B.BoostError) as e:
+            B.boost_modulus_from_ratio(bad)
+        assert e.value.code == B.ERR_INVALID
+    for hbm, link in ((10, 1), (3330, 350), (6452.2, 55.0), (100.0, 25.0), (7.0, 7.0)):
+        assert B.boost_modulus_from_bandwidths(hbm, link) == op.modulus_from_bandwidths(hbm, link)
+
+
+def test_placement_tables_bit_exact():
+    rng = random.Random(11)
+    cases = [(4096 * 4096 * 2, 1 / 16, B.POLICY_MODULO, 0, 1)]
+    for _ in range(300):
+        n_bytes = rng.randint(0, 700) * B.PAGE_BYTES + rng.choice([0, 0, 1, 4096, B.PAGE_BYTES - 1])
+        ratio = rng.choice([0.0, 1 / 256, 1 / 128, 1 / 64, 1 / 32, 1 / 16, 1 / 8, 1 / 12, 0.1, 0.3, 0.5,
+                            rng.uniform(0.001, 0.5)])
+        policy = rng.choice([B.POLICY_MODULO, B.POLICY_CONTIGUOUS, B.POLICY_RANDOM])
+        s = rng.choice([1, 1, 2, 7]) if policy == B.POLICY_MODULO else 1
+        cases.append((n_bytes, ratio, policy, rng.getrandbits(64), s))
+    for n_bytes, ratio, policy, seed, s in cases:
+        got, _ = B.boost_place_pages_ex(None, n_bytes, ratio, 0, policy, seed, s)
+        want = op.place_pages(n_bytes, ratio, policy, seed, s)
+        assert got.tolist() == want, (n_bytes, ratio, policy, seed, s)
+    # the plain entry point is modulo placement
+    assert B.boost_place_pages(None, 32 << 20, 1 / 16).tolist() == [0] * 15 + [1]
+
+
+def test_placement_full_size_sweep_config():
+    # configuration 3: 1 .. 64 GiB buffers, the stated host ratios, three placements
+    for gib in (1, 4, 16, 64):
+        for ratio in (0, 1 / 256, 1 / 128, 1 / 64, 1 / 32, 1 / 16, 1 / 8):
+            for policy in (B.POLICY_MODULO, B.POLICY_CONTIGUOUS, B.POLICY_RANDOM):
+                if gib == 64 and policy == B.POLICY_RANDOM and ratio not in (1 / 16,):
+                    continue  # keep the pure-Python oracle within seconds
+                got, _ = B.boost_place_pages_ex(None, gib << 30, ratio, 0, policy, 9, 1)
+                assert got.tolist() == op.place_pages(gib << 30, ratio, policy, 9, 1)
+
+
+def test_placement_errors_and_flags():
+    with pytest.raises(B.BoostError) as e:
+        B.boost_place_pages(4096, 1 << 21, 0.1)           # misaligned buffer address
+    assert e.value.code == B.ERR_ALIGN
+    with pytest.raises(B.BoostError) as e:
+        B.boost_place_pages_ex(None, 1 << 22, 0.1, 0, 7, 0, 1)
+    assert e.value.code == B.ERR_INVALID
+    with pytest.raises(B.BoostError):
+        B.boost_place_pages_ex(None, 1 << 22, 0.1, 0, B.POLICY_RANDOM, 0, 2)
+    tier = np.zeros(2, np.uint8)
+    n = B.C.c_size_t(0)
+    rc = B.lib().boost_place_pages(None, 10 << 21, 0.25, 0, tier.ctypes.data, 2, B.C.addressof(n))
+    assert rc == B.ERR_CAPACITY and n.value == 10
+    _, flags = B.boost_place_pages_ex(None, 64 << 21, 1 / 16, 8)
+    assert flags == 1                                        # a wave of 8 pages is shorter than the period
+    _, flags = B.boost_place_pages_ex(None, 64 << 21, 1 / 16, 16)
+    assert flags == 0
+
+
+def test_wave_stats_match_oracle():
+    rng = random.Random(3)
+    for _ in range(120):
+        p = rng.randint(1, 300)
+        ratio = rng.choice([1 / 8, 1 / 12, 1 / 16, 0.1, 1 / 64])
+        policy = rng.choice([0, 1, 2])
+        tier = op.place_pages(p * B.PAGE_BYTES, ratio, policy, rng.getrandbits(32))
+        tile = B.PAGE_BYTES // rng.choice([1, 2, 8, 16, 128])
+        g = rng.choice([1, 7, 148, 296, 592, 1000])
+        want = op.wave_stats(tier, tile, g, ratio)
+        got = B.boost_wave_stats(np.array(tier, np.uint8), tile, g, ratio)
+        for k in ("n_waves", "n_host_pages", "n_zero_waves", "n_over_waves"):
+            assert got[k] == want[k], (k, p, ratio, policy, tile, g)
+        for k in ("mean", "var", "min", "max"):
+            assert abs(got[k] - want[k]) < 1e-12, k
+    with pytest.raises(B.BoostError):
+        B.boost_wave_stats(np.zeros(4, np.uint8), 3000, 4, 0.1)
+
+
+def test_tier_order_and_page_table():
+    tier = np.array(op.place_pages(77 * B.PAGE_BYTES, 1 / 8, op.POLICY_RANDOM, 4), np.uint8)
+    order, n_host = B.boost_tier_order(tier)
+    want, want_n = op.tier_order(tier.tolist())
+    assert order.tolist() == want and n_host == want_n
+    hbm, host = 0x7F0000000000, 0x200000000
+    table = B.boost_page_table(tier, hbm, 100 * B.PAGE_BYTES, host, 100 * B.PAGE_BYTES)
+    # every page gets its own 2 MiB slot inside the slab of its tier, in page order
+    hbm_slots = [int(a) for a, t in zip(table, tier) if t == 0]
+    host_slots = [int(a) for a, t in zip(table, tier) if t == 1]
+    assert hbm_slots == [hbm + i * B.PAGE_BYTES for i in range(len(hbm_slots))]
+    assert host_slots == [host + i * B.PAGE_BYTES for i in range(len(host_slots))]
+    with pytest.raises(B.BoostError) as e:
+        B.boost_page_table(tier, hbm, 3 * B.PAGE_BYTES, host, 100 * B.PAGE_BYTES)
+    assert e.value.code == B.ERR_CAPACITY
+    with pytest.raises(B.BoostError) as e:
+        B.boost_page_table(tier, hbm + 4096, 100 * B.PAGE_BYTES, host, 100 * B.PAGE_BYTES)
+    assert e.value.code == B.ERR_ALIGN
+
+
+def same_state(pool, ref):
+    q = pool.query()
+    rq = ref.query()
+    assert q["free_lo"] == rq["free_lo"] and q["free_hi"] == rq["free_hi"]
+    assert q["live_blocks"] == rq["live_blocks"] and q["n_requests"] == rq["n_requests"]
+    assert q["live_host_chunks"] == rq["live_host_chunks"] and q["live_chunks"] == rq["live_chunks"]
+
+
+@pytest.mark.parametrize("geom", [(2048, 8, 8), (1536, 4, 12), (2560, 8, 5), (512, 8, 0),
+                                  (1024, 4, 8), (512, 8, 2), (5120, 8, 5), (1024, 2, 3)])
+def test_pool_traces_bit_exact(geom):
+    n, h, m = geom
+    pool, ref = B.KVPool(n, h, m), okp.KVPool(n, h, m)
+    q = pool.query()
+    assert q["n_pages"] == ref.n_pages and q["n_host_pages"] == ref.n_host_pages
+    assert q["host_heads_lo"] == ref.k_lo
+    first_hi = ref.kind.index(okp.KIND_HI) if okp.KIND_HI in ref.kind else n
+    assert q["first_hi_block"] == first_hi
+    assert pool.page_tiers().tolist() == ref.page_tiers()
+    rng = random.Random(n * 131 + h * 7 + m)
+    live = []
+    rid = 0
+    for step in range(1500):
+        r = rng.random()
+        if live and r < 0.3:
+            victim = live.pop(rng.randrange(len(live)))
+            pool.free(victim)
+            ref.free_request(victim)
+        elif live and r < 0.65:
+            target = rng.choice(live)
+            k = rng.randint(1, 40)
+            try:
+                want = ref.alloc(target, k)
+            except okp.PoolError as e:
+                with pytest.raises(B.BoostError) as ge:
+                    pool.alloc(target, k)
+                assert ge.value.code == e.code
+            else:
+                assert pool.alloc(target, k).tolist() == want
+                assert pool.request_kind(target) == ref.request_kind[target]
+        else:
+            k = rng.randint(1, n // 6)
+            try:
+                want = ref.alloc(rid, k)
+            except okp.PoolError as e:
+                with pytest.raises(B.BoostError) as ge:
+                    pool.alloc(rid, k)
+                assert ge.value.code == e.code
+            else:
+                assert pool.alloc(rid, k).tolist() == want
+                assert pool.request_kind(rid) == ref.request_kind[rid]
+                live.append(rid)
+            rid += 1
+        if step % 50 == 0:
+            same_state(pool, ref)
+    same_state(pool, ref)
+    with pytest.raises(B.BoostError) as e:
+        pool.free(10 ** 9)
+    assert e.value.code == B.ERR_INVALID
+    with pytest.raises(B.BoostError):
+        pool.alloc(1, 0)
+    pool.close()
+
+
+def test_pool_bad_geometry():
+    for args in ((500, 8, 8), (0, 8, 8), (512, 0, 8), (512, 8, 1)):
+        with pytest.raises(B.BoostError) as e:
+            B.KVPool(*args)
+        assert e.value.code == B.ERR_INVALID
+
+
+def test_pool_config5_geometry():
+    # batch 128, contexts up to 4096 -> 24.6k blocks; 1/5 of the KV pages on the host, 8 heads
+    n = 25600
+    pool, ref = B.KVPool(n, 8, 5), okp.KVPool(n, 8, 5)
+    q = pool.query()
+    assert q["host_heads_lo"] == 1 and q["first_hi_block"] == int(0.4 * n) == ref.kind.index(1)
+    assert q["n_host_pages"] * 5 == q["n_pages"]
+    pool.close()
