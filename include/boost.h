@@ -289,6 +289,112 @@ int boost_paged_attn_decode_tiered(const void* q /*device*/, const void* const* 
                                    void* workspace /*device*/, size_t workspace_bytes,
                                    void* out /*device*/, void* stream);
 
+/* --------------------------------------------------- glue of a decode step
+ * The paper does not describe these operators (it treats decode as weight kernels plus
+ * attention, Sec. 2.1, Sec. 5.4); shapes follow the public Llama-3 architecture.  All
+ * tensors are bf16 row-major in device memory unless stated otherwise. */
+
+/* out[b, :] = table[tokens[b], :];  table [vocab, hidden]; tokens device int32 [B]. */
+int boost_embed_gather(const void* table /*device*/, uint32_t vocab, uint32_t hidden,
+                       const int32_t* tokens /*device*/, uint32_t B, void* out /*device*/, void* stream);
+
+/* out = x * rsqrt(mean(x^2) + eps) * weight, row by row; x, out [B, hidden]; weight [hidden]. */
+int boost_rmsnorm(const void* x /*device*/, const void* weight /*device*/, uint32_t B, uint32_t hidden,
+                  float eps, void* out /*device*/, void* stream);
+
+/* Rotary embedding and KV append.  qkv [B, (Hq + 2 Hkv) * D] holds the query heads, then the
+ * key heads, then the value heads of the new token of every sequence; its position is
+ * ctx_lens[b] - 1.  Queries and keys are rotated (rotate-half pairing: element i with
+ * i + D/2, angle = position * rope_base^(-2i/D)); rotated queries go to q_out [B, Hq, D];
+ * rotated keys and the values are written into the paged cache (layout of
+ * boost_kv_scatter) at block_table[b][pos / 16], slot pos % 16.  status_word: device
+ * uint32 that receives error bits (bit 1 = a block index out of range).  D = 128. */
+int boost_rope_kv_append(const void* qkv /*device*/, void* q_out /*device*/,
+                         const void* const* k_page_ptr /*device*/, const void* const* v_page_ptr /*device*/,
+                         uint32_t n_pool_blocks, const int32_t* block_table /*device*/, uint32_t max_blocks,
+                         const int32_t* ctx_lens /*device*/, uint32_t B, uint32_t Hq, uint32_t Hkv,
+                         uint32_t D, float rope_base, void* status_word /*device*/, void* stream);
+
+/* out[b, f] = silu(gate_up[b, f]) * gate_up[b, F + f];  gate_up [B, 2F]; out [B, F]. */
+int boost_swiglu(const void* gate_up /*device*/, uint32_t B, uint32_t F, void* out /*device*/, void* stream);
+
+/* out[b] = index of the largest of logits[b, :] (fp32), lowest index on ties. */
+int boost_argmax(const float* logits /*device*/, uint32_t B, uint32_t V, int32_t* out /*device*/,
+                 void* stream);
+
+/* ------------------------------------------------------- whole decode step */
+
+/* A packed, tiered weight as consumed by boost_gemv_tiered. */
+typedef struct {
+  const void* const* page_ptr; /* device */
+  const uint32_t* order;       /* device */
+  uint64_t n_pages, n_host_pages;
+  uint32_t N, K;
+} boost_weight_t;
+
+typedef struct {
+  boost_weight_t wqkv; /* [(Hq + 2 Hkv) D, hidden]: query rows, key rows, value rows */
+  boost_weight_t wo;   /* [hidden, Hq D] */
+  boost_weight_t wgu;  /* [2 F, hidden]: gate rows, then up rows */
+  boost_weight_t wd;   /* [hidden, F] */
+  const void* norm1;   /* device bf16 [hidden] */
+  const void* norm2;
+  const void* const* k_page_ptr; /* device: pages of this layer's K tensor */
+  const void* const* v_page_ptr;
+} boost_llama_layer_t;
+
+typedef struct {
+  uint32_t n_layers, hidden, ffn, n_q_heads, n_kv_heads, head_dim, vocab;
+  float rms_eps, rope_base;
+  const void* embed;  /* device bf16 [vocab, hidden] */
+  const void* norm_f; /* device bf16 [hidden] */
+  boost_weight_t lm_head; /* [vocab, hidden] */
+  const boost_llama_layer_t* layers; /* host array of n_layers entries */
+  const uint8_t* kv_tier;            /* host: tier of every page of a K (or V) tensor, or NULL */
+  uint64_t n_kv_pages;
+  uint32_t n_pool_blocks;
+} boost_llama_model_t;
+
+/* Device scratch of a decode step for up to B_max sequences (all bf16 unless noted):
+ * h, xn [B, hidden]; qkv [B, (Hq+2Hkv) D]; q_rot, attn [B, Hq D]; gu [B, 2F]; act [B, F];
+ * logits fp32 [B, vocab]; gemv_ws >= the largest boost_gemv_workspace_bytes over the model's
+ * weights; attn_ws >= boost_paged_attn_workspace_bytes; both zero-filled once and 256-byte
+ * aligned; tokens_dev / ctx_dev / next_dev int32 [B] and table_dev int32 [B, max_blocks] are
+ * staging buffers used by boost_llama_decode_step_host only. */
+typedef struct {
+  void *h, *xn, *qkv, *q_rot, *attn, *gu, *act;
+  float* logits;
+  void* gemv_ws;
+  size_t gemv_ws_bytes;
+  void* attn_ws;
+  size_t attn_ws_bytes;
+  int32_t *tokens_dev, *ctx_dev, *table_dev, *next_dev;
+} boost_llama_scratch_t;
+
+/* One decode step for B sequences: embedding, n_layers x (RMSNorm, QKV product, RoPE + KV
+ * append, paged attention, output product + residual, RMSNorm, gate/up product, SwiGLU,
+ * down product + residual), final RMSNorm, LM head, argmax.  Every product is
+ * boost_gemv_tiered, attention is boost_paged_attn_decode_tiered.  Activations between
+ * kernels are bf16; logits stay fp32.  tokens, block_table [B, max_blocks], ctx_lens (new
+ * token included) and next_tokens are device arrays.  Launches are asynchronous on stream.
+ * Returns the number of kernels launched in *n_launches_out when it is not NULL. */
+int boost_llama_decode_step(const boost_llama_model_t* model /*host*/,
+                            const boost_llama_scratch_t* scratch /*host*/,
+                            const int32_t* tokens /*device*/, const int32_t* block_table /*device*/,
+                            uint32_t max_blocks, const int32_t* ctx_lens /*device*/, uint32_t B,
+                            int32_t* next_tokens /*device*/, uint32_t* n_launches_out /*host*/,
+                            void* stream);
+
+/* As above with HOST buffers (pinned memory recommended): copies tokens, block_table and
+ * ctx_lens to the staging buffers of `scratch`, runs the step, copies next_tokens back and
+ * waits for the stream, so the result is valid on return. */
+int boost_llama_decode_step_host(const boost_llama_model_t* model /*host*/,
+                                 const boost_llama_scratch_t* scratch /*host*/,
+                                 const int32_t* tokens /*host*/, const int32_t* block_table /*host*/,
+                                 uint32_t max_blocks, const int32_t* ctx_lens /*host*/, uint32_t B,
+                                 int32_t* next_tokens /*host*/, uint32_t* n_launches_out /*host*/,
+                                 void* stream);
+
 #ifdef __cplusplus
 }
 #endif

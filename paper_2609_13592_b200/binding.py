@@ -48,6 +48,33 @@ class WeightLayout(C.Structure):
                 ("splits", C.c_uint32), ("bytes", C.c_uint64), ("n_pages", C.c_uint64)]
 
 
+class Weight(C.Structure):
+    _fields_ = [("page_ptr", C.c_void_p), ("order", C.c_void_p), ("n_pages", C.c_uint64),
+                ("n_host_pages", C.c_uint64), ("N", C.c_uint32), ("K", C.c_uint32)]
+
+
+class LlamaLayer(C.Structure):
+    _fields_ = [("wqkv", Weight), ("wo", Weight), ("wgu", Weight), ("wd", Weight),
+                ("norm1", C.c_void_p), ("norm2", C.c_void_p),
+                ("k_page_ptr", C.c_void_p), ("v_page_ptr", C.c_void_p)]
+
+
+class LlamaModel(C.Structure):
+    _fields_ = [(n, C.c_uint32) for n in
+                ("n_layers", "hidden", "ffn", "n_q_heads", "n_kv_heads", "head_dim", "vocab")] + \
+               [("rms_eps", C.c_float), ("rope_base", C.c_float),
+                ("embed", C.c_void_p), ("norm_f", C.c_void_p), ("lm_head", Weight),
+                ("layers", C.POINTER(LlamaLayer)), ("kv_tier", C.c_void_p),
+                ("n_kv_pages", C.c_uint64), ("n_pool_blocks", C.c_uint32)]
+
+
+class LlamaScratch(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in ("h", "xn", "qkv", "q_rot", "attn", "gu", "act", "logits")] + \
+               [("gemv_ws", C.c_void_p), ("gemv_ws_bytes", C.c_size_t),
+                ("attn_ws", C.c_void_p), ("attn_ws_bytes", C.c_size_t)] + \
+               [(n, C.c_void_p) for n in ("tokens_dev", "ctx_dev", "table_dev", "next_dev")]
+
+
 _vp, _sz, _u32, _u64, _i32, _dbl, _int, _flt = (C.c_void_p, C.c_size_t, C.c_uint32, C.c_uint64,
                                                  C.c_int32, C.c_double, C.c_int, C.c_float)
 
@@ -82,6 +109,14 @@ SIGNATURES = {
     "boost_paged_attn_workspace_bytes": (_sz, [_u32, _u32, _u32, _u32]),
     "boost_paged_attn_decode_tiered": (_int, [_vp, _vp, _vp, _vp, _sz, _u32, _vp, _u32, _vp,
                                               _u32, _u32, _u32, _u32, _flt, _vp, _sz, _vp, _vp]),
+    "boost_embed_gather": (_int, [_vp, _u32, _u32, _vp, _u32, _vp, _vp]),
+    "boost_rmsnorm": (_int, [_vp, _vp, _u32, _u32, _flt, _vp, _vp]),
+    "boost_rope_kv_append": (_int, [_vp, _vp, _vp, _vp, _u32, _vp, _u32, _vp, _u32, _u32, _u32, _u32,
+                                    _flt, _vp, _vp]),
+    "boost_swiglu": (_int, [_vp, _u32, _u32, _vp, _vp]),
+    "boost_argmax": (_int, [_vp, _u32, _u32, _vp, _vp]),
+    "boost_llama_decode_step": (_int, [_vp, _vp, _vp, _vp, _u32, _vp, _u32, _vp, _vp, _vp]),
+    "boost_llama_decode_step_host": (_int, [_vp, _vp, _vp, _vp, _u32, _vp, _u32, _vp, _vp, _vp]),
 }
 
 _lib = None
@@ -320,3 +355,53 @@ def boost_paged_attn_decode_tiered(q, k_page_ptr, v_page_ptr, kv_tier, n_kv_page
         _ptr(q), _ptr(k_page_ptr), _ptr(v_page_ptr), _ptr(tier), n_kv_pages, n_pool_blocks,
         _ptr(block_table), max_blocks, _ptr(ctx_lens), b, hq, hkv, d, scale, _ptr(workspace),
         workspace_bytes, _ptr(out), _stream(stream)), "boost_paged_attn_decode_tiered")
+
+
+# ----------------------------------------------------------------------- glue
+
+def boost_embed_gather(table, vocab, hidden, tokens, b, out, stream=None):
+    _check(lib().boost_embed_gather(_ptr(table), vocab, hidden, _ptr(tokens), b, _ptr(out), _stream(stream)),
+           "boost_embed_gather")
+
+
+def boost_rmsnorm(x, weight, b, hidden, eps, out, stream=None):
+    _check(lib().boost_rmsnorm(_ptr(x), _ptr(weight), b, hidden, eps, _ptr(out), _stream(stream)),
+           "boost_rmsnorm")
+
+
+def boost_rope_kv_append(qkv, q_out, k_page_ptr, v_page_ptr, n_pool_blocks, block_table, max_blocks,
+                         ctx_lens, b, hq, hkv, d, rope_base, status_word, stream=None):
+    _check(lib().boost_rope_kv_append(_ptr(qkv), _ptr(q_out), _ptr(k_page_ptr), _ptr(v_page_ptr),
+                                      n_pool_blocks, _ptr(block_table), max_blocks, _ptr(ctx_lens), b, hq,
+                                      hkv, d, rope_base, _ptr(status_word), _stream(stream)),
+           "boost_rope_kv_append")
+
+
+def boost_swiglu(gate_up, b, f, out, stream=None):
+    _check(lib().boost_swiglu(_ptr(gate_up), b, f, _ptr(out), _stream(stream)), "boost_swiglu")
+
+
+def boost_argmax(logits, b, v, out, stream=None):
+    _check(lib().boost_argmax(_ptr(logits), b, v, _ptr(out), _stream(stream)), "boost_argmax")
+
+
+def boost_llama_decode_step(model, scratch, tokens, block_table, max_blocks, ctx_lens, b, next_tokens,
+                            stream=None):
+    """model / scratch: LlamaModel / LlamaScratch structures; returns the number of launches."""
+    n = C.c_uint32(0)
+    _check(lib().boost_llama_decode_step(C.addressof(model), C.addressof(scratch), _ptr(tokens),
+                                         _ptr(block_table), max_blocks, _ptr(ctx_lens), b,
+                                         _ptr(next_tokens), C.addressof(n), _stream(stream)),
+           "boost_llama_decode_step")
+    return n.value
+
+
+def boost_llama_decode_step_host(model, scratch, tokens, block_table, max_blocks, ctx_lens, b, next_tokens,
+                                 stream=None):
+    """Host-buffer variant: tokens / block_table / ctx_lens / next_tokens are host arrays."""
+    n = C.c_uint32(0)
+    _check(lib().boost_llama_decode_step_host(C.addressof(model), C.addressof(scratch), _ptr(tokens),
+                                              _ptr(block_table), max_blocks, _ptr(ctx_lens), b,
+                                              _ptr(next_tokens), C.addressof(n), _stream(stream)),
+           "boost_llama_decode_step_host")
+    return n.value

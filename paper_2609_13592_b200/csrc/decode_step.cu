@@ -1,0 +1,84 @@
+// One decode step of a Llama-shaped model as a fixed sequence of launches on one stream.
+// Host code only: every step of the path runs in the kernels of the other files.
+#include <cuda_runtime.h>
+
+#include "host_common.h"
+
+namespace {
+
+struct Launcher {
+  void* stream;
+  uint32_t count = 0;
+  int rc = BOOST_OK;
+  bool ok() const { return rc == BOOST_OK; }
+  void run(int r) {
+    if (rc == BOOST_OK) { rc = r; ++count; }
+  }
+};
+
+int gemv(const boost_weight_t& w, const void* x, uint32_t B, void* y, int y_dtype, const void* residual,
+         const boost_llama_scratch_t* s, void* stream) {
+  return boost_gemv_tiered(w.page_ptr, w.order, (size_t)w.n_pages, (size_t)w.n_host_pages, w.N, w.K, x, B, y,
+                           y_dtype, residual, s->gemv_ws, s->gemv_ws_bytes, stream);
+}
+
+}  // namespace
+
+extern "C" int boost_llama_decode_step(const boost_llama_model_t* m, const boost_llama_scratch_t* s,
+                                       const int32_t* tokens, const int32_t* block_table,
+                                       uint32_t max_blocks, const int32_t* ctx_lens, uint32_t B,
+                                       int32_t* next_tokens, uint32_t* n_launches_out, void* stream) {
+  if (!m || !s || !tokens || !block_table || !ctx_lens || !next_tokens) return BOOST_ERR_INVALID;
+  if (B == 0 || B > 128 || !m->layers || m->n_layers == 0) return BOOST_ERR_INVALID;
+  if (!s->h || !s->xn || !s->qkv || !s->q_rot || !s->attn || !s->gu || !s->act || !s->logits ||
+      !s->gemv_ws || !s->attn_ws)
+    return BOOST_ERR_INVALID;
+  const uint32_t hq = m->n_q_heads, hkv = m->n_kv_heads, d = m->head_dim;
+  if (m->hidden != hq * d && m->hidden == 0) return BOOST_ERR_INVALID;
+  const float scale = 1.0f / sqrtf((float)d);
+  Launcher L{stream};
+  L.run(boost_embed_gather(m->embed, m->vocab, m->hidden, tokens, B, s->h, stream));
+  for (uint32_t li = 0; li < m->n_layers && L.ok(); ++li) {
+    const boost_llama_layer_t& ly = m->layers[li];
+    L.run(boost_rmsnorm(s->h, ly.norm1, B, m->hidden, m->rms_eps, s->xn, stream));
+    L.run(gemv(ly.wqkv, s->xn, B, s->qkv, 1, nullptr, s, stream));
+    L.run(boost_rope_kv_append(s->qkv, s->q_rot, ly.k_page_ptr, ly.v_page_ptr, m->n_pool_blocks, block_table,
+                               max_blocks, ctx_lens, B, hq, hkv, d, m->rope_base, s->attn_ws, stream));
+    L.run(boost_paged_attn_decode_tiered(s->q_rot, ly.k_page_ptr, ly.v_page_ptr, m->kv_tier,
+                                         (size_t)m->n_kv_pages, m->n_pool_blocks, block_table, max_blocks,
+                                         ctx_lens, B, hq, hkv, d, scale, s->attn_ws, s->attn_ws_bytes,
+                                         s->attn, stream));
+    L.run(gemv(ly.wo, s->attn, B, s->h, 1, s->h, s, stream));       // h += attn Wo^T
+    L.run(boost_rmsnorm(s->h, ly.norm2, B, m->hidden, m->rms_eps, s->xn, stream));
+    L.run(gemv(ly.wgu, s->xn, B, s->gu, 1, nullptr, s, stream));
+    L.run(boost_swiglu(s->gu, B, m->ffn, s->act, stream));
+    L.run(gemv(ly.wd, s->act, B, s->h, 1, s->h, s, stream));        // h += act Wd^T
+  }
+  L.run(boost_rmsnorm(s->h, m->norm_f, B, m->hidden, m->rms_eps, s->xn, stream));
+  L.run(gemv(m->lm_head, s->xn, B, s->logits, 0, nullptr, s, stream));
+  L.run(boost_argmax(s->logits, B, m->vocab, next_tokens, stream));
+  if (n_launches_out) *n_launches_out = L.count;
+  return L.rc;
+}
+
+extern "C" int boost_llama_decode_step_host(const boost_llama_model_t* m, const boost_llama_scratch_t* s,
+                                            const int32_t* tokens, const int32_t* block_table,
+                                            uint32_t max_blocks, const int32_t* ctx_lens, uint32_t B,
+                                            int32_t* next_tokens, uint32_t* n_launches_out, void* stream) {
+  if (!m || !s || !tokens || !block_table || !ctx_lens || !next_tokens) return BOOST_ERR_INVALID;
+  if (!s->tokens_dev || !s->ctx_dev || !s->table_dev || !s->next_dev) return BOOST_ERR_INVALID;
+  cudaStream_t st = (cudaStream_t)stream;
+  int rc = boosth::check(cudaMemcpyAsync(s->tokens_dev, tokens, (size_t)B * 4, cudaMemcpyHostToDevice, st));
+  if (rc == BOOST_OK)
+    rc = boosth::check(cudaMemcpyAsync(s->ctx_dev, ctx_lens, (size_t)B * 4, cudaMemcpyHostToDevice, st));
+  if (rc == BOOST_OK)
+    rc = boosth::check(cudaMemcpyAsync(s->table_dev, block_table, (size_t)B * max_blocks * 4,
+                                       cudaMemcpyHostToDevice, st));
+  if (rc != BOOST_OK) return rc;
+  rc = boost_llama_decode_step(m, s, s->tokens_dev, s->table_dev, max_blocks, s->ctx_dev, B, s->next_dev,
+                               n_launches_out, stream);
+  if (rc != BOOST_OK) return rc;
+  rc = boosth::check(cudaMemcpyAsync(next_tokens, s->next_dev, (size_t)B * 4, cudaMemcpyDeviceToHost, st));
+  if (rc != BOOST_OK) return rc;
+  return boosth::check(cudaStreamSynchronize(st));
+}

@@ -1,0 +1,180 @@
+"""GPU parity: the small operators of a decode step and the whole step against the oracle."""
+import numpy as np
+import pytest
+
+from oracle import decode as od
+from oracle import kv_pool as okp
+from oracle import linalg as ol
+from paper_2609_13592_b200 import binding as B
+from paper_2609_13592_b200 import synth
+from tests.helpers import assert_chain_close, assert_close_to_oracle
+
+torch = pytest.importorskip("torch")
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def dev():
+    if not torch.cuda.is_available():
+        pytest.skip("needs a CUDA device")
+    from paper_2609_13592_b200 import build
+    build.build_library()
+    B.lib()
+    return torch.device("cuda:0")
+
+
+def bf16_tensor(bits, dev):
+    return torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).to(dev).view(torch.bfloat16)
+
+
+def bits_of(t):
+    return t.contiguous().view(torch.int16).cpu().numpy().view(np.uint16)
+
+
+def test_embed_rmsnorm_swiglu_argmax(dev):
+    rng = np.random.default_rng(0)
+    vocab, hid, n_seq, ffn = 300, 512, 5, 384
+    table = synth.normal_bf16((vocab, hid), 0.02, 1)
+    tokens = np.array([0, 299, 17, 17, 123], np.int32)
+    out = torch.zeros(n_seq, hid, dtype=torch.bfloat16, device=dev)
+    B.boost_embed_gather(bf16_tensor(table, dev), vocab, hid, torch.from_numpy(tokens).to(dev), n_seq, out)
+    assert np.array_equal(bits_of(out), table[tokens])
+
+    x = synth.normal_bf16((n_seq, hid), 1.0, 2)
+    w = synth.f32_to_bf16_bits(1.0 + 0.1 * rng.standard_normal(hid).astype(np.float32))
+    y = torch.zeros(n_seq, hid, dtype=torch.bfloat16, device=dev)
+    B.boost_rmsnorm(bf16_tensor(x, dev), bf16_tensor(w, dev), n_seq, hid, od.RMS_EPS, y)
+    assert_close_to_oracle(y.float().cpu().numpy(), od.rmsnorm(ol.bf16_bits_to_f64(x), w), "rmsnorm")
+
+    gu = synth.normal_bf16((n_seq, 2 * ffn), 2.0, 3)
+    act = torch.zeros(n_seq, ffn, dtype=torch.bfloat16, device=dev)
+    B.boost_swiglu(bf16_tensor(gu, dev), n_seq, ffn, act)
+    g64 = ol.bf16_bits_to_f64(gu)
+    assert_close_to_oracle(act.float().cpu().numpy(), od.silu(g64[:, :ffn]) * g64[:, ffn:], "swiglu")
+
+    v = 128256
+    logits = rng.standard_normal((4, v)).astype(np.float32)
+    logits[1, 5000] = logits[1, 70000] = 9.0           # tie: lowest index wins
+    logits[2, v - 1] = 10.0
+    logits[3, 0] = 11.0
+    got = torch.zeros(4, dtype=torch.int32, device=dev)
+    B.boost_argmax(torch.from_numpy(logits).to(dev), 4, v, got)
+    torch.cuda.synchronize()
+    assert got.cpu().numpy().tolist() == np.argmax(logits, axis=-1).tolist() == [int(np.argmax(logits[0])), 5000, v - 1, 0]
+
+
+def test_rope_kv_append(dev):
+    from paper_2609_13592_b200.tiers import TieredKVCache
+    hq, hkv, d, n_blocks = 8, 2, 128, 512
+    pool = B.KVPool(n_blocks, hkv, 4)
+    cache = TieredKVCache(pool, hkv, n_blocks, d, dev)
+    k0 = synth.normal_bf16((hkv, n_blocks, 16, d), 1.0, 5)
+    v0 = synth.normal_bf16((hkv, n_blocks, 16, d), 1.0, 6)
+    cache.load(bf16_tensor(k0, dev), bf16_tensor(v0, dev))
+    ctx = np.array([1, 16, 17, 4000, 0], np.int32)
+    n_seq = len(ctx)
+    table = np.zeros((n_seq, 256), np.int32)
+    used = iter(np.random.default_rng(1).permutation(n_blocks))
+    for b in range(n_seq):
+        for j in range((ctx[b] + 15) // 16):
+            table[b, j] = next(used)
+    qkv = synth.normal_bf16((n_seq, (hq + 2 * hkv) * d), 1.0, 7)
+    q_out = torch.zeros(n_seq, hq, d, dtype=torch.bfloat16, device=dev)
+    status = torch.zeros(4, dtype=torch.int32, device=dev)
+    B.boost_rope_kv_append(bf16_tensor(qkv, dev), q_out, cache.k.page_ptr, cache.v.page_ptr, n_blocks,
+                           torch.from_numpy(table).to(dev), 256, torch.from_numpy(ctx).to(dev), n_seq, hq, hkv,
+                           d, od.ROPE_BASE, status)
+    torch.cuda.synchronize()
+    assert int(status[0]) == 0
+    x = ol.bf16_bits_to_f64(qkv)
+    pos = np.maximum(ctx - 1, 0)
+    q_ref = od.rope(x[:, :hq * d].reshape(n_seq, hq, d), pos)
+    k_ref = od.rope(x[:, hq * d:(hq + hkv) * d].reshape(n_seq, hkv, d), pos)
+    v_ref = x[:, (hq + hkv) * d:].reshape(n_seq, hkv, d)
+    live = ctx > 0
+    assert_close_to_oracle(q_out.float().cpu().numpy()[live], q_ref[live], "rope q")
+    k_now, v_now = (bits_of(t) for t in cache.dump())
+    k_want, v_want = k0.copy(), v0.copy()
+    for b in range(n_seq):
+        if ctx[b] == 0:
+            continue
+        blk, slot = table[b, pos[b] // 16], pos[b] % 16
+        assert_close_to_oracle(ol.bf16_bits_to_f64(k_now[:, blk, slot]), k_ref[b], "rope k")
+        assert np.array_equal(ol.bf16_bits_to_f64(v_now[:, blk, slot]), v_ref[b])
+        k_want[:, blk, slot] = k_now[:, blk, slot]
+        v_want[:, blk, slot] = v_now[:, blk, slot]
+    # nothing else in the cache was touched
+    assert np.array_equal(k_now, k_want) and np.array_equal(v_now, v_want)
+    pool.close()
+
+
+def build_decoder(dev, cfg, w, n_pool_blocks, kv_modulus, weight_ratio, max_batch, max_blocks):
+    from paper_2609_13592_b200.llama import LlamaDecoder
+
+    def get_weight(name, layer):
+        src = w[name] if layer is None else w["layers"][layer][name]
+        return bf16_tensor(src, dev)
+
+    return LlamaDecoder(cfg, get_weight, weight_ratio, n_pool_blocks, kv_modulus, max_batch, max_blocks, dev)
+
+
+@pytest.mark.parametrize("n_seq,kv_modulus,weight_ratio", [(3, 4, 0.5), (1, 0, 0.0), (20, 2, 0.25)])
+def test_decode_steps_match_oracle(dev, n_seq, kv_modulus, weight_ratio):
+    cfg = dict(synth.TINY_LLAMA)
+    w = synth.llama_weights(cfg, seed=n_seq, std=0.05)
+    hkv, d, nl = cfg["n_kv_heads"], cfg["head_dim"], cfg["n_layers"]
+    n_pool_blocks, max_blocks = 512, 8
+    dec = build_decoder(dev, cfg, w, n_pool_blocks, kv_modulus, weight_ratio, max(n_seq, 4), max_blocks)
+    ref_pool = okp.KVPool(n_pool_blocks, hkv, kv_modulus, 16 * d * 2)
+    assert dec.kv_tier.tolist() == ref_pool.page_tiers()
+    # start each sequence with a random prefix already in the cache (prefill stand-in)
+    rng = np.random.default_rng(10 + n_seq)
+    prefix = rng.integers(0, 40, size=n_seq)
+    k_host = [synth.normal_bf16((hkv, n_pool_blocks, 16, d), 1.0, 100 + li) for li in range(nl)]
+    v_host = [synth.normal_bf16((hkv, n_pool_blocks, 16, d), 1.0, 200 + li) for li in range(nl)]
+    for li in range(nl):
+        B.boost_kv_scatter(bf16_tensor(k_host[li], dev), hkv, n_pool_blocks, d, dec.layers[li]["k"].page_ptr,
+                           dec.layers[li]["k"].n_pages)
+        B.boost_kv_scatter(bf16_tensor(v_host[li], dev), hkv, n_pool_blocks, d, dec.layers[li]["v"].page_ptr,
+                           dec.layers[li]["v"].n_pages)
+    table = np.zeros((n_seq, max_blocks), np.int32)
+    n_have = np.zeros(n_seq, np.int64)
+    ctx = prefix.astype(np.int64).copy()
+    tokens = rng.integers(0, cfg["vocab"], size=n_seq).astype(np.int32)
+    tok_pin = torch.zeros(n_seq, dtype=torch.int32).pin_memory()
+    ctx_pin = torch.zeros(n_seq, dtype=torch.int32).pin_memory()
+    tab_pin = torch.zeros(n_seq, max_blocks, dtype=torch.int32).pin_memory()
+    nxt_pin = torch.zeros(n_seq, dtype=torch.int32).pin_memory()
+    for step in range(20):
+        ctx += 1                                           # the new token joins the context
+        for b in range(n_seq):                             # blocks through the pool, both sides
+            while n_have[b] * 16 < ctx[b]:
+                got = dec.pool.alloc(b, 1).tolist()
+                assert got == ref_pool.alloc(b, 1)
+                table[b, n_have[b]] = got[0]
+                n_have[b] += 1
+        tok_pin.numpy()[:] = tokens
+        ctx_pin.numpy()[:] = ctx
+        tab_pin.numpy()[:] = table
+        n_launch = dec.step_host(tok_pin.numpy(), tab_pin.numpy(), ctx_pin.numpy(), nxt_pin.numpy())
+        assert n_launch == 1 + 10 * nl + 3
+        ref = od.decode_step(cfg, w, tokens, k_host, v_host, table, ctx)
+        logits = dec.buf["logits"][:n_seq].cpu().numpy()
+        assert_chain_close(logits, ref["logits"], f"logits step {step}")
+        got_next = nxt_pin.numpy().copy()
+        # the device's own argmax of its own logits (integer work: exact) ...
+        assert np.array_equal(got_next, np.argmax(logits, axis=-1))
+        # ... and against the oracle wherever its top two logits are separated by more than the tolerance
+        top2 = np.sort(ref["logits"], axis=-1)[:, -2:]
+        clear = (top2[:, 1] - top2[:, 0]) > 4e-2
+        assert np.array_equal(got_next[clear], ref["next_tokens"][clear])
+        tokens = ref["next_tokens"].astype(np.int32)       # both sides continue from the oracle's choice
+    assert dec.status_words() == [0, 0]
+    # the device cache now holds what the oracle's cache holds (new K/V rounded to bf16 on both sides)
+    for li in range(nl):
+        for name, host in (("k", k_host), ("v", v_host)):
+            t = torch.empty(hkv, n_pool_blocks, 16, d, dtype=torch.bfloat16, device=dev)
+            B.boost_kv_gather(t, hkv, n_pool_blocks, d, dec.layers[li][name].page_ptr, dec.layers[li][name].n_pages)
+            got = ol.bf16_bits_to_f64(bits_of(t))
+            want = ol.bf16_bits_to_f64(host[li])
+            assert_chain_close(got, want, f"cache {name}{li}")
