@@ -39,19 +39,31 @@ def assert_close_to_oracle(got, ref, what=""):
     return int((np.abs(ref) < floor).sum())
 
 
-def assert_chain_close(got, ref, what=""):
-    """Outputs of a CHAIN of kernels with bf16 tensors in between (a whole decode step).
-    One bf16 rounding that falls the other way on the two sides moves an intermediate by
-    2^-8 relative and every output by about that fraction of the output's typical size, so
-    element-wise relative error near zero crossings is not meaningful here: the error is
-    bounded by 2e-2 absolute and by 1e-2 of max(|ref|, rms(ref)).  Each kernel of the chain
-    is held to the strict tolerance in its own test."""
+CHAIN_REL_TOL = 3e-2
+
+
+def chain_error(got, ref):
+    """max |got - ref| / max(|ref|, rms(ref)) and max abs error."""
     import numpy as np
     got = np.asarray(got, dtype=np.float64)
     ref = np.asarray(ref, dtype=np.float64)
-    assert got.shape == ref.shape and np.isfinite(got).all(), what
+    assert got.shape == ref.shape and np.isfinite(got).all()
     err = np.abs(got - ref)
     rms = float(np.sqrt((ref * ref).mean())) if ref.size else 0.0
     denom = np.maximum(np.abs(ref), rms if rms > 0 else 1.0)
-    assert err.max(initial=0.0) <= ABS_TOL, f"{what}: max abs err {err.max():.3e}"
-    assert (err / denom).max(initial=0.0) <= REL_TOL, f"{what}: max err / max(|ref|, rms) {(err / denom).max():.3e}"
+    return float((err / denom).max(initial=0.0)), float(err.max(initial=0.0))
+
+
+def assert_chain_close(got, ref, what=""):
+    """Outputs of a CHAIN of kernels with bf16 tensors in between (a whole decode step).
+    Where the fp32 device value and the fp64 oracle value of an intermediate fall on
+    different sides of a bf16 rounding boundary, that intermediate differs by one bf16 ulp
+    (2^-8 relative) and the outputs move by a fraction of their typical size: about 1.3 % of
+    rms(logits) per such event in the 256-wide test model (measured with a numpy fp32
+    emulation of the same chain, no CUDA involved).  Element-wise relative error is
+    therefore not meaningful for a chain; the bound is 2e-2 absolute and 3e-2 of
+    max(|ref|, rms(ref)).  Every kernel of the chain is held to the strict tolerance in its
+    own test, and callers also check that most rows agree to 1e-4 (no such event)."""
+    rel, abs_err = chain_error(got, ref)
+    assert abs_err <= ABS_TOL, f"{what}: max abs err {abs_err:.3e}"
+    assert rel <= CHAIN_REL_TOL, f"{what}: max err / max(|ref|, rms) {rel:.3e}"

@@ -46,7 +46,7 @@ def test_embed_rmsnorm_swiglu_argmax(dev):
     B.boost_rmsnorm(bf16_tensor(x, dev), bf16_tensor(w, dev), n_seq, hid, od.RMS_EPS, y)
     assert_close_to_oracle(y.float().cpu().numpy(), od.rmsnorm(ol.bf16_bits_to_f64(x), w), "rmsnorm")
 
-    gu = synth.normal_bf16((n_seq, 2 * ffn), 2.0, 3)
+    gu = synth.normal_bf16((n_seq, 2 * ffn), 0.4, 3)   # outputs stay below 4: half a bf16 ulp < 2e-2
     act = torch.zeros(n_seq, ffn, dtype=torch.bfloat16, device=dev)
     B.boost_swiglu(bf16_tensor(gu, dev), n_seq, ffn, act)
     g64 = ol.bf16_bits_to_f64(gu)
@@ -118,25 +118,35 @@ def build_decoder(dev, cfg, w, n_pool_blocks, kv_modulus, weight_ratio, max_batc
     return LlamaDecoder(cfg, get_weight, weight_ratio, n_pool_blocks, kv_modulus, max_batch, max_blocks, dev)
 
 
+def load_caches(dev, dec, k_host, v_host):
+    hkv, d = dec.cfg["n_kv_heads"], dec.cfg["head_dim"]
+    for li, ly in enumerate(dec.layers):
+        B.boost_kv_scatter(bf16_tensor(k_host[li], dev), hkv, dec.n_pool_blocks, d, ly["k"].page_ptr, ly["k"].n_pages)
+        B.boost_kv_scatter(bf16_tensor(v_host[li], dev), hkv, dec.n_pool_blocks, d, ly["v"].page_ptr, ly["v"].n_pages)
+
+
+def dump_cache(dev, dec, li, name):
+    hkv, d = dec.cfg["n_kv_heads"], dec.cfg["head_dim"]
+    t = torch.empty(hkv, dec.n_pool_blocks, 16, d, dtype=torch.bfloat16, device=dev)
+    B.boost_kv_gather(t, hkv, dec.n_pool_blocks, d, dec.layers[li][name].page_ptr, dec.layers[li][name].n_pages)
+    return bits_of(t)
+
+
 @pytest.mark.parametrize("n_seq,kv_modulus,weight_ratio", [(3, 4, 0.5), (1, 0, 0.0), (20, 2, 0.25)])
 def test_decode_steps_match_oracle(dev, n_seq, kv_modulus, weight_ratio):
+    from tests.helpers import chain_error
     cfg = dict(synth.TINY_LLAMA)
-    w = synth.llama_weights(cfg, seed=n_seq, std=0.05)
+    w = synth.llama_weights(cfg, seed=n_seq, std=0.02)
     hkv, d, nl = cfg["n_kv_heads"], cfg["head_dim"], cfg["n_layers"]
     n_pool_blocks, max_blocks = 512, 8
     dec = build_decoder(dev, cfg, w, n_pool_blocks, kv_modulus, weight_ratio, max(n_seq, 4), max_blocks)
     ref_pool = okp.KVPool(n_pool_blocks, hkv, kv_modulus, 16 * d * 2)
     assert dec.kv_tier.tolist() == ref_pool.page_tiers()
-    # start each sequence with a random prefix already in the cache (prefill stand-in)
+    # every sequence starts with a random prefix already in the cache (prefill stand-in)
     rng = np.random.default_rng(10 + n_seq)
     prefix = rng.integers(0, 40, size=n_seq)
     k_host = [synth.normal_bf16((hkv, n_pool_blocks, 16, d), 1.0, 100 + li) for li in range(nl)]
     v_host = [synth.normal_bf16((hkv, n_pool_blocks, 16, d), 1.0, 200 + li) for li in range(nl)]
-    for li in range(nl):
-        B.boost_kv_scatter(bf16_tensor(k_host[li], dev), hkv, n_pool_blocks, d, dec.layers[li]["k"].page_ptr,
-                           dec.layers[li]["k"].n_pages)
-        B.boost_kv_scatter(bf16_tensor(v_host[li], dev), hkv, n_pool_blocks, d, dec.layers[li]["v"].page_ptr,
-                           dec.layers[li]["v"].n_pages)
     table = np.zeros((n_seq, max_blocks), np.int32)
     n_have = np.zeros(n_seq, np.int64)
     ctx = prefix.astype(np.int64).copy()
@@ -145,7 +155,11 @@ def test_decode_steps_match_oracle(dev, n_seq, kv_modulus, weight_ratio):
     ctx_pin = torch.zeros(n_seq, dtype=torch.int32).pin_memory()
     tab_pin = torch.zeros(n_seq, max_blocks, dtype=torch.int32).pin_memory()
     nxt_pin = torch.zeros(n_seq, dtype=torch.int32).pin_memory()
-    for step in range(20):
+    exact_rows = total_rows = 0
+    for step in range(16):
+        # both sides start every step from the same cache, so that a bf16 rounding that fell
+        # differently in an earlier step does not carry over
+        load_caches(dev, dec, k_host, v_host)
         ctx += 1                                           # the new token joins the context
         for b in range(n_seq):                             # blocks through the pool, both sides
             while n_have[b] * 16 < ctx[b]:
@@ -157,24 +171,31 @@ def test_decode_steps_match_oracle(dev, n_seq, kv_modulus, weight_ratio):
         ctx_pin.numpy()[:] = ctx
         tab_pin.numpy()[:] = table
         n_launch = dec.step_host(tok_pin.numpy(), tab_pin.numpy(), ctx_pin.numpy(), nxt_pin.numpy())
-        assert n_launch == 1 + 10 * nl + 3
+        assert n_launch == 1 + 9 * nl + 3
         ref = od.decode_step(cfg, w, tokens, k_host, v_host, table, ctx)
         logits = dec.buf["logits"][:n_seq].cpu().numpy()
         assert_chain_close(logits, ref["logits"], f"logits step {step}")
+        for b in range(n_seq):
+            total_rows += 1
+            exact_rows += chain_error(logits[b], ref["logits"][b])[0] < 1e-4
         got_next = nxt_pin.numpy().copy()
         # the device's own argmax of its own logits (integer work: exact) ...
         assert np.array_equal(got_next, np.argmax(logits, axis=-1))
-        # ... and against the oracle wherever its top two logits are separated by more than the tolerance
+        # ... and against the oracle wherever its top two logits are clearly separated
         top2 = np.sort(ref["logits"], axis=-1)[:, -2:]
         clear = (top2[:, 1] - top2[:, 0]) > 4e-2
         assert np.array_equal(got_next[clear], ref["next_tokens"][clear])
+        # the K/V rows written by this step
+        pos = ctx - 1
+        for li in range(nl):
+            for name, host in (("k", k_host), ("v", v_host)):
+                now = dump_cache(dev, dec, li, name)
+                for b in range(n_seq):
+                    blk, slot = table[b, pos[b] // 16], pos[b] % 16
+                    assert_chain_close(ol.bf16_bits_to_f64(now[:, blk, slot]),
+                                       ol.bf16_bits_to_f64(host[li][:, blk, slot]), f"new {name} row")
+                    now[:, blk, slot] = host[li][:, blk, slot]
+                assert np.array_equal(now, host[li])       # nothing else was written
         tokens = ref["next_tokens"].astype(np.int32)       # both sides continue from the oracle's choice
     assert dec.status_words() == [0, 0]
-    # the device cache now holds what the oracle's cache holds (new K/V rounded to bf16 on both sides)
-    for li in range(nl):
-        for name, host in (("k", k_host), ("v", v_host)):
-            t = torch.empty(hkv, n_pool_blocks, 16, d, dtype=torch.bfloat16, device=dev)
-            B.boost_kv_gather(t, hkv, n_pool_blocks, d, dec.layers[li][name].page_ptr, dec.layers[li][name].n_pages)
-            got = ol.bf16_bits_to_f64(bits_of(t))
-            want = ol.bf16_bits_to_f64(host[li])
-            assert_chain_close(got, want, f"cache {name}{li}")
+    assert exact_rows >= 0.6 * total_rows, (exact_rows, total_rows)
