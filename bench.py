@@ -1,0 +1,478 @@
+#!/usr/bin/env python
+"""Benchmark of the tiered decode hot path on B200.
+
+Default workload (N = 1): one Llama-3-8B-shaped decode step - 32 layers, hidden 4096, FFN
+14336, 32 query / 8 KV heads, vocab 128256, bf16 random-init weights N(0, 0.02^2), batch
+32, context 2048 - with weight pages placed by modulo placement at the host share that the
+measured host-link / HBM bandwidth ratio gives, KV cache in HBM.  A step runs every kernel
+of the path (embedding, 32 x [RMSNorm, QKV, RoPE + KV append, paged attention, output
+projection, RMSNorm, gate/up, SwiGLU, down], final norm, LM head, argmax) through the C ABI.
+
+  python bench.py --gpus N --steps K --warmup W            # this repository's kernels
+  python bench.py --impl reference ...                      # the CPU oracle on the host cores
+
+Prints ONE JSON line on rank 0.  With N > 1 every rank runs an independent replica (the
+path does not shard across GPUs; no collective on the data path) and the value is the sum
+over ranks divided by the slowest rank's time.
+"""
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+WORKLOAD = "llama3_8b_shaped_decode_step_b32_ctx2048_tiered_weights"
+FALLBACK_HBM_GBS = 6650.0
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as fh:
+            p = json.load(fh)
+        return float(p["hbm_gbs"]), "measured (MEASURED_PEAKS.json)"
+    return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index):
+        self.gpu_index = gpu_index
+        self.proc = None
+        self.tmp = None
+
+    def start(self):
+        try:
+            self.tmp = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.gpu_index), f"--query-gpu={self.QUERY}",
+                 "--format=csv,noheader,nounits", "-lms", "100"], stdout=self.tmp, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        self.tmp.flush()
+        self.tmp.seek(0)
+        clocks, reasons, mx = [], set(), None
+        for line in self.tmp.read().splitlines():
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                clocks.append(float(f[1]))
+                mx = float(f[2])
+            except ValueError:
+                continue
+            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"),
+                                 f[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        try:
+            os.unlink(self.tmp.name)
+        except OSError:
+            pass
+        if clocks:
+            out.update(sm_mhz=float(np.median(clocks)), sm_max_mhz=mx, reasons=sorted(reasons),
+                       samples=len(clocks))
+        return out
+
+
+# --------------------------------------------------------------------------- CPU oracle leg
+
+def cpu_oracle_sample(batch, ctx, seed=0):
+    """Times the CPU oracle (as it stands) on a bounded sample of the default workload: one of
+    the 32 layers plus the LM head at full batch and context; the layer time is scaled by 32.
+    Returns (tokens_per_s, description, threads)."""
+    from oracle import decode as od
+    from paper_2609_13592_b200 import synth
+    cfg = dict(synth.LLAMA3_8B, n_layers=1)
+    hq, hkv, d, hid, ffn, vocab = (cfg[k] for k in ("n_q_heads", "n_kv_heads", "head_dim", "hidden", "ffn", "vocab"))
+    head = synth.normal_bf16((vocab, hid), 0.02, seed + 1)
+    layer = {"norm1": synth.f32_to_bf16_bits(np.ones(hid, np.float32)),
+             "norm2": synth.f32_to_bf16_bits(np.ones(hid, np.float32)),
+             "wqkv": synth.normal_bf16(((hq + 2 * hkv) * d, hid), 0.02, seed + 2),
+             "wo": synth.normal_bf16((hid, hq * d), 0.02, seed + 3),
+             "wgu": synth.normal_bf16((2 * ffn, hid), 0.02, seed + 4),
+             "wd": synth.normal_bf16((hid, ffn), 0.02, seed + 5)}
+    w = {"embed": head, "lm_head": head, "norm_f": layer["norm1"], "layers": [layer]}
+    n_blk_seq = (ctx + 15) // 16
+    n_blocks = batch * n_blk_seq
+    kc = [synth.normal_bf16((hkv, n_blocks, 16, d), 1.0, seed + 6)]
+    vc = [synth.normal_bf16((hkv, n_blocks, 16, d), 1.0, seed + 7)]
+    table = np.arange(n_blocks, dtype=np.int64).reshape(batch, n_blk_seq)
+    tokens = np.arange(batch) * 97 % vocab
+    ctx_lens = np.full(batch, ctx)
+    t0 = time.perf_counter()
+    od.decode_step(cfg, w, tokens, kc, vc, table, ctx_lens, n_layers=0)
+    t_head = time.perf_counter() - t0
+    t0 = time.perf_counter()
+    od.decode_step(cfg, w, tokens, kc, vc, table, ctx_lens, n_layers=1)
+    t_one = time.perf_counter() - t0
+    t_layer = max(t_one - t_head, 1e-9)
+    t_step = 32 * t_layer + t_head
+    try:
+        from threadpoolctl import threadpool_info
+        threads = max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
+    except Exception:
+        threads = os.cpu_count() or 1
+    desc = (f"1 of 32 layers + LM head at batch {batch}, context {ctx} "
+            f"(layer {t_layer:.2f} s x 32 + head {t_head:.2f} s)")
+    return batch / t_step, desc, threads, t_one + t_head
+
+
+def run_reference(args, rank, world):
+    if rank != 0:
+        return
+    steps, vals = max(1, min(args.steps, 3)), []
+    for _ in range(max(0, min(args.warmup, 1))):
+        cpu_oracle_sample(32, 2048)
+    desc, threads = "", 1
+    t_total = 0.0
+    for _ in range(steps):
+        v, desc, threads, t = cpu_oracle_sample(32, 2048)
+        vals.append(v)
+        t_total += t
+    value = float(np.mean(vals))
+    line = {"impl": "reference", "metric": "decode_tokens_per_s", "value": value, "unit": "tokens/s",
+            "n_gpus": args.gpus, "steps": steps, "warmup": min(args.warmup, 1),
+            "ms_per_step": 1000.0 * 32 / value, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": WORKLOAD, "note": "CPU oracle on the host cores, bounded sample per step"},
+            "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": threads, "kind": "oracle", "sample": desc},
+            "e2e": {"value": value, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+# ------------------------------------------------------------------------------ device leg
+
+def measure_stream(dev, n_pages, tier_value, reps=5):
+    """GB/s of the tiered stream-reduce kernel over n_pages pages all in one tier."""
+    import torch
+    from paper_2609_13592_b200 import binding as B
+    from paper_2609_13592_b200.tiers import TieredBuffer
+    tier = np.full(n_pages, tier_value, np.uint8)
+    buf = TieredBuffer(n_pages * B.PAGE_BYTES, device=dev, tier=tier)
+    ws_bytes = B.boost_stream_reduce_workspace_bytes(n_pages)
+    ws = torch.zeros(ws_bytes, dtype=torch.uint8, device=dev)
+    sums = torch.zeros(n_pages, dtype=torch.float32, device=dev)
+    best = float("inf")
+    for i in range(reps + 2):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        B.boost_stream_reduce_tiered(buf.page_ptr, buf.order, n_pages, buf.n_host, sums, ws, ws_bytes)
+        e1.record()
+        torch.cuda.synchronize(dev)
+        if i >= 2:
+            best = min(best, e0.elapsed_time(e1))
+    del buf
+    return n_pages * B.PAGE_BYTES / best / 1e6
+
+
+def build_decoder(dev, cfg, host_ratio, batch, n_pool_blocks, max_blocks, seed):
+    import torch
+    from paper_2609_13592_b200.llama import LlamaDecoder
+    hq, hkv, d, hid, ffn, vocab = (cfg[k] for k in ("n_q_heads", "n_kv_heads", "head_dim", "hidden", "ffn", "vocab"))
+    shapes = {"embed": (vocab, hid), "lm_head": (vocab, hid), "wqkv": ((hq + 2 * hkv) * d, hid),
+              "wo": (hid, hq * d), "wgu": (2 * ffn, hid), "wd": (hid, ffn)}
+    names = ["embed", "norm_f", "lm_head", "norm1", "wqkv", "wo", "norm2", "wgu", "wd"]
+
+    def get_weight(name, layer):
+        g = torch.Generator(device=dev)
+        g.manual_seed(seed * 100003 + (0 if layer is None else layer + 1) * 101 + names.index(name))
+        if name.startswith("norm"):
+            return (1.0 + 0.02 * torch.randn(hid, generator=g, device=dev)).to(torch.bfloat16)
+        return (0.02 * torch.randn(shapes[name], generator=g, device=dev)).to(torch.bfloat16)
+
+    dec = LlamaDecoder(cfg, get_weight, host_ratio, n_pool_blocks, 0, batch, max_blocks, dev)
+    g = torch.Generator(device=dev)
+    g.manual_seed(seed + 7)
+    for ly in dec.layers:                      # synthetic context: KV ~ N(0, 1)
+        for name in ("k", "v"):
+            ly[name]._hbm.view(torch.bfloat16).normal_(0.0, 1.0, generator=g)
+    torch.cuda.synchronize(dev)
+    return dec
+
+
+class StepDriver:
+    """Holds the per-step inputs of a run of consecutive decode steps of one decoder."""
+
+    def __init__(self, dec, dev, batch, ctx0, n_steps, max_blocks):
+        import torch
+        self.dec, self.dev, self.batch, self.ctx0, self.max_blocks = dec, dev, batch, ctx0, max_blocks
+        need0 = (ctx0 + 15) // 16
+        self.table = np.zeros((batch, max_blocks), np.int32)
+        self.n_have = np.zeros(batch, np.int64)
+        for j in range(need0):                 # round-robin growth through the wave-aware pool
+            for b in range(batch):
+                self.table[b, j] = dec.pool.alloc(b, 1)[0]
+        self.n_have[:] = need0
+        self.ctx = np.full(batch, ctx0 - 1, np.int64)   # the first step brings it to ctx0
+        self.torch = torch
+
+    def advance(self):
+        """Next step's context lengths; new blocks come from the pool when a sequence crosses
+        a block boundary."""
+        self.ctx += 1
+        for b in range(self.batch):
+            while self.n_have[b] * 16 < self.ctx[b]:
+                self.table[b, self.n_have[b]] = self.dec.pool.alloc(b, 1)[0]
+                self.n_have[b] += 1
+        return self.ctx
+
+    def release(self):
+        for b in range(self.batch):
+            self.dec.pool.free(b)
+
+
+def timed_device_steps(dec, dev, batch, ctx0, warmup, steps, max_blocks, dist_ctx):
+    """Device-resident loop: inputs already in HBM; K steps between two events."""
+    import torch
+    drv = StepDriver(dec, dev, batch, ctx0, warmup + steps, max_blocks)
+    ctx_all = np.zeros((warmup + steps, batch), np.int32)
+    for i in range(warmup + steps):
+        ctx_all[i] = drv.advance()
+    ctx_dev = torch.from_numpy(ctx_all).to(dev)
+    table_dev = torch.from_numpy(drv.table).to(dev)
+    tok = [torch.arange(batch, dtype=torch.int32, device=dev) * 97 % dec.cfg["vocab"],
+           torch.zeros(batch, dtype=torch.int32, device=dev)]
+    stream = torch.cuda.current_stream(dev)
+    launches = 0
+    for i in range(warmup):
+        dec.step(tok[i % 2], table_dev, ctx_dev[i], tok[(i + 1) % 2], stream)
+    dist_ctx.barrier()
+    torch.cuda.synchronize(dev)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for i in range(warmup, warmup + steps):
+        launches += dec.step(tok[i % 2], table_dev, ctx_dev[i], tok[(i + 1) % 2], stream)
+    e1.record(stream)
+    torch.cuda.synchronize(dev)
+    dist_ctx.barrier()
+    ms = e0.elapsed_time(e1)
+    kv_tokens = int(ctx_all[warmup:].sum())
+    # per-kind device time of one more step (events around every launch)
+    i = warmup + steps - 1
+    from paper_2609_13592_b200 import binding as B
+    kind_ms, kind_n = B.boost_llama_decode_step_profile(dec.model, dec.scratch, tok[i % 2], table_dev,
+                                                        max_blocks, ctx_dev[i], batch, tok[(i + 1) % 2], stream)
+    drv.release()
+    return ms, launches, kv_tokens, kind_ms, kind_n
+
+
+def timed_host_steps(dec, dev, batch, ctx0, warmup, steps, max_blocks, dist_ctx):
+    """End-to-end loop through the host-buffer entry point: per step the tokens, context
+    lengths and block table go host -> device and the next tokens come back."""
+    import torch
+    drv = StepDriver(dec, dev, batch, ctx0, warmup + steps, max_blocks)
+    tok_pin = torch.zeros(batch, dtype=torch.int32).pin_memory()
+    ctx_pin = torch.zeros(batch, dtype=torch.int32).pin_memory()
+    tab_pin = torch.zeros(batch, max_blocks, dtype=torch.int32).pin_memory()
+    nxt_pin = torch.zeros(batch, dtype=torch.int32).pin_memory()
+    tok_pin.numpy()[:] = np.arange(batch) * 97 % dec.cfg["vocab"]
+    stream = torch.cuda.current_stream(dev)
+
+    def one_step():
+        ctx_pin.numpy()[:] = drv.advance()
+        tab_pin.numpy()[:] = drv.table
+        dec.step_host(tok_pin.numpy(), tab_pin.numpy(), ctx_pin.numpy(), nxt_pin.numpy(), stream)
+        tok_pin.numpy()[:] = nxt_pin.numpy()         # the generated token is the next input
+
+    for _ in range(warmup):
+        one_step()
+    dist_ctx.barrier()
+    torch.cuda.synchronize(dev)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(steps):
+        one_step()
+    e1.record(stream)
+    torch.cuda.synchronize(dev)
+    dist_ctx.barrier()
+    ms = e0.elapsed_time(e1)
+    drv.release()
+    h2d = batch * 4 * 2 + batch * max_blocks * 4
+    d2h = batch * 4
+    return ms, h2d, d2h
+
+
+class DistCtx:
+    def __init__(self, rank, world, dev):
+        self.rank, self.world, self.dev = rank, world, dev
+        self.dist = None
+        if world > 1:
+            import torch.distributed as dist
+            dist.init_process_group(backend="nccl", device_id=dev)
+            self.dist = dist
+
+    def barrier(self):
+        if self.dist is not None:
+            self.dist.barrier()
+
+    def max(self, x):
+        if self.dist is None:
+            return x
+        import torch
+        t = torch.tensor([x], dtype=torch.float64, device=self.dev)
+        self.dist.all_reduce(t, op=self.dist.ReduceOp.MAX)
+        return float(t.item())
+
+    def close(self):
+        if self.dist is not None:
+            self.dist.destroy_process_group()
+
+
+def run_ours(args, rank, world, local_rank):
+    import torch
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the path has no CPU fallback")
+    from paper_2609_13592_b200 import binding as B
+    from paper_2609_13592_b200 import build as libbuild
+    from paper_2609_13592_b200 import synth
+    libbuild.build_library()
+    B.lib()
+    dev = torch.device(f"cuda:{local_rank}")
+    torch.cuda.set_device(dev)
+    dist_ctx = DistCtx(rank, world, dev)
+    hbm_peak, peak_src = load_peaks()
+
+    # host-link and HBM read bandwidth of this machine, measured in this run with the same kernel
+    link_gbs = measure_stream(dev, 64, 1)            # 128 MiB of host-mapped pinned pages
+    hbm_read_gbs = measure_stream(dev, 1024, 0)      # 2 GiB in HBM
+    modulus = B.boost_modulus_from_bandwidths(hbm_peak, link_gbs)
+    host_ratio = 1.0 / modulus
+
+    cfg = dict(synth.LLAMA3_8B)
+    if args.layers:
+        cfg["n_layers"] = args.layers
+    batch, ctx0 = args.batch, args.ctx
+    total_steps = args.warmup + args.steps
+    blocks_per_seq = (ctx0 + total_steps + 15) // 16 + 1
+    max_blocks = blocks_per_seq
+    n_pool_blocks = -(-batch * blocks_per_seq // 512) * 512
+
+    results = {}
+    clocks = None
+    for label, ratio in (("hbm_only", 0.0), ("tiered", host_ratio)):
+        dec = build_decoder(dev, cfg, ratio, batch, n_pool_blocks, max_blocks, seed=1)
+        sampler = ClockSampler(local_rank)
+        if label == "tiered":
+            sampler.start()
+        ms, launches, kv_tokens, kind_ms, kind_n = timed_device_steps(dec, dev, batch, ctx0, args.warmup,
+                                                                     args.steps, max_blocks, dist_ctx)
+        if label == "tiered":
+            clocks = sampler.stop()
+        r = {"ms": dist_ctx.max(ms), "launches": launches, "kv_tokens": kv_tokens, "kind_ms": kind_ms,
+             "kind_n": kind_n, "weight_bytes": dec.weight_bytes(), "kv_bytes_per_token": dec.kv_bytes_per_token(),
+             "host_pages": dec.host_weight_pages(), "status": dec.status_words()}
+        if label == "tiered":
+            e_ms, h2d, d2h = timed_host_steps(dec, dev, batch, ctx0, args.warmup, args.steps, max_blocks, dist_ctx)
+            r.update(e2e_ms=dist_ctx.max(e_ms), h2d=h2d, d2h=d2h)
+        results[label] = r
+        del dec
+        torch.cuda.empty_cache()
+
+    if rank == 0:
+        t = results["tiered"]
+        ms_step = t["ms"] / args.steps
+        value = world * batch / (ms_step / 1e3)
+        bytes_step = t["weight_bytes"] + t["kv_tokens"] / args.steps * t["kv_bytes_per_token"]
+        combined = bytes_step / (ms_step / 1e3) / 1e9
+        roof = hbm_peak + link_gbs
+        gemv_ms, gemv_n = t["kind_ms"][0], t["kind_n"][0]
+        gemv_gbs = t["weight_bytes"] / (gemv_ms / 1e3) / 1e9
+        attn_ms, attn_n = t["kind_ms"][1], t["kind_n"][1]
+        attn_bytes = t["kv_tokens"] / args.steps * t["kv_bytes_per_token"]
+        attn_gbs = attn_bytes / (attn_ms / 1e3) / 1e9
+        hb = results["hbm_only"]
+        hb_ms = hb["ms"] / args.steps
+        line = {
+            "metric": "decode_tokens_per_s", "value": value, "unit": "tokens/s", "n_gpus": world,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": WORKLOAD, "batch": batch, "context": ctx0, "layers": cfg["n_layers"],
+                       "weight_placement": f"modulo, host share 1/{modulus} per tensor",
+                       "kv_placement": "HBM", "l2": "inputs larger than L2 (weights 15 GB per step)",
+                       "multi_gpu": "replicas only" if world > 1 else "single GPU"},
+            "tpot_ms": ms_step,
+            "combined_read_gbs": combined,
+            "combined_roofline_gbs": roof,
+            "combined_roofline_frac": combined / roof,
+            "hbm_peak_gbs": hbm_peak, "hbm_peak_source": peak_src,
+            "host_link": {"type": "PCIe (zero-copy SM loads of pinned host memory)", "read_gbs": link_gbs,
+                          "alpha": link_gbs / hbm_peak, "modulus": modulus},
+            "hbm_read_gbs_stream_kernel": hbm_read_gbs,
+            "algorithmic_bytes_per_step": bytes_step,
+            "host_weight_pages": t["host_pages"],
+            "hbm_only": {"ms_per_step": hb_ms, "value": world * batch / (hb_ms / 1e3),
+                         "tiered_over_hbm_only_time": ms_step / hb_ms},
+            "roofline": {"bound": "hbm", "kernel": "gemv_tiered_kernel (weight products, M_b = 32)",
+                         "achieved": gemv_gbs, "peak": hbm_peak, "unit": "GB/s", "frac": gemv_gbs / hbm_peak,
+                         "traffic": None, "launches_per_step": gemv_n, "avg_launch_us": 1e3 * gemv_ms / max(gemv_n, 1),
+                         "peak_source": peak_src},
+            "roofline_attention": {"bound": "hbm", "kernel": "paged_attn_kernel", "achieved": attn_gbs,
+                                   "peak": hbm_peak, "unit": "GB/s", "frac": attn_gbs / hbm_peak,
+                                   "launches_per_step": attn_n, "avg_launch_us": 1e3 * attn_ms / max(attn_n, 1)},
+            "kernel_time_share": {"gemv": t["kind_ms"][0], "attention": t["kind_ms"][1], "glue": t["kind_ms"][2],
+                                  "unit": "ms of one step, events around every launch"},
+            "e2e": {"value": world * batch / (t["e2e_ms"] / args.steps / 1e3), "unit": "tokens/s",
+                    "h2d_bytes_per_step": t["h2d"], "d2h_bytes_per_step": t["d2h"],
+                    "ms_per_step": t["e2e_ms"] / args.steps},
+            "gpu_launches": t["launches"],
+            "clocks": clocks,
+            "device_status_words": t["status"],
+        }
+        if not args.no_cpu_baseline and world == 1:
+            v, desc, threads, _ = cpu_oracle_sample(batch, ctx0)
+            line["cpu_baseline"] = {"value": v, "unit": "tokens/s", "cores": threads, "kind": "oracle",
+                                    "sample": desc}
+        elif world > 1:
+            line["cpu_baseline"] = None
+        print(json.dumps(line), flush=True)
+    dist_ctx.close()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--batch", type=int, default=32)
+    ap.add_argument("--ctx", type=int, default=2048)
+    ap.add_argument("--layers", type=int, default=0, help="override the layer count (0 = 32)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.impl == "reference":
+        run_reference(args, rank, world)
+    else:
+        run_ours(args, rank, world, local_rank)
+
+
+if __name__ == "__main__":
+    main()

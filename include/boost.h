@@ -385,6 +385,18 @@ int boost_llama_decode_step(const boost_llama_model_t* model /*host*/,
                             int32_t* next_tokens /*device*/, uint32_t* n_launches_out /*host*/,
                             void* stream);
 
+/* Measurement aid: runs one step as boost_llama_decode_step does, with a pair of CUDA
+ * events around every launch, waits for the stream and returns the summed device time and
+ * the number of launches per kind of kernel: [0] weight products (boost_gemv_tiered),
+ * [1] attention, [2] everything else.  kind_ms_out / kind_launches_out: host arrays of 3.
+ * Creates and destroys its events; not for use inside a timed region. */
+int boost_llama_decode_step_profile(const boost_llama_model_t* model /*host*/,
+                                    const boost_llama_scratch_t* scratch /*host*/,
+                                    const int32_t* tokens /*device*/, const int32_t* block_table /*device*/,
+                                    uint32_t max_blocks, const int32_t* ctx_lens /*device*/, uint32_t B,
+                                    int32_t* next_tokens /*device*/, float* kind_ms_out /*host*/,
+                                    uint32_t* kind_launches_out /*host*/, void* stream);
+
 /* As above with HOST buffers (pinned memory recommended): copies tokens, block_table and
  * ctx_lens to the staging buffers of `scratch`, runs the step, copies next_tokens back and
  * waits for the stream, so the result is valid on return. */

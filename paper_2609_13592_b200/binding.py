@@ -116,6 +116,7 @@ SIGNATURES = {
     "boost_swiglu": (_int, [_vp, _u32, _u32, _vp, _vp]),
     "boost_argmax": (_int, [_vp, _u32, _u32, _vp, _vp]),
     "boost_llama_decode_step": (_int, [_vp, _vp, _vp, _vp, _u32, _vp, _u32, _vp, _vp, _vp]),
+    "boost_llama_decode_step_profile": (_int, [_vp, _vp, _vp, _vp, _u32, _vp, _u32, _vp, _vp, _vp, _vp]),
     "boost_llama_decode_step_host": (_int, [_vp, _vp, _vp, _vp, _u32, _vp, _u32, _vp, _vp, _vp]),
 }
 
@@ -405,3 +406,15 @@ def boost_llama_decode_step_host(model, scratch, tokens, block_table, max_blocks
                                               _ptr(next_tokens), C.addressof(n), _stream(stream)),
            "boost_llama_decode_step_host")
     return n.value
+
+
+def boost_llama_decode_step_profile(model, scratch, tokens, block_table, max_blocks, ctx_lens, b, next_tokens,
+                                    stream=None):
+    """-> (ms per kind [gemv, attn, glue], launches per kind)."""
+    ms = (C.c_float * 3)()
+    n = (C.c_uint32 * 3)()
+    _check(lib().boost_llama_decode_step_profile(C.addressof(model), C.addressof(scratch), _ptr(tokens),
+                                                 _ptr(block_table), max_blocks, _ptr(ctx_lens), b,
+                                                 _ptr(next_tokens), C.addressof(ms), C.addressof(n),
+                                                 _stream(stream)), "boost_llama_decode_step_profile")
+    return list(ms), list(n)

@@ -6,13 +6,32 @@
 
 namespace {
 
+enum Kind { kKindGemv = 0, kKindAttn = 1, kKindGlue = 2, kNumKinds = 3 };
+
+// Issues the launches of a step in order; optionally brackets each with a pair of events so
+// that the time of every kind of kernel can be read back afterwards.
 struct Launcher {
   void* stream;
+  bool timed = false;
   uint32_t count = 0;
   int rc = BOOST_OK;
+  cudaEvent_t ev[2 * 512];
+  int kind_of[512];
   bool ok() const { return rc == BOOST_OK; }
-  void run(int r) {
-    if (rc == BOOST_OK) { rc = r; ++count; }
+  template <typename F>
+  void run(int kind, F&& f) {
+    if (rc != BOOST_OK) return;
+    if (timed && count < 512) {
+      rc = boosth::check(cudaEventRecord(ev[2 * count], (cudaStream_t)stream));
+      if (rc != BOOST_OK) return;
+    }
+    rc = f();
+    if (rc != BOOST_OK) return;
+    if (timed && count < 512) {
+      rc = boosth::check(cudaEventRecord(ev[2 * count + 1], (cudaStream_t)stream));
+      kind_of[count] = kind;
+    }
+    ++count;
   }
 };
 
@@ -22,43 +41,81 @@ int gemv(const boost_weight_t& w, const void* x, uint32_t B, void* y, int y_dtyp
                            y_dtype, residual, s->gemv_ws, s->gemv_ws_bytes, stream);
 }
 
+int run_step(Launcher& L, const boost_llama_model_t* m, const boost_llama_scratch_t* s, const int32_t* tokens,
+             const int32_t* block_table, uint32_t max_blocks, const int32_t* ctx_lens, uint32_t B,
+             int32_t* next_tokens) {
+  if (!m || !s || !tokens || !block_table || !ctx_lens || !next_tokens) return BOOST_ERR_INVALID;
+  if (B == 0 || B > 128 || !m->layers || m->n_layers == 0) return BOOST_ERR_INVALID;
+  if (!s->h || !s->xn || !s->qkv || !s->q_rot || !s->attn || !s->gu || !s->act || !s->logits ||
+      !s->gemv_ws || !s->attn_ws)
+    return BOOST_ERR_INVALID;
+  void* stream = L.stream;
+  const uint32_t hq = m->n_q_heads, hkv = m->n_kv_heads, d = m->head_dim;
+  const float scale = 1.0f / sqrtf((float)d);
+  L.run(kKindGlue, [&] { return boost_embed_gather(m->embed, m->vocab, m->hidden, tokens, B, s->h, stream); });
+  for (uint32_t li = 0; li < m->n_layers && L.ok(); ++li) {
+    const boost_llama_layer_t& ly = m->layers[li];
+    L.run(kKindGlue, [&] { return boost_rmsnorm(s->h, ly.norm1, B, m->hidden, m->rms_eps, s->xn, stream); });
+    L.run(kKindGemv, [&] { return gemv(ly.wqkv, s->xn, B, s->qkv, 1, nullptr, s, stream); });
+    L.run(kKindGlue, [&] {
+      return boost_rope_kv_append(s->qkv, s->q_rot, ly.k_page_ptr, ly.v_page_ptr, m->n_pool_blocks, block_table,
+                                  max_blocks, ctx_lens, B, hq, hkv, d, m->rope_base, s->attn_ws, stream);
+    });
+    L.run(kKindAttn, [&] {
+      return boost_paged_attn_decode_tiered(s->q_rot, ly.k_page_ptr, ly.v_page_ptr, m->kv_tier,
+                                            (size_t)m->n_kv_pages, m->n_pool_blocks, block_table, max_blocks,
+                                            ctx_lens, B, hq, hkv, d, scale, s->attn_ws, s->attn_ws_bytes,
+                                            s->attn, stream);
+    });
+    L.run(kKindGemv, [&] { return gemv(ly.wo, s->attn, B, s->h, 1, s->h, s, stream); });     // h += attn Wo^T
+    L.run(kKindGlue, [&] { return boost_rmsnorm(s->h, ly.norm2, B, m->hidden, m->rms_eps, s->xn, stream); });
+    L.run(kKindGemv, [&] { return gemv(ly.wgu, s->xn, B, s->gu, 1, nullptr, s, stream); });
+    L.run(kKindGlue, [&] { return boost_swiglu(s->gu, B, m->ffn, s->act, stream); });
+    L.run(kKindGemv, [&] { return gemv(ly.wd, s->act, B, s->h, 1, s->h, s, stream); });      // h += act Wd^T
+  }
+  L.run(kKindGlue, [&] { return boost_rmsnorm(s->h, m->norm_f, B, m->hidden, m->rms_eps, s->xn, stream); });
+  L.run(kKindGemv, [&] { return gemv(m->lm_head, s->xn, B, s->logits, 0, nullptr, s, stream); });
+  L.run(kKindGlue, [&] { return boost_argmax(s->logits, B, m->vocab, next_tokens, stream); });
+  return L.rc;
+}
+
 }  // namespace
 
 extern "C" int boost_llama_decode_step(const boost_llama_model_t* m, const boost_llama_scratch_t* s,
                                        const int32_t* tokens, const int32_t* block_table,
                                        uint32_t max_blocks, const int32_t* ctx_lens, uint32_t B,
                                        int32_t* next_tokens, uint32_t* n_launches_out, void* stream) {
-  if (!m || !s || !tokens || !block_table || !ctx_lens || !next_tokens) return BOOST_ERR_INVALID;
-  if (B == 0 || B > 128 || !m->layers || m->n_layers == 0) return BOOST_ERR_INVALID;
-  if (!s->h || !s->xn || !s->qkv || !s->q_rot || !s->attn || !s->gu || !s->act || !s->logits ||
-      !s->gemv_ws || !s->attn_ws)
-    return BOOST_ERR_INVALID;
-  const uint32_t hq = m->n_q_heads, hkv = m->n_kv_heads, d = m->head_dim;
-  if (m->hidden != hq * d && m->hidden == 0) return BOOST_ERR_INVALID;
-  const float scale = 1.0f / sqrtf((float)d);
-  Launcher L{stream};
-  L.run(boost_embed_gather(m->embed, m->vocab, m->hidden, tokens, B, s->h, stream));
-  for (uint32_t li = 0; li < m->n_layers && L.ok(); ++li) {
-    const boost_llama_layer_t& ly = m->layers[li];
-    L.run(boost_rmsnorm(s->h, ly.norm1, B, m->hidden, m->rms_eps, s->xn, stream));
-    L.run(gemv(ly.wqkv, s->xn, B, s->qkv, 1, nullptr, s, stream));
-    L.run(boost_rope_kv_append(s->qkv, s->q_rot, ly.k_page_ptr, ly.v_page_ptr, m->n_pool_blocks, block_table,
-                               max_blocks, ctx_lens, B, hq, hkv, d, m->rope_base, s->attn_ws, stream));
-    L.run(boost_paged_attn_decode_tiered(s->q_rot, ly.k_page_ptr, ly.v_page_ptr, m->kv_tier,
-                                         (size_t)m->n_kv_pages, m->n_pool_blocks, block_table, max_blocks,
-                                         ctx_lens, B, hq, hkv, d, scale, s->attn_ws, s->attn_ws_bytes,
-                                         s->attn, stream));
-    L.run(gemv(ly.wo, s->attn, B, s->h, 1, s->h, s, stream));       // h += attn Wo^T
-    L.run(boost_rmsnorm(s->h, ly.norm2, B, m->hidden, m->rms_eps, s->xn, stream));
-    L.run(gemv(ly.wgu, s->xn, B, s->gu, 1, nullptr, s, stream));
-    L.run(boost_swiglu(s->gu, B, m->ffn, s->act, stream));
-    L.run(gemv(ly.wd, s->act, B, s->h, 1, s->h, s, stream));        // h += act Wd^T
-  }
-  L.run(boost_rmsnorm(s->h, m->norm_f, B, m->hidden, m->rms_eps, s->xn, stream));
-  L.run(gemv(m->lm_head, s->xn, B, s->logits, 0, nullptr, s, stream));
-  L.run(boost_argmax(s->logits, B, m->vocab, next_tokens, stream));
+  static thread_local Launcher L;
+  L.stream = stream; L.timed = false; L.count = 0; L.rc = BOOST_OK;
+  const int rc = run_step(L, m, s, tokens, block_table, max_blocks, ctx_lens, B, next_tokens);
   if (n_launches_out) *n_launches_out = L.count;
-  return L.rc;
+  return rc;
+}
+
+extern "C" int boost_llama_decode_step_profile(const boost_llama_model_t* m, const boost_llama_scratch_t* s,
+                                               const int32_t* tokens, const int32_t* block_table,
+                                               uint32_t max_blocks, const int32_t* ctx_lens, uint32_t B,
+                                               int32_t* next_tokens, float* kind_ms_out,
+                                               uint32_t* kind_launches_out, void* stream) {
+  if (!kind_ms_out || !kind_launches_out || !m) return BOOST_ERR_INVALID;
+  if (1 + 9 * (uint64_t)m->n_layers + 3 > 512) return BOOST_ERR_UNSUPPORTED;
+  static thread_local Launcher L;
+  L.stream = stream; L.timed = true; L.count = 0; L.rc = BOOST_OK;
+  const uint32_t n_events = 2 * (1 + 9 * m->n_layers + 3);
+  uint32_t made = 0;
+  int rc = BOOST_OK;
+  for (; made < n_events && rc == BOOST_OK; ++made) rc = boosth::check(cudaEventCreate(&L.ev[made]));
+  if (rc == BOOST_OK) rc = run_step(L, m, s, tokens, block_table, max_blocks, ctx_lens, B, next_tokens);
+  if (rc == BOOST_OK) rc = boosth::check(cudaStreamSynchronize((cudaStream_t)stream));
+  for (int k = 0; k < kNumKinds; ++k) { kind_ms_out[k] = 0.f; kind_launches_out[k] = 0; }
+  for (uint32_t i = 0; i < L.count && rc == BOOST_OK; ++i) {
+    float ms = 0.f;
+    rc = boosth::check(cudaEventElapsedTime(&ms, L.ev[2 * i], L.ev[2 * i + 1]));
+    kind_ms_out[L.kind_of[i]] += ms;
+    kind_launches_out[L.kind_of[i]] += 1;
+  }
+  for (uint32_t i = 0; i < made; ++i) cudaEventDestroy(L.ev[i]);
+  return rc;
 }
 
 extern "C" int boost_llama_decode_step_host(const boost_llama_model_t* m, const boost_llama_scratch_t* s,
