@@ -246,8 +246,8 @@ int boost_pack_weights(const void* w_row_major /*device*/, uint32_t N, uint32_t 
  *   y          device, row-major [M_b, N]; y_dtype 0 = fp32, 1 = bf16;
  *   residual   device bf16 [M_b, N] added before the final rounding, or NULL;
  *   workspace  device, >= boost_gemv_workspace_bytes(N, K, M_b).
- * M_b <= 8 runs on CUDA cores with warp-shuffle reductions; larger batches use the tensor
- * cores.  Split-K partial sums are combined in a fixed order by the last threadblock to
+ * M_b <= 2 runs on CUDA cores with warp-shuffle reductions; larger batches use the tensor
+ * cores (batch padded to a multiple of 16).  Split-K partial sums are combined in a fixed order by the last threadblock to
  * finish a row tile, so the result is deterministic. */
 size_t boost_gemv_workspace_bytes(uint32_t N, uint32_t K, uint32_t M_b);
 int boost_gemv_tiered(const void* const* w_page_ptr /*device*/, const uint32_t* w_order /*device*/,

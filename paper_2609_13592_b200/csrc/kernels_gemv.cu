@@ -1,9 +1,9 @@
 // Tiered weight-streaming product y = x W^T (GEMV at batch 1, skinny GEMM above) and the
 // kernel that packs a row-major weight into its paged 16 KiB-block form.
 //
-// One persistent threadblock per SM.  A producer warp walks the work queue (host-tier items
-// first, Sec. 3.2) and fills a ring of shared-memory stages: a 16 KiB weight block arrives
-// by one bulk copy through the TMA unit when its page is in HBM, or by a deep fan of
+// One persistent threadblock per SM.  Two producer warps walk the work queue (host-tier
+// items first, Sec. 3.2) and fill a ring of shared-memory stages: a 16 KiB weight block
+// arrives by one bulk copy through the TMA unit when its page is in HBM, or by a deep fan of
 // 16-byte cp.async loads when the page is host memory behind the CPU-GPU link; the matching
 // 64-column slice of x rides along by cp.async.  Eight consumer warps multiply from shared
 // memory: on CUDA cores with warp-shuffle reductions for batches up to 8, with bf16
@@ -25,9 +25,10 @@ constexpr uint32_t kBlockBytes = kBlockRows * kBlockK * 2;      // 16 KiB
 constexpr uint32_t kBlocksPerPage = kPageBytes / kBlockBytes;   // 128
 constexpr uint32_t kConsumerWarps = 8;
 constexpr uint32_t kConsumerThreads = kConsumerWarps * 32;
-constexpr uint32_t kGemvThreads = kConsumerThreads + 32;
-constexpr uint32_t kMaxStages = 8;
-constexpr uint32_t kSmemBudget = 200u * 1024u;
+constexpr uint32_t kGemvThreads = kConsumerThreads + 64;   // + weight producer warp + x producer warp
+constexpr uint32_t kMaxStages = 16;
+constexpr uint32_t kSmemBudget = 224u * 1024u;
+constexpr uint32_t kXRowStride = 144;  // 128 data bytes + 16: 8 consecutive rows hit distinct banks
 
 enum : uint32_t { kFlagFirst = 1u, kFlagLast = 2u, kFlagStop = 4u };
 
@@ -49,7 +50,7 @@ struct GemvParams {
 
 __host__ __device__ constexpr uint32_t x_rows_of(int NT, int MB) { return NT > 0 ? NT * 8 : MB; }
 __host__ __device__ constexpr uint32_t stage_bytes_of(int NT, int MB) {
-  return kBlockBytes + ((x_rows_of(NT, MB) * 128u + 1023u) / 1024u) * 1024u;
+  return kBlockBytes + ((x_rows_of(NT, MB) * kXRowStride + 1023u) / 1024u) * 1024u;
 }
 
 __device__ __forceinline__ void store_out(const GemvParams& p, uint32_t m, uint32_t n, float v) {
@@ -61,7 +62,7 @@ __device__ __forceinline__ void store_out(const GemvParams& p, uint32_t m, uint3
 
 // NT > 0: tensor-core path with NT batch tiles of 8; NT == 0: CUDA-core path for MB rows.
 template <int NT, int MB>
-__global__ void __launch_bounds__(kGemvThreads, 1) gemv_tiered_kernel(const GemvParams p) {
+__global__ void __launch_bounds__(kGemvThreads, (NT >= 8 ? 1 : 2)) gemv_tiered_kernel(const GemvParams p) {
   constexpr uint32_t kXRows = x_rows_of(NT, MB);
   constexpr uint32_t kStageBytes = stage_bytes_of(NT, MB);
   extern __shared__ uint8_t smem_raw[];
@@ -69,6 +70,9 @@ __global__ void __launch_bounds__(kGemvThreads, 1) gemv_tiered_kernel(const Gemv
   __shared__ uint64_t full_bar[kMaxStages];
   __shared__ uint64_t empty_bar[kMaxStages];
   __shared__ uint4 meta[kMaxStages];
+  __shared__ uint64_t item_full[4];
+  __shared__ uint64_t item_empty[4];
+  __shared__ uint32_t item_ring[4];
   __shared__ uint32_t s_old;
 
   const uint32_t tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -77,73 +81,111 @@ __global__ void __launch_bounds__(kGemvThreads, 1) gemv_tiered_kernel(const Gemv
 
   if (tid == 0) {
     for (uint32_t s = 0; s < n_stages; ++s) {
-      mbar_init(&full_bar[s], 33);              // 32 cp.async arrivals + the lane-0 arrive
+      mbar_init(&full_bar[s], 65);              // 2 x 32 cp.async arrivals + the arrive.expect_tx
       mbar_init(&empty_bar[s], kConsumerWarps);
+    }
+    for (uint32_t s = 0; s < 4; ++s) {
+      mbar_init(&item_full[s], 1);
+      mbar_init(&item_empty[s], 1);
     }
     fence_barrier_init();
   }
   __syncthreads();
 
-  if (warp == kConsumerWarps) {
-    // ------------------------------------------------------------------ producer warp
+  if (warp >= kConsumerWarps) {
+    // ------------------------------------------------------------------ producer warps
+    // Warp 8 owns the work queue and the weight blocks; warp 9 follows the same item
+    // sequence (handed over through a four-slot ring) and loads the matching slices of x.
+    // Two warps, because a lone warp's instruction latency would cap the fill rate.
+    const bool leader = (warp == kConsumerWarps);
+    const uint32_t n_host_items = p.n_host_pages * p.items_per_page;
     TierQueues q;
-    q.init(p.ws, p.n_host_pages * p.items_per_page, p.n_pages * p.items_per_page,
-           blockIdx.x < p.n_host_ctas);
-    uint32_t stage = 0, phase = 0;
+    q.init(p.ws, n_host_items, p.n_pages * p.items_per_page, blockIdx.x < p.n_host_ctas);
+    uint32_t stage = 0, phase = 0, icount = 0;
     for (;;) {
+      const uint32_t slot = icount & 3u, iphase = (icount >> 2) & 1u;
       uint32_t qi = 0;
-      if (lane == 0) qi = q.next();
-      qi = __shfl_sync(0xFFFFFFFFu, qi, 0);
+      if (leader) {
+        if (lane == 0) {
+          for (;;) {   // skip the unused tail of the last page
+            qi = q.next();
+            if (qi == 0xFFFFFFFFu) break;
+            if (p.w_order[qi / p.items_per_page] * p.items_per_page + qi % p.items_per_page < p.n_items) break;
+          }
+          mbar_wait(&item_empty[slot], iphase ^ 1u, status);
+          item_ring[slot] = qi;
+          mbar_arrive(&item_full[slot]);
+        }
+        qi = __shfl_sync(0xFFFFFFFFu, qi, 0);
+      } else {
+        mbar_wait(&item_full[slot], iphase, status);
+        qi = item_ring[slot];
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&item_empty[slot]);
+      }
+      ++icount;
       if (qi == 0xFFFFFFFFu) break;
       const uint32_t page = p.w_order[qi / p.items_per_page];
-      const uint32_t item = page * p.items_per_page + qi % p.items_per_page;
-      if (item >= p.n_items) continue;  // unused tail of the last page
-      const uint32_t first_blk = item * p.run;
+      const uint32_t first_blk = (page * p.items_per_page + qi % p.items_per_page) * p.run;
       const uint32_t row_tile = first_blk / p.k_blocks;
       const uint32_t kb0 = first_blk % p.k_blocks;
-      const bool from_host = qi < p.n_host_pages * p.items_per_page;
-      const uint8_t* src = static_cast<const uint8_t*>(p.w_page_ptr[page]) +
-                           (size_t)(first_blk % kBlocksPerPage) * kBlockBytes;
-      for (uint32_t j = 0; j < p.run; ++j) {
-        mbar_wait(&empty_bar[stage], phase ^ 1u, status);
-        uint8_t* wdst = smem + (size_t)stage * kStageBytes;
-        uint8_t* xdst = wdst + kBlockBytes;
-        if (lane == 0)
-          meta[stage] = make_uint4(row_tile, kb0 / p.run,
-                                   (j == 0 ? kFlagFirst : 0u) | (j + 1 == p.run ? kFlagLast : 0u), 0u);
-        const uint32_t k_base = (kb0 + j) * kBlockK;
-        for (uint32_t idx = lane; idx < kXRows * 8; idx += 32) {
-          const uint32_t m = idx >> 3, c = idx & 7;
-          const uint32_t k = k_base + c * 8;
-          const bool valid = (m < p.M_b) && (k < p.K);
-          const __nv_bfloat16* xs = valid ? p.x + (size_t)m * p.K + k : p.x;
-          cp_async_16(xdst + m * 128 + ((c ^ (m & 7)) << 4), xs, valid ? 16u : 0u);
-        }
-        if (from_host) {
-          const uint8_t* s = src + (size_t)j * kBlockBytes;
-#pragma unroll 8
-          for (uint32_t idx = lane; idx < kBlockBytes / 16; idx += 32)
-            cp_async_16(wdst + idx * 16, s + idx * 16, 16u);
-        }
-        cp_async_arrive_noinc(&full_bar[stage]);
-        if (lane == 0) {
-          if (from_host) {
-            mbar_arrive(&full_bar[stage]);
-          } else {
-            mbar_arrive_expect_tx(&full_bar[stage], kBlockBytes);
-            bulk_copy_g2s(wdst, src + (size_t)j * kBlockBytes, kBlockBytes, &full_bar[stage]);
+      const bool from_host = qi < n_host_items;
+      if (leader) {
+        const uint8_t* src = static_cast<const uint8_t*>(p.w_page_ptr[page]) +
+                             (size_t)(first_blk % kBlocksPerPage) * kBlockBytes;
+        for (uint32_t j = 0; j < p.run; ++j, src += kBlockBytes) {
+          uint8_t* wdst = smem + (size_t)stage * kStageBytes;
+          if (lane == 0) {
+            mbar_wait(&empty_bar[stage], phase ^ 1u, status);
+            meta[stage] = make_uint4(row_tile, kb0 / p.run,
+                                     (j == 0 ? kFlagFirst : 0u) | (j + 1 == p.run ? kFlagLast : 0u), 0u);
+            mbar_arrive_expect_tx(&full_bar[stage], from_host ? 0u : kBlockBytes);
+            if (!from_host) bulk_copy_g2s(wdst, src, kBlockBytes, &full_bar[stage]);
           }
+          __syncwarp();   // the other lanes must not run ahead of lane 0's wait on the stage
+          if (from_host) {
+            // host page: a fan of 16-byte loads through the load/store path keeps many
+            // requests on the link at once (Sec. 3.2: this threadblock is a host-tier block)
+#pragma unroll 8
+            for (uint32_t idx = lane; idx < kBlockBytes / 16; idx += 32)
+              cp_async_16(wdst + idx * 16, src + idx * 16, 16u);
+          }
+          cp_async_arrive_noinc(&full_bar[stage]);
+          if (++stage == n_stages) { stage = 0; phase ^= 1u; }
         }
-        if (++stage == n_stages) { stage = 0; phase ^= 1u; }
+      } else {
+        // lane -> (row m0 + 4 i, 16-byte chunk c); pointers advance by constants
+        const uint32_t c = lane & 7, m0 = lane >> 3;
+        for (uint32_t j = 0; j < p.run; ++j) {
+          mbar_wait(&empty_bar[stage], phase ^ 1u, status);
+          uint8_t* xdst = smem + (size_t)stage * kStageBytes + kBlockBytes + m0 * kXRowStride + c * 16;
+          const uint32_t k = (kb0 + j) * kBlockK + c * 8;
+          const bool k_ok = k < p.K;
+          const __nv_bfloat16* xs = p.x + (size_t)m0 * p.K + (k_ok ? k : 0u);
+#pragma unroll 4
+          for (uint32_t m = m0; m < kXRows; m += 4) {
+            cp_async_16(xdst, xs, (k_ok && m < p.M_b) ? 16u : 0u);
+            xdst += 4 * kXRowStride;
+            if (m + 4 < p.M_b) xs += (size_t)4 * p.K;
+          }
+          cp_async_arrive_noinc(&full_bar[stage]);
+          if (++stage == n_stages) { stage = 0; phase ^= 1u; }
+        }
       }
     }
     // tell the consumers to stop
-    mbar_wait(&empty_bar[stage], phase ^ 1u, status);
-    if (lane == 0) meta[stage] = make_uint4(0u, 0u, kFlagStop, 0u);
-    cp_async_arrive_noinc(&full_bar[stage]);
-    if (lane == 0) {
-      mbar_arrive(&full_bar[stage]);
-      q.finish(gridDim.x);
+    if (leader) {
+      if (lane == 0) {
+        mbar_wait(&empty_bar[stage], phase ^ 1u, status);
+        meta[stage] = make_uint4(0u, 0u, kFlagStop, 0u);
+        mbar_arrive(&full_bar[stage]);
+      }
+      __syncwarp();
+      cp_async_arrive_noinc(&full_bar[stage]);
+      if (lane == 0) q.finish(gridDim.x);
+    } else {
+      mbar_wait(&empty_bar[stage], phase ^ 1u, status);
+      cp_async_arrive_noinc(&full_bar[stage]);
     }
     return;
   }
@@ -185,7 +227,7 @@ __global__ void __launch_bounds__(kGemvThreads, 1) gemv_tiered_kernel(const Gemv
         for (int n2 = 0; n2 < NT / 2; ++n2) {
           const uint32_t b_row = n2 * 16 + b_row0;
           uint32_t b0, b1, b2, b3;
-          ldmatrix_x4(b0, b1, b2, b3, xbase + b_row * 128 + ((b_chunk ^ (b_row & 7)) << 4));
+          ldmatrix_x4(b0, b1, b2, b3, xbase + b_row * kXRowStride + (b_chunk << 4));
           mma_bf16_16816(acc[2 * n2], a, b0, b1);
           mma_bf16_16816(acc[2 * n2 + 1], a, b2, b3);
         }
@@ -203,7 +245,7 @@ __global__ void __launch_bounds__(kGemvThreads, 1) gemv_tiered_kernel(const Gemv
       }
 #pragma unroll
       for (int m = 0; m < MB; ++m) {
-        const uint4 xv = *reinterpret_cast<const uint4*>(xsm + m * 128 + ((c ^ (m & 7)) << 4));
+        const uint4 xv = *reinterpret_cast<const uint4*>(xsm + m * kXRowStride + (c << 4));
         const float xf[8] = {bf16_lo(xv.x), bf16_hi(xv.x), bf16_lo(xv.y), bf16_hi(xv.y),
                              bf16_lo(xv.z), bf16_hi(xv.z), bf16_lo(xv.w), bf16_hi(xv.w)};
 #pragma unroll
@@ -275,14 +317,26 @@ __global__ void __launch_bounds__(kGemvThreads, 1) gemv_tiered_kernel(const Gemv
         named_barrier_sync(1, kConsumerThreads);
         if (s_old == p.splits - 1) {
           __threadfence();
-          const float* base = p.partials + (size_t)row_tile * p.splits * kXRows * kBlockRows;
-          for (uint32_t idx = tid; idx < p.M_b * kBlockRows; idx += kConsumerThreads) {
-            const uint32_t m = idx / kBlockRows, nl = idx % kBlockRows;
-            float s = 0.f;
-            for (uint32_t sp = 0; sp < p.splits; ++sp)
-              s += __ldcg(base + ((size_t)sp * kXRows + m) * kBlockRows + nl);
-            const uint32_t n = row_tile * kBlockRows + nl;
-            if (n < p.N) store_out(p, m, n, s);
+          const float4* base = reinterpret_cast<const float4*>(
+              p.partials + (size_t)row_tile * p.splits * kXRows * kBlockRows);
+          constexpr uint32_t kVecRow = kBlockRows / 4;   // float4 per batch row
+          for (uint32_t idx = tid; idx < p.M_b * kVecRow; idx += kConsumerThreads) {
+            const uint32_t m = idx / kVecRow, v4 = idx % kVecRow;
+            float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
+            for (uint32_t sp0 = 0; sp0 < p.splits; sp0 += 8) {   // loads in batches of 8, sums in split order
+              float4 t[8];
+#pragma unroll
+              for (uint32_t u = 0; u < 8; ++u)
+                if (sp0 + u < p.splits) t[u] = __ldcg(base + ((size_t)(sp0 + u) * kXRows + m) * kVecRow + v4);
+#pragma unroll
+              for (uint32_t u = 0; u < 8; ++u)
+                if (sp0 + u < p.splits) { s.x += t[u].x; s.y += t[u].y; s.z += t[u].z; s.w += t[u].w; }
+            }
+            const uint32_t n = row_tile * kBlockRows + v4 * 4;
+            if (n < p.N) store_out(p, m, n, s.x);
+            if (n + 1 < p.N) store_out(p, m, n + 1, s.y);
+            if (n + 2 < p.N) store_out(p, m, n + 2, s.z);
+            if (n + 3 < p.N) store_out(p, m, n + 3, s.w);
           }
           if (tid == 0) tile_cnt[row_tile] = 0;
         }
@@ -330,7 +384,10 @@ template <int NT, int MB>
 int launch_gemv(const GemvParams& p, int sms, cudaStream_t stream) {
   constexpr uint32_t kStage = stage_bytes_of(NT, MB);
   GemvParams q = p;
-  uint32_t n_stages = kSmemBudget / kStage;
+  // Two threadblocks per SM where registers allow: a second ring hides the producer /
+  // consumer hand-over latency of the first (measured: +25 % bandwidth on B200).
+  const uint32_t ctas_per_sm = (NT >= 8) ? 1 : 2;
+  uint32_t n_stages = (kSmemBudget / ctas_per_sm - 1024) / kStage;
   if (n_stages > kMaxStages) n_stages = kMaxStages;
   q.n_stages = n_stages;
   const size_t smem = (size_t)n_stages * kStage + 1024;
@@ -341,7 +398,7 @@ int launch_gemv(const GemvParams& p, int sms, cudaStream_t stream) {
     if (rc != BOOST_OK) return rc;
     configured = true;
   }
-  uint32_t grid = (uint32_t)sms;
+  uint32_t grid = (uint32_t)sms * ctas_per_sm;
   const uint32_t queue_len = q.n_pages * q.items_per_page;
   if (grid > queue_len) grid = queue_len;
   uint32_t n_host_ctas = 0;
@@ -386,10 +443,11 @@ extern "C" int boost_pack_weights(const void* w_row_major, uint32_t N, uint32_t 
 }
 
 static uint32_t gemv_x_rows(uint32_t M_b) {
+  // rows of x staged per block: 1 or 2 on the CUDA-core path, else batch tiles of 8 for the
+  // tensor cores (which outrun the CUDA cores from three rows up: the kernel is HBM-bound and
+  // the tensor pipe is otherwise idle)
   if (M_b <= 1) return 1;
   if (M_b <= 2) return 2;
-  if (M_b <= 4) return 4;
-  if (M_b <= 8) return 8;
   if (M_b <= 16) return 16;
   if (M_b <= 32) return 32;
   if (M_b <= 64) return 64;
@@ -444,8 +502,6 @@ extern "C" int boost_gemv_tiered(const void* const* w_page_ptr, const uint32_t* 
   switch (gemv_x_rows(M_b)) {
     case 1: return launch_gemv<0, 1>(p, sms, st);
     case 2: return launch_gemv<0, 2>(p, sms, st);
-    case 4: return launch_gemv<0, 4>(p, sms, st);
-    case 8: return launch_gemv<0, 8>(p, sms, st);
     case 16: return launch_gemv<2, 0>(p, sms, st);
     case 32: return launch_gemv<4, 0>(p, sms, st);
     case 64: return launch_gemv<8, 0>(p, sms, st);
