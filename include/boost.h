@@ -215,6 +215,28 @@ int boost_stream_reduce_tiered(const void* const* page_ptr /*device*/,
                                size_t n_host_pages, float* per_page_sum /*device*/,
                                void* workspace /*device*/, size_t workspace_bytes, void* stream);
 
+/* boost_stream_reduce_tiered for callers that cannot allocate.  (The paper has no
+ * counterpart: this entry point exists for integration, not for the method.)
+ * Who needs it: an engine that gave all device memory to its own pools at start-up, so a
+ * later cudaMalloc fails; a plug-in that must stay inside a host framework's allocator; any
+ * caller on a path where allocating CUDA calls are not allowed.  The scratch that the
+ * kernel needs lives in a fixed array inside the library (about 272 KiB, held by every GPU
+ * that loads the library until the process exits), so the call allocates nothing - no
+ * cudaMalloc, cudaFree or allocating library routine - and takes no workspace argument.
+ *   - n_pages may be at most boost_stream_reduce_static_max_pages() (4096 pages, 8 GiB);
+ *     larger buffers return BOOST_ERR_CAPACITY and must use boost_stream_reduce_tiered.
+ *   - The first call on each device looks up the array's device address (with that device
+ *     current); make that first call outside any stream capture.
+ *   - All calls on a device share the one array: the call clears the counters it needs on
+ *     `stream` before the kernel, but two calls that overlap on the GPU (different streams,
+ *     or a graph replayed concurrently) race on it and give wrong sums.
+ * Inputs, outputs and results are those of boost_stream_reduce_tiered. */
+size_t boost_stream_reduce_static_max_pages(void);
+int boost_stream_reduce_tiered_static(const void* const* page_ptr /*device*/,
+                                      const uint32_t* order /*device*/, size_t n_pages,
+                                      size_t n_host_pages, float* per_page_sum /*device*/,
+                                      void* stream);
+
 /* Weight tensors are stored in pages as a stream of 16 KiB blocks.  Block (t, kb) holds
  * rows [128 t, 128 t + 128) and columns [64 kb, 64 kb + 64) of the row-major [N, K] bf16
  * matrix W (zero padded), at byte offset (t * ceil(K/64) + kb) * 16 KiB of the tensor; row

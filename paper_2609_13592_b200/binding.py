@@ -100,6 +100,8 @@ SIGNATURES = {
     "boost_kv_pool_destroy": (_int, [_vp]),
     "boost_stream_reduce_workspace_bytes": (_sz, [_sz]),
     "boost_stream_reduce_tiered": (_int, [_vp, _vp, _sz, _sz, _vp, _vp, _sz, _vp]),
+    "boost_stream_reduce_static_max_pages": (_sz, []),
+    "boost_stream_reduce_tiered_static": (_int, [_vp, _vp, _sz, _sz, _vp, _vp]),
     "boost_weight_layout": (_int, [_u32, _u32, _vp]),
     "boost_pack_weights": (_int, [_vp, _u32, _u32, _vp, _sz, _vp]),
     "boost_gemv_workspace_bytes": (_sz, [_u32, _u32, _u32]),
@@ -310,6 +312,18 @@ def boost_stream_reduce_tiered(page_ptr, order, n_pages, n_host_pages, per_page_
     _check(lib().boost_stream_reduce_tiered(_ptr(page_ptr), _ptr(order), n_pages, n_host_pages,
                                             _ptr(per_page_sum), _ptr(workspace), workspace_bytes,
                                             _stream(stream)), "boost_stream_reduce_tiered")
+
+
+def boost_stream_reduce_static_max_pages():
+    return lib().boost_stream_reduce_static_max_pages()
+
+
+def boost_stream_reduce_tiered_static(page_ptr, order, n_pages, n_host_pages, per_page_sum, stream=None):
+    """Stream reduce with the library's built-in scratch: for callers that cannot allocate a
+    workspace (see include/boost.h).  At most boost_stream_reduce_static_max_pages() pages."""
+    _check(lib().boost_stream_reduce_tiered_static(_ptr(page_ptr), _ptr(order), n_pages, n_host_pages,
+                                                   _ptr(per_page_sum), _stream(stream)),
+           "boost_stream_reduce_tiered_static")
 
 
 def boost_weight_layout(n, k):

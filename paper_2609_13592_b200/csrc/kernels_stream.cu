@@ -3,6 +3,8 @@
 // tensor is materialised into its tiers.
 #include <cuda_runtime.h>
 
+#include <mutex>
+
 #include "device_common.cuh"
 #include "host_common.h"
 
@@ -177,4 +179,67 @@ extern "C" int boost_stream_reduce_tiered(const void* const* page_ptr, const uin
       page_ptr, order, (uint32_t)n_pages, (uint32_t)n_host_pages, per_page_sum,
       static_cast<uint32_t*>(workspace), n_host_ctas);
   return boosth::check_launch();
+}
+
+// ---------------------------------------------------------------------------------------
+// Stream reduce for callers that may not allocate.
+//
+// Some users of this library cannot obtain scratch memory at call time: a serving engine
+// that has handed all of the GPU's memory to its own pools at start-up (a later cudaMalloc
+// simply fails), a plug-in that runs under a host framework's allocator and is forbidden
+// to go around it, or code on a path where the allocating CUDA calls are not permitted.
+// For them the scratch of the stream-reduce kernel lives in a fixed array inside the
+// library image.  Every GPU that loads the library carries these kStaticScratchBytes
+// until the process exits, which is why the limit is modest.
+constexpr size_t kStaticMaxPages = 4096;   // buffers of up to 8 GiB
+constexpr size_t kStaticScratchBytes =
+    (size_t)boostk::kWsHeaderWords * 4 + kStaticMaxPages * 4 + kStaticMaxPages * kTilesPerPage * 4;
+
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+
+namespace {
+
+// In host code `g_static_scratch` is only a handle for the runtime, not an address a kernel
+// can use; the device address is looked up once per device, with that device current.
+void* g_static_scratch_dev[64] = {nullptr};
+std::mutex g_static_scratch_mutex;
+
+int static_scratch_address(void** out) {
+  int dev = 0;
+  int rc = boosth::check(cudaGetDevice(&dev));
+  if (rc != BOOST_OK) return rc;
+  if (dev < 0 || dev >= 64) return BOOST_ERR_UNSUPPORTED;
+  std::lock_guard<std::mutex> lock(g_static_scratch_mutex);
+  if (g_static_scratch_dev[dev] == nullptr) {
+    void* p = nullptr;
+    rc = boosth::check(cudaGetSymbolAddress(&p, g_static_scratch));
+    if (rc != BOOST_OK) return rc;
+    if (p == nullptr) return BOOST_ERR_CUDA;
+    g_static_scratch_dev[dev] = p;
+  }
+  *out = g_static_scratch_dev[dev];
+  return BOOST_OK;
+}
+
+}  // namespace
+
+extern "C" size_t boost_stream_reduce_static_max_pages(void) { return kStaticMaxPages; }
+
+extern "C" int boost_stream_reduce_tiered_static(const void* const* page_ptr, const uint32_t* order,
+                                                 size_t n_pages, size_t n_host_pages,
+                                                 float* per_page_sum, void* stream) {
+  if (n_pages == 0) return BOOST_OK;
+  if (!page_ptr || !order || !per_page_sum) return BOOST_ERR_INVALID;
+  if (n_host_pages > n_pages) return BOOST_ERR_INVALID;
+  if (n_pages > kStaticMaxPages) return BOOST_ERR_CAPACITY;   // larger buffers need the caller's own workspace
+  void* scratch = nullptr;
+  int rc = static_scratch_address(&scratch);
+  if (rc != BOOST_OK) return rc;
+  // The array keeps whatever the previous call left.  The queue words and the per-page
+  // counters must start at zero; the per-tile partial sums are overwritten before use.
+  const size_t counters = (size_t)boostk::kWsHeaderWords * 4 + n_pages * 4;
+  rc = boosth::check(cudaMemsetAsync(scratch, 0, counters, (cudaStream_t)stream));
+  if (rc != BOOST_OK) return rc;
+  return boost_stream_reduce_tiered(page_ptr, order, n_pages, n_host_pages, per_page_sum, scratch,
+                                    kStaticScratchBytes, stream);
 }
