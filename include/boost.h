@@ -380,7 +380,7 @@ typedef struct {
 /* Device scratch of a decode step for up to B_max sequences (all bf16 unless noted):
  * h, xn [B, hidden]; qkv [B, (Hq+2Hkv) D]; q_rot, attn [B, Hq D]; gu [B, 2F]; act [B, F];
  * logits fp32 [B, vocab]; gemv_ws >= the largest boost_gemv_workspace_bytes over the model's
- * weights; attn_ws >= boost_paged_attn_workspace_bytes; both zero-filled once and 256-byte
+ * weights plus 33024 bytes (one set of queue words per launch of a step); attn_ws >= boost_paged_attn_workspace_bytes; both zero-filled once and 256-byte
  * aligned; tokens_dev / ctx_dev / next_dev int32 [B] and table_dev int32 [B, max_blocks] are
  * staging buffers used by boost_llama_decode_step_host only. */
 typedef struct {

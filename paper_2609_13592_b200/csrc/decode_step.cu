@@ -35,10 +35,20 @@ struct Launcher {
   }
 };
 
+// The tail of the GEMV workspace holds one set of queue words per launch of a step, so that a
+// weight product can take work and stream weights while the kernel before it is still running.
+constexpr size_t kQueueSlots = 512;
+constexpr size_t kQueueSlotBytes = 64;
+constexpr size_t kQueueRegionBytes = kQueueSlots * kQueueSlotBytes;
+
 int gemv(const boost_weight_t& w, const void* x, uint32_t B, void* y, int y_dtype, const void* residual,
-         const boost_llama_scratch_t* s, void* stream) {
-  return boost_gemv_tiered(w.page_ptr, w.order, (size_t)w.n_pages, (size_t)w.n_host_pages, w.N, w.K, x, B, y,
-                           y_dtype, residual, s->gemv_ws, s->gemv_ws_bytes, stream);
+         const boost_llama_scratch_t* s, uint32_t launch_index, void* stream) {
+  if (s->gemv_ws_bytes <= kQueueRegionBytes + 256) return BOOST_ERR_CAPACITY;
+  const size_t usable = (s->gemv_ws_bytes - kQueueRegionBytes) & ~(size_t)255;
+  uint8_t* slots = static_cast<uint8_t*>(s->gemv_ws) + usable;
+  uint32_t* queue = reinterpret_cast<uint32_t*>(slots + (launch_index % kQueueSlots) * kQueueSlotBytes);
+  return boosth::gemv_tiered_launch(w.page_ptr, w.order, (size_t)w.n_pages, (size_t)w.n_host_pages, w.N, w.K, x,
+                                    B, y, y_dtype, residual, s->gemv_ws, usable, queue, stream);
 }
 
 int run_step(Launcher& L, const boost_llama_model_t* m, const boost_llama_scratch_t* s, const int32_t* tokens,
@@ -56,7 +66,7 @@ int run_step(Launcher& L, const boost_llama_model_t* m, const boost_llama_scratc
   for (uint32_t li = 0; li < m->n_layers && L.ok(); ++li) {
     const boost_llama_layer_t& ly = m->layers[li];
     L.run(kKindGlue, [&] { return boost_rmsnorm(s->h, ly.norm1, B, m->hidden, m->rms_eps, s->xn, stream); });
-    L.run(kKindGemv, [&] { return gemv(ly.wqkv, s->xn, B, s->qkv, 1, nullptr, s, stream); });
+    L.run(kKindGemv, [&] { return gemv(ly.wqkv, s->xn, B, s->qkv, 1, nullptr, s, L.count, stream); });
     L.run(kKindGlue, [&] {
       return boost_rope_kv_append(s->qkv, s->q_rot, ly.k_page_ptr, ly.v_page_ptr, m->n_pool_blocks, block_table,
                                   max_blocks, ctx_lens, B, hq, hkv, d, m->rope_base, s->attn_ws, stream);
@@ -67,14 +77,14 @@ int run_step(Launcher& L, const boost_llama_model_t* m, const boost_llama_scratc
                                             ctx_lens, B, hq, hkv, d, scale, s->attn_ws, s->attn_ws_bytes,
                                             s->attn, stream);
     });
-    L.run(kKindGemv, [&] { return gemv(ly.wo, s->attn, B, s->h, 1, s->h, s, stream); });     // h += attn Wo^T
+    L.run(kKindGemv, [&] { return gemv(ly.wo, s->attn, B, s->h, 1, s->h, s, L.count, stream); });     // h += attn Wo^T
     L.run(kKindGlue, [&] { return boost_rmsnorm(s->h, ly.norm2, B, m->hidden, m->rms_eps, s->xn, stream); });
-    L.run(kKindGemv, [&] { return gemv(ly.wgu, s->xn, B, s->gu, 1, nullptr, s, stream); });
+    L.run(kKindGemv, [&] { return gemv(ly.wgu, s->xn, B, s->gu, 1, nullptr, s, L.count, stream); });
     L.run(kKindGlue, [&] { return boost_swiglu(s->gu, B, m->ffn, s->act, stream); });
-    L.run(kKindGemv, [&] { return gemv(ly.wd, s->act, B, s->h, 1, s->h, s, stream); });      // h += act Wd^T
+    L.run(kKindGemv, [&] { return gemv(ly.wd, s->act, B, s->h, 1, s->h, s, L.count, stream); });      // h += act Wd^T
   }
   L.run(kKindGlue, [&] { return boost_rmsnorm(s->h, m->norm_f, B, m->hidden, m->rms_eps, s->xn, stream); });
-  L.run(kKindGemv, [&] { return gemv(m->lm_head, s->xn, B, s->logits, 0, nullptr, s, stream); });
+  L.run(kKindGemv, [&] { return gemv(m->lm_head, s->xn, B, s->logits, 0, nullptr, s, L.count, stream); });
   L.run(kKindGlue, [&] { return boost_argmax(s->logits, B, m->vocab, next_tokens, stream); });
   return L.rc;
 }

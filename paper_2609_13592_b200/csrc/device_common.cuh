@@ -91,6 +91,15 @@ __device__ __forceinline__ void cp_async_arrive_noinc(uint64_t* bar) {
 }
 __device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
 
+// Programmatic dependent launch: let the next kernel of the stream start its prologue now,
+// and wait (before touching anything an earlier kernel produces or still reads) until all
+// earlier kernels have completed and their writes are visible.  No-ops when the kernel was
+// launched without the programmatic-serialization attribute.
+__device__ __forceinline__ void pdl_launch_dependents() {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 __device__ __forceinline__ void named_barrier_sync(uint32_t id, uint32_t n_threads) {
   asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(n_threads) : "memory");
 }
@@ -129,30 +138,42 @@ __device__ __forceinline__ void mma_bf16_16816(float (&d)[4], const uint32_t (&a
       : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
 
-// Two work queues in the workspace header: threadblocks with `host_first` take items of the
-// host-tier queue [0, n_host_items) until it is empty and then help with the HBM queue
-// [n_host_items, n_items); the others do the reverse.  Returns the queue position or
-// 0xFFFFFFFF when both queues are empty.  Called by one thread per threadblock.
+// Two work queues: threadblocks with `host_first` take items of the host-tier queue
+// [0, n_host_items) until it is empty and then help with the HBM queue
+// [n_host_items, n_items); the others do the reverse.  Every threadblock owns its first
+// item by position (no atomic on the critical path of a short kernel); later items come from
+// two atomic counters in `ws`.  Returns the queue position or 0xFFFFFFFF when both queues are
+// empty.  Called by one thread per threadblock.
 struct TierQueues {
   uint32_t* ws;
-  uint32_t n_host_items, n_items;
+  uint32_t n_host_items, n_hbm_items;
+  uint32_t host_base, hbm_base;     // items handed out by position
+  uint32_t first_host, first_hbm;   // this threadblock's own first items (or none)
   bool host_first;
   bool host_open, hbm_open;
-  __device__ __forceinline__ void init(uint32_t* workspace, uint32_t n_host, uint32_t n_all, bool hf) {
-    ws = workspace; n_host_items = n_host; n_items = n_all; host_first = hf;
-    host_open = n_host > 0; hbm_open = n_all > n_host;
+  __device__ __forceinline__ void init(uint32_t* workspace, uint32_t n_host, uint32_t n_all, uint32_t n_host_ctas,
+                                       uint32_t cta, uint32_t n_ctas) {
+    ws = workspace; n_host_items = n_host; n_hbm_items = n_all - n_host;
+    host_first = cta < n_host_ctas;
+    host_base = min(n_host_ctas, n_host_items);
+    hbm_base = min(n_ctas - n_host_ctas, n_hbm_items);
+    first_host = (host_first && cta < n_host_items) ? cta : 0xFFFFFFFFu;
+    first_hbm = (!host_first && cta - n_host_ctas < n_hbm_items) ? n_host_items + cta - n_host_ctas : 0xFFFFFFFFu;
+    host_open = n_host_items > 0; hbm_open = n_hbm_items > 0;
   }
   __device__ __forceinline__ uint32_t take_host() {
+    if (first_host != 0xFFFFFFFFu) { const uint32_t i = first_host; first_host = 0xFFFFFFFFu; return i; }
     if (!host_open) return 0xFFFFFFFFu;
-    const uint32_t i = atomicAdd(ws + kWsHostNext, 1u);
+    const uint32_t i = host_base + atomicAdd(ws + kWsHostNext, 1u);
     if (i < n_host_items) return i;
     host_open = false;
     return 0xFFFFFFFFu;
   }
   __device__ __forceinline__ uint32_t take_hbm() {
+    if (first_hbm != 0xFFFFFFFFu) { const uint32_t i = first_hbm; first_hbm = 0xFFFFFFFFu; return i; }
     if (!hbm_open) return 0xFFFFFFFFu;
-    const uint32_t i = atomicAdd(ws + kWsHbmNext, 1u);
-    if (i < n_items - n_host_items) return n_host_items + i;
+    const uint32_t i = hbm_base + atomicAdd(ws + kWsHbmNext, 1u);
+    if (i < n_hbm_items) return n_host_items + i;
     hbm_open = false;
     return 0xFFFFFFFFu;
   }

@@ -17,6 +17,33 @@ inline int check(cudaError_t e) {
   return BOOST_ERR_CUDA;
 }
 
+// Launch a kernel of the decode chain with programmatic stream serialization allowed: it may
+// start while its predecessor drains, and waits inside (griddepcontrol.wait) before it touches
+// anything the predecessor produces.
+template <typename... KArgs, typename... Args>
+inline int launch_chained(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                          Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return check(cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...));
+}
+
+// boost_gemv_tiered with a private set of queue words (16 zeroed uint32 that no other launch
+// in flight uses): the kernel may then take work and stream weights before its predecessor
+// has finished.  queue_words = nullptr gives the public behaviour.
+int gemv_tiered_launch(const void* const* w_page_ptr, const uint32_t* w_order, size_t n_pages,
+                       size_t n_host_pages, uint32_t N, uint32_t K, const void* x, uint32_t M_b, void* y,
+                       int y_dtype, const void* residual, void* workspace, size_t workspace_bytes,
+                       uint32_t* queue_words, void* stream);
+
 // Launch check: picks up configuration errors of the launch just made.
 inline int check_launch() { return check(cudaGetLastError()); }
 

@@ -59,6 +59,8 @@ __global__ void __launch_bounds__(kAttnThreads, 3) paged_attn_kernel(const AttnP
 
   const uint32_t tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   uint32_t* status = p.ws + kWsStatus;
+  pdl_launch_dependents();
+  pdl_wait();   // the newest K/V rows and q come from the kernel just before this one
 
   // threadblock -> (g, b, split); the highest-numbered KV heads (the host-resident ones
   // under linear placement) come first
@@ -397,6 +399,6 @@ extern "C" int boost_paged_attn_decode_tiered(const void* q, const void* const* 
   }
   const uint64_t grid = (uint64_t)Hkv * B * p.max_splits;
   if (grid > 0x7FFFFFFFull) return BOOST_ERR_INVALID;
-  paged_attn_kernel<<<(unsigned)grid, kAttnThreads, smem, (cudaStream_t)stream>>>(p);
-  return boosth::check_launch();
+  return boosth::launch_chained(paged_attn_kernel, dim3((unsigned)grid), dim3(kAttnThreads), smem,
+                                (cudaStream_t)stream, p);
 }

@@ -43,6 +43,8 @@ struct GemvParams {
   int y_dtype;
   const __nv_bfloat16* residual;
   uint32_t* ws;        // header, then one counter per row tile
+  uint32_t* queue;     // queue words: the header, or a private set (then weights may stream early)
+  uint32_t early;      // 1: private queue words
   float* partials;     // [row_tile][split][x_rows][128]
   uint32_t n_host_ctas;
   uint32_t n_stages;
@@ -79,6 +81,7 @@ __global__ void __launch_bounds__(kGemvThreads, (NT >= 8 ? 1 : 2)) gemv_tiered_k
   const uint32_t n_stages = p.n_stages;
   uint32_t* status = p.ws + kWsStatus;
 
+  pdl_launch_dependents();
   if (tid == 0) {
     for (uint32_t s = 0; s < n_stages; ++s) {
       mbar_init(&full_bar[s], 65);              // 2 x 32 cp.async arrivals + the arrive.expect_tx
@@ -100,7 +103,11 @@ __global__ void __launch_bounds__(kGemvThreads, (NT >= 8 ? 1 : 2)) gemv_tiered_k
     const bool leader = (warp == kConsumerWarps);
     const uint32_t n_host_items = p.n_host_pages * p.items_per_page;
     TierQueues q;
-    q.init(p.ws, n_host_items, p.n_pages * p.items_per_page, blockIdx.x < p.n_host_ctas);
+    q.init(p.queue, n_host_items, p.n_pages * p.items_per_page, p.n_host_ctas, blockIdx.x, gridDim.x);
+    // Weights are never written by the decode chain, so with private queue words the weight
+    // warp starts streaming while the previous kernel is still running; x is produced by
+    // that kernel, so the x warp (and the consumers) wait for it.
+    if (!leader || !p.early) pdl_wait();
     uint32_t stage = 0, phase = 0, icount = 0;
     for (;;) {
       const uint32_t slot = icount & 3u, iphase = (icount >> 2) & 1u;
@@ -201,6 +208,7 @@ __global__ void __launch_bounds__(kGemvThreads, (NT >= 8 ? 1 : 2)) gemv_tiered_k
 
   uint32_t* tile_cnt = p.ws + kWsHeaderWords;
   uint32_t stage = 0, phase = 0;
+  pdl_wait();
   for (;;) {
     mbar_wait(&full_bar[stage], phase, status);
     const uint4 mt = meta[stage];
@@ -408,8 +416,7 @@ int launch_gemv(const GemvParams& p, int sms, cudaStream_t stream) {
     if (n_host_ctas > grid) n_host_ctas = grid;
   }
   q.n_host_ctas = n_host_ctas;
-  gemv_tiered_kernel<NT, MB><<<grid, kGemvThreads, smem, stream>>>(q);
-  return boosth::check_launch();
+  return boosth::launch_chained(gemv_tiered_kernel<NT, MB>, dim3(grid), dim3(kGemvThreads), smem, stream, q);
 }
 
 }  // namespace
@@ -467,6 +474,14 @@ extern "C" int boost_gemv_tiered(const void* const* w_page_ptr, const uint32_t* 
                                  const void* x, uint32_t M_b, void* y, int y_dtype,
                                  const void* residual, void* workspace, size_t workspace_bytes,
                                  void* stream) {
+  return boosth::gemv_tiered_launch(w_page_ptr, w_order, n_pages, n_host_pages, N, K, x, M_b, y, y_dtype,
+                                    residual, workspace, workspace_bytes, nullptr, stream);
+}
+
+int boosth::gemv_tiered_launch(const void* const* w_page_ptr, const uint32_t* w_order, size_t n_pages,
+                               size_t n_host_pages, uint32_t N, uint32_t K, const void* x, uint32_t M_b,
+                               void* y, int y_dtype, const void* residual, void* workspace,
+                               size_t workspace_bytes, uint32_t* queue_words, void* stream) {
   if (!w_page_ptr || !w_order || !x || !y || !workspace) return BOOST_ERR_INVALID;
   if (M_b == 0 || M_b > 128 || (y_dtype != 0 && y_dtype != 1)) return BOOST_ERR_INVALID;
   boost_weight_layout_t lay;
@@ -495,6 +510,8 @@ extern "C" int boost_gemv_tiered(const void* const* w_page_ptr, const uint32_t* 
   p.y = y; p.y_dtype = y_dtype;
   p.residual = static_cast<const __nv_bfloat16*>(residual);
   p.ws = static_cast<uint32_t*>(workspace);
+  p.queue = queue_words ? queue_words : p.ws;
+  p.early = queue_words ? 1u : 0u;
   const size_t header = ((size_t)(kWsHeaderWords + lay.n_row_tiles) * 4 + 255) / 256 * 256;
   p.partials = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + header);
   p.n_host_ctas = 0; p.n_stages = 0;

@@ -20,6 +20,8 @@ constexpr uint32_t kChunkBytes = kTok * kD * 2;
 __global__ void __launch_bounds__(256)
 embed_gather_kernel(const uint4* __restrict__ table, uint32_t vocab, uint32_t row_vecs,
                     const int32_t* __restrict__ tokens, uint4* __restrict__ out) {
+  pdl_launch_dependents();
+  pdl_wait();
   const uint32_t b = blockIdx.x;
   int32_t t = tokens[b];
   if (t < 0 || (uint32_t)t >= vocab) t = 0;
@@ -31,6 +33,8 @@ embed_gather_kernel(const uint4* __restrict__ table, uint32_t vocab, uint32_t ro
 __global__ void __launch_bounds__(256)
 rmsnorm_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restrict__ w,
                uint32_t hidden, float eps, __nv_bfloat16* __restrict__ out) {
+  pdl_launch_dependents();
+  pdl_wait();
   __shared__ float s_part[8];
   __shared__ float s_scale;
   const size_t row = (size_t)blockIdx.x * hidden;
@@ -75,6 +79,8 @@ rope_kv_append_kernel(const __nv_bfloat16* __restrict__ qkv, __nv_bfloat16* __re
                       uint32_t n_pool_blocks, const int32_t* __restrict__ block_table, uint32_t max_blocks,
                       const int32_t* __restrict__ ctx_lens, uint32_t B, uint32_t Hq, uint32_t Hkv,
                       double log2_base, uint32_t* __restrict__ status) {
+  pdl_launch_dependents();
+  pdl_wait();
   const uint32_t half = kD / 2;
   const uint32_t heads = Hq + 2 * Hkv;
   const uint32_t idx = blockIdx.x * blockDim.x + threadIdx.x;
@@ -121,6 +127,8 @@ rope_kv_append_kernel(const __nv_bfloat16* __restrict__ qkv, __nv_bfloat16* __re
 // act = silu(gate) * up with gate = gu[:, :F], up = gu[:, F:]
 __global__ void __launch_bounds__(256)
 swiglu_kernel(const __nv_bfloat16* __restrict__ gu, uint32_t B, uint32_t F, __nv_bfloat16* __restrict__ out) {
+  pdl_launch_dependents();
+  pdl_wait();
   const size_t n = (size_t)B * F / 2;
   const size_t stride = (size_t)gridDim.x * blockDim.x;
   for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += stride) {
@@ -137,6 +145,8 @@ swiglu_kernel(const __nv_bfloat16* __restrict__ gu, uint32_t B, uint32_t F, __nv
 // argmax over fp32 logits, lowest index on ties; one threadblock per row
 __global__ void __launch_bounds__(1024)
 argmax_kernel(const float* __restrict__ logits, uint32_t V, int32_t* __restrict__ out) {
+  pdl_launch_dependents();
+  pdl_wait();
   __shared__ float s_val[32];
   __shared__ uint32_t s_idx[32];
   const float* row = logits + (size_t)blockIdx.x * V;
@@ -175,9 +185,8 @@ extern "C" int boost_embed_gather(const void* table, uint32_t vocab, uint32_t hi
   if (B == 0) return BOOST_OK;
   if (!table || !tokens || !out || vocab == 0 || hidden == 0) return BOOST_ERR_INVALID;
   if (hidden % 8 != 0 || ((uintptr_t)table % 16) || ((uintptr_t)out % 16)) return BOOST_ERR_ALIGN;
-  embed_gather_kernel<<<B, 256, 0, (cudaStream_t)stream>>>(static_cast<const uint4*>(table), vocab, hidden / 8,
-                                                         tokens, static_cast<uint4*>(out));
-  return boosth::check_launch();
+  return boosth::launch_chained(embed_gather_kernel, dim3(B), dim3(256), 0, (cudaStream_t)stream,
+                                static_cast<const uint4*>(table), vocab, hidden / 8, tokens, static_cast<uint4*>(out));
 }
 
 extern "C" int boost_rmsnorm(const void* x, const void* weight, uint32_t B, uint32_t hidden, float eps,
@@ -185,10 +194,9 @@ extern "C" int boost_rmsnorm(const void* x, const void* weight, uint32_t B, uint
   if (B == 0) return BOOST_OK;
   if (!x || !weight || !out || hidden == 0) return BOOST_ERR_INVALID;
   if (hidden % 2 != 0 || ((uintptr_t)x % 4) || ((uintptr_t)out % 4) || ((uintptr_t)weight % 4)) return BOOST_ERR_ALIGN;
-  rmsnorm_kernel<<<B, 256, 0, (cudaStream_t)stream>>>(static_cast<const __nv_bfloat16*>(x),
-                                                     static_cast<const __nv_bfloat16*>(weight), hidden, eps,
-                                                     static_cast<__nv_bfloat16*>(out));
-  return boosth::check_launch();
+  return boosth::launch_chained(rmsnorm_kernel, dim3(B), dim3(256), 0, (cudaStream_t)stream,
+                                static_cast<const __nv_bfloat16*>(x), static_cast<const __nv_bfloat16*>(weight),
+                                hidden, eps, static_cast<__nv_bfloat16*>(out));
 }
 
 extern "C" int boost_rope_kv_append(const void* qkv, void* q_out, const void* const* k_page_ptr,
@@ -203,11 +211,11 @@ extern "C" int boost_rope_kv_append(const void* qkv, void* q_out, const void* co
   if (Hq == 0 || Hkv == 0 || max_blocks == 0 || n_pool_blocks == 0 || !(rope_base > 1.f)) return BOOST_ERR_INVALID;
   const uint64_t n = (uint64_t)B * (Hq + 2 * Hkv) * (kD / 2);
   if (n > 0x7FFFFFFFull) return BOOST_ERR_INVALID;
-  rope_kv_append_kernel<<<(unsigned)((n + 255) / 256), 256, 0, (cudaStream_t)stream>>>(
-      static_cast<const __nv_bfloat16*>(qkv), static_cast<__nv_bfloat16*>(q_out), k_page_ptr, v_page_ptr,
-      n_pool_blocks, block_table, max_blocks, ctx_lens, B, Hq, Hkv, log2((double)rope_base),
-      static_cast<uint32_t*>(status_word));
-  return boosth::check_launch();
+  return boosth::launch_chained(rope_kv_append_kernel, dim3((unsigned)((n + 255) / 256)), dim3(256), 0,
+                                (cudaStream_t)stream, static_cast<const __nv_bfloat16*>(qkv),
+                                static_cast<__nv_bfloat16*>(q_out), k_page_ptr, v_page_ptr, n_pool_blocks,
+                                block_table, max_blocks, ctx_lens, B, Hq, Hkv, log2((double)rope_base),
+                                static_cast<uint32_t*>(status_word));
 }
 
 extern "C" int boost_swiglu(const void* gate_up, uint32_t B, uint32_t F, void* out, void* stream) {
@@ -218,14 +226,12 @@ extern "C" int boost_swiglu(const void* gate_up, uint32_t B, uint32_t F, void* o
   size_t blocks = (n + 255) / 256;
   const size_t cap = (size_t)(boosth::sm_count() > 0 ? boosth::sm_count() : 148) * 8;
   if (blocks > cap) blocks = cap;
-  swiglu_kernel<<<(unsigned)blocks, 256, 0, (cudaStream_t)stream>>>(static_cast<const __nv_bfloat16*>(gate_up), B, F,
-                                                                   static_cast<__nv_bfloat16*>(out));
-  return boosth::check_launch();
+  return boosth::launch_chained(swiglu_kernel, dim3((unsigned)blocks), dim3(256), 0, (cudaStream_t)stream,
+                                static_cast<const __nv_bfloat16*>(gate_up), B, F, static_cast<__nv_bfloat16*>(out));
 }
 
 extern "C" int boost_argmax(const float* logits, uint32_t B, uint32_t V, int32_t* out, void* stream) {
   if (B == 0) return BOOST_OK;
   if (!logits || !out || V == 0) return BOOST_ERR_INVALID;
-  argmax_kernel<<<B, 1024, 0, (cudaStream_t)stream>>>(logits, V, out);
-  return boosth::check_launch();
+  return boosth::launch_chained(argmax_kernel, dim3(B), dim3(1024), 0, (cudaStream_t)stream, logits, V, out);
 }

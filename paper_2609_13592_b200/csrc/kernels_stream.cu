@@ -67,7 +67,7 @@ stream_reduce_kernel(const void* const* __restrict__ page_ptr, const uint32_t* _
   float* tile_part = reinterpret_cast<float*>(ws + kWsHeaderWords + n_pages);
 
   TierQueues q;
-  q.init(ws, n_host_pages * kTilesPerPage, n_pages * kTilesPerPage, blockIdx.x < n_host_ctas);
+  q.init(ws, n_host_pages * kTilesPerPage, n_pages * kTilesPerPage, n_host_ctas, blockIdx.x, gridDim.x);
   const uint32_t tid = threadIdx.x;
 
   for (;;) {
