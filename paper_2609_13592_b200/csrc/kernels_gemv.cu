@@ -11,6 +11,7 @@
 // so a threadblock reads one tier at a time.
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
+#include <stdlib.h>
 
 #include "device_common.cuh"
 #include "host_common.h"
@@ -31,6 +32,21 @@ constexpr uint32_t kSmemBudget = 224u * 1024u;
 constexpr uint32_t kXRowStride = 144;  // 128 data bytes + 16: 8 consecutive rows hit distinct banks
 
 enum : uint32_t { kFlagFirst = 1u, kFlagLast = 2u, kFlagStop = 4u };
+
+#ifdef BOOST_TRACE
+// Debug build only: per-threadblock time stamps (global timer, ns) for timeline analysis.
+__device__ unsigned long long* g_trace = nullptr;
+__device__ __forceinline__ unsigned long long gtime() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+  return t;
+}
+#define TRACE(slot) do { if (g_trace && (threadIdx.x & 31) == 0) g_trace[(size_t)blockIdx.x * 16 + (slot)] = gtime(); } while (0)
+#define TRACE_ONCE(slot) do { if (g_trace && (threadIdx.x & 31) == 0 && g_trace[(size_t)blockIdx.x * 16 + (slot)] == 0) g_trace[(size_t)blockIdx.x * 16 + (slot)] = gtime(); } while (0)
+#else
+#define TRACE(slot) do { } while (0)
+#define TRACE_ONCE(slot) do { } while (0)
+#endif
 
 struct GemvParams {
   const void* const* w_page_ptr;
@@ -62,6 +78,24 @@ __device__ __forceinline__ void store_out(const GemvParams& p, uint32_t m, uint3
   else static_cast<__nv_bfloat16*>(p.y)[idx] = __float2bfloat16_rn(v);
 }
 
+// four consecutive outputs of one batch row; N % 4 == 0 and n % 4 == 0
+__device__ __forceinline__ void store_out4(const GemvParams& p, uint32_t m, uint32_t n, float4 v) {
+  const size_t idx = (size_t)m * p.N + n;
+  if (p.residual) {
+    const uint2 r = *reinterpret_cast<const uint2*>(p.residual + idx);
+    v.x += bf16_lo(r.x); v.y += bf16_hi(r.x); v.z += bf16_lo(r.y); v.w += bf16_hi(r.y);
+  }
+  if (p.y_dtype == 0) {
+    *reinterpret_cast<float4*>(static_cast<float*>(p.y) + idx) = v;
+  } else {
+    const __nv_bfloat162 lo = __floats2bfloat162_rn(v.x, v.y), hi = __floats2bfloat162_rn(v.z, v.w);
+    uint2 o;
+    o.x = *reinterpret_cast<const uint32_t*>(&lo);
+    o.y = *reinterpret_cast<const uint32_t*>(&hi);
+    *reinterpret_cast<uint2*>(static_cast<__nv_bfloat16*>(p.y) + idx) = o;
+  }
+}
+
 // NT > 0: tensor-core path with NT batch tiles of 8; NT == 0: CUDA-core path for MB rows.
 template <int NT, int MB>
 __global__ void __launch_bounds__(kGemvThreads, (NT >= 8 ? 1 : 2)) gemv_tiered_kernel(const GemvParams p) {
@@ -81,6 +115,7 @@ __global__ void __launch_bounds__(kGemvThreads, (NT >= 8 ? 1 : 2)) gemv_tiered_k
   const uint32_t n_stages = p.n_stages;
   uint32_t* status = p.ws + kWsStatus;
 
+  if (tid == 0) TRACE(0);
   pdl_launch_dependents();
   if (tid == 0) {
     for (uint32_t s = 0; s < n_stages; ++s) {
@@ -131,6 +166,7 @@ __global__ void __launch_bounds__(kGemvThreads, (NT >= 8 ? 1 : 2)) gemv_tiered_k
         if (lane == 0) mbar_arrive(&item_empty[slot]);
       }
       ++icount;
+      if (leader) TRACE_ONCE(1);
       if (qi == 0xFFFFFFFFu) break;
       const uint32_t page = p.w_order[qi / p.items_per_page];
       const uint32_t first_blk = (page * p.items_per_page + qi % p.items_per_page) * p.run;
@@ -212,6 +248,7 @@ __global__ void __launch_bounds__(kGemvThreads, (NT >= 8 ? 1 : 2)) gemv_tiered_k
   for (;;) {
     mbar_wait(&full_bar[stage], phase, status);
     const uint4 mt = meta[stage];
+    if (warp == 0) TRACE_ONCE(2);
     if (mt.z & kFlagStop) break;
     if (mt.z & kFlagFirst) {
 #pragma unroll
@@ -270,6 +307,7 @@ __global__ void __launch_bounds__(kGemvThreads, (NT >= 8 ? 1 : 2)) gemv_tiered_k
     if (++stage == n_stages) { stage = 0; phase ^= 1u; }
 
     if (mt.z & kFlagLast) {
+      if (warp == 0) { TRACE_ONCE(3); TRACE(5); }
       const uint32_t row_tile = mt.x, split = mt.y;
       if constexpr (NT == 0) {
         // finish the dot products: sum over the 8 lanes that share a row
@@ -328,30 +366,56 @@ __global__ void __launch_bounds__(kGemvThreads, (NT >= 8 ? 1 : 2)) gemv_tiered_k
           const float4* base = reinterpret_cast<const float4*>(
               p.partials + (size_t)row_tile * p.splits * kXRows * kBlockRows);
           constexpr uint32_t kVecRow = kBlockRows / 4;   // float4 per batch row
-          for (uint32_t idx = tid; idx < p.M_b * kVecRow; idx += kConsumerThreads) {
-            const uint32_t m = idx / kVecRow, v4 = idx % kVecRow;
-            float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
-            for (uint32_t sp0 = 0; sp0 < p.splits; sp0 += 8) {   // loads in batches of 8, sums in split order
-              float4 t[8];
+          // Each thread owns two float4 outputs at a time and walks the splits in order, four
+          // splits (eight independent loads) per round, so the L2 latency is paid once per
+          // round and not once per load.
+          const uint32_t n_vec = p.M_b * kVecRow;
+          for (uint32_t idx0 = tid; idx0 < n_vec; idx0 += 2 * kConsumerThreads) {
+            const uint32_t idx1 = idx0 + kConsumerThreads;
+            const bool two = idx1 < n_vec;
+            float4 a0 = make_float4(0.f, 0.f, 0.f, 0.f), a1 = a0;
+            for (uint32_t sp0 = 0; sp0 < p.splits; sp0 += 4) {
+              float4 t0[4], t1[4];
 #pragma unroll
-              for (uint32_t u = 0; u < 8; ++u)
-                if (sp0 + u < p.splits) t[u] = __ldcg(base + ((size_t)(sp0 + u) * kXRows + m) * kVecRow + v4);
+              for (uint32_t u = 0; u < 4; ++u) {
+                if (sp0 + u < p.splits) {
+                  const float4* src = base + (size_t)(sp0 + u) * kXRows * kVecRow;
+                  t0[u] = __ldcg(src + idx0);
+                  if (two) t1[u] = __ldcg(src + idx1);
+                }
+              }
 #pragma unroll
-              for (uint32_t u = 0; u < 8; ++u)
-                if (sp0 + u < p.splits) { s.x += t[u].x; s.y += t[u].y; s.z += t[u].z; s.w += t[u].w; }
+              for (uint32_t u = 0; u < 4; ++u) {
+                if (sp0 + u < p.splits) {
+                  a0.x += t0[u].x; a0.y += t0[u].y; a0.z += t0[u].z; a0.w += t0[u].w;
+                  if (two) { a1.x += t1[u].x; a1.y += t1[u].y; a1.z += t1[u].z; a1.w += t1[u].w; }
+                }
+              }
             }
-            const uint32_t n = row_tile * kBlockRows + v4 * 4;
-            if (n < p.N) store_out(p, m, n, s.x);
-            if (n + 1 < p.N) store_out(p, m, n + 1, s.y);
-            if (n + 2 < p.N) store_out(p, m, n + 2, s.z);
-            if (n + 3 < p.N) store_out(p, m, n + 3, s.w);
+            for (int i = 0; i < (two ? 2 : 1); ++i) {
+              const uint32_t idx = i ? idx1 : idx0;
+              const float4 v = i ? a1 : a0;
+              const uint32_t m = idx / kVecRow, v4 = idx % kVecRow;
+              const uint32_t n = row_tile * kBlockRows + v4 * 4;
+              if (n + 3 < p.N && (p.N & 3u) == 0) {
+                store_out4(p, m, n, v);
+              } else {
+                if (n < p.N) store_out(p, m, n, v.x);
+                if (n + 1 < p.N) store_out(p, m, n + 1, v.y);
+                if (n + 2 < p.N) store_out(p, m, n + 2, v.z);
+                if (n + 3 < p.N) store_out(p, m, n + 3, v.w);
+              }
+            }
           }
           if (tid == 0) tile_cnt[row_tile] = 0;
+          if (warp == 0) TRACE(8);
         }
         named_barrier_sync(1, kConsumerThreads);
       }
+      if (warp == 0) { TRACE_ONCE(4); TRACE(6); }
     }
   }
+  if (warp == 0) TRACE(7);
 }
 
 // Packed form: 16-byte chunk `pos` of row r of block (t, kb) holds columns
@@ -377,11 +441,12 @@ pack_weights_kernel(const uint4* __restrict__ w, uint32_t N, uint32_t K, uint32_
 
 uint32_t pick_run(uint32_t n_row_tiles, uint32_t k_blocks) {
   // Run length of a work item in blocks: a power of two that divides the row tile's
-  // k_blocks (and so the 128 blocks of a page).  Longer runs mean fewer split-K partial
-  // sums; shorter runs mean more items to balance over the SMs.  Take the longest run that
-  // leaves about three items per SM, else the longest that leaves one per SM, else 1.
+  // k_blocks (and so the 128 blocks of a page).  Every run ends with a split-K partial sum
+  // that is written, fenced and later re-read, and on B200 that costs more than a coarse
+  // split of the work (measured): take the longest run that still leaves one item per SM,
+  // else the longest that leaves 64 items, else single blocks.
   const uint64_t total = (uint64_t)n_row_tiles * k_blocks;
-  const uint64_t wanted[2] = {444, 148};
+  const uint64_t wanted[2] = {148, 64};
   for (int pass = 0; pass < 2; ++pass)
     for (uint32_t run = 32; run >= 1; run >>= 1)
       if (k_blocks % run == 0 && total / run >= wanted[pass]) return run;
@@ -406,8 +471,13 @@ int launch_gemv(const GemvParams& p, int sms, cudaStream_t stream) {
     if (rc != BOOST_OK) return rc;
     configured = true;
   }
-  uint32_t grid = (uint32_t)sms * ctas_per_sm;
+  // Threadblocks share HBM bandwidth, so what has to be even is the number of items per
+  // threadblock: use as many blocks as give every block the same count (rounded up).
+  const uint32_t max_ctas = (uint32_t)sms * ctas_per_sm;
   const uint32_t queue_len = q.n_pages * q.items_per_page;
+  const uint32_t items = q.n_items ? q.n_items : 1;
+  const uint32_t per_cta = (items + max_ctas - 1) / max_ctas;
+  uint32_t grid = (items + per_cta - 1) / per_cta;
   if (grid > queue_len) grid = queue_len;
   uint32_t n_host_ctas = 0;
   if (q.n_host_pages) {
@@ -426,6 +496,10 @@ extern "C" int boost_weight_layout(uint32_t N, uint32_t K, boost_weight_layout_t
   out->n_row_tiles = (N + kBlockRows - 1) / kBlockRows;
   out->k_blocks = (K + kBlockK - 1) / kBlockK;
   out->blocks_per_item = pick_run(out->n_row_tiles, out->k_blocks);
+  if (const char* e = getenv("BOOST_RUN")) {   // experiment hook
+    const uint32_t r = (uint32_t)atoi(e);
+    if (r && out->k_blocks % r == 0 && 128 % r == 0) out->blocks_per_item = r;
+  }
   out->splits = out->k_blocks / out->blocks_per_item;
   out->bytes = (uint64_t)out->n_row_tiles * out->k_blocks * kBlockBytes;
   out->n_pages = (out->bytes + kPageBytes - 1) / kPageBytes;
@@ -525,3 +599,9 @@ int boosth::gemv_tiered_launch(const void* const* w_page_ptr, const uint32_t* w_
     default: return launch_gemv<16, 0>(p, sms, st);
   }
 }
+
+#ifdef BOOST_TRACE
+extern "C" int boost_debug_set_trace(void* ptr) {
+  return boosth::check(cudaMemcpyToSymbol(g_trace, &ptr, sizeof(ptr)));
+}
+#endif
