@@ -79,6 +79,7 @@ __global__ void __launch_bounds__(kAttnThreads, (NH == 1 ? 3 : 2)) paged_attn_ke
   __shared__ uint64_t full_bar[kMaxStages];
   __shared__ uint64_t empty_bar[kMaxStages];
   __shared__ uint4 meta[kMaxStages];
+  __shared__ uint32_t meta_ctx[kMaxStages];
   __shared__ float merge_ml[kAttnWarps][kMaxGroup][2];
   __shared__ uint32_t s_old;
 
@@ -138,6 +139,7 @@ __global__ void __launch_bounds__(kAttnThreads, (NH == 1 ? 3 : 2)) paged_attn_ke
             mbar_wait(&empty_bar[stage], phase ^ 1u, status);
             const uint32_t flags = (i == 0 ? kAFirst : 0u) | (i + 1 == n_emit ? kALast : 0u) | (nb ? 0u : kANoData);
             meta[stage] = make_uint4(b, g | (split << 16), (blk0 + i) * kTok, flags | (i << 16));
+            meta_ctx[stage] = ctx;
             const bool bulk = nb && !from_host;
             mbar_arrive_expect_tx(&full_bar[stage], bulk ? kStageBytes : 0u);
             if (bulk) {
@@ -215,16 +217,19 @@ __global__ void __launch_bounds__(kAttnThreads, (NH == 1 ? 3 : 2)) paged_attn_ke
       }
     }
     const uint32_t b = mt.x, g = mt.y & 0xFFFFu, split = mt.y >> 16;
-    const uint32_t ctx = (uint32_t)max(p.ctx_lens[b], 0);
+    const uint32_t ctx = meta_ctx[stage];
     if (!(flags & kANoData) && ((mt.w >> 16) & 3u) == warp) {
       const uint32_t kbase = smem_u32(stage_sm + (size_t)stage * kStageBytes);
       const uint32_t vbase = kbase + kChunkBytes;
       const uint32_t tok = (lane & 7) + ((lane >> 4) << 3);     // ldmatrix row of this lane
       const uint32_t sub = (lane >> 3) & 1;                     // which 16-byte chunk of a pair
       // S^T = K q^T: rows = 16 tokens, columns = heads
-      float s[NH][4];
+      float s[NH][4], s2[NH][4];   // two accumulation chains, added at the end
 #pragma unroll
-      for (int nh = 0; nh < NH; ++nh) { s[nh][0] = s[nh][1] = s[nh][2] = s[nh][3] = 0.f; }
+      for (int nh = 0; nh < NH; ++nh) {
+        s[nh][0] = s[nh][1] = s[nh][2] = s[nh][3] = 0.f;
+        s2[nh][0] = s2[nh][1] = s2[nh][2] = s2[nh][3] = 0.f;
+      }
 #pragma unroll
       for (uint32_t ks = 0; ks < 8; ++ks) {
         // A fragment of K: m0 tokens 0-7 / chunk 2ks, m1 tokens 8-15 / chunk 2ks, m2, m3 chunk 2ks+1
@@ -233,8 +238,12 @@ __global__ void __launch_bounds__(kAttnThreads, (NH == 1 ? 3 : 2)) paged_attn_ke
         uint32_t a[4];
         ldmatrix_x4(a[0], a[1], a[2], a[3], kbase + a_tok * 256 + ((a_chunk ^ (a_tok & 7)) << 4));
 #pragma unroll
-        for (int nh = 0; nh < NH; ++nh) mma_bf16_16816(s[nh], a, qb[nh][ks][0], qb[nh][ks][1]);
+        for (int nh = 0; nh < NH; ++nh) mma_bf16_16816((ks & 1) ? s2[nh] : s[nh], a, qb[nh][ks][0], qb[nh][ks][1]);
       }
+#pragma unroll
+      for (int nh = 0; nh < NH; ++nh)
+#pragma unroll
+        for (int r = 0; r < 4; ++r) s[nh][r] += s2[nh][r];
       // mask the tail of the last block, scale into the log2 domain; online softmax per head
       const uint32_t t_lo = mt.z + gq, t_hi = t_lo + 8;
       uint32_t pa[NH][3][2];
@@ -345,9 +354,11 @@ __global__ void __launch_bounds__(kAttnThreads, (NH == 1 ? 3 : 2)) paged_attn_ke
     if (!single) {
       // the last split of (b, g) to arrive combines all splits, in split order
       uint32_t* cnt = p.ws + kWsHeaderWords + b * p.Hkv + g;
-      __threadfence();
       named_barrier_sync(1, kConsumerThreads);
-      if (tid == 0) s_old = atomicAdd(cnt, 1u);
+      if (tid == 0) {
+        __threadfence();   // cumulative: publishes the partials of all 128 threads (ordered by the barrier)
+        s_old = atomicAdd(cnt, 1u);
+      }
       named_barrier_sync(1, kConsumerThreads);
       if (s_old == n_splits - 1) {
         __threadfence();

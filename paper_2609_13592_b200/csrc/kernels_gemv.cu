@@ -357,9 +357,11 @@ __global__ void __launch_bounds__(kGemvThreads, (NT >= 8 ? 1 : 2)) gemv_tiered_k
       if (!direct) {
         // the threadblock that delivers the last partial sum of a row tile adds them up in
         // split order (fixed order: deterministic) and writes the output
-        __threadfence();
         named_barrier_sync(1, kConsumerThreads);
-        if (tid == 0) s_old = atomicAdd(tile_cnt + row_tile, 1u);
+        if (tid == 0) {
+          __threadfence();   // cumulative: publishes the partials of all consumer threads (ordered by the barrier)
+          s_old = atomicAdd(tile_cnt + row_tile, 1u);
+        }
         named_barrier_sync(1, kConsumerThreads);
         if (s_old == p.splits - 1) {
           __threadfence();
