@@ -1,20 +1,19 @@
 // Tiered paged decode attention (split-KV) over the KV cache of a boost_kv_pool, and the
 // copies that move a logical [Hkv][N][16][D] cache into and out of its pages.
 //
-// Persistent threadblocks, two per SM.  A work item is a KV-head chunk run: sequence b, KV
+// Persistent grid of autonomous warps.  A work item is a KV-head chunk run: sequence b, KV
 // head g, blocks [16 s, 16 s + 16) of the sequence (Sec. 3.3: attention threadblocks work
 // on KV head chunks); items of the highest-numbered heads - the ones linear placement puts
-// on the host tier - are handed out first.  A producer warp walks the items and fills a
-// ring of 8 KiB stages, one KV block (K chunk + V chunk) per stage: two 4 KiB bulk copies
-// through the TMA unit for HBM pages, a fan of 16-byte cp.async loads for host pages; the
-// query rows of the item ride along with its first block.  Four consumer warps take the
-// blocks of an item round-robin, each with its own running softmax state.  The products
-// are bf16 tensor-core MMAs with the 16 tokens of a block as the 16-row dimension and the
-// query heads of the group as the 8-wide dimension (S^T = K q^T, O^T += V^T P^T, so a group of
-// four heads wastes half a tile instead of three quarters); P goes in as three bf16 terms,
-// transposed in registers with movmatrix; the online softmax is fp32.  At the end of
-// an item the warps merge through shared memory, and the last split of a (b, g) pair to
-// finish combines all splits in split order.
+// on the host tier - are handed out first.  Each warp takes whole items and streams their
+// KV blocks through its own two-stage ring in shared memory: per block two 4 KiB bulk
+// copies through the TMA unit (K chunk, V chunk) when the page is in HBM, a fan of 16-byte
+// cp.async loads when it is host memory.  Twelve such warps per SM keep about 150 KiB in
+// flight with no producer warp, no block-wide barrier and no cross-warp merge.  The
+// products are bf16 tensor-core MMAs with the 16 tokens of a block as the 16-row dimension
+// and the query heads of the group as the 8-wide dimension (S^T = K q^T, O^T += V^T P^T: a
+// group of four heads wastes half a tile instead of three quarters); P goes in as three
+// bf16 terms, transposed in registers with movmatrix; the online softmax is fp32.  The
+// last split of a (b, g) pair to finish combines all splits in split order.
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <math_constants.h>
@@ -32,16 +31,10 @@ constexpr uint32_t kChunkBytes = kTok * kD * 2;          // 4 KiB
 constexpr uint32_t kChunksPerPage = kPageBytes / kChunkBytes;
 constexpr uint32_t kItemBlocks = 16;                     // KV blocks per work item
 constexpr uint32_t kStageBytes = 2 * kChunkBytes;        // K chunk + V chunk
-constexpr uint32_t kAttnWarps = 4;                       // consumer warps
-constexpr uint32_t kConsumerThreads = kAttnWarps * 32;
-constexpr uint32_t kAttnThreads = kConsumerThreads + 32; // + producer warp
+constexpr uint32_t kAttnWarps = 4;                       // warps per threadblock
+constexpr uint32_t kAttnThreads = kAttnWarps * 32;
+constexpr uint32_t kWarpStages = 2;                      // ring depth of one warp
 constexpr uint32_t kMaxGroup = 16;
-constexpr uint32_t kMaxStages = 12;
-constexpr uint32_t kQRowStride = 272;                    // 256 data bytes + 16: rows hit distinct banks
-constexpr uint32_t kAttnSmemBudget3 = 74u * 1024u;       // three threadblocks per SM (groups up to 8)
-constexpr uint32_t kAttnSmemBudget2 = 111u * 1024u;      // two per SM (groups up to 16)
-
-enum : uint32_t { kAFirst = 1u, kALast = 2u, kAStop = 4u, kANoData = 8u };
 
 struct AttnParams {
   const __nv_bfloat16* q;
@@ -52,7 +45,7 @@ struct AttnParams {
   const int32_t* block_table;
   uint32_t max_blocks;
   const int32_t* ctx_lens;
-  uint32_t B, Hq, Hkv, group, max_splits, n_items, n_stages;
+  uint32_t B, Hq, Hkv, group, max_splits, n_items;
   float scale_log2e;
   uint32_t* ws;        // header (status, item counter, done counter) + one counter per (b, g)
   float* part_ml;      // [B][Hq][max_splits][2]
@@ -71,315 +64,261 @@ template <int NH>
 __global__ void __launch_bounds__(kAttnThreads, (NH == 1 ? 3 : 2)) paged_attn_kernel(const AttnParams p) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~uintptr_t(127));
-  const uint32_t n_stages = p.n_stages;
-  uint8_t* stage_sm = smem;                                        // [n_stages][K 4 KiB | V 4 KiB]
-  uint8_t* q_sm = smem + (size_t)n_stages * kStageBytes;           // [n_stages][group][kQRowStride]
-  const uint32_t q_slot_bytes = p.group * kQRowStride;             // query rows travel with an item's first stage
-  float* merge_o = reinterpret_cast<float*>(q_sm + (size_t)n_stages * q_slot_bytes);  // [warps][group][128]
-  __shared__ uint64_t full_bar[kMaxStages];
-  __shared__ uint64_t empty_bar[kMaxStages];
-  __shared__ uint4 meta[kMaxStages];
-  __shared__ uint32_t meta_ctx[kMaxStages];
-  __shared__ float merge_ml[kAttnWarps][kMaxGroup][2];
-  __shared__ uint32_t s_old;
+  __shared__ uint64_t full_bar[kAttnWarps][kWarpStages];
 
   const uint32_t tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  uint8_t* ring = smem + (size_t)warp * kWarpStages * kStageBytes;   // this warp's stages
   uint32_t* status = p.ws + kWsStatus;
   pdl_launch_dependents();
-  if (tid == 0) {
-    for (uint32_t s = 0; s < n_stages; ++s) {
-      mbar_init(&full_bar[s], 33);   // 32 cp.async arrivals + the arrive.expect_tx
-      mbar_init(&empty_bar[s], kAttnWarps);
-    }
+  if (lane == 0) {
+    for (uint32_t s = 0; s < kWarpStages; ++s) mbar_init(&full_bar[warp][s], 33);   // 32 cp.async arrivals + arrive.expect_tx
     fence_barrier_init();
   }
+  __syncwarp();
   pdl_wait();   // q and the newest K/V rows come from the kernels just before this one
-  __syncthreads();
 
-  if (warp == kAttnWarps) {
-    // ------------------------------------------------------------------ producer warp
-    uint32_t stage = 0, phase = 0;
-    uint32_t id = blockIdx.x;   // first item by position, later ones from the counter
-    const uint32_t per_head = p.B * p.max_splits;
-    while (id < p.n_items) {
-      const uint32_t g = p.Hkv - 1 - id / per_head;     // host-resident heads first
-      const uint32_t b = (id % per_head) / p.max_splits;
-      const uint32_t split = id % p.max_splits;
-      const uint32_t ctx = (uint32_t)max(p.ctx_lens[b], 0);
-      const uint32_t n_blk = (ctx + kTok - 1) / kTok;
-      const uint32_t n_splits = n_blk ? (n_blk + kItemBlocks - 1) / kItemBlocks : 1;
-      if (split < n_splits) {
-        const uint32_t blk0 = split * kItemBlocks;
-        const uint32_t nb = min(kItemBlocks, n_blk - min(n_blk, blk0));
-        // every lane resolves one block of the item: table entry, page, addresses
-        const uint8_t* ksrc = nullptr;
-        const uint8_t* vsrc = nullptr;
-        uint32_t host_bit = 0;
-        if (lane < nb) {
-          int32_t blk = p.block_table[(size_t)b * p.max_blocks + blk0 + lane];
-          if (blk < 0 || (uint32_t)blk >= p.n_pool_blocks) {   // bad table entry: record, read block 0
-            atomicOr(status, kErrBadIndex);
-            blk = 0;
-          }
-          const uint32_t lin = g * p.n_pool_blocks + (uint32_t)blk;
-          const uint32_t page = lin / kChunksPerPage;
-          const size_t in_page = (size_t)(lin % kChunksPerPage) * kChunkBytes;
-          ksrc = static_cast<const uint8_t*>(p.k_page_ptr[page]) + in_page;
-          vsrc = static_cast<const uint8_t*>(p.v_page_ptr[page]) + in_page;
-          host_bit = page >= p.first_host_page ? 1u : 0u;
-        }
-        const uint32_t n_emit = nb ? nb : 1u;   // an empty sequence still gets one (data-less) stage
-        for (uint32_t i = 0; i < n_emit; ++i) {
-          const uint8_t* ks = reinterpret_cast<const uint8_t*>(__shfl_sync(0xFFFFFFFFu, (unsigned long long)ksrc, i));
-          const uint8_t* vs = reinterpret_cast<const uint8_t*>(__shfl_sync(0xFFFFFFFFu, (unsigned long long)vsrc, i));
-          const bool from_host = __shfl_sync(0xFFFFFFFFu, host_bit, i) != 0;
-          uint8_t* kdst = stage_sm + (size_t)stage * kStageBytes;
-          uint8_t* vdst = kdst + kChunkBytes;
-          if (lane == 0) {
-            mbar_wait(&empty_bar[stage], phase ^ 1u, status);
-            const uint32_t flags = (i == 0 ? kAFirst : 0u) | (i + 1 == n_emit ? kALast : 0u) | (nb ? 0u : kANoData);
-            meta[stage] = make_uint4(b, g | (split << 16), (blk0 + i) * kTok, flags | (i << 16));
-            meta_ctx[stage] = ctx;
-            const bool bulk = nb && !from_host;
-            mbar_arrive_expect_tx(&full_bar[stage], bulk ? kStageBytes : 0u);
-            if (bulk) {
-              bulk_copy_g2s(kdst, ks, kChunkBytes, &full_bar[stage]);
-              bulk_copy_g2s(vdst, vs, kChunkBytes, &full_bar[stage]);
-            }
-          }
-          __syncwarp();
-          if (nb && from_host) {
-#pragma unroll
-            for (uint32_t c = lane; c < kChunkBytes / 16; c += 32) {
-              cp_async_16(kdst + c * 16, ks + c * 16, 16u);
-              cp_async_16(vdst + c * 16, vs + c * 16, 16u);
-            }
-          }
-          if (i == 0) {
-            // the item's query rows: group x 256 bytes into this item's slot
-            const uint8_t* qsrc = reinterpret_cast<const uint8_t*>(p.q + ((size_t)b * p.Hq + g * p.group) * kD);
-            uint8_t* qdst = q_sm + (size_t)stage * q_slot_bytes;
-            for (uint32_t c = lane; c < p.group * 16; c += 32)
-              cp_async_16(qdst + (c >> 4) * kQRowStride + (c & 15) * 16, qsrc + c * 16, 16u);
-          }
-          cp_async_arrive_noinc(&full_bar[stage]);
-          if (++stage == n_stages) { stage = 0; phase ^= 1u; }
-        }
-      }
-      uint32_t nxt = 0;
-      if (lane == 0) nxt = gridDim.x + atomicAdd(p.ws + kWsHbmNext, 1u);
-      id = __shfl_sync(0xFFFFFFFFu, nxt, 0);
-    }
-    // tell the consumers to stop, then the last threadblock out resets the counters
-    if (lane == 0) {
-      mbar_wait(&empty_bar[stage], phase ^ 1u, status);
-      meta[stage] = make_uint4(0u, 0u, 0u, kAStop);
-      mbar_arrive(&full_bar[stage]);
-    }
-    __syncwarp();
-    cp_async_arrive_noinc(&full_bar[stage]);
-    if (lane == 0) {
-      __threadfence();
-      const uint32_t d = atomicAdd(p.ws + kWsDone, 1u);
-      if (d == gridDim.x - 1) { p.ws[kWsHbmNext] = 0; p.ws[kWsDone] = 0; __threadfence(); }
-    }
-    return;
-  }
-
-  // -------------------------------------------------------------------- consumer warps
-  // Fragment coordinates: rows g, g+8 (tokens for S^T, d for O^T), columns c0, c0+1 (heads).
+  // Fragment coordinates: rows gq, gq+8 (tokens for S^T, d for O^T), columns c0, c0+1 (heads).
   const uint32_t gq = lane >> 2, c0 = (lane & 3) * 2;
-  uint32_t qb[NH][8][2];      // q^T as the B operand: k = d, n = head
-  float o[NH][8][4];          // O^T: 8 tiles of 16 d, columns = heads
-  float m_run[NH][2], l_run[NH][2];
-  uint32_t stage = 0, phase = 0;
-  for (;;) {
-    mbar_wait(&full_bar[stage], phase, status);
-    const uint4 mt = meta[stage];
-    const uint32_t flags = mt.w & 0xFFu;
-    if (flags & kAStop) break;
-    if (flags & kAFirst) {
-      // the item's query rows sit in the slot of its first stage, ours until we release it
-      const uint8_t* qs = q_sm + (size_t)stage * q_slot_bytes;
+  const uint32_t n_warps = gridDim.x * kAttnWarps;
+  const uint32_t per_head = p.B * p.max_splits;
+  uint32_t phase_mask = 0;                       // bit s = phase to wait for on stage s
+  uint32_t id = blockIdx.x * kAttnWarps + warp;  // first item by position, later ones from the counter
+
+  while (id < p.n_items) {
+    const uint32_t g = p.Hkv - 1 - id / per_head;     // host-resident heads first
+    const uint32_t b = (id % per_head) / p.max_splits;
+    const uint32_t split = id % p.max_splits;
+    const uint32_t ctx = (uint32_t)max(p.ctx_lens[b], 0);
+    const uint32_t n_blk = (ctx + kTok - 1) / kTok;
+    const uint32_t n_splits = n_blk ? (n_blk + kItemBlocks - 1) / kItemBlocks : 1;
+    if (split < n_splits) {
+      const uint32_t blk0 = split * kItemBlocks;
+      const uint32_t nb = min(kItemBlocks, n_blk - min(n_blk, blk0));
+      // every lane resolves one block of the item: table entry, page, addresses
+      const uint8_t* ksrc = nullptr;
+      const uint8_t* vsrc = nullptr;
+      uint32_t host_bit = 0;
+      if (lane < nb) {
+        int32_t blk = p.block_table[(size_t)b * p.max_blocks + blk0 + lane];
+        if (blk < 0 || (uint32_t)blk >= p.n_pool_blocks) {   // bad table entry: record, read block 0
+          atomicOr(status, kErrBadIndex);
+          blk = 0;
+        }
+        const uint32_t lin = g * p.n_pool_blocks + (uint32_t)blk;
+        const uint32_t page = lin / kChunksPerPage;
+        const size_t in_page = (size_t)(lin % kChunksPerPage) * kChunkBytes;
+        ksrc = static_cast<const uint8_t*>(p.k_page_ptr[page]) + in_page;
+        vsrc = static_cast<const uint8_t*>(p.v_page_ptr[page]) + in_page;
+        host_bit = page >= p.first_host_page ? 1u : 0u;
+      }
+      // request block i of the item into stage i % kWarpStages
+      auto request = [&](uint32_t i) {
+        const uint32_t st = i % kWarpStages;
+        const uint8_t* ks = reinterpret_cast<const uint8_t*>(__shfl_sync(0xFFFFFFFFu, (unsigned long long)ksrc, i));
+        const uint8_t* vs = reinterpret_cast<const uint8_t*>(__shfl_sync(0xFFFFFFFFu, (unsigned long long)vsrc, i));
+        const bool from_host = __shfl_sync(0xFFFFFFFFu, host_bit, i) != 0;
+        uint8_t* kdst = ring + (size_t)st * kStageBytes;
+        uint8_t* vdst = kdst + kChunkBytes;
+        if (lane == 0) {
+          mbar_arrive_expect_tx(&full_bar[warp][st], from_host ? 0u : kStageBytes);
+          if (!from_host) {
+            bulk_copy_g2s(kdst, ks, kChunkBytes, &full_bar[warp][st]);
+            bulk_copy_g2s(vdst, vs, kChunkBytes, &full_bar[warp][st]);
+          }
+        }
+        if (from_host) {
+          // host page: a fan of 16-byte loads through the load/store path (Sec. 3.2)
+#pragma unroll
+          for (uint32_t c = lane; c < kChunkBytes / 16; c += 32) {
+            cp_async_16(kdst + c * 16, ks + c * 16, 16u);
+            cp_async_16(vdst + c * 16, vs + c * 16, 16u);
+          }
+        }
+        cp_async_arrive_noinc(&full_bar[warp][st]);
+      };
+      for (uint32_t i = 0; i < min(nb, kWarpStages); ++i) request(i);
+
+      // q^T as the B operand (k = d, n = head), straight from global while the blocks fly
+      uint32_t qb[NH][8][2];
+      float o[NH][8][4];          // O^T: 8 tiles of 16 d, columns = heads
+      float m_run[NH][2], l_run[NH][2];
 #pragma unroll
       for (int nh = 0; nh < NH; ++nh) {
         const uint32_t head = nh * 8 + gq;
+        const uint8_t* qs = reinterpret_cast<const uint8_t*>(p.q + ((size_t)b * p.Hq + g * p.group + head) * kD);
 #pragma unroll
         for (uint32_t ks = 0; ks < 8; ++ks) {
-          const uint8_t* src = qs + head * kQRowStride + (ks * 16 + c0) * 2;
-          qb[nh][ks][0] = head < p.group ? *reinterpret_cast<const uint32_t*>(src) : 0u;
-          qb[nh][ks][1] = head < p.group ? *reinterpret_cast<const uint32_t*>(src + 16) : 0u;
+          qb[nh][ks][0] = head < p.group ? *reinterpret_cast<const uint32_t*>(qs + (ks * 16 + c0) * 2) : 0u;
+          qb[nh][ks][1] = head < p.group ? *reinterpret_cast<const uint32_t*>(qs + (ks * 16 + c0) * 2 + 16) : 0u;
         }
 #pragma unroll
         for (int i = 0; i < 8; ++i) { o[nh][i][0] = o[nh][i][1] = o[nh][i][2] = o[nh][i][3] = 0.f; }
         m_run[nh][0] = m_run[nh][1] = -CUDART_INF_F;
         l_run[nh][0] = l_run[nh][1] = 0.f;
       }
-    }
-    const uint32_t b = mt.x, g = mt.y & 0xFFFFu, split = mt.y >> 16;
-    const uint32_t ctx = meta_ctx[stage];
-    if (!(flags & kANoData) && ((mt.w >> 16) & 3u) == warp) {
-      const uint32_t kbase = smem_u32(stage_sm + (size_t)stage * kStageBytes);
-      const uint32_t vbase = kbase + kChunkBytes;
-      const uint32_t tok = (lane & 7) + ((lane >> 4) << 3);     // ldmatrix row of this lane
-      const uint32_t sub = (lane >> 3) & 1;                     // which 16-byte chunk of a pair
-      // S^T = K q^T: rows = 16 tokens, columns = heads
-      float s[NH][4], s2[NH][4];   // two accumulation chains, added at the end
+
+      for (uint32_t i = 0; i < nb; ++i) {
+        const uint32_t st = i % kWarpStages;
+        mbar_wait(&full_bar[warp][st], (phase_mask >> st) & 1u, status);
+        phase_mask ^= 1u << st;
+        const uint32_t kbase = smem_u32(ring + (size_t)st * kStageBytes);
+        const uint32_t vbase = kbase + kChunkBytes;
+        const uint32_t tok = (lane & 7) + ((lane >> 4) << 3);     // ldmatrix row of this lane (V^T)
+        const uint32_t sub = (lane >> 3) & 1;                     // which 16-byte chunk of a pair
+        // S^T = K q^T: rows = 16 tokens, columns = heads; two accumulation chains
+        float s[NH][4], s2[NH][4];
 #pragma unroll
-      for (int nh = 0; nh < NH; ++nh) {
-        s[nh][0] = s[nh][1] = s[nh][2] = s[nh][3] = 0.f;
-        s2[nh][0] = s2[nh][1] = s2[nh][2] = s2[nh][3] = 0.f;
+        for (int nh = 0; nh < NH; ++nh) {
+          s[nh][0] = s[nh][1] = s[nh][2] = s[nh][3] = 0.f;
+          s2[nh][0] = s2[nh][1] = s2[nh][2] = s2[nh][3] = 0.f;
+        }
+#pragma unroll
+        for (uint32_t ks = 0; ks < 8; ++ks) {
+          // A fragment of K: m0 tokens 0-7 / chunk 2ks, m1 tokens 8-15 / chunk 2ks, m2, m3 chunk 2ks+1
+          const uint32_t a_tok = (lane & 7) + (((lane >> 3) & 1) << 3);
+          const uint32_t a_chunk = 2 * ks + (lane >> 4);
+          uint32_t a[4];
+          ldmatrix_x4(a[0], a[1], a[2], a[3], kbase + a_tok * 256 + ((a_chunk ^ (a_tok & 7)) << 4));
+#pragma unroll
+          for (int nh = 0; nh < NH; ++nh) mma_bf16_16816((ks & 1) ? s2[nh] : s[nh], a, qb[nh][ks][0], qb[nh][ks][1]);
+        }
+        // mask the tail of the last block, scale into the log2 domain; online softmax per head
+        const uint32_t t_lo = (blk0 + i) * kTok + gq, t_hi = t_lo + 8;
+        uint32_t pa[NH][3][2];
+#pragma unroll
+        for (int nh = 0; nh < NH; ++nh) {
+          float pf[4];
+#pragma unroll
+          for (int r = 0; r < 4; ++r) {
+            const uint32_t t = (r & 2) ? t_hi : t_lo;
+            const float v = s[nh][r] + s2[nh][r];
+            s[nh][r] = (t < ctx) ? v * p.scale_log2e : -CUDART_INF_F;
+          }
+#pragma unroll
+          for (int h = 0; h < 2; ++h) {
+            float mx = fmaxf(s[nh][h], s[nh][2 + h]);
+            mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, 4));
+            mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, 8));
+            mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, 16));
+            const float m_new = fmaxf(m_run[nh][h], mx);      // finite: a block has a valid token
+            const float corr = exp2f(m_run[nh][h] - m_new);   // exp2(-inf) = 0 on the first block
+            pf[h] = exp2f(s[nh][h] - m_new);
+            pf[2 + h] = exp2f(s[nh][2 + h] - m_new);
+            float sum = pf[h] + pf[2 + h];
+            sum += __shfl_xor_sync(0xFFFFFFFFu, sum, 4);
+            sum += __shfl_xor_sync(0xFFFFFFFFu, sum, 8);
+            sum += __shfl_xor_sync(0xFFFFFFFFu, sum, 16);
+            l_run[nh][h] = l_run[nh][h] * corr + sum;
+            m_run[nh][h] = m_new;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) { o[nh][j][h] *= corr; o[nh][j][2 + h] *= corr; }
+          }
+          // P^T as the B operand (k = token, n = head).  A single bf16 rounding of P would put
+          // an error of 2^-9 * sqrt(sum p^2 v^2) on every output, far above 1 % of the outputs
+          // that are close to zero; P is split into three bf16 terms (24 bits) multiplied term
+          // by term.  The accumulator layout (token rows) becomes the operand layout (token as
+          // k) by an 8x8 transpose across the warp.
+          float x0 = pf[0], x1 = pf[1], x2 = pf[2], x3 = pf[3];
+#pragma unroll
+          for (int t = 0; t < 3; ++t) {
+            const __nv_bfloat162 lo = __floats2bfloat162_rn(x0, x1), hi = __floats2bfloat162_rn(x2, x3);
+            pa[nh][t][0] = movmatrix_trans(*reinterpret_cast<const uint32_t*>(&lo));   // tokens 0-7
+            pa[nh][t][1] = movmatrix_trans(*reinterpret_cast<const uint32_t*>(&hi));   // tokens 8-15
+            x0 -= __low2float(lo); x1 -= __high2float(lo);
+            x2 -= __low2float(hi); x3 -= __high2float(hi);
+          }
+        }
+        // O^T += V^T P^T: rows = d (8 tiles of 16), k = 16 tokens
+#pragma unroll
+        for (uint32_t dt = 0; dt < 8; ++dt) {
+          // A fragment of V^T: m0 d-chunk 2dt / tokens 0-7, m1 chunk 2dt+1 / tokens 0-7, m2, m3 tokens 8-15
+          const uint32_t chunk = 2 * dt + sub;
+          uint32_t a[4];
+          ldmatrix_x4_trans(a[0], a[1], a[2], a[3], vbase + tok * 256 + ((chunk ^ (tok & 7)) << 4));
+#pragma unroll
+          for (int nh = 0; nh < NH; ++nh)
+#pragma unroll
+            for (int t = 2; t >= 0; --t) mma_bf16_16816(o[nh][dt], a, pa[nh][t][0], pa[nh][t][1]);
+        }
+        __syncwarp();   // every lane is done with this stage before it is refilled
+        if (i + kWarpStages < nb) request(i + kWarpStages);
       }
-#pragma unroll
-      for (uint32_t ks = 0; ks < 8; ++ks) {
-        // A fragment of K: m0 tokens 0-7 / chunk 2ks, m1 tokens 8-15 / chunk 2ks, m2, m3 chunk 2ks+1
-        const uint32_t a_tok = (lane & 7) + (((lane >> 3) & 1) << 3);
-        const uint32_t a_chunk = 2 * ks + (lane >> 4);
-        uint32_t a[4];
-        ldmatrix_x4(a[0], a[1], a[2], a[3], kbase + a_tok * 256 + ((a_chunk ^ (a_tok & 7)) << 4));
-#pragma unroll
-        for (int nh = 0; nh < NH; ++nh) mma_bf16_16816((ks & 1) ? s2[nh] : s[nh], a, qb[nh][ks][0], qb[nh][ks][1]);
-      }
+
+      // ---- end of the item: this warp holds the whole chunk run
+      const bool single = (n_splits == 1);
 #pragma unroll
       for (int nh = 0; nh < NH; ++nh)
 #pragma unroll
-        for (int r = 0; r < 4; ++r) s[nh][r] += s2[nh][r];
-      // mask the tail of the last block, scale into the log2 domain; online softmax per head
-      const uint32_t t_lo = mt.z + gq, t_hi = t_lo + 8;
-      uint32_t pa[NH][3][2];
-#pragma unroll
-      for (int nh = 0; nh < NH; ++nh) {
-        float pf[4];
-#pragma unroll
-        for (int r = 0; r < 4; ++r) {
-          const uint32_t t = (r & 2) ? t_hi : t_lo;
-          s[nh][r] = (t < ctx) ? s[nh][r] * p.scale_log2e : -CUDART_INF_F;
-        }
-#pragma unroll
         for (int h = 0; h < 2; ++h) {
-          float mx = fmaxf(s[nh][h], s[nh][2 + h]);
-          mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, 4));
-          mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, 8));
-          mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, 16));
-          const float m_new = fmaxf(m_run[nh][h], mx);      // finite: a block has a valid token
-          const float corr = exp2f(m_run[nh][h] - m_new);   // exp2(-inf) = 0 on the first block
-          pf[h] = exp2f(s[nh][h] - m_new);
-          pf[2 + h] = exp2f(s[nh][2 + h] - m_new);
-          float sum = pf[h] + pf[2 + h];
-          sum += __shfl_xor_sync(0xFFFFFFFFu, sum, 4);
-          sum += __shfl_xor_sync(0xFFFFFFFFu, sum, 8);
-          sum += __shfl_xor_sync(0xFFFFFFFFu, sum, 16);
-          l_run[nh][h] = l_run[nh][h] * corr + sum;
-          m_run[nh][h] = m_new;
+          const uint32_t head = nh * 8 + c0 + h;
+          if (head >= p.group) continue;
+          const uint32_t hq = g * p.group + head;
+          if (single) {
+            const float inv = l_run[nh][h] > 0.f ? 1.f / l_run[nh][h] : 0.f;
+            __nv_bfloat16* dst = p.out + ((size_t)b * p.Hq + hq) * kD;
 #pragma unroll
-          for (int i = 0; i < 8; ++i) { o[nh][i][h] *= corr; o[nh][i][2 + h] *= corr; }
-        }
-        // P^T as the B operand (k = token, n = head).  A single bf16 rounding of P would put
-        // an error of 2^-9 * sqrt(sum p^2 v^2) on every output, far above 1 % of the outputs
-        // that are close to zero; P is split into three bf16 terms (24 bits) multiplied term by
-        // term.  The accumulator layout (token rows) is turned into the operand layout (token
-        // as k) by an 8x8 transpose across the warp.
-        float x0 = pf[0], x1 = pf[1], x2 = pf[2], x3 = pf[3];
+            for (int j = 0; j < 8; ++j) {
+              dst[j * 16 + gq] = __float2bfloat16_rn(o[nh][j][h] * inv);
+              dst[j * 16 + gq + 8] = __float2bfloat16_rn(o[nh][j][2 + h] * inv);
+            }
+          } else {
+            const size_t slot = ((size_t)b * p.Hq + hq) * p.max_splits + split;
+            float* dst = p.part_o + slot * kD;
 #pragma unroll
-        for (int t = 0; t < 3; ++t) {
-          const __nv_bfloat162 lo = __floats2bfloat162_rn(x0, x1), hi = __floats2bfloat162_rn(x2, x3);
-          pa[nh][t][0] = movmatrix_trans(*reinterpret_cast<const uint32_t*>(&lo));   // tokens 0-7
-          pa[nh][t][1] = movmatrix_trans(*reinterpret_cast<const uint32_t*>(&hi));   // tokens 8-15
-          x0 -= __low2float(lo); x1 -= __high2float(lo);
-          x2 -= __low2float(hi); x3 -= __high2float(hi);
-        }
-      }
-      // O^T += V^T P^T: rows = d (8 tiles of 16), k = 16 tokens
-#pragma unroll
-      for (uint32_t dt = 0; dt < 8; ++dt) {
-        // A fragment of V^T: m0 d-chunk 2dt / tokens 0-7, m1 chunk 2dt+1 / tokens 0-7, m2, m3 tokens 8-15
-        const uint32_t chunk = 2 * dt + sub;
-        uint32_t a[4];
-        ldmatrix_x4_trans(a[0], a[1], a[2], a[3], vbase + tok * 256 + ((chunk ^ (tok & 7)) << 4));
-#pragma unroll
-        for (int nh = 0; nh < NH; ++nh)
-#pragma unroll
-          for (int t = 2; t >= 0; --t) mma_bf16_16816(o[nh][dt], a, pa[nh][t][0], pa[nh][t][1]);
-      }
-    }
-    __syncwarp();
-    if (lane == 0) mbar_arrive(&empty_bar[stage]);
-    if (++stage == n_stages) { stage = 0; phase ^= 1u; }
-    if (!(flags & kALast)) continue;
-
-    // ---- end of the item: merge the warps (disjoint sets of blocks) through shared memory
-#pragma unroll
-    for (int nh = 0; nh < NH; ++nh)
-#pragma unroll
-      for (int h = 0; h < 2; ++h) {
-        const uint32_t head = nh * 8 + c0 + h;
-        if (head < p.group) {
-          if (gq == 0) { merge_ml[warp][head][0] = m_run[nh][h]; merge_ml[warp][head][1] = l_run[nh][h]; }
-          float* dst = merge_o + ((size_t)warp * p.group + head) * kD;
-#pragma unroll
-          for (int i = 0; i < 8; ++i) {
-            dst[i * 16 + gq] = o[nh][i][h];
-            dst[i * 16 + gq + 8] = o[nh][i][2 + h];
+            for (int j = 0; j < 8; ++j) {
+              __stcg(dst + j * 16 + gq, o[nh][j][h]);
+              __stcg(dst + j * 16 + gq + 8, o[nh][j][2 + h]);
+            }
+            if (gq == 0) { __stcg(p.part_ml + slot * 2, m_run[nh][h]); __stcg(p.part_ml + slot * 2 + 1, l_run[nh][h]); }
           }
         }
-      }
-    named_barrier_sync(1, kConsumerThreads);
-
-    const uint32_t n_blk = (ctx + kTok - 1) / kTok;
-    const uint32_t n_splits = n_blk ? (n_blk + kItemBlocks - 1) / kItemBlocks : 1;
-    const bool single = (n_splits == 1);
-    // thread d of 128 owns output column d; loop over the query heads of the group
-    for (uint32_t r = 0; r < p.group; ++r) {
-      float m_all = -CUDART_INF_F;
-#pragma unroll
-      for (uint32_t w = 0; w < kAttnWarps; ++w) m_all = fmaxf(m_all, merge_ml[w][r][0]);
-      float acc = 0.f, l_all = 0.f;
-#pragma unroll
-      for (uint32_t w = 0; w < kAttnWarps; ++w) {
-        const float mw = merge_ml[w][r][0];
-        const float f = (mw == -CUDART_INF_F) ? 0.f : exp2f(mw - m_all);
-        acc += f * merge_o[((size_t)w * p.group + r) * kD + tid];
-        l_all += f * merge_ml[w][r][1];
-      }
-      const uint32_t hq = g * p.group + r;
-      if (single) {
-        const float v = l_all > 0.f ? acc / l_all : 0.f;
-        p.out[((size_t)b * p.Hq + hq) * kD + tid] = __float2bfloat16_rn(v);
-      } else {
-        const size_t slot = ((size_t)b * p.Hq + hq) * p.max_splits + split;
-        __stcg(p.part_o + slot * kD + tid, acc);
-        if (tid == 0) { __stcg(p.part_ml + slot * 2, m_all); __stcg(p.part_ml + slot * 2 + 1, l_all); }
-      }
-    }
-    if (!single) {
-      // the last split of (b, g) to arrive combines all splits, in split order
-      uint32_t* cnt = p.ws + kWsHeaderWords + b * p.Hkv + g;
-      named_barrier_sync(1, kConsumerThreads);
-      if (tid == 0) {
-        __threadfence();   // cumulative: publishes the partials of all 128 threads (ordered by the barrier)
-        s_old = atomicAdd(cnt, 1u);
-      }
-      named_barrier_sync(1, kConsumerThreads);
-      if (s_old == n_splits - 1) {
-        __threadfence();
-        for (uint32_t r = 0; r < p.group; ++r) {
-          const uint32_t hq = g * p.group + r;
-          const size_t slot0 = ((size_t)b * p.Hq + hq) * p.max_splits;
-          float m_all = -CUDART_INF_F;
-          for (uint32_t sp = 0; sp < n_splits; ++sp) m_all = fmaxf(m_all, __ldcg(p.part_ml + (slot0 + sp) * 2));
-          float acc = 0.f, l_all = 0.f;
-          for (uint32_t sp = 0; sp < n_splits; ++sp) {
-            const float ms = __ldcg(p.part_ml + (slot0 + sp) * 2);
-            const float f = (ms == -CUDART_INF_F) ? 0.f : exp2f(ms - m_all);
-            acc += f * __ldcg(p.part_o + (slot0 + sp) * kD + tid);
-            l_all += f * __ldcg(p.part_ml + (slot0 + sp) * 2 + 1);
-          }
-          p.out[((size_t)b * p.Hq + hq) * kD + tid] = __float2bfloat16_rn(l_all > 0.f ? acc / l_all : 0.f);
+      if (!single) {
+        // the last split of (b, g) to arrive combines all splits, in split order
+        uint32_t* cnt = p.ws + kWsHeaderWords + b * p.Hkv + g;
+        __syncwarp();
+        uint32_t old = 0;
+        if (lane == 0) {
+          __threadfence();   // cumulative: publishes the partials of the whole warp
+          old = atomicAdd(cnt, 1u);
         }
-        if (tid == 0) *cnt = 0;
+        old = __shfl_sync(0xFFFFFFFFu, old, 0);
+        if (old == n_splits - 1) {
+          __threadfence();
+          for (uint32_t r = 0; r < p.group; ++r) {
+            const uint32_t hq = g * p.group + r;
+            const size_t slot0 = ((size_t)b * p.Hq + hq) * p.max_splits;
+            float m_all = -CUDART_INF_F;
+            for (uint32_t sp = 0; sp < n_splits; ++sp) m_all = fmaxf(m_all, __ldcg(p.part_ml + (slot0 + sp) * 2));
+            float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+            float l_all = 0.f;
+            for (uint32_t sp = 0; sp < n_splits; ++sp) {
+              const float ms = __ldcg(p.part_ml + (slot0 + sp) * 2);
+              const float f = (ms == -CUDART_INF_F) ? 0.f : exp2f(ms - m_all);
+              const float4 v = __ldcg(reinterpret_cast<const float4*>(p.part_o + (slot0 + sp) * kD) + lane);
+              acc.x += f * v.x; acc.y += f * v.y; acc.z += f * v.z; acc.w += f * v.w;
+              l_all += f * __ldcg(p.part_ml + (slot0 + sp) * 2 + 1);
+            }
+            const float inv = l_all > 0.f ? 1.f / l_all : 0.f;
+            const __nv_bfloat162 lo = __floats2bfloat162_rn(acc.x * inv, acc.y * inv);
+            const __nv_bfloat162 hi = __floats2bfloat162_rn(acc.z * inv, acc.w * inv);
+            uint2 ov;
+            ov.x = *reinterpret_cast<const uint32_t*>(&lo);
+            ov.y = *reinterpret_cast<const uint32_t*>(&hi);
+            *reinterpret_cast<uint2*>(p.out + ((size_t)b * p.Hq + hq) * kD + lane * 4) = ov;
+          }
+          if (lane == 0) *cnt = 0;
+        }
       }
     }
-    named_barrier_sync(1, kConsumerThreads);   // the merge buffers are free again
+    uint32_t nxt = 0;
+    if (lane == 0) nxt = n_warps + atomicAdd(p.ws + kWsHbmNext, 1u);
+    id = __shfl_sync(0xFFFFFFFFu, nxt, 0);
+  }
+  // the last warp out resets the counters for the next launch
+  if (lane == 0) {
+    __threadfence();
+    const uint32_t d = atomicAdd(p.ws + kWsDone, 1u);
+    if (d == n_warps - 1) { p.ws[kWsHbmNext] = 0; p.ws[kWsDone] = 0; __threadfence(); }
   }
 }
 
@@ -488,24 +427,19 @@ extern "C" int boost_paged_attn_decode_tiered(const void* q, const void* const* 
   p.part_ml = reinterpret_cast<float*>(base);
   p.part_o = p.part_ml + (size_t)B * Hq * p.max_splits * 2;
   p.out = static_cast<__nv_bfloat16*>(out);
-  const size_t fixed = (size_t)kAttnWarps * p.group * kD * 4 + 128;
-  const uint32_t budget = p.group <= 8 ? kAttnSmemBudget3 : kAttnSmemBudget2;
-  uint32_t n_stages = (uint32_t)((budget - fixed) / (kStageBytes + p.group * kQRowStride));
-  if (n_stages > kMaxStages) n_stages = kMaxStages;
-  p.n_stages = n_stages;
-  const size_t smem = (size_t)n_stages * (kStageBytes + p.group * kQRowStride) + fixed;
+  const size_t smem = (size_t)kAttnWarps * kWarpStages * kStageBytes + 128;
   static bool configured = false;
   if (!configured) {
-    int rc = boosth::check(cudaFuncSetAttribute(paged_attn_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kAttnSmemBudget2));
+    int rc = boosth::check(cudaFuncSetAttribute(paged_attn_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     if (rc == BOOST_OK)
-      rc = boosth::check(cudaFuncSetAttribute(paged_attn_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kAttnSmemBudget2));
+      rc = boosth::check(cudaFuncSetAttribute(paged_attn_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     if (rc != BOOST_OK) return rc;
     configured = true;
   }
   const int sms = boosth::sm_count();
   if (sms <= 0) return BOOST_ERR_CUDA;
   uint32_t grid = (uint32_t)sms * (p.group <= 8 ? 3 : 2);
-  if (grid > p.n_items) grid = p.n_items;
+  if (grid * kAttnWarps > p.n_items) grid = (p.n_items + kAttnWarps - 1) / kAttnWarps;
   if (p.group <= 8)
     return boosth::launch_chained(paged_attn_kernel<1>, dim3(grid), dim3(kAttnThreads), smem, (cudaStream_t)stream, p);
   return boosth::launch_chained(paged_attn_kernel<2>, dim3(grid), dim3(kAttnThreads), smem, (cudaStream_t)stream, p);
