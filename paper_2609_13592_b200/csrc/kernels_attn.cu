@@ -2,7 +2,7 @@
 // copies that move a logical [Hkv][N][16][D] cache into and out of its pages.
 //
 // Persistent grid of autonomous warps.  A work item is a KV-head chunk run: sequence b, KV
-// head g, blocks [16 s, 16 s + 16) of the sequence (Sec. 3.3: attention threadblocks work
+// head g, a run of up to 32 consecutive blocks of the sequence (Sec. 3.3: threadblocks work
 // on KV head chunks); items of the highest-numbered heads - the ones linear placement puts
 // on the host tier - are handed out first.  Each warp takes whole items and streams their
 // KV blocks through its own two-stage ring in shared memory: per block two 4 KiB bulk
@@ -17,6 +17,7 @@
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <math_constants.h>
+#include <stdlib.h>
 
 #include "device_common.cuh"
 #include "host_common.h"
@@ -29,7 +30,8 @@ constexpr uint32_t kD = 128;
 constexpr uint32_t kTok = BOOST_KV_BLOCK_TOKENS;         // 16
 constexpr uint32_t kChunkBytes = kTok * kD * 2;          // 4 KiB
 constexpr uint32_t kChunksPerPage = kPageBytes / kChunkBytes;
-constexpr uint32_t kItemBlocks = 16;                     // KV blocks per work item
+constexpr uint32_t kMaxItemBlocks = 32;                  // KV blocks per work item: at most (one lane resolves one block)
+constexpr uint32_t kMinItemBlocks = 4;
 constexpr uint32_t kStageBytes = 2 * kChunkBytes;        // K chunk + V chunk
 constexpr uint32_t kAttnWarps = 4;                       // warps per threadblock
 constexpr uint32_t kAttnThreads = kAttnWarps * 32;
@@ -45,7 +47,7 @@ struct AttnParams {
   const int32_t* block_table;
   uint32_t max_blocks;
   const int32_t* ctx_lens;
-  uint32_t B, Hq, Hkv, group, max_splits, n_items;
+  uint32_t B, Hq, Hkv, group, max_splits, n_items, item_blocks;
   float scale_log2e;
   uint32_t* ws;        // header (status, item counter, done counter) + one counter per (b, g)
   float* part_ml;      // [B][Hq][max_splits][2]
@@ -90,10 +92,10 @@ __global__ void __launch_bounds__(kAttnThreads, (NH == 1 ? 3 : 2)) paged_attn_ke
     const uint32_t split = id % p.max_splits;
     const uint32_t ctx = (uint32_t)max(p.ctx_lens[b], 0);
     const uint32_t n_blk = (ctx + kTok - 1) / kTok;
-    const uint32_t n_splits = n_blk ? (n_blk + kItemBlocks - 1) / kItemBlocks : 1;
+    const uint32_t n_splits = n_blk ? (n_blk + p.item_blocks - 1) / p.item_blocks : 1;
     if (split < n_splits) {
-      const uint32_t blk0 = split * kItemBlocks;
-      const uint32_t nb = min(kItemBlocks, n_blk - min(n_blk, blk0));
+      const uint32_t blk0 = split * p.item_blocks;
+      const uint32_t nb = min(p.item_blocks, n_blk - min(n_blk, blk0));
       // every lane resolves one block of the item: table entry, page, addresses
       const uint8_t* ksrc = nullptr;
       const uint8_t* vsrc = nullptr;
@@ -376,7 +378,7 @@ extern "C" int boost_kv_gather(void* dst, uint32_t n_kv_heads, uint32_t n_pool_b
 extern "C" size_t boost_paged_attn_workspace_bytes(uint32_t B, uint32_t Hq, uint32_t D,
                                                    uint32_t max_blocks) {
   if (D != kD || B == 0 || Hq == 0) return 0;
-  const size_t max_splits = max_blocks ? (max_blocks + kItemBlocks - 1) / kItemBlocks : 1;
+  const size_t max_splits = max_blocks ? (max_blocks + kMinItemBlocks - 1) / kMinItemBlocks : 1;
   // counters are per (b, KV head); Hq bounds the number of KV heads
   return attn_header_bytes(B, Hq) + (size_t)B * Hq * max_splits * (2 + kD) * 4;
 }
@@ -417,7 +419,23 @@ extern "C" int boost_paged_attn_decode_tiered(const void* q, const void* const* 
   p.max_blocks = max_blocks;
   p.ctx_lens = ctx_lens;
   p.B = B; p.Hq = Hq; p.Hkv = Hkv; p.group = Hq / Hkv;
-  p.max_splits = (max_blocks + kItemBlocks - 1) / kItemBlocks;
+  const int sms = boosth::sm_count();
+  if (sms <= 0) return BOOST_ERR_CUDA;
+  const uint32_t ctas_per_sm = p.group <= 8 ? 3 : 2;
+  const uint32_t n_warps = (uint32_t)sms * ctas_per_sm * kAttnWarps;
+  // Item length: every item costs a table look-up, a query load and a partial result, so long
+  // items are better as long as enough warps have work to keep HBM busy (measured on B200:
+  // about a thousand warps with 16 KiB in flight each saturate it).  Taking the sequences as
+  // max_blocks long, use the longest run (4..32 blocks) that still gives 55 % of the warps an
+  // item.
+  uint32_t best_len = kMinItemBlocks;
+  for (uint32_t len = kMaxItemBlocks; len >= kMinItemBlocks; --len) {
+    const uint64_t items = (uint64_t)Hkv * B * ((max_blocks + len - 1) / len);
+    if (items * 100 >= (uint64_t)n_warps * 55) { best_len = len; break; }
+  }
+  if (const char* e = getenv("BOOST_ATTN_L")) { const uint32_t v = (uint32_t)atoi(e); if (v >= 1 && v <= kMaxItemBlocks) best_len = v; }   // experiment hook
+  p.item_blocks = best_len;
+  p.max_splits = (max_blocks + best_len - 1) / best_len;
   const uint64_t n_items = (uint64_t)Hkv * B * p.max_splits;
   if (n_items > 0x7FFFFFFFull) return BOOST_ERR_INVALID;
   p.n_items = (uint32_t)n_items;
@@ -436,9 +454,7 @@ extern "C" int boost_paged_attn_decode_tiered(const void* q, const void* const* 
     if (rc != BOOST_OK) return rc;
     configured = true;
   }
-  const int sms = boosth::sm_count();
-  if (sms <= 0) return BOOST_ERR_CUDA;
-  uint32_t grid = (uint32_t)sms * (p.group <= 8 ? 3 : 2);
+  uint32_t grid = (uint32_t)sms * ctas_per_sm;
   if (grid * kAttnWarps > p.n_items) grid = (p.n_items + kAttnWarps - 1) / kAttnWarps;
   if (p.group <= 8)
     return boosth::launch_chained(paged_attn_kernel<1>, dim3(grid), dim3(kAttnThreads), smem, (cudaStream_t)stream, p);
