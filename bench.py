@@ -317,6 +317,19 @@ def timed_host_steps(dec, dev, batch, ctx0, warmup, steps, max_blocks, dist_ctx)
     return ms, h2d, d2h
 
 
+def aggregate_replicas(ms, dist, device):
+    """Slowest rank's time: MAX all-reduce over the ranks (each rank ran its own replica)."""
+    import torch
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def replica_job_value(batch, world, ms_per_step):
+    """Whole-job decode tokens/s of `world` independent replicas of `batch` sequences."""
+    return world * batch / (ms_per_step / 1e3)
+
+
 class DistCtx:
     def __init__(self, rank, world, dev):
         self.rank, self.world, self.dev = rank, world, dev
@@ -333,10 +346,7 @@ class DistCtx:
     def max(self, x):
         if self.dist is None:
             return x
-        import torch
-        t = torch.tensor([x], dtype=torch.float64, device=self.dev)
-        self.dist.all_reduce(t, op=self.dist.ReduceOp.MAX)
-        return float(t.item())
+        return aggregate_replicas(x, self.dist, self.dev)
 
     def close(self):
         if self.dist is not None:
@@ -360,7 +370,8 @@ def run_ours(args, rank, world, local_rank):
     # host-link and HBM read bandwidth of this machine, measured in this run with the same kernel
     link_gbs = measure_stream(dev, 64, 1)            # 128 MiB of host-mapped pinned pages
     hbm_read_gbs = measure_stream(dev, 1024, 0)      # 2 GiB in HBM
-    modulus = B.boost_modulus_from_bandwidths(hbm_peak, link_gbs)
+    # K = HBM read bandwidth / link bandwidth, both measured with the same kernel in this run
+    modulus = B.boost_modulus_from_bandwidths(max(hbm_read_gbs, hbm_peak), link_gbs)
     host_ratio = 1.0 / modulus
 
     cfg = dict(synth.LLAMA3_8B)
@@ -396,7 +407,7 @@ def run_ours(args, rank, world, local_rank):
     if rank == 0:
         t = results["tiered"]
         ms_step = t["ms"] / args.steps
-        value = world * batch / (ms_step / 1e3)
+        value = replica_job_value(batch, world, ms_step)
         bytes_step = t["weight_bytes"] + t["kv_tokens"] / args.steps * t["kv_bytes_per_token"]
         combined = bytes_step / (ms_step / 1e3) / 1e9
         roof = hbm_peak + link_gbs
@@ -453,6 +464,63 @@ def run_ours(args, rank, world, local_rank):
     dist_ctx.close()
 
 
+def run_stream_sweep(args):
+    """Configuration 3: tiered streaming-read sweep.  A bf16 buffer of 1 / 4 / 16 (/ 64) GiB is
+    reduced by the stream-reduce kernel (full waves of 4 threadblocks per SM) with the host
+    share in {0, 1/256, ..., 1/8} under modulo, contiguous and random placement.  Prints one
+    JSON document with combined GB/s and the per-wave host-share statistics of each point."""
+    import torch
+    from paper_2609_13592_b200 import binding as B
+    from paper_2609_13592_b200 import build as libbuild
+    from paper_2609_13592_b200.tiers import Slabs, TieredBuffer
+    libbuild.build_library()
+    dev = torch.device("cuda:0")
+    torch.cuda.set_device(dev)
+    hbm_peak, peak_src = load_peaks()
+    link = measure_stream(dev, 64, 1)
+    sms = torch.cuda.get_device_properties(dev).multi_processor_count
+    ratios = [0.0, 1 / 256, 1 / 128, 1 / 64, 1 / 32, 1 / 16, 1 / 8]
+    policies = [("modulo", B.POLICY_MODULO), ("contiguous", B.POLICY_CONTIGUOUS), ("random", B.POLICY_RANDOM)]
+    sizes = [int(x) for x in args.sweep_gib.split(",")]
+    points = []
+    for gib in sizes:
+        n_pages = gib * 512
+        slabs = Slabs(n_pages, n_pages // 8 + n_pages // 32 + 8, dev)
+        ws_bytes = B.boost_stream_reduce_workspace_bytes(n_pages)
+        ws = torch.zeros(ws_bytes, dtype=torch.uint8, device=dev)
+        sums = torch.zeros(n_pages, dtype=torch.float32, device=dev)
+        for ratio in ratios:
+            for name, pol in policies:
+                seeds = range(args.sweep_seeds) if (pol == B.POLICY_RANDOM and ratio > 0) else [0]
+                gbs, var = [], []
+                n_host = 0
+                for seed in seeds:
+                    buf = TieredBuffer(n_pages * B.PAGE_BYTES, ratio, pol, seed=seed, device=dev, slabs=slabs)
+                    n_host = buf.n_host
+                    st = B.boost_wave_stats(buf.tier, 128 * 1024, sms * 4, ratio)
+                    best = float("inf")
+                    for i in range(5):
+                        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                        e0.record()
+                        B.boost_stream_reduce_tiered(buf.page_ptr, buf.order, n_pages, buf.n_host, sums, ws, ws_bytes)
+                        e1.record()
+                        torch.cuda.synchronize(dev)
+                        if i >= 1:
+                            best = min(best, e0.elapsed_time(e1))
+                    gbs.append(n_pages * B.PAGE_BYTES / best / 1e6)
+                    var.append(st["var"])
+                    del buf
+                bound = min(hbm_peak + link, link / ratio * 1.0) if ratio > 0 else hbm_peak
+                points.append({"gib": gib, "host_ratio": ratio, "placement": name, "host_pages": n_host,
+                               "combined_gbs": float(np.mean(gbs)), "gbs_min": float(min(gbs)),
+                               "gbs_max": float(max(gbs)), "wave_host_share_var": float(np.mean(var)),
+                               "tier_bound_gbs": bound, "seeds": len(list(seeds))})
+        del slabs, ws, sums
+        torch.cuda.empty_cache()
+    print(json.dumps({"workload": "c3_tiered_stream_sweep", "hbm_peak_gbs": hbm_peak, "hbm_peak_source": peak_src,
+                      "host_link_gbs": link, "combined_roofline_gbs": hbm_peak + link, "points": points}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -463,12 +531,19 @@ def main():
     ap.add_argument("--ctx", type=int, default=2048)
     ap.add_argument("--layers", type=int, default=0, help="override the layer count (0 = 32)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--workload", default="decode", choices=["decode", "stream_sweep"],
+                    help="decode: the benchmark line; stream_sweep: the placement sweep of configuration 3")
+    ap.add_argument("--sweep-gib", default="1,4,16")
+    ap.add_argument("--sweep-seeds", type=int, default=5)
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    if args.impl == "reference":
+    if args.workload == "stream_sweep":
+        if rank == 0:
+            run_stream_sweep(args)
+    elif args.impl == "reference":
         run_reference(args, rank, world)
     else:
         run_ours(args, rank, world, local_rank)

@@ -19,11 +19,25 @@ def _aligned(t, align=PAGE):
     return (p + align - 1) // align * align
 
 
+class Slabs:
+    """An HBM slab and a pinned host slab that several TieredBuffers may map their pages onto
+    (for placement sweeps, where only the page table changes between runs)."""
+
+    def __init__(self, hbm_pages, host_pages, device="cuda"):
+        self.device = torch.device(device)
+        self.hbm_pages, self.host_pages = hbm_pages, host_pages
+        self._hbm = torch.empty(hbm_pages * PAGE + PAGE, dtype=torch.uint8, device=self.device)
+        self.hbm_base = _aligned(self._hbm)
+        self._host = torch.empty(max(host_pages, 1) * PAGE + PAGE, dtype=torch.uint8, pin_memory=True)
+        self.host_base_cpu = _aligned(self._host)
+        self.host_base = B.boost_host_device_pointer(self.host_base_cpu)
+
+
 class TieredBuffer:
     """A buffer of n_bytes cut into 2 MiB pages placed over HBM and pinned host memory."""
 
     def __init__(self, n_bytes, host_ratio=0.0, policy=B.POLICY_MODULO, seed=0, superpage_pages=1,
-                 device="cuda", tier=None, wave_size=0):
+                 device="cuda", tier=None, wave_size=0, slabs=None):
         self.n_bytes = int(n_bytes)
         self.device = torch.device(device)
         if tier is None:
@@ -35,9 +49,16 @@ class TieredBuffer:
         self.n_pages = int(tier.size)
         self.n_host = int((tier == B.TIER_HOST).sum())
         self.n_hbm = self.n_pages - self.n_host
-        self._hbm = torch.empty(self.n_hbm * PAGE + PAGE, dtype=torch.uint8, device=self.device)
-        self.hbm_base = _aligned(self._hbm)
-        if self.n_host:
+        if slabs is not None:
+            assert self.n_hbm <= slabs.hbm_pages and self.n_host <= slabs.host_pages
+            self._hbm, self.hbm_base = slabs._hbm, slabs.hbm_base
+            self._host, self.host_base_cpu, self.host_base = slabs._host, slabs.host_base_cpu, slabs.host_base
+        else:
+            self._hbm = torch.empty(self.n_hbm * PAGE + PAGE, dtype=torch.uint8, device=self.device)
+            self.hbm_base = _aligned(self._hbm)
+        if slabs is not None:
+            pass
+        elif self.n_host:
             self._host = torch.empty(self.n_host * PAGE + PAGE, dtype=torch.uint8, pin_memory=True)
             self.host_base_cpu = _aligned(self._host)
             self.host_base = B.boost_host_device_pointer(self.host_base_cpu)
