@@ -259,6 +259,17 @@ int boost_weight_layout(uint32_t N, uint32_t K, boost_weight_layout_t* out /*hos
 int boost_pack_weights(const void* w_row_major /*device*/, uint32_t N, uint32_t K,
                        const void* const* w_page_ptr /*device*/, size_t n_pages, void* stream);
 
+/* boost_pack_weights with two load-time transformations that let the small operators of a
+ * decode step disappear into the products (the paper does not discuss those operators):
+ *   row_mode 1  rows 0..63 of packed row tile t are rows [64 t, 64 t + 64) of the first half of
+ *               W and rows 64..127 the same rows of the second half, so that gate row j and up
+ *               row j of a [gate; up] matrix meet in one threadblock (N % 128 == 0);
+ *   col_scale   bf16 [K] or NULL: W[n, k] is multiplied by col_scale[k] and rounded to bf16 -
+ *               an RMSNorm weight folded into the matrix it feeds. */
+int boost_pack_weights_ex(const void* w_row_major /*device*/, uint32_t N, uint32_t K,
+                          const void* const* w_page_ptr /*device*/, size_t n_pages, int row_mode,
+                          const void* col_scale /*device*/, void* stream);
+
 /* y[m, n] = sum_k x[m, k] * W[n, k] (+ residual[m, n]), fp32 accumulation: the
  * weight-streaming product that dominates decode (Sec. 2.1, Sec. 3.1; the two-pointer
  * handwritten matmul of Sec. 3.1 is the closest thing the paper describes).
@@ -277,6 +288,47 @@ int boost_gemv_tiered(const void* const* w_page_ptr /*device*/, const uint32_t* 
                       const void* x /*device*/, uint32_t M_b, void* y /*device*/, int y_dtype,
                       const void* residual /*device*/, void* workspace /*device*/,
                       size_t workspace_bytes, void* stream);
+
+/* Epilogues of boost_gemv_tiered_fused.  All are applied by the threadblock that combines the
+ * split-K partial sums of a row tile, in fixed order. */
+enum {
+  BOOST_EPI_PLAIN = 0,      /* y = acc (* row scale) (+ residual) */
+  BOOST_EPI_SWIGLU = 1,     /* weight packed with row_mode 1 from [gate; up]: y[m, j] =
+                               silu(bf16(gate_j)) * bf16(up_j), y bf16 [M_b, N/2] */
+  BOOST_EPI_ROPE_APPEND = 2 /* N = (Hq + 2 Hkv) * 128, row tile = head: rotate q and k heads
+                               (as boost_rope_kv_append), write q to q_out and k, v into the
+                               paged cache; y is not written */
+};
+
+typedef struct {
+  int mode;
+  /* Row scale rsqrt(sum_t ssq_in[t][m] / K + rms_eps): RMSNorm of x whose weight was folded
+   * into W (boost_pack_weights_ex col_scale).  ssq_in [ssq_in_tiles][ssq_stride] fp32 holds,
+   * per 128-column tile of x, the sum of squares of row m; NULL = no scale. */
+  const float* ssq_in; /* device */
+  uint32_t ssq_in_tiles, ssq_stride;
+  float rms_eps;
+  /* PLAIN with bf16 output only: ssq_out[t][m] = sum of squares of the (rounded) outputs of
+   * row tile t, i.e. the ssq_in of a product that consumes y.  NULL = not wanted. */
+  float* ssq_out; /* device */
+  /* ROPE_APPEND only */
+  void* q_out;                   /* device bf16 [M_b, Hq, 128] */
+  const void* const* k_page_ptr; /* device */
+  const void* const* v_page_ptr; /* device */
+  uint32_t n_pool_blocks;
+  const int32_t* block_table;    /* device [M_b, max_blocks] */
+  uint32_t max_blocks;
+  const int32_t* ctx_lens;       /* device [M_b], new token included */
+  uint32_t n_q_heads, n_kv_heads;
+  float rope_base;
+} boost_gemv_epilogue_t;
+
+/* boost_gemv_tiered with an epilogue descriptor (NULL = plain). */
+int boost_gemv_tiered_fused(const void* const* w_page_ptr /*device*/, const uint32_t* w_order /*device*/,
+                            size_t n_pages, size_t n_host_pages, uint32_t N, uint32_t K,
+                            const void* x /*device*/, uint32_t M_b, void* y /*device*/, int y_dtype,
+                            const void* residual /*device*/, const boost_gemv_epilogue_t* epilogue /*host*/,
+                            void* workspace /*device*/, size_t workspace_bytes, void* stream);
 
 /* Copy a logical KV cache [n_kv_heads][n_pool_blocks][16][D] (contiguous device buffer,
  * bf16) into the pages of a K or V tensor, or back.  Chunk (h, b) lands at byte offset
@@ -320,6 +372,13 @@ int boost_paged_attn_decode_tiered(const void* q /*device*/, const void* const* 
 int boost_embed_gather(const void* table /*device*/, uint32_t vocab, uint32_t hidden,
                        const int32_t* tokens /*device*/, uint32_t B, void* out /*device*/, void* stream);
 
+/* As boost_embed_gather; also writes ssq_out[t][b] (fp32, row pitch ssq_stride >= B) = sum of
+ * squares of columns [128 t, 128 t + 128) of row b, the row statistics a following
+ * boost_gemv_tiered_fused needs for its RMS scale.  hidden % 128 == 0. */
+int boost_embed_gather_ssq(const void* table /*device*/, uint32_t vocab, uint32_t hidden,
+                           const int32_t* tokens /*device*/, uint32_t B, void* out /*device*/,
+                           float* ssq_out /*device*/, uint32_t ssq_stride, void* stream);
+
 /* out = x * rsqrt(mean(x^2) + eps) * weight, row by row; x, out [B, hidden]; weight [hidden]. */
 int boost_rmsnorm(const void* x /*device*/, const void* weight /*device*/, uint32_t B, uint32_t hidden,
                   float eps, void* out /*device*/, void* stream);
@@ -355,12 +414,10 @@ typedef struct {
 } boost_weight_t;
 
 typedef struct {
-  boost_weight_t wqkv; /* [(Hq + 2 Hkv) D, hidden]: query rows, key rows, value rows */
+  boost_weight_t wqkv; /* [(Hq + 2 Hkv) D, hidden]: query, key, value rows; packed with col_scale = norm-1 weight */
   boost_weight_t wo;   /* [hidden, Hq D] */
-  boost_weight_t wgu;  /* [2 F, hidden]: gate rows, then up rows */
+  boost_weight_t wgu;  /* [2 F, hidden]: gate rows then up rows; packed with row_mode 1, col_scale = norm-2 weight */
   boost_weight_t wd;   /* [hidden, F] */
-  const void* norm1;   /* device bf16 [hidden] */
-  const void* norm2;
   const void* const* k_page_ptr; /* device: pages of this layer's K tensor */
   const void* const* v_page_ptr;
 } boost_llama_layer_t;
@@ -368,24 +425,27 @@ typedef struct {
 typedef struct {
   uint32_t n_layers, hidden, ffn, n_q_heads, n_kv_heads, head_dim, vocab;
   float rms_eps, rope_base;
-  const void* embed;  /* device bf16 [vocab, hidden] */
-  const void* norm_f; /* device bf16 [hidden] */
-  boost_weight_t lm_head; /* [vocab, hidden] */
+  const void* embed;      /* device bf16 [vocab, hidden] */
+  boost_weight_t lm_head; /* [vocab, hidden]; packed with col_scale = final norm weight */
   const boost_llama_layer_t* layers; /* host array of n_layers entries */
   const uint8_t* kv_tier;            /* host: tier of every page of a K (or V) tensor, or NULL */
   uint64_t n_kv_pages;
   uint32_t n_pool_blocks;
 } boost_llama_model_t;
 
-/* Device scratch of a decode step for up to B_max sequences (all bf16 unless noted):
- * h, xn [B, hidden]; qkv [B, (Hq+2Hkv) D]; q_rot, attn [B, Hq D]; gu [B, 2F]; act [B, F];
- * logits fp32 [B, vocab]; gemv_ws >= the largest boost_gemv_workspace_bytes over the model's
- * weights plus 33024 bytes (one set of queue words per launch of a step); attn_ws >= boost_paged_attn_workspace_bytes; both zero-filled once and 256-byte
- * aligned; tokens_dev / ctx_dev / next_dev int32 [B] and table_dev int32 [B, max_blocks] are
- * staging buffers used by boost_llama_decode_step_host only. */
+/* Device scratch of a decode step for up to ssq_stride sequences (bf16 unless noted):
+ * h [B, hidden] (residual stream); q_rot, attn [B, Hq D]; act [B, F]; logits fp32 [B, vocab];
+ * ssq_a, ssq_b fp32 [hidden / 128][ssq_stride] (row statistics for the RMS scales);
+ * gemv_ws >= the largest boost_gemv_workspace_bytes over the model's weights plus 33024
+ * bytes (one set of queue words per launch of a step); attn_ws >=
+ * boost_paged_attn_workspace_bytes; both zero-filled once and 256-byte aligned; tokens_dev /
+ * ctx_dev / next_dev int32 [B] and table_dev int32 [B, max_blocks] are staging buffers used by
+ * boost_llama_decode_step_host only. */
 typedef struct {
-  void *h, *xn, *qkv, *q_rot, *attn, *gu, *act;
+  void *h, *q_rot, *attn, *act;
   float* logits;
+  float *ssq_a, *ssq_b;
+  uint32_t ssq_stride;
   void* gemv_ws;
   size_t gemv_ws_bytes;
   void* attn_ws;
@@ -395,9 +455,11 @@ typedef struct {
 
 /* One decode step for B sequences: embedding, n_layers x (RMSNorm, QKV product, RoPE + KV
  * append, paged attention, output product + residual, RMSNorm, gate/up product, SwiGLU,
- * down product + residual), final RMSNorm, LM head, argmax.  Every product is
- * boost_gemv_tiered, attention is boost_paged_attn_decode_tiered.  Activations between
- * kernels are bf16; logits stay fp32.  tokens, block_table [B, max_blocks], ctx_lens (new
+ * down product + residual), final RMSNorm, LM head, argmax - as 1 + 5 n_layers + 2 launches:
+ * every small operator rides in the epilogue of a weight product (boost_gemv_tiered_fused:
+ * RMSNorm as a row scale with its weight folded into the matrix, RoPE + KV append after the
+ * QKV product, SwiGLU after the gate/up product, the row statistics of the residual stream
+ * after the output and down products).  Activations between kernels are bf16; logits fp32.  tokens, block_table [B, max_blocks], ctx_lens (new
  * token included) and next_tokens are device arrays.  Launches are asynchronous on stream.
  * Returns the number of kernels launched in *n_launches_out when it is not NULL. */
 int boost_llama_decode_step(const boost_llama_model_t* model /*host*/,

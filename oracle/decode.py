@@ -13,6 +13,15 @@ unpinned by the paper, pinned only by textbook special cases in the tests.
 All arithmetic is fp64.  Tensors that the device path stores as bf16 between
 kernels are rounded to bf16 here at the same places (marked "-> bf16"), so that
 32 layers of rounding do not separate the two; logits stay unrounded.
+
+RMSNorm in the step is evaluated in its factored form, the way an inference
+engine prepares a model for decoding: the norm weight is folded into the matrix
+it feeds when the model is loaded, W' = bf16(W * gamma) (one rounding, at load
+time), and the step computes rs * (h W'^T) with rs = 1/sqrt(mean(h^2) + eps)
+taken from the bf16 residual stream h.  This is x*rsqrt(mean(x^2)+eps)*gamma
+followed by the product, with the normalised activations never stored; the
+paper is silent on all of this (it treats decode as weight products plus
+attention), so the choice is this repository's and is stated in its design notes.
 """
 import numpy as np
 
@@ -46,6 +55,16 @@ def rope(x, positions, base=ROPE_BASE):
     return np.concatenate([x1 * c - x2 * s, x2 * c + x1 * s], axis=-1)
 
 
+def fold_norm_weight(w_bits, gamma_bits):
+    """W' = bf16(W * gamma): the RMSNorm weight folded into the matrix it feeds (load time)."""
+    return f64_to_bf16_bits(bf16_bits_to_f64(w_bits) * bf16_bits_to_f64(gamma_bits)[None, :])
+
+
+def rms_scale(x, eps=RMS_EPS):
+    """1 / sqrt(mean(x^2) + eps), row-wise.  x: fp64 [B, H] -> [B, 1]."""
+    return 1.0 / np.sqrt((x * x).mean(axis=-1, keepdims=True) + eps)
+
+
 def silu(x):
     return x / (1.0 + np.exp(-x))
 
@@ -77,8 +96,8 @@ def decode_step(cfg, weights, tokens, k_caches, v_caches, block_table, ctx_lens,
     h = bf16_bits_to_f64(weights["embed"][tokens])              # [B, hidden], bf16 values
     for li in range(n_layers):
         lw = weights["layers"][li]
-        _, xn = _round_bf16(rmsnorm(h, lw["norm1"]))             # -> bf16
-        _, qkv = _round_bf16(xn @ bf16_bits_to_f64(lw["wqkv"]).T)  # -> bf16
+        wqkv = bf16_bits_to_f64(fold_norm_weight(lw["wqkv"], lw["norm1"]))     # load-time fold -> bf16
+        _, qkv = _round_bf16(rms_scale(h) * (h @ wqkv.T))        # rmsnorm + product -> bf16
         q = qkv[:, :hq * d].reshape(n_seq, hq, d)
         k = qkv[:, hq * d:(hq + hkv) * d].reshape(n_seq, hkv, d)
         v = qkv[:, (hq + hkv) * d:].reshape(n_seq, hkv, d)
@@ -94,20 +113,20 @@ def decode_step(cfg, weights, tokens, k_caches, v_caches, block_table, ctx_lens,
                                       block_table, ctx_lens, scale)
         _, attn = _round_bf16(attn.reshape(n_seq, hq * d))       # -> bf16
         _, h = _round_bf16(h + attn @ bf16_bits_to_f64(lw["wo"]).T)   # residual -> bf16
-        _, xn2 = _round_bf16(rmsnorm(h, lw["norm2"]))            # -> bf16
-        _, gu = _round_bf16(xn2 @ bf16_bits_to_f64(lw["wgu"]).T)  # -> bf16
+        wgu = bf16_bits_to_f64(fold_norm_weight(lw["wgu"], lw["norm2"]))       # load-time fold -> bf16
+        _, gu = _round_bf16(rms_scale(h) * (h @ wgu.T))          # rmsnorm + product -> bf16
         f = gu.shape[1] // 2
         _, act = _round_bf16(silu(gu[:, :f]) * gu[:, f:])        # -> bf16
         _, h = _round_bf16(h + act @ bf16_bits_to_f64(lw["wd"]).T)    # residual -> bf16
         if keep:
             trace[f"h{li}"] = h.copy()
             if li == 0:
-                trace.update(xn=xn, qkv=qkv, q_rope=bf16_bits_to_f64(q_bits),
+                trace.update(qkv=qkv, q_rope=bf16_bits_to_f64(q_bits),
                              k_rope=bf16_bits_to_f64(k_bits), attn=attn, act=act)
-    _, xf = _round_bf16(rmsnorm(h, weights["norm_f"]))           # -> bf16
-    logits = xf @ bf16_bits_to_f64(weights["lm_head"]).T         # fp64, not rounded
+    w_head = bf16_bits_to_f64(fold_norm_weight(weights["lm_head"], weights["norm_f"]))   # load-time fold -> bf16
+    logits = rms_scale(h) * (h @ w_head.T)                       # fp64, not rounded
     # The device takes the argmax of fp32 logits: decide in that precision, lowest index on ties.
     next_tokens = np.argmax(logits.astype(np.float32), axis=-1).astype(np.int64)
-    out = {"logits": logits, "next_tokens": next_tokens, "h_final": h, "xf": xf}
+    out = {"logits": logits, "next_tokens": next_tokens, "h_final": h}
     out.update(trace)
     return out

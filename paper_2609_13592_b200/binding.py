@@ -53,9 +53,17 @@ class Weight(C.Structure):
                 ("n_host_pages", C.c_uint64), ("N", C.c_uint32), ("K", C.c_uint32)]
 
 
+class GemvEpilogue(C.Structure):
+    _fields_ = [("mode", C.c_int), ("ssq_in", C.c_void_p), ("ssq_in_tiles", C.c_uint32),
+                ("ssq_stride", C.c_uint32), ("rms_eps", C.c_float), ("ssq_out", C.c_void_p),
+                ("q_out", C.c_void_p), ("k_page_ptr", C.c_void_p), ("v_page_ptr", C.c_void_p),
+                ("n_pool_blocks", C.c_uint32), ("block_table", C.c_void_p), ("max_blocks", C.c_uint32),
+                ("ctx_lens", C.c_void_p), ("n_q_heads", C.c_uint32), ("n_kv_heads", C.c_uint32),
+                ("rope_base", C.c_float)]
+
+
 class LlamaLayer(C.Structure):
     _fields_ = [("wqkv", Weight), ("wo", Weight), ("wgu", Weight), ("wd", Weight),
-                ("norm1", C.c_void_p), ("norm2", C.c_void_p),
                 ("k_page_ptr", C.c_void_p), ("v_page_ptr", C.c_void_p)]
 
 
@@ -63,17 +71,20 @@ class LlamaModel(C.Structure):
     _fields_ = [(n, C.c_uint32) for n in
                 ("n_layers", "hidden", "ffn", "n_q_heads", "n_kv_heads", "head_dim", "vocab")] + \
                [("rms_eps", C.c_float), ("rope_base", C.c_float),
-                ("embed", C.c_void_p), ("norm_f", C.c_void_p), ("lm_head", Weight),
+                ("embed", C.c_void_p), ("lm_head", Weight),
                 ("layers", C.POINTER(LlamaLayer)), ("kv_tier", C.c_void_p),
                 ("n_kv_pages", C.c_uint64), ("n_pool_blocks", C.c_uint32)]
 
 
 class LlamaScratch(C.Structure):
-    _fields_ = [(n, C.c_void_p) for n in ("h", "xn", "qkv", "q_rot", "attn", "gu", "act", "logits")] + \
-               [("gemv_ws", C.c_void_p), ("gemv_ws_bytes", C.c_size_t),
+    _fields_ = [(n, C.c_void_p) for n in ("h", "q_rot", "attn", "act", "logits", "ssq_a", "ssq_b")] + \
+               [("ssq_stride", C.c_uint32),
+                ("gemv_ws", C.c_void_p), ("gemv_ws_bytes", C.c_size_t),
                 ("attn_ws", C.c_void_p), ("attn_ws_bytes", C.c_size_t)] + \
                [(n, C.c_void_p) for n in ("tokens_dev", "ctx_dev", "table_dev", "next_dev")]
 
+
+EPI_PLAIN, EPI_SWIGLU, EPI_ROPE_APPEND = 0, 1, 2
 
 _vp, _sz, _u32, _u64, _i32, _dbl, _int, _flt = (C.c_void_p, C.c_size_t, C.c_uint32, C.c_uint64,
                                                  C.c_int32, C.c_double, C.c_int, C.c_float)
@@ -104,6 +115,9 @@ SIGNATURES = {
     "boost_stream_reduce_tiered_static": (_int, [_vp, _vp, _sz, _sz, _vp, _vp]),
     "boost_weight_layout": (_int, [_u32, _u32, _vp]),
     "boost_pack_weights": (_int, [_vp, _u32, _u32, _vp, _sz, _vp]),
+    "boost_pack_weights_ex": (_int, [_vp, _u32, _u32, _vp, _sz, _int, _vp, _vp]),
+    "boost_gemv_tiered_fused": (_int, [_vp, _vp, _sz, _sz, _u32, _u32, _vp, _u32, _vp, _int, _vp, _vp, _vp, _sz, _vp]),
+    "boost_embed_gather_ssq": (_int, [_vp, _u32, _u32, _vp, _u32, _vp, _vp, _u32, _vp]),
     "boost_gemv_workspace_bytes": (_sz, [_u32, _u32, _u32]),
     "boost_gemv_tiered": (_int, [_vp, _vp, _sz, _sz, _u32, _u32, _vp, _u32, _vp, _int, _vp, _vp, _sz, _vp]),
     "boost_kv_scatter": (_int, [_vp, _u32, _u32, _u32, _vp, _sz, _vp]),
@@ -335,6 +349,26 @@ def boost_weight_layout(n, k):
 def boost_pack_weights(w_row_major, n, k, w_page_ptr, n_pages, stream=None):
     _check(lib().boost_pack_weights(_ptr(w_row_major), n, k, _ptr(w_page_ptr), n_pages, _stream(stream)),
            "boost_pack_weights")
+
+
+def boost_pack_weights_ex(w_row_major, n, k, w_page_ptr, n_pages, row_mode=0, col_scale=None, stream=None):
+    _check(lib().boost_pack_weights_ex(_ptr(w_row_major), n, k, _ptr(w_page_ptr), n_pages, row_mode,
+                                       _ptr(col_scale), _stream(stream)), "boost_pack_weights_ex")
+
+
+def boost_gemv_tiered_fused(w_page_ptr, w_order, n_pages, n_host_pages, n, k, x, m_b, y, y_dtype, residual,
+                            epilogue, workspace, workspace_bytes, stream=None):
+    """epilogue: a GemvEpilogue structure or None (plain)."""
+    _check(lib().boost_gemv_tiered_fused(_ptr(w_page_ptr), _ptr(w_order), n_pages, n_host_pages, n, k,
+                                         _ptr(x), m_b, _ptr(y), y_dtype, _ptr(residual),
+                                         None if epilogue is None else C.addressof(epilogue),
+                                         _ptr(workspace), workspace_bytes, _stream(stream)),
+           "boost_gemv_tiered_fused")
+
+
+def boost_embed_gather_ssq(table, vocab, hidden, tokens, b, out, ssq_out, ssq_stride, stream=None):
+    _check(lib().boost_embed_gather_ssq(_ptr(table), vocab, hidden, _ptr(tokens), b, _ptr(out),
+                                        _ptr(ssq_out), ssq_stride, _stream(stream)), "boost_embed_gather_ssq")
 
 
 def boost_gemv_workspace_bytes(n, k, m_b):

@@ -42,13 +42,13 @@ constexpr size_t kQueueSlotBytes = 64;
 constexpr size_t kQueueRegionBytes = kQueueSlots * kQueueSlotBytes;
 
 int gemv(const boost_weight_t& w, const void* x, uint32_t B, void* y, int y_dtype, const void* residual,
-         const boost_llama_scratch_t* s, uint32_t launch_index, void* stream) {
+         const boost_gemv_epilogue_t* epi, const boost_llama_scratch_t* s, uint32_t launch_index, void* stream) {
   if (s->gemv_ws_bytes <= kQueueRegionBytes + 256) return BOOST_ERR_CAPACITY;
   const size_t usable = (s->gemv_ws_bytes - kQueueRegionBytes) & ~(size_t)255;
   uint8_t* slots = static_cast<uint8_t*>(s->gemv_ws) + usable;
   uint32_t* queue = reinterpret_cast<uint32_t*>(slots + (launch_index % kQueueSlots) * kQueueSlotBytes);
   return boosth::gemv_tiered_launch(w.page_ptr, w.order, (size_t)w.n_pages, (size_t)w.n_host_pages, w.N, w.K, x,
-                                    B, y, y_dtype, residual, s->gemv_ws, usable, queue, stream);
+                                    B, y, y_dtype, residual, s->gemv_ws, usable, epi, queue, stream);
 }
 
 int run_step(Launcher& L, const boost_llama_model_t* m, const boost_llama_scratch_t* s, const int32_t* tokens,
@@ -56,35 +56,68 @@ int run_step(Launcher& L, const boost_llama_model_t* m, const boost_llama_scratc
              int32_t* next_tokens) {
   if (!m || !s || !tokens || !block_table || !ctx_lens || !next_tokens) return BOOST_ERR_INVALID;
   if (B == 0 || B > 128 || !m->layers || m->n_layers == 0) return BOOST_ERR_INVALID;
-  if (!s->h || !s->xn || !s->qkv || !s->q_rot || !s->attn || !s->gu || !s->act || !s->logits ||
-      !s->gemv_ws || !s->attn_ws)
+  if (!s->h || !s->q_rot || !s->attn || !s->act || !s->logits || !s->ssq_a || !s->ssq_b || !s->gemv_ws ||
+      !s->attn_ws || s->ssq_stride < B)
     return BOOST_ERR_INVALID;
+  if (m->hidden % 128 != 0 || m->head_dim != 128) return BOOST_ERR_UNSUPPORTED;
   void* stream = L.stream;
   const uint32_t hq = m->n_q_heads, hkv = m->n_kv_heads, d = m->head_dim;
   const float scale = 1.0f / sqrtf((float)d);
-  L.run(kKindGlue, [&] { return boost_embed_gather(m->embed, m->vocab, m->hidden, tokens, B, s->h, stream); });
+  const uint32_t h_tiles = m->hidden / 128;
+
+  // epilogue descriptors: x = residual stream h with row statistics in ssq_a / ssq_b
+  boost_gemv_epilogue_t scaled = {};
+  scaled.mode = BOOST_EPI_PLAIN;
+  scaled.ssq_in_tiles = h_tiles;
+  scaled.ssq_stride = s->ssq_stride;
+  scaled.rms_eps = m->rms_eps;
+  boost_gemv_epilogue_t stats = {};
+  stats.mode = BOOST_EPI_PLAIN;
+  stats.ssq_stride = s->ssq_stride;
+
+  L.run(kKindGlue, [&] {
+    return boost_embed_gather_ssq(m->embed, m->vocab, m->hidden, tokens, B, s->h, s->ssq_a, s->ssq_stride, stream);
+  });
   for (uint32_t li = 0; li < m->n_layers && L.ok(); ++li) {
     const boost_llama_layer_t& ly = m->layers[li];
-    L.run(kKindGlue, [&] { return boost_rmsnorm(s->h, ly.norm1, B, m->hidden, m->rms_eps, s->xn, stream); });
-    L.run(kKindGemv, [&] { return gemv(ly.wqkv, s->xn, B, s->qkv, 1, nullptr, s, L.count, stream); });
-    L.run(kKindGlue, [&] {
-      return boost_rope_kv_append(s->qkv, s->q_rot, ly.k_page_ptr, ly.v_page_ptr, m->n_pool_blocks, block_table,
-                                  max_blocks, ctx_lens, B, hq, hkv, d, m->rope_base, s->attn_ws, stream);
-    });
+    // q, k, v = rope(rmsnorm(h) Wqkv^T): row scale from ssq_a, RoPE + KV append in the epilogue
+    boost_gemv_epilogue_t qkv = scaled;
+    qkv.mode = BOOST_EPI_ROPE_APPEND;
+    qkv.ssq_in = s->ssq_a;
+    qkv.q_out = s->q_rot;
+    qkv.k_page_ptr = ly.k_page_ptr;
+    qkv.v_page_ptr = ly.v_page_ptr;
+    qkv.n_pool_blocks = m->n_pool_blocks;
+    qkv.block_table = block_table;
+    qkv.max_blocks = max_blocks;
+    qkv.ctx_lens = ctx_lens;
+    qkv.n_q_heads = hq;
+    qkv.n_kv_heads = hkv;
+    qkv.rope_base = m->rope_base;
+    L.run(kKindGemv, [&] { return gemv(ly.wqkv, s->h, B, nullptr, 1, nullptr, &qkv, s, L.count, stream); });
     L.run(kKindAttn, [&] {
       return boost_paged_attn_decode_tiered(s->q_rot, ly.k_page_ptr, ly.v_page_ptr, m->kv_tier,
                                             (size_t)m->n_kv_pages, m->n_pool_blocks, block_table, max_blocks,
                                             ctx_lens, B, hq, hkv, d, scale, s->attn_ws, s->attn_ws_bytes,
                                             s->attn, stream);
     });
-    L.run(kKindGemv, [&] { return gemv(ly.wo, s->attn, B, s->h, 1, s->h, s, L.count, stream); });     // h += attn Wo^T
-    L.run(kKindGlue, [&] { return boost_rmsnorm(s->h, ly.norm2, B, m->hidden, m->rms_eps, s->xn, stream); });
-    L.run(kKindGemv, [&] { return gemv(ly.wgu, s->xn, B, s->gu, 1, nullptr, s, L.count, stream); });
-    L.run(kKindGlue, [&] { return boost_swiglu(s->gu, B, m->ffn, s->act, stream); });
-    L.run(kKindGemv, [&] { return gemv(ly.wd, s->act, B, s->h, 1, s->h, s, L.count, stream); });      // h += act Wd^T
+    // h += attn Wo^T, row statistics of the new h into ssq_b
+    boost_gemv_epilogue_t wo = stats;
+    wo.ssq_out = s->ssq_b;
+    L.run(kKindGemv, [&] { return gemv(ly.wo, s->attn, B, s->h, 1, s->h, &wo, s, L.count, stream); });
+    // act = swiglu(rmsnorm(h) Wgu^T): row scale from ssq_b
+    boost_gemv_epilogue_t gu = scaled;
+    gu.mode = BOOST_EPI_SWIGLU;
+    gu.ssq_in = s->ssq_b;
+    L.run(kKindGemv, [&] { return gemv(ly.wgu, s->h, B, s->act, 1, nullptr, &gu, s, L.count, stream); });
+    // h += act Wd^T, row statistics of the new h into ssq_a
+    boost_gemv_epilogue_t wd = stats;
+    wd.ssq_out = s->ssq_a;
+    L.run(kKindGemv, [&] { return gemv(ly.wd, s->act, B, s->h, 1, s->h, &wd, s, L.count, stream); });
   }
-  L.run(kKindGlue, [&] { return boost_rmsnorm(s->h, m->norm_f, B, m->hidden, m->rms_eps, s->xn, stream); });
-  L.run(kKindGemv, [&] { return gemv(m->lm_head, s->xn, B, s->logits, 0, nullptr, s, L.count, stream); });
+  boost_gemv_epilogue_t head = scaled;
+  head.ssq_in = s->ssq_a;
+  L.run(kKindGemv, [&] { return gemv(m->lm_head, s->h, B, s->logits, 0, nullptr, &head, s, L.count, stream); });
   L.run(kKindGlue, [&] { return boost_argmax(s->logits, B, m->vocab, next_tokens, stream); });
   return L.rc;
 }
@@ -108,10 +141,10 @@ extern "C" int boost_llama_decode_step_profile(const boost_llama_model_t* m, con
                                                int32_t* next_tokens, float* kind_ms_out,
                                                uint32_t* kind_launches_out, void* stream) {
   if (!kind_ms_out || !kind_launches_out || !m) return BOOST_ERR_INVALID;
-  if (1 + 9 * (uint64_t)m->n_layers + 3 > 512) return BOOST_ERR_UNSUPPORTED;
+  if (1 + 5 * (uint64_t)m->n_layers + 2 > 512) return BOOST_ERR_UNSUPPORTED;
   static thread_local Launcher L;
   L.stream = stream; L.timed = true; L.count = 0; L.rc = BOOST_OK;
-  const uint32_t n_events = 2 * (1 + 9 * m->n_layers + 3);
+  const uint32_t n_events = 2 * (1 + 5 * m->n_layers + 2);
   uint32_t made = 0;
   int rc = BOOST_OK;
   for (; made < n_events && rc == BOOST_OK; ++made) rc = boosth::check(cudaEventCreate(&L.ev[made]));

@@ -42,7 +42,7 @@ inline int launch_chained(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_
 int gemv_tiered_launch(const void* const* w_page_ptr, const uint32_t* w_order, size_t n_pages,
                        size_t n_host_pages, uint32_t N, uint32_t K, const void* x, uint32_t M_b, void* y,
                        int y_dtype, const void* residual, void* workspace, size_t workspace_bytes,
-                       uint32_t* queue_words, void* stream);
+                       const boost_gemv_epilogue_t* epilogue, uint32_t* queue_words, void* stream);
 
 // Launch check: picks up configuration errors of the launch just made.
 inline int check_launch() { return check(cudaGetLastError()); }

@@ -32,6 +32,7 @@ constexpr uint32_t kSmemBudget = 224u * 1024u;
 constexpr uint32_t kXRowStride = 144;  // 128 data bytes + 16: 8 consecutive rows hit distinct banks
 
 enum : uint32_t { kFlagFirst = 1u, kFlagLast = 2u, kFlagStop = 4u };
+enum : uint32_t { kEpiPlain = 0u, kEpiSwiglu = 1u, kEpiRope = 2u };
 
 #ifdef BOOST_TRACE
 // Debug build only: per-threadblock time stamps (global timer, ns) for timeline analysis.
@@ -61,6 +62,19 @@ struct GemvParams {
   uint32_t* ws;        // header, then one counter per row tile
   uint32_t* queue;     // queue words: the header, or a private set (then weights may stream early)
   uint32_t early;      // 1: private queue words
+  // epilogue
+  uint32_t epi;              // kEpiPlain / kEpiSwiglu / kEpiRope
+  const float* ssq_in;       // [ssq_in_tiles][ssq_stride]: sums of squares of the rows of x by 128-column tile, or null
+  uint32_t ssq_in_tiles, ssq_stride, x_cols;
+  float rms_eps;
+  float* ssq_out;            // [n_row_tiles][ssq_stride]: the same for the rows of y (plain epilogue, bf16 output), or null
+  __nv_bfloat16* q_out;      // rope epilogue: rotated queries [M_b, Hq, 128]
+  const void* const* k_page_ptr;
+  const void* const* v_page_ptr;
+  const int32_t* block_table;
+  const int32_t* ctx_lens;
+  uint32_t n_pool_blocks, max_blocks, Hq, Hkv;
+  double log2_rope_base;
   float* partials;     // [row_tile][split][x_rows][128]
   uint32_t n_host_ctas;
   uint32_t n_stages;
@@ -78,21 +92,172 @@ __device__ __forceinline__ void store_out(const GemvParams& p, uint32_t m, uint3
   else static_cast<__nv_bfloat16*>(p.y)[idx] = __float2bfloat16_rn(v);
 }
 
-// four consecutive outputs of one batch row; N % 4 == 0 and n % 4 == 0
-__device__ __forceinline__ void store_out4(const GemvParams& p, uint32_t m, uint32_t n, float4 v) {
-  const size_t idx = (size_t)m * p.N + n;
-  if (p.residual) {
-    const uint2 r = *reinterpret_cast<const uint2*>(p.residual + idx);
-    v.x += bf16_lo(r.x); v.y += bf16_hi(r.x); v.z += bf16_lo(r.y); v.w += bf16_hi(r.y);
-  }
-  if (p.y_dtype == 0) {
-    *reinterpret_cast<float4*>(static_cast<float*>(p.y) + idx) = v;
-  } else {
-    const __nv_bfloat162 lo = __floats2bfloat162_rn(v.x, v.y), hi = __floats2bfloat162_rn(v.z, v.w);
-    uint2 o;
-    o.x = *reinterpret_cast<const uint32_t*>(&lo);
-    o.y = *reinterpret_cast<const uint32_t*>(&hi);
-    *reinterpret_cast<uint2*>(static_cast<__nv_bfloat16*>(p.y) + idx) = o;
+__device__ __forceinline__ uint2 pack4_bf16(float a, float b, float c, float d) {
+  const __nv_bfloat162 lo = __floats2bfloat162_rn(a, b), hi = __floats2bfloat162_rn(c, d);
+  uint2 o;
+  o.x = *reinterpret_cast<const uint32_t*>(&lo);
+  o.y = *reinterpret_cast<const uint32_t*>(&hi);
+  return o;
+}
+__device__ __forceinline__ float round_bf16(float v) { return __bfloat162float(__float2bfloat16_rn(v)); }
+
+// Sum the split-K partial sums of one row tile in split order and finish the outputs.
+// Thread -> (batch row m, columns [4 v, 4 v + 4) and their partners 64 columns on): the
+// partners are what SwiGLU (gate / up) and the rotary embedding (d / d + 64) pair up.
+//   plain   y = sum (* row scale) (+ residual); optionally the sum of squares of the bf16
+//           outputs per row, for the RMS scale of the next product;
+//   swiglu  rows 0..63 of the tile are gate rows, 64..127 the matching up rows:
+//           out[m, 64 t + j] = silu(bf16(gate)) * bf16(up);
+//   rope    the tile is one head of [q heads | k heads | v heads]: q and k are rotated
+//           (rotate-half pairing, angle = position * base^(-2i/128), in double), q goes to
+//           q_out, k and v into the paged cache at the position of the new token.
+// The row scale is rsqrt(mean(x^2) + eps) from per-tile sums of squares of the rows of x:
+// RMSNorm whose weight has been folded into the packed matrix.
+template <uint32_t kXRows>
+__device__ __noinline__ void combine_tile(const GemvParams& p, uint32_t row_tile, uint32_t tid, uint32_t* status) {
+  const float4* base = reinterpret_cast<const float4*>(p.partials + (size_t)row_tile * p.splits * kXRows * kBlockRows);
+  constexpr uint32_t kVecRow = kBlockRows / 4;   // float4 per batch row
+  const uint32_t n_pairs = p.M_b * 16;
+  for (uint32_t pidx0 = 0; pidx0 < n_pairs; pidx0 += kConsumerThreads) {
+    const uint32_t pidx = pidx0 + tid;
+    const bool valid = pidx < n_pairs;
+    const uint32_t m = valid ? (pidx >> 4) : 0u, v = pidx & 15u;
+    const uint32_t off = m * kVecRow + v;
+    float4 lo = make_float4(0.f, 0.f, 0.f, 0.f), hi = lo;
+    if (valid) {
+      // four splits (eight independent loads) per round: the L2 latency is paid per round
+      for (uint32_t sp0 = 0; sp0 < p.splits; sp0 += 4) {
+        float4 t0[4], t1[4];
+#pragma unroll
+        for (uint32_t u = 0; u < 4; ++u) {
+          if (sp0 + u < p.splits) {
+            const float4* src = base + (size_t)(sp0 + u) * kXRows * kVecRow + off;
+            t0[u] = __ldcg(src);
+            t1[u] = __ldcg(src + 16);
+          }
+        }
+#pragma unroll
+        for (uint32_t u = 0; u < 4; ++u) {
+          if (sp0 + u < p.splits) {
+            lo.x += t0[u].x; lo.y += t0[u].y; lo.z += t0[u].z; lo.w += t0[u].w;
+            hi.x += t1[u].x; hi.y += t1[u].y; hi.z += t1[u].z; hi.w += t1[u].w;
+          }
+        }
+      }
+      if (p.ssq_in) {
+        float ss = 0.f;
+        for (uint32_t t0 = 0; t0 < p.ssq_in_tiles; t0 += 8) {
+          float q[8];
+#pragma unroll
+          for (uint32_t u = 0; u < 8; ++u)
+            if (t0 + u < p.ssq_in_tiles) q[u] = __ldcg(p.ssq_in + (size_t)(t0 + u) * p.ssq_stride + m);
+#pragma unroll
+          for (uint32_t u = 0; u < 8; ++u)
+            if (t0 + u < p.ssq_in_tiles) ss += q[u];
+        }
+        const float rs = rsqrtf(ss / (float)p.x_cols + p.rms_eps);
+        lo.x *= rs; lo.y *= rs; lo.z *= rs; lo.w *= rs;
+        hi.x *= rs; hi.y *= rs; hi.z *= rs; hi.w *= rs;
+      }
+    }
+    if (p.epi == kEpiPlain) {
+      float sq = 0.f;
+      if (valid) {
+        const float4 val[2] = {lo, hi};
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
+          const uint32_t n = row_tile * kBlockRows + half * 64 + v * 4;
+          float e[4] = {val[half].x, val[half].y, val[half].z, val[half].w};
+          if (n + 3 < p.N && (p.N & 3u) == 0) {
+            const size_t idx = (size_t)m * p.N + n;
+            if (p.residual) {
+              const uint2 r = *reinterpret_cast<const uint2*>(p.residual + idx);
+              e[0] += bf16_lo(r.x); e[1] += bf16_hi(r.x); e[2] += bf16_lo(r.y); e[3] += bf16_hi(r.y);
+            }
+            if (p.y_dtype == 0) {
+              *reinterpret_cast<float4*>(static_cast<float*>(p.y) + idx) = make_float4(e[0], e[1], e[2], e[3]);
+            } else {
+              *reinterpret_cast<uint2*>(static_cast<__nv_bfloat16*>(p.y) + idx) = pack4_bf16(e[0], e[1], e[2], e[3]);
+#pragma unroll
+              for (int j = 0; j < 4; ++j) { const float b = round_bf16(e[j]); sq = fmaf(b, b, sq); }
+            }
+          } else {
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+              if (n + j < p.N) {
+                float x = e[j];
+                if (p.residual) x += __bfloat162float(p.residual[(size_t)m * p.N + n + j]);
+                if (p.y_dtype == 0) static_cast<float*>(p.y)[(size_t)m * p.N + n + j] = x;
+                else {
+                  static_cast<__nv_bfloat16*>(p.y)[(size_t)m * p.N + n + j] = __float2bfloat16_rn(x);
+                  const float b = round_bf16(x);
+                  sq = fmaf(b, b, sq);
+                }
+              }
+          }
+        }
+      }
+      if (p.ssq_out) {   // sum over the 16 threads that share row m (a fixed butterfly order)
+        sq += __shfl_xor_sync(0xFFFFFFFFu, sq, 1);
+        sq += __shfl_xor_sync(0xFFFFFFFFu, sq, 2);
+        sq += __shfl_xor_sync(0xFFFFFFFFu, sq, 4);
+        sq += __shfl_xor_sync(0xFFFFFFFFu, sq, 8);
+        if (valid && v == 0) p.ssq_out[(size_t)row_tile * p.ssq_stride + m] = sq;
+      }
+    } else if (p.epi == kEpiSwiglu) {
+      if (valid) {
+        const float g[4] = {round_bf16(lo.x), round_bf16(lo.y), round_bf16(lo.z), round_bf16(lo.w)};
+        const float u[4] = {round_bf16(hi.x), round_bf16(hi.y), round_bf16(hi.z), round_bf16(hi.w)};
+        float a[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) a[j] = g[j] / (1.f + expf(-g[j])) * u[j];
+        const size_t idx = (size_t)m * (p.N / 2) + row_tile * 64 + v * 4;
+        *reinterpret_cast<uint2*>(static_cast<__nv_bfloat16*>(p.y) + idx) = pack4_bf16(a[0], a[1], a[2], a[3]);
+      }
+    } else {   // kEpiRope
+      const int32_t ctx = valid ? p.ctx_lens[m] : 0;
+      if (valid && ctx > 0) {
+        const uint32_t pos = (uint32_t)ctx - 1u;
+        const uint32_t head = row_tile;
+        float x1[4] = {round_bf16(lo.x), round_bf16(lo.y), round_bf16(lo.z), round_bf16(lo.w)};
+        float x2[4] = {round_bf16(hi.x), round_bf16(hi.y), round_bf16(hi.z), round_bf16(hi.w)};
+        if (head < p.Hq + p.Hkv) {
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            const uint32_t i = v * 4 + j;
+            const double inv_freq = exp2(-(double)(2 * i) / (double)kBlockRows * p.log2_rope_base);
+            double sn, cs;
+            sincos((double)pos * inv_freq, &sn, &cs);
+            const float y1 = (float)((double)x1[j] * cs - (double)x2[j] * sn);
+            const float y2 = (float)((double)x2[j] * cs + (double)x1[j] * sn);
+            x1[j] = y1; x2[j] = y2;
+          }
+        }
+        const uint2 o1 = pack4_bf16(x1[0], x1[1], x1[2], x1[3]), o2 = pack4_bf16(x2[0], x2[1], x2[2], x2[3]);
+        const uint32_t d = v * 4;
+        if (head < p.Hq) {
+          __nv_bfloat16* dst = p.q_out + ((size_t)m * p.Hq + head) * kBlockRows;
+          *reinterpret_cast<uint2*>(dst + d) = o1;
+          *reinterpret_cast<uint2*>(dst + d + 64) = o2;
+        } else {
+          const bool is_k = head < p.Hq + p.Hkv;
+          const uint32_t kvh = is_k ? head - p.Hq : head - p.Hq - p.Hkv;
+          const uint32_t bi = pos / BOOST_KV_BLOCK_TOKENS, slot = pos % BOOST_KV_BLOCK_TOKENS;
+          const int32_t blk = bi < p.max_blocks ? p.block_table[(size_t)m * p.max_blocks + bi] : -1;
+          if (blk < 0 || (uint32_t)blk >= p.n_pool_blocks) {
+            atomicOr(status, kErrBadIndex);
+          } else {
+            const void* const* pages = is_k ? p.k_page_ptr : p.v_page_ptr;
+            // chunk (kvh, blk): token `slot` at slot*256, 16-byte piece c at position c ^ (slot & 7)
+            const size_t chunk = ((size_t)kvh * p.n_pool_blocks + (uint32_t)blk) * 4096u + slot * 256u;
+            const size_t off1 = chunk + ((((d >> 3) ^ (slot & 7u))) << 4) + (d & 7u) * 2u;
+            const size_t off2 = chunk + (((((d + 64) >> 3) ^ (slot & 7u))) << 4) + (d & 7u) * 2u;
+            *reinterpret_cast<uint2*>(static_cast<uint8_t*>(const_cast<void*>(pages[off1 / kPageBytes])) + off1 % kPageBytes) = o1;
+            *reinterpret_cast<uint2*>(static_cast<uint8_t*>(const_cast<void*>(pages[off2 / kPageBytes])) + off2 % kPageBytes) = o2;
+          }
+        }
+      }
+    }
   }
 }
 
@@ -322,7 +487,8 @@ __global__ void __launch_bounds__(kGemvThreads, (NT >= 8 ? 1 : 2)) gemv_tiered_k
             acc[j][m] = s;
           }
       }
-      const bool direct = (p.splits == 1);
+      // without splits (and without a row scale, pairing or row statistics) the sums go straight out
+      const bool direct = (p.splits == 1) && p.epi == kEpiPlain && !p.ssq_in && !p.ssq_out;
       float* part = p.partials + ((size_t)row_tile * p.splits + split) * kXRows * kBlockRows;
       if constexpr (NT > 0) {
 #pragma unroll
@@ -365,50 +531,7 @@ __global__ void __launch_bounds__(kGemvThreads, (NT >= 8 ? 1 : 2)) gemv_tiered_k
         named_barrier_sync(1, kConsumerThreads);
         if (s_old == p.splits - 1) {
           __threadfence();
-          const float4* base = reinterpret_cast<const float4*>(
-              p.partials + (size_t)row_tile * p.splits * kXRows * kBlockRows);
-          constexpr uint32_t kVecRow = kBlockRows / 4;   // float4 per batch row
-          // Each thread owns two float4 outputs at a time and walks the splits in order, four
-          // splits (eight independent loads) per round, so the L2 latency is paid once per
-          // round and not once per load.
-          const uint32_t n_vec = p.M_b * kVecRow;
-          for (uint32_t idx0 = tid; idx0 < n_vec; idx0 += 2 * kConsumerThreads) {
-            const uint32_t idx1 = idx0 + kConsumerThreads;
-            const bool two = idx1 < n_vec;
-            float4 a0 = make_float4(0.f, 0.f, 0.f, 0.f), a1 = a0;
-            for (uint32_t sp0 = 0; sp0 < p.splits; sp0 += 4) {
-              float4 t0[4], t1[4];
-#pragma unroll
-              for (uint32_t u = 0; u < 4; ++u) {
-                if (sp0 + u < p.splits) {
-                  const float4* src = base + (size_t)(sp0 + u) * kXRows * kVecRow;
-                  t0[u] = __ldcg(src + idx0);
-                  if (two) t1[u] = __ldcg(src + idx1);
-                }
-              }
-#pragma unroll
-              for (uint32_t u = 0; u < 4; ++u) {
-                if (sp0 + u < p.splits) {
-                  a0.x += t0[u].x; a0.y += t0[u].y; a0.z += t0[u].z; a0.w += t0[u].w;
-                  if (two) { a1.x += t1[u].x; a1.y += t1[u].y; a1.z += t1[u].z; a1.w += t1[u].w; }
-                }
-              }
-            }
-            for (int i = 0; i < (two ? 2 : 1); ++i) {
-              const uint32_t idx = i ? idx1 : idx0;
-              const float4 v = i ? a1 : a0;
-              const uint32_t m = idx / kVecRow, v4 = idx % kVecRow;
-              const uint32_t n = row_tile * kBlockRows + v4 * 4;
-              if (n + 3 < p.N && (p.N & 3u) == 0) {
-                store_out4(p, m, n, v);
-              } else {
-                if (n < p.N) store_out(p, m, n, v.x);
-                if (n + 1 < p.N) store_out(p, m, n + 1, v.y);
-                if (n + 2 < p.N) store_out(p, m, n + 2, v.z);
-                if (n + 3 < p.N) store_out(p, m, n + 3, v.w);
-              }
-            }
-          }
+          combine_tile<kXRows>(p, row_tile, tid, status);
           if (tid == 0) tile_cnt[row_tile] = 0;
           if (warp == 0) TRACE(8);
         }
@@ -421,19 +544,38 @@ __global__ void __launch_bounds__(kGemvThreads, (NT >= 8 ? 1 : 2)) gemv_tiered_k
 }
 
 // Packed form: 16-byte chunk `pos` of row r of block (t, kb) holds columns
-// [64 kb + 8 c, +8) of weight row 128 t + r with c = pos ^ (r & 7).
+// [64 kb + 8 c, +8) of packed row 128 t + r with c = pos ^ (r & 7).  Packed row -> weight row:
+// identity, or (row_mode 1) rows 0..63 of a tile = rows [64 t, 64 t + 64) of the first half of
+// W and rows 64..127 the same rows of the second half (gate and up rows side by side).
+// col_scale (bf16 [K], optional) multiplies column k: an RMSNorm weight folded into W.
 __global__ void __launch_bounds__(256)
 pack_weights_kernel(const uint4* __restrict__ w, uint32_t N, uint32_t K, uint32_t k_blocks,
-                    size_t n_chunks, const void* const* __restrict__ page_ptr) {
+                    size_t n_chunks, const void* const* __restrict__ page_ptr, int row_mode,
+                    const uint4* __restrict__ col_scale) {
   const size_t stride = (size_t)gridDim.x * blockDim.x;
   for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n_chunks; i += stride) {
     const size_t blk = i / (kBlockBytes / 16);
     const uint32_t in_blk = (uint32_t)(i % (kBlockBytes / 16));
     const uint32_t r = in_blk >> 3, pos = in_blk & 7, c = pos ^ (r & 7);
     const uint32_t t = (uint32_t)(blk / k_blocks), kb = (uint32_t)(blk % k_blocks);
-    const uint32_t row = t * kBlockRows + r, k = kb * kBlockK + c * 8;
+    uint32_t row = t * kBlockRows + r;
+    if (row_mode == 1) row = (r < 64) ? t * 64 + r : N / 2 + t * 64 + (r - 64);
+    const uint32_t k = kb * kBlockK + c * 8;
     uint4 v = make_uint4(0u, 0u, 0u, 0u);
-    if (row < N && k < K) v = w[((size_t)row * K + k) / 8];
+    if (row < N && k < K) {
+      v = w[((size_t)row * K + k) / 8];
+      if (col_scale) {
+        const uint4 g = col_scale[k / 8];
+        const uint32_t wv[4] = {v.x, v.y, v.z, v.w}, gv[4] = {g.x, g.y, g.z, g.w};
+        uint32_t o[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const __nv_bfloat162 pr = __floats2bfloat162_rn(bf16_lo(wv[j]) * bf16_lo(gv[j]), bf16_hi(wv[j]) * bf16_hi(gv[j]));
+          o[j] = *reinterpret_cast<const uint32_t*>(&pr);
+        }
+        v = make_uint4(o[0], o[1], o[2], o[3]);
+      }
+    }
     const size_t off = i * 16;
     uint4* dst = reinterpret_cast<uint4*>(static_cast<uint8_t*>(const_cast<void*>(page_ptr[off / kPageBytes])) +
                                           off % kPageBytes);
@@ -508,21 +650,30 @@ extern "C" int boost_weight_layout(uint32_t N, uint32_t K, boost_weight_layout_t
   return BOOST_OK;
 }
 
-extern "C" int boost_pack_weights(const void* w_row_major, uint32_t N, uint32_t K,
-                                  const void* const* w_page_ptr, size_t n_pages, void* stream) {
+extern "C" int boost_pack_weights_ex(const void* w_row_major, uint32_t N, uint32_t K,
+                                     const void* const* w_page_ptr, size_t n_pages, int row_mode,
+                                     const void* col_scale, void* stream) {
   boost_weight_layout_t lay;
   const int rc = boost_weight_layout(N, K, &lay);
   if (rc != BOOST_OK) return rc;
   if (!w_row_major || !w_page_ptr) return BOOST_ERR_INVALID;
-  if (K % 8 != 0 || ((uintptr_t)w_row_major % 16) != 0) return BOOST_ERR_ALIGN;
+  if (row_mode != 0 && row_mode != 1) return BOOST_ERR_INVALID;
+  if (row_mode == 1 && N % 128 != 0) return BOOST_ERR_INVALID;
+  if (K % 8 != 0 || ((uintptr_t)w_row_major % 16) != 0 || ((uintptr_t)col_scale % 16) != 0) return BOOST_ERR_ALIGN;
   if (n_pages < lay.n_pages) return BOOST_ERR_CAPACITY;
   const size_t n_chunks = lay.bytes / 16;
   size_t blocks = (n_chunks + 255) / 256;
   const size_t cap = (size_t)(boosth::sm_count() > 0 ? boosth::sm_count() : 148) * 16;
   if (blocks > cap) blocks = cap;
   pack_weights_kernel<<<(unsigned)blocks, 256, 0, (cudaStream_t)stream>>>(
-      static_cast<const uint4*>(w_row_major), N, K, lay.k_blocks, n_chunks, w_page_ptr);
+      static_cast<const uint4*>(w_row_major), N, K, lay.k_blocks, n_chunks, w_page_ptr, row_mode,
+      static_cast<const uint4*>(col_scale));
   return boosth::check_launch();
+}
+
+extern "C" int boost_pack_weights(const void* w_row_major, uint32_t N, uint32_t K,
+                                  const void* const* w_page_ptr, size_t n_pages, void* stream) {
+  return boost_pack_weights_ex(w_row_major, N, K, w_page_ptr, n_pages, 0, nullptr, stream);
 }
 
 static uint32_t gemv_x_rows(uint32_t M_b) {
@@ -541,7 +692,7 @@ extern "C" size_t boost_gemv_workspace_bytes(uint32_t N, uint32_t K, uint32_t M_
   boost_weight_layout_t lay;
   if (boost_weight_layout(N, K, &lay) != BOOST_OK || M_b == 0 || M_b > 128) return 0;
   size_t header = ((size_t)(kWsHeaderWords + lay.n_row_tiles) * 4 + 255) / 256 * 256;
-  size_t partials = lay.splits > 1 ? (size_t)lay.n_row_tiles * lay.splits * gemv_x_rows(M_b) * kBlockRows * 4 : 0;
+  size_t partials = (size_t)lay.n_row_tiles * lay.splits * gemv_x_rows(M_b) * kBlockRows * 4;
   return header + partials;
 }
 
@@ -551,14 +702,36 @@ extern "C" int boost_gemv_tiered(const void* const* w_page_ptr, const uint32_t* 
                                  const void* residual, void* workspace, size_t workspace_bytes,
                                  void* stream) {
   return boosth::gemv_tiered_launch(w_page_ptr, w_order, n_pages, n_host_pages, N, K, x, M_b, y, y_dtype,
-                                    residual, workspace, workspace_bytes, nullptr, stream);
+                                    residual, workspace, workspace_bytes, nullptr, nullptr, stream);
+}
+
+extern "C" int boost_gemv_tiered_fused(const void* const* w_page_ptr, const uint32_t* w_order,
+                                       size_t n_pages, size_t n_host_pages, uint32_t N, uint32_t K,
+                                       const void* x, uint32_t M_b, void* y, int y_dtype,
+                                       const void* residual, const boost_gemv_epilogue_t* epilogue,
+                                       void* workspace, size_t workspace_bytes, void* stream) {
+  return boosth::gemv_tiered_launch(w_page_ptr, w_order, n_pages, n_host_pages, N, K, x, M_b, y, y_dtype,
+                                    residual, workspace, workspace_bytes, epilogue, nullptr, stream);
 }
 
 int boosth::gemv_tiered_launch(const void* const* w_page_ptr, const uint32_t* w_order, size_t n_pages,
                                size_t n_host_pages, uint32_t N, uint32_t K, const void* x, uint32_t M_b,
                                void* y, int y_dtype, const void* residual, void* workspace,
-                               size_t workspace_bytes, uint32_t* queue_words, void* stream) {
-  if (!w_page_ptr || !w_order || !x || !y || !workspace) return BOOST_ERR_INVALID;
+                               size_t workspace_bytes, const boost_gemv_epilogue_t* epi,
+                               uint32_t* queue_words, void* stream) {
+  const int mode = epi ? epi->mode : BOOST_EPI_PLAIN;
+  if (!w_page_ptr || !w_order || !x || !workspace) return BOOST_ERR_INVALID;
+  if (!y && mode != BOOST_EPI_ROPE_APPEND) return BOOST_ERR_INVALID;
+  if (mode != BOOST_EPI_PLAIN && mode != BOOST_EPI_SWIGLU && mode != BOOST_EPI_ROPE_APPEND) return BOOST_ERR_INVALID;
+  if (mode == BOOST_EPI_SWIGLU && (N % 128 != 0 || y_dtype != 1 || residual)) return BOOST_ERR_INVALID;
+  if (mode == BOOST_EPI_ROPE_APPEND) {
+    if (!epi->q_out || !epi->k_page_ptr || !epi->v_page_ptr || !epi->block_table || !epi->ctx_lens ||
+        epi->n_pool_blocks == 0 || epi->max_blocks == 0 || !(epi->rope_base > 1.f) || residual)
+      return BOOST_ERR_INVALID;
+    if ((uint64_t)(epi->n_q_heads + 2 * epi->n_kv_heads) * 128 != N) return BOOST_ERR_INVALID;
+  }
+  if (epi && epi->ssq_in && (epi->ssq_in_tiles == 0 || epi->ssq_stride < M_b)) return BOOST_ERR_INVALID;
+  if (epi && epi->ssq_out && (mode != BOOST_EPI_PLAIN || y_dtype != 1 || epi->ssq_stride < M_b)) return BOOST_ERR_INVALID;
   if (M_b == 0 || M_b > 128 || (y_dtype != 0 && y_dtype != 1)) return BOOST_ERR_INVALID;
   boost_weight_layout_t lay;
   const int rc = boost_weight_layout(N, K, &lay);
@@ -588,6 +761,23 @@ int boosth::gemv_tiered_launch(const void* const* w_page_ptr, const uint32_t* w_
   p.ws = static_cast<uint32_t*>(workspace);
   p.queue = queue_words ? queue_words : p.ws;
   p.early = queue_words ? 1u : 0u;
+  p.epi = (uint32_t)mode;
+  p.ssq_in = epi ? epi->ssq_in : nullptr;
+  p.ssq_in_tiles = epi ? epi->ssq_in_tiles : 0;
+  p.ssq_stride = epi ? epi->ssq_stride : 0;
+  p.x_cols = K;
+  p.rms_eps = epi ? epi->rms_eps : 0.f;
+  p.ssq_out = epi ? epi->ssq_out : nullptr;
+  p.q_out = epi ? static_cast<__nv_bfloat16*>(epi->q_out) : nullptr;
+  p.k_page_ptr = epi ? epi->k_page_ptr : nullptr;
+  p.v_page_ptr = epi ? epi->v_page_ptr : nullptr;
+  p.block_table = epi ? epi->block_table : nullptr;
+  p.ctx_lens = epi ? epi->ctx_lens : nullptr;
+  p.n_pool_blocks = epi ? epi->n_pool_blocks : 0;
+  p.max_blocks = epi ? epi->max_blocks : 0;
+  p.Hq = epi ? epi->n_q_heads : 0;
+  p.Hkv = epi ? epi->n_kv_heads : 0;
+  p.log2_rope_base = (epi && epi->rope_base > 1.f) ? log2((double)epi->rope_base) : 0.0;
   const size_t header = ((size_t)(kWsHeaderWords + lay.n_row_tiles) * 4 + 255) / 256 * 256;
   p.partials = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + header);
   p.n_host_ctas = 0; p.n_stages = 0;

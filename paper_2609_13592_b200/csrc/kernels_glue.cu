@@ -17,16 +17,37 @@ constexpr uint32_t kD = 128;
 constexpr uint32_t kTok = BOOST_KV_BLOCK_TOKENS;
 constexpr uint32_t kChunkBytes = kTok * kD * 2;
 
+// ssq (optional): ssq[tile][b] = sum of squares of columns [128 tile, 128 tile + 128) of row b,
+// the row statistics a following product needs for its RMS scale.  A tile is 16 vectors of 8
+// values, read by 16 consecutive threads and summed with a fixed butterfly.
 __global__ void __launch_bounds__(256)
 embed_gather_kernel(const uint4* __restrict__ table, uint32_t vocab, uint32_t row_vecs,
-                    const int32_t* __restrict__ tokens, uint4* __restrict__ out) {
+                    const int32_t* __restrict__ tokens, uint4* __restrict__ out,
+                    float* __restrict__ ssq, uint32_t ssq_stride) {
   pdl_launch_dependents();
   pdl_wait();
   const uint32_t b = blockIdx.x;
   int32_t t = tokens[b];
   if (t < 0 || (uint32_t)t >= vocab) t = 0;
-  for (uint32_t i = threadIdx.x; i < row_vecs; i += blockDim.x)
-    out[(size_t)b * row_vecs + i] = table[(size_t)t * row_vecs + i];
+  const uint32_t n_iter = (row_vecs + blockDim.x - 1) / blockDim.x;
+  for (uint32_t it = 0; it < n_iter; ++it) {
+    const uint32_t i = it * blockDim.x + threadIdx.x;
+    float sq = 0.f;
+    if (i < row_vecs) {
+      const uint4 v = table[(size_t)t * row_vecs + i];
+      out[(size_t)b * row_vecs + i] = v;
+      const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+      for (int j = 0; j < 4; ++j) { sq = fmaf(bf16_lo(w[j]), bf16_lo(w[j]), sq); sq = fmaf(bf16_hi(w[j]), bf16_hi(w[j]), sq); }
+    }
+    if (ssq) {
+      sq += __shfl_xor_sync(0xFFFFFFFFu, sq, 1);
+      sq += __shfl_xor_sync(0xFFFFFFFFu, sq, 2);
+      sq += __shfl_xor_sync(0xFFFFFFFFu, sq, 4);
+      sq += __shfl_xor_sync(0xFFFFFFFFu, sq, 8);
+      if (i < row_vecs && (i & 15u) == 0) ssq[(size_t)(i >> 4) * ssq_stride + b] = sq;
+    }
+  }
 }
 
 // out = x * rsqrt(mean(x^2) + eps) * w, one threadblock per row, fp32 arithmetic.
@@ -182,11 +203,19 @@ argmax_kernel(const float* __restrict__ logits, uint32_t V, int32_t* __restrict_
 
 extern "C" int boost_embed_gather(const void* table, uint32_t vocab, uint32_t hidden,
                                   const int32_t* tokens, uint32_t B, void* out, void* stream) {
+  return boost_embed_gather_ssq(table, vocab, hidden, tokens, B, out, nullptr, 0, stream);
+}
+
+extern "C" int boost_embed_gather_ssq(const void* table, uint32_t vocab, uint32_t hidden,
+                                      const int32_t* tokens, uint32_t B, void* out, float* ssq_out,
+                                      uint32_t ssq_stride, void* stream) {
   if (B == 0) return BOOST_OK;
   if (!table || !tokens || !out || vocab == 0 || hidden == 0) return BOOST_ERR_INVALID;
   if (hidden % 8 != 0 || ((uintptr_t)table % 16) || ((uintptr_t)out % 16)) return BOOST_ERR_ALIGN;
+  if (ssq_out && (hidden % 128 != 0 || ssq_stride < B)) return BOOST_ERR_INVALID;
   return boosth::launch_chained(embed_gather_kernel, dim3(B), dim3(256), 0, (cudaStream_t)stream,
-                                static_cast<const uint4*>(table), vocab, hidden / 8, tokens, static_cast<uint4*>(out));
+                                static_cast<const uint4*>(table), vocab, hidden / 8, tokens, static_cast<uint4*>(out),
+                                ssq_out, ssq_stride);
 }
 
 extern "C" int boost_rmsnorm(const void* x, const void* weight, uint32_t B, uint32_t hidden, float eps,

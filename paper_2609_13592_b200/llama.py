@@ -43,34 +43,34 @@ class LlamaDecoder:
         self.n_pool_blocks = n_pool_blocks
         kv_bytes = hkv * n_pool_blocks * 16 * d * 2
 
-        def tiered(name, layer):
+        def tiered(name, layer, norm=None, row_mode=0):
+            # norm: name of the RMSNorm weight folded into this matrix at load time
             w = get_weight(name, layer).contiguous()
-            tw = TieredWeight(w, weight_host_ratio, weight_policy, device=self.device)
-            del w
+            g = get_weight(norm, layer).contiguous() if norm else None
+            tw = TieredWeight(w, weight_host_ratio, weight_policy, device=self.device, row_mode=row_mode,
+                              col_scale=g)
+            del w, g
             return tw
 
         self.embed = get_weight("embed", None).contiguous()
-        self.norm_f = get_weight("norm_f", None).contiguous()
-        self.lm_head = tiered("lm_head", None)
+        self.lm_head = tiered("lm_head", None, norm="norm_f")
         self.layers = []
         self._layer_structs = (B.LlamaLayer * nl)()
         for li in range(nl):
-            ly = {k: tiered(k, li) for k in ("wqkv", "wo", "wgu", "wd")}
-            ly["norm1"] = get_weight("norm1", li).contiguous()
-            ly["norm2"] = get_weight("norm2", li).contiguous()
+            ly = {"wqkv": tiered("wqkv", li, norm="norm1"), "wo": tiered("wo", li),
+                  "wgu": tiered("wgu", li, norm="norm2", row_mode=1), "wd": tiered("wd", li)}
             ly["k"] = TieredBuffer(kv_bytes, device=self.device, tier=self.kv_tier)
             ly["v"] = TieredBuffer(kv_bytes, device=self.device, tier=self.kv_tier)
             self.layers.append(ly)
             st = self._layer_structs[li]
             st.wqkv, st.wo = _weight_struct(ly["wqkv"]), _weight_struct(ly["wo"])
             st.wgu, st.wd = _weight_struct(ly["wgu"]), _weight_struct(ly["wd"])
-            st.norm1, st.norm2 = ly["norm1"].data_ptr(), ly["norm2"].data_ptr()
             st.k_page_ptr, st.v_page_ptr = ly["k"].page_ptr.data_ptr(), ly["v"].page_ptr.data_ptr()
         self._kv_tier_c = np.ascontiguousarray(self.kv_tier, dtype=np.uint8)
         m = B.LlamaModel()
         m.n_layers, m.hidden, m.ffn, m.n_q_heads, m.n_kv_heads = nl, hid, ffn, hq, hkv
         m.head_dim, m.vocab, m.rms_eps, m.rope_base = d, vocab, RMS_EPS, ROPE_BASE
-        m.embed, m.norm_f, m.lm_head = self.embed.data_ptr(), self.norm_f.data_ptr(), _weight_struct(self.lm_head)
+        m.embed, m.lm_head = self.embed.data_ptr(), _weight_struct(self.lm_head)
         m.layers = C.cast(self._layer_structs, C.POINTER(B.LlamaLayer))
         m.kv_tier = self._kv_tier_c.ctypes.data
         m.n_kv_pages, m.n_pool_blocks = int(self.kv_tier.size), n_pool_blocks
@@ -79,11 +79,11 @@ class LlamaDecoder:
         bm = max_batch
         bf = dict(dtype=torch.bfloat16, device=self.device)
         self.buf = {
-            "h": torch.zeros(bm, hid, **bf), "xn": torch.zeros(bm, hid, **bf),
-            "qkv": torch.zeros(bm, (hq + 2 * hkv) * d, **bf), "q_rot": torch.zeros(bm, hq * d, **bf),
-            "attn": torch.zeros(bm, hq * d, **bf), "gu": torch.zeros(bm, 2 * ffn, **bf),
-            "act": torch.zeros(bm, ffn, **bf),
+            "h": torch.zeros(bm, hid, **bf), "q_rot": torch.zeros(bm, hq * d, **bf),
+            "attn": torch.zeros(bm, hq * d, **bf), "act": torch.zeros(bm, ffn, **bf),
             "logits": torch.zeros(bm, vocab, dtype=torch.float32, device=self.device),
+            "ssq_a": torch.zeros(hid // 128, bm, dtype=torch.float32, device=self.device),
+            "ssq_b": torch.zeros(hid // 128, bm, dtype=torch.float32, device=self.device),
             "tokens_dev": torch.zeros(bm, dtype=torch.int32, device=self.device),
             "ctx_dev": torch.zeros(bm, dtype=torch.int32, device=self.device),
             "table_dev": torch.zeros(bm, max_blocks, dtype=torch.int32, device=self.device),
@@ -95,9 +95,10 @@ class LlamaDecoder:
         self._gemv_ws_t, gemv_ws = aligned_workspace(gemv_bytes, self.device)
         self._attn_ws_t, attn_ws = aligned_workspace(attn_bytes, self.device)
         s = B.LlamaScratch()
-        for k in ("h", "xn", "qkv", "q_rot", "attn", "gu", "act", "logits",
+        for k in ("h", "q_rot", "attn", "act", "logits", "ssq_a", "ssq_b",
                   "tokens_dev", "ctx_dev", "table_dev", "next_dev"):
             setattr(s, k, self.buf[k].data_ptr())
+        s.ssq_stride = bm
         s.gemv_ws, s.gemv_ws_bytes, s.attn_ws, s.attn_ws_bytes = gemv_ws, gemv_bytes, attn_ws, attn_bytes
         self.scratch = s
         self._gemv_ws_ptr, self._attn_ws_ptr = gemv_ws, attn_ws

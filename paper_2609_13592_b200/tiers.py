@@ -87,12 +87,14 @@ class TieredWeight:
     """A row-major bf16 weight [N, K] packed into tiered pages for boost_gemv_tiered."""
 
     def __init__(self, w, host_ratio=0.0, policy=B.POLICY_MODULO, seed=0, device="cuda", tier=None,
-                 superpage_pages=1):
+                 superpage_pages=1, row_mode=0, col_scale=None):
+        """row_mode 1 interleaves the two halves of the rows (gate / up) per 64 rows; col_scale
+        (bf16 [K]) is an RMSNorm weight folded into the matrix (see boost_pack_weights_ex)."""
         assert w.dtype == torch.bfloat16 and w.dim() == 2 and w.is_cuda and w.is_contiguous()
         self.N, self.K = int(w.shape[0]), int(w.shape[1])
         self.layout = B.boost_weight_layout(self.N, self.K)
         self.buf = TieredBuffer(self.layout["bytes"], host_ratio, policy, seed, superpage_pages, device, tier)
-        B.boost_pack_weights(w, self.N, self.K, self.buf.page_ptr, self.buf.n_pages)
+        B.boost_pack_weights_ex(w, self.N, self.K, self.buf.page_ptr, self.buf.n_pages, row_mode, col_scale)
         torch.cuda.current_stream().synchronize()
         self._ws = {}
 
@@ -113,16 +115,24 @@ class TieredWeight:
             out.append(int(ws[off:off + 4].cpu().numpy().view(np.uint32)[0]))
         return out
 
-    def gemv(self, x, y=None, y_dtype=torch.float32, residual=None, workspace=None, stream=None):
-        """y = x @ W^T (+ residual); x bf16 [M_b, K] (or [K])."""
+    def gemv(self, x, y=None, y_dtype=torch.float32, residual=None, workspace=None, stream=None,
+             epilogue=None):
+        """y = x @ W^T (+ residual); x bf16 [M_b, K] (or [K]).  epilogue: a binding.GemvEpilogue
+        (then y may be None for the RoPE-append mode)."""
         x2 = x.reshape(-1, self.K)
         m_b = x2.shape[0]
-        if y is None:
-            y = torch.empty(m_b, self.N, dtype=y_dtype, device=x.device)
+        if y is None and (epilogue is None or epilogue.mode != B.EPI_ROPE_APPEND):
+            n_out = self.N // 2 if (epilogue is not None and epilogue.mode == B.EPI_SWIGLU) else self.N
+            y = torch.empty(m_b, n_out, dtype=y_dtype, device=x.device)
         ws_ptr, ws_bytes = workspace if workspace is not None else self.workspace(m_b)
-        B.boost_gemv_tiered(self.buf.page_ptr, self.buf.order, self.buf.n_pages, self.buf.n_host,
-                            self.N, self.K, x2, m_b, y, 0 if y.dtype == torch.float32 else 1, residual,
-                            ws_ptr, ws_bytes, stream)
+        y_code = 1 if (y is None or y.dtype != torch.float32) else 0
+        if epilogue is None:
+            B.boost_gemv_tiered(self.buf.page_ptr, self.buf.order, self.buf.n_pages, self.buf.n_host,
+                                self.N, self.K, x2, m_b, y, y_code, residual, ws_ptr, ws_bytes, stream)
+        else:
+            B.boost_gemv_tiered_fused(self.buf.page_ptr, self.buf.order, self.buf.n_pages, self.buf.n_host,
+                                      self.N, self.K, x2, m_b, y, y_code, residual, epilogue, ws_ptr, ws_bytes,
+                                      stream)
         return y
 
 

@@ -171,7 +171,7 @@ def test_decode_steps_match_oracle(dev, n_seq, kv_modulus, weight_ratio):
         ctx_pin.numpy()[:] = ctx
         tab_pin.numpy()[:] = table
         n_launch = dec.step_host(tok_pin.numpy(), tab_pin.numpy(), ctx_pin.numpy(), nxt_pin.numpy())
-        assert n_launch == 1 + 9 * nl + 3
+        assert n_launch == 1 + 5 * nl + 2
         ref = od.decode_step(cfg, w, tokens, k_host, v_host, table, ctx)
         logits = dec.buf["logits"][:n_seq].cpu().numpy()
         assert_chain_close(logits, ref["logits"], f"logits step {step}")
@@ -199,3 +199,97 @@ def test_decode_steps_match_oracle(dev, n_seq, kv_modulus, weight_ratio):
         tokens = ref["next_tokens"].astype(np.int32)       # both sides continue from the oracle's choice
     assert dec.status_words() == [0, 0]
     assert exact_rows >= 0.6 * total_rows, (exact_rows, total_rows)
+
+
+def test_fused_product_epilogues_match_oracle(dev):
+    """boost_gemv_tiered_fused: RMS row scale with folded norm weight + row statistics, SwiGLU,
+    RoPE + KV append - each against the oracle's operators applied one after the other."""
+    from paper_2609_13592_b200.tiers import TieredKVCache, TieredWeight
+    m_b, hid, ffn, hq, hkv, d = 20, 512, 384, 4, 2, 128
+    x_bits = synth.normal_bf16((m_b, hid), 1.0, 1)
+    gamma = synth.f32_to_bf16_bits(1.0 + 0.1 * np.random.default_rng(2).standard_normal(hid).astype(np.float32))
+    x = bf16_tensor(x_bits, dev)
+    x64 = ol.bf16_bits_to_f64(x_bits)
+    rs = od.rms_scale(x64)
+    stride = 32
+    # row statistics of x as the embedding kernel produces them (gather rows 0..m_b-1 of x itself)
+    ssq = torch.zeros(hid // 128, stride, dtype=torch.float32, device=dev)
+    xcopy = torch.zeros_like(x)
+    B.boost_embed_gather_ssq(x, m_b, hid, torch.arange(m_b, dtype=torch.int32, device=dev), m_b, xcopy, ssq, stride)
+    torch.cuda.synchronize()
+    assert torch.equal(xcopy, x)
+    want_ssq = (x64.reshape(m_b, hid // 128, 128) ** 2).sum(-1).T
+    assert np.allclose(ssq.cpu().numpy()[:, :m_b], want_ssq, rtol=1e-5)
+
+    def epilogue(mode, **kw):
+        e = B.GemvEpilogue()
+        e.mode, e.ssq_in, e.ssq_in_tiles, e.ssq_stride, e.rms_eps = mode, ssq.data_ptr(), hid // 128, stride, od.RMS_EPS
+        for k, v in kw.items():
+            setattr(e, k, v)
+        return e
+
+    # 1. plain: y = rs * (x W'^T) + residual, bf16, with the row statistics of y
+    w_bits = synth.normal_bf16((640, hid), 0.05, 3)
+    res_bits = synth.normal_bf16((m_b, 640), 1.0, 4)
+    w = TieredWeight(bf16_tensor(w_bits, dev), 0.5, device=dev, col_scale=bf16_tensor(gamma, dev))
+    ssq_out = torch.zeros(5, stride, dtype=torch.float32, device=dev)
+    y = w.gemv(x, y_dtype=torch.bfloat16, residual=bf16_tensor(res_bits, dev),
+               epilogue=epilogue(B.EPI_PLAIN, ssq_out=ssq_out.data_ptr()))
+    torch.cuda.synchronize()
+    wf = ol.bf16_bits_to_f64(od.fold_norm_weight(w_bits, gamma))
+    ref = rs * (x64 @ wf.T) + ol.bf16_bits_to_f64(res_bits)
+    assert_close_to_oracle(y.float().cpu().numpy(), ref, "scaled product + residual")
+    y64 = y.float().cpu().numpy().astype(np.float64)
+    assert np.allclose(ssq_out.cpu().numpy()[:, :m_b], (y64.reshape(m_b, 5, 128) ** 2).sum(-1).T, rtol=1e-5)
+
+    # 2. SwiGLU: [gate; up] packed with interleaved rows
+    wgu_bits = synth.normal_bf16((2 * ffn, hid), 0.05, 5)
+    wgu = TieredWeight(bf16_tensor(wgu_bits, dev), 0.25, device=dev, row_mode=1, col_scale=bf16_tensor(gamma, dev))
+    act = wgu.gemv(x, y_dtype=torch.bfloat16, epilogue=epilogue(B.EPI_SWIGLU))
+    torch.cuda.synchronize()
+    assert tuple(act.shape) == (m_b, ffn)
+    gu = ol.bf16_bits_to_f64(ol.f64_to_bf16_bits(rs * (x64 @ ol.bf16_bits_to_f64(od.fold_norm_weight(wgu_bits, gamma)).T)))
+    assert_chain_close(act.float().cpu().numpy(), od.silu(gu[:, :ffn]) * gu[:, ffn:], "fused swiglu")
+
+    # 3. RoPE + KV append after the QKV product
+    n_blocks = 512
+    pool = B.KVPool(n_blocks, hkv, 4)
+    cache = TieredKVCache(pool, hkv, n_blocks, d, dev)
+    k0 = synth.normal_bf16((hkv, n_blocks, 16, d), 1.0, 6)
+    v0 = synth.normal_bf16((hkv, n_blocks, 16, d), 1.0, 7)
+    cache.load(bf16_tensor(k0, dev), bf16_tensor(v0, dev))
+    ctx = np.array([1, 16, 17, 100, 0] * 4, np.int32)
+    table = np.zeros((m_b, 8), np.int32)
+    used = iter(np.random.default_rng(8).permutation(n_blocks))
+    for b in range(m_b):
+        for j in range((ctx[b] + 15) // 16):
+            table[b, j] = next(used)
+    wqkv_bits = synth.normal_bf16(((hq + 2 * hkv) * d, hid), 0.05, 9)
+    wqkv = TieredWeight(bf16_tensor(wqkv_bits, dev), 0.5, device=dev, col_scale=bf16_tensor(gamma, dev))
+    q_out = torch.zeros(m_b, hq, d, dtype=torch.bfloat16, device=dev)
+    table_d, ctx_d = torch.from_numpy(table).to(dev), torch.from_numpy(ctx).to(dev)
+    wqkv.gemv(x, epilogue=epilogue(B.EPI_ROPE_APPEND, q_out=q_out.data_ptr(), k_page_ptr=cache.k.page_ptr.data_ptr(),
+                                   v_page_ptr=cache.v.page_ptr.data_ptr(), n_pool_blocks=n_blocks,
+                                   block_table=table_d.data_ptr(), max_blocks=8, ctx_lens=ctx_d.data_ptr(),
+                                   n_q_heads=hq, n_kv_heads=hkv, rope_base=od.ROPE_BASE))
+    torch.cuda.synchronize()
+    assert wqkv.status_words() == [0]
+    qkv = ol.bf16_bits_to_f64(ol.f64_to_bf16_bits(rs * (x64 @ ol.bf16_bits_to_f64(od.fold_norm_weight(wqkv_bits, gamma)).T)))
+    pos = np.maximum(ctx - 1, 0)
+    q_ref = od.rope(qkv[:, :hq * d].reshape(m_b, hq, d), pos)
+    k_ref = od.rope(qkv[:, hq * d:(hq + hkv) * d].reshape(m_b, hkv, d), pos)
+    v_ref = qkv[:, (hq + hkv) * d:].reshape(m_b, hkv, d)
+    live = ctx > 0
+    assert_chain_close(q_out.float().cpu().numpy()[live], q_ref[live], "fused rope q")
+    k_now, v_now = (bits_of(t) for t in cache.dump())
+    k_want, v_want = k0.copy(), v0.copy()
+    for b in range(m_b):
+        if ctx[b] == 0:
+            continue
+        blk, slot = table[b, pos[b] // 16], pos[b] % 16
+        assert_chain_close(ol.bf16_bits_to_f64(k_now[:, blk, slot]), k_ref[b], "fused rope k")
+        assert_chain_close(ol.bf16_bits_to_f64(v_now[:, blk, slot]), v_ref[b], "fused v")
+        k_want[:, blk, slot] = k_now[:, blk, slot]
+        v_want[:, blk, slot] = v_now[:, blk, slot]
+    assert np.array_equal(k_now, k_want) and np.array_equal(v_now, v_want)   # nothing else was touched
+    pool.close()

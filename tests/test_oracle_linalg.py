@@ -219,10 +219,16 @@ def test_decode_step_reduces_to_known_cases():
     wz = dict(w, layers=[dict(l, wo=np.zeros_like(l["wo"]), wd=np.zeros_like(l["wd"])) for l in w["layers"]])
     out = od.decode_step(cfg, wz, tokens, kc, vc, table, [1, 1, 1])
     h0 = ol.bf16_bits_to_f64(w["embed"][tokens])
-    xf = ol.bf16_bits_to_f64(ol.f64_to_bf16_bits(od.rmsnorm(h0, w["norm_f"])))
-    want = xf @ ol.bf16_bits_to_f64(w["lm_head"]).T
-    assert np.array_equal(out["logits"], want)
-    assert np.array_equal(out["next_tokens"], want.astype(np.float32).argmax(-1))
+    # textbook RMSNorm then the product, nothing rounded: the step's factored form (norm weight
+    # folded into the matrix with one bf16 rounding) must agree to that rounding
+    want = od.rmsnorm(h0, w["norm_f"]) @ ol.bf16_bits_to_f64(w["lm_head"]).T
+    assert np.abs(out["logits"] - want).max() <= 2.0 ** -6 * np.sqrt((want ** 2).mean())
+    # and exactly with the folded matrix written out by hand
+    folded = ol.bf16_bits_to_f64(ol.f64_to_bf16_bits(
+        ol.bf16_bits_to_f64(w["lm_head"]) * ol.bf16_bits_to_f64(w["norm_f"])[None, :]))
+    exact = (h0 @ folded.T) / np.sqrt((h0 * h0).mean(-1, keepdims=True) + od.RMS_EPS)
+    assert np.allclose(out["logits"], exact, rtol=1e-12, atol=1e-12)
+    assert np.array_equal(out["next_tokens"], out["logits"].astype(np.float32).argmax(-1))
     # the step wrote the new token's K/V at position ctx-1 of the right block and nowhere else
     assert kc[0][:, 0, 0].any() and not kc[0][:, 0, 1:].any() and not kc[0][:, 1].any()
     assert kc[0][:, 2, 0].any() and vc[1][:, 4, 0].any()
