@@ -320,7 +320,7 @@ typedef struct {
   uint32_t max_blocks;
   const int32_t* ctx_lens;       /* device [M_b], new token included */
   uint32_t n_q_heads, n_kv_heads;
-  float rope_base;
+  const float* rope_table;       /* device, from boost_rope_table: (cos, sin) [M_b][64] */
 } boost_gemv_epilogue_t;
 
 /* boost_gemv_tiered with an epilogue descriptor (NULL = plain). */
@@ -396,6 +396,12 @@ int boost_rope_kv_append(const void* qkv /*device*/, void* q_out /*device*/,
                          const int32_t* ctx_lens /*device*/, uint32_t B, uint32_t Hq, uint32_t Hkv,
                          uint32_t D, float rope_base, void* status_word /*device*/, void* stream);
 
+/* table[b][i] = (cos, sin) of (ctx_lens[b] - 1) * rope_base^(-2i/D), i < D/2, fp32 pairs,
+ * evaluated in double: the rotary angles of the new token of every sequence.  They are the
+ * same for all layers of a step, so a step computes them once.  D = 128. */
+int boost_rope_table(const int32_t* ctx_lens /*device*/, uint32_t B, uint32_t D, float rope_base,
+                     float* table /*device, B * D/2 * 2 floats*/, void* stream);
+
 /* out[b, f] = silu(gate_up[b, f]) * gate_up[b, F + f];  gate_up [B, 2F]; out [B, F]. */
 int boost_swiglu(const void* gate_up /*device*/, uint32_t B, uint32_t F, void* out /*device*/, void* stream);
 
@@ -435,7 +441,8 @@ typedef struct {
 
 /* Device scratch of a decode step for up to ssq_stride sequences (bf16 unless noted):
  * h [B, hidden] (residual stream); q_rot, attn [B, Hq D]; act [B, F]; logits fp32 [B, vocab];
- * ssq_a, ssq_b fp32 [hidden / 128][ssq_stride] (row statistics for the RMS scales);
+ * ssq_a, ssq_b fp32 [hidden / 128][ssq_stride] (row statistics for the RMS scales); rope_table
+ * fp32 [B][64][2];
  * gemv_ws >= the largest boost_gemv_workspace_bytes over the model's weights plus 33024
  * bytes (one set of queue words per launch of a step); attn_ws >=
  * boost_paged_attn_workspace_bytes; both zero-filled once and 256-byte aligned; tokens_dev /
@@ -446,6 +453,7 @@ typedef struct {
   float* logits;
   float *ssq_a, *ssq_b;
   uint32_t ssq_stride;
+  float* rope_table; /* fp32 [B][64][2] */
   void* gemv_ws;
   size_t gemv_ws_bytes;
   void* attn_ws;
@@ -455,7 +463,7 @@ typedef struct {
 
 /* One decode step for B sequences: embedding, n_layers x (RMSNorm, QKV product, RoPE + KV
  * append, paged attention, output product + residual, RMSNorm, gate/up product, SwiGLU,
- * down product + residual), final RMSNorm, LM head, argmax - as 1 + 5 n_layers + 2 launches:
+ * down product + residual), final RMSNorm, LM head, argmax - as 2 + 5 n_layers + 2 launches:
  * every small operator rides in the epilogue of a weight product (boost_gemv_tiered_fused:
  * RMSNorm as a row scale with its weight folded into the matrix, RoPE + KV append after the
  * QKV product, SwiGLU after the gate/up product, the row statistics of the residual stream

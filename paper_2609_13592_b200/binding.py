@@ -59,7 +59,7 @@ class GemvEpilogue(C.Structure):
                 ("q_out", C.c_void_p), ("k_page_ptr", C.c_void_p), ("v_page_ptr", C.c_void_p),
                 ("n_pool_blocks", C.c_uint32), ("block_table", C.c_void_p), ("max_blocks", C.c_uint32),
                 ("ctx_lens", C.c_void_p), ("n_q_heads", C.c_uint32), ("n_kv_heads", C.c_uint32),
-                ("rope_base", C.c_float)]
+                ("rope_table", C.c_void_p)]
 
 
 class LlamaLayer(C.Structure):
@@ -78,7 +78,7 @@ class LlamaModel(C.Structure):
 
 class LlamaScratch(C.Structure):
     _fields_ = [(n, C.c_void_p) for n in ("h", "q_rot", "attn", "act", "logits", "ssq_a", "ssq_b")] + \
-               [("ssq_stride", C.c_uint32),
+               [("ssq_stride", C.c_uint32), ("rope_table", C.c_void_p),
                 ("gemv_ws", C.c_void_p), ("gemv_ws_bytes", C.c_size_t),
                 ("attn_ws", C.c_void_p), ("attn_ws_bytes", C.c_size_t)] + \
                [(n, C.c_void_p) for n in ("tokens_dev", "ctx_dev", "table_dev", "next_dev")]
@@ -129,6 +129,7 @@ SIGNATURES = {
     "boost_rmsnorm": (_int, [_vp, _vp, _u32, _u32, _flt, _vp, _vp]),
     "boost_rope_kv_append": (_int, [_vp, _vp, _vp, _vp, _u32, _vp, _u32, _vp, _u32, _u32, _u32, _u32,
                                     _flt, _vp, _vp]),
+    "boost_rope_table": (_int, [_vp, _u32, _u32, _flt, _vp, _vp]),
     "boost_swiglu": (_int, [_vp, _u32, _u32, _vp, _vp]),
     "boost_argmax": (_int, [_vp, _u32, _u32, _vp, _vp]),
     "boost_llama_decode_step": (_int, [_vp, _vp, _vp, _vp, _u32, _vp, _u32, _vp, _vp, _vp]),
@@ -424,6 +425,10 @@ def boost_rope_kv_append(qkv, q_out, k_page_ptr, v_page_ptr, n_pool_blocks, bloc
                                       n_pool_blocks, _ptr(block_table), max_blocks, _ptr(ctx_lens), b, hq,
                                       hkv, d, rope_base, _ptr(status_word), _stream(stream)),
            "boost_rope_kv_append")
+
+
+def boost_rope_table(ctx_lens, b, d, rope_base, table, stream=None):
+    _check(lib().boost_rope_table(_ptr(ctx_lens), b, d, rope_base, _ptr(table), _stream(stream)), "boost_rope_table")
 
 
 def boost_swiglu(gate_up, b, f, out, stream=None):

@@ -56,7 +56,7 @@ int run_step(Launcher& L, const boost_llama_model_t* m, const boost_llama_scratc
              int32_t* next_tokens) {
   if (!m || !s || !tokens || !block_table || !ctx_lens || !next_tokens) return BOOST_ERR_INVALID;
   if (B == 0 || B > 128 || !m->layers || m->n_layers == 0) return BOOST_ERR_INVALID;
-  if (!s->h || !s->q_rot || !s->attn || !s->act || !s->logits || !s->ssq_a || !s->ssq_b || !s->gemv_ws ||
+  if (!s->h || !s->q_rot || !s->attn || !s->act || !s->logits || !s->ssq_a || !s->ssq_b || !s->rope_table || !s->gemv_ws ||
       !s->attn_ws || s->ssq_stride < B)
     return BOOST_ERR_INVALID;
   if (m->hidden % 128 != 0 || m->head_dim != 128) return BOOST_ERR_UNSUPPORTED;
@@ -75,6 +75,7 @@ int run_step(Launcher& L, const boost_llama_model_t* m, const boost_llama_scratc
   stats.mode = BOOST_EPI_PLAIN;
   stats.ssq_stride = s->ssq_stride;
 
+  L.run(kKindGlue, [&] { return boost_rope_table(ctx_lens, B, d, m->rope_base, s->rope_table, stream); });
   L.run(kKindGlue, [&] {
     return boost_embed_gather_ssq(m->embed, m->vocab, m->hidden, tokens, B, s->h, s->ssq_a, s->ssq_stride, stream);
   });
@@ -93,7 +94,7 @@ int run_step(Launcher& L, const boost_llama_model_t* m, const boost_llama_scratc
     qkv.ctx_lens = ctx_lens;
     qkv.n_q_heads = hq;
     qkv.n_kv_heads = hkv;
-    qkv.rope_base = m->rope_base;
+    qkv.rope_table = s->rope_table;
     L.run(kKindGemv, [&] { return gemv(ly.wqkv, s->h, B, nullptr, 1, nullptr, &qkv, s, L.count, stream); });
     L.run(kKindAttn, [&] {
       return boost_paged_attn_decode_tiered(s->q_rot, ly.k_page_ptr, ly.v_page_ptr, m->kv_tier,
@@ -141,10 +142,10 @@ extern "C" int boost_llama_decode_step_profile(const boost_llama_model_t* m, con
                                                int32_t* next_tokens, float* kind_ms_out,
                                                uint32_t* kind_launches_out, void* stream) {
   if (!kind_ms_out || !kind_launches_out || !m) return BOOST_ERR_INVALID;
-  if (1 + 5 * (uint64_t)m->n_layers + 2 > 512) return BOOST_ERR_UNSUPPORTED;
+  if (2 + 5 * (uint64_t)m->n_layers + 2 > 512) return BOOST_ERR_UNSUPPORTED;
   static thread_local Launcher L;
   L.stream = stream; L.timed = true; L.count = 0; L.rc = BOOST_OK;
-  const uint32_t n_events = 2 * (1 + 5 * m->n_layers + 2);
+  const uint32_t n_events = 2 * (2 + 5 * m->n_layers + 2);
   uint32_t made = 0;
   int rc = BOOST_OK;
   for (; made < n_events && rc == BOOST_OK; ++made) rc = boosth::check(cudaEventCreate(&L.ev[made]));

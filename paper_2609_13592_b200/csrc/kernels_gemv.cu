@@ -74,7 +74,7 @@ struct GemvParams {
   const int32_t* block_table;
   const int32_t* ctx_lens;
   uint32_t n_pool_blocks, max_blocks, Hq, Hkv;
-  double log2_rope_base;
+  const float* rope_table;   // rope epilogue: (cos, sin) [M_b][64] of this step's positions
   float* partials;     // [row_tile][split][x_rows][128]
   uint32_t n_host_ctas;
   uint32_t n_stages;
@@ -109,12 +109,12 @@ __device__ __forceinline__ float round_bf16(float v) { return __bfloat162float(_
 //   swiglu  rows 0..63 of the tile are gate rows, 64..127 the matching up rows:
 //           out[m, 64 t + j] = silu(bf16(gate)) * bf16(up);
 //   rope    the tile is one head of [q heads | k heads | v heads]: q and k are rotated
-//           (rotate-half pairing, angle = position * base^(-2i/128), in double), q goes to
-//           q_out, k and v into the paged cache at the position of the new token.
+//           (rotate-half pairing, cos / sin from the step's table), q goes to q_out, k and v
+//           into the paged cache at the position of the new token.
 // The row scale is rsqrt(mean(x^2) + eps) from per-tile sums of squares of the rows of x:
 // RMSNorm whose weight has been folded into the packed matrix.
 template <uint32_t kXRows>
-__device__ __noinline__ void combine_tile(const GemvParams& p, uint32_t row_tile, uint32_t tid, uint32_t* status) {
+__device__ __forceinline__ void combine_tile(const GemvParams& p, uint32_t row_tile, uint32_t tid, uint32_t* status) {
   const float4* base = reinterpret_cast<const float4*>(p.partials + (size_t)row_tile * p.splits * kXRows * kBlockRows);
   constexpr uint32_t kVecRow = kBlockRows / 4;   // float4 per batch row
   const uint32_t n_pairs = p.M_b * 16;
@@ -222,14 +222,14 @@ __device__ __noinline__ void combine_tile(const GemvParams& p, uint32_t row_tile
         float x1[4] = {round_bf16(lo.x), round_bf16(lo.y), round_bf16(lo.z), round_bf16(lo.w)};
         float x2[4] = {round_bf16(hi.x), round_bf16(hi.y), round_bf16(hi.z), round_bf16(hi.w)};
         if (head < p.Hq + p.Hkv) {
+          // cos / sin of position * base^(-2i/128) for i = 4v .. 4v+3, from the step's table
+          const float4 cs01 = __ldg(reinterpret_cast<const float4*>(p.rope_table + ((size_t)m * 64 + v * 4) * 2));
+          const float4 cs23 = __ldg(reinterpret_cast<const float4*>(p.rope_table + ((size_t)m * 64 + v * 4 + 2) * 2));
+          const float cs[4] = {cs01.x, cs01.z, cs23.x, cs23.z}, sn[4] = {cs01.y, cs01.w, cs23.y, cs23.w};
 #pragma unroll
           for (int j = 0; j < 4; ++j) {
-            const uint32_t i = v * 4 + j;
-            const double inv_freq = exp2(-(double)(2 * i) / (double)kBlockRows * p.log2_rope_base);
-            double sn, cs;
-            sincos((double)pos * inv_freq, &sn, &cs);
-            const float y1 = (float)((double)x1[j] * cs - (double)x2[j] * sn);
-            const float y2 = (float)((double)x2[j] * cs + (double)x1[j] * sn);
+            const float y1 = x1[j] * cs[j] - x2[j] * sn[j];
+            const float y2 = x2[j] * cs[j] + x1[j] * sn[j];
             x1[j] = y1; x2[j] = y2;
           }
         }
@@ -263,7 +263,7 @@ __device__ __noinline__ void combine_tile(const GemvParams& p, uint32_t row_tile
 
 // NT > 0: tensor-core path with NT batch tiles of 8; NT == 0: CUDA-core path for MB rows.
 template <int NT, int MB>
-__global__ void __launch_bounds__(kGemvThreads, (NT >= 8 ? 1 : 2)) gemv_tiered_kernel(const GemvParams p) {
+__global__ void __launch_bounds__(kGemvThreads, (NT >= 8 ? 1 : 2)) gemv_tiered_kernel(const __grid_constant__ GemvParams p) {
   constexpr uint32_t kXRows = x_rows_of(NT, MB);
   constexpr uint32_t kStageBytes = stage_bytes_of(NT, MB);
   extern __shared__ uint8_t smem_raw[];
@@ -726,7 +726,7 @@ int boosth::gemv_tiered_launch(const void* const* w_page_ptr, const uint32_t* w_
   if (mode == BOOST_EPI_SWIGLU && (N % 128 != 0 || y_dtype != 1 || residual)) return BOOST_ERR_INVALID;
   if (mode == BOOST_EPI_ROPE_APPEND) {
     if (!epi->q_out || !epi->k_page_ptr || !epi->v_page_ptr || !epi->block_table || !epi->ctx_lens ||
-        epi->n_pool_blocks == 0 || epi->max_blocks == 0 || !(epi->rope_base > 1.f) || residual)
+        epi->n_pool_blocks == 0 || epi->max_blocks == 0 || !epi->rope_table || residual)
       return BOOST_ERR_INVALID;
     if ((uint64_t)(epi->n_q_heads + 2 * epi->n_kv_heads) * 128 != N) return BOOST_ERR_INVALID;
   }
@@ -777,7 +777,7 @@ int boosth::gemv_tiered_launch(const void* const* w_page_ptr, const uint32_t* w_
   p.max_blocks = epi ? epi->max_blocks : 0;
   p.Hq = epi ? epi->n_q_heads : 0;
   p.Hkv = epi ? epi->n_kv_heads : 0;
-  p.log2_rope_base = (epi && epi->rope_base > 1.f) ? log2((double)epi->rope_base) : 0.0;
+  p.rope_table = epi ? epi->rope_table : nullptr;
   const size_t header = ((size_t)(kWsHeaderWords + lay.n_row_tiles) * 4 + 255) / 256 * 256;
   p.partials = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + header);
   p.n_host_ctas = 0; p.n_stages = 0;

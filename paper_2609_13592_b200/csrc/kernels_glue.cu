@@ -145,6 +145,20 @@ rope_kv_append_kernel(const __nv_bfloat16* __restrict__ qkv, __nv_bfloat16* __re
   *reinterpret_cast<__nv_bfloat16*>(p2) = __float2bfloat16_rn(y2);
 }
 
+// (cos, sin) of the rotary angles of the new token of every sequence, in double.
+__global__ void __launch_bounds__(64)
+rope_table_kernel(const int32_t* __restrict__ ctx_lens, double log2_base, float2* __restrict__ table) {
+  pdl_launch_dependents();
+  pdl_wait();
+  const uint32_t b = blockIdx.x, i = threadIdx.x;
+  const int32_t ctx = ctx_lens[b];
+  const double pos = ctx > 0 ? (double)(ctx - 1) : 0.0;
+  const double inv_freq = exp2(-(double)(2 * i) / (double)kD * log2_base);
+  double sn, cs;
+  sincos(pos * inv_freq, &sn, &cs);
+  table[(size_t)b * (kD / 2) + i] = make_float2((float)cs, (float)sn);
+}
+
 // act = silu(gate) * up with gate = gu[:, :F], up = gu[:, F:]
 __global__ void __launch_bounds__(256)
 swiglu_kernel(const __nv_bfloat16* __restrict__ gu, uint32_t B, uint32_t F, __nv_bfloat16* __restrict__ out) {
@@ -245,6 +259,16 @@ extern "C" int boost_rope_kv_append(const void* qkv, void* q_out, const void* co
                                 static_cast<__nv_bfloat16*>(q_out), k_page_ptr, v_page_ptr, n_pool_blocks,
                                 block_table, max_blocks, ctx_lens, B, Hq, Hkv, log2((double)rope_base),
                                 static_cast<uint32_t*>(status_word));
+}
+
+extern "C" int boost_rope_table(const int32_t* ctx_lens, uint32_t B, uint32_t D, float rope_base, float* table,
+                                void* stream) {
+  if (B == 0) return BOOST_OK;
+  if (!ctx_lens || !table || !(rope_base > 1.f)) return BOOST_ERR_INVALID;
+  if (D != kD) return BOOST_ERR_UNSUPPORTED;
+  if ((uintptr_t)table % 16) return BOOST_ERR_ALIGN;
+  return boosth::launch_chained(rope_table_kernel, dim3(B), dim3(kD / 2), 0, (cudaStream_t)stream, ctx_lens,
+                                log2((double)rope_base), reinterpret_cast<float2*>(table));
 }
 
 extern "C" int boost_swiglu(const void* gate_up, uint32_t B, uint32_t F, void* out, void* stream) {

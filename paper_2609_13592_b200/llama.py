@@ -84,6 +84,7 @@ class LlamaDecoder:
             "logits": torch.zeros(bm, vocab, dtype=torch.float32, device=self.device),
             "ssq_a": torch.zeros(hid // 128, bm, dtype=torch.float32, device=self.device),
             "ssq_b": torch.zeros(hid // 128, bm, dtype=torch.float32, device=self.device),
+            "rope_table": torch.zeros(bm, d // 2, 2, dtype=torch.float32, device=self.device),
             "tokens_dev": torch.zeros(bm, dtype=torch.int32, device=self.device),
             "ctx_dev": torch.zeros(bm, dtype=torch.int32, device=self.device),
             "table_dev": torch.zeros(bm, max_blocks, dtype=torch.int32, device=self.device),
@@ -95,7 +96,7 @@ class LlamaDecoder:
         self._gemv_ws_t, gemv_ws = aligned_workspace(gemv_bytes, self.device)
         self._attn_ws_t, attn_ws = aligned_workspace(attn_bytes, self.device)
         s = B.LlamaScratch()
-        for k in ("h", "q_rot", "attn", "act", "logits", "ssq_a", "ssq_b",
+        for k in ("h", "q_rot", "attn", "act", "logits", "ssq_a", "ssq_b", "rope_table",
                   "tokens_dev", "ctx_dev", "table_dev", "next_dev"):
             setattr(s, k, self.buf[k].data_ptr())
         s.ssq_stride = bm

@@ -171,7 +171,7 @@ def test_decode_steps_match_oracle(dev, n_seq, kv_modulus, weight_ratio):
         ctx_pin.numpy()[:] = ctx
         tab_pin.numpy()[:] = table
         n_launch = dec.step_host(tok_pin.numpy(), tab_pin.numpy(), ctx_pin.numpy(), nxt_pin.numpy())
-        assert n_launch == 1 + 5 * nl + 2
+        assert n_launch == 2 + 5 * nl + 2
         ref = od.decode_step(cfg, w, tokens, k_host, v_host, table, ctx)
         logits = dec.buf["logits"][:n_seq].cpu().numpy()
         assert_chain_close(logits, ref["logits"], f"logits step {step}")
@@ -268,10 +268,12 @@ def test_fused_product_epilogues_match_oracle(dev):
     wqkv = TieredWeight(bf16_tensor(wqkv_bits, dev), 0.5, device=dev, col_scale=bf16_tensor(gamma, dev))
     q_out = torch.zeros(m_b, hq, d, dtype=torch.bfloat16, device=dev)
     table_d, ctx_d = torch.from_numpy(table).to(dev), torch.from_numpy(ctx).to(dev)
+    rope_table = torch.zeros(m_b, d // 2, 2, dtype=torch.float32, device=dev)
+    B.boost_rope_table(ctx_d, m_b, d, od.ROPE_BASE, rope_table)
     wqkv.gemv(x, epilogue=epilogue(B.EPI_ROPE_APPEND, q_out=q_out.data_ptr(), k_page_ptr=cache.k.page_ptr.data_ptr(),
                                    v_page_ptr=cache.v.page_ptr.data_ptr(), n_pool_blocks=n_blocks,
                                    block_table=table_d.data_ptr(), max_blocks=8, ctx_lens=ctx_d.data_ptr(),
-                                   n_q_heads=hq, n_kv_heads=hkv, rope_base=od.ROPE_BASE))
+                                   n_q_heads=hq, n_kv_heads=hkv, rope_table=rope_table.data_ptr()))
     torch.cuda.synchronize()
     assert wqkv.status_words() == [0]
     qkv = ol.bf16_bits_to_f64(ol.f64_to_bf16_bits(rs * (x64 @ ol.bf16_bits_to_f64(od.fold_norm_weight(wqkv_bits, gamma)).T)))
