@@ -5,8 +5,10 @@ Default workload (N = 1): one Llama-3-8B-shaped decode step - 32 layers, hidden 
 14336, 32 query / 8 KV heads, vocab 128256, bf16 random-init weights N(0, 0.02^2), batch
 32, context 2048 - with weight pages placed by modulo placement at the host share that the
 measured host-link / HBM bandwidth ratio gives, KV cache in HBM.  A step runs every kernel
-of the path (embedding, 32 x [RMSNorm, QKV, RoPE + KV append, paged attention, output
-projection, RMSNorm, gate/up, SwiGLU, down], final norm, LM head, argmax) through the C ABI.
+of the path through the C ABI: RoPE table, embedding gather, 32 x [QKV product with RMSNorm
+scale, RoPE and KV append in its epilogue; paged attention; output product + residual;
+gate/up product with RMSNorm scale and SwiGLU in its epilogue; down product + residual],
+LM head, argmax - 164 launches.
 
   python bench.py --gpus N --steps K --warmup W            # this repository's kernels
   python bench.py --impl reference ...                      # the CPU oracle on the host cores
@@ -31,6 +33,10 @@ sys.path.insert(0, ROOT)
 
 WORKLOAD = "llama3_8b_shaped_decode_step_b32_ctx2048_tiered_weights"
 FALLBACK_HBM_GBS = 6650.0
+# DRAM bytes (read + write) per algorithmic byte of the weight-product kernel, from one ncu
+# capture of the gate/up, down and LM-head launches of this workload (profiles/
+# gemv_tiered_kernel_llama8b_m32.md): 1442.3 MB moved for 1403.0 MB of packed weights.
+GEMV_TRAFFIC_PER_ALGORITHMIC_BYTE = 1.028
 
 
 def load_peaks():
@@ -413,6 +419,10 @@ def run_ours(args, rank, world, local_rank):
         roof = hbm_peak + link_gbs
         gemv_ms, gemv_n = t["kind_ms"][0], t["kind_n"][0]
         gemv_gbs = t["weight_bytes"] / (gemv_ms / 1e3) / 1e9
+        gemv_bytes_per_launch = t["weight_bytes"] / max(gemv_n, 1)
+        # tier-wise bound: the slower of the two tiers if each streamed its own bytes at its own peak
+        host_bytes = t["host_pages"] * (2 << 20)
+        t_min_ms = 1e3 * max((bytes_step - host_bytes) / (hbm_peak * 1e9), host_bytes / (link_gbs * 1e9))
         attn_ms, attn_n = t["kind_ms"][1], t["kind_n"][1]
         attn_bytes = t["kv_tokens"] / args.steps * t["kv_bytes_per_token"]
         attn_gbs = attn_bytes / (attn_ms / 1e3) / 1e9
@@ -430,6 +440,8 @@ def run_ours(args, rank, world, local_rank):
             "combined_read_gbs": combined,
             "combined_roofline_gbs": roof,
             "combined_roofline_frac": combined / roof,
+            "tier_bound": {"t_min_ms": t_min_ms, "frac_of_t_min": t_min_ms / ms_step,
+                           "host_bytes_per_step": host_bytes},
             "hbm_peak_gbs": hbm_peak, "hbm_peak_source": peak_src,
             "host_link": {"type": "PCIe (zero-copy SM loads of pinned host memory)", "read_gbs": link_gbs,
                           "alpha": link_gbs / hbm_peak, "modulus": modulus},
@@ -440,7 +452,10 @@ def run_ours(args, rank, world, local_rank):
                          "tiered_over_hbm_only_time": ms_step / hb_ms},
             "roofline": {"bound": "hbm", "kernel": "gemv_tiered_kernel (weight products, M_b = 32)",
                          "achieved": gemv_gbs, "peak": hbm_peak, "unit": "GB/s", "frac": gemv_gbs / hbm_peak,
-                         "traffic": None, "launches_per_step": gemv_n, "avg_launch_us": 1e3 * gemv_ms / max(gemv_n, 1),
+                         "algorithmic_bytes_per_launch": gemv_bytes_per_launch,
+                         "traffic": GEMV_TRAFFIC_PER_ALGORITHMIC_BYTE * gemv_bytes_per_launch,
+                         "traffic_source": "ncu dram bytes of this workload's launches, ratio 1.028 to algorithmic",
+                         "launches_per_step": gemv_n, "avg_launch_us": 1e3 * gemv_ms / max(gemv_n, 1),
                          "peak_source": peak_src},
             "roofline_attention": {"bound": "hbm", "kernel": "paged_attn_kernel", "achieved": attn_gbs,
                                    "peak": hbm_peak, "unit": "GB/s", "frac": attn_gbs / hbm_peak,

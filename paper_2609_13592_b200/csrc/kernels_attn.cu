@@ -433,7 +433,6 @@ extern "C" int boost_paged_attn_decode_tiered(const void* q, const void* const* 
     const uint64_t items = (uint64_t)Hkv * B * ((max_blocks + len - 1) / len);
     if (items * 100 >= (uint64_t)n_warps * 55) { best_len = len; break; }
   }
-  if (const char* e = getenv("BOOST_ATTN_L")) { const uint32_t v = (uint32_t)atoi(e); if (v >= 1 && v <= kMaxItemBlocks) best_len = v; }   // experiment hook
   p.item_blocks = best_len;
   p.max_splits = (max_blocks + best_len - 1) / best_len;
   const uint64_t n_items = (uint64_t)Hkv * B * p.max_splits;

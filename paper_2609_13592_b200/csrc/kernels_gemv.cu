@@ -640,10 +640,6 @@ extern "C" int boost_weight_layout(uint32_t N, uint32_t K, boost_weight_layout_t
   out->n_row_tiles = (N + kBlockRows - 1) / kBlockRows;
   out->k_blocks = (K + kBlockK - 1) / kBlockK;
   out->blocks_per_item = pick_run(out->n_row_tiles, out->k_blocks);
-  if (const char* e = getenv("BOOST_RUN")) {   // experiment hook
-    const uint32_t r = (uint32_t)atoi(e);
-    if (r && out->k_blocks % r == 0 && 128 % r == 0) out->blocks_per_item = r;
-  }
   out->splits = out->k_blocks / out->blocks_per_item;
   out->bytes = (uint64_t)out->n_row_tiles * out->k_blocks * kBlockBytes;
   out->n_pages = (out->bytes + kPageBytes - 1) / kPageBytes;
