@@ -443,8 +443,8 @@ typedef struct {
  * h [B, hidden] (residual stream); q_rot, attn [B, Hq D]; act [B, F]; logits fp32 [B, vocab];
  * ssq_a, ssq_b fp32 [hidden / 128][ssq_stride] (row statistics for the RMS scales); rope_table
  * fp32 [B][64][2];
- * gemv_ws >= the largest boost_gemv_workspace_bytes over the model's weights plus 33024
- * bytes (one set of queue words per launch of a step); attn_ws >=
+ * gemv_ws >= boost_llama_gemv_workspace_bytes(model, B) (counters sized for the widest
+ * product, the largest set of partial sums, one set of queue words per launch); attn_ws >=
  * boost_paged_attn_workspace_bytes; both zero-filled once and 256-byte aligned; tokens_dev /
  * ctx_dev / next_dev int32 [B] and table_dev int32 [B, max_blocks] are staging buffers used by
  * boost_llama_decode_step_host only. */
@@ -460,6 +460,10 @@ typedef struct {
   size_t attn_ws_bytes;
   int32_t *tokens_dev, *ctx_dev, *table_dev, *next_dev;
 } boost_llama_scratch_t;
+
+/* Size of scratch->gemv_ws for steps of up to B sequences of this model (Sec. 2.1 treats the
+ * step as a chain of weight products; they share one workspace).  0 on invalid arguments. */
+size_t boost_llama_gemv_workspace_bytes(const boost_llama_model_t* model /*host*/, uint32_t B);
 
 /* One decode step for B sequences: embedding, n_layers x (RMSNorm, QKV product, RoPE + KV
  * append, paged attention, output product + residual, RMSNorm, gate/up product, SwiGLU,

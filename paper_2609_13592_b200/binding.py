@@ -132,6 +132,7 @@ SIGNATURES = {
     "boost_rope_table": (_int, [_vp, _u32, _u32, _flt, _vp, _vp]),
     "boost_swiglu": (_int, [_vp, _u32, _u32, _vp, _vp]),
     "boost_argmax": (_int, [_vp, _u32, _u32, _vp, _vp]),
+    "boost_llama_gemv_workspace_bytes": (C.c_size_t, [_vp, _u32]),
     "boost_llama_decode_step": (_int, [_vp, _vp, _vp, _vp, _u32, _vp, _u32, _vp, _vp, _vp]),
     "boost_llama_decode_step_profile": (_int, [_vp, _vp, _vp, _vp, _u32, _vp, _u32, _vp, _vp, _vp, _vp]),
     "boost_llama_decode_step_host": (_int, [_vp, _vp, _vp, _vp, _u32, _vp, _u32, _vp, _vp, _vp]),
@@ -437,6 +438,10 @@ def boost_swiglu(gate_up, b, f, out, stream=None):
 
 def boost_argmax(logits, b, v, out, stream=None):
     _check(lib().boost_argmax(_ptr(logits), b, v, _ptr(out), _stream(stream)), "boost_argmax")
+
+
+def boost_llama_gemv_workspace_bytes(model, b):
+    return int(lib().boost_llama_gemv_workspace_bytes(C.addressof(model), b))
 
 
 def boost_llama_decode_step(model, scratch, tokens, block_table, max_blocks, ctx_lens, b, next_tokens,

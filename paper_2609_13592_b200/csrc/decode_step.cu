@@ -41,14 +41,27 @@ constexpr size_t kQueueSlots = 512;
 constexpr size_t kQueueSlotBytes = 64;
 constexpr size_t kQueueRegionBytes = kQueueSlots * kQueueSlotBytes;
 
+// All products of a step share one workspace: the counter area is sized for the product with
+// the most row tiles, so that no product's partial sums lie where another keeps its counters.
+uint32_t max_row_tiles(const boost_llama_model_t* m) {
+  uint32_t n = m->lm_head.N;
+  for (uint32_t li = 0; li < m->n_layers; ++li) {
+    const boost_llama_layer_t& ly = m->layers[li];
+    const uint32_t ns[4] = {ly.wqkv.N, ly.wo.N, ly.wgu.N, ly.wd.N};
+    for (uint32_t v : ns) n = v > n ? v : n;
+  }
+  return (n + 127) / 128;
+}
+
 int gemv(const boost_weight_t& w, const void* x, uint32_t B, void* y, int y_dtype, const void* residual,
-         const boost_gemv_epilogue_t* epi, const boost_llama_scratch_t* s, uint32_t launch_index, void* stream) {
+         const boost_gemv_epilogue_t* epi, const boost_llama_scratch_t* s, uint32_t launch_index,
+         uint32_t header_tiles, void* stream) {
   if (s->gemv_ws_bytes <= kQueueRegionBytes + 256) return BOOST_ERR_CAPACITY;
   const size_t usable = (s->gemv_ws_bytes - kQueueRegionBytes) & ~(size_t)255;
   uint8_t* slots = static_cast<uint8_t*>(s->gemv_ws) + usable;
   uint32_t* queue = reinterpret_cast<uint32_t*>(slots + (launch_index % kQueueSlots) * kQueueSlotBytes);
   return boosth::gemv_tiered_launch(w.page_ptr, w.order, (size_t)w.n_pages, (size_t)w.n_host_pages, w.N, w.K, x,
-                                    B, y, y_dtype, residual, s->gemv_ws, usable, epi, queue, stream);
+                                    B, y, y_dtype, residual, s->gemv_ws, usable, epi, queue, header_tiles, stream);
 }
 
 int run_step(Launcher& L, const boost_llama_model_t* m, const boost_llama_scratch_t* s, const int32_t* tokens,
@@ -64,6 +77,7 @@ int run_step(Launcher& L, const boost_llama_model_t* m, const boost_llama_scratc
   const uint32_t hq = m->n_q_heads, hkv = m->n_kv_heads, d = m->head_dim;
   const float scale = 1.0f / sqrtf((float)d);
   const uint32_t h_tiles = m->hidden / 128;
+  const uint32_t tiles = max_row_tiles(m);
 
   // epilogue descriptors: x = residual stream h with row statistics in ssq_a / ssq_b
   boost_gemv_epilogue_t scaled = {};
@@ -95,7 +109,7 @@ int run_step(Launcher& L, const boost_llama_model_t* m, const boost_llama_scratc
     qkv.n_q_heads = hq;
     qkv.n_kv_heads = hkv;
     qkv.rope_table = s->rope_table;
-    L.run(kKindGemv, [&] { return gemv(ly.wqkv, s->h, B, nullptr, 1, nullptr, &qkv, s, L.count, stream); });
+    L.run(kKindGemv, [&] { return gemv(ly.wqkv, s->h, B, nullptr, 1, nullptr, &qkv, s, L.count, tiles, stream); });
     L.run(kKindAttn, [&] {
       return boost_paged_attn_decode_tiered(s->q_rot, ly.k_page_ptr, ly.v_page_ptr, m->kv_tier,
                                             (size_t)m->n_kv_pages, m->n_pool_blocks, block_table, max_blocks,
@@ -105,25 +119,39 @@ int run_step(Launcher& L, const boost_llama_model_t* m, const boost_llama_scratc
     // h += attn Wo^T, row statistics of the new h into ssq_b
     boost_gemv_epilogue_t wo = stats;
     wo.ssq_out = s->ssq_b;
-    L.run(kKindGemv, [&] { return gemv(ly.wo, s->attn, B, s->h, 1, s->h, &wo, s, L.count, stream); });
+    L.run(kKindGemv, [&] { return gemv(ly.wo, s->attn, B, s->h, 1, s->h, &wo, s, L.count, tiles, stream); });
     // act = swiglu(rmsnorm(h) Wgu^T): row scale from ssq_b
     boost_gemv_epilogue_t gu = scaled;
     gu.mode = BOOST_EPI_SWIGLU;
     gu.ssq_in = s->ssq_b;
-    L.run(kKindGemv, [&] { return gemv(ly.wgu, s->h, B, s->act, 1, nullptr, &gu, s, L.count, stream); });
+    L.run(kKindGemv, [&] { return gemv(ly.wgu, s->h, B, s->act, 1, nullptr, &gu, s, L.count, tiles, stream); });
     // h += act Wd^T, row statistics of the new h into ssq_a
     boost_gemv_epilogue_t wd = stats;
     wd.ssq_out = s->ssq_a;
-    L.run(kKindGemv, [&] { return gemv(ly.wd, s->act, B, s->h, 1, s->h, &wd, s, L.count, stream); });
+    L.run(kKindGemv, [&] { return gemv(ly.wd, s->act, B, s->h, 1, s->h, &wd, s, L.count, tiles, stream); });
   }
   boost_gemv_epilogue_t head = scaled;
   head.ssq_in = s->ssq_a;
-  L.run(kKindGemv, [&] { return gemv(m->lm_head, s->h, B, s->logits, 0, nullptr, &head, s, L.count, stream); });
+  L.run(kKindGemv, [&] { return gemv(m->lm_head, s->h, B, s->logits, 0, nullptr, &head, s, L.count, tiles, stream); });
   L.run(kKindGlue, [&] { return boost_argmax(s->logits, B, m->vocab, next_tokens, stream); });
   return L.rc;
 }
 
 }  // namespace
+
+extern "C" size_t boost_llama_gemv_workspace_bytes(const boost_llama_model_t* m, uint32_t B) {
+  if (!m || !m->layers || B == 0 || B > 128) return 0;
+  size_t partial = boosth::gemv_partial_bytes(m->lm_head.N, m->lm_head.K, B);
+  for (uint32_t li = 0; li < m->n_layers; ++li) {
+    const boost_llama_layer_t& ly = m->layers[li];
+    const boost_weight_t* ws[4] = {&ly.wqkv, &ly.wo, &ly.wgu, &ly.wd};
+    for (const boost_weight_t* w : ws) {
+      const size_t b = boosth::gemv_partial_bytes(w->N, w->K, B);
+      partial = b > partial ? b : partial;
+    }
+  }
+  return boosth::gemv_header_bytes(max_row_tiles(m)) + partial + kQueueRegionBytes + 256;
+}
 
 extern "C" int boost_llama_decode_step(const boost_llama_model_t* m, const boost_llama_scratch_t* s,
                                        const int32_t* tokens, const int32_t* block_table,

@@ -38,11 +38,19 @@ inline int launch_chained(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_
 
 // boost_gemv_tiered with a private set of queue words (16 zeroed uint32 that no other launch
 // in flight uses): the kernel may then take work and stream weights before its predecessor
-// has finished.  queue_words = nullptr gives the public behaviour.
+// has finished.  queue_words = nullptr gives the public behaviour.  header_row_tiles: size the
+// counter area at the head of the workspace for this many row tiles (0 = the product's own),
+// so that products of different shapes that share one workspace keep their counters clear of
+// each other's partial sums.
 int gemv_tiered_launch(const void* const* w_page_ptr, const uint32_t* w_order, size_t n_pages,
                        size_t n_host_pages, uint32_t N, uint32_t K, const void* x, uint32_t M_b, void* y,
                        int y_dtype, const void* residual, void* workspace, size_t workspace_bytes,
-                       const boost_gemv_epilogue_t* epilogue, uint32_t* queue_words, void* stream);
+                       const boost_gemv_epilogue_t* epilogue, uint32_t* queue_words, uint32_t header_row_tiles,
+                       void* stream);
+
+// Bytes of the counter area for n_row_tiles row tiles, and of the partial sums of one product.
+size_t gemv_header_bytes(uint32_t n_row_tiles);
+size_t gemv_partial_bytes(uint32_t N, uint32_t K, uint32_t M_b);
 
 // Launch check: picks up configuration errors of the launch just made.
 inline int check_launch() { return check(cudaGetLastError()); }

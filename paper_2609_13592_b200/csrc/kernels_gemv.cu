@@ -684,12 +684,20 @@ static uint32_t gemv_x_rows(uint32_t M_b) {
   return 128;
 }
 
+size_t boosth::gemv_header_bytes(uint32_t n_row_tiles) {
+  return ((size_t)(kWsHeaderWords + n_row_tiles) * 4 + 255) / 256 * 256;
+}
+
+size_t boosth::gemv_partial_bytes(uint32_t N, uint32_t K, uint32_t M_b) {
+  boost_weight_layout_t lay;
+  if (boost_weight_layout(N, K, &lay) != BOOST_OK || M_b == 0 || M_b > 128) return 0;
+  return (size_t)lay.n_row_tiles * lay.splits * gemv_x_rows(M_b) * kBlockRows * 4;
+}
+
 extern "C" size_t boost_gemv_workspace_bytes(uint32_t N, uint32_t K, uint32_t M_b) {
   boost_weight_layout_t lay;
   if (boost_weight_layout(N, K, &lay) != BOOST_OK || M_b == 0 || M_b > 128) return 0;
-  size_t header = ((size_t)(kWsHeaderWords + lay.n_row_tiles) * 4 + 255) / 256 * 256;
-  size_t partials = (size_t)lay.n_row_tiles * lay.splits * gemv_x_rows(M_b) * kBlockRows * 4;
-  return header + partials;
+  return boosth::gemv_header_bytes(lay.n_row_tiles) + boosth::gemv_partial_bytes(N, K, M_b);
 }
 
 extern "C" int boost_gemv_tiered(const void* const* w_page_ptr, const uint32_t* w_order,
@@ -698,7 +706,7 @@ extern "C" int boost_gemv_tiered(const void* const* w_page_ptr, const uint32_t* 
                                  const void* residual, void* workspace, size_t workspace_bytes,
                                  void* stream) {
   return boosth::gemv_tiered_launch(w_page_ptr, w_order, n_pages, n_host_pages, N, K, x, M_b, y, y_dtype,
-                                    residual, workspace, workspace_bytes, nullptr, nullptr, stream);
+                                    residual, workspace, workspace_bytes, nullptr, nullptr, 0, stream);
 }
 
 extern "C" int boost_gemv_tiered_fused(const void* const* w_page_ptr, const uint32_t* w_order,
@@ -707,14 +715,14 @@ extern "C" int boost_gemv_tiered_fused(const void* const* w_page_ptr, const uint
                                        const void* residual, const boost_gemv_epilogue_t* epilogue,
                                        void* workspace, size_t workspace_bytes, void* stream) {
   return boosth::gemv_tiered_launch(w_page_ptr, w_order, n_pages, n_host_pages, N, K, x, M_b, y, y_dtype,
-                                    residual, workspace, workspace_bytes, epilogue, nullptr, stream);
+                                    residual, workspace, workspace_bytes, epilogue, nullptr, 0, stream);
 }
 
 int boosth::gemv_tiered_launch(const void* const* w_page_ptr, const uint32_t* w_order, size_t n_pages,
                                size_t n_host_pages, uint32_t N, uint32_t K, const void* x, uint32_t M_b,
                                void* y, int y_dtype, const void* residual, void* workspace,
                                size_t workspace_bytes, const boost_gemv_epilogue_t* epi,
-                               uint32_t* queue_words, void* stream) {
+                               uint32_t* queue_words, uint32_t header_row_tiles, void* stream) {
   const int mode = epi ? epi->mode : BOOST_EPI_PLAIN;
   if (!w_page_ptr || !w_order || !x || !workspace) return BOOST_ERR_INVALID;
   if (!y && mode != BOOST_EPI_ROPE_APPEND) return BOOST_ERR_INVALID;
@@ -734,7 +742,8 @@ int boosth::gemv_tiered_launch(const void* const* w_page_ptr, const uint32_t* w_
   if (rc != BOOST_OK) return rc;
   if (n_pages != lay.n_pages || n_host_pages > n_pages) return BOOST_ERR_INVALID;
   if (K % 8 != 0 || ((uintptr_t)x % 16) != 0 || ((uintptr_t)workspace % 256) != 0) return BOOST_ERR_ALIGN;
-  if (workspace_bytes < boost_gemv_workspace_bytes(N, K, M_b)) return BOOST_ERR_CAPACITY;
+  const size_t header = gemv_header_bytes(header_row_tiles > lay.n_row_tiles ? header_row_tiles : lay.n_row_tiles);
+  if (workspace_bytes < header + gemv_partial_bytes(N, K, M_b)) return BOOST_ERR_CAPACITY;
   const int sms = boosth::sm_count();
   if (sms <= 0) return BOOST_ERR_CUDA;
 
@@ -774,7 +783,6 @@ int boosth::gemv_tiered_launch(const void* const* w_page_ptr, const uint32_t* w_
   p.Hq = epi ? epi->n_q_heads : 0;
   p.Hkv = epi ? epi->n_kv_heads : 0;
   p.rope_table = epi ? epi->rope_table : nullptr;
-  const size_t header = ((size_t)(kWsHeaderWords + lay.n_row_tiles) * 4 + 255) / 256 * 256;
   p.partials = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + header);
   p.n_host_ctas = 0; p.n_stages = 0;
   cudaStream_t st = (cudaStream_t)stream;

@@ -90,8 +90,8 @@ class LlamaDecoder:
             "table_dev": torch.zeros(bm, max_blocks, dtype=torch.int32, device=self.device),
             "next_dev": torch.zeros(bm, dtype=torch.int32, device=self.device),
         }
-        shapes = [(hq + 2 * hkv) * d, hid], [hid, hq * d], [2 * ffn, hid], [hid, ffn], [vocab, hid]
-        gemv_bytes = max(B.boost_gemv_workspace_bytes(n, k, bm) for n, k in shapes) + 33024
+        gemv_bytes = B.boost_llama_gemv_workspace_bytes(m, bm)
+        assert gemv_bytes > 0
         attn_bytes = B.boost_paged_attn_workspace_bytes(bm, hq, d, max_blocks)
         self._gemv_ws_t, gemv_ws = aligned_workspace(gemv_bytes, self.device)
         self._attn_ws_t, attn_ws = aligned_workspace(attn_bytes, self.device)

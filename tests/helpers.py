@@ -54,7 +54,7 @@ def chain_error(got, ref):
     return float((err / denom).max(initial=0.0)), float(err.max(initial=0.0))
 
 
-def assert_chain_close(got, ref, what=""):
+def assert_chain_close(got, ref, what="", wide=False):
     """Outputs of a CHAIN of kernels with bf16 tensors in between (a whole decode step).
     Where the fp32 device value and the fp64 oracle value of an intermediate fall on
     different sides of a bf16 rounding boundary, that intermediate differs by one bf16 ulp
@@ -63,7 +63,14 @@ def assert_chain_close(got, ref, what=""):
     emulation of the same chain, no CUDA involved).  Element-wise relative error is
     therefore not meaningful for a chain; the bound is 2e-2 absolute and 3e-2 of
     max(|ref|, rms(ref)).  Every kernel of the chain is held to the strict tolerance in its
-    own test, and callers also check that most rows agree to 1e-4 (no such event)."""
+    own test, and callers also check that most rows agree to 1e-4 (no such event).
+
+    wide=True is for the full-size model, whose bf16 activations reach magnitudes well above
+    1 (rms 1 - 2.5, elements beyond 10): one rounding flip alone is up to 2^-7 |value| (more
+    than 2e-2 from 2.6 on), a small element of the residual stream is the difference of
+    large ones, and the logits sum 4096 such elements; the 2e-2 absolute bound is dropped
+    there and only the bound relative to max(|ref|, rms(ref)) applies."""
     rel, abs_err = chain_error(got, ref)
-    assert abs_err <= ABS_TOL, f"{what}: max abs err {abs_err:.3e}"
+    if not wide:
+        assert abs_err <= ABS_TOL, f"{what}: max abs err {abs_err:.3e}"
     assert rel <= CHAIN_REL_TOL, f"{what}: max err / max(|ref|, rms) {rel:.3e}"

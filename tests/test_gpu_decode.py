@@ -295,3 +295,51 @@ def test_fused_product_epilogues_match_oracle(dev):
         v_want[:, blk, slot] = v_now[:, blk, slot]
     assert np.array_equal(k_now, k_want) and np.array_equal(v_now, v_want)   # nothing else was touched
     pool.close()
+
+
+def test_full_size_step_matches_oracle_on_samples(dev):
+    """One layer + LM head at the bench's shapes (hidden 4096, FFN 14336, 32 / 8 heads, vocab
+    128256, batch 32, context about 2048, weight host share 1/131, block tables 133 wide): the
+    launch configuration that bench.py times.  The oracle computes the layer in full and the
+    logits of every 61st vocabulary row (so every 128-row tile of the LM head is sampled)."""
+    cfg = dict(synth.LLAMA3_8B)
+    cfg["n_layers"] = 1
+    hq, hkv, d, hid, ffn, vocab = (cfg[k] for k in ("n_q_heads", "n_kv_heads", "head_dim", "hidden", "ffn", "vocab"))
+    n_seq, max_blocks, n_pool_blocks = 32, 133, 4608
+    head = synth.normal_bf16((vocab, hid), 0.02, 11)
+    gam = lambda s: synth.f32_to_bf16_bits(1.0 + 0.02 * np.random.default_rng(s).standard_normal(hid).astype(np.float32))
+    w = {"embed": head, "lm_head": head, "norm_f": gam(1), "layers": [{
+        "norm1": gam(2), "wqkv": synth.normal_bf16(((hq + 2 * hkv) * d, hid), 0.02, 12),
+        "wo": synth.normal_bf16((hid, hq * d), 0.02, 13), "norm2": gam(3),
+        "wgu": synth.normal_bf16((2 * ffn, hid), 0.02, 14), "wd": synth.normal_bf16((hid, ffn), 0.02, 15)}]}
+    dec = build_decoder(dev, cfg, w, n_pool_blocks, 0, 1.0 / 131, n_seq, max_blocks)
+    assert dec.host_weight_pages() > 0
+    k_host = [synth.normal_bf16((hkv, n_pool_blocks, 16, d), 1.0, 21)]
+    v_host = [synth.normal_bf16((hkv, n_pool_blocks, 16, d), 1.0, 22)]
+    load_caches(dev, dec, k_host, v_host)
+    rng = np.random.default_rng(5)
+    ctx = rng.integers(1900, 2101, size=n_seq).astype(np.int32)
+    table = np.zeros((n_seq, max_blocks), np.int32)
+    for j in range(max_blocks):                      # round-robin growth through the pool
+        for b in range(n_seq):
+            if j * 16 < ctx[b]:
+                table[b, j] = dec.pool.alloc(b, 1)[0]
+    tokens = rng.integers(0, vocab, size=n_seq).astype(np.int32)
+    nxt = np.zeros(n_seq, np.int32)
+    n_launch = dec.step_host(tokens, table, ctx, nxt)
+    assert n_launch == 2 + 5 + 2
+    assert dec.status_words() == [0, 0]
+
+    rows = np.arange(0, vocab, 61)
+    w_ref = dict(w)
+    w_ref["lm_head"] = head[rows]
+    ref = od.decode_step(cfg, w_ref, tokens, k_host, v_host, table, ctx, n_layers=1, keep=True)
+    assert_chain_close(dec.buf["act"].float().cpu().numpy(), ref["act"], "SwiGLU output, full width", wide=True)
+    assert_chain_close(dec.buf["h"].float().cpu().numpy(), ref["h_final"], "residual stream, full width", wide=True)
+    logits = dec.buf["logits"].cpu().numpy()
+    assert_chain_close(logits[:, rows], ref["logits"], "sampled logits", wide=True)
+    # integer work: the device's argmax of its own logits, lowest index on ties
+    assert np.array_equal(nxt, np.argmax(logits, axis=-1))
+    # every logit was written by this step: the buffer starts at zero, and an fp32 sum that
+    # cancels exactly is a once-in-10^7 event per element
+    assert logits.size - np.count_nonzero(logits) <= 4
