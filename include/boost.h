@@ -330,6 +330,42 @@ int boost_gemv_tiered_fused(const void* const* w_page_ptr /*device*/, const uint
                             const void* residual /*device*/, const boost_gemv_epilogue_t* epilogue /*host*/,
                             void* workspace /*device*/, size_t workspace_bytes, void* stream);
 
+/* A packed, tiered weight as consumed by boost_gemv_tiered. */
+typedef struct {
+  const void* const* page_ptr; /* device */
+  const uint32_t* order;       /* device */
+  uint64_t n_pages, n_host_pages;
+  uint32_t N, K;
+} boost_weight_t;
+
+/* One product of a chain: y = x W^T with the epilogue of boost_gemv_tiered_fused
+ * (has_epilogue = 0: plain). */
+typedef struct {
+  boost_weight_t w;
+  const void* x;        /* device, bf16 [M_b, w.K] */
+  void* y;              /* device (see boost_gemv_tiered_fused) */
+  int y_dtype;
+  const void* residual; /* device or NULL */
+  int has_epilogue;
+  boost_gemv_epilogue_t epilogue;
+} boost_gemv_call_t;
+
+/* A chain of 1..4 weight products in ONE launch, each of which may take what the previous
+ * ones wrote (as its x, its residual or its row statistics): the results equal those of the
+ * same calls of boost_gemv_tiered_fused made one after the other.  Sec. 2.1 describes decode as
+ * a chain of weight-streaming products; because weights do not depend on activations, the
+ * persistent threadblocks stream the next product's weight pages (both tiers, host pages
+ * first, as in boost_gemv_tiered) while the tail of the current product drains, and meet at
+ * a grid-wide counter between products.  All calls share M_b and the workspace.
+ *   workspace  device, 256-byte aligned, >= boost_gemv_chain_workspace_bytes, zero-filled
+ *              once (the kernel leaves its counters at zero); word 0 collects error bits
+ *              (bit 0: a bounded wait ran out, including the wait between products).
+ * Errors: INVALID (n_calls outside 1..4, a call that boost_gemv_tiered_fused would reject),
+ * ALIGN, CAPACITY, UNSUPPORTED (the device cannot hold one threadblock), CUDA. */
+size_t boost_gemv_chain_workspace_bytes(const boost_gemv_call_t* calls /*host*/, uint32_t n_calls, uint32_t M_b);
+int boost_gemv_tiered_chain(const boost_gemv_call_t* calls /*host*/, uint32_t n_calls, uint32_t M_b,
+                            void* workspace /*device*/, size_t workspace_bytes, void* stream);
+
 /* Copy a logical KV cache [n_kv_heads][n_pool_blocks][16][D] (contiguous device buffer,
  * bf16) into the pages of a K or V tensor, or back.  Chunk (h, b) lands at byte offset
  * (h*n_pool_blocks + b) * 4 KiB of the tensor; inside a chunk token t occupies 256 bytes at
@@ -410,14 +446,6 @@ int boost_argmax(const float* logits /*device*/, uint32_t B, uint32_t V, int32_t
                  void* stream);
 
 /* ------------------------------------------------------- whole decode step */
-
-/* A packed, tiered weight as consumed by boost_gemv_tiered. */
-typedef struct {
-  const void* const* page_ptr; /* device */
-  const uint32_t* order;       /* device */
-  uint64_t n_pages, n_host_pages;
-  uint32_t N, K;
-} boost_weight_t;
 
 typedef struct {
   boost_weight_t wqkv; /* [(Hq + 2 Hkv) D, hidden]: query, key, value rows; packed with col_scale = norm-1 weight */

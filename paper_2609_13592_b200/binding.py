@@ -62,6 +62,11 @@ class GemvEpilogue(C.Structure):
                 ("rope_table", C.c_void_p)]
 
 
+class GemvCall(C.Structure):
+    _fields_ = [("w", Weight), ("x", C.c_void_p), ("y", C.c_void_p), ("y_dtype", C.c_int),
+                ("residual", C.c_void_p), ("has_epilogue", C.c_int), ("epilogue", GemvEpilogue)]
+
+
 class LlamaLayer(C.Structure):
     _fields_ = [("wqkv", Weight), ("wo", Weight), ("wgu", Weight), ("wd", Weight),
                 ("k_page_ptr", C.c_void_p), ("v_page_ptr", C.c_void_p)]
@@ -132,6 +137,8 @@ SIGNATURES = {
     "boost_rope_table": (_int, [_vp, _u32, _u32, _flt, _vp, _vp]),
     "boost_swiglu": (_int, [_vp, _u32, _u32, _vp, _vp]),
     "boost_argmax": (_int, [_vp, _u32, _u32, _vp, _vp]),
+    "boost_gemv_chain_workspace_bytes": (C.c_size_t, [_vp, _u32, _u32]),
+    "boost_gemv_tiered_chain": (_int, [_vp, _u32, _u32, _vp, _sz, _vp]),
     "boost_llama_gemv_workspace_bytes": (C.c_size_t, [_vp, _u32]),
     "boost_llama_decode_step": (_int, [_vp, _vp, _vp, _vp, _u32, _vp, _u32, _vp, _vp, _vp]),
     "boost_llama_decode_step_profile": (_int, [_vp, _vp, _vp, _vp, _u32, _vp, _u32, _vp, _vp, _vp, _vp]),
@@ -366,6 +373,30 @@ def boost_gemv_tiered_fused(w_page_ptr, w_order, n_pages, n_host_pages, n, k, x,
                                          None if epilogue is None else C.addressof(epilogue),
                                          _ptr(workspace), workspace_bytes, _stream(stream)),
            "boost_gemv_tiered_fused")
+
+
+def gemv_calls(calls):
+    """calls: list of dict(w=Weight, x, y, y_dtype (0 fp32 / 1 bf16), residual=None, epilogue=None)
+    -> ctypes array of GemvCall."""
+    arr = (GemvCall * len(calls))()
+    for c, d in zip(arr, calls):
+        c.w, c.x, c.y, c.y_dtype = d["w"], _ptr(d["x"]), _ptr(d.get("y")), d["y_dtype"]
+        c.residual = _ptr(d.get("residual"))
+        epi = d.get("epilogue")
+        c.has_epilogue = 0 if epi is None else 1
+        if epi is not None:
+            c.epilogue = epi
+    return arr
+
+
+def boost_gemv_chain_workspace_bytes(calls, m_b):
+    return int(lib().boost_gemv_chain_workspace_bytes(C.addressof(calls), len(calls), m_b))
+
+
+def boost_gemv_tiered_chain(calls, m_b, workspace, workspace_bytes, stream=None):
+    """calls: the array made by gemv_calls; one launch for the whole chain."""
+    _check(lib().boost_gemv_tiered_chain(C.addressof(calls), len(calls), m_b, _ptr(workspace), workspace_bytes,
+                                         _stream(stream)), "boost_gemv_tiered_chain")
 
 
 def boost_embed_gather_ssq(table, vocab, hidden, tokens, b, out, ssq_out, ssq_stride, stream=None):

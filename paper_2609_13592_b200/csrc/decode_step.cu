@@ -53,15 +53,25 @@ uint32_t max_row_tiles(const boost_llama_model_t* m) {
   return (n + 127) / 128;
 }
 
-int gemv(const boost_weight_t& w, const void* x, uint32_t B, void* y, int y_dtype, const void* residual,
-         const boost_gemv_epilogue_t* epi, const boost_llama_scratch_t* s, uint32_t launch_index,
-         uint32_t header_tiles, void* stream) {
-  if (s->gemv_ws_bytes <= kQueueRegionBytes + 256) return BOOST_ERR_CAPACITY;
-  const size_t usable = (s->gemv_ws_bytes - kQueueRegionBytes) & ~(size_t)255;
-  uint8_t* slots = static_cast<uint8_t*>(s->gemv_ws) + usable;
-  uint32_t* queue = reinterpret_cast<uint32_t*>(slots + (launch_index % kQueueSlots) * kQueueSlotBytes);
-  return boosth::gemv_tiered_launch(w.page_ptr, w.order, (size_t)w.n_pages, (size_t)w.n_host_pages, w.N, w.K, x,
-                                    B, y, y_dtype, residual, s->gemv_ws, usable, epi, queue, header_tiles, stream);
+// Sync words of a launch: `n_calls + 1` slots from the region at the tail of the workspace.
+struct SyncSlots {
+  uint32_t next = 0;
+  uint32_t* take(const boost_llama_scratch_t* s, size_t usable, uint32_t n) {
+    if (next + n > kQueueSlots) next = 0;
+    uint8_t* slots = static_cast<uint8_t*>(s->gemv_ws) + usable;
+    uint32_t* r = reinterpret_cast<uint32_t*>(slots + (size_t)next * kQueueSlotBytes);
+    next += n;
+    return r;
+  }
+};
+
+boost_gemv_call_t call_of(const boost_weight_t& w, const void* x, void* y, int y_dtype, const void* residual,
+                          const boost_gemv_epilogue_t& epi) {
+  boost_gemv_call_t c = {};
+  c.w = w; c.x = x; c.y = y; c.y_dtype = y_dtype; c.residual = residual;
+  c.has_epilogue = 1;
+  c.epilogue = epi;
+  return c;
 }
 
 int run_step(Launcher& L, const boost_llama_model_t* m, const boost_llama_scratch_t* s, const int32_t* tokens,
@@ -73,11 +83,14 @@ int run_step(Launcher& L, const boost_llama_model_t* m, const boost_llama_scratc
       !s->attn_ws || s->ssq_stride < B)
     return BOOST_ERR_INVALID;
   if (m->hidden % 128 != 0 || m->head_dim != 128) return BOOST_ERR_UNSUPPORTED;
+  if (s->gemv_ws_bytes <= kQueueRegionBytes + 256) return BOOST_ERR_CAPACITY;
+  const size_t usable = (s->gemv_ws_bytes - kQueueRegionBytes) & ~(size_t)255;
   void* stream = L.stream;
   const uint32_t hq = m->n_q_heads, hkv = m->n_kv_heads, d = m->head_dim;
   const float scale = 1.0f / sqrtf((float)d);
   const uint32_t h_tiles = m->hidden / 128;
   const uint32_t tiles = max_row_tiles(m);
+  SyncSlots slots;
 
   // epilogue descriptors: x = residual stream h with row statistics in ssq_a / ssq_b
   boost_gemv_epilogue_t scaled = {};
@@ -89,13 +102,8 @@ int run_step(Launcher& L, const boost_llama_model_t* m, const boost_llama_scratc
   stats.mode = BOOST_EPI_PLAIN;
   stats.ssq_stride = s->ssq_stride;
 
-  L.run(kKindGlue, [&] { return boost_rope_table(ctx_lens, B, d, m->rope_base, s->rope_table, stream); });
-  L.run(kKindGlue, [&] {
-    return boost_embed_gather_ssq(m->embed, m->vocab, m->hidden, tokens, B, s->h, s->ssq_a, s->ssq_stride, stream);
-  });
-  for (uint32_t li = 0; li < m->n_layers && L.ok(); ++li) {
-    const boost_llama_layer_t& ly = m->layers[li];
-    // q, k, v = rope(rmsnorm(h) Wqkv^T): row scale from ssq_a, RoPE + KV append in the epilogue
+  // q, k, v = rope(rmsnorm(h) Wqkv^T): row scale from ssq_a, RoPE + KV append in the epilogue
+  auto qkv_call = [&](const boost_llama_layer_t& ly) {
     boost_gemv_epilogue_t qkv = scaled;
     qkv.mode = BOOST_EPI_ROPE_APPEND;
     qkv.ssq_in = s->ssq_a;
@@ -109,30 +117,48 @@ int run_step(Launcher& L, const boost_llama_model_t* m, const boost_llama_scratc
     qkv.n_q_heads = hq;
     qkv.n_kv_heads = hkv;
     qkv.rope_table = s->rope_table;
-    L.run(kKindGemv, [&] { return gemv(ly.wqkv, s->h, B, nullptr, 1, nullptr, &qkv, s, L.count, tiles, stream); });
+    return call_of(ly.wqkv, s->h, nullptr, 1, nullptr, qkv);
+  };
+  auto chain = [&](const boost_gemv_call_t* calls, uint32_t n) {
+    return boosth::gemv_chain_launch(calls, n, B, s->gemv_ws, usable, slots.take(s, usable, n + 1), tiles, stream);
+  };
+
+  L.run(kKindGlue, [&] { return boost_rope_table(ctx_lens, B, d, m->rope_base, s->rope_table, stream); });
+  L.run(kKindGlue, [&] {
+    return boost_embed_gather_ssq(m->embed, m->vocab, m->hidden, tokens, B, s->h, s->ssq_a, s->ssq_stride, stream);
+  });
+  {
+    const boost_gemv_call_t first = qkv_call(m->layers[0]);
+    L.run(kKindGemv, [&] { return chain(&first, 1); });
+  }
+  for (uint32_t li = 0; li < m->n_layers && L.ok(); ++li) {
+    const boost_llama_layer_t& ly = m->layers[li];
     L.run(kKindAttn, [&] {
       return boost_paged_attn_decode_tiered(s->q_rot, ly.k_page_ptr, ly.v_page_ptr, m->kv_tier,
                                             (size_t)m->n_kv_pages, m->n_pool_blocks, block_table, max_blocks,
                                             ctx_lens, B, hq, hkv, d, scale, s->attn_ws, s->attn_ws_bytes,
                                             s->attn, stream);
     });
-    // h += attn Wo^T, row statistics of the new h into ssq_b
+    // One launch for the four products between two attention kernels:
+    //   h += attn Wo^T                       (row statistics of the new h into ssq_b)
+    //   act = swiglu(rmsnorm(h) Wgu^T)       (row scale from ssq_b)
+    //   h += act Wd^T                        (row statistics of the new h into ssq_a)
+    //   next layer's q, k, v - or the logits = rmsnorm(h) Whead^T after the last layer
     boost_gemv_epilogue_t wo = stats;
     wo.ssq_out = s->ssq_b;
-    L.run(kKindGemv, [&] { return gemv(ly.wo, s->attn, B, s->h, 1, s->h, &wo, s, L.count, tiles, stream); });
-    // act = swiglu(rmsnorm(h) Wgu^T): row scale from ssq_b
     boost_gemv_epilogue_t gu = scaled;
     gu.mode = BOOST_EPI_SWIGLU;
     gu.ssq_in = s->ssq_b;
-    L.run(kKindGemv, [&] { return gemv(ly.wgu, s->h, B, s->act, 1, nullptr, &gu, s, L.count, tiles, stream); });
-    // h += act Wd^T, row statistics of the new h into ssq_a
     boost_gemv_epilogue_t wd = stats;
     wd.ssq_out = s->ssq_a;
-    L.run(kKindGemv, [&] { return gemv(ly.wd, s->act, B, s->h, 1, s->h, &wd, s, L.count, tiles, stream); });
+    boost_gemv_epilogue_t head = scaled;
+    head.ssq_in = s->ssq_a;
+    boost_gemv_call_t calls[4] = {
+        call_of(ly.wo, s->attn, s->h, 1, s->h, wo), call_of(ly.wgu, s->h, s->act, 1, nullptr, gu),
+        call_of(ly.wd, s->act, s->h, 1, s->h, wd),
+        li + 1 < m->n_layers ? qkv_call(m->layers[li + 1]) : call_of(m->lm_head, s->h, s->logits, 0, nullptr, head)};
+    L.run(kKindGemv, [&] { return chain(calls, 4); });
   }
-  boost_gemv_epilogue_t head = scaled;
-  head.ssq_in = s->ssq_a;
-  L.run(kKindGemv, [&] { return gemv(m->lm_head, s->h, B, s->logits, 0, nullptr, &head, s, L.count, tiles, stream); });
   L.run(kKindGlue, [&] { return boost_argmax(s->logits, B, m->vocab, next_tokens, stream); });
   return L.rc;
 }
@@ -170,10 +196,10 @@ extern "C" int boost_llama_decode_step_profile(const boost_llama_model_t* m, con
                                                int32_t* next_tokens, float* kind_ms_out,
                                                uint32_t* kind_launches_out, void* stream) {
   if (!kind_ms_out || !kind_launches_out || !m) return BOOST_ERR_INVALID;
-  if (2 + 5 * (uint64_t)m->n_layers + 2 > 512) return BOOST_ERR_UNSUPPORTED;
+  if (4 + 2 * (uint64_t)m->n_layers > 512) return BOOST_ERR_UNSUPPORTED;
   static thread_local Launcher L;
   L.stream = stream; L.timed = true; L.count = 0; L.rc = BOOST_OK;
-  const uint32_t n_events = 2 * (2 + 5 * m->n_layers + 2);
+  const uint32_t n_events = 2 * (4 + 2 * m->n_layers);
   uint32_t made = 0;
   int rc = BOOST_OK;
   for (; made < n_events && rc == BOOST_OK; ++made) rc = boosth::check(cudaEventCreate(&L.ev[made]));

@@ -100,6 +100,24 @@ __device__ __forceinline__ void pdl_launch_dependents() {
 }
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
+// Wait until the counter at `ctr` (raised once by every threadblock of the grid) reaches
+// `target`: the grid barrier between two phases of one persistent kernel.  All threadblocks of
+// such a kernel are resident at once (the host sizes the grid from the occupancy), so the
+// counter always gets there; the wait is bounded all the same and records a timeout.
+__device__ __forceinline__ void grid_counter_wait(const uint32_t* ctr, uint32_t target, uint32_t* status) {
+  const long long t0 = clock64();
+  for (;;) {
+    uint32_t v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(ctr) : "memory");
+    if (v >= target) return;
+    if (clock64() - t0 > kWaitLimitCycles) {
+      atomicOr(status, kErrWaitTimeout);
+      return;
+    }
+    __nanosleep(32);
+  }
+}
+
 __device__ __forceinline__ void named_barrier_sync(uint32_t id, uint32_t n_threads) {
   asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(n_threads) : "memory");
 }

@@ -48,6 +48,12 @@ int gemv_tiered_launch(const void* const* w_page_ptr, const uint32_t* w_order, s
                        const boost_gemv_epilogue_t* epilogue, uint32_t* queue_words, uint32_t header_row_tiles,
                        void* stream);
 
+// A chain of 1..4 products in one launch (see boost_gemv_tiered_chain).  sync_words: 16 zeroed
+// uint32 per product (its queue words) followed by 16 more (phase counters), private to this
+// launch among the launches in flight.
+int gemv_chain_launch(const boost_gemv_call_t* calls, uint32_t n_calls, uint32_t M_b, void* workspace,
+                      size_t workspace_bytes, uint32_t* sync_words, uint32_t header_row_tiles, void* stream);
+
 // Bytes of the counter area for n_row_tiles row tiles, and of the partial sums of one product.
 size_t gemv_header_bytes(uint32_t n_row_tiles);
 size_t gemv_partial_bytes(uint32_t N, uint32_t K, uint32_t M_b);

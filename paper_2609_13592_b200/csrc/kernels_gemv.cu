@@ -31,19 +31,21 @@ constexpr uint32_t kMaxStages = 16;
 constexpr uint32_t kSmemBudget = 224u * 1024u;
 constexpr uint32_t kXRowStride = 144;  // 128 data bytes + 16: 8 consecutive rows hit distinct banks
 
-enum : uint32_t { kFlagFirst = 1u, kFlagLast = 2u, kFlagStop = 4u };
+enum : uint32_t { kFlagFirst = 1u, kFlagLast = 2u, kFlagStop = 4u, kFlagPhaseEnd = 8u };
+constexpr uint32_t kMaxPhases = 4;
 enum : uint32_t { kEpiPlain = 0u, kEpiSwiglu = 1u, kEpiRope = 2u };
 
 #ifdef BOOST_TRACE
 // Debug build only: per-threadblock time stamps (global timer, ns) for timeline analysis.
+// 64 slots per threadblock: 0 start, 7 exit, 8 + 8 * phase + k for the events of a phase.
 __device__ unsigned long long* g_trace = nullptr;
 __device__ __forceinline__ unsigned long long gtime() {
   unsigned long long t;
   asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
   return t;
 }
-#define TRACE(slot) do { if (g_trace && (threadIdx.x & 31) == 0) g_trace[(size_t)blockIdx.x * 16 + (slot)] = gtime(); } while (0)
-#define TRACE_ONCE(slot) do { if (g_trace && (threadIdx.x & 31) == 0 && g_trace[(size_t)blockIdx.x * 16 + (slot)] == 0) g_trace[(size_t)blockIdx.x * 16 + (slot)] = gtime(); } while (0)
+#define TRACE(slot) do { if (g_trace && (threadIdx.x & 31) == 0) g_trace[(size_t)blockIdx.x * 64 + (slot)] = gtime(); } while (0)
+#define TRACE_ONCE(slot) do { if (g_trace && (threadIdx.x & 31) == 0 && g_trace[(size_t)blockIdx.x * 64 + (slot)] == 0) g_trace[(size_t)blockIdx.x * 64 + (slot)] = gtime(); } while (0)
 #else
 #define TRACE(slot) do { } while (0)
 #define TRACE_ONCE(slot) do { } while (0)
@@ -78,6 +80,30 @@ struct GemvParams {
   float* partials;     // [row_tile][split][x_rows][128]
   uint32_t n_host_ctas;
   uint32_t n_stages;
+  uint32_t active_ctas;   // threadblocks [0, active_ctas) take this product's items (an even share each)
+  // Even partition (weights with no host page): threadblock c of active_ctas streams the blocks
+  // [c T / G, (c + 1) T / G) of the packed matrix, T = total_blocks, cut into segments at row-tile
+  // boundaries; a row tile's partial sums then come from the consecutive threadblocks that
+  // touch it.  Every SM carries the same number of bytes, which is what HBM-bound work needs.
+  uint32_t even_part, total_blocks;
+  uint32_t max_seg;       // partial-sum slots per row tile (= splits with the queues)
+};
+
+// First / last threadblock of the even partition that holds a block of row tile `t`.
+__device__ __forceinline__ uint32_t part_owner(uint64_t block, uint32_t G, uint32_t T) {
+  return (uint32_t)(((block + 1) * G - 1) / T);
+}
+
+// A launch runs one product, or a chain of up to kMaxPhases products in which each takes the
+// previous one's output (as its x, its residual or its row statistics).  The threadblocks stay
+// resident; between two phases they meet at a grid-wide counter, and because weights do not
+// depend on activations the weight warps stream the next phase's blocks into their rings
+// while the tail of the current phase (last items, partial sums, combine) is still running.
+// M_b, ws, n_stages and early are those of phase 0.
+struct ChainParams {
+  uint32_t n_phases;
+  uint32_t* bar;   // n_phases > 1: counters [kMaxPhases + 1], zero at rest (one per phase boundary, one for the exit)
+  GemvParams ph[kMaxPhases];
 };
 
 __host__ __device__ constexpr uint32_t x_rows_of(int NT, int MB) { return NT > 0 ? NT * 8 : MB; }
@@ -87,7 +113,7 @@ __host__ __device__ constexpr uint32_t stage_bytes_of(int NT, int MB) {
 
 __device__ __forceinline__ void store_out(const GemvParams& p, uint32_t m, uint32_t n, float v) {
   const size_t idx = (size_t)m * p.N + n;
-  if (p.residual) v += __bfloat162float(p.residual[idx]);
+  if (p.residual) v += bf16_lo((uint32_t)__ldcg(reinterpret_cast<const unsigned short*>(p.residual) + idx));
   if (p.y_dtype == 0) static_cast<float*>(p.y)[idx] = v;
   else static_cast<__nv_bfloat16*>(p.y)[idx] = __float2bfloat16_rn(v);
 }
@@ -114,8 +140,9 @@ __device__ __forceinline__ float round_bf16(float v) { return __bfloat162float(_
 // The row scale is rsqrt(mean(x^2) + eps) from per-tile sums of squares of the rows of x:
 // RMSNorm whose weight has been folded into the packed matrix.
 template <uint32_t kXRows>
-__device__ __forceinline__ void combine_tile(const GemvParams& p, uint32_t row_tile, uint32_t tid, uint32_t* status) {
-  const float4* base = reinterpret_cast<const float4*>(p.partials + (size_t)row_tile * p.splits * kXRows * kBlockRows);
+__device__ __forceinline__ void combine_tile(const GemvParams& p, uint32_t row_tile, uint32_t n_seg, uint32_t tid,
+                                             uint32_t* status) {
+  const float4* base = reinterpret_cast<const float4*>(p.partials + (size_t)row_tile * p.max_seg * kXRows * kBlockRows);
   constexpr uint32_t kVecRow = kBlockRows / 4;   // float4 per batch row
   const uint32_t n_pairs = p.M_b * 16;
   for (uint32_t pidx0 = 0; pidx0 < n_pairs; pidx0 += kConsumerThreads) {
@@ -124,13 +151,31 @@ __device__ __forceinline__ void combine_tile(const GemvParams& p, uint32_t row_t
     const uint32_t m = valid ? (pidx >> 4) : 0u, v = pidx & 15u;
     const uint32_t off = m * kVecRow + v;
     float4 lo = make_float4(0.f, 0.f, 0.f, 0.f), hi = lo;
+    // Everything this thread needs from memory is requested before the first use, so that the
+    // L2 round trips overlap: its share of the row statistics, the residual, the partial sums.
+    float ss = 0.f, ss0 = 0.f, ss1 = 0.f;
+    if (p.ssq_in && valid) {
+      // the 16 threads of row m take every 16th tile each; a butterfly adds the shares
+      if (v < p.ssq_in_tiles) ss0 = __ldcg(p.ssq_in + (size_t)v * p.ssq_stride + m);
+      if (v + 16 < p.ssq_in_tiles) ss1 = __ldcg(p.ssq_in + (size_t)(v + 16) * p.ssq_stride + m);
+      for (uint32_t t0 = v + 32; t0 < p.ssq_in_tiles; t0 += 16) ss += __ldcg(p.ssq_in + (size_t)t0 * p.ssq_stride + m);
+    }
+    const bool vec_out = (p.N & 3u) == 0;   // then n + 3 < N for every n = 4 v' < N
+    uint2 res[2] = {make_uint2(0u, 0u), make_uint2(0u, 0u)};
+    if (valid && p.epi == kEpiPlain && p.residual && vec_out) {
+#pragma unroll
+      for (int half = 0; half < 2; ++half) {
+        const uint32_t n = row_tile * kBlockRows + half * 64 + v * 4;
+        if (n < p.N) res[half] = __ldcg(reinterpret_cast<const uint2*>(p.residual + (size_t)m * p.N + n));   // L2: an earlier phase may have rewritten it
+      }
+    }
     if (valid) {
       // four splits (eight independent loads) per round: the L2 latency is paid per round
-      for (uint32_t sp0 = 0; sp0 < p.splits; sp0 += 4) {
+      for (uint32_t sp0 = 0; sp0 < n_seg; sp0 += 4) {
         float4 t0[4], t1[4];
 #pragma unroll
         for (uint32_t u = 0; u < 4; ++u) {
-          if (sp0 + u < p.splits) {
+          if (sp0 + u < n_seg) {
             const float4* src = base + (size_t)(sp0 + u) * kXRows * kVecRow + off;
             t0[u] = __ldcg(src);
             t1[u] = __ldcg(src + 16);
@@ -138,27 +183,22 @@ __device__ __forceinline__ void combine_tile(const GemvParams& p, uint32_t row_t
         }
 #pragma unroll
         for (uint32_t u = 0; u < 4; ++u) {
-          if (sp0 + u < p.splits) {
+          if (sp0 + u < n_seg) {
             lo.x += t0[u].x; lo.y += t0[u].y; lo.z += t0[u].z; lo.w += t0[u].w;
             hi.x += t1[u].x; hi.y += t1[u].y; hi.z += t1[u].z; hi.w += t1[u].w;
           }
         }
       }
-      if (p.ssq_in) {
-        float ss = 0.f;
-        for (uint32_t t0 = 0; t0 < p.ssq_in_tiles; t0 += 8) {
-          float q[8];
-#pragma unroll
-          for (uint32_t u = 0; u < 8; ++u)
-            if (t0 + u < p.ssq_in_tiles) q[u] = __ldcg(p.ssq_in + (size_t)(t0 + u) * p.ssq_stride + m);
-#pragma unroll
-          for (uint32_t u = 0; u < 8; ++u)
-            if (t0 + u < p.ssq_in_tiles) ss += q[u];
-        }
-        const float rs = rsqrtf(ss / (float)p.x_cols + p.rms_eps);
-        lo.x *= rs; lo.y *= rs; lo.z *= rs; lo.w *= rs;
-        hi.x *= rs; hi.y *= rs; hi.z *= rs; hi.w *= rs;
-      }
+    }
+    if (p.ssq_in) {
+      ss += ss0 + ss1;
+      ss += __shfl_xor_sync(0xFFFFFFFFu, ss, 1);
+      ss += __shfl_xor_sync(0xFFFFFFFFu, ss, 2);
+      ss += __shfl_xor_sync(0xFFFFFFFFu, ss, 4);
+      ss += __shfl_xor_sync(0xFFFFFFFFu, ss, 8);
+      const float rs = rsqrtf(ss / (float)p.x_cols + p.rms_eps);
+      lo.x *= rs; lo.y *= rs; lo.z *= rs; lo.w *= rs;
+      hi.x *= rs; hi.y *= rs; hi.z *= rs; hi.w *= rs;
     }
     if (p.epi == kEpiPlain) {
       float sq = 0.f;
@@ -168,10 +208,10 @@ __device__ __forceinline__ void combine_tile(const GemvParams& p, uint32_t row_t
         for (int half = 0; half < 2; ++half) {
           const uint32_t n = row_tile * kBlockRows + half * 64 + v * 4;
           float e[4] = {val[half].x, val[half].y, val[half].z, val[half].w};
-          if (n + 3 < p.N && (p.N & 3u) == 0) {
+          if (n + 3 < p.N && vec_out) {
             const size_t idx = (size_t)m * p.N + n;
             if (p.residual) {
-              const uint2 r = *reinterpret_cast<const uint2*>(p.residual + idx);
+              const uint2 r = res[half];
               e[0] += bf16_lo(r.x); e[1] += bf16_hi(r.x); e[2] += bf16_lo(r.y); e[3] += bf16_hi(r.y);
             }
             if (p.y_dtype == 0) {
@@ -186,7 +226,7 @@ __device__ __forceinline__ void combine_tile(const GemvParams& p, uint32_t row_t
             for (int j = 0; j < 4; ++j)
               if (n + j < p.N) {
                 float x = e[j];
-                if (p.residual) x += __bfloat162float(p.residual[(size_t)m * p.N + n + j]);
+                if (p.residual) x += bf16_lo((uint32_t)__ldcg(reinterpret_cast<const unsigned short*>(p.residual) + (size_t)m * p.N + n + j));
                 if (p.y_dtype == 0) static_cast<float*>(p.y)[(size_t)m * p.N + n + j] = x;
                 else {
                   static_cast<__nv_bfloat16*>(p.y)[(size_t)m * p.N + n + j] = __float2bfloat16_rn(x);
@@ -263,7 +303,7 @@ __device__ __forceinline__ void combine_tile(const GemvParams& p, uint32_t row_t
 
 // NT > 0: tensor-core path with NT batch tiles of 8; NT == 0: CUDA-core path for MB rows.
 template <int NT, int MB>
-__global__ void __launch_bounds__(kGemvThreads, (NT >= 8 ? 1 : 2)) gemv_tiered_kernel(const __grid_constant__ GemvParams p) {
+__global__ void __launch_bounds__(kGemvThreads, (NT >= 8 ? 1 : 2)) gemv_tiered_kernel(const __grid_constant__ ChainParams cp) {
   constexpr uint32_t kXRows = x_rows_of(NT, MB);
   constexpr uint32_t kStageBytes = stage_bytes_of(NT, MB);
   extern __shared__ uint8_t smem_raw[];
@@ -277,8 +317,9 @@ __global__ void __launch_bounds__(kGemvThreads, (NT >= 8 ? 1 : 2)) gemv_tiered_k
   __shared__ uint32_t s_old;
 
   const uint32_t tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const uint32_t n_stages = p.n_stages;
-  uint32_t* status = p.ws + kWsStatus;
+  const uint32_t n_stages = cp.ph[0].n_stages;
+  const uint32_t n_phases = cp.n_phases;
+  uint32_t* status = cp.ph[0].ws + kWsStatus;
 
   if (tid == 0) TRACE(0);
   pdl_launch_dependents();
@@ -301,99 +342,155 @@ __global__ void __launch_bounds__(kGemvThreads, (NT >= 8 ? 1 : 2)) gemv_tiered_k
     // sequence (handed over through a four-slot ring) and loads the matching slices of x.
     // Two warps, because a lone warp's instruction latency would cap the fill rate.
     const bool leader = (warp == kConsumerWarps);
-    const uint32_t n_host_items = p.n_host_pages * p.items_per_page;
-    TierQueues q;
-    q.init(p.queue, n_host_items, p.n_pages * p.items_per_page, p.n_host_ctas, blockIdx.x, gridDim.x);
-    // Weights are never written by the decode chain, so with private queue words the weight
-    // warp starts streaming while the previous kernel is still running; x is produced by
-    // that kernel, so the x warp (and the consumers) wait for it.
-    if (!leader || !p.early) pdl_wait();
     uint32_t stage = 0, phase = 0, icount = 0;
-    for (;;) {
-      const uint32_t slot = icount & 3u, iphase = (icount >> 2) & 1u;
-      uint32_t qi = 0;
+    for (uint32_t ph = 0; ph < n_phases; ++ph) {
+      const GemvParams& p = cp.ph[ph];
+      const uint32_t n_host_items = p.n_host_pages * p.items_per_page;
+      TierQueues q;
+      const bool active = blockIdx.x < p.active_ctas;
+      if (active && !p.even_part) q.init(p.queue, n_host_items, p.n_pages * p.items_per_page, p.n_host_ctas, blockIdx.x, p.active_ctas);
+      if (ph == 0) {
+        // Weights are never written by the decode chain, so with private queue words the weight
+        // warp starts streaming while the previous kernel is still running; x is produced by
+        // that kernel, so the x warp (and the consumers) wait for it.
+        if (!leader || !p.early) pdl_wait();
+      } else if (!leader) {
+        // x of this phase is what the previous phase wrote: wait until every threadblock has
+        // finished it.  The weight warp does not wait: it fills the ring meanwhile.
+        if (lane == 0) grid_counter_wait(cp.bar + (ph - 1), gridDim.x, status);
+        __syncwarp();
+      }
+      if (!leader) TRACE(8 + 8 * ph + 2);
+      if (p.even_part) {
+        // Even partition: both warps walk the same static block range, no queue.
+        const uint32_t G = p.active_ctas, T = p.total_blocks;
+        if (blockIdx.x < G) {
+          const uint32_t b0 = (uint32_t)((uint64_t)blockIdx.x * T / G), b1 = (uint32_t)((uint64_t)(blockIdx.x + 1) * T / G);
+          uint32_t row_tile = b0 / p.k_blocks, kb = b0 % p.k_blocks;
+          uint32_t seg = blockIdx.x - part_owner((uint64_t)row_tile * p.k_blocks, G, T);
+          if (leader && b0 < b1) TRACE_ONCE(8 + 8 * ph + 0);
+          const uint32_t c = lane & 7, m0 = lane >> 3;
+          for (uint32_t b = b0; b < b1; ++b) {
+            const bool seg_first = (b == b0) || kb == 0, seg_last = (b + 1 == b1) || (kb + 1 == p.k_blocks);
+            if (leader) {
+              uint8_t* wdst = smem + (size_t)stage * kStageBytes;
+              if (lane == 0) {
+                const uint8_t* src = static_cast<const uint8_t*>(p.w_page_ptr[b / kBlocksPerPage]) +
+                                     (size_t)(b % kBlocksPerPage) * kBlockBytes;
+                mbar_wait(&empty_bar[stage], phase ^ 1u, status);
+                meta[stage] = make_uint4(row_tile, seg, (seg_first ? kFlagFirst : 0u) | (seg_last ? kFlagLast : 0u), ph);
+                mbar_arrive_expect_tx(&full_bar[stage], kBlockBytes);
+                bulk_copy_g2s(wdst, src, kBlockBytes, &full_bar[stage]);
+              }
+              __syncwarp();
+              cp_async_arrive_noinc(&full_bar[stage]);
+            } else {
+              mbar_wait(&empty_bar[stage], phase ^ 1u, status);
+              uint8_t* xdst = smem + (size_t)stage * kStageBytes + kBlockBytes + m0 * kXRowStride + c * 16;
+              const uint32_t k = kb * kBlockK + c * 8;
+              const bool k_ok = k < p.K;
+              const __nv_bfloat16* xs = p.x + (size_t)m0 * p.K + (k_ok ? k : 0u);
+#pragma unroll 4
+              for (uint32_t m = m0; m < kXRows; m += 4) {
+                cp_async_16(xdst, xs, (k_ok && m < p.M_b) ? 16u : 0u);
+                xdst += 4 * kXRowStride;
+                if (m + 4 < p.M_b) xs += (size_t)4 * p.K;
+              }
+              cp_async_arrive_noinc(&full_bar[stage]);
+            }
+            if (++stage == n_stages) { stage = 0; phase ^= 1u; }
+            if (++kb == p.k_blocks) { kb = 0; ++row_tile; seg = 0; }
+          }
+        }
+      } else
+      for (;;) {
+        const uint32_t slot = icount & 3u, iphase = (icount >> 2) & 1u;
+        uint32_t qi = 0;
+        if (leader) {
+          if (lane == 0) {
+            for (;;) {   // skip the unused tail of the last page
+              qi = active ? q.next() : 0xFFFFFFFFu;
+              if (qi == 0xFFFFFFFFu) break;
+              if (p.w_order[qi / p.items_per_page] * p.items_per_page + qi % p.items_per_page < p.n_items) break;
+            }
+            mbar_wait(&item_empty[slot], iphase ^ 1u, status);
+            item_ring[slot] = qi;
+            mbar_arrive(&item_full[slot]);
+          }
+          qi = __shfl_sync(0xFFFFFFFFu, qi, 0);
+        } else {
+          mbar_wait(&item_full[slot], iphase, status);
+          qi = item_ring[slot];
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&item_empty[slot]);
+        }
+        ++icount;
+        if (leader && qi != 0xFFFFFFFFu) TRACE_ONCE(8 + 8 * ph + 0);
+        if (qi == 0xFFFFFFFFu) break;
+        const uint32_t page = p.w_order[qi / p.items_per_page];
+        const uint32_t first_blk = (page * p.items_per_page + qi % p.items_per_page) * p.run;
+        const uint32_t row_tile = first_blk / p.k_blocks;
+        const uint32_t kb0 = first_blk % p.k_blocks;
+        const bool from_host = qi < n_host_items;
+        if (leader) {
+          const uint8_t* src = static_cast<const uint8_t*>(p.w_page_ptr[page]) +
+                               (size_t)(first_blk % kBlocksPerPage) * kBlockBytes;
+          for (uint32_t j = 0; j < p.run; ++j, src += kBlockBytes) {
+            uint8_t* wdst = smem + (size_t)stage * kStageBytes;
+            if (lane == 0) {
+              mbar_wait(&empty_bar[stage], phase ^ 1u, status);
+              meta[stage] = make_uint4(row_tile, kb0 / p.run,
+                                       (j == 0 ? kFlagFirst : 0u) | (j + 1 == p.run ? kFlagLast : 0u), ph);
+              mbar_arrive_expect_tx(&full_bar[stage], from_host ? 0u : kBlockBytes);
+              if (!from_host) bulk_copy_g2s(wdst, src, kBlockBytes, &full_bar[stage]);
+            }
+            __syncwarp();   // the other lanes must not run ahead of lane 0's wait on the stage
+            if (from_host) {
+              // host page: a fan of 16-byte loads through the load/store path keeps many
+              // requests on the link at once (Sec. 3.2: this threadblock is a host-tier block)
+#pragma unroll 8
+              for (uint32_t idx = lane; idx < kBlockBytes / 16; idx += 32)
+                cp_async_16(wdst + idx * 16, src + idx * 16, 16u);
+            }
+            cp_async_arrive_noinc(&full_bar[stage]);
+            if (++stage == n_stages) { stage = 0; phase ^= 1u; }
+          }
+        } else {
+          // lane -> (row m0 + 4 i, 16-byte chunk c); pointers advance by constants
+          const uint32_t c = lane & 7, m0 = lane >> 3;
+          for (uint32_t j = 0; j < p.run; ++j) {
+            mbar_wait(&empty_bar[stage], phase ^ 1u, status);
+            uint8_t* xdst = smem + (size_t)stage * kStageBytes + kBlockBytes + m0 * kXRowStride + c * 16;
+            const uint32_t k = (kb0 + j) * kBlockK + c * 8;
+            const bool k_ok = k < p.K;
+            const __nv_bfloat16* xs = p.x + (size_t)m0 * p.K + (k_ok ? k : 0u);
+#pragma unroll 4
+            for (uint32_t m = m0; m < kXRows; m += 4) {
+              cp_async_16(xdst, xs, (k_ok && m < p.M_b) ? 16u : 0u);
+              xdst += 4 * kXRowStride;
+              if (m + 4 < p.M_b) xs += (size_t)4 * p.K;
+            }
+            cp_async_arrive_noinc(&full_bar[stage]);
+            if (++stage == n_stages) { stage = 0; phase ^= 1u; }
+          }
+        }
+      }
+      // a stage without data tells the consumers that the phase (or the launch) is over
+      if (leader) TRACE(8 + 8 * ph + 1);
       if (leader) {
         if (lane == 0) {
-          for (;;) {   // skip the unused tail of the last page
-            qi = q.next();
-            if (qi == 0xFFFFFFFFu) break;
-            if (p.w_order[qi / p.items_per_page] * p.items_per_page + qi % p.items_per_page < p.n_items) break;
-          }
-          mbar_wait(&item_empty[slot], iphase ^ 1u, status);
-          item_ring[slot] = qi;
-          mbar_arrive(&item_full[slot]);
-        }
-        qi = __shfl_sync(0xFFFFFFFFu, qi, 0);
-      } else {
-        mbar_wait(&item_full[slot], iphase, status);
-        qi = item_ring[slot];
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&item_empty[slot]);
-      }
-      ++icount;
-      if (leader) TRACE_ONCE(1);
-      if (qi == 0xFFFFFFFFu) break;
-      const uint32_t page = p.w_order[qi / p.items_per_page];
-      const uint32_t first_blk = (page * p.items_per_page + qi % p.items_per_page) * p.run;
-      const uint32_t row_tile = first_blk / p.k_blocks;
-      const uint32_t kb0 = first_blk % p.k_blocks;
-      const bool from_host = qi < n_host_items;
-      if (leader) {
-        const uint8_t* src = static_cast<const uint8_t*>(p.w_page_ptr[page]) +
-                             (size_t)(first_blk % kBlocksPerPage) * kBlockBytes;
-        for (uint32_t j = 0; j < p.run; ++j, src += kBlockBytes) {
-          uint8_t* wdst = smem + (size_t)stage * kStageBytes;
-          if (lane == 0) {
-            mbar_wait(&empty_bar[stage], phase ^ 1u, status);
-            meta[stage] = make_uint4(row_tile, kb0 / p.run,
-                                     (j == 0 ? kFlagFirst : 0u) | (j + 1 == p.run ? kFlagLast : 0u), 0u);
-            mbar_arrive_expect_tx(&full_bar[stage], from_host ? 0u : kBlockBytes);
-            if (!from_host) bulk_copy_g2s(wdst, src, kBlockBytes, &full_bar[stage]);
-          }
-          __syncwarp();   // the other lanes must not run ahead of lane 0's wait on the stage
-          if (from_host) {
-            // host page: a fan of 16-byte loads through the load/store path keeps many
-            // requests on the link at once (Sec. 3.2: this threadblock is a host-tier block)
-#pragma unroll 8
-            for (uint32_t idx = lane; idx < kBlockBytes / 16; idx += 32)
-              cp_async_16(wdst + idx * 16, src + idx * 16, 16u);
-          }
-          cp_async_arrive_noinc(&full_bar[stage]);
-          if (++stage == n_stages) { stage = 0; phase ^= 1u; }
-        }
-      } else {
-        // lane -> (row m0 + 4 i, 16-byte chunk c); pointers advance by constants
-        const uint32_t c = lane & 7, m0 = lane >> 3;
-        for (uint32_t j = 0; j < p.run; ++j) {
           mbar_wait(&empty_bar[stage], phase ^ 1u, status);
-          uint8_t* xdst = smem + (size_t)stage * kStageBytes + kBlockBytes + m0 * kXRowStride + c * 16;
-          const uint32_t k = (kb0 + j) * kBlockK + c * 8;
-          const bool k_ok = k < p.K;
-          const __nv_bfloat16* xs = p.x + (size_t)m0 * p.K + (k_ok ? k : 0u);
-#pragma unroll 4
-          for (uint32_t m = m0; m < kXRows; m += 4) {
-            cp_async_16(xdst, xs, (k_ok && m < p.M_b) ? 16u : 0u);
-            xdst += 4 * kXRowStride;
-            if (m + 4 < p.M_b) xs += (size_t)4 * p.K;
-          }
-          cp_async_arrive_noinc(&full_bar[stage]);
-          if (++stage == n_stages) { stage = 0; phase ^= 1u; }
+          meta[stage] = make_uint4(0u, 0u, ph + 1 == n_phases ? kFlagStop : kFlagPhaseEnd, ph);
+          mbar_arrive(&full_bar[stage]);
         }
-      }
-    }
-    // tell the consumers to stop
-    if (leader) {
-      if (lane == 0) {
+        __syncwarp();
+        cp_async_arrive_noinc(&full_bar[stage]);
+        if (lane == 0 && active && !p.even_part) q.finish(p.active_ctas);
+      } else {
         mbar_wait(&empty_bar[stage], phase ^ 1u, status);
-        meta[stage] = make_uint4(0u, 0u, kFlagStop, 0u);
-        mbar_arrive(&full_bar[stage]);
+        cp_async_arrive_noinc(&full_bar[stage]);
       }
-      __syncwarp();
-      cp_async_arrive_noinc(&full_bar[stage]);
-      if (lane == 0) q.finish(gridDim.x);
-    } else {
-      mbar_wait(&empty_bar[stage], phase ^ 1u, status);
-      cp_async_arrive_noinc(&full_bar[stage]);
+      if (++stage == n_stages) { stage = 0; phase ^= 1u; }
     }
     return;
   }
@@ -407,14 +504,40 @@ __global__ void __launch_bounds__(kGemvThreads, (NT >= 8 ? 1 : 2)) gemv_tiered_k
 #pragma unroll
     for (int j = 0; j < kAccM; ++j) acc[i][j] = 0.f;
 
-  uint32_t* tile_cnt = p.ws + kWsHeaderWords;
+  uint32_t* tile_cnt = cp.ph[0].ws + kWsHeaderWords;
   uint32_t stage = 0, phase = 0;
   pdl_wait();
   for (;;) {
     mbar_wait(&full_bar[stage], phase, status);
     const uint4 mt = meta[stage];
-    if (warp == 0) TRACE_ONCE(2);
-    if (mt.z & kFlagStop) break;
+    if (mt.z & (kFlagStop | kFlagPhaseEnd)) {
+      if (warp == 0) TRACE(8 + 8 * mt.w + 4);
+      if (n_phases > 1) {
+        // every consumer thread has finished this phase's items, combines included: publish
+        // them and tell the grid (the x warps of all threadblocks wait for the count)
+        named_barrier_sync(1, kConsumerThreads);
+        if (tid == 0) {
+          __threadfence();
+          if (mt.z & kFlagPhaseEnd) {
+            atomicAdd(cp.bar + mt.w, 1u);
+          } else {
+            // last threadblock out puts the counters back to zero for the next launch; by then
+            // every x warp has passed every phase boundary (its stop stage came after them)
+            const uint32_t old = atomicAdd(cp.bar + kMaxPhases, 1u);
+            if (old == gridDim.x - 1) {
+              for (uint32_t i = 0; i <= kMaxPhases; ++i) cp.bar[i] = 0u;
+              __threadfence();
+            }
+          }
+        }
+      }
+      if (mt.z & kFlagStop) break;
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&empty_bar[stage]);
+      if (++stage == n_stages) { stage = 0; phase ^= 1u; }
+      continue;
+    }
+    if (warp == 0 && (mt.z & kFlagFirst)) TRACE_ONCE(8 + 8 * mt.w + 3);
     if (mt.z & kFlagFirst) {
 #pragma unroll
       for (int i = 0; i < kAccN; ++i)
@@ -472,7 +595,8 @@ __global__ void __launch_bounds__(kGemvThreads, (NT >= 8 ? 1 : 2)) gemv_tiered_k
     if (++stage == n_stages) { stage = 0; phase ^= 1u; }
 
     if (mt.z & kFlagLast) {
-      if (warp == 0) { TRACE_ONCE(3); TRACE(5); }
+      if (warp == 0) TRACE(8 + 8 * mt.w + 6);
+      const GemvParams& p = cp.ph[mt.w];
       const uint32_t row_tile = mt.x, split = mt.y;
       if constexpr (NT == 0) {
         // finish the dot products: sum over the 8 lanes that share a row
@@ -488,8 +612,15 @@ __global__ void __launch_bounds__(kGemvThreads, (NT >= 8 ? 1 : 2)) gemv_tiered_k
           }
       }
       // without splits (and without a row scale, pairing or row statistics) the sums go straight out
-      const bool direct = (p.splits == 1) && p.epi == kEpiPlain && !p.ssq_in && !p.ssq_out;
-      float* part = p.partials + ((size_t)row_tile * p.splits + split) * kXRows * kBlockRows;
+      // partial sums of this row tile: one per split of the queue items, or one per
+      // threadblock of the even partition that holds some of its blocks
+      uint32_t n_seg = p.splits;
+      if (p.even_part) {
+        const uint64_t t0 = (uint64_t)row_tile * p.k_blocks;
+        n_seg = part_owner(t0 + p.k_blocks - 1, p.active_ctas, p.total_blocks) - part_owner(t0, p.active_ctas, p.total_blocks) + 1;
+      }
+      const bool direct = (n_seg == 1) && p.epi == kEpiPlain && !p.ssq_in && !p.ssq_out;
+      float* part = p.partials + ((size_t)row_tile * p.max_seg + split) * kXRows * kBlockRows;
       if constexpr (NT > 0) {
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt)
@@ -529,15 +660,14 @@ __global__ void __launch_bounds__(kGemvThreads, (NT >= 8 ? 1 : 2)) gemv_tiered_k
           s_old = atomicAdd(tile_cnt + row_tile, 1u);
         }
         named_barrier_sync(1, kConsumerThreads);
-        if (s_old == p.splits - 1) {
+        if (s_old == n_seg - 1) {
           __threadfence();
-          combine_tile<kXRows>(p, row_tile, tid, status);
+          combine_tile<kXRows>(p, row_tile, n_seg, tid, status);
           if (tid == 0) tile_cnt[row_tile] = 0;
-          if (warp == 0) TRACE(8);
+          if (warp == 0) TRACE(8 + 8 * mt.w + 5);
         }
         named_barrier_sync(1, kConsumerThreads);
       }
-      if (warp == 0) { TRACE_ONCE(4); TRACE(6); }
     }
   }
   if (warp == 0) TRACE(7);
@@ -598,39 +728,61 @@ uint32_t pick_run(uint32_t n_row_tiles, uint32_t k_blocks) {
 }
 
 template <int NT, int MB>
-int launch_gemv(const GemvParams& p, int sms, cudaStream_t stream) {
+int launch_gemv(const ChainParams& chain, int sms, cudaStream_t stream) {
   constexpr uint32_t kStage = stage_bytes_of(NT, MB);
-  GemvParams q = p;
+  ChainParams c = chain;
   // Two threadblocks per SM where registers allow: a second ring hides the producer /
   // consumer hand-over latency of the first (measured: +25 % bandwidth on B200).
-  const uint32_t ctas_per_sm = (NT >= 8) ? 1 : 2;
+  uint32_t ctas_per_sm = (NT >= 8) ? 1 : 2;
   uint32_t n_stages = (kSmemBudget / ctas_per_sm - 1024) / kStage;
   if (n_stages > kMaxStages) n_stages = kMaxStages;
-  q.n_stages = n_stages;
   const size_t smem = (size_t)n_stages * kStage + 1024;
   static bool configured = false;
+  static int resident = 0;   // threadblocks of this kernel that one SM holds at this shared-memory size
   if (!configured) {
-    const int rc = boosth::check(cudaFuncSetAttribute(gemv_tiered_kernel<NT, MB>,
-                                                      cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(kSmemBudget + 1024)));
+    int rc = boosth::check(cudaFuncSetAttribute(gemv_tiered_kernel<NT, MB>,
+                                                cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(kSmemBudget + 1024)));
+    if (rc != BOOST_OK) return rc;
+    rc = boosth::check(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&resident, gemv_tiered_kernel<NT, MB>,
+                                                                     (int)kGemvThreads, smem));
     if (rc != BOOST_OK) return rc;
     configured = true;
   }
-  // Threadblocks share HBM bandwidth, so what has to be even is the number of items per
-  // threadblock: use as many blocks as give every block the same count (rounded up).
-  const uint32_t max_ctas = (uint32_t)sms * ctas_per_sm;
-  const uint32_t queue_len = q.n_pages * q.items_per_page;
-  const uint32_t items = q.n_items ? q.n_items : 1;
-  const uint32_t per_cta = (items + max_ctas - 1) / max_ctas;
-  uint32_t grid = (items + per_cta - 1) / per_cta;
-  if (grid > queue_len) grid = queue_len;
-  uint32_t n_host_ctas = 0;
-  if (q.n_host_pages) {
-    n_host_ctas = 8;
-    if (n_host_ctas > q.n_host_pages * q.items_per_page) n_host_ctas = q.n_host_pages * q.items_per_page;
-    if (n_host_ctas > grid) n_host_ctas = grid;
+  if (c.n_phases > 1) {
+    // the phases of a chain meet at grid-wide counters: every threadblock must be resident
+    if (resident < 1) return BOOST_ERR_UNSUPPORTED;
+    if ((uint32_t)resident < ctas_per_sm) ctas_per_sm = (uint32_t)resident;
   }
-  q.n_host_ctas = n_host_ctas;
-  return boosth::launch_chained(gemv_tiered_kernel<NT, MB>, dim3(grid), dim3(kGemvThreads), smem, stream, q);
+  const uint32_t max_ctas = (uint32_t)sms * ctas_per_sm;
+  uint32_t grid = 0;
+  for (uint32_t i = 0; i < c.n_phases; ++i) {
+    GemvParams& q = c.ph[i];
+    q.n_stages = n_stages;
+    // Threadblocks share HBM bandwidth, so what has to be even is the number of items per
+    // threadblock: use as many blocks as give every block the same count (rounded up).
+    const uint32_t queue_len = q.n_pages * q.items_per_page;
+    const uint32_t items = q.n_items ? q.n_items : 1;
+    const uint32_t per_cta = (items + max_ctas - 1) / max_ctas;
+    uint32_t g = (items + per_cta - 1) / per_cta;
+    if (g > queue_len) g = queue_len;
+    if (q.even_part) g = q.total_blocks < max_ctas ? q.total_blocks : max_ctas;
+    q.active_ctas = g;
+    if (g > grid) grid = g;
+  }
+  // a chain keeps one grid for all phases: the full machine, so that threadblocks that run
+  // out of items in one phase stream ahead in the next
+  if (c.n_phases > 1) grid = max_ctas;
+  for (uint32_t i = 0; i < c.n_phases; ++i) {
+    GemvParams& q = c.ph[i];
+    uint32_t n_host_ctas = 0;
+    if (q.n_host_pages) {
+      n_host_ctas = 8;
+      if (n_host_ctas > q.n_host_pages * q.items_per_page) n_host_ctas = q.n_host_pages * q.items_per_page;
+      if (n_host_ctas > q.active_ctas) n_host_ctas = q.active_ctas;
+    }
+    q.n_host_ctas = n_host_ctas;
+  }
+  return boosth::launch_chained(gemv_tiered_kernel<NT, MB>, dim3(grid), dim3(kGemvThreads), smem, stream, c);
 }
 
 }  // namespace
@@ -688,10 +840,23 @@ size_t boosth::gemv_header_bytes(uint32_t n_row_tiles) {
   return ((size_t)(kWsHeaderWords + n_row_tiles) * 4 + 255) / 256 * 256;
 }
 
+// Partial-sum slots per row tile: the splits of the queue items, or (even partition over G
+// threadblocks, each at least floor(T / G) blocks long) the most threadblocks a tile can touch.
+static uint32_t partial_slots(const boost_weight_layout_t& lay, uint32_t M_b) {
+  int sms = boosth::sm_count();
+  if (sms <= 0) sms = 148;
+  const uint64_t T = (uint64_t)lay.n_row_tiles * lay.k_blocks;
+  uint64_t G = (uint64_t)sms * (gemv_x_rows(M_b) >= 64 ? 1 : 2);
+  if (G > T) G = T;
+  const uint32_t per = (uint32_t)(T / G);
+  const uint32_t even = (lay.k_blocks + per - 1) / per + 1;
+  return even > lay.splits ? even : lay.splits;
+}
+
 size_t boosth::gemv_partial_bytes(uint32_t N, uint32_t K, uint32_t M_b) {
   boost_weight_layout_t lay;
   if (boost_weight_layout(N, K, &lay) != BOOST_OK || M_b == 0 || M_b > 128) return 0;
-  return (size_t)lay.n_row_tiles * lay.splits * gemv_x_rows(M_b) * kBlockRows * 4;
+  return (size_t)lay.n_row_tiles * partial_slots(lay, M_b) * gemv_x_rows(M_b) * kBlockRows * 4;
 }
 
 extern "C" size_t boost_gemv_workspace_bytes(uint32_t N, uint32_t K, uint32_t M_b) {
@@ -718,11 +883,14 @@ extern "C" int boost_gemv_tiered_fused(const void* const* w_page_ptr, const uint
                                     residual, workspace, workspace_bytes, epilogue, nullptr, 0, stream);
 }
 
-int boosth::gemv_tiered_launch(const void* const* w_page_ptr, const uint32_t* w_order, size_t n_pages,
-                               size_t n_host_pages, uint32_t N, uint32_t K, const void* x, uint32_t M_b,
-                               void* y, int y_dtype, const void* residual, void* workspace,
-                               size_t workspace_bytes, const boost_gemv_epilogue_t* epi,
-                               uint32_t* queue_words, uint32_t header_row_tiles, void* stream) {
+namespace {
+
+// Checks one product's arguments and fills its kernel parameters.  `header` = bytes of the
+// counter area at the head of the workspace (the same for all products that share it).
+int fill_params(GemvParams& p, const void* const* w_page_ptr, const uint32_t* w_order, size_t n_pages,
+                size_t n_host_pages, uint32_t N, uint32_t K, const void* x, uint32_t M_b, void* y, int y_dtype,
+                const void* residual, void* workspace, size_t workspace_bytes, const boost_gemv_epilogue_t* epi,
+                uint32_t* queue_words, uint32_t header_row_tiles) {
   const int mode = epi ? epi->mode : BOOST_EPI_PLAIN;
   if (!w_page_ptr || !w_order || !x || !workspace) return BOOST_ERR_INVALID;
   if (!y && mode != BOOST_EPI_ROPE_APPEND) return BOOST_ERR_INVALID;
@@ -742,12 +910,10 @@ int boosth::gemv_tiered_launch(const void* const* w_page_ptr, const uint32_t* w_
   if (rc != BOOST_OK) return rc;
   if (n_pages != lay.n_pages || n_host_pages > n_pages) return BOOST_ERR_INVALID;
   if (K % 8 != 0 || ((uintptr_t)x % 16) != 0 || ((uintptr_t)workspace % 256) != 0) return BOOST_ERR_ALIGN;
-  const size_t header = gemv_header_bytes(header_row_tiles > lay.n_row_tiles ? header_row_tiles : lay.n_row_tiles);
-  if (workspace_bytes < header + gemv_partial_bytes(N, K, M_b)) return BOOST_ERR_CAPACITY;
-  const int sms = boosth::sm_count();
-  if (sms <= 0) return BOOST_ERR_CUDA;
+  const size_t header =
+      boosth::gemv_header_bytes(header_row_tiles > lay.n_row_tiles ? header_row_tiles : lay.n_row_tiles);
+  if (workspace_bytes < header + boosth::gemv_partial_bytes(N, K, M_b)) return BOOST_ERR_CAPACITY;
 
-  GemvParams p;
   p.w_page_ptr = w_page_ptr;
   p.w_order = w_order;
   p.n_pages = (uint32_t)n_pages;
@@ -757,6 +923,9 @@ int boosth::gemv_tiered_launch(const void* const* w_page_ptr, const uint32_t* w_
   p.k_blocks = lay.k_blocks;
   p.run = lay.blocks_per_item;
   p.splits = lay.splits;
+  p.even_part = n_host_pages == 0 ? 1u : 0u;
+  p.total_blocks = lay.n_row_tiles * lay.k_blocks;
+  p.max_seg = partial_slots(lay, M_b);
   p.items_per_page = kBlocksPerPage / lay.blocks_per_item;
   p.n_items = (uint32_t)((uint64_t)lay.n_row_tiles * lay.k_blocks / lay.blocks_per_item);
   p.x = static_cast<const __nv_bfloat16*>(x);
@@ -785,15 +954,87 @@ int boosth::gemv_tiered_launch(const void* const* w_page_ptr, const uint32_t* w_
   p.rope_table = epi ? epi->rope_table : nullptr;
   p.partials = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + header);
   p.n_host_ctas = 0; p.n_stages = 0;
+  return BOOST_OK;
+}
+
+int launch_routed(const ChainParams& c, uint32_t M_b, void* stream) {
+  const int sms = boosth::sm_count();
+  if (sms <= 0) return BOOST_ERR_CUDA;
   cudaStream_t st = (cudaStream_t)stream;
   switch (gemv_x_rows(M_b)) {
-    case 1: return launch_gemv<0, 1>(p, sms, st);
-    case 2: return launch_gemv<0, 2>(p, sms, st);
-    case 16: return launch_gemv<2, 0>(p, sms, st);
-    case 32: return launch_gemv<4, 0>(p, sms, st);
-    case 64: return launch_gemv<8, 0>(p, sms, st);
-    default: return launch_gemv<16, 0>(p, sms, st);
+    case 1: return launch_gemv<0, 1>(c, sms, st);
+    case 2: return launch_gemv<0, 2>(c, sms, st);
+    case 16: return launch_gemv<2, 0>(c, sms, st);
+    case 32: return launch_gemv<4, 0>(c, sms, st);
+    case 64: return launch_gemv<8, 0>(c, sms, st);
+    default: return launch_gemv<16, 0>(c, sms, st);
   }
+}
+
+}  // namespace
+
+int boosth::gemv_tiered_launch(const void* const* w_page_ptr, const uint32_t* w_order, size_t n_pages,
+                               size_t n_host_pages, uint32_t N, uint32_t K, const void* x, uint32_t M_b,
+                               void* y, int y_dtype, const void* residual, void* workspace,
+                               size_t workspace_bytes, const boost_gemv_epilogue_t* epi,
+                               uint32_t* queue_words, uint32_t header_row_tiles, void* stream) {
+  ChainParams c;
+  c.n_phases = 1;
+  c.bar = nullptr;
+  const int rc = fill_params(c.ph[0], w_page_ptr, w_order, n_pages, n_host_pages, N, K, x, M_b, y, y_dtype, residual,
+                             workspace, workspace_bytes, epi, queue_words, header_row_tiles);
+  if (rc != BOOST_OK) return rc;
+  return launch_routed(c, M_b, stream);
+}
+
+int boosth::gemv_chain_launch(const boost_gemv_call_t* calls, uint32_t n_calls, uint32_t M_b, void* workspace,
+                              size_t workspace_bytes, uint32_t* sync_words, uint32_t header_row_tiles,
+                              void* stream) {
+  if (!calls || n_calls == 0 || n_calls > kMaxPhases || !sync_words) return BOOST_ERR_INVALID;
+  uint32_t tiles = header_row_tiles;
+  for (uint32_t i = 0; i < n_calls; ++i) {
+    const uint32_t t = (calls[i].w.N + kBlockRows - 1) / kBlockRows;
+    tiles = t > tiles ? t : tiles;
+  }
+  ChainParams c;
+  c.n_phases = n_calls;
+  c.bar = n_calls > 1 ? sync_words + 16 * n_calls : nullptr;
+  for (uint32_t i = 0; i < n_calls; ++i) {
+    const boost_gemv_call_t& g = calls[i];
+    const int rc = fill_params(c.ph[i], g.w.page_ptr, g.w.order, (size_t)g.w.n_pages, (size_t)g.w.n_host_pages, g.w.N,
+                               g.w.K, g.x, M_b, g.y, g.y_dtype, g.residual, workspace, workspace_bytes,
+                               g.has_epilogue ? &g.epilogue : nullptr, sync_words + 16 * i, tiles);
+    if (rc != BOOST_OK) return rc;
+  }
+  return launch_routed(c, M_b, stream);
+}
+
+extern "C" size_t boost_gemv_chain_workspace_bytes(const boost_gemv_call_t* calls, uint32_t n_calls, uint32_t M_b) {
+  if (!calls || n_calls == 0 || n_calls > kMaxPhases) return 0;
+  uint32_t tiles = 0;
+  size_t partial = 0;
+  for (uint32_t i = 0; i < n_calls; ++i) {
+    const uint32_t t = (calls[i].w.N + kBlockRows - 1) / kBlockRows;
+    tiles = t > tiles ? t : tiles;
+    const size_t b = boosth::gemv_partial_bytes(calls[i].w.N, calls[i].w.K, M_b);
+    if (b == 0) return 0;
+    partial = b > partial ? b : partial;
+  }
+  return boosth::gemv_header_bytes(tiles) + (partial + 255) / 256 * 256 + 64 * (size_t)(n_calls + 1);
+}
+
+extern "C" int boost_gemv_tiered_chain(const boost_gemv_call_t* calls, uint32_t n_calls, uint32_t M_b,
+                                       void* workspace, size_t workspace_bytes, void* stream) {
+  const size_t need = boost_gemv_chain_workspace_bytes(calls, n_calls, M_b);
+  if (need == 0) return BOOST_ERR_INVALID;
+  if (!workspace) return BOOST_ERR_INVALID;
+  if (((uintptr_t)workspace % 256) != 0) return BOOST_ERR_ALIGN;
+  if (workspace_bytes < need) return BOOST_ERR_CAPACITY;
+  // the tail of the workspace holds the queue words of every product and the phase counters
+  const size_t sync_bytes = 64 * (size_t)(n_calls + 1);
+  const size_t usable = (workspace_bytes - sync_bytes) & ~(size_t)255;
+  uint32_t* sync_words = reinterpret_cast<uint32_t*>(static_cast<uint8_t*>(workspace) + usable);
+  return boosth::gemv_chain_launch(calls, n_calls, M_b, workspace, usable, sync_words, 0, stream);
 }
 
 #ifdef BOOST_TRACE

@@ -98,6 +98,11 @@ class TieredWeight:
         torch.cuda.current_stream().synchronize()
         self._ws = {}
 
+    def struct(self):
+        """The weight as the binding.Weight structure that chains and the decode step take."""
+        return B.Weight(self.buf.page_ptr.data_ptr(), self.buf.order.data_ptr(), self.buf.n_pages, self.buf.n_host,
+                        self.N, self.K)
+
     def workspace(self, m_b):
         n = B.boost_gemv_workspace_bytes(self.N, self.K, m_b)
         ws = self._ws.get(n)

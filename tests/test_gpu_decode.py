@@ -171,7 +171,7 @@ def test_decode_steps_match_oracle(dev, n_seq, kv_modulus, weight_ratio):
         ctx_pin.numpy()[:] = ctx
         tab_pin.numpy()[:] = table
         n_launch = dec.step_host(tok_pin.numpy(), tab_pin.numpy(), ctx_pin.numpy(), nxt_pin.numpy())
-        assert n_launch == 2 + 5 * nl + 2
+        assert n_launch == 4 + 2 * nl
         ref = od.decode_step(cfg, w, tokens, k_host, v_host, table, ctx)
         logits = dec.buf["logits"][:n_seq].cpu().numpy()
         assert_chain_close(logits, ref["logits"], f"logits step {step}")
@@ -327,7 +327,7 @@ def test_full_size_step_matches_oracle_on_samples(dev):
     tokens = rng.integers(0, vocab, size=n_seq).astype(np.int32)
     nxt = np.zeros(n_seq, np.int32)
     n_launch = dec.step_host(tokens, table, ctx, nxt)
-    assert n_launch == 2 + 5 + 2
+    assert n_launch == 4 + 2
     assert dec.status_words() == [0, 0]
 
     rows = np.arange(0, vocab, 61)
@@ -343,3 +343,80 @@ def test_full_size_step_matches_oracle_on_samples(dev):
     # every logit was written by this step: the buffer starts at zero, and an fp32 sum that
     # cancels exactly is a once-in-10^7 event per element
     assert logits.size - np.count_nonzero(logits) <= 4
+
+
+@pytest.mark.parametrize("m_b", [1, 24, 70])
+def test_gemv_chain_matches_separate_launches_and_oracle(dev, m_b):
+    """boost_gemv_tiered_chain: four dependent products in one launch (output product with
+    residual and row statistics -> gate/up with row scale and SwiGLU -> down product with
+    residual and statistics -> a scaled product with fp32 output and a ragged row count) give
+    bit for bit what the same calls of boost_gemv_tiered_fused give one after the other, and
+    agree with the oracle's operators; repeated launches reuse the workspace."""
+    from paper_2609_13592_b200.tiers import TieredWeight, aligned_workspace
+    kin, hid, ffn, n_out, stride = 768, 1024, 1536, 2000, 128
+    x_bits = synth.normal_bf16((m_b, kin), 1.0, 1)
+    h0_bits = synth.normal_bf16((m_b, hid), 1.0, 2)
+    g1 = synth.f32_to_bf16_bits(1.0 + 0.1 * np.random.default_rng(3).standard_normal(hid).astype(np.float32))
+    g2 = synth.f32_to_bf16_bits(1.0 + 0.1 * np.random.default_rng(4).standard_normal(hid).astype(np.float32))
+    wb = [synth.normal_bf16((hid, kin), 0.03, 5), synth.normal_bf16((2 * ffn, hid), 0.03, 6),
+          synth.normal_bf16((hid, ffn), 0.03, 7), synth.normal_bf16((n_out, hid), 0.03, 8)]
+    w = [TieredWeight(bf16_tensor(wb[0], dev), 0.5, device=dev),
+         TieredWeight(bf16_tensor(wb[1], dev), 0.25, device=dev, row_mode=1, col_scale=bf16_tensor(g1, dev)),
+         TieredWeight(bf16_tensor(wb[2], dev), 0.5, device=dev),
+         TieredWeight(bf16_tensor(wb[3], dev), 0.25, device=dev, col_scale=bf16_tensor(g2, dev))]
+    x = bf16_tensor(x_bits, dev)
+
+    def buffers():
+        return {"h": bf16_tensor(h0_bits, dev).clone(), "act": torch.zeros(m_b, ffn, dtype=torch.bfloat16, device=dev),
+                "logits": torch.zeros(m_b, n_out, dtype=torch.float32, device=dev),
+                "ssq_b": torch.zeros(hid // 128, stride, dtype=torch.float32, device=dev),
+                "ssq_a": torch.zeros(hid // 128, stride, dtype=torch.float32, device=dev)}
+
+    def epi(mode=B.EPI_PLAIN, ssq_in=None, ssq_out=None):
+        e = B.GemvEpilogue()
+        e.mode, e.ssq_stride, e.rms_eps, e.ssq_in_tiles = mode, stride, od.RMS_EPS, hid // 128
+        e.ssq_in = None if ssq_in is None else ssq_in.data_ptr()
+        e.ssq_out = None if ssq_out is None else ssq_out.data_ptr()
+        return e
+
+    def calls_for(b):
+        return [dict(w=w[0].struct(), x=x, y=b["h"], y_dtype=1, residual=b["h"], epilogue=epi(ssq_out=b["ssq_b"])),
+                dict(w=w[1].struct(), x=b["h"], y=b["act"], y_dtype=1, epilogue=epi(B.EPI_SWIGLU, ssq_in=b["ssq_b"])),
+                dict(w=w[2].struct(), x=b["act"], y=b["h"], y_dtype=1, residual=b["h"], epilogue=epi(ssq_out=b["ssq_a"])),
+                dict(w=w[3].struct(), x=b["h"], y=b["logits"], y_dtype=0, epilogue=epi(ssq_in=b["ssq_a"]))]
+
+    # the same four calls, one launch each
+    sep = buffers()
+    for c, tw in zip(calls_for(sep), w):
+        tw.gemv(c["x"], y=c["y"], residual=c.get("residual"), epilogue=c["epilogue"])
+    torch.cuda.synchronize()
+    assert all(tw.status_words() == [0] for tw in w)
+
+    # one launch for the chain, several times over the same workspace
+    probe = B.gemv_calls(calls_for(sep))
+    ws_bytes = B.boost_gemv_chain_workspace_bytes(probe, m_b)
+    assert ws_bytes > 0
+    ws_t, ws_ptr = aligned_workspace(ws_bytes, dev)
+    for rep in range(6):
+        got = buffers()
+        arr = B.gemv_calls(calls_for(got))
+        B.boost_gemv_tiered_chain(arr, m_b, ws_ptr, ws_bytes)
+        torch.cuda.synchronize()
+        for name in ("h", "act", "logits", "ssq_a", "ssq_b"):
+            assert torch.equal(got[name], sep[name]), (name, rep)
+    off = ws_ptr - ws_t.data_ptr()
+    assert int(ws_t[off:off + 4].cpu().numpy().view(np.uint32)[0]) == 0          # status word
+    tail = ws_t[off + ws_bytes - 64 * 5:off + ws_bytes]
+    assert int(tail.count_nonzero()) == 0                                         # queue words and phase counters reset
+
+    # the oracle's operators one after the other, bf16 where the device stores bf16
+    rnd = lambda a: ol.bf16_bits_to_f64(ol.f64_to_bf16_bits(a))
+    x64, h64 = ol.bf16_bits_to_f64(x_bits), ol.bf16_bits_to_f64(h0_bits)
+    h1 = rnd(h64 + x64 @ ol.bf16_bits_to_f64(wb[0]).T)
+    gu = rnd(od.rms_scale(h1) * (h1 @ ol.bf16_bits_to_f64(od.fold_norm_weight(wb[1], g1)).T))
+    act = rnd(od.silu(gu[:, :ffn]) * gu[:, ffn:])
+    h2 = rnd(h1 + act @ ol.bf16_bits_to_f64(wb[2]).T)
+    logits = od.rms_scale(h2) * (h2 @ ol.bf16_bits_to_f64(od.fold_norm_weight(wb[3], g2)).T)
+    assert_chain_close(got["act"].float().cpu().numpy(), act, "chain: SwiGLU output", wide=True)
+    assert_chain_close(got["h"].float().cpu().numpy(), h2, "chain: residual stream", wide=True)
+    assert_chain_close(got["logits"].cpu().numpy(), logits, "chain: scaled product", wide=True)
