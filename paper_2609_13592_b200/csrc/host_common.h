@@ -36,6 +36,27 @@ inline int launch_chained(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_
   return check(cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...));
 }
 
+// The same for a kernel whose threadblocks form clusters of cluster_x along x.
+template <typename... KArgs, typename... Args>
+inline int launch_chained_cluster(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, unsigned cluster_x,
+                                  cudaStream_t stream, Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[2];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  attr[1].id = cudaLaunchAttributeClusterDimension;
+  attr[1].val.clusterDim.x = cluster_x;
+  attr[1].val.clusterDim.y = 1;
+  attr[1].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 2;
+  return check(cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...));
+}
+
 // boost_gemv_tiered with a private set of queue words (16 zeroed uint32 that no other launch
 // in flight uses): the kernel may then take work and stream weights before its predecessor
 // has finished.  queue_words = nullptr gives the public behaviour.  header_row_tiles: size the

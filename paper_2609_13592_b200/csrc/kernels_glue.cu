@@ -177,40 +177,77 @@ swiglu_kernel(const __nv_bfloat16* __restrict__ gu, uint32_t B, uint32_t F, __nv
   }
 }
 
-// argmax over fp32 logits, lowest index on ties; one threadblock per row
-__global__ void __launch_bounds__(1024)
+// argmax over fp32 logits, lowest index on ties.  One cluster of kArgmaxCluster threadblocks
+// per row: each scans a slice of the row, and the first block of the cluster reads the others'
+// candidates out of their shared memory (distributed shared memory), so no scratch in global
+// memory and no second launch are needed.
+constexpr uint32_t kArgmaxCluster = 8;
+constexpr uint32_t kArgmaxThreads = 512;
+
+__device__ __forceinline__ void take_better(float& best, uint32_t& best_i, float v, uint32_t i) {
+  if (v > best || (v == best && i < best_i)) { best = v; best_i = i; }
+}
+
+__global__ void __launch_bounds__(kArgmaxThreads)
 argmax_kernel(const float* __restrict__ logits, uint32_t V, int32_t* __restrict__ out) {
   pdl_launch_dependents();
   pdl_wait();
   __shared__ float s_val[32];
   __shared__ uint32_t s_idx[32];
-  const float* row = logits + (size_t)blockIdx.x * V;
+  __shared__ float s_best;
+  __shared__ uint32_t s_best_i;
+  uint32_t rank;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(rank));
+  const float* row = logits + (size_t)blockIdx.y * V;
+  const uint32_t slice = (V + kArgmaxCluster - 1) / kArgmaxCluster;
+  const uint32_t i0 = rank * slice, i1 = min(V, i0 + slice);
   float best = -CUDART_INF_F;
-  uint32_t best_i = 0xFFFFFFFFu;
-  for (uint32_t i = threadIdx.x; i < V; i += blockDim.x) {
-    const float v = row[i];
-    if (v > best || best_i == 0xFFFFFFFFu) { best = v; best_i = i; }   // ascending i: first max wins
+  uint32_t best_i = 0xFFFFFFFFu;   // "nothing yet": loses every tie, and any value beats -inf or equals it
+  uint32_t i = i0 + threadIdx.x;
+  for (; i + 3 * kArgmaxThreads < i1; i += 4 * kArgmaxThreads) {   // four loads in flight
+    const float v0 = row[i], v1 = row[i + kArgmaxThreads], v2 = row[i + 2 * kArgmaxThreads], v3 = row[i + 3 * kArgmaxThreads];
+    take_better(best, best_i, v0, i);
+    take_better(best, best_i, v1, i + kArgmaxThreads);
+    take_better(best, best_i, v2, i + 2 * kArgmaxThreads);
+    take_better(best, best_i, v3, i + 3 * kArgmaxThreads);
   }
+  for (; i < i1; i += kArgmaxThreads) take_better(best, best_i, row[i], i);
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) {
     const float ov = __shfl_xor_sync(0xFFFFFFFFu, best, o);
     const uint32_t oi = __shfl_xor_sync(0xFFFFFFFFu, best_i, o);
-    if (ov > best || (ov == best && oi < best_i)) { best = ov; best_i = oi; }
+    take_better(best, best_i, ov, oi);
   }
   if ((threadIdx.x & 31) == 0) { s_val[threadIdx.x >> 5] = best; s_idx[threadIdx.x >> 5] = best_i; }
   __syncthreads();
   if (threadIdx.x < 32) {
-    const uint32_t n_warps = blockDim.x / 32;
+    const uint32_t n_warps = kArgmaxThreads / 32;
     best = threadIdx.x < n_warps ? s_val[threadIdx.x] : -CUDART_INF_F;
     best_i = threadIdx.x < n_warps ? s_idx[threadIdx.x] : 0xFFFFFFFFu;
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) {
       const float ov = __shfl_xor_sync(0xFFFFFFFFu, best, o);
       const uint32_t oi = __shfl_xor_sync(0xFFFFFFFFu, best_i, o);
-      if (ov > best || (ov == best && oi < best_i)) { best = ov; best_i = oi; }
+      take_better(best, best_i, ov, oi);
     }
-    if (threadIdx.x == 0) out[blockIdx.x] = (int32_t)best_i;
+    if (threadIdx.x == 0) { s_best = best; s_best_i = best_i; }
   }
+  // every block's candidate is in its shared memory: the first block of the cluster collects them
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+  if (rank == 0 && threadIdx.x == 0) {
+    for (uint32_t r = 1; r < kArgmaxCluster; ++r) {
+      uint32_t a_val, a_idx, ri;
+      float rv;
+      asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(a_val) : "r"(smem_u32(&s_best)), "r"(r));
+      asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(a_idx) : "r"(smem_u32(&s_best_i)), "r"(r));
+      asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(rv) : "r"(a_val) : "memory");
+      asm volatile("ld.shared::cluster.u32 %0, [%1];" : "=r"(ri) : "r"(a_idx) : "memory");
+      take_better(best, best_i, rv, ri);
+    }
+    out[blockIdx.y] = best_i == 0xFFFFFFFFu ? 0 : (int32_t)best_i;   // a row of NaNs: index 0
+  }
+  // nobody leaves (and gives up its shared memory) before the collector has read it
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
 
 }  // namespace
@@ -286,5 +323,7 @@ extern "C" int boost_swiglu(const void* gate_up, uint32_t B, uint32_t F, void* o
 extern "C" int boost_argmax(const float* logits, uint32_t B, uint32_t V, int32_t* out, void* stream) {
   if (B == 0) return BOOST_OK;
   if (!logits || !out || V == 0) return BOOST_ERR_INVALID;
-  return boosth::launch_chained(argmax_kernel, dim3(B), dim3(1024), 0, (cudaStream_t)stream, logits, V, out);
+  if (B > 65535) return BOOST_ERR_UNSUPPORTED;
+  return boosth::launch_chained_cluster(argmax_kernel, dim3(kArgmaxCluster, B), dim3(kArgmaxThreads), 0, kArgmaxCluster,
+                                        (cudaStream_t)stream, logits, V, out);
 }
