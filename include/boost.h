@@ -321,6 +321,10 @@ typedef struct {
   const int32_t* ctx_lens;       /* device [M_b], new token included */
   uint32_t n_q_heads, n_kv_heads;
   const float* rope_table;       /* device, from boost_rope_table: (cos, sin) [M_b][64] */
+  /* Optional second pair of page tables of the same cache: the new K / V rows are written
+   * through both (the prefetch-to-HBM variant keeps a staged copy of host pages in HBM). */
+  const void* const* k_page_ptr2; /* device or NULL */
+  const void* const* v_page_ptr2; /* device or NULL */
 } boost_gemv_epilogue_t;
 
 /* boost_gemv_tiered with an epilogue descriptor (NULL = plain). */
@@ -488,6 +492,50 @@ typedef struct {
   size_t attn_ws_bytes;
   int32_t *tokens_dev, *ctx_dev, *table_dev, *next_dev;
 } boost_llama_scratch_t;
+
+/* Prefetch-to-HBM comparison variant (Sec. 2.5: the alternative to concurrent access is to
+ * copy host-resident data into HBM ahead of its use; its gain is bounded by 1 - alpha).  The
+ * host pages of every layer's K and V tensor occupy one contiguous range of the pinned slab
+ * (boost_page_table puts them in consecutive slots); the copy engine brings that range into
+ * one of two staging buffers in HBM while earlier layers compute, and the attention kernel
+ * reads the staged copy through a second page table in which host pages point into the
+ * staging buffer.  The new token's K / V rows are written to both copies.
+ *   host_bytes                 bytes of host pages per tensor (a multiple of 2 MiB; the same
+ *                              for every layer: the pool places all layers alike);
+ *   k_stage / v_stage          device, two staging buffers of host_bytes each, 2 MiB aligned;
+ *   layers[l].k_host_src ...   host (pinned) address of the first host page of layer l;
+ *   layers[l].k_page_ptr_staged  device array like the layer's k_page_ptr with every host
+ *                              page replaced by its slot in staging buffer l % 2. */
+typedef struct {
+  const void* k_host_src; /* pinned host */
+  const void* v_host_src;
+  const void* const* k_page_ptr_staged; /* device */
+  const void* const* v_page_ptr_staged;
+} boost_kv_prefetch_layer_t;
+
+typedef struct {
+  uint64_t host_bytes;
+  void* k_stage[2];
+  void* v_stage[2];
+  const boost_kv_prefetch_layer_t* layers; /* host array of n_layers entries */
+} boost_kv_prefetch_t;
+
+/* Copy stream and events of the prefetch variant; one per model instance. */
+typedef struct boost_prefetch_ctx boost_prefetch_ctx;
+int boost_prefetch_ctx_create(uint32_t n_layers, boost_prefetch_ctx** out /*host*/);
+void boost_prefetch_ctx_destroy(boost_prefetch_ctx* ctx);
+
+/* boost_llama_decode_step with the host pages of the KV cache staged into HBM by the copy
+ * engine, layer l + 2 while layers l and l + 1 compute.  Same results as
+ * boost_llama_decode_step (the attention kernel reads identical bytes from another address).
+ * model->kv_tier may name host pages; they are never read by the SMs in this variant. */
+int boost_llama_decode_step_prefetch(const boost_llama_model_t* model /*host*/,
+                                     const boost_llama_scratch_t* scratch /*host*/,
+                                     const boost_kv_prefetch_t* prefetch /*host*/, boost_prefetch_ctx* ctx,
+                                     const int32_t* tokens /*device*/, const int32_t* block_table /*device*/,
+                                     uint32_t max_blocks, const int32_t* ctx_lens /*device*/, uint32_t B,
+                                     int32_t* next_tokens /*device*/, uint32_t* n_launches_out /*host*/,
+                                     void* stream);
 
 /* Size of scratch->gemv_ws for steps of up to B sequences of this model (Sec. 2.1 treats the
  * step as a chain of weight products; they share one workspace).  0 on invalid arguments. */

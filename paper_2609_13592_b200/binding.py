@@ -59,7 +59,7 @@ class GemvEpilogue(C.Structure):
                 ("q_out", C.c_void_p), ("k_page_ptr", C.c_void_p), ("v_page_ptr", C.c_void_p),
                 ("n_pool_blocks", C.c_uint32), ("block_table", C.c_void_p), ("max_blocks", C.c_uint32),
                 ("ctx_lens", C.c_void_p), ("n_q_heads", C.c_uint32), ("n_kv_heads", C.c_uint32),
-                ("rope_table", C.c_void_p)]
+                ("rope_table", C.c_void_p), ("k_page_ptr2", C.c_void_p), ("v_page_ptr2", C.c_void_p)]
 
 
 class GemvCall(C.Structure):
@@ -79,6 +79,16 @@ class LlamaModel(C.Structure):
                 ("embed", C.c_void_p), ("lm_head", Weight),
                 ("layers", C.POINTER(LlamaLayer)), ("kv_tier", C.c_void_p),
                 ("n_kv_pages", C.c_uint64), ("n_pool_blocks", C.c_uint32)]
+
+
+class KVPrefetchLayer(C.Structure):
+    _fields_ = [("k_host_src", C.c_void_p), ("v_host_src", C.c_void_p),
+                ("k_page_ptr_staged", C.c_void_p), ("v_page_ptr_staged", C.c_void_p)]
+
+
+class KVPrefetch(C.Structure):
+    _fields_ = [("host_bytes", C.c_uint64), ("k_stage", C.c_void_p * 2), ("v_stage", C.c_void_p * 2),
+                ("layers", C.POINTER(KVPrefetchLayer))]
 
 
 class LlamaScratch(C.Structure):
@@ -141,6 +151,9 @@ SIGNATURES = {
     "boost_gemv_tiered_chain": (_int, [_vp, _u32, _u32, _vp, _sz, _vp]),
     "boost_llama_gemv_workspace_bytes": (C.c_size_t, [_vp, _u32]),
     "boost_llama_decode_step": (_int, [_vp, _vp, _vp, _vp, _u32, _vp, _u32, _vp, _vp, _vp]),
+    "boost_prefetch_ctx_create": (_int, [_u32, _vp]),
+    "boost_prefetch_ctx_destroy": (None, [_vp]),
+    "boost_llama_decode_step_prefetch": (_int, [_vp, _vp, _vp, _vp, _vp, _vp, _u32, _vp, _u32, _vp, _vp, _vp]),
     "boost_llama_decode_step_profile": (_int, [_vp, _vp, _vp, _vp, _u32, _vp, _u32, _vp, _vp, _vp, _vp]),
     "boost_llama_decode_step_host": (_int, [_vp, _vp, _vp, _vp, _u32, _vp, _u32, _vp, _vp, _vp]),
 }
@@ -483,6 +496,27 @@ def boost_llama_decode_step(model, scratch, tokens, block_table, max_blocks, ctx
                                          _ptr(block_table), max_blocks, _ptr(ctx_lens), b,
                                          _ptr(next_tokens), C.addressof(n), _stream(stream)),
            "boost_llama_decode_step")
+    return n.value
+
+
+def boost_prefetch_ctx_create(n_layers):
+    h = C.c_void_p()
+    _check(lib().boost_prefetch_ctx_create(n_layers, C.addressof(h)), "boost_prefetch_ctx_create")
+    return h
+
+
+def boost_prefetch_ctx_destroy(handle):
+    lib().boost_prefetch_ctx_destroy(handle)
+
+
+def boost_llama_decode_step_prefetch(model, scratch, prefetch, ctx, tokens, block_table, max_blocks, ctx_lens, b,
+                                     next_tokens, stream=None):
+    """Prefetch-to-HBM variant of boost_llama_decode_step; prefetch: a KVPrefetch structure."""
+    n = C.c_uint32(0)
+    _check(lib().boost_llama_decode_step_prefetch(C.addressof(model), C.addressof(scratch), C.addressof(prefetch),
+                                                  ctx, _ptr(tokens), _ptr(block_table), max_blocks,
+                                                  _ptr(ctx_lens), b, _ptr(next_tokens), C.addressof(n),
+                                                  _stream(stream)), "boost_llama_decode_step_prefetch")
     return n.value
 
 

@@ -2,6 +2,8 @@
 // Host code only: every step of the path runs in the kernels of the other files.
 #include <cuda_runtime.h>
 
+#include <new>
+
 #include "host_common.h"
 
 namespace {
@@ -74,9 +76,22 @@ boost_gemv_call_t call_of(const boost_weight_t& w, const void* x, void* y, int y
   return c;
 }
 
+}  // namespace
+
+// Copy stream and events of the prefetch-to-HBM variant.
+struct boost_prefetch_ctx {
+  cudaStream_t copy_stream = nullptr;
+  uint32_t n_layers = 0;
+  cudaEvent_t* copy_done = nullptr;   // [n_layers]: layer's host pages are in its staging buffer
+  cudaEvent_t* attn_done = nullptr;   // [n_layers]: the attention kernel of the layer has been issued and finished
+  cudaEvent_t step_begin = nullptr;   // everything issued to the compute stream before this step
+};
+
+namespace {
+
 int run_step(Launcher& L, const boost_llama_model_t* m, const boost_llama_scratch_t* s, const int32_t* tokens,
              const int32_t* block_table, uint32_t max_blocks, const int32_t* ctx_lens, uint32_t B,
-             int32_t* next_tokens) {
+             int32_t* next_tokens, const boost_kv_prefetch_t* pf = nullptr, boost_prefetch_ctx* pc = nullptr) {
   if (!m || !s || !tokens || !block_table || !ctx_lens || !next_tokens) return BOOST_ERR_INVALID;
   if (B == 0 || B > 128 || !m->layers || m->n_layers == 0) return BOOST_ERR_INVALID;
   if (!s->h || !s->q_rot || !s->attn || !s->act || !s->logits || !s->ssq_a || !s->ssq_b || !s->rope_table || !s->gemv_ws ||
@@ -117,8 +132,44 @@ int run_step(Launcher& L, const boost_llama_model_t* m, const boost_llama_scratc
     qkv.n_q_heads = hq;
     qkv.n_kv_heads = hkv;
     qkv.rope_table = s->rope_table;
+    if (pf) {
+      const uint32_t li = (uint32_t)(&ly - m->layers);
+      qkv.k_page_ptr2 = pf->layers[li].k_page_ptr_staged;
+      qkv.v_page_ptr2 = pf->layers[li].v_page_ptr_staged;
+    }
     return call_of(ly.wqkv, s->h, nullptr, 1, nullptr, qkv);
   };
+  // Prefetch variant: the copy engine stages layer l's host pages into buffer l % 2.  A buffer
+  // is free again once the attention kernel two layers back has finished; the staged copy must
+  // be complete before the product that appends the new rows of layer l is launched.
+  cudaStream_t cs = pc ? pc->copy_stream : nullptr;
+  auto stage_layer = [&](uint32_t li) -> int {
+    if (pf->host_bytes == 0) return BOOST_OK;
+    int rc = BOOST_OK;
+    if (li >= 2) rc = boosth::check(cudaStreamWaitEvent(cs, pc->attn_done[li - 2], 0));
+    if (rc == BOOST_OK)
+      rc = boosth::check(cudaMemcpyAsync(pf->k_stage[li & 1], pf->layers[li].k_host_src, pf->host_bytes,
+                                         cudaMemcpyHostToDevice, cs));
+    if (rc == BOOST_OK)
+      rc = boosth::check(cudaMemcpyAsync(pf->v_stage[li & 1], pf->layers[li].v_host_src, pf->host_bytes,
+                                         cudaMemcpyHostToDevice, cs));
+    if (rc == BOOST_OK) rc = boosth::check(cudaEventRecord(pc->copy_done[li], cs));
+    return rc;
+  };
+  auto wait_staged = [&](uint32_t li) -> int {
+    if (pf->host_bytes == 0) return BOOST_OK;
+    return boosth::check(cudaStreamWaitEvent((cudaStream_t)stream, pc->copy_done[li], 0));
+  };
+  if (pf) {
+    if (!pc || pc->n_layers < m->n_layers || !pf->layers) return BOOST_ERR_INVALID;
+    // the copies of this step come after everything already on the compute stream: the previous
+    // step (which read the staging buffers and wrote new rows into the host pages), cache loads
+    L.rc = boosth::check(cudaEventRecord(pc->step_begin, (cudaStream_t)stream));
+    if (L.ok()) L.rc = boosth::check(cudaStreamWaitEvent(cs, pc->step_begin, 0));
+    for (uint32_t li = 0; li < 2 && li < m->n_layers && L.ok(); ++li) L.rc = stage_layer(li);
+    if (L.ok()) L.rc = wait_staged(0);
+    if (!L.ok()) return L.rc;
+  }
   auto chain = [&](const boost_gemv_call_t* calls, uint32_t n) {
     return boosth::gemv_chain_launch(calls, n, B, s->gemv_ws, usable, slots.take(s, usable, n + 1), tiles, stream);
   };
@@ -134,11 +185,18 @@ int run_step(Launcher& L, const boost_llama_model_t* m, const boost_llama_scratc
   for (uint32_t li = 0; li < m->n_layers && L.ok(); ++li) {
     const boost_llama_layer_t& ly = m->layers[li];
     L.run(kKindAttn, [&] {
-      return boost_paged_attn_decode_tiered(s->q_rot, ly.k_page_ptr, ly.v_page_ptr, m->kv_tier,
-                                            (size_t)m->n_kv_pages, m->n_pool_blocks, block_table, max_blocks,
-                                            ctx_lens, B, hq, hkv, d, scale, s->attn_ws, s->attn_ws_bytes,
-                                            s->attn, stream);
+      // prefetch variant: every page is read from HBM (host pages from their staged copy)
+      return boost_paged_attn_decode_tiered(s->q_rot, pf ? pf->layers[li].k_page_ptr_staged : ly.k_page_ptr,
+                                            pf ? pf->layers[li].v_page_ptr_staged : ly.v_page_ptr,
+                                            pf ? nullptr : m->kv_tier, (size_t)m->n_kv_pages, m->n_pool_blocks,
+                                            block_table, max_blocks, ctx_lens, B, hq, hkv, d, scale, s->attn_ws,
+                                            s->attn_ws_bytes, s->attn, stream);
     });
+    if (pf && L.ok()) {
+      L.rc = boosth::check(cudaEventRecord(pc->attn_done[li], (cudaStream_t)stream));
+      if (L.ok() && li + 2 < m->n_layers) L.rc = stage_layer(li + 2);
+      if (L.ok() && li + 1 < m->n_layers) L.rc = wait_staged(li + 1);
+    }
     // One launch for the four products between two attention kernels:
     //   h += attn Wo^T                       (row statistics of the new h into ssq_b)
     //   act = swiglu(rmsnorm(h) Wgu^T)       (row scale from ssq_b)
@@ -186,6 +244,57 @@ extern "C" int boost_llama_decode_step(const boost_llama_model_t* m, const boost
   static thread_local Launcher L;
   L.stream = stream; L.timed = false; L.count = 0; L.rc = BOOST_OK;
   const int rc = run_step(L, m, s, tokens, block_table, max_blocks, ctx_lens, B, next_tokens);
+  if (n_launches_out) *n_launches_out = L.count;
+  return rc;
+}
+
+extern "C" int boost_prefetch_ctx_create(uint32_t n_layers, boost_prefetch_ctx** out) {
+  if (!out || n_layers == 0) return BOOST_ERR_INVALID;
+  boost_prefetch_ctx* c = new (std::nothrow) boost_prefetch_ctx;
+  if (!c) return BOOST_ERR_INVALID;
+  c->n_layers = n_layers;
+  c->copy_done = new (std::nothrow) cudaEvent_t[n_layers]();
+  c->attn_done = new (std::nothrow) cudaEvent_t[n_layers]();
+  int rc = (c->copy_done && c->attn_done) ? BOOST_OK : BOOST_ERR_INVALID;
+  if (rc == BOOST_OK) rc = boosth::check(cudaStreamCreateWithFlags(&c->copy_stream, cudaStreamNonBlocking));
+  for (uint32_t i = 0; i < n_layers && rc == BOOST_OK; ++i) {
+    rc = boosth::check(cudaEventCreateWithFlags(&c->copy_done[i], cudaEventDisableTiming));
+    if (rc == BOOST_OK) rc = boosth::check(cudaEventCreateWithFlags(&c->attn_done[i], cudaEventDisableTiming));
+  }
+  if (rc == BOOST_OK) rc = boosth::check(cudaEventCreateWithFlags(&c->step_begin, cudaEventDisableTiming));
+  if (rc != BOOST_OK) {
+    boost_prefetch_ctx_destroy(c);
+    return rc;
+  }
+  *out = c;
+  return BOOST_OK;
+}
+
+extern "C" void boost_prefetch_ctx_destroy(boost_prefetch_ctx* c) {
+  if (!c) return;
+  for (uint32_t i = 0; i < c->n_layers; ++i) {
+    if (c->copy_done && c->copy_done[i]) cudaEventDestroy(c->copy_done[i]);
+    if (c->attn_done && c->attn_done[i]) cudaEventDestroy(c->attn_done[i]);
+  }
+  if (c->step_begin) cudaEventDestroy(c->step_begin);
+  if (c->copy_stream) cudaStreamDestroy(c->copy_stream);
+  delete[] c->copy_done;
+  delete[] c->attn_done;
+  delete c;
+}
+
+extern "C" int boost_llama_decode_step_prefetch(const boost_llama_model_t* m, const boost_llama_scratch_t* s,
+                                                const boost_kv_prefetch_t* prefetch, boost_prefetch_ctx* ctx,
+                                                const int32_t* tokens, const int32_t* block_table,
+                                                uint32_t max_blocks, const int32_t* ctx_lens, uint32_t B,
+                                                int32_t* next_tokens, uint32_t* n_launches_out, void* stream) {
+  if (!prefetch || !ctx) return BOOST_ERR_INVALID;
+  if (prefetch->host_bytes % BOOST_PAGE_BYTES != 0) return BOOST_ERR_INVALID;
+  if (prefetch->host_bytes && (!prefetch->k_stage[0] || !prefetch->k_stage[1] || !prefetch->v_stage[0] || !prefetch->v_stage[1]))
+    return BOOST_ERR_INVALID;
+  static thread_local Launcher L;
+  L.stream = stream; L.timed = false; L.count = 0; L.rc = BOOST_OK;
+  const int rc = run_step(L, m, s, tokens, block_table, max_blocks, ctx_lens, B, next_tokens, prefetch, ctx);
   if (n_launches_out) *n_launches_out = L.count;
   return rc;
 }

@@ -73,6 +73,8 @@ struct GemvParams {
   __nv_bfloat16* q_out;      // rope epilogue: rotated queries [M_b, Hq, 128]
   const void* const* k_page_ptr;
   const void* const* v_page_ptr;
+  const void* const* k_page_ptr2;   // optional second copy of the cache (staged host pages)
+  const void* const* v_page_ptr2;
   const int32_t* block_table;
   const int32_t* ctx_lens;
   uint32_t n_pool_blocks, max_blocks, Hq, Hkv;
@@ -294,6 +296,11 @@ __device__ __forceinline__ void combine_tile(const GemvParams& p, uint32_t row_t
             const size_t off2 = chunk + (((((d + 64) >> 3) ^ (slot & 7u))) << 4) + (d & 7u) * 2u;
             *reinterpret_cast<uint2*>(static_cast<uint8_t*>(const_cast<void*>(pages[off1 / kPageBytes])) + off1 % kPageBytes) = o1;
             *reinterpret_cast<uint2*>(static_cast<uint8_t*>(const_cast<void*>(pages[off2 / kPageBytes])) + off2 % kPageBytes) = o2;
+            const void* const* pages2 = is_k ? p.k_page_ptr2 : p.v_page_ptr2;
+            if (pages2) {
+              *reinterpret_cast<uint2*>(static_cast<uint8_t*>(const_cast<void*>(pages2[off1 / kPageBytes])) + off1 % kPageBytes) = o1;
+              *reinterpret_cast<uint2*>(static_cast<uint8_t*>(const_cast<void*>(pages2[off2 / kPageBytes])) + off2 % kPageBytes) = o2;
+            }
           }
         }
       }
@@ -945,6 +952,8 @@ int fill_params(GemvParams& p, const void* const* w_page_ptr, const uint32_t* w_
   p.q_out = epi ? static_cast<__nv_bfloat16*>(epi->q_out) : nullptr;
   p.k_page_ptr = epi ? epi->k_page_ptr : nullptr;
   p.v_page_ptr = epi ? epi->v_page_ptr : nullptr;
+  p.k_page_ptr2 = epi ? epi->k_page_ptr2 : nullptr;
+  p.v_page_ptr2 = epi ? epi->v_page_ptr2 : nullptr;
   p.block_table = epi ? epi->block_table : nullptr;
   p.ctx_lens = epi ? epi->ctx_lens : nullptr;
   p.n_pool_blocks = epi ? epi->n_pool_blocks : 0;

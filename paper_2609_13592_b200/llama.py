@@ -32,7 +32,7 @@ class LlamaDecoder:
     """
 
     def __init__(self, cfg, get_weight, weight_host_ratio=0.0, n_pool_blocks=512, kv_host_modulus=0,
-                 max_batch=32, max_blocks=8, device="cuda", weight_policy=B.POLICY_MODULO):
+                 max_batch=32, max_blocks=8, device="cuda", weight_policy=B.POLICY_MODULO, kv_prefetch=False):
         self.cfg = dict(cfg)
         self.device = torch.device(device)
         self.max_batch, self.max_blocks = max_batch, max_blocks
@@ -103,7 +103,40 @@ class LlamaDecoder:
         s.gemv_ws, s.gemv_ws_bytes, s.attn_ws, s.attn_ws_bytes = gemv_ws, gemv_bytes, attn_ws, attn_bytes
         self.scratch = s
         self._gemv_ws_ptr, self._attn_ws_ptr = gemv_ws, attn_ws
+        self._prefetch = None
+        if kv_prefetch:
+            self._make_prefetch()
         torch.cuda.synchronize(self.device)
+
+    def _make_prefetch(self):
+        """Structures of the prefetch-to-HBM variant: two staging buffers per tensor kind, and
+        per layer a page table whose host pages point into staging buffer (layer % 2)."""
+        n_host = self.layers[0]["k"].n_host
+        host_bytes = n_host * B.PAGE_BYTES
+        self._stage_t = [torch.empty(host_bytes + B.PAGE_BYTES, dtype=torch.uint8, device=self.device) for _ in range(4)]
+        stage = [(t.data_ptr() + B.PAGE_BYTES - 1) // B.PAGE_BYTES * B.PAGE_BYTES for t in self._stage_t]
+        self._pf_layers = (B.KVPrefetchLayer * len(self.layers))()
+        self._pf_tables = []
+        for li, ly in enumerate(self.layers):
+            kt = ly["k"].staged_page_ptr(stage[li % 2])
+            vt = ly["v"].staged_page_ptr(stage[2 + li % 2])
+            self._pf_tables += [kt, vt]
+            e = self._pf_layers[li]
+            e.k_host_src, e.v_host_src = ly["k"].host_base_cpu or None, ly["v"].host_base_cpu or None
+            e.k_page_ptr_staged, e.v_page_ptr_staged = kt.data_ptr(), vt.data_ptr()
+        pf = B.KVPrefetch()
+        pf.host_bytes = host_bytes
+        pf.k_stage[0], pf.k_stage[1], pf.v_stage[0], pf.v_stage[1] = stage
+        pf.layers = C.cast(self._pf_layers, C.POINTER(B.KVPrefetchLayer))
+        self._prefetch = pf
+        self._prefetch_ctx = B.boost_prefetch_ctx_create(len(self.layers))
+
+    def step_prefetch(self, tokens, block_table, ctx_lens, next_tokens, stream=None):
+        """Device-buffer step of the prefetch-to-HBM variant (the decoder was built with kv_prefetch=True)."""
+        assert self._prefetch is not None
+        return B.boost_llama_decode_step_prefetch(self.model, self.scratch, self._prefetch, self._prefetch_ctx,
+                                                  tokens, block_table, block_table.shape[1], ctx_lens,
+                                                  tokens.shape[0], next_tokens, stream)
 
     # bytes the kernels must read per step (algorithmic): all weight pages plus live KV
     def weight_bytes(self):

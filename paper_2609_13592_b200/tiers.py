@@ -73,6 +73,13 @@ class TieredBuffer:
         self.order_host = order
         self.order = torch.from_numpy(order.view(np.int32).copy()).to(self.device)
 
+    def staged_page_ptr(self, stage_base):
+        """Page table in which every host page points at its slot of a staging buffer in HBM
+        (device address stage_base, n_host pages long) instead of the pinned slab."""
+        table = B.boost_page_table(self.tier, self.hbm_base, self.n_hbm * PAGE, stage_base or None,
+                                   self.n_host * PAGE)
+        return torch.from_numpy(table.view(np.int64).copy()).to(self.device)
+
     def scatter_from(self, flat, stream=None):
         """Copy a contiguous device tensor (any dtype) of n_bytes into the pages."""
         assert flat.is_cuda and flat.is_contiguous() and flat.numel() * flat.element_size() == self.n_bytes

@@ -420,3 +420,52 @@ def test_gemv_chain_matches_separate_launches_and_oracle(dev, m_b):
     assert_chain_close(got["act"].float().cpu().numpy(), act, "chain: SwiGLU output", wide=True)
     assert_chain_close(got["h"].float().cpu().numpy(), h2, "chain: residual stream", wide=True)
     assert_chain_close(got["logits"].cpu().numpy(), logits, "chain: scaled product", wide=True)
+
+
+def test_prefetch_variant_matches_tiered_step(dev):
+    """boost_llama_decode_step_prefetch (host KV pages staged into HBM by the copy engine, two
+    layers ahead) gives bit for bit the logits, tokens and cache contents of the step that
+    reads the host pages in place: the same bytes reach the same arithmetic."""
+    from paper_2609_13592_b200.llama import LlamaDecoder
+    cfg = dict(synth.TINY_LLAMA)
+    cfg["n_layers"] = 5                                   # staging buffers are reused: 0, 1, 0, 1, 0
+    w = synth.llama_weights(cfg, seed=9, std=0.02)
+    hkv, d, nl = cfg["n_kv_heads"], cfg["head_dim"], cfg["n_layers"]
+    n_seq, n_pool_blocks, max_blocks = 6, 512, 8
+
+    def get_weight(name, layer):
+        return bf16_tensor(w[name] if layer is None else w["layers"][layer][name], dev)
+
+    decs = [LlamaDecoder(cfg, get_weight, 0.25, n_pool_blocks, 2, n_seq, max_blocks, dev, kv_prefetch=pf)
+            for pf in (False, True)]
+    assert decs[1].layers[0]["k"].n_host > 0
+    k_host = [synth.normal_bf16((hkv, n_pool_blocks, 16, d), 1.0, 300 + li) for li in range(nl)]
+    v_host = [synth.normal_bf16((hkv, n_pool_blocks, 16, d), 1.0, 400 + li) for li in range(nl)]
+    for dec in decs:
+        load_caches(dev, dec, k_host, v_host)
+    rng = np.random.default_rng(3)
+    ctx = rng.integers(5, 60, size=n_seq).astype(np.int32)
+    table = np.zeros((n_seq, max_blocks), np.int32)
+    for b in range(n_seq):
+        for j in range(max_blocks):
+            got = [dec.pool.alloc(b, 1)[0] for dec in decs]
+            assert got[0] == got[1]
+            table[b, j] = got[0]
+    table_dev = torch.from_numpy(table).to(dev)
+    tok0 = torch.from_numpy(rng.integers(0, cfg["vocab"], size=n_seq).astype(np.int32)).to(dev)
+    tok = [tok0, tok0.clone()]
+    nxt = [torch.zeros(n_seq, dtype=torch.int32, device=dev) for _ in decs]
+    for step in range(6):
+        ctx += 1
+        ctx_dev = torch.from_numpy(ctx).to(dev)
+        n0 = decs[0].step(tok[0], table_dev, ctx_dev, nxt[0])
+        n1 = decs[1].step_prefetch(tok[1], table_dev, ctx_dev, nxt[1])
+        torch.cuda.synchronize()
+        assert n0 == n1 == 4 + 2 * nl
+        assert torch.equal(decs[0].buf["logits"][:n_seq], decs[1].buf["logits"][:n_seq]), step
+        assert torch.equal(nxt[0], nxt[1])
+        tok = [nxt[0].clone(), nxt[1].clone()]
+    for li in range(nl):
+        for name in ("k", "v"):
+            assert np.array_equal(dump_cache(dev, decs[0], li, name), dump_cache(dev, decs[1], li, name))
+    assert decs[0].status_words() == [0, 0] and decs[1].status_words() == [0, 0]
