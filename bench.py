@@ -196,7 +196,7 @@ def measure_stream(dev, n_pages, tier_value, reps=5):
     return n_pages * B.PAGE_BYTES / best / 1e6
 
 
-def build_decoder(dev, cfg, host_ratio, batch, n_pool_blocks, max_blocks, seed):
+def build_decoder(dev, cfg, host_ratio, batch, n_pool_blocks, max_blocks, seed, kv_host_modulus=0, kv_prefetch=False):
     import torch
     from paper_2609_13592_b200.llama import LlamaDecoder
     hq, hkv, d, hid, ffn, vocab = (cfg[k] for k in ("n_q_heads", "n_kv_heads", "head_dim", "hidden", "ffn", "vocab"))
@@ -211,12 +211,18 @@ def build_decoder(dev, cfg, host_ratio, batch, n_pool_blocks, max_blocks, seed):
             return (1.0 + 0.02 * torch.randn(hid, generator=g, device=dev)).to(torch.bfloat16)
         return (0.02 * torch.randn(shapes[name], generator=g, device=dev)).to(torch.bfloat16)
 
-    dec = LlamaDecoder(cfg, get_weight, host_ratio, n_pool_blocks, 0, batch, max_blocks, dev)
+    dec = LlamaDecoder(cfg, get_weight, host_ratio, n_pool_blocks, kv_host_modulus, batch, max_blocks, dev,
+                       kv_prefetch=kv_prefetch)
     g = torch.Generator(device=dev)
     g.manual_seed(seed + 7)
     for ly in dec.layers:                      # synthetic context: KV ~ N(0, 1)
         for name in ("k", "v"):
-            ly[name]._hbm.view(torch.bfloat16).normal_(0.0, 1.0, generator=g)
+            hbm = ly[name]._hbm.view(torch.bfloat16)
+            hbm.normal_(0.0, 1.0, generator=g)
+            if ly[name]._host is not None:     # host pages: a copy of device-generated values
+                host = ly[name]._host.view(torch.bfloat16)
+                n = min(host.numel(), hbm.numel())
+                host[:n].copy_(hbm[:n])
     torch.cuda.synchronize(dev)
     return dec
 
@@ -227,14 +233,16 @@ class StepDriver:
     def __init__(self, dec, dev, batch, ctx0, n_steps, max_blocks):
         import torch
         self.dec, self.dev, self.batch, self.ctx0, self.max_blocks = dec, dev, batch, ctx0, max_blocks
+        ctx0 = np.broadcast_to(np.asarray(ctx0, np.int64), (batch,))   # one length, or one per sequence
         need0 = (ctx0 + 15) // 16
         self.table = np.zeros((batch, max_blocks), np.int32)
         self.n_have = np.zeros(batch, np.int64)
-        for j in range(need0):                 # round-robin growth through the wave-aware pool
+        for j in range(int(need0.max())):      # round-robin growth through the wave-aware pool
             for b in range(batch):
-                self.table[b, j] = dec.pool.alloc(b, 1)[0]
+                if j < need0[b]:
+                    self.table[b, j] = dec.pool.alloc(b, 1)[0]
         self.n_have[:] = need0
-        self.ctx = np.full(batch, ctx0 - 1, np.int64)   # the first step brings it to ctx0
+        self.ctx = ctx0 - 1                             # the first step brings it to ctx0
         self.torch = torch
 
     def advance(self):
@@ -252,9 +260,10 @@ class StepDriver:
             self.dec.pool.free(b)
 
 
-def timed_device_steps(dec, dev, batch, ctx0, warmup, steps, max_blocks, dist_ctx):
+def timed_device_steps(dec, dev, batch, ctx0, warmup, steps, max_blocks, dist_ctx, prefetch=False, profile=True):
     """Device-resident loop: inputs already in HBM; K steps between two events."""
     import torch
+    step_fn = dec.step_prefetch if prefetch else dec.step
     drv = StepDriver(dec, dev, batch, ctx0, warmup + steps, max_blocks)
     ctx_all = np.zeros((warmup + steps, batch), np.int32)
     for i in range(warmup + steps):
@@ -266,18 +275,21 @@ def timed_device_steps(dec, dev, batch, ctx0, warmup, steps, max_blocks, dist_ct
     stream = torch.cuda.current_stream(dev)
     launches = 0
     for i in range(warmup):
-        dec.step(tok[i % 2], table_dev, ctx_dev[i], tok[(i + 1) % 2], stream)
+        step_fn(tok[i % 2], table_dev, ctx_dev[i], tok[(i + 1) % 2], stream)
     dist_ctx.barrier()
     torch.cuda.synchronize(dev)
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record(stream)
     for i in range(warmup, warmup + steps):
-        launches += dec.step(tok[i % 2], table_dev, ctx_dev[i], tok[(i + 1) % 2], stream)
+        launches += step_fn(tok[i % 2], table_dev, ctx_dev[i], tok[(i + 1) % 2], stream)
     e1.record(stream)
     torch.cuda.synchronize(dev)
     dist_ctx.barrier()
     ms = e0.elapsed_time(e1)
     kv_tokens = int(ctx_all[warmup:].sum())
+    if not profile:
+        drv.release()
+        return ms, launches, kv_tokens, None, None
     # per-kind device time of one more step (events around every launch)
     i = warmup + steps - 1
     from paper_2609_13592_b200 import binding as B
@@ -479,6 +491,73 @@ def run_ours(args, rank, world, local_rank):
     dist_ctx.close()
 
 
+def run_kv_spill(args):
+    """Configuration 5: Llama-3-8B-shaped decode, batch 128, context lengths uniform in
+    [2048, 4096]; the pool keeps one page in five of every KV tensor in host memory (an HBM
+    budget of 80 % of the pages).  Three runs of the same kernels: host pages read in place by
+    the SMs (the tiered path), the prefetch-to-HBM variant (copy engine, two layers ahead), and
+    HBM-only at the largest batch whose blocks fit the 80 % budget.  One JSON line."""
+    import torch
+    from paper_2609_13592_b200 import binding as B
+    from paper_2609_13592_b200 import build as libbuild
+    from paper_2609_13592_b200 import synth
+    libbuild.build_library()
+    B.lib()
+    dev = torch.device("cuda:0")
+    torch.cuda.set_device(dev)
+    hbm_peak, peak_src = load_peaks()
+    link_gbs = measure_stream(dev, 64, 1)
+    cfg = dict(synth.LLAMA3_8B)
+    if args.layers:
+        cfg["n_layers"] = args.layers
+    batch = args.batch if args.batch != 32 else 128
+    steps, warmup = min(args.steps, 5), 3
+    total_steps = warmup + steps
+    ctx0 = synth.ctx_lens_uniform(batch, 2048, 4096, seed=5).astype(np.int64)
+    blocks = (ctx0 + total_steps + 15) // 16 + 1
+    max_blocks = int(blocks.max())
+    n_pool_blocks = -(-int(blocks.sum()) // 512) * 512
+    # HBM-only comparison: the longest prefix of the batch whose blocks fit 80 % of the pool
+    budget = int(0.8 * n_pool_blocks) // 512 * 512
+    small = int(np.searchsorted(np.cumsum(blocks), budget, side="right"))
+    null = DistCtx(0, 1, dev)
+    out = {}
+    for label, b_run, pool_blocks, modulus, prefetch in (("tiered", batch, n_pool_blocks, 5, False),
+                                                         ("prefetch", batch, n_pool_blocks, 5, True),
+                                                         ("hbm_only", small, budget, 0, False)):
+        dec = build_decoder(dev, cfg, 0.0, b_run, pool_blocks, max_blocks, seed=1, kv_host_modulus=modulus,
+                            kv_prefetch=prefetch)
+        ms, launches, kv_tokens, _, _ = timed_device_steps(dec, dev, b_run, ctx0[:b_run], warmup, steps, max_blocks,
+                                                           null, prefetch=prefetch, profile=False)
+        host_pages = dec.layers[0]["k"].n_host
+        kv_bytes = kv_tokens / steps * dec.kv_bytes_per_token()
+        host_share = host_pages / dec.layers[0]["k"].n_pages
+        out[label] = {"batch": b_run, "ms_per_step": ms / steps, "tokens_per_s": b_run / (ms / steps / 1e3),
+                      "kv_bytes_per_step": kv_bytes, "host_kv_bytes_per_step": kv_bytes * host_share,
+                      "weight_bytes": dec.weight_bytes(), "launches_per_step": launches // steps,
+                      "pool_blocks": pool_blocks, "kv_host_pages_per_tensor": host_pages,
+                      "status": dec.status_words()}
+        del dec
+        torch.cuda.empty_cache()
+    t = out["tiered"]
+    bytes_step = t["weight_bytes"] + t["kv_bytes_per_step"]
+    t_min_ms = 1e3 * max((bytes_step - t["host_kv_bytes_per_step"]) / (hbm_peak * 1e9),
+                         t["host_kv_bytes_per_step"] / (link_gbs * 1e9))
+    line = {"metric": "decode_tokens_per_s", "value": t["tokens_per_s"], "unit": "tokens/s", "n_gpus": 1,
+            "steps": steps, "warmup": warmup, "ms_per_step": t["ms_per_step"], "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": "llama3_8b_shaped_decode_b128_ctx2048_4096_kv_spill_one_page_in_five",
+                       "batch": batch, "layers": cfg["n_layers"], "kv_placement": "pool, host modulus 5",
+                       "weight_placement": "HBM"},
+            "host_link_gbs": link_gbs, "hbm_peak_gbs": hbm_peak, "hbm_peak_source": peak_src,
+            "combined_read_gbs": bytes_step / (t["ms_per_step"] / 1e3) / 1e9,
+            "combined_roofline_gbs": hbm_peak + link_gbs,
+            "tier_bound": {"t_min_ms": t_min_ms, "frac_of_t_min": t_min_ms / t["ms_per_step"],
+                           "note": "the host share (20 %) is far above the link share of this box, so the step is link-bound"},
+            "runs": out}
+    print(json.dumps(line), flush=True)
+
+
 def run_stream_sweep(args):
     """Configuration 3: tiered streaming-read sweep.  A bf16 buffer of 1 / 4 / 16 (/ 64) GiB is
     reduced by the stream-reduce kernel (full waves of 4 threadblocks per SM) with the host
@@ -546,8 +625,10 @@ def main():
     ap.add_argument("--ctx", type=int, default=2048)
     ap.add_argument("--layers", type=int, default=0, help="override the layer count (0 = 32)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--workload", default="decode", choices=["decode", "stream_sweep"],
-                    help="decode: the benchmark line; stream_sweep: the placement sweep of configuration 3")
+    ap.add_argument("--workload", default="decode", choices=["decode", "stream_sweep", "kv_spill"],
+                    help="decode: the benchmark line; stream_sweep: the placement sweep of configuration 3; "
+                         "kv_spill: configuration 5 (batch 128, one KV page in five on the host) with its "
+                         "HBM-only and prefetch-to-HBM comparison runs")
     ap.add_argument("--sweep-gib", default="1,4,16")
     ap.add_argument("--sweep-seeds", type=int, default=5)
     args = ap.parse_args()
@@ -555,7 +636,10 @@ def main():
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    if args.workload == "stream_sweep":
+    if args.workload == "kv_spill":
+        if rank == 0:
+            run_kv_spill(args)
+    elif args.workload == "stream_sweep":
         if rank == 0:
             run_stream_sweep(args)
     elif args.impl == "reference":
