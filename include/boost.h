@@ -327,6 +327,13 @@ typedef struct {
   const void* const* v_page_ptr2; /* device or NULL */
 } boost_gemv_epilogue_t;
 
+/* Batches of at least m_b rows run on the tcgen05 kernel (operands from shared memory through
+ * matrix descriptors, accumulators in tensor memory), smaller ones down to 3 rows on the
+ * mma.sync kernel; 1 and 2 rows always use the CUDA cores.  Process-wide; the results of the
+ * two tensor-core kernels agree to fp32 rounding.  Default 33 (measured crossover on B200).  The paper has no counterpart
+ * (its matrix products are library kernels, Sec. 4.1). */
+int boost_gemv_set_tc_min_batch(uint32_t m_b);
+
 /* boost_gemv_tiered with an epilogue descriptor (NULL = plain). */
 int boost_gemv_tiered_fused(const void* const* w_page_ptr /*device*/, const uint32_t* w_order /*device*/,
                             size_t n_pages, size_t n_host_pages, uint32_t N, uint32_t K,

@@ -55,15 +55,17 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
 // Bounded wait on an mbarrier phase.  On a timeout the error is recorded in *status and the
 // caller simply carries on (its data is wrong, the host sees the status word), so that no
 // thread is left behind waiting for an arrival that never comes.
-__device__ __forceinline__ void mbar_wait(uint64_t* bar, uint32_t parity, uint32_t* status) {
-  if (mbar_try_wait(bar, parity)) return;
+// Returns false when it gave up.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, uint32_t* status) {
+  if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
   while (!mbar_try_wait(bar, parity)) {
     if (clock64() - t0 > kWaitLimitCycles) {
       atomicOr(status, kErrWaitTimeout);
-      return;
+      return false;
     }
   }
+  return true;
 }
 
 // Bulk asynchronous copy global -> shared through the TMA unit; completion is counted in
@@ -128,6 +130,69 @@ __device__ __forceinline__ uint4 ld_stream_16(const void* p) {
                : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
                : "l"(p));
   return v;
+}
+
+// ---- 5th-generation tensor cores (tcgen05): accumulators live in tensor memory (TMEM), the
+// operands are read from shared memory through 64-bit matrix descriptors, one thread issues.
+
+// Allocate n_cols (a power of two >= 32) TMEM columns; the base address lands in *dst_smem.
+// Executed by one whole warp, which also frees them with tmem_dealloc.
+__device__ __forceinline__ void tmem_alloc(uint32_t* dst_smem, uint32_t n_cols) {
+  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(dst_smem)), "r"(n_cols)
+               : "memory");
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t n_cols) {
+  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(n_cols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before_sync() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after_sync() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+// Writes made through the load/store path (cp.async, st.shared) become visible to the
+// asynchronous proxy, through which the tensor cores read shared memory.
+__device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+// Shared-memory matrix descriptor of a K-major bf16 tile in the 128-byte swizzle: rows of
+// 128 bytes (64 values of k), 16-byte chunk c of row r stored at chunk c ^ (r & 7), groups of
+// 8 rows 1024 bytes apart, tile base 1024-byte aligned.  `addr` may be advanced by 32 bytes
+// per 16 values of k inside the row.
+__device__ __forceinline__ uint64_t umma_desc_k_sw128(uint32_t addr) {
+  return (uint64_t)((addr >> 4) & 0x3FFFu)   // start address
+         | ((uint64_t)1 << 16)               // leading byte offset (unused inside one swizzle row): 16 B
+         | ((uint64_t)(1024 >> 4) << 32)     // stride byte offset: 8-row groups 1024 B apart
+         | ((uint64_t)1 << 46)               // descriptor version of this architecture
+         | ((uint64_t)2 << 61);              // layout type: 128-byte swizzle
+}
+// Instruction descriptor: D fp32 = A bf16 (K-major, M rows) x B bf16 (K-major, N rows)^T.
+__device__ __forceinline__ constexpr uint32_t umma_idesc_bf16_f32(uint32_t M, uint32_t N) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((N >> 3) << 17) | ((M >> 4) << 24);
+}
+// D[tmem] (+)= A[smem] * B[smem]^T, K = 16; accumulate = 0 overwrites D.
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                          uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, {%5, %5, %5, %5}, p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(0u)
+      : "memory");
+}
+// Arrive (count one) on `bar` when every MMA this thread has issued so far has completed.
+__device__ __forceinline__ void umma_commit(uint64_t* bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
+               : "memory");
+}
+// 16 consecutive fp32 columns of this thread's TMEM lane (lane = 32 * (warp % 4) + lane id).
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, float (&v)[16]) {
+  uint32_t r[16];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr)
+      : "memory");
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+  for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
 }
 
 // Two bf16 packed in a 32-bit word -> two floats (bf16 is the top half of an fp32).

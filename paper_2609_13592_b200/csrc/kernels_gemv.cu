@@ -141,13 +141,13 @@ __device__ __forceinline__ float round_bf16(float v) { return __bfloat162float(_
 //           into the paged cache at the position of the new token.
 // The row scale is rsqrt(mean(x^2) + eps) from per-tile sums of squares of the rows of x:
 // RMSNorm whose weight has been folded into the packed matrix.
-template <uint32_t kXRows>
+template <uint32_t kXRows, uint32_t kThreads = kConsumerThreads>
 __device__ __forceinline__ void combine_tile(const GemvParams& p, uint32_t row_tile, uint32_t n_seg, uint32_t tid,
                                              uint32_t* status) {
   const float4* base = reinterpret_cast<const float4*>(p.partials + (size_t)row_tile * p.max_seg * kXRows * kBlockRows);
   constexpr uint32_t kVecRow = kBlockRows / 4;   // float4 per batch row
   const uint32_t n_pairs = p.M_b * 16;
-  for (uint32_t pidx0 = 0; pidx0 < n_pairs; pidx0 += kConsumerThreads) {
+  for (uint32_t pidx0 = 0; pidx0 < n_pairs; pidx0 += kThreads) {
     const uint32_t pidx = pidx0 + tid;
     const bool valid = pidx < n_pairs;
     const uint32_t m = valid ? (pidx >> 4) : 0u, v = pidx & 15u;
@@ -377,13 +377,20 @@ __global__ void __launch_bounds__(kGemvThreads, (NT >= 8 ? 1 : 2)) gemv_tiered_k
           uint32_t seg = blockIdx.x - part_owner((uint64_t)row_tile * p.k_blocks, G, T);
           if (leader && b0 < b1) TRACE_ONCE(8 + 8 * ph + 0);
           const uint32_t c = lane & 7, m0 = lane >> 3;
+          // the page address is looked up once per page, not once per block: a table look-up per
+          // block would put an L2 round trip between any two copies of this warp
+          const uint8_t* page_base = nullptr;
+          uint32_t page_of_base = 0xFFFFFFFFu;
           for (uint32_t b = b0; b < b1; ++b) {
             const bool seg_first = (b == b0) || kb == 0, seg_last = (b + 1 == b1) || (kb + 1 == p.k_blocks);
             if (leader) {
               uint8_t* wdst = smem + (size_t)stage * kStageBytes;
               if (lane == 0) {
-                const uint8_t* src = static_cast<const uint8_t*>(p.w_page_ptr[b / kBlocksPerPage]) +
-                                     (size_t)(b % kBlocksPerPage) * kBlockBytes;
+                if (b / kBlocksPerPage != page_of_base) {
+                  page_of_base = b / kBlocksPerPage;
+                  page_base = static_cast<const uint8_t*>(p.w_page_ptr[page_of_base]);
+                }
+                const uint8_t* src = page_base + (size_t)(b % kBlocksPerPage) * kBlockBytes;
                 mbar_wait(&empty_bar[stage], phase ^ 1u, status);
                 meta[stage] = make_uint4(row_tile, seg, (seg_first ? kFlagFirst : 0u) | (seg_last ? kFlagLast : 0u), ph);
                 mbar_arrive_expect_tx(&full_bar[stage], kBlockBytes);
@@ -680,6 +687,338 @@ __global__ void __launch_bounds__(kGemvThreads, (NT >= 8 ? 1 : 2)) gemv_tiered_k
   if (warp == 0) TRACE(7);
 }
 
+// ---------------------------------------------------------------------------------------------
+// The same product on the 5th-generation tensor cores, for batches where it is a real dense
+// contraction.  A packed weight block is already the A operand the hardware wants (128 rows,
+// K-major, 128-byte swizzle); the activations of the block's 64 columns are staged as the B
+// operand (NPAD rows, same layout); one thread issues four tcgen05.mma (K = 16 each) per block
+// and the 128 x NPAD fp32 accumulator lives in tensor memory, double-buffered so that the
+// next segment accumulates while four epilogue warps read the finished one back
+// (tcgen05.ld), write the partial sums and run the same combine as the kernel above.
+// Warps: 0-7 epilogue (warp w reads TMEM lanes 32 (w % 4) .. + 31 = weight rows, and the half
+// w / 4 of the accumulator's columns), 8 MMA issue and TMEM allocation, 9 weight producer,
+// 10-13 activation producers.  One threadblock per SM (the driver keeps kernels that allocate
+// tensor memory at one per SM at this shared-memory size) with the whole shared memory as its
+// ring: no warp reads an operand back, so the ring's bandwidth is all HBM's.
+constexpr uint32_t kTcEpiWarps = 8;
+constexpr uint32_t kTcEpiThreads = kTcEpiWarps * 32;
+constexpr uint32_t kTcXWarps = 4;   // activation producer warps: rows m with (m / 4) % 4 == their index
+constexpr uint32_t kTcThreads = kTcEpiThreads + 64 + 32 * kTcXWarps;
+
+__host__ __device__ constexpr uint32_t tc_stage_bytes(uint32_t npad) { return kBlockBytes + npad * 128u; }
+
+template <uint32_t NPAD>
+__global__ void __launch_bounds__(kTcThreads, 1) gemv_tc_kernel(const __grid_constant__ ChainParams cp) {
+  constexpr uint32_t kStageBytes = tc_stage_bytes(NPAD);
+  constexpr uint32_t kTmemCols = 2 * NPAD < 32 ? 32 : 2 * NPAD;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  __shared__ uint64_t full_bar[kMaxStages];
+  __shared__ uint64_t empty_bar[kMaxStages];
+  __shared__ uint4 meta[kMaxStages];
+  __shared__ uint64_t item_full[4];
+  __shared__ uint64_t item_empty[4];
+  __shared__ uint32_t item_ring[4];
+  __shared__ uint64_t acc_full[2];
+  __shared__ uint64_t acc_empty[2];
+  __shared__ uint4 acc_meta[2];
+  __shared__ uint32_t s_old;
+  __shared__ uint32_t s_tmem;
+  __shared__ uint32_t s_go[2];          // epilogue: thread 0's wait on an accumulator succeeded
+  __shared__ volatile uint32_t s_abort; // a bounded wait ran out somewhere: everybody winds down
+
+  const uint32_t tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const uint32_t n_stages = cp.ph[0].n_stages;
+  const uint32_t n_phases = cp.n_phases;
+  uint32_t* status = cp.ph[0].ws + kWsStatus;
+
+  pdl_launch_dependents();
+  if (tid == 0) {
+    for (uint32_t s = 0; s < n_stages; ++s) {
+      mbar_init(&full_bar[s], 33 + 32 * kTcXWarps);   // cp.async arrivals of the producer warps + the arrive.expect_tx
+      mbar_init(&empty_bar[s], 1);   // the commit of the MMAs that read the stage
+    }
+    for (uint32_t s = 0; s < 4; ++s) {
+      mbar_init(&item_full[s], 1);
+      mbar_init(&item_empty[s], kTcXWarps);
+    }
+    for (uint32_t s = 0; s < 2; ++s) {
+      mbar_init(&acc_full[s], 1);
+      mbar_init(&acc_empty[s], kTcEpiWarps);
+    }
+    s_abort = 0;
+    fence_barrier_init();
+  }
+  if (warp == kTcEpiWarps) tmem_alloc(&s_tmem, kTmemCols);
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem_base = s_tmem;
+
+  if (warp > kTcEpiWarps) {
+    // ------------------------------------------------------------------ producer warps (as above)
+    const bool leader = (warp == kTcEpiWarps + 1);
+    const uint32_t xw = warp - (kTcEpiWarps + 2);   // index among the activation producer warps
+    uint32_t stage = 0, phase = 0, icount = 0;
+    for (uint32_t ph = 0; ph < n_phases; ++ph) {
+      const GemvParams& p = cp.ph[ph];
+      const uint32_t n_host_items = p.n_host_pages * p.items_per_page;
+      TierQueues q;
+      const bool active = blockIdx.x < p.active_ctas;
+      if (active && !p.even_part) q.init(p.queue, n_host_items, p.n_pages * p.items_per_page, p.n_host_ctas, blockIdx.x, p.active_ctas);
+      if (ph == 0) {
+        if (!leader || !p.early) pdl_wait();
+      } else if (!leader) {
+        if (lane == 0) grid_counter_wait(cp.bar + (ph - 1), gridDim.x, status);
+        __syncwarp();
+      }
+      // one block: the weight warp copies it, the activation warp stages x[:, 64 kb .. 64 kb + 64)
+      // as NPAD rows of 128 bytes in the 128-byte swizzle (rows >= M_b are zero)
+      auto produce = [&](const uint8_t* src, bool from_host, uint32_t row_tile, uint32_t seg, uint32_t flags, uint32_t kb) {
+        if (s_abort) return;
+        if (leader) {
+          uint8_t* wdst = smem + (size_t)stage * kStageBytes;
+          if (lane == 0) {
+            if (!mbar_wait(&empty_bar[stage], phase ^ 1u, status)) s_abort = 1;
+            meta[stage] = make_uint4(row_tile, seg, flags, ph);
+            mbar_arrive_expect_tx(&full_bar[stage], from_host ? 0u : kBlockBytes);
+            if (!from_host) bulk_copy_g2s(wdst, src, kBlockBytes, &full_bar[stage]);
+          }
+          __syncwarp();
+          if (from_host) {
+#pragma unroll 8
+            for (uint32_t idx = lane; idx < kBlockBytes / 16; idx += 32) cp_async_16(wdst + idx * 16, src + idx * 16, 16u);
+          }
+          cp_async_arrive_noinc(&full_bar[stage]);
+        } else {
+          if (!mbar_wait(&empty_bar[stage], phase ^ 1u, status)) s_abort = 1;
+          const uint32_t c = lane & 7, m0 = (lane >> 3) + 4 * xw;
+          uint8_t* xbase = smem + (size_t)stage * kStageBytes + kBlockBytes;
+          const uint32_t k = kb * kBlockK + c * 8;
+          const bool k_ok = k < p.K;
+#pragma unroll 4
+          for (uint32_t m = m0; m < NPAD; m += 4 * kTcXWarps) {
+            const bool live = k_ok && m < p.M_b;
+            cp_async_16(xbase + m * 128 + ((c ^ (m & 7)) << 4), p.x + (live ? (size_t)m * p.K + k : 0u), live ? 16u : 0u);
+          }
+          cp_async_arrive_noinc(&full_bar[stage]);
+        }
+        if (++stage == n_stages) { stage = 0; phase ^= 1u; }
+      };
+      if (p.even_part) {
+        const uint32_t G = p.active_ctas, T = p.total_blocks;
+        if (blockIdx.x < G) {
+          const uint32_t b0 = (uint32_t)((uint64_t)blockIdx.x * T / G), b1 = (uint32_t)((uint64_t)(blockIdx.x + 1) * T / G);
+          uint32_t row_tile = b0 / p.k_blocks, kb = b0 % p.k_blocks;
+          uint32_t seg = blockIdx.x - part_owner((uint64_t)row_tile * p.k_blocks, G, T);
+          const uint8_t* page_base = nullptr;   // looked up once per page (an L2 round trip)
+          uint32_t page_of_base = 0xFFFFFFFFu;
+          for (uint32_t b = b0; b < b1; ++b) {
+            const bool seg_first = (b == b0) || kb == 0, seg_last = (b + 1 == b1) || (kb + 1 == p.k_blocks);
+            const uint8_t* src = nullptr;
+            if (leader && lane == 0) {
+              if (b / kBlocksPerPage != page_of_base) {
+                page_of_base = b / kBlocksPerPage;
+                page_base = static_cast<const uint8_t*>(p.w_page_ptr[page_of_base]);
+              }
+              src = page_base + (size_t)(b % kBlocksPerPage) * kBlockBytes;
+            }
+            produce(src, false, row_tile, seg, (seg_first ? kFlagFirst : 0u) | (seg_last ? kFlagLast : 0u), kb);
+            if (++kb == p.k_blocks) { kb = 0; ++row_tile; seg = 0; }
+          }
+        }
+      } else {
+        for (;;) {
+          const uint32_t slot = icount & 3u, iphase = (icount >> 2) & 1u;
+          uint32_t qi = 0;
+          if (leader) {
+            if (lane == 0) {
+              for (;;) {   // skip the unused tail of the last page
+                qi = active ? q.next() : 0xFFFFFFFFu;
+                if (qi == 0xFFFFFFFFu) break;
+                if (p.w_order[qi / p.items_per_page] * p.items_per_page + qi % p.items_per_page < p.n_items) break;
+              }
+              if (!mbar_wait(&item_empty[slot], iphase ^ 1u, status)) { s_abort = 1; qi = 0xFFFFFFFFu; }
+              item_ring[slot] = qi;
+              mbar_arrive(&item_full[slot]);
+            }
+            qi = __shfl_sync(0xFFFFFFFFu, qi, 0);
+          } else {
+            const bool got = mbar_wait(&item_full[slot], iphase, status);
+            qi = got ? item_ring[slot] : 0xFFFFFFFFu;
+            if (!got) s_abort = 1;
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&item_empty[slot]);
+          }
+          ++icount;
+          if (qi == 0xFFFFFFFFu) break;
+          const uint32_t page = p.w_order[qi / p.items_per_page];
+          const uint32_t first_blk = (page * p.items_per_page + qi % p.items_per_page) * p.run;
+          const uint32_t row_tile = first_blk / p.k_blocks, kb0 = first_blk % p.k_blocks;
+          const bool from_host = qi < n_host_items;
+          const uint8_t* src = static_cast<const uint8_t*>(p.w_page_ptr[page]) + (size_t)(first_blk % kBlocksPerPage) * kBlockBytes;
+          for (uint32_t j = 0; j < p.run; ++j, src += kBlockBytes)
+            produce(src, from_host, row_tile, kb0 / p.run, (j == 0 ? kFlagFirst : 0u) | (j + 1 == p.run ? kFlagLast : 0u), kb0 + j);
+        }
+      }
+      // a stage without data tells the MMA warp that the phase (or the launch) is over
+      if (leader) {
+        if (lane == 0) {
+          mbar_wait(&empty_bar[stage], phase ^ 1u, status);
+          meta[stage] = make_uint4(0u, 0u, ph + 1 == n_phases ? kFlagStop : kFlagPhaseEnd, ph);
+          mbar_arrive(&full_bar[stage]);
+        }
+        __syncwarp();
+        cp_async_arrive_noinc(&full_bar[stage]);
+        if (lane == 0 && active && !p.even_part) q.finish(p.active_ctas);
+      } else {
+        mbar_wait(&empty_bar[stage], phase ^ 1u, status);
+        cp_async_arrive_noinc(&full_bar[stage]);
+      }
+      if (++stage == n_stages) { stage = 0; phase ^= 1u; }
+    }
+    return;
+  }
+
+  if (warp == kTcEpiWarps) {
+    // ------------------------------------------------------------------ MMA warp: one thread issues
+    if (lane == 0) {
+      constexpr uint32_t idesc = umma_idesc_bf16_f32(kBlockRows, NPAD);
+      uint32_t stage = 0, phase = 0, buf = 0, buf_phase = 0, accumulate = 0;
+      for (;;) {
+        if (s_abort || !mbar_wait(&full_bar[stage], phase, status)) { s_abort = 1; break; }
+        const uint4 mt = meta[stage];
+        if (mt.z & (kFlagStop | kFlagPhaseEnd)) {
+          // hand the marker to the epilogue warps in order with the segments
+          if (!mbar_wait(&acc_empty[buf], buf_phase ^ 1u, status)) { s_abort = 1; break; }
+          acc_meta[buf] = mt;
+          mbar_arrive(&acc_full[buf]);
+          if (++buf == 2) { buf = 0; buf_phase ^= 1u; }
+          mbar_arrive(&empty_bar[stage]);
+          if (++stage == n_stages) { stage = 0; phase ^= 1u; }
+          if (mt.z & kFlagStop) break;
+          continue;
+        }
+        if (mt.z & kFlagFirst) {
+          if (!mbar_wait(&acc_empty[buf], buf_phase ^ 1u, status)) { s_abort = 1; break; }   // the epilogue has read this accumulator
+          accumulate = 0;
+        }
+        fence_proxy_async_smem();   // x (and host-tier weight blocks) were written through the load/store path
+        tc_fence_after_sync();
+        const uint32_t wbase = smem_u32(smem + (size_t)stage * kStageBytes);
+        const uint32_t xbase = wbase + kBlockBytes;
+#pragma unroll
+        for (uint32_t ks = 0; ks < kBlockK / 16; ++ks) {
+          umma_bf16(tmem_base + buf * NPAD, umma_desc_k_sw128(wbase + ks * 32), umma_desc_k_sw128(xbase + ks * 32), idesc,
+                    accumulate);
+          accumulate = 1;
+        }
+        umma_commit(&empty_bar[stage]);   // the stage is free once these MMAs have read it
+        if (mt.z & kFlagLast) {
+          acc_meta[buf] = mt;
+          umma_commit(&acc_full[buf]);    // the accumulator is complete once they have finished
+          if (++buf == 2) { buf = 0; buf_phase ^= 1u; }
+        }
+        if (++stage == n_stages) { stage = 0; phase ^= 1u; }
+      }
+    }
+    __syncwarp();
+    named_barrier_sync(2, kTcEpiThreads + 32);   // the epilogue warps have read everything
+    tmem_dealloc(tmem_base, kTmemCols);
+    return;
+  }
+
+  // -------------------------------------------------------------------- epilogue warps
+  uint32_t* tile_cnt = cp.ph[0].ws + kWsHeaderWords;
+  uint32_t buf = 0, buf_phase = 0;
+  pdl_wait();
+  for (;;) {
+    // thread 0 waits for the accumulator (or marker) and tells the others, so that all 128
+    // threads take the same way out if the wait runs out
+    if (tid == 0) {
+      const bool ok = mbar_wait(&acc_full[buf], buf_phase, status);
+      if (!ok) s_abort = 1;
+      s_go[buf] = ok ? 1u : 0u;
+    }
+    named_barrier_sync(1, kTcEpiThreads);
+    if (!s_go[buf]) break;
+    const uint4 mt = acc_meta[buf];
+    if (mt.z & (kFlagStop | kFlagPhaseEnd)) {
+      if (n_phases > 1) {
+        named_barrier_sync(1, kTcEpiThreads);
+        if (tid == 0) {
+          __threadfence();
+          if (mt.z & kFlagPhaseEnd) {
+            atomicAdd(cp.bar + mt.w, 1u);
+          } else {
+            const uint32_t old = atomicAdd(cp.bar + kMaxPhases, 1u);
+            if (old == gridDim.x - 1) {
+              for (uint32_t i = 0; i <= kMaxPhases; ++i) cp.bar[i] = 0u;
+              __threadfence();
+            }
+          }
+        }
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&acc_empty[buf]);
+      if (++buf == 2) { buf = 0; buf_phase ^= 1u; }
+      if (mt.z & kFlagStop) break;
+      continue;
+    }
+    tc_fence_after_sync();
+    const GemvParams& p = cp.ph[mt.w];
+    const uint32_t row_tile = mt.x, split = mt.y;
+    uint32_t n_seg = p.splits;
+    if (p.even_part) {
+      const uint64_t t0 = (uint64_t)row_tile * p.k_blocks;
+      n_seg = part_owner(t0 + p.k_blocks - 1, p.active_ctas, p.total_blocks) - part_owner(t0, p.active_ctas, p.total_blocks) + 1;
+    }
+    const bool direct = (n_seg == 1) && p.epi == kEpiPlain && !p.ssq_in && !p.ssq_out;
+    float* part = p.partials + ((size_t)row_tile * p.max_seg + split) * NPAD * kBlockRows;
+    const uint32_t quarter = warp & 3u, half = warp >> 2;
+    const uint32_t nl = quarter * 32 + lane;                                 // weight row of this thread = its TMEM lane
+    const uint32_t taddr = tmem_base + ((quarter * 32u) << 16) + buf * NPAD;
+    // warps 0-3 read the first half of the columns, warps 4-7 the second (16 columns: the first group reads all)
+    constexpr uint32_t kColsPerGroup = NPAD >= 32 ? NPAD / 2 : NPAD;
+    const uint32_t c_begin = half * kColsPerGroup;
+    const uint32_t c_end = (NPAD >= 32 || half == 0) ? c_begin + kColsPerGroup : c_begin;
+    for (uint32_t c0 = c_begin; c0 < c_end; c0 += 16) {
+      float v[16];
+      tmem_ld16(taddr + c0, v);
+#pragma unroll
+      for (uint32_t j = 0; j < 16; ++j) {
+        const uint32_t m = c0 + j;                                           // batch row = accumulator column
+        if (direct) {
+          const uint32_t n = row_tile * kBlockRows + nl;
+          if (m < p.M_b && n < p.N) store_out(p, m, n, v[j]);
+        } else {
+          __stcg(part + m * kBlockRows + nl, v[j]);
+        }
+      }
+    }
+    // the accumulator may be overwritten
+    tc_fence_before_sync();
+    __syncwarp();
+    if (lane == 0) mbar_arrive(&acc_empty[buf]);
+    if (++buf == 2) { buf = 0; buf_phase ^= 1u; }
+    if (!direct) {
+      named_barrier_sync(1, kTcEpiThreads);
+      if (tid == 0) {
+        __threadfence();
+        s_old = atomicAdd(tile_cnt + row_tile, 1u);
+      }
+      named_barrier_sync(1, kTcEpiThreads);
+      if (s_old == n_seg - 1) {
+        __threadfence();
+        combine_tile<NPAD, kTcEpiThreads>(p, row_tile, n_seg, tid, status);
+        if (tid == 0) tile_cnt[row_tile] = 0;
+      }
+      named_barrier_sync(1, kTcEpiThreads);
+    }
+  }
+  named_barrier_sync(2, kTcEpiThreads + 32);
+}
+
 // Packed form: 16-byte chunk `pos` of row r of block (t, kb) holds columns
 // [64 kb + 8 c, +8) of packed row 128 t + r with c = pos ^ (r & 7).  Packed row -> weight row:
 // identity, or (row_mode 1) rows 0..63 of a tile = rows [64 t, 64 t + 64) of the first half of
@@ -734,31 +1073,31 @@ uint32_t pick_run(uint32_t n_row_tiles, uint32_t k_blocks) {
   return 1;
 }
 
-template <int NT, int MB>
-int launch_gemv(const ChainParams& chain, int sms, cudaStream_t stream) {
-  constexpr uint32_t kStage = stage_bytes_of(NT, MB);
+// Common launch path of the two kernels: ring depth from the shared-memory budget, grid and
+// per-phase threadblock counts, host-tier threadblocks.  `state` keeps what is set up once per
+// kernel instantiation.
+struct KernelState {
+  bool configured = false;
+  int resident = 0;   // threadblocks of the kernel that one SM holds at its shared-memory size
+};
+
+int launch_planned(void (*kernel)(ChainParams), KernelState& state, uint32_t threads, uint32_t stage_bytes,
+                   uint32_t ctas_per_sm, const ChainParams& chain, int sms, cudaStream_t stream) {
   ChainParams c = chain;
-  // Two threadblocks per SM where registers allow: a second ring hides the producer /
-  // consumer hand-over latency of the first (measured: +25 % bandwidth on B200).
-  uint32_t ctas_per_sm = (NT >= 8) ? 1 : 2;
-  uint32_t n_stages = (kSmemBudget / ctas_per_sm - 1024) / kStage;
+  uint32_t n_stages = (kSmemBudget / ctas_per_sm - 1024) / stage_bytes;
   if (n_stages > kMaxStages) n_stages = kMaxStages;
-  const size_t smem = (size_t)n_stages * kStage + 1024;
-  static bool configured = false;
-  static int resident = 0;   // threadblocks of this kernel that one SM holds at this shared-memory size
-  if (!configured) {
-    int rc = boosth::check(cudaFuncSetAttribute(gemv_tiered_kernel<NT, MB>,
-                                                cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(kSmemBudget + 1024)));
+  const size_t smem = (size_t)n_stages * stage_bytes + 1024;
+  if (!state.configured) {
+    int rc = boosth::check(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(kSmemBudget + 1024)));
     if (rc != BOOST_OK) return rc;
-    rc = boosth::check(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&resident, gemv_tiered_kernel<NT, MB>,
-                                                                     (int)kGemvThreads, smem));
+    rc = boosth::check(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&state.resident, kernel, (int)threads, smem));
     if (rc != BOOST_OK) return rc;
-    configured = true;
+    state.configured = true;
   }
   if (c.n_phases > 1) {
     // the phases of a chain meet at grid-wide counters: every threadblock must be resident
-    if (resident < 1) return BOOST_ERR_UNSUPPORTED;
-    if ((uint32_t)resident < ctas_per_sm) ctas_per_sm = (uint32_t)resident;
+    if (state.resident < 1) return BOOST_ERR_UNSUPPORTED;
+    if ((uint32_t)state.resident < ctas_per_sm) ctas_per_sm = (uint32_t)state.resident;
   }
   const uint32_t max_ctas = (uint32_t)sms * ctas_per_sm;
   uint32_t grid = 0;
@@ -789,7 +1128,22 @@ int launch_gemv(const ChainParams& chain, int sms, cudaStream_t stream) {
     }
     q.n_host_ctas = n_host_ctas;
   }
-  return boosth::launch_chained(gemv_tiered_kernel<NT, MB>, dim3(grid), dim3(kGemvThreads), smem, stream, c);
+  return boosth::launch_chained(kernel, dim3(grid), dim3(threads), smem, stream, c);
+}
+
+// Two threadblocks per SM where registers allow: a second ring hides the producer / consumer
+// hand-over latency of the first (measured: +25 % bandwidth on B200).
+template <int NT, int MB>
+int launch_gemv(const ChainParams& chain, int sms, cudaStream_t stream) {
+  static KernelState state;
+  return launch_planned(gemv_tiered_kernel<NT, MB>, state, kGemvThreads, stage_bytes_of(NT, MB), (NT >= 8) ? 1 : 2, chain,
+                        sms, stream);
+}
+
+template <uint32_t NPAD>
+int launch_gemv_tc(const ChainParams& chain, int sms, cudaStream_t stream) {
+  static KernelState state;
+  return launch_planned(gemv_tc_kernel<NPAD>, state, kTcThreads, tc_stage_bytes(NPAD), 1, chain, sms, stream);
 }
 
 }  // namespace
@@ -853,7 +1207,7 @@ static uint32_t partial_slots(const boost_weight_layout_t& lay, uint32_t M_b) {
   int sms = boosth::sm_count();
   if (sms <= 0) sms = 148;
   const uint64_t T = (uint64_t)lay.n_row_tiles * lay.k_blocks;
-  uint64_t G = (uint64_t)sms * (gemv_x_rows(M_b) >= 64 ? 1 : 2);
+  uint64_t G = (uint64_t)sms * 2;   // the most threadblocks any of the kernels keeps on an SM
   if (G > T) G = T;
   const uint32_t per = (uint32_t)(T / G);
   const uint32_t even = (lay.k_blocks + per - 1) / per + 1;
@@ -966,17 +1320,25 @@ int fill_params(GemvParams& p, const void* const* w_page_ptr, const uint32_t* w_
   return BOOST_OK;
 }
 
+// Batches from this size on take the tcgen05 kernel, smaller ones (from 3 rows) mma.sync.
+// Measured on B200 on Llama-3-8B-shaped matrices: up to 32 rows the mma.sync kernel (two
+// threadblocks per SM) streams faster; at 64 rows the tcgen05 kernel is 1.5 x, at 128 rows
+// 1.8 x faster, because the mma.sync kernel re-reads the activation tile from shared memory in
+// every warp.
+uint32_t g_tc_min_batch = 33;
+
 int launch_routed(const ChainParams& c, uint32_t M_b, void* stream) {
   const int sms = boosth::sm_count();
   if (sms <= 0) return BOOST_ERR_CUDA;
   cudaStream_t st = (cudaStream_t)stream;
+  const bool tc = M_b >= g_tc_min_batch;
   switch (gemv_x_rows(M_b)) {
     case 1: return launch_gemv<0, 1>(c, sms, st);
     case 2: return launch_gemv<0, 2>(c, sms, st);
-    case 16: return launch_gemv<2, 0>(c, sms, st);
-    case 32: return launch_gemv<4, 0>(c, sms, st);
-    case 64: return launch_gemv<8, 0>(c, sms, st);
-    default: return launch_gemv<16, 0>(c, sms, st);
+    case 16: return tc ? launch_gemv_tc<16>(c, sms, st) : launch_gemv<2, 0>(c, sms, st);
+    case 32: return tc ? launch_gemv_tc<32>(c, sms, st) : launch_gemv<4, 0>(c, sms, st);
+    case 64: return tc ? launch_gemv_tc<64>(c, sms, st) : launch_gemv<8, 0>(c, sms, st);
+    default: return tc ? launch_gemv_tc<128>(c, sms, st) : launch_gemv<16, 0>(c, sms, st);
   }
 }
 
@@ -1044,6 +1406,12 @@ extern "C" int boost_gemv_tiered_chain(const boost_gemv_call_t* calls, uint32_t 
   const size_t usable = (workspace_bytes - sync_bytes) & ~(size_t)255;
   uint32_t* sync_words = reinterpret_cast<uint32_t*>(static_cast<uint8_t*>(workspace) + usable);
   return boosth::gemv_chain_launch(calls, n_calls, M_b, workspace, usable, sync_words, 0, stream);
+}
+
+// Routing threshold between the two tensor-core kernels (measurement and tests).
+extern "C" int boost_gemv_set_tc_min_batch(uint32_t m_b) {
+  g_tc_min_batch = m_b;
+  return BOOST_OK;
 }
 
 #ifdef BOOST_TRACE
