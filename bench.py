@@ -5,10 +5,11 @@ Default workload (N = 1): one Llama-3-8B-shaped decode step - 32 layers, hidden 
 14336, 32 query / 8 KV heads, vocab 128256, bf16 random-init weights N(0, 0.02^2), batch
 32, context 2048 - with weight pages placed by modulo placement at the host share that the
 measured host-link / HBM bandwidth ratio gives, KV cache in HBM.  A step runs every kernel
-of the path through the C ABI: RoPE table, embedding gather, 32 x [QKV product with RMSNorm
-scale, RoPE and KV append in its epilogue; paged attention; output product + residual;
-gate/up product with RMSNorm scale and SwiGLU in its epilogue; down product + residual],
-LM head, argmax - 164 launches.
+of the path through the C ABI: RoPE table, embedding gather, the first layer's QKV product
+(RMSNorm scale, RoPE and KV append in its epilogue), then 32 x [paged attention; ONE launch
+for the output product + residual, the gate/up product with RMSNorm scale and SwiGLU, the
+down product + residual and the next layer's QKV product - the LM head after the last
+layer], argmax - 68 launches.
 
   python bench.py --gpus N --steps K --warmup W            # this repository's kernels
   python bench.py --impl reference ...                      # the CPU oracle on the host cores
@@ -34,9 +35,9 @@ sys.path.insert(0, ROOT)
 WORKLOAD = "llama3_8b_shaped_decode_step_b32_ctx2048_tiered_weights"
 FALLBACK_HBM_GBS = 6650.0
 # DRAM bytes (read + write) per algorithmic byte of the weight-product kernel, from one ncu
-# capture of the gate/up, down and LM-head launches of this workload (profiles/
-# gemv_tiered_kernel_llama8b_m32.md): 1442.3 MB moved for 1403.0 MB of packed weights.
-GEMV_TRAFFIC_PER_ALGORITHMIC_BYTE = 1.028
+# capture of two full-size chain launches of this workload (profiles/
+# gemv_tiered_kernel_chain_llama8b_m32.md): 1955.5 MB moved for 1872.8 MB of packed weights.
+GEMV_TRAFFIC_PER_ALGORITHMIC_BYTE = 1.044
 
 
 def load_peaks():
@@ -466,7 +467,7 @@ def run_ours(args, rank, world, local_rank):
                          "achieved": gemv_gbs, "peak": hbm_peak, "unit": "GB/s", "frac": gemv_gbs / hbm_peak,
                          "algorithmic_bytes_per_launch": gemv_bytes_per_launch,
                          "traffic": GEMV_TRAFFIC_PER_ALGORITHMIC_BYTE * gemv_bytes_per_launch,
-                         "traffic_source": "ncu dram bytes of this workload's launches, ratio 1.028 to algorithmic",
+                         "traffic_source": "ncu dram bytes of this workload's launches, ratio 1.044 to algorithmic",
                          "launches_per_step": gemv_n, "avg_launch_us": 1e3 * gemv_ms / max(gemv_n, 1),
                          "peak_source": peak_src},
             "roofline_attention": {"bound": "hbm", "kernel": "paged_attn_kernel", "achieved": attn_gbs,
