@@ -38,6 +38,14 @@ constexpr uint32_t kAttnThreads = kAttnWarps * 32;
 constexpr uint32_t kWarpStages = 2;                      // ring depth of one warp
 constexpr uint32_t kMaxGroup = 16;
 
+#ifdef BOOST_TRACE
+// Debug build only: per-warp time stamps (global timer, ns), 8 slots per warp.
+__device__ unsigned long long* g_attn_trace = nullptr;
+#define ATRACE(slot) do { if (g_attn_trace && (threadIdx.x & 31) == 0) { unsigned long long t_; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_)); g_attn_trace[((size_t)blockIdx.x * 4 + (threadIdx.x >> 5)) * 8 + (slot)] = t_; } } while (0)
+#else
+#define ATRACE(slot) do { } while (0)
+#endif
+
 struct AttnParams {
   const __nv_bfloat16* q;
   const void* const* k_page_ptr;
@@ -77,7 +85,12 @@ __global__ void __launch_bounds__(kAttnThreads, (NH == 1 ? 3 : 2)) paged_attn_ke
     fence_barrier_init();
   }
   __syncwarp();
-  pdl_wait();   // q and the newest K/V rows come from the kernels just before this one
+  ATRACE(0);
+  // The kernels just before this one produce q and the newest K / V row of every sequence
+  // (in its last block).  Context lengths, block tables and all older blocks are not theirs:
+  // the first item's look-ups, and its first blocks unless one of them is the sequence's
+  // last, are requested before the wait on those kernels.
+  bool waited = false;
 
   // Fragment coordinates: rows gq, gq+8 (tokens for S^T, d for O^T), columns c0, c0+1 (heads).
   const uint32_t gq = lane >> 2, c0 = (lane & 3) * 2;
@@ -94,8 +107,11 @@ __global__ void __launch_bounds__(kAttnThreads, (NH == 1 ? 3 : 2)) paged_attn_ke
     const uint32_t n_blk = (ctx + kTok - 1) / kTok;
     const uint32_t n_splits = n_blk ? (n_blk + p.item_blocks - 1) / p.item_blocks : 1;
     if (split < n_splits) {
-      const uint32_t blk0 = split * p.item_blocks;
-      const uint32_t nb = min(p.item_blocks, n_blk - min(n_blk, blk0));
+      // the sequence's blocks in n_splits runs of equal length (the last may be shorter by a
+      // few): a 129-block sequence is 5 runs of 26, not 4 of 32 and one of 1
+      const uint32_t run_len = n_blk ? (n_blk + n_splits - 1) / n_splits : 0;
+      const uint32_t blk0 = split * run_len;
+      const uint32_t nb = min(run_len, n_blk - min(n_blk, blk0));
       // every lane resolves one block of the item: table entry, page, addresses
       const uint8_t* ksrc = nullptr;
       const uint8_t* vsrc = nullptr;
@@ -138,7 +154,17 @@ __global__ void __launch_bounds__(kAttnThreads, (NH == 1 ? 3 : 2)) paged_attn_ke
         }
         cp_async_arrive_noinc(&full_bar[warp][st]);
       };
-      for (uint32_t i = 0; i < min(nb, kWarpStages); ++i) request(i);
+      const uint32_t n_first = min(nb, kWarpStages);
+      const bool early = !waited && blk0 + n_first + 1 <= n_blk;   // none of them is the last block
+      if (early)
+        for (uint32_t i = 0; i < n_first; ++i) request(i);
+      if (!waited) {
+        pdl_wait();
+        waited = true;
+        ATRACE(1);
+      }
+      if (!early)
+        for (uint32_t i = 0; i < n_first; ++i) request(i);
 
       // q^T as the B operand (k = d, n = head), straight from global while the blocks fly
       uint32_t qb[NH][8][2];
@@ -162,6 +188,7 @@ __global__ void __launch_bounds__(kAttnThreads, (NH == 1 ? 3 : 2)) paged_attn_ke
       for (uint32_t i = 0; i < nb; ++i) {
         const uint32_t st = i % kWarpStages;
         mbar_wait(&full_bar[warp][st], (phase_mask >> st) & 1u, status);
+        if (i == 0) ATRACE(2);
         phase_mask ^= 1u << st;
         const uint32_t kbase = smem_u32(ring + (size_t)st * kStageBytes);
         const uint32_t vbase = kbase + kChunkBytes;
@@ -246,6 +273,7 @@ __global__ void __launch_bounds__(kAttnThreads, (NH == 1 ? 3 : 2)) paged_attn_ke
         if (i + kWarpStages < nb) request(i + kWarpStages);
       }
 
+      ATRACE(3);
       // ---- end of the item: this warp holds the whole chunk run
       const bool single = (n_splits == 1);
 #pragma unroll
@@ -284,8 +312,60 @@ __global__ void __launch_bounds__(kAttnThreads, (NH == 1 ? 3 : 2)) paged_attn_ke
           old = atomicAdd(cnt, 1u);
         }
         old = __shfl_sync(0xFFFFFFFFu, old, 0);
+        ATRACE(4);
         if (old == n_splits - 1) {
           __threadfence();
+          if (p.group == 4) {
+            // four heads side by side: 8 lanes per head, 16 outputs per lane, the loads of two
+            // splits (8 x 16 bytes per lane) in flight at a time
+            const uint32_t r = lane >> 3, c = lane & 7;
+            const uint32_t hq = g * p.group + r;
+            const size_t slot0 = ((size_t)b * p.Hq + hq) * p.max_splits;
+            float m_all = -CUDART_INF_F;
+            for (uint32_t sp = c; sp < n_splits; sp += 8) m_all = fmaxf(m_all, __ldcg(p.part_ml + (slot0 + sp) * 2));
+            m_all = fmaxf(m_all, __shfl_xor_sync(0xFFFFFFFFu, m_all, 1));
+            m_all = fmaxf(m_all, __shfl_xor_sync(0xFFFFFFFFu, m_all, 2));
+            m_all = fmaxf(m_all, __shfl_xor_sync(0xFFFFFFFFu, m_all, 4));
+            float4 acc[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) acc[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+            float l_all = 0.f;
+            for (uint32_t sp0 = 0; sp0 < n_splits; sp0 += 2) {
+              float4 v[2][4];
+              float2 ml[2];
+#pragma unroll
+              for (uint32_t u = 0; u < 2; ++u)
+                if (sp0 + u < n_splits) {
+                  ml[u] = __ldcg(reinterpret_cast<const float2*>(p.part_ml + (slot0 + sp0 + u) * 2));
+#pragma unroll
+                  for (int j = 0; j < 4; ++j)
+                    v[u][j] = __ldcg(reinterpret_cast<const float4*>(p.part_o + (slot0 + sp0 + u) * kD) + c * 4 + j);
+                }
+#pragma unroll
+              for (uint32_t u = 0; u < 2; ++u)
+                if (sp0 + u < n_splits) {
+                  const float f = (ml[u].x == -CUDART_INF_F) ? 0.f : exp2f(ml[u].x - m_all);
+                  l_all += f * ml[u].y;
+#pragma unroll
+                  for (int j = 0; j < 4; ++j) {
+                    acc[j].x += f * v[u][j].x; acc[j].y += f * v[u][j].y; acc[j].z += f * v[u][j].z; acc[j].w += f * v[u][j].w;
+                  }
+                }
+            }
+            const float inv = l_all > 0.f ? 1.f / l_all : 0.f;
+            __nv_bfloat16* dst = p.out + ((size_t)b * p.Hq + hq) * kD + c * 16;
+#pragma unroll
+            for (int j = 0; j < 4; j += 2) {
+              const __nv_bfloat162 w0 = __floats2bfloat162_rn(acc[j].x * inv, acc[j].y * inv);
+              const __nv_bfloat162 w1 = __floats2bfloat162_rn(acc[j].z * inv, acc[j].w * inv);
+              const __nv_bfloat162 w2 = __floats2bfloat162_rn(acc[j + 1].x * inv, acc[j + 1].y * inv);
+              const __nv_bfloat162 w3 = __floats2bfloat162_rn(acc[j + 1].z * inv, acc[j + 1].w * inv);
+              uint4 ov;
+              ov.x = *reinterpret_cast<const uint32_t*>(&w0); ov.y = *reinterpret_cast<const uint32_t*>(&w1);
+              ov.z = *reinterpret_cast<const uint32_t*>(&w2); ov.w = *reinterpret_cast<const uint32_t*>(&w3);
+              *reinterpret_cast<uint4*>(dst + j * 4) = ov;
+            }
+          } else
           for (uint32_t r = 0; r < p.group; ++r) {
             const uint32_t hq = g * p.group + r;
             const size_t slot0 = ((size_t)b * p.Hq + hq) * p.max_splits;
@@ -309,6 +389,7 @@ __global__ void __launch_bounds__(kAttnThreads, (NH == 1 ? 3 : 2)) paged_attn_ke
             *reinterpret_cast<uint2*>(p.out + ((size_t)b * p.Hq + hq) * kD + lane * 4) = ov;
           }
           if (lane == 0) *cnt = 0;
+          ATRACE(5);
         }
       }
     }
@@ -316,6 +397,7 @@ __global__ void __launch_bounds__(kAttnThreads, (NH == 1 ? 3 : 2)) paged_attn_ke
     if (lane == 0) nxt = n_warps + atomicAdd(p.ws + kWsHbmNext, 1u);
     id = __shfl_sync(0xFFFFFFFFu, nxt, 0);
   }
+  ATRACE(6);
   // the last warp out resets the counters for the next launch
   if (lane == 0) {
     __threadfence();
@@ -364,6 +446,12 @@ size_t attn_header_bytes(uint32_t B, uint32_t Hkv_upper) {
 }
 
 }  // namespace
+
+#ifdef BOOST_TRACE
+extern "C" int boost_debug_set_attn_trace(void* ptr) {
+  return boosth::check(cudaMemcpyToSymbol(g_attn_trace, &ptr, sizeof(ptr)));
+}
+#endif
 
 extern "C" int boost_kv_scatter(const void* src, uint32_t n_kv_heads, uint32_t n_pool_blocks,
                                 uint32_t D, const void* const* page_ptr, size_t n_pages, void* stream) {
