@@ -559,6 +559,70 @@ def run_kv_spill(args):
     print(json.dumps(line), flush=True)
 
 
+def run_gemv_sweep(args):
+    """Weight-product sweep over the Llama-3-8B matrix shapes, batch 1 .. 128 and three host
+    shares (0, the measured link share, 1/16): where tiering is free, where the link binds, and
+    where each of the three product kernels (CUDA cores, mma.sync, tcgen05) takes over.  Every
+    point: a CUDA graph of back-to-back launches over rotating copies of the weight that
+    together exceed twice the L2.  Prints one JSON document."""
+    import torch
+    from paper_2609_13592_b200 import binding as B
+    from paper_2609_13592_b200 import build as libbuild
+    from paper_2609_13592_b200.tiers import TieredWeight
+    libbuild.build_library()
+    B.lib()
+    dev = torch.device("cuda:0")
+    torch.cuda.set_device(dev)
+    hbm_peak, peak_src = load_peaks()
+    link = measure_stream(dev, 64, 1)
+    modulus = B.boost_modulus_from_bandwidths(hbm_peak, link)
+    shapes = {"qkv": (6144, 4096), "o": (4096, 4096), "gate_up": (28672, 4096), "down": (4096, 14336),
+              "lm_head": (128256, 4096)}
+    ratios = [("hbm_only", 0.0), (f"link_share_1/{modulus}", 1.0 / modulus), ("1/16", 1.0 / 16)]
+    batches = [1, 2, 4, 8, 16, 32, 64, 128]
+    points = []
+    g = torch.Generator(device=dev)
+    g.manual_seed(3)
+    for name, (n, k) in shapes.items():
+        n_copies = max(2, int(np.ceil(2 * 126e6 / (n * k * 2))))
+        for label, ratio in ratios:
+            ws = [TieredWeight((0.02 * torch.randn(n, k, generator=g, device=dev)).to(torch.bfloat16), ratio, device=dev)
+                  for _ in range(n_copies)]
+            host_pages, pages = ws[0].buf.n_host, ws[0].buf.n_pages
+            for mb in batches:
+                x = torch.randn(mb, k, generator=g, device=dev).to(torch.bfloat16)
+                y = torch.empty(mb, n, dtype=torch.bfloat16, device=dev)
+                for w in ws:
+                    w.gemv(x, y=y)
+                torch.cuda.synchronize(dev)
+                graph = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(graph):
+                    for w in ws:
+                        w.gemv(x, y=y)
+                graph.replay()
+                torch.cuda.synchronize(dev)
+                reps = 5 if host_pages > 8 else 10
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                for _ in range(reps):
+                    graph.replay()
+                e1.record()
+                torch.cuda.synchronize(dev)
+                us = e0.elapsed_time(e1) * 1e3 / (reps * n_copies)
+                nbytes = ws[0].layout["bytes"]
+                host_bytes = host_pages * B.PAGE_BYTES
+                t_min_us = 1e6 * max((nbytes - host_bytes) / (hbm_peak * 1e9), host_bytes / (link * 1e9))
+                points.append({"matrix": name, "N": n, "K": k, "batch": mb, "placement": label, "pages": pages,
+                               "host_pages": host_pages, "us": us, "gbs": nbytes / us / 1e3,
+                               "tier_bound_us": t_min_us, "frac_of_tier_bound": t_min_us / us,
+                               "status": ws[0].status_words()})
+                del graph
+            del ws
+            torch.cuda.empty_cache()
+    print(json.dumps({"workload": "weight_product_shape_batch_sweep", "hbm_peak_gbs": hbm_peak, "hbm_peak_source": peak_src,
+                      "host_link_gbs": link, "points": points}))
+
+
 def run_stream_sweep(args):
     """Configuration 3: tiered streaming-read sweep.  A bf16 buffer of 1 / 4 / 16 (/ 64) GiB is
     reduced by the stream-reduce kernel (full waves of 4 threadblocks per SM) with the host
@@ -626,10 +690,11 @@ def main():
     ap.add_argument("--ctx", type=int, default=2048)
     ap.add_argument("--layers", type=int, default=0, help="override the layer count (0 = 32)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--workload", default="decode", choices=["decode", "stream_sweep", "kv_spill"],
+    ap.add_argument("--workload", default="decode", choices=["decode", "stream_sweep", "kv_spill", "gemv_sweep"],
                     help="decode: the benchmark line; stream_sweep: the placement sweep of configuration 3; "
                          "kv_spill: configuration 5 (batch 128, one KV page in five on the host) with its "
-                         "HBM-only and prefetch-to-HBM comparison runs")
+                         "HBM-only and prefetch-to-HBM comparison runs; gemv_sweep: weight products over shapes, "
+                         "batch sizes and host shares")
     ap.add_argument("--sweep-gib", default="1,4,16")
     ap.add_argument("--sweep-seeds", type=int, default=5)
     args = ap.parse_args()
@@ -640,6 +705,9 @@ def main():
     if args.workload == "kv_spill":
         if rank == 0:
             run_kv_spill(args)
+    elif args.workload == "gemv_sweep":
+        if rank == 0:
+            run_gemv_sweep(args)
     elif args.workload == "stream_sweep":
         if rank == 0:
             run_stream_sweep(args)
