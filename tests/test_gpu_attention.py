@@ -158,3 +158,43 @@ def test_attention_argument_errors(dev):
             call(**kwargs)
         assert e.value.code == code, kwargs
     del args
+
+
+def test_attention_config5_shape_on_sampled_sequences(dev):
+    """Configuration 5's attention launch: batch 128, context lengths uniform in [2048, 4096]
+    (seed 5), 32 / 8 heads, a pool of 25088 blocks with host modulus 5 (one page in five of the
+    K and V tensors in host memory), blocks through the wave-aware pool.  The device computes
+    all 128 sequences; the oracle computes every head of 6 sampled sequences (the longest, the
+    shortest and four drawn with seed 7)."""
+    from paper_2609_13592_b200.tiers import TieredKVCache, aligned_workspace
+    n_seq, hq, hkv, d, n_blocks, modulus = 128, 32, 8, 128, 25088, 5
+    ctx = synth.ctx_lens_uniform(n_seq, 2048, 4096, seed=5)
+    assert int(((ctx + 15) // 16).sum()) <= n_blocks
+    pool, ref_pool = B.KVPool(n_blocks, hkv, modulus), okp.KVPool(n_blocks, hkv, modulus)
+    table = build_tables(pool, ref_pool, ctx.tolist(), churn=False)
+    k_bits = synth.normal_bf16((hkv, n_blocks, 16, d), 1.0, 50)
+    v_bits = synth.normal_bf16((hkv, n_blocks, 16, d), 1.0, 51)
+    q_bits = synth.normal_bf16((n_seq, hq, d), 1.0, 52)
+    cache = TieredKVCache(pool, hkv, n_blocks, d, dev)
+    assert cache.tier.tolist() == ref_pool.page_tiers()
+    assert int((cache.tier == 1).sum()) == cache.tier.size // 5
+    cache.load(bf16_tensor(k_bits, dev), bf16_tensor(v_bits, dev))
+    max_blocks = table.shape[1]
+    ws_bytes = B.boost_paged_attn_workspace_bytes(n_seq, hq, d, max_blocks)
+    ws_t, ws = aligned_workspace(ws_bytes, dev)
+    out = torch.full((n_seq, hq, d), float("nan"), dtype=torch.bfloat16, device=dev)
+    scale = 1.0 / math.sqrt(d)
+    B.boost_paged_attn_decode_tiered(bf16_tensor(q_bits, dev), cache.k.page_ptr, cache.v.page_ptr, cache.tier,
+                                     cache.n_pages, n_blocks, torch.from_numpy(table).to(dev), max_blocks,
+                                     torch.from_numpy(ctx.astype(np.int32)).to(dev), n_seq, hq, hkv, d, scale,
+                                     ws, ws_bytes, out)
+    torch.cuda.synchronize()
+    got = out.float().cpu().numpy()
+    assert np.isfinite(got).all()
+    off = ws - ws_t.data_ptr()
+    assert int(ws_t[off:off + 4].cpu().numpy().view(np.uint32)[0]) == 0     # status word
+    sel = sorted({int(np.argmax(ctx)), int(np.argmin(ctx)),
+                  *np.random.default_rng(7).choice(n_seq, size=4, replace=False).tolist()})
+    ref = ol.paged_attention_decode(q_bits[sel], k_bits, v_bits, table[sel], ctx[sel].tolist(), scale)
+    assert_close_to_oracle(got[sel], ref, "config 5 attention, sampled sequences")
+    pool.close()

@@ -214,3 +214,14 @@ def test_gemv_tcgen05_and_mma_sync_kernels_agree(dev, m_b):
         B.boost_gemv_set_tc_min_batch(33)
     for ratio in (0.0, 1 / 4):
         assert np.allclose(outs[("tcgen05", ratio)], outs[("mma_sync", ratio)], rtol=2e-5, atol=2e-6)
+
+
+@pytest.mark.parametrize("ratio", [0.0, 1 / 64])
+def test_gemv_full_size_batch128(dev, ratio):
+    """The gate/up matrix of the bench model (28672 x 4096) at batch 128, the launch of
+    configuration 5 (tcgen05 kernel): all outputs against the oracle; with all pages in HBM
+    (even partition) and with one page in 64 on the host (queue items, host pages first)."""
+    w, y, ref, _ = run_gemv(dev, 28672, 4096, 128, ratio, seed=21)
+    assert w.buf.n_host == (0 if ratio == 0 else w.buf.n_pages // 64)
+    assert_close_to_oracle(y, ref, f"28672 x 4096, batch 128, host ratio {ratio}", floor_rms=2e-3)
+    assert w.status_words() == [0]
