@@ -1,19 +1,20 @@
 // Tiered paged decode attention (split-KV) over the KV cache of a boost_kv_pool, and the
 // copies that move a logical [Hkv][N][16][D] cache into and out of its pages.
 //
-// Persistent grid of autonomous warps.  A work item is a KV-head chunk run: sequence b, KV
-// head g, a run of up to 32 consecutive blocks of the sequence (Sec. 3.3: threadblocks work
-// on KV head chunks); items of the highest-numbered heads - the ones linear placement puts
-// on the host tier - are handed out first.  Each warp takes whole items and streams their
-// KV blocks through its own two-stage ring in shared memory: per block two 4 KiB bulk
-// copies through the TMA unit (K chunk, V chunk) when the page is in HBM, a fan of 16-byte
-// cp.async loads when it is host memory.  Twelve such warps per SM keep about 150 KiB in
-// flight with no producer warp, no block-wide barrier and no cross-warp merge.  The
-// products are bf16 tensor-core MMAs with the 16 tokens of a block as the 16-row dimension
-// and the query heads of the group as the 8-wide dimension (S^T = K q^T, O^T += V^T P^T: a
-// group of four heads wastes half a tile instead of three quarters); P goes in as three
-// bf16 terms, transposed in registers with movmatrix; the online softmax is fp32.  The
-// last split of a (b, g) pair to finish combines all splits in split order.
+// Persistent grid.  A work item is a KV-head chunk run: sequence b, KV head g, a run of
+// consecutive blocks of the sequence (Sec. 3.3: threadblocks work on KV head chunks); items
+// of the highest-numbered heads - the ones linear placement puts on the host tier - are
+// handed out first.  The four warps of a threadblock take a quarter of the run each and
+// stream it on their own, through their own two-stage rings in shared memory: per block two
+// 4 KiB bulk copies through the TMA unit (K chunk, V chunk) when the page is in HBM, a fan of
+// 16-byte cp.async loads when it is host memory.  Twelve such warps per SM keep about
+// 150 KiB in flight with no producer warp and no barrier while they stream.  The products
+// are bf16 tensor-core MMAs with the 16 tokens of a block as the 16-row dimension and the
+// query heads of the group as the 8-wide dimension (S^T = K q^T, O^T += V^T P^T: a group of
+// four heads wastes half a tile instead of three quarters); P goes in as three bf16 terms,
+// transposed in registers with movmatrix; the online softmax is fp32.  The four quarters are
+// merged in shared memory; only a sequence longer than one item leaves partial results in
+// global memory, and the last of its items to finish combines them in run order.
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <math_constants.h>
@@ -30,13 +31,14 @@ constexpr uint32_t kD = 128;
 constexpr uint32_t kTok = BOOST_KV_BLOCK_TOKENS;         // 16
 constexpr uint32_t kChunkBytes = kTok * kD * 2;          // 4 KiB
 constexpr uint32_t kChunksPerPage = kPageBytes / kChunkBytes;
-constexpr uint32_t kMaxItemBlocks = 32;                  // KV blocks per work item: at most (one lane resolves one block)
+constexpr uint32_t kMaxItemBlocks = 64;                  // KV blocks per warp and work item: at most (one lane resolves two blocks)
 constexpr uint32_t kMinItemBlocks = 4;
 constexpr uint32_t kStageBytes = 2 * kChunkBytes;        // K chunk + V chunk
 constexpr uint32_t kAttnWarps = 4;                       // warps per threadblock
 constexpr uint32_t kAttnThreads = kAttnWarps * 32;
 constexpr uint32_t kWarpStages = 2;                      // ring depth of one warp
 constexpr uint32_t kMaxGroup = 16;
+constexpr uint32_t kParkStride = kD + 4;                 // floats per parked head: 128 outputs, m, l, padding
 
 #ifdef BOOST_TRACE
 // Debug build only: per-warp time stamps (global timer, ns), 8 slots per warp.
@@ -94,10 +96,13 @@ __global__ void __launch_bounds__(kAttnThreads, (NH == 1 ? 3 : 2)) paged_attn_ke
 
   // Fragment coordinates: rows gq, gq+8 (tokens for S^T, d for O^T), columns c0, c0+1 (heads).
   const uint32_t gq = lane >> 2, c0 = (lane & 3) * 2;
-  const uint32_t n_warps = gridDim.x * kAttnWarps;
   const uint32_t per_head = p.B * p.max_splits;
   uint32_t phase_mask = 0;                       // bit s = phase to wait for on stage s
-  uint32_t id = blockIdx.x * kAttnWarps + warp;  // first item by position, later ones from the counter
+  // A work item belongs to the threadblock: (sequence b, KV head g, a run of blocks); its four
+  // warps take a quarter of the run each and stream it on their own; their results meet in
+  // shared memory.  First item by position, later ones from the counter.
+  __shared__ uint32_t s_next, s_old;
+  uint32_t id = blockIdx.x;
 
   while (id < p.n_items) {
     const uint32_t g = p.Hkv - 1 - id / per_head;     // host-resident heads first
@@ -105,36 +110,47 @@ __global__ void __launch_bounds__(kAttnThreads, (NH == 1 ? 3 : 2)) paged_attn_ke
     const uint32_t split = id % p.max_splits;
     const uint32_t ctx = (uint32_t)max(p.ctx_lens[b], 0);
     const uint32_t n_blk = (ctx + kTok - 1) / kTok;
-    const uint32_t n_splits = n_blk ? (n_blk + p.item_blocks - 1) / p.item_blocks : 1;
+    const uint32_t cta_max = kAttnWarps * p.item_blocks;
+    const uint32_t n_splits = n_blk ? (n_blk + cta_max - 1) / cta_max : 1;
     if (split < n_splits) {
       // the sequence's blocks in n_splits runs of equal length (the last may be shorter by a
-      // few): a 129-block sequence is 5 runs of 26, not 4 of 32 and one of 1
+      // few), each run in four quarters
       const uint32_t run_len = n_blk ? (n_blk + n_splits - 1) / n_splits : 0;
-      const uint32_t blk0 = split * run_len;
-      const uint32_t nb = min(run_len, n_blk - min(n_blk, blk0));
-      // every lane resolves one block of the item: table entry, page, addresses
-      const uint8_t* ksrc = nullptr;
-      const uint8_t* vsrc = nullptr;
-      uint32_t host_bit = 0;
-      if (lane < nb) {
-        int32_t blk = p.block_table[(size_t)b * p.max_blocks + blk0 + lane];
-        if (blk < 0 || (uint32_t)blk >= p.n_pool_blocks) {   // bad table entry: record, read block 0
-          atomicOr(status, kErrBadIndex);
-          blk = 0;
+      const uint32_t cblk0 = split * run_len;
+      const uint32_t cnb = min(run_len, n_blk - min(n_blk, cblk0));
+      const uint32_t sub_len = (cnb + kAttnWarps - 1) / kAttnWarps;
+      const uint32_t blk0 = cblk0 + warp * sub_len;
+      const uint32_t nb = min(sub_len, cnb - min(cnb, warp * sub_len));
+      // every lane resolves up to two blocks of the warp's run (lane and lane + 32): table
+      // entry, page, addresses (K and V sit at the same offset of their tensors)
+      const uint8_t* ksrc[2] = {nullptr, nullptr};
+      size_t v_minus_k[2] = {0, 0};
+      uint32_t host_bits = 0;
+#pragma unroll
+      for (uint32_t h = 0; h < 2; ++h) {
+        if (lane + 32 * h < nb) {
+          int32_t blk = p.block_table[(size_t)b * p.max_blocks + blk0 + lane + 32 * h];
+          if (blk < 0 || (uint32_t)blk >= p.n_pool_blocks) {   // bad table entry: record, read block 0
+            atomicOr(status, kErrBadIndex);
+            blk = 0;
+          }
+          const uint32_t lin = g * p.n_pool_blocks + (uint32_t)blk;
+          const uint32_t page = lin / kChunksPerPage;
+          const size_t in_page = (size_t)(lin % kChunksPerPage) * kChunkBytes;
+          ksrc[h] = static_cast<const uint8_t*>(p.k_page_ptr[page]) + in_page;
+          v_minus_k[h] = (size_t)(static_cast<const uint8_t*>(p.v_page_ptr[page]) + in_page - ksrc[h]);
+          host_bits |= (page >= p.first_host_page ? 1u : 0u) << h;
         }
-        const uint32_t lin = g * p.n_pool_blocks + (uint32_t)blk;
-        const uint32_t page = lin / kChunksPerPage;
-        const size_t in_page = (size_t)(lin % kChunksPerPage) * kChunkBytes;
-        ksrc = static_cast<const uint8_t*>(p.k_page_ptr[page]) + in_page;
-        vsrc = static_cast<const uint8_t*>(p.v_page_ptr[page]) + in_page;
-        host_bit = page >= p.first_host_page ? 1u : 0u;
       }
-      // request block i of the item into stage i % kWarpStages
+      // request block i of the run into stage i % kWarpStages
       auto request = [&](uint32_t i) {
         const uint32_t st = i % kWarpStages;
-        const uint8_t* ks = reinterpret_cast<const uint8_t*>(__shfl_sync(0xFFFFFFFFu, (unsigned long long)ksrc, i));
-        const uint8_t* vs = reinterpret_cast<const uint8_t*>(__shfl_sync(0xFFFFFFFFu, (unsigned long long)vsrc, i));
-        const bool from_host = __shfl_sync(0xFFFFFFFFu, host_bit, i) != 0;
+        const uint32_t h = i >> 5, src_lane = i & 31u;
+        const unsigned long long k_all = (unsigned long long)(h ? ksrc[1] : ksrc[0]);
+        const unsigned long long d_all = (unsigned long long)(h ? v_minus_k[1] : v_minus_k[0]);
+        const uint8_t* ks = reinterpret_cast<const uint8_t*>(__shfl_sync(0xFFFFFFFFu, k_all, src_lane));
+        const uint8_t* vs = ks + __shfl_sync(0xFFFFFFFFu, d_all, src_lane);
+        const bool from_host = ((__shfl_sync(0xFFFFFFFFu, host_bits, src_lane) >> h) & 1u) != 0;
         uint8_t* kdst = ring + (size_t)st * kStageBytes;
         uint8_t* vdst = kdst + kChunkBytes;
         if (lane == 0) {
@@ -274,111 +290,105 @@ __global__ void __launch_bounds__(kAttnThreads, (NH == 1 ? 3 : 2)) paged_attn_ke
       }
 
       ATRACE(3);
-      // ---- end of the item: this warp holds the whole chunk run
-      const bool single = (n_splits == 1);
+      // ---- end of the run: the four warps' (m, l, O) meet in shared memory.  Each warp parks
+      // its result in its own (now idle) ring space: per head 128 outputs, then m and l.
+      float* park = reinterpret_cast<float*>(ring);
 #pragma unroll
       for (int nh = 0; nh < NH; ++nh)
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
           const uint32_t head = nh * 8 + c0 + h;
           if (head >= p.group) continue;
-          const uint32_t hq = g * p.group + head;
-          if (single) {
-            const float inv = l_run[nh][h] > 0.f ? 1.f / l_run[nh][h] : 0.f;
-            __nv_bfloat16* dst = p.out + ((size_t)b * p.Hq + hq) * kD;
+          float* dst = park + head * kParkStride;
 #pragma unroll
-            for (int j = 0; j < 8; ++j) {
-              dst[j * 16 + gq] = __float2bfloat16_rn(o[nh][j][h] * inv);
-              dst[j * 16 + gq + 8] = __float2bfloat16_rn(o[nh][j][2 + h] * inv);
-            }
-          } else {
-            const size_t slot = ((size_t)b * p.Hq + hq) * p.max_splits + split;
-            float* dst = p.part_o + slot * kD;
-#pragma unroll
-            for (int j = 0; j < 8; ++j) {
-              __stcg(dst + j * 16 + gq, o[nh][j][h]);
-              __stcg(dst + j * 16 + gq + 8, o[nh][j][2 + h]);
-            }
-            if (gq == 0) { __stcg(p.part_ml + slot * 2, m_run[nh][h]); __stcg(p.part_ml + slot * 2 + 1, l_run[nh][h]); }
+          for (int j = 0; j < 8; ++j) {
+            dst[j * 16 + gq] = o[nh][j][h];
+            dst[j * 16 + gq + 8] = o[nh][j][2 + h];
           }
+          if (gq == 0) { dst[kD] = m_run[nh][h]; dst[kD + 1] = l_run[nh][h]; }
         }
+      __syncthreads();
+      // warp w merges heads w, w + 4, ...: lane = four consecutive outputs
+      const bool single = (n_splits == 1);
+      for (uint32_t r = warp; r < p.group; r += kAttnWarps) {
+        const uint32_t hq = g * p.group + r;
+        float mw[kAttnWarps], lw[kAttnWarps];
+        float m_all = -CUDART_INF_F;
+#pragma unroll
+        for (uint32_t w = 0; w < kAttnWarps; ++w) {
+          const float* src = reinterpret_cast<const float*>(smem + (size_t)w * kWarpStages * kStageBytes) + r * kParkStride;
+          mw[w] = src[kD]; lw[w] = src[kD + 1];
+          m_all = fmaxf(m_all, mw[w]);
+        }
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        float l_all = 0.f;
+#pragma unroll
+        for (uint32_t w = 0; w < kAttnWarps; ++w) {
+          if (mw[w] == -CUDART_INF_F) continue;   // a quarter without blocks
+          const float f = exp2f(mw[w] - m_all);
+          const float4 v = *(reinterpret_cast<const float4*>(reinterpret_cast<const float*>(smem + (size_t)w * kWarpStages * kStageBytes) + r * kParkStride) + lane);
+          acc.x += f * v.x; acc.y += f * v.y; acc.z += f * v.z; acc.w += f * v.w;
+          l_all += f * lw[w];
+        }
+        if (single) {
+          const float inv = l_all > 0.f ? 1.f / l_all : 0.f;
+          const __nv_bfloat162 lo = __floats2bfloat162_rn(acc.x * inv, acc.y * inv);
+          const __nv_bfloat162 hi = __floats2bfloat162_rn(acc.z * inv, acc.w * inv);
+          uint2 ov;
+          ov.x = *reinterpret_cast<const uint32_t*>(&lo);
+          ov.y = *reinterpret_cast<const uint32_t*>(&hi);
+          *reinterpret_cast<uint2*>(p.out + ((size_t)b * p.Hq + hq) * kD + lane * 4) = ov;
+        } else {
+          const size_t slot = ((size_t)b * p.Hq + hq) * p.max_splits + split;
+          __stcg(reinterpret_cast<float4*>(p.part_o + slot * kD) + lane, acc);
+          if (lane == 0) { __stcg(p.part_ml + slot * 2, m_all); __stcg(p.part_ml + slot * 2 + 1, l_all); }
+        }
+      }
       if (!single) {
-        // the last split of (b, g) to arrive combines all splits, in split order
+        // the last run of (b, g) to arrive combines all runs, in run order
         uint32_t* cnt = p.ws + kWsHeaderWords + b * p.Hkv + g;
-        __syncwarp();
-        uint32_t old = 0;
-        if (lane == 0) {
-          __threadfence();   // cumulative: publishes the partials of the whole warp
-          old = atomicAdd(cnt, 1u);
+        __syncthreads();
+        if (tid == 0) {
+          __threadfence();   // cumulative: publishes the partial results of the whole threadblock
+          s_old = atomicAdd(cnt, 1u);
         }
-        old = __shfl_sync(0xFFFFFFFFu, old, 0);
+        __syncthreads();
         ATRACE(4);
-        if (old == n_splits - 1) {
+        if (s_old == n_splits - 1) {
           __threadfence();
-          if (p.group == 4) {
-            // four heads side by side: 8 lanes per head, 16 outputs per lane, the loads of two
-            // splits (8 x 16 bytes per lane) in flight at a time
-            const uint32_t r = lane >> 3, c = lane & 7;
+          for (uint32_t r = warp; r < p.group; r += kAttnWarps) {
             const uint32_t hq = g * p.group + r;
             const size_t slot0 = ((size_t)b * p.Hq + hq) * p.max_splits;
+            // lane i looks after the (m, l) pair of runs i, i + 32, ...; the outputs are summed
+            // in run order, eight loads in flight at a time
             float m_all = -CUDART_INF_F;
-            for (uint32_t sp = c; sp < n_splits; sp += 8) m_all = fmaxf(m_all, __ldcg(p.part_ml + (slot0 + sp) * 2));
-            m_all = fmaxf(m_all, __shfl_xor_sync(0xFFFFFFFFu, m_all, 1));
-            m_all = fmaxf(m_all, __shfl_xor_sync(0xFFFFFFFFu, m_all, 2));
-            m_all = fmaxf(m_all, __shfl_xor_sync(0xFFFFFFFFu, m_all, 4));
-            float4 acc[4];
+            for (uint32_t sp = lane; sp < n_splits; sp += 32) m_all = fmaxf(m_all, __ldcg(p.part_ml + (slot0 + sp) * 2));
 #pragma unroll
-            for (int j = 0; j < 4; ++j) acc[j] = make_float4(0.f, 0.f, 0.f, 0.f);
-            float l_all = 0.f;
-            for (uint32_t sp0 = 0; sp0 < n_splits; sp0 += 2) {
-              float4 v[2][4];
-              float2 ml[2];
-#pragma unroll
-              for (uint32_t u = 0; u < 2; ++u)
-                if (sp0 + u < n_splits) {
-                  ml[u] = __ldcg(reinterpret_cast<const float2*>(p.part_ml + (slot0 + sp0 + u) * 2));
-#pragma unroll
-                  for (int j = 0; j < 4; ++j)
-                    v[u][j] = __ldcg(reinterpret_cast<const float4*>(p.part_o + (slot0 + sp0 + u) * kD) + c * 4 + j);
-                }
-#pragma unroll
-              for (uint32_t u = 0; u < 2; ++u)
-                if (sp0 + u < n_splits) {
-                  const float f = (ml[u].x == -CUDART_INF_F) ? 0.f : exp2f(ml[u].x - m_all);
-                  l_all += f * ml[u].y;
-#pragma unroll
-                  for (int j = 0; j < 4; ++j) {
-                    acc[j].x += f * v[u][j].x; acc[j].y += f * v[u][j].y; acc[j].z += f * v[u][j].z; acc[j].w += f * v[u][j].w;
-                  }
-                }
-            }
-            const float inv = l_all > 0.f ? 1.f / l_all : 0.f;
-            __nv_bfloat16* dst = p.out + ((size_t)b * p.Hq + hq) * kD + c * 16;
-#pragma unroll
-            for (int j = 0; j < 4; j += 2) {
-              const __nv_bfloat162 w0 = __floats2bfloat162_rn(acc[j].x * inv, acc[j].y * inv);
-              const __nv_bfloat162 w1 = __floats2bfloat162_rn(acc[j].z * inv, acc[j].w * inv);
-              const __nv_bfloat162 w2 = __floats2bfloat162_rn(acc[j + 1].x * inv, acc[j + 1].y * inv);
-              const __nv_bfloat162 w3 = __floats2bfloat162_rn(acc[j + 1].z * inv, acc[j + 1].w * inv);
-              uint4 ov;
-              ov.x = *reinterpret_cast<const uint32_t*>(&w0); ov.y = *reinterpret_cast<const uint32_t*>(&w1);
-              ov.z = *reinterpret_cast<const uint32_t*>(&w2); ov.w = *reinterpret_cast<const uint32_t*>(&w3);
-              *reinterpret_cast<uint4*>(dst + j * 4) = ov;
-            }
-          } else
-          for (uint32_t r = 0; r < p.group; ++r) {
-            const uint32_t hq = g * p.group + r;
-            const size_t slot0 = ((size_t)b * p.Hq + hq) * p.max_splits;
-            float m_all = -CUDART_INF_F;
-            for (uint32_t sp = 0; sp < n_splits; ++sp) m_all = fmaxf(m_all, __ldcg(p.part_ml + (slot0 + sp) * 2));
+            for (int sh = 16; sh >= 1; sh >>= 1) m_all = fmaxf(m_all, __shfl_xor_sync(0xFFFFFFFFu, m_all, sh));
             float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
             float l_all = 0.f;
-            for (uint32_t sp = 0; sp < n_splits; ++sp) {
-              const float ms = __ldcg(p.part_ml + (slot0 + sp) * 2);
-              const float f = (ms == -CUDART_INF_F) ? 0.f : exp2f(ms - m_all);
-              const float4 v = __ldcg(reinterpret_cast<const float4*>(p.part_o + (slot0 + sp) * kD) + lane);
-              acc.x += f * v.x; acc.y += f * v.y; acc.z += f * v.z; acc.w += f * v.w;
-              l_all += f * __ldcg(p.part_ml + (slot0 + sp) * 2 + 1);
+            for (uint32_t base = 0; base < n_splits; base += 32) {
+              float f_mine = 0.f, lf = 0.f;
+              if (base + lane < n_splits) {
+                const float2 ml = __ldcg(reinterpret_cast<const float2*>(p.part_ml + (slot0 + base + lane) * 2));
+                f_mine = (ml.x == -CUDART_INF_F) ? 0.f : exp2f(ml.x - m_all);
+                lf = f_mine * ml.y;
+              }
+#pragma unroll
+              for (int sh = 16; sh >= 1; sh >>= 1) lf += __shfl_xor_sync(0xFFFFFFFFu, lf, sh);
+              l_all += lf;
+              const uint32_t n_here = min(32u, n_splits - base);
+              for (uint32_t j0 = 0; j0 < n_here; j0 += 8) {
+                float4 v[8];
+#pragma unroll
+                for (uint32_t u = 0; u < 8; ++u)
+                  if (j0 + u < n_here) v[u] = __ldcg(reinterpret_cast<const float4*>(p.part_o + (slot0 + base + j0 + u) * kD) + lane);
+#pragma unroll
+                for (uint32_t u = 0; u < 8; ++u) {
+                  const float f = __shfl_sync(0xFFFFFFFFu, f_mine, (j0 + u) & 31u);
+                  if (j0 + u < n_here) { acc.x += f * v[u].x; acc.y += f * v[u].y; acc.z += f * v[u].z; acc.w += f * v[u].w; }
+                }
+              }
             }
             const float inv = l_all > 0.f ? 1.f / l_all : 0.f;
             const __nv_bfloat162 lo = __floats2bfloat162_rn(acc.x * inv, acc.y * inv);
@@ -388,21 +398,28 @@ __global__ void __launch_bounds__(kAttnThreads, (NH == 1 ? 3 : 2)) paged_attn_ke
             ov.y = *reinterpret_cast<const uint32_t*>(&hi);
             *reinterpret_cast<uint2*>(p.out + ((size_t)b * p.Hq + hq) * kD + lane * 4) = ov;
           }
-          if (lane == 0) *cnt = 0;
+          if (tid == 0) *cnt = 0;
           ATRACE(5);
         }
       }
+      // the ring is written by bulk copies again: order the parked values' reads and writes before them
+      __syncthreads();
+      fence_proxy_async_smem();
+    } else if (!waited) {
+      pdl_wait();   // keep every thread's first pass through the dependency wait
+      waited = true;
     }
-    uint32_t nxt = 0;
-    if (lane == 0) nxt = n_warps + atomicAdd(p.ws + kWsHbmNext, 1u);
-    id = __shfl_sync(0xFFFFFFFFu, nxt, 0);
+    if (tid == 0) s_next = gridDim.x + atomicAdd(p.ws + kWsHbmNext, 1u);
+    __syncthreads();
+    id = s_next;
+    __syncthreads();
   }
   ATRACE(6);
-  // the last warp out resets the counters for the next launch
-  if (lane == 0) {
+  // the last threadblock out resets the counters for the next launch
+  if (tid == 0) {
     __threadfence();
     const uint32_t d = atomicAdd(p.ws + kWsDone, 1u);
-    if (d == n_warps - 1) { p.ws[kWsHbmNext] = 0; p.ws[kWsDone] = 0; __threadfence(); }
+    if (d == gridDim.x - 1) { p.ws[kWsHbmNext] = 0; p.ws[kWsDone] = 0; __threadfence(); }
   }
 }
 
@@ -511,18 +528,19 @@ extern "C" int boost_paged_attn_decode_tiered(const void* q, const void* const* 
   if (sms <= 0) return BOOST_ERR_CUDA;
   const uint32_t ctas_per_sm = p.group <= 8 ? 3 : 2;
   const uint32_t n_warps = (uint32_t)sms * ctas_per_sm * kAttnWarps;
-  // Item length: every item costs a table look-up, a query load and a partial result, so long
-  // items are better as long as enough warps have work to keep HBM busy (measured on B200:
+  // Run length: an item (four warps, a quarter of the run each) costs a table look-up, a query
+  // load and, when a sequence needs several items, a partial result in global memory, so long
+  // runs are better as long as enough warps have work to keep HBM busy (measured on B200:
   // about a thousand warps with 16 KiB in flight each saturate it).  Taking the sequences as
-  // max_blocks long, use the longest run (4..32 blocks) that still gives 55 % of the warps an
-  // item.
+  // max_blocks long, use the longest quarter (4..64 blocks) that still gives 55 % of the
+  // warps work.
   uint32_t best_len = kMinItemBlocks;
   for (uint32_t len = kMaxItemBlocks; len >= kMinItemBlocks; --len) {
-    const uint64_t items = (uint64_t)Hkv * B * ((max_blocks + len - 1) / len);
-    if (items * 100 >= (uint64_t)n_warps * 55) { best_len = len; break; }
+    const uint64_t items = (uint64_t)Hkv * B * ((max_blocks + kAttnWarps * len - 1) / (kAttnWarps * len));
+    if (items * kAttnWarps * 100 >= (uint64_t)n_warps * 55) { best_len = len; break; }
   }
   p.item_blocks = best_len;
-  p.max_splits = (max_blocks + best_len - 1) / best_len;
+  p.max_splits = (max_blocks + kAttnWarps * best_len - 1) / (kAttnWarps * best_len);
   const uint64_t n_items = (uint64_t)Hkv * B * p.max_splits;
   if (n_items > 0x7FFFFFFFull) return BOOST_ERR_INVALID;
   p.n_items = (uint32_t)n_items;
@@ -542,7 +560,7 @@ extern "C" int boost_paged_attn_decode_tiered(const void* q, const void* const* 
     configured = true;
   }
   uint32_t grid = (uint32_t)sms * ctas_per_sm;
-  if (grid * kAttnWarps > p.n_items) grid = (p.n_items + kAttnWarps - 1) / kAttnWarps;
+  if (grid > p.n_items) grid = p.n_items;
   if (p.group <= 8)
     return boosth::launch_chained(paged_attn_kernel<1>, dim3(grid), dim3(kAttnThreads), smem, (cudaStream_t)stream, p);
   return boosth::launch_chained(paged_attn_kernel<2>, dim3(grid), dim3(kAttnThreads), smem, (cudaStream_t)stream, p);
