@@ -132,7 +132,7 @@ def dump_cache(dev, dec, li, name):
     return bits_of(t)
 
 
-@pytest.mark.parametrize("n_seq,kv_modulus,weight_ratio", [(3, 4, 0.5), (1, 0, 0.0), (20, 2, 0.25)])
+@pytest.mark.parametrize("n_seq,kv_modulus,weight_ratio", [(3, 4, 0.5), (1, 0, 0.0), (20, 2, 0.25), (40, 4, 0.25)])
 def test_decode_steps_match_oracle(dev, n_seq, kv_modulus, weight_ratio):
     from tests.helpers import chain_error
     cfg = dict(synth.TINY_LLAMA)
