@@ -31,7 +31,7 @@ constexpr uint32_t kMaxStages = 16;
 constexpr uint32_t kSmemBudget = 224u * 1024u;
 constexpr uint32_t kXRowStride = 144;  // 128 data bytes + 16: 8 consecutive rows hit distinct banks
 
-enum : uint32_t { kFlagFirst = 1u, kFlagLast = 2u, kFlagStop = 4u, kFlagPhaseEnd = 8u };
+enum : uint32_t { kFlagFirst = 1u, kFlagLast = 2u, kFlagStop = 4u, kFlagPhaseEnd = 8u, kFlagPair = 16u, kFlagSecond = 32u, kFlagHost = 64u };
 constexpr uint32_t kMaxPhases = 4;
 enum : uint32_t { kEpiPlain = 0u, kEpiSwiglu = 1u, kEpiRope = 2u };
 
@@ -89,6 +89,7 @@ struct GemvParams {
   // touch it.  Every SM carries the same number of bytes, which is what HBM-bound work needs.
   uint32_t even_part, total_blocks;
   uint32_t max_seg;       // partial-sum slots per row tile (= splits with the queues)
+  uint32_t tiles_per_unit;   // tcgen05 kernel, even partition: 1, or 2 = adjacent row tiles share an activation tile
 };
 
 // First / last threadblock of the even partition that holds a block of row tile `t`.
@@ -705,12 +706,13 @@ constexpr uint32_t kTcEpiThreads = kTcEpiWarps * 32;
 constexpr uint32_t kTcXWarps = 4;   // activation producer warps: rows m with (m / 4) % 4 == their index
 constexpr uint32_t kTcThreads = kTcEpiThreads + 64 + 32 * kTcXWarps;
 
-__host__ __device__ constexpr uint32_t tc_stage_bytes(uint32_t npad) { return kBlockBytes + npad * 128u; }
+// a stage: two weight blocks (the same 64 columns of two adjacent row tiles) and one activation tile
+__host__ __device__ constexpr uint32_t tc_stage_bytes(uint32_t npad) { return 2 * kBlockBytes + npad * 128u; }
 
 template <uint32_t NPAD>
 __global__ void __launch_bounds__(kTcThreads, 1) gemv_tc_kernel(const __grid_constant__ ChainParams cp) {
   constexpr uint32_t kStageBytes = tc_stage_bytes(NPAD);
-  constexpr uint32_t kTmemCols = 2 * NPAD < 32 ? 32 : 2 * NPAD;
+  constexpr uint32_t kTmemCols = 4 * NPAD < 32 ? 32 : 4 * NPAD;   // two accumulators (a pair of row tiles), double-buffered
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   __shared__ uint64_t full_bar[kMaxStages];
@@ -774,15 +776,22 @@ __global__ void __launch_bounds__(kTcThreads, 1) gemv_tc_kernel(const __grid_con
       }
       // one block: the weight warp copies it, the activation warp stages x[:, 64 kb .. 64 kb + 64)
       // as NPAD rows of 128 bytes in the 128-byte swizzle (rows >= M_b are zero)
-      auto produce = [&](const uint8_t* src, bool from_host, uint32_t row_tile, uint32_t seg, uint32_t flags, uint32_t kb) {
+      // one stage: the weight warp copies the weight block (two blocks in pair mode), the
+      // activation warps stage x[:, 64 kb .. 64 kb + 64) as NPAD rows of 128 bytes in the
+      // 128-byte swizzle (rows >= M_b are zero)
+      auto produce = [&](const uint8_t* src, const uint8_t* src1, bool from_host, uint32_t row_tile, uint32_t seg,
+                         uint32_t flags, uint32_t kb) {
         if (s_abort) return;
         if (leader) {
           uint8_t* wdst = smem + (size_t)stage * kStageBytes;
           if (lane == 0) {
             if (!mbar_wait(&empty_bar[stage], phase ^ 1u, status)) s_abort = 1;
-            meta[stage] = make_uint4(row_tile, seg, flags, ph);
-            mbar_arrive_expect_tx(&full_bar[stage], from_host ? 0u : kBlockBytes);
-            if (!from_host) bulk_copy_g2s(wdst, src, kBlockBytes, &full_bar[stage]);
+            meta[stage] = make_uint4(row_tile, seg, flags | (from_host ? kFlagHost : 0u), ph);
+            mbar_arrive_expect_tx(&full_bar[stage], from_host ? 0u : ((flags & kFlagSecond) ? 2 * kBlockBytes : kBlockBytes));
+            if (!from_host) {
+              bulk_copy_g2s(wdst, src, kBlockBytes, &full_bar[stage]);
+              if (flags & kFlagSecond) bulk_copy_g2s(wdst + kBlockBytes, src1, kBlockBytes, &full_bar[stage]);
+            }
           }
           __syncwarp();
           if (from_host) {
@@ -793,7 +802,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) gemv_tc_kernel(const __grid_con
         } else {
           if (!mbar_wait(&empty_bar[stage], phase ^ 1u, status)) s_abort = 1;
           const uint32_t c = lane & 7, m0 = (lane >> 3) + 4 * xw;
-          uint8_t* xbase = smem + (size_t)stage * kStageBytes + kBlockBytes;
+          uint8_t* xbase = smem + (size_t)stage * kStageBytes + 2 * kBlockBytes;
           const uint32_t k = kb * kBlockK + c * 8;
           const bool k_ok = k < p.K;
 #pragma unroll 4
@@ -806,25 +815,37 @@ __global__ void __launch_bounds__(kTcThreads, 1) gemv_tc_kernel(const __grid_con
         if (++stage == n_stages) { stage = 0; phase ^= 1u; }
       };
       if (p.even_part) {
-        const uint32_t G = p.active_ctas, T = p.total_blocks;
+        // The unit is (row tile, kb) or, for long matrices, (pair of adjacent row tiles, kb): both
+        // weight blocks then meet the same activation tile, which halves the activation traffic
+        // from L2 and its share of the ring (short matrices keep single tiles: pairs would double
+        // the partial sums per tile).  Threadblock c of G takes units [c T2 / G, (c + 1) T2 / G).
+        const uint32_t G = p.active_ctas, tpu = p.tiles_per_unit;
+        const uint32_t n_pairs = (p.n_row_tiles + tpu - 1) / tpu, T2 = n_pairs * p.k_blocks;
         if (blockIdx.x < G) {
-          const uint32_t b0 = (uint32_t)((uint64_t)blockIdx.x * T / G), b1 = (uint32_t)((uint64_t)(blockIdx.x + 1) * T / G);
-          uint32_t row_tile = b0 / p.k_blocks, kb = b0 % p.k_blocks;
-          uint32_t seg = blockIdx.x - part_owner((uint64_t)row_tile * p.k_blocks, G, T);
-          const uint8_t* page_base = nullptr;   // looked up once per page (an L2 round trip)
-          uint32_t page_of_base = 0xFFFFFFFFu;
-          for (uint32_t b = b0; b < b1; ++b) {
-            const bool seg_first = (b == b0) || kb == 0, seg_last = (b + 1 == b1) || (kb + 1 == p.k_blocks);
-            const uint8_t* src = nullptr;
+          const uint32_t u0 = (uint32_t)((uint64_t)blockIdx.x * T2 / G), u1 = (uint32_t)((uint64_t)(blockIdx.x + 1) * T2 / G);
+          uint32_t pair = u0 / p.k_blocks, kb = u0 % p.k_blocks;
+          uint32_t seg = blockIdx.x - part_owner((uint64_t)pair * p.k_blocks, G, T2);
+          const uint8_t* page_base[2] = {nullptr, nullptr};   // looked up once per page (an L2 round trip)
+          uint32_t page_of_base[2] = {0xFFFFFFFFu, 0xFFFFFFFFu};
+          for (uint32_t u = u0; u < u1; ++u) {
+            const bool seg_first = (u == u0) || kb == 0, seg_last = (u + 1 == u1) || (kb + 1 == p.k_blocks);
+            const bool second = tpu == 2 && 2 * pair + 1 < p.n_row_tiles;
+            const uint8_t* src[2] = {nullptr, nullptr};
             if (leader && lane == 0) {
-              if (b / kBlocksPerPage != page_of_base) {
-                page_of_base = b / kBlocksPerPage;
-                page_base = static_cast<const uint8_t*>(p.w_page_ptr[page_of_base]);
+#pragma unroll
+              for (uint32_t h = 0; h < 2; ++h) {
+                if (h == 1 && !second) break;
+                const uint32_t b = (tpu * pair + h) * p.k_blocks + kb;
+                if (b / kBlocksPerPage != page_of_base[h]) {
+                  page_of_base[h] = b / kBlocksPerPage;
+                  page_base[h] = static_cast<const uint8_t*>(p.w_page_ptr[page_of_base[h]]);
+                }
+                src[h] = page_base[h] + (size_t)(b % kBlocksPerPage) * kBlockBytes;
               }
-              src = page_base + (size_t)(b % kBlocksPerPage) * kBlockBytes;
             }
-            produce(src, false, row_tile, seg, (seg_first ? kFlagFirst : 0u) | (seg_last ? kFlagLast : 0u), kb);
-            if (++kb == p.k_blocks) { kb = 0; ++row_tile; seg = 0; }
+            produce(src[0], src[1], false, tpu * pair, seg,
+                    kFlagPair | (second ? kFlagSecond : 0u) | (seg_first ? kFlagFirst : 0u) | (seg_last ? kFlagLast : 0u), kb);
+            if (++kb == p.k_blocks) { kb = 0; ++pair; seg = 0; }
           }
         }
       } else {
@@ -858,7 +879,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) gemv_tc_kernel(const __grid_con
           const bool from_host = qi < n_host_items;
           const uint8_t* src = static_cast<const uint8_t*>(p.w_page_ptr[page]) + (size_t)(first_blk % kBlocksPerPage) * kBlockBytes;
           for (uint32_t j = 0; j < p.run; ++j, src += kBlockBytes)
-            produce(src, from_host, row_tile, kb0 / p.run, (j == 0 ? kFlagFirst : 0u) | (j + 1 == p.run ? kFlagLast : 0u), kb0 + j);
+            produce(src, nullptr, from_host, row_tile, kb0 / p.run, (j == 0 ? kFlagFirst : 0u) | (j + 1 == p.run ? kFlagLast : 0u), kb0 + j);
         }
       }
       // a stage without data tells the MMA warp that the phase (or the launch) is over
@@ -906,11 +927,13 @@ __global__ void __launch_bounds__(kTcThreads, 1) gemv_tc_kernel(const __grid_con
         fence_proxy_async_smem();   // x (and host-tier weight blocks) were written through the load/store path
         tc_fence_after_sync();
         const uint32_t wbase = smem_u32(smem + (size_t)stage * kStageBytes);
-        const uint32_t xbase = wbase + kBlockBytes;
+        const uint32_t xbase = wbase + 2 * kBlockBytes;
+        const uint32_t d0 = tmem_base + buf * 2 * NPAD;   // accumulator of the first row tile; the second follows it
 #pragma unroll
         for (uint32_t ks = 0; ks < kBlockK / 16; ++ks) {
-          umma_bf16(tmem_base + buf * NPAD, umma_desc_k_sw128(wbase + ks * 32), umma_desc_k_sw128(xbase + ks * 32), idesc,
-                    accumulate);
+          const uint64_t xdesc = umma_desc_k_sw128(xbase + ks * 32);
+          umma_bf16(d0, umma_desc_k_sw128(wbase + ks * 32), xdesc, idesc, accumulate);
+          if (mt.z & kFlagSecond) umma_bf16(d0 + NPAD, umma_desc_k_sw128(wbase + kBlockBytes + ks * 32), xdesc, idesc, accumulate);
           accumulate = 1;
         }
         umma_commit(&empty_bar[stage]);   // the stage is free once these MMAs have read it
@@ -967,53 +990,62 @@ __global__ void __launch_bounds__(kTcThreads, 1) gemv_tc_kernel(const __grid_con
     }
     tc_fence_after_sync();
     const GemvParams& p = cp.ph[mt.w];
-    const uint32_t row_tile = mt.x, split = mt.y;
+    const uint32_t split = mt.y;
+    const uint32_t n_tiles = (mt.z & kFlagSecond) ? 2u : 1u;   // row tiles in this accumulator
     uint32_t n_seg = p.splits;
     if (p.even_part) {
-      const uint64_t t0 = (uint64_t)row_tile * p.k_blocks;
-      n_seg = part_owner(t0 + p.k_blocks - 1, p.active_ctas, p.total_blocks) - part_owner(t0, p.active_ctas, p.total_blocks) + 1;
+      const uint32_t tpu = p.tiles_per_unit;
+      const uint32_t T2 = ((p.n_row_tiles + tpu - 1) / tpu) * p.k_blocks;
+      const uint64_t u0 = (uint64_t)(mt.x / tpu) * p.k_blocks;
+      n_seg = part_owner(u0 + p.k_blocks - 1, p.active_ctas, T2) - part_owner(u0, p.active_ctas, T2) + 1;
     }
     const bool direct = (n_seg == 1) && p.epi == kEpiPlain && !p.ssq_in && !p.ssq_out;
-    float* part = p.partials + ((size_t)row_tile * p.max_seg + split) * NPAD * kBlockRows;
     const uint32_t quarter = warp & 3u, half = warp >> 2;
     const uint32_t nl = quarter * 32 + lane;                                 // weight row of this thread = its TMEM lane
-    const uint32_t taddr = tmem_base + ((quarter * 32u) << 16) + buf * NPAD;
     // warps 0-3 read the first half of the columns, warps 4-7 the second (16 columns: the first group reads all)
     constexpr uint32_t kColsPerGroup = NPAD >= 32 ? NPAD / 2 : NPAD;
     const uint32_t c_begin = half * kColsPerGroup;
     const uint32_t c_end = (NPAD >= 32 || half == 0) ? c_begin + kColsPerGroup : c_begin;
-    for (uint32_t c0 = c_begin; c0 < c_end; c0 += 16) {
-      float v[16];
-      tmem_ld16(taddr + c0, v);
+    for (uint32_t ti = 0; ti < n_tiles; ++ti) {
+      const uint32_t row_tile = mt.x + ti;
+      float* part = p.partials + ((size_t)row_tile * p.max_seg + split) * NPAD * kBlockRows;
+      const uint32_t taddr = tmem_base + ((quarter * 32u) << 16) + buf * 2 * NPAD + ti * NPAD;
+      for (uint32_t c0 = c_begin; c0 < c_end; c0 += 16) {
+        float v[16];
+        tmem_ld16(taddr + c0, v);
 #pragma unroll
-      for (uint32_t j = 0; j < 16; ++j) {
-        const uint32_t m = c0 + j;                                           // batch row = accumulator column
-        if (direct) {
-          const uint32_t n = row_tile * kBlockRows + nl;
-          if (m < p.M_b && n < p.N) store_out(p, m, n, v[j]);
-        } else {
-          __stcg(part + m * kBlockRows + nl, v[j]);
+        for (uint32_t j = 0; j < 16; ++j) {
+          const uint32_t m = c0 + j;                                         // batch row = accumulator column
+          if (direct) {
+            const uint32_t n = row_tile * kBlockRows + nl;
+            if (m < p.M_b && n < p.N) store_out(p, m, n, v[j]);
+          } else {
+            __stcg(part + m * kBlockRows + nl, v[j]);
+          }
         }
       }
     }
-    // the accumulator may be overwritten
+    // the accumulators may be overwritten
     tc_fence_before_sync();
     __syncwarp();
     if (lane == 0) mbar_arrive(&acc_empty[buf]);
     if (++buf == 2) { buf = 0; buf_phase ^= 1u; }
     if (!direct) {
-      named_barrier_sync(1, kTcEpiThreads);
-      if (tid == 0) {
-        __threadfence();
-        s_old = atomicAdd(tile_cnt + row_tile, 1u);
+      for (uint32_t ti = 0; ti < n_tiles; ++ti) {
+        const uint32_t row_tile = mt.x + ti;
+        named_barrier_sync(1, kTcEpiThreads);
+        if (tid == 0) {
+          __threadfence();
+          s_old = atomicAdd(tile_cnt + row_tile, 1u);
+        }
+        named_barrier_sync(1, kTcEpiThreads);
+        if (s_old == n_seg - 1) {
+          __threadfence();
+          combine_tile<NPAD, kTcEpiThreads>(p, row_tile, n_seg, tid, status);
+          if (tid == 0) tile_cnt[row_tile] = 0;
+        }
+        named_barrier_sync(1, kTcEpiThreads);
       }
-      named_barrier_sync(1, kTcEpiThreads);
-      if (s_old == n_seg - 1) {
-        __threadfence();
-        combine_tile<NPAD, kTcEpiThreads>(p, row_tile, n_seg, tid, status);
-        if (tid == 0) tile_cnt[row_tile] = 0;
-      }
-      named_barrier_sync(1, kTcEpiThreads);
     }
   }
   named_barrier_sync(2, kTcEpiThreads + 32);
@@ -1081,8 +1113,9 @@ struct KernelState {
   int resident = 0;   // threadblocks of the kernel that one SM holds at its shared-memory size
 };
 
+// pairs: the even partition counts (pair of row tiles, k block) units instead of blocks.
 int launch_planned(void (*kernel)(ChainParams), KernelState& state, uint32_t threads, uint32_t stage_bytes,
-                   uint32_t ctas_per_sm, const ChainParams& chain, int sms, cudaStream_t stream) {
+                   uint32_t ctas_per_sm, bool pairs, const ChainParams& chain, int sms, cudaStream_t stream) {
   ChainParams c = chain;
   uint32_t n_stages = (kSmemBudget / ctas_per_sm - 1024) / stage_bytes;
   if (n_stages > kMaxStages) n_stages = kMaxStages;
@@ -1111,7 +1144,13 @@ int launch_planned(void (*kernel)(ChainParams), KernelState& state, uint32_t thr
     const uint32_t per_cta = (items + max_ctas - 1) / max_ctas;
     uint32_t g = (items + per_cta - 1) / per_cta;
     if (g > queue_len) g = queue_len;
-    if (q.even_part) g = q.total_blocks < max_ctas ? q.total_blocks : max_ctas;
+    if (q.even_part) {
+      // at least one unit per threadblock: the partial-sum slots of a row tile are sized for that
+      // pairs of row tiles where every threadblock still gets a long run (32 units or more)
+      q.tiles_per_unit = (pairs && (uint64_t)((q.n_row_tiles + 1) / 2) * q.k_blocks >= 32ull * max_ctas) ? 2u : 1u;
+      const uint32_t units = ((q.n_row_tiles + q.tiles_per_unit - 1) / q.tiles_per_unit) * q.k_blocks;
+      g = units < max_ctas ? units : max_ctas;
+    }
     q.active_ctas = g;
     if (g > grid) grid = g;
   }
@@ -1136,14 +1175,14 @@ int launch_planned(void (*kernel)(ChainParams), KernelState& state, uint32_t thr
 template <int NT, int MB>
 int launch_gemv(const ChainParams& chain, int sms, cudaStream_t stream) {
   static KernelState state;
-  return launch_planned(gemv_tiered_kernel<NT, MB>, state, kGemvThreads, stage_bytes_of(NT, MB), (NT >= 8) ? 1 : 2, chain,
-                        sms, stream);
+  return launch_planned(gemv_tiered_kernel<NT, MB>, state, kGemvThreads, stage_bytes_of(NT, MB), (NT >= 8) ? 1 : 2, false,
+                        chain, sms, stream);
 }
 
 template <uint32_t NPAD>
 int launch_gemv_tc(const ChainParams& chain, int sms, cudaStream_t stream) {
   static KernelState state;
-  return launch_planned(gemv_tc_kernel<NPAD>, state, kTcThreads, tc_stage_bytes(NPAD), 1, chain, sms, stream);
+  return launch_planned(gemv_tc_kernel<NPAD>, state, kTcThreads, tc_stage_bytes(NPAD), 1, true, chain, sms, stream);
 }
 
 }  // namespace
@@ -1287,6 +1326,7 @@ int fill_params(GemvParams& p, const void* const* w_page_ptr, const uint32_t* w_
   p.even_part = n_host_pages == 0 ? 1u : 0u;
   p.total_blocks = lay.n_row_tiles * lay.k_blocks;
   p.max_seg = partial_slots(lay, M_b);
+  p.tiles_per_unit = 1;
   p.items_per_page = kBlocksPerPage / lay.blocks_per_item;
   p.n_items = (uint32_t)((uint64_t)lay.n_row_tiles * lay.k_blocks / lay.blocks_per_item);
   p.x = static_cast<const __nv_bfloat16*>(x);
