@@ -640,6 +640,10 @@ def run_stream_sweep(args):
     sms = torch.cuda.get_device_properties(dev).multi_processor_count
     ratios = [0.0, 1 / 256, 1 / 128, 1 / 64, 1 / 32, 1 / 16, 1 / 8]
     policies = [("modulo", B.POLICY_MODULO), ("contiguous", B.POLICY_CONTIGUOUS), ("random", B.POLICY_RANDOM)]
+    if args.sweep_ratios:     # a subset, for a profiler capture of single points
+        ratios = [float(x) for x in args.sweep_ratios.split(",")]
+    if args.sweep_policies:
+        policies = [pp for pp in policies if pp[0] in args.sweep_policies.split(",")]
     sizes = [int(x) for x in args.sweep_gib.split(",")]
     points = []
     for gib in sizes:
@@ -697,6 +701,8 @@ def main():
                          "batch sizes and host shares")
     ap.add_argument("--sweep-gib", default="1,4,16")
     ap.add_argument("--sweep-seeds", type=int, default=5)
+    ap.add_argument("--sweep-ratios", default="", help="stream_sweep: comma-separated host shares (default: the full list)")
+    ap.add_argument("--sweep-policies", default="", help="stream_sweep: subset of modulo,contiguous,random")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     rank = int(os.environ.get("RANK", "0"))

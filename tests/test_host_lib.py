@@ -214,3 +214,52 @@ def test_pool_config5_geometry():
     assert q["host_heads_lo"] == 1 and q["first_hi_block"] == int(0.4 * n) == ref.kind.index(1)
     assert q["n_host_pages"] * 5 == q["n_pages"]
     pool.close()
+
+
+def test_chain_and_step_workspace_sizes_and_argument_checks():
+    """Host-side logic of the chained products: workspace sizes grow with what they must hold,
+    and calls that cannot be valid are refused before any CUDA work (no GPU needed)."""
+    import ctypes as C
+    lib = B.lib()
+
+    def call(n, k):
+        c = B.GemvCall()
+        c.w = B.Weight(0, 0, B.boost_weight_layout(n, k)["n_pages"], 0, n, k)
+        c.y_dtype = 1
+        return c
+
+    def chain(shapes):
+        arr = (B.GemvCall * len(shapes))()
+        for i, (n, k) in enumerate(shapes):
+            arr[i] = call(n, k)
+        return arr
+
+    one = chain([(4096, 4096)])
+    four = chain([(4096, 4096), (28672, 4096), (4096, 14336), (6144, 4096)])
+    w1 = B.boost_gemv_chain_workspace_bytes(one, 32)
+    w4 = B.boost_gemv_chain_workspace_bytes(four, 32)
+    assert 0 < w1 < w4
+    # a chain needs at least what its largest product needs alone
+    assert w4 >= max(B.boost_gemv_workspace_bytes(n, k, 32) for n, k in [(4096, 4096), (28672, 4096), (4096, 14336), (6144, 4096)])
+    assert B.boost_gemv_chain_workspace_bytes(four, 128) > w4          # partial sums grow with the batch
+    assert lib.boost_gemv_chain_workspace_bytes(C.addressof(four), 5, 32) == 0   # more than four products
+    assert lib.boost_gemv_chain_workspace_bytes(C.addressof(four), 0, 32) == 0
+    assert B.boost_gemv_chain_workspace_bytes(four, 0) == 0 and B.boost_gemv_chain_workspace_bytes(four, 129) == 0
+    for n_calls in (0, 5):
+        rc = lib.boost_gemv_tiered_chain(C.addressof(four), n_calls, 32, None, 1 << 30, None)
+        assert rc == B.ERR_INVALID
+    assert lib.boost_gemv_tiered_chain(C.addressof(four), 4, 32, None, 1 << 30, None) == B.ERR_INVALID   # no workspace
+    assert lib.boost_gemv_tiered_chain(C.addressof(four), 4, 32, 256, 1024, None) == B.ERR_CAPACITY
+    assert lib.boost_gemv_tiered_chain(C.addressof(four), 4, 32, 257, 1 << 30, None) == B.ERR_ALIGN
+
+    # decode-step workspace: counters for the widest product + the largest partial sums + queue words
+    layers = (B.LlamaLayer * 2)()
+    for ly in layers:
+        ly.wqkv, ly.wo, ly.wgu, ly.wd = call(6144, 4096).w, call(4096, 4096).w, call(28672, 4096).w, call(4096, 14336).w
+    m = B.LlamaModel()
+    m.n_layers, m.lm_head = 2, call(128256, 4096).w
+    m.layers = C.cast(layers, C.POINTER(B.LlamaLayer))
+    s32, s128 = B.boost_llama_gemv_workspace_bytes(m, 32), B.boost_llama_gemv_workspace_bytes(m, 128)
+    assert s32 >= B.boost_gemv_workspace_bytes(128256, 4096, 32) and s128 > s32
+    assert B.boost_llama_gemv_workspace_bytes(m, 0) == 0 and B.boost_llama_gemv_workspace_bytes(m, 129) == 0
+    B.boost_gemv_set_tc_min_batch(33)
