@@ -172,6 +172,53 @@ def run_reference(args, rank, world):
     print(json.dumps(line), flush=True)
 
 
+def run_reference_configs(args):
+    """The CPU oracle, as it stands, timed on configurations 1 - 3 on this machine's host cores: with
+    one thread and with all of them (the BLAS calls inside numpy are what threads).  One JSON
+    document; the decode-step sample of configuration 4 is the default `--impl reference` line."""
+    from oracle import kv_pool as okp
+    from oracle import linalg as ol
+    from oracle import placement as op
+    from paper_2609_13592_b200 import synth
+    try:
+        from threadpoolctl import threadpool_limits
+    except Exception:
+        threadpool_limits = None
+    # inputs (not timed)
+    w1, x1 = synth.normal_bf16((4096, 4096), 0.02, 1), synth.normal_bf16((1, 4096), 1.0, 2)
+    ctx2 = synth.ctx_lens_uniform(8, 512, 4096, seed=2).tolist()
+    pool = okp.KVPool(2560, 8, 8, 16 * 128 * 2)
+    table = np.zeros((8, 256), np.int64)
+    for b, c in enumerate(ctx2):
+        blocks = pool.alloc(b, (c + 15) // 16)
+        table[b, :len(blocks)] = blocks
+    k2, v2 = synth.normal_bf16((8, 2560, 16, 128), 1.0, 20), synth.normal_bf16((8, 2560, 16, 128), 1.0, 21)
+    q2 = synth.normal_bf16((8, 32, 128), 1.0, 22)
+    page_elems = (2 << 20) // 2
+    buf3 = synth.small_int_bf16(0, 512 * page_elems) if hasattr(synth, "small_int_bf16") else \
+        synth.f32_to_bf16_bits(synth.small_int_values(0, 512 * page_elems).astype(np.float32))
+
+    def timed(fn):
+        t0 = time.perf_counter()
+        fn()
+        return time.perf_counter() - t0
+
+    cases = {
+        "c1_place_pages_and_gemv_4096x4096_batch1": lambda: (op.place_pages(4096 * 4096 * 2, 1 / 16), ol.gemm(x1, w1)),
+        "c2_attention_batch8_ctx512_4096": lambda: ol.paged_attention_decode(q2, k2, v2, table, ctx2, 1.0 / np.sqrt(128.0)),
+        "c3_stream_sum_1gib": lambda: ol.stream_sum(buf3, page_elems),
+    }
+    out = {}
+    for name, fn in cases.items():
+        row = {"all_cores_s": timed(fn)}
+        if threadpool_limits is not None:
+            with threadpool_limits(limits=1):
+                row["one_thread_s"] = timed(fn)
+        out[name] = row
+    print(json.dumps({"impl": "reference", "workload": "oracle_on_configs_1_to_3", "cores": os.cpu_count(),
+                      "seconds": out}), flush=True)
+
+
 # ------------------------------------------------------------------------------ device leg
 
 def measure_stream(dev, n_pages, tier_value, reps=5):
@@ -694,11 +741,12 @@ def main():
     ap.add_argument("--ctx", type=int, default=2048)
     ap.add_argument("--layers", type=int, default=0, help="override the layer count (0 = 32)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--workload", default="decode", choices=["decode", "stream_sweep", "kv_spill", "gemv_sweep"],
+    ap.add_argument("--workload", default="decode", choices=["decode", "stream_sweep", "kv_spill", "gemv_sweep", "oracle_configs"],
                     help="decode: the benchmark line; stream_sweep: the placement sweep of configuration 3; "
                          "kv_spill: configuration 5 (batch 128, one KV page in five on the host) with its "
                          "HBM-only and prefetch-to-HBM comparison runs; gemv_sweep: weight products over shapes, "
-                         "batch sizes and host shares")
+                         "batch sizes and host shares; oracle_configs (with --impl reference): the CPU oracle timed on "
+                         "configurations 1 - 3")
     ap.add_argument("--sweep-gib", default="1,4,16")
     ap.add_argument("--sweep-seeds", type=int, default=5)
     ap.add_argument("--sweep-ratios", default="", help="stream_sweep: comma-separated host shares (default: the full list)")
@@ -717,6 +765,9 @@ def main():
     elif args.workload == "stream_sweep":
         if rank == 0:
             run_stream_sweep(args)
+    elif args.impl == "reference" and args.workload == "oracle_configs":
+        if rank == 0:
+            run_reference_configs(args)
     elif args.impl == "reference":
         run_reference(args, rank, world)
     else:
