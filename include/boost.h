@@ -548,15 +548,21 @@ int boost_llama_decode_step_prefetch(const boost_llama_model_t* model /*host*/,
  * step as a chain of weight products; they share one workspace).  0 on invalid arguments. */
 size_t boost_llama_gemv_workspace_bytes(const boost_llama_model_t* model /*host*/, uint32_t B);
 
-/* One decode step for B sequences: embedding, n_layers x (RMSNorm, QKV product, RoPE + KV
- * append, paged attention, output product + residual, RMSNorm, gate/up product, SwiGLU,
- * down product + residual), final RMSNorm, LM head, argmax - as 2 + 5 n_layers + 2 launches:
- * every small operator rides in the epilogue of a weight product (boost_gemv_tiered_fused:
- * RMSNorm as a row scale with its weight folded into the matrix, RoPE + KV append after the
- * QKV product, SwiGLU after the gate/up product, the row statistics of the residual stream
- * after the output and down products).  Activations between kernels are bf16; logits fp32.  tokens, block_table [B, max_blocks], ctx_lens (new
- * token included) and next_tokens are device arrays.  Launches are asynchronous on stream.
- * Returns the number of kernels launched in *n_launches_out when it is not NULL. */
+/* One decode step for B sequences (Sec. 2.1: a chain of weight-streaming products and
+ * attention kernels): embedding, n_layers x (RMSNorm, QKV product, RoPE + KV append, paged
+ * attention, output product + residual, RMSNorm, gate/up product, SwiGLU, down product +
+ * residual), final RMSNorm, LM head, argmax - as 4 + 2 n_layers launches: RoPE table,
+ * embedding gather, the first layer's QKV product, then per layer the attention kernel and
+ * ONE chain launch (boost_gemv_tiered_chain) for the output, gate/up and down products and the
+ * next layer's QKV product (the LM head after the last layer), then argmax.  Every small
+ * operator rides in the epilogue of a weight product (RMSNorm as a row scale with its weight
+ * folded into the matrix, RoPE + KV append after the QKV product, SwiGLU after the gate/up
+ * product, the row statistics of the residual stream after the output and down products).
+ * Activations between kernels are bf16; logits fp32.  tokens, block_table [B, max_blocks],
+ * ctx_lens (new token included) and next_tokens are device arrays.  Launches are
+ * asynchronous on stream.  Returns the number of kernels launched in *n_launches_out when
+ * it is not NULL.  Errors: INVALID, UNSUPPORTED (head_dim != 128, hidden % 128 != 0),
+ * CAPACITY (scratch->gemv_ws too small), CUDA. */
 int boost_llama_decode_step(const boost_llama_model_t* model /*host*/,
                             const boost_llama_scratch_t* scratch /*host*/,
                             const int32_t* tokens /*device*/, const int32_t* block_table /*device*/,
