@@ -280,8 +280,15 @@ int boost_pack_weights_ex(const void* w_row_major /*device*/, uint32_t N, uint32
  *   residual   device bf16 [M_b, N] added before the final rounding, or NULL;
  *   workspace  device, >= boost_gemv_workspace_bytes(N, K, M_b).
  * M_b <= 2 runs on CUDA cores with warp-shuffle reductions; larger batches use the tensor
- * cores (batch padded to a multiple of 16).  Split-K partial sums are combined in a fixed order by the last threadblock to
- * finish a row tile, so the result is deterministic. */
+ * cores (mma.sync up to 32 rows, tcgen05 with accumulators in tensor memory above; see
+ * boost_gemv_set_tc_min_batch).  A weight with host pages is cut into work items handed out
+ * host pages first; a weight entirely in HBM is cut evenly over the threadblocks.  Split-K
+ * partial sums are combined in a fixed order by the last threadblock to finish a row tile, so
+ * the result is deterministic (to the bit for a given placement, device and batch; across
+ * placements the order of the fp32 sums, hence the last bits, may differ).
+ * Errors: INVALID, ALIGN (x not 16-byte, workspace not 256-byte aligned, K % 8 != 0), CAPACITY,
+ * CUDA.  Word 0 of the workspace collects error bits of the kernel (bit 0: a bounded wait ran
+ * out; bit 1: a block index out of range in the RoPE / KV-append epilogue). */
 size_t boost_gemv_workspace_bytes(uint32_t N, uint32_t K, uint32_t M_b);
 int boost_gemv_tiered(const void* const* w_page_ptr /*device*/, const uint32_t* w_order /*device*/,
                       size_t n_pages, size_t n_host_pages, uint32_t N, uint32_t K,
