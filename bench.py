@@ -606,6 +606,123 @@ def run_kv_spill(args):
     print(json.dumps(line), flush=True)
 
 
+def run_pool_churn(args):
+    """KV pool under serving-like churn (Sec. 5.9, Sec. 5.10): Poisson arrivals with a
+    long-generation length mix are replayed on the wave-aware pool at about 80 % utilisation for
+    12 000 decode steps; the host share of the live KV chunks is recorded after every step
+    (rolling median and min - max band over 500 steps, against the configured 1/M and the 1/H
+    granularity bound), and at five steps the attention kernel is timed on the batch as the
+    churned pool laid it out, on the same batch laid out by an unused pool, and with every KV
+    page in HBM.  Three pools: four KV heads with one page in twelve on the host, eight KV
+    heads with one page in eight, and eight KV heads at the measured link share.  Prints one
+    JSON document."""
+    import math
+    import torch
+    from paper_2609_13592_b200 import binding as B
+    from paper_2609_13592_b200 import build as libbuild
+    from paper_2609_13592_b200 import serving, synth
+    from paper_2609_13592_b200.tiers import TieredKVCache, aligned_workspace
+    libbuild.build_library()
+    B.lib()
+    dev = torch.device("cuda:0")
+    torch.cuda.set_device(dev)
+    hbm_peak, peak_src = load_peaks()
+    link = measure_stream(dev, 64, 1)
+    link_modulus = B.boost_modulus_from_bandwidths(hbm_peak, link)
+    d, n_steps, window = 128, args.churn_steps, 500
+    snaps = [int(n_steps * f) - 1 for f in (1 / 3, 1 / 2, 2 / 3, 5 / 6, 1.0)]
+    pools = [dict(name="4_kv_heads_one_page_in_12", n_blocks=12 * 1024, hkv=4, hq=32, modulus=12, rate=0.045, max_batch=96),
+             dict(name="8_kv_heads_one_page_in_8", n_blocks=8 * 1024, hkv=8, hq=32, modulus=8, rate=0.028, max_batch=64),
+             dict(name=f"8_kv_heads_link_share_one_page_in_{link_modulus}", n_blocks=64 * 1024, hkv=8, hq=32,
+                  modulus=link_modulus, rate=0.22, max_batch=384)]
+    g = torch.Generator(device=dev)
+    g.manual_seed(11)
+    scale = 1.0 / math.sqrt(d)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+
+    def time_attention(cache, table, ctx, hq, hkv, n_blocks, reps=20):
+        n_seq, max_blocks = table.shape
+        ws_bytes = B.boost_paged_attn_workspace_bytes(n_seq, hq, d, max_blocks)
+        ws_t, ws = aligned_workspace(ws_bytes, dev)
+        q = torch.randn(n_seq, hq, d, generator=g, device=dev).to(torch.bfloat16)
+        out = torch.empty(n_seq, hq, d, dtype=torch.bfloat16, device=dev)
+        table_d, ctx_d = torch.from_numpy(table).to(dev), torch.from_numpy(ctx).to(dev)
+        # every launch starts with a cold L2 (the flush buffer is twice its size) and is queued
+        # while the flush still runs, so the events see the kernel and not the host's launch path
+        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(reps + 3)]
+        for e0, e1 in ev:
+            flush.zero_()
+            e0.record()
+            B.boost_paged_attn_decode_tiered(q, cache.k.page_ptr, cache.v.page_ptr, cache.tier, cache.n_pages, n_blocks,
+                                             table_d, max_blocks, ctx_d, n_seq, hq, hkv, d, scale, ws, ws_bytes, out)
+            e1.record()
+        torch.cuda.synchronize(dev)
+        times = [e0.elapsed_time(e1) * 1e3 for e0, e1 in ev[3:]]
+        off = ws - ws_t.data_ptr()
+        status = int(ws_t[off:off + 4].cpu().numpy().view(np.uint32)[0])
+        assert bool(torch.isfinite(out.float()).all())
+        return float(np.median(times)), status
+
+    results = []
+    for pc in pools:
+        n_blocks, hkv, hq, m = pc["n_blocks"], pc["hkv"], pc["hq"], pc["modulus"]
+        pool = B.KVPool(n_blocks, hkv, m)
+        trace = synth.serving_churn_trace(n_blocks, n_steps, pc["rate"], pc["max_batch"], seed=7)
+        shares, batch_sizes, live_blocks, snapshots, stats = serving.replay_churn(pool, trace, snaps)
+        warm = n_steps // 4
+        s = shares[warm:]
+        medians = [float(np.median(s[i:i + window])) for i in range(0, len(s) - window, 50)]
+        lows = [float(s[i:i + window].min()) for i in range(0, len(s) - window, 50)]
+        highs = [float(s[i:i + window].max()) for i in range(0, len(s) - window, 50)]
+        info = pool.query()
+        cache = TieredKVCache(pool, hkv, n_blocks, d, dev)
+        hbm_pool = B.KVPool(n_blocks, hkv, 0)
+        hbm_cache = TieredKVCache(hbm_pool, hkv, n_blocks, d, dev)
+        for c in (cache, hbm_cache):
+            for buf in (c.k, c.v):
+                t = torch.randn(hkv, n_blocks, 16, d, generator=g, device=dev, dtype=torch.bfloat16)
+                B.boost_kv_scatter(t, hkv, n_blocks, d, buf.page_ptr, buf.n_pages)
+                torch.cuda.synchronize(dev)
+                del t
+        points = []
+        for sn in snapshots:
+            ctx, table = sn["ctx_lens"], sn["table"]
+            host_b, all_b = serving.host_kv_bytes(table, ctx, dict(info, n_kv_heads=hkv), d)
+            fresh_pool = B.KVPool(n_blocks, hkv, m)
+            fresh = serving.fresh_tables(fresh_pool, ctx)
+            fresh_host_b, _ = serving.host_kv_bytes(fresh, ctx, dict(info, n_kv_heads=hkv), d)
+            fresh_pool.close()
+            us_churn, st1 = time_attention(cache, table, ctx, hq, hkv, n_blocks)
+            us_fresh, st2 = time_attention(cache, fresh, ctx, hq, hkv, n_blocks)
+            us_hbm, st3 = time_attention(hbm_cache, table, ctx, hq, hkv, n_blocks)
+
+            def bound_us(host_bytes):
+                return 1e6 * max((all_b - host_bytes) / (hbm_peak * 1e9), host_bytes / (link * 1e9))
+            points.append({"step": sn["step"], "batch": int(len(ctx)), "tokens": int(ctx.sum()), "max_ctx": int(ctx.max()),
+                           "kv_bytes": all_b, "host_share_churned": host_b / all_b, "host_share_fresh": fresh_host_b / all_b,
+                           "us_churned": us_churn, "us_fresh": us_fresh, "us_hbm_only": us_hbm,
+                           "tier_bound_us_churned": bound_us(host_b), "tier_bound_us_fresh": bound_us(fresh_host_b),
+                           "frac_of_tier_bound_churned": bound_us(host_b) / us_churn,
+                           "frac_of_tier_bound_fresh": bound_us(fresh_host_b) / us_fresh,
+                           "hbm_only_gbs": all_b / us_hbm / 1e3, "status": [st1, st2, st3]})
+        results.append({"pool": pc["name"], "n_blocks": n_blocks, "n_kv_heads": hkv, "n_q_heads": hq, "host_modulus": m,
+                        "target_share": info["n_host_pages"] / info["n_pages"], "granularity_bound": 1.0 / hkv,
+                        "arrivals_per_step": pc["rate"], "max_batch": pc["max_batch"], "steps": n_steps,
+                        "trace": stats, "mean_batch": float(batch_sizes[warm:].mean()),
+                        "mean_utilisation": float(live_blocks[warm:].mean() / n_blocks),
+                        "peak_utilisation": float(live_blocks.max() / n_blocks),
+                        "share_after_warm_in": {"min": float(s.min()), "median": float(np.median(s)), "max": float(s.max())},
+                        "rolling_median_band": [min(medians), max(medians)],
+                        "rolling_min_max_band": [min(lows), max(highs)],
+                        "attention": points})
+        pool.close()
+        hbm_pool.close()
+        del cache, hbm_cache
+        torch.cuda.empty_cache()
+    print(json.dumps({"workload": "kv_pool_under_serving_churn", "hbm_peak_gbs": hbm_peak, "hbm_peak_source": peak_src,
+                      "host_link_gbs": link, "pools": results}))
+
+
 def run_gemv_sweep(args):
     """Weight-product sweep over the Llama-3-8B matrix shapes, batch 1 .. 128 and three host
     shares (0, the measured link share, 1/16): where tiering is free, where the link binds, and
@@ -741,12 +858,14 @@ def main():
     ap.add_argument("--ctx", type=int, default=2048)
     ap.add_argument("--layers", type=int, default=0, help="override the layer count (0 = 32)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--workload", default="decode", choices=["decode", "stream_sweep", "kv_spill", "gemv_sweep", "oracle_configs"],
+    ap.add_argument("--workload", default="decode", choices=["decode", "stream_sweep", "kv_spill", "gemv_sweep", "pool_churn", "oracle_configs"],
                     help="decode: the benchmark line; stream_sweep: the placement sweep of configuration 3; "
                          "kv_spill: configuration 5 (batch 128, one KV page in five on the host) with its "
                          "HBM-only and prefetch-to-HBM comparison runs; gemv_sweep: weight products over shapes, "
-                         "batch sizes and host shares; oracle_configs (with --impl reference): the CPU oracle timed on "
+                         "batch sizes and host shares; pool_churn: the KV pool under serving-like arrivals, realised host "
+                         "share over time and attention timed on churned against fresh layouts; oracle_configs (with --impl reference): the CPU oracle timed on "
                          "configurations 1 - 3")
+    ap.add_argument("--churn-steps", type=int, default=12000, help="pool_churn: decode steps replayed")
     ap.add_argument("--sweep-gib", default="1,4,16")
     ap.add_argument("--sweep-seeds", type=int, default=5)
     ap.add_argument("--sweep-ratios", default="", help="stream_sweep: comma-separated host shares (default: the full list)")
@@ -762,6 +881,9 @@ def main():
     elif args.workload == "gemv_sweep":
         if rank == 0:
             run_gemv_sweep(args)
+    elif args.workload == "pool_churn":
+        if rank == 0:
+            run_pool_churn(args)
     elif args.workload == "stream_sweep":
         if rank == 0:
             run_stream_sweep(args)

@@ -405,6 +405,10 @@ int boost_kv_gather(void* dst /*device*/, uint32_t n_kv_heads, uint32_t n_pool_b
  *                a linear placement (HBM pages, then host pages), else UNSUPPORTED;
  *   block_table  device int32 [B, max_blocks]; ctx_lens device int32 [B] (tokens cached,
  *                the current one included); query head j reads KV head j / (Hq/Hkv);
+ *                the kernel cuts the sequences into work items from ctx_lens itself, and
+ *                reads ctx_lens and block_table before it waits for the kernel launched
+ *                just before it on the stream when that kernel is one of this library's
+ *                (which write neither); the newest K / V rows and q are read after it;
  *   out          device bf16 [B, Hq, D];
  *   workspace    device, >= boost_paged_attn_workspace_bytes(B, Hq, D, max_blocks). */
 size_t boost_paged_attn_workspace_bytes(uint32_t B, uint32_t Hq, uint32_t D, uint32_t max_blocks);

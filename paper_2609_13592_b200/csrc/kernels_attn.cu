@@ -15,6 +15,9 @@
 // transposed in registers with movmatrix; the online softmax is fp32.  The four quarters are
 // merged in shared memory; only a sequence longer than one item leaves partial results in
 // global memory, and the last of its items to finish combines them in run order.
+// The run length is not fixed by the host: every threadblock derives it, and a dense list of
+// the items, from the context lengths when it starts (before the wait on the preceding
+// kernel), so the decomposition follows the batch's real mix of lengths.
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <math_constants.h>
@@ -39,6 +42,8 @@ constexpr uint32_t kAttnThreads = kAttnWarps * 32;
 constexpr uint32_t kWarpStages = 2;                      // ring depth of one warp
 constexpr uint32_t kMaxGroup = 16;
 constexpr uint32_t kParkStride = kD + 4;                 // floats per parked head: 128 outputs, m, l, padding
+constexpr uint32_t kMaxListedSeqs = 1024;                // batches up to this size get a dense item list
+constexpr uint32_t kTailPieces = 4;                      // the runs of the last KV head are cut in this many items
 
 #ifdef BOOST_TRACE
 // Debug build only: per-warp time stamps (global timer, ns), 8 slots per warp.
@@ -57,10 +62,11 @@ struct AttnParams {
   const int32_t* block_table;
   uint32_t max_blocks;
   const int32_t* ctx_lens;
-  uint32_t B, Hq, Hkv, group, max_splits, n_items, item_blocks;
+  uint32_t B, Hq, Hkv, group;
+  uint32_t cta_slots;         // threadblocks the device holds at once (the balance target)
   float scale_log2e;
   uint32_t* ws;        // header (status, item counter, done counter) + one counter per (b, g)
-  float* part_ml;      // [B][Hq][max_splits][2]
+  float* part_ml;      // [B][Hq][max_splits][2], max_splits from the run length chosen on the device
   float* part_o;       // [B][Hq][max_splits][128]
   __nv_bfloat16* out;
 };
@@ -96,28 +102,120 @@ __global__ void __launch_bounds__(kAttnThreads, (NH == 1 ? 3 : 2)) paged_attn_ke
 
   // Fragment coordinates: rows gq, gq+8 (tokens for S^T, d for O^T), columns c0, c0+1 (heads).
   const uint32_t gq = lane >> 2, c0 = (lane & 3) * 2;
-  const uint32_t per_head = p.B * p.max_splits;
   uint32_t phase_mask = 0;                       // bit s = phase to wait for on stage s
   // A work item belongs to the threadblock: (sequence b, KV head g, a run of blocks); its four
   // warps take a quarter of the run each and stream it on their own; their results meet in
   // shared memory.  First item by position, later ones from the counter.
   __shared__ uint32_t s_next, s_old;
+  __shared__ uint32_t s_warp_sum[kAttnWarps], s_warp_max[kAttnWarps];
+  __shared__ uint32_t s_first_item[kMaxListedSeqs + 1];   // first item of every sequence within a head
+
+  // ---- run length.  Every threadblock derives the same decomposition from the context
+  // lengths.  An item costs a table look-up, a query load and, when a sequence needs several
+  // items, a partial result in global memory, so long runs are better; but the kernel ends with
+  // its longest item, and about 55 % of the threadblocks the device holds saturate HBM
+  // (measured on B200: about a thousand warps with 16 KiB in flight each).  With u KV blocks
+  // per threadblock slot on average: when the sequences are about equally long, a run is at
+  // most 1.75 u blocks, so that share of the slots gets one item each and all end together;
+  // with a mix of lengths (longest above 1.25 times the mean) items differ in length anyway,
+  // and runs of at most u give every slot a few items to even out through the queue.
+  uint32_t my_blocks = 0, my_max = 0;
+  for (uint32_t b = tid; b < p.B; b += kAttnThreads) {
+    const uint32_t n = ((uint32_t)max(p.ctx_lens[b], 0) + kTok - 1) / kTok;
+    my_blocks += n;
+    my_max = max(my_max, n);
+  }
+#pragma unroll
+  for (int sh = 16; sh >= 1; sh >>= 1) {
+    my_blocks += __shfl_xor_sync(0xFFFFFFFFu, my_blocks, sh);
+    my_max = max(my_max, __shfl_xor_sync(0xFFFFFFFFu, my_max, sh));
+  }
+  if (lane == 0) { s_warp_sum[warp] = my_blocks; s_warp_max[warp] = my_max; }
+  __syncthreads();
+  uint64_t total_blocks = 0;
+  uint32_t longest = 0;
+#pragma unroll
+  for (uint32_t w = 0; w < kAttnWarps; ++w) { total_blocks += s_warp_sum[w]; longest = max(longest, s_warp_max[w]); }
+  const bool mixed = (uint64_t)longest * p.B * 4 > total_blocks * 5;
+  const uint64_t quarters = mixed ? 4 : 7;   // run cap in quarters of u
+  const uint64_t run_cap = (total_blocks * p.Hkv * quarters + (uint64_t)p.cta_slots * 4 - 1) / ((uint64_t)p.cta_slots * 4);
+  const uint32_t item_blocks = (uint32_t)min((uint64_t)kMaxItemBlocks, max((uint64_t)kMinItemBlocks, (run_cap + kAttnWarps - 1) / kAttnWarps));
+  const uint32_t cta_max = kAttnWarps * item_blocks;
+  const uint32_t max_splits = (p.max_blocks + cta_max - 1) / cta_max;
+  // ---- item list.  Up to kMaxListedSeqs sequences: items are numbered densely, sequence by
+  // sequence (s_first_item = running count of runs), so no threadblock draws an empty item.
+  // Larger batches: every sequence has max_splits numbers and the unused ones are skipped.
+  const bool listed = p.B <= kMaxListedSeqs;
+  uint32_t per_head = p.B * max_splits;
+  if (listed) {
+    uint32_t carry = 0;
+    for (uint32_t b0 = 0; b0 < p.B; b0 += kAttnThreads) {
+      const uint32_t b = b0 + tid;
+      const uint32_t n_blk = b < p.B ? ((uint32_t)max(p.ctx_lens[b], 0) + kTok - 1) / kTok : 0;
+      const uint32_t mine = b < p.B ? (n_blk ? (n_blk + cta_max - 1) / cta_max : 1u) : 0u;
+      uint32_t incl = mine;
+#pragma unroll
+      for (int sh = 1; sh < 32; sh <<= 1) {
+        const uint32_t up = __shfl_up_sync(0xFFFFFFFFu, incl, sh);
+        if ((int)lane >= sh) incl += up;
+      }
+      __syncthreads();   // s_warp_sum is free again
+      if (lane == 31) s_warp_sum[warp] = incl;
+      __syncthreads();
+      uint32_t before = carry, round_total = 0;
+#pragma unroll
+      for (uint32_t w = 0; w < kAttnWarps; ++w) {
+        if (w < warp) before += s_warp_sum[w];
+        round_total += s_warp_sum[w];
+      }
+      if (b < p.B) s_first_item[b] = before + incl - mine;
+      carry += round_total;
+    }
+    if (tid == 0) s_first_item[p.B] = carry;
+    __syncthreads();
+    per_head = carry;
+  }
+  // The queue ends with KV head 0.  With a mix of lengths its runs are cut in kTailPieces
+  // items each, so the threadblocks run out of work within a short item of one another.
+  const uint32_t tail_k = mixed ? kTailPieces : 1u;
+  const uint32_t n_long = (p.Hkv - 1) * per_head;
+  const uint32_t n_items = n_long + per_head * tail_k;
+  const uint32_t slots_per = max_splits * tail_k;      // partial results of one (sequence, query head)
+  ATRACE(7);
   uint32_t id = blockIdx.x;
 
-  while (id < p.n_items) {
-    const uint32_t g = p.Hkv - 1 - id / per_head;     // host-resident heads first
-    const uint32_t b = (id % per_head) / p.max_splits;
-    const uint32_t split = id % p.max_splits;
+  while (id < n_items) {
+    const bool tail = id >= n_long;
+    const uint32_t g = tail ? 0u : p.Hkv - 1 - id / per_head;     // host-resident heads first
+    const uint32_t k_pieces = tail ? tail_k : 1u;
+    const uint32_t in_head = tail ? (id - n_long) / tail_k : id % per_head;
+    const uint32_t piece = tail ? (id - n_long) % tail_k : 0u;
+    uint32_t b, split;
+    if (listed) {
+      // the sequence whose range of items holds in_head: last b with s_first_item[b] <= in_head
+      uint32_t lo = 0, hi = p.B;
+      while (hi - lo > 1) {
+        const uint32_t mid = (lo + hi) >> 1;
+        if (s_first_item[mid] <= in_head) lo = mid; else hi = mid;
+      }
+      b = lo;
+      split = in_head - s_first_item[lo];
+    } else {
+      b = in_head / max_splits;
+      split = in_head % max_splits;
+    }
     const uint32_t ctx = (uint32_t)max(p.ctx_lens[b], 0);
     const uint32_t n_blk = (ctx + kTok - 1) / kTok;
-    const uint32_t cta_max = kAttnWarps * p.item_blocks;
     const uint32_t n_splits = n_blk ? (n_blk + cta_max - 1) / cta_max : 1;
     if (split < n_splits) {
       // the sequence's blocks in n_splits runs of equal length (the last may be shorter by a
       // few), each run in four quarters
       const uint32_t run_len = n_blk ? (n_blk + n_splits - 1) / n_splits : 0;
-      const uint32_t cblk0 = split * run_len;
-      const uint32_t cnb = min(run_len, n_blk - min(n_blk, cblk0));
+      const uint32_t rblk0 = split * run_len;
+      const uint32_t rnb = min(run_len, n_blk - min(n_blk, rblk0));
+      const uint32_t piece_len = (rnb + k_pieces - 1) / k_pieces;
+      const uint32_t cblk0 = rblk0 + piece * piece_len;
+      const uint32_t cnb = min(piece_len, rnb - min(rnb, piece * piece_len));
       const uint32_t sub_len = (cnb + kAttnWarps - 1) / kAttnWarps;
       const uint32_t blk0 = cblk0 + warp * sub_len;
       const uint32_t nb = min(sub_len, cnb - min(cnb, warp * sub_len));
@@ -309,7 +407,8 @@ __global__ void __launch_bounds__(kAttnThreads, (NH == 1 ? 3 : 2)) paged_attn_ke
         }
       __syncthreads();
       // warp w merges heads w, w + 4, ...: lane = four consecutive outputs
-      const bool single = (n_splits == 1);
+      const uint32_t n_parts = n_splits * k_pieces;   // items of this (sequence, KV head)
+      const bool single = (n_parts == 1);
       for (uint32_t r = warp; r < p.group; r += kAttnWarps) {
         const uint32_t hq = g * p.group + r;
         float mw[kAttnWarps], lw[kAttnWarps];
@@ -339,7 +438,7 @@ __global__ void __launch_bounds__(kAttnThreads, (NH == 1 ? 3 : 2)) paged_attn_ke
           ov.y = *reinterpret_cast<const uint32_t*>(&hi);
           *reinterpret_cast<uint2*>(p.out + ((size_t)b * p.Hq + hq) * kD + lane * 4) = ov;
         } else {
-          const size_t slot = ((size_t)b * p.Hq + hq) * p.max_splits + split;
+          const size_t slot = ((size_t)b * p.Hq + hq) * slots_per + split * k_pieces + piece;
           __stcg(reinterpret_cast<float4*>(p.part_o + slot * kD) + lane, acc);
           if (lane == 0) { __stcg(p.part_ml + slot * 2, m_all); __stcg(p.part_ml + slot * 2 + 1, l_all); }
         }
@@ -354,22 +453,22 @@ __global__ void __launch_bounds__(kAttnThreads, (NH == 1 ? 3 : 2)) paged_attn_ke
         }
         __syncthreads();
         ATRACE(4);
-        if (s_old == n_splits - 1) {
+        if (s_old == n_parts - 1) {
           __threadfence();
           for (uint32_t r = warp; r < p.group; r += kAttnWarps) {
             const uint32_t hq = g * p.group + r;
-            const size_t slot0 = ((size_t)b * p.Hq + hq) * p.max_splits;
+            const size_t slot0 = ((size_t)b * p.Hq + hq) * slots_per;
             // lane i looks after the (m, l) pair of runs i, i + 32, ...; the outputs are summed
             // in run order, eight loads in flight at a time
             float m_all = -CUDART_INF_F;
-            for (uint32_t sp = lane; sp < n_splits; sp += 32) m_all = fmaxf(m_all, __ldcg(p.part_ml + (slot0 + sp) * 2));
+            for (uint32_t sp = lane; sp < n_parts; sp += 32) m_all = fmaxf(m_all, __ldcg(p.part_ml + (slot0 + sp) * 2));
 #pragma unroll
             for (int sh = 16; sh >= 1; sh >>= 1) m_all = fmaxf(m_all, __shfl_xor_sync(0xFFFFFFFFu, m_all, sh));
             float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
             float l_all = 0.f;
-            for (uint32_t base = 0; base < n_splits; base += 32) {
+            for (uint32_t base = 0; base < n_parts; base += 32) {
               float f_mine = 0.f, lf = 0.f;
-              if (base + lane < n_splits) {
+              if (base + lane < n_parts) {
                 const float2 ml = __ldcg(reinterpret_cast<const float2*>(p.part_ml + (slot0 + base + lane) * 2));
                 f_mine = (ml.x == -CUDART_INF_F) ? 0.f : exp2f(ml.x - m_all);
                 lf = f_mine * ml.y;
@@ -377,7 +476,7 @@ __global__ void __launch_bounds__(kAttnThreads, (NH == 1 ? 3 : 2)) paged_attn_ke
 #pragma unroll
               for (int sh = 16; sh >= 1; sh >>= 1) lf += __shfl_xor_sync(0xFFFFFFFFu, lf, sh);
               l_all += lf;
-              const uint32_t n_here = min(32u, n_splits - base);
+              const uint32_t n_here = min(32u, n_parts - base);
               for (uint32_t j0 = 0; j0 < n_here; j0 += 8) {
                 float4 v[8];
 #pragma unroll
@@ -458,6 +557,12 @@ int launch_kv_copy(void* flat, uint32_t n_kv_heads, uint32_t n_pool_blocks, uint
   return boosth::check_launch();
 }
 
+// Partial results a (sequence, query head) can have: the shortest runs, each cut in pieces.
+size_t partial_slots(uint32_t max_blocks) {
+  const size_t runs = max_blocks ? (max_blocks + kAttnWarps * kMinItemBlocks - 1) / (kAttnWarps * kMinItemBlocks) : 1;
+  return runs * kTailPieces;
+}
+
 size_t attn_header_bytes(uint32_t B, uint32_t Hkv_upper) {
   return ((size_t)(kWsHeaderWords + (size_t)B * Hkv_upper) * 4 + 255) / 256 * 256;
 }
@@ -483,7 +588,7 @@ extern "C" int boost_kv_gather(void* dst, uint32_t n_kv_heads, uint32_t n_pool_b
 extern "C" size_t boost_paged_attn_workspace_bytes(uint32_t B, uint32_t Hq, uint32_t D,
                                                    uint32_t max_blocks) {
   if (D != kD || B == 0 || Hq == 0) return 0;
-  const size_t max_splits = max_blocks ? (max_blocks + kMinItemBlocks - 1) / kMinItemBlocks : 1;
+  const size_t max_splits = partial_slots(max_blocks);
   // counters are per (b, KV head); Hq bounds the number of KV heads
   return attn_header_bytes(B, Hq) + (size_t)B * Hq * max_splits * (2 + kD) * 4;
 }
@@ -527,28 +632,16 @@ extern "C" int boost_paged_attn_decode_tiered(const void* q, const void* const* 
   const int sms = boosth::sm_count();
   if (sms <= 0) return BOOST_ERR_CUDA;
   const uint32_t ctas_per_sm = p.group <= 8 ? 3 : 2;
-  const uint32_t n_warps = (uint32_t)sms * ctas_per_sm * kAttnWarps;
-  // Run length: an item (four warps, a quarter of the run each) costs a table look-up, a query
-  // load and, when a sequence needs several items, a partial result in global memory, so long
-  // runs are better as long as enough warps have work to keep HBM busy (measured on B200:
-  // about a thousand warps with 16 KiB in flight each saturate it).  Taking the sequences as
-  // max_blocks long, use the longest quarter (4..64 blocks) that still gives 55 % of the
-  // warps work.
-  uint32_t best_len = kMinItemBlocks;
-  for (uint32_t len = kMaxItemBlocks; len >= kMinItemBlocks; --len) {
-    const uint64_t items = (uint64_t)Hkv * B * ((max_blocks + kAttnWarps * len - 1) / (kAttnWarps * len));
-    if (items * kAttnWarps * 100 >= (uint64_t)n_warps * 55) { best_len = len; break; }
-  }
-  p.item_blocks = best_len;
-  p.max_splits = (max_blocks + kAttnWarps * best_len - 1) / (kAttnWarps * best_len);
-  const uint64_t n_items = (uint64_t)Hkv * B * p.max_splits;
-  if (n_items > 0x7FFFFFFFull) return BOOST_ERR_INVALID;
-  p.n_items = (uint32_t)n_items;
+  p.cta_slots = (uint32_t)sms * ctas_per_sm;
+  // every sequence is at least one item per KV head, at most one per kMinItemBlocks-long quarter run
+  const uint64_t max_items = (uint64_t)Hkv * B * partial_slots(max_blocks);
+  if (max_items > 0x7FFFFFFFull) return BOOST_ERR_INVALID;
   p.scale_log2e = scale * 1.4426950408889634f;
   p.ws = static_cast<uint32_t*>(workspace);
   uint8_t* base = static_cast<uint8_t*>(workspace) + attn_header_bytes(B, Hq);
   p.part_ml = reinterpret_cast<float*>(base);
-  p.part_o = p.part_ml + (size_t)B * Hq * p.max_splits * 2;
+  // room for the shortest runs; the kernel indexes with the max_splits of the run length it picks
+  p.part_o = p.part_ml + (size_t)B * Hq * partial_slots(max_blocks) * 2;
   p.out = static_cast<__nv_bfloat16*>(out);
   const size_t smem = (size_t)kAttnWarps * kWarpStages * kStageBytes + 128;
   static bool configured = false;
@@ -559,8 +652,8 @@ extern "C" int boost_paged_attn_decode_tiered(const void* q, const void* const* 
     if (rc != BOOST_OK) return rc;
     configured = true;
   }
-  uint32_t grid = (uint32_t)sms * ctas_per_sm;
-  if (grid > p.n_items) grid = p.n_items;
+  uint32_t grid = p.cta_slots;
+  if (grid > max_items) grid = (uint32_t)max_items;
   if (p.group <= 8)
     return boosth::launch_chained(paged_attn_kernel<1>, dim3(grid), dim3(kAttnThreads), smem, (cudaStream_t)stream, p);
   return boosth::launch_chained(paged_attn_kernel<2>, dim3(grid), dim3(kAttnThreads), smem, (cudaStream_t)stream, p);

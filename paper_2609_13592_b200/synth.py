@@ -91,3 +91,73 @@ def llama_weights(cfg, seed, std=0.02):
             "wd": normal_bf16((hid, ffn), std, b + 5),
         })
     return w
+
+
+def serving_churn_trace(n_blocks, n_steps, arrivals_per_step, max_batch, seed, prompt_lo=64, prompt_hi=1024,
+                        out_median=1500.0, out_sigma=0.8, out_cap=8192, block_tokens=16):
+    """Allocation trace of a continuously batched decode server, one decode step at a time
+    (a stand-in for the paper's serving runs with Poisson arrivals and a long-generation
+    length mix, Sec. 5.9, Sec. 5.10; shapes only, no dataset items).
+
+    Arrivals per step are Poisson; a request has a prompt of U[prompt_lo, prompt_hi] tokens
+    and generates a log-normal number of tokens (median out_median, log-sigma out_sigma,
+    capped).  Waiting requests are admitted first come first served while fewer than
+    max_batch are running and the pool has room for the prompt plus one block per running
+    request; every running request grows by one token per step and needs a new block every
+    block_tokens tokens; a request that cannot grow is dropped (counted).  Admission counts
+    free blocks only, so the trace does not depend on which blocks a pool hands out.
+
+    Yields, per step, (ops, live, stats): ops is the list of ("alloc", request, n_blocks) and
+    ("free", request) calls of the step in order, live maps each running request to its
+    context length after the step (the generator's own dict: read, do not change), stats
+    counts arrivals, admissions, completions and drops so far."""
+    rng = np.random.Generator(np.random.PCG64(seed))
+    free = int(n_blocks)
+    live, left, held = {}, {}, {}
+    waiting = []
+    next_id = 0
+    stats = {"arrived": 0, "admitted": 0, "finished": 0, "dropped": 0}
+
+    def blocks_of(tokens):
+        return -(-tokens // block_tokens)
+
+    for _ in range(n_steps):
+        ops = []
+        for _ in range(int(rng.poisson(arrivals_per_step))):
+            prompt = int(rng.integers(prompt_lo, prompt_hi + 1))
+            out = int(min(out_cap, max(1, round(float(rng.lognormal(np.log(out_median), out_sigma))))))
+            waiting.append((prompt, out))
+            stats["arrived"] += 1
+        # completions of the previous step give their blocks back before anything is handed out
+        for r in [r for r, n in left.items() if n <= 0]:
+            ops.append(("free", r))
+            free += held.pop(r)
+            del live[r], left[r]
+            stats["finished"] += 1
+        # running requests take their next token
+        for r in list(live):
+            if live[r] % block_tokens == 0:
+                if free == 0:
+                    ops.append(("free", r))
+                    free += held.pop(r)
+                    del live[r], left[r]
+                    stats["dropped"] += 1
+                    continue
+                ops.append(("alloc", r, 1))
+                free -= 1
+                held[r] += 1
+            live[r] += 1
+            left[r] -= 1
+        # admissions: the prompt is cached and the first token generated in this step
+        while waiting and len(live) < max_batch:
+            prompt, out = waiting[0]
+            need = blocks_of(prompt + 1)
+            if free < need + len(live):
+                break
+            waiting.pop(0)
+            r, next_id = next_id, next_id + 1
+            ops.append(("alloc", r, need))
+            free -= need
+            held[r], live[r], left[r] = need, prompt + 1, out - 1
+            stats["admitted"] += 1
+        yield ops, live, dict(stats, waiting=len(waiting), free_blocks=free)

@@ -198,3 +198,58 @@ def test_attention_config5_shape_on_sampled_sequences(dev):
     ref = ol.paged_attention_decode(q_bits[sel], k_bits, v_bits, table[sel], ctx[sel].tolist(), scale)
     assert_close_to_oracle(got[sel], ref, "config 5 attention, sampled sequences")
     pool.close()
+
+
+def test_attention_on_a_pool_under_serving_churn(dev):
+    """Four KV heads (eight query heads each), one KV page in twelve on the host, the batch as a
+    pool leaves it after 7000 decode steps of Poisson arrivals with a long-generation length
+    mix at about 80 % utilisation (Sec. 5.10): about 95 sequences of up to 6000 tokens whose
+    blocks are scattered over the pool, so a sequence takes several work items and its
+    partial results meet in global memory.  The library and the oracle pool replay the trace
+    side by side; the oracle computes the longest, the shortest and three more sequences."""
+    from paper_2609_13592_b200 import serving
+    from paper_2609_13592_b200.tiers import TieredKVCache, aligned_workspace
+    hq, hkv, d, n_blocks, modulus = 32, 4, 128, 12 * 1024, 12
+    pool, ref_pool = B.KVPool(n_blocks, hkv, modulus), okp.KVPool(n_blocks, hkv, modulus)
+
+    class Both:
+        def alloc(self, r, n):
+            got = pool.alloc(r, n)
+            assert got.tolist() == ref_pool.alloc(r, n)
+            return got
+
+        def free(self, r):
+            pool.free(r)
+            ref_pool.free_request(r)
+
+        def query(self):
+            return pool.query()
+
+    trace = synth.serving_churn_trace(n_blocks, 7000, 0.045, 96, seed=7)
+    _, _, _, snapshots, _ = serving.replay_churn(Both(), trace, [6999])
+    ctx, table = snapshots[0]["ctx_lens"], snapshots[0]["table"]
+    n_seq, max_blocks = table.shape
+    assert n_seq >= 40 and ctx.max() > 4096 + 64
+    k_bits = synth.normal_bf16((hkv, n_blocks, 16, d), 1.0, 60)
+    v_bits = synth.normal_bf16((hkv, n_blocks, 16, d), 1.0, 61)
+    q_bits = synth.normal_bf16((n_seq, hq, d), 1.0, 62)
+    cache = TieredKVCache(pool, hkv, n_blocks, d, dev)
+    assert cache.tier.tolist() == ref_pool.page_tiers() and int((cache.tier == 1).sum()) * 12 == cache.tier.size
+    cache.load(bf16_tensor(k_bits, dev), bf16_tensor(v_bits, dev))
+    ws_bytes = B.boost_paged_attn_workspace_bytes(n_seq, hq, d, max_blocks)
+    ws_t, ws = aligned_workspace(ws_bytes, dev)
+    out = torch.full((n_seq, hq, d), float("nan"), dtype=torch.bfloat16, device=dev)
+    scale = 1.0 / math.sqrt(d)
+    B.boost_paged_attn_decode_tiered(bf16_tensor(q_bits, dev), cache.k.page_ptr, cache.v.page_ptr, cache.tier,
+                                     cache.n_pages, n_blocks, torch.from_numpy(table).to(dev), max_blocks,
+                                     torch.from_numpy(ctx).to(dev), n_seq, hq, hkv, d, scale, ws, ws_bytes, out)
+    torch.cuda.synchronize()
+    got = out.float().cpu().numpy()
+    assert np.isfinite(got).all()
+    off = ws - ws_t.data_ptr()
+    assert int(ws_t[off:off + 4].cpu().numpy().view(np.uint32)[0]) == 0     # status word
+    sel = sorted({int(np.argmax(ctx)), int(np.argmin(ctx)),
+                  *np.random.default_rng(9).choice(n_seq, size=3, replace=False).tolist()})
+    ref = ol.paged_attention_decode(q_bits[sel], k_bits, v_bits, table[sel], ctx[sel].tolist(), scale)
+    assert_close_to_oracle(got[sel], ref, "attention on a churned pool, sampled sequences")
+    pool.close()

@@ -199,6 +199,38 @@ def test_pool_traces_bit_exact(geom):
     pool.close()
 
 
+def test_pool_under_serving_churn_bit_exact_and_near_target():
+    # Sec. 5.10: four KV heads, one page in twelve on the host, Poisson arrivals with a
+    # long-generation length mix at about 80 % pool utilisation.  The library hands out the
+    # same blocks as the oracle throughout, and the realised host share of the live KV
+    # chunks stays within a point of the target, far below the 1/H granularity bound.
+    from paper_2609_13592_b200 import synth
+    n, h, m = 12 * 1024, 4, 12
+    pool, ref = B.KVPool(n, h, m), okp.KVPool(n, h, m)
+    shares = []
+    for step, (ops, live, stats) in enumerate(synth.serving_churn_trace(n, 5000, 0.045, 96, seed=7)):
+        for op in ops:
+            if op[0] == "alloc":
+                assert pool.alloc(op[1], op[2]).tolist() == ref.alloc(op[1], op[2])
+            else:
+                pool.free(op[1])
+                ref.free_request(op[1])
+        q = pool.query()
+        assert q["n_requests"] == len(live)
+        assert q["live_blocks"] == sum(-(-c // 16) for c in live.values()) == n - stats["free_blocks"]
+        if step % 100 == 0:
+            same_state(pool, ref)
+        if step >= 2500:
+            shares.append(q["live_host_chunks"] / q["live_chunks"])
+    same_state(pool, ref)
+    assert stats["admitted"] > 150 and stats["finished"] > 100
+    window = 500
+    medians = [float(np.median(shares[i:i + window])) for i in range(0, len(shares) - window, 50)]
+    assert max(abs(x - 1.0 / m) for x in medians) < 0.01
+    assert max(shares) < 0.5 / h
+    pool.close()
+
+
 def test_pool_bad_geometry():
     for args in ((500, 8, 8), (0, 8, 8), (512, 0, 8), (512, 8, 1)):
         with pytest.raises(B.BoostError) as e:
