@@ -383,7 +383,11 @@ __global__ void __launch_bounds__(kAttnThreads, (NH == 1 ? 3 : 2)) paged_attn_ke
 #pragma unroll
             for (int t = 2; t >= 0; --t) mma_bf16_16816(o[nh][dt], a, pa[nh][t][0], pa[nh][t][1]);
         }
-        __syncwarp();   // every lane is done with this stage before it is refilled
+        // Every lane is done with this stage before it is refilled, and its loads have been
+        // performed: they went through the generic proxy, the refill is a bulk copy through the
+        // async proxy, which nothing else keeps behind loads still in flight.
+        __threadfence_block();
+        __syncwarp();
         if (i + kWarpStages < nb) request(i + kWarpStages);
       }
 
@@ -501,9 +505,10 @@ __global__ void __launch_bounds__(kAttnThreads, (NH == 1 ? 3 : 2)) paged_attn_ke
           ATRACE(5);
         }
       }
-      // the ring is written by bulk copies again: order the parked values' reads and writes before them
-      __syncthreads();
+      // the ring is written by bulk copies again: every thread orders its reads and writes of the
+      // parked values before them (proxy fence), then all meet
       fence_proxy_async_smem();
+      __syncthreads();
     } else if (!waited) {
       pdl_wait();   // keep every thread's first pass through the dependency wait
       waited = true;

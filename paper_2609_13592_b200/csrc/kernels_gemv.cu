@@ -605,6 +605,14 @@ __global__ void __launch_bounds__(kGemvThreads, (NT >= 8 ? 1 : 2)) gemv_tiered_k
         }
       }
     }
+    // Every read of the stage must have been performed before the stage is released: the loads
+    // went through the generic proxy, the refill is a bulk copy through the async proxy, and the
+    // release alone does not keep the refill behind loads that are still in flight (the MMAs
+    // that use them may be scheduled after it).  Seen on B200 as torn weight rows in one launch
+    // in four when threadblocks have an SM to themselves and the producer reacts at once.  A
+    // CTA-scope fence in every reading thread closes it (1.3 % of the step; fence.proxy.async in
+    // the same place also does, at 2.4 %).
+    __threadfence_block();
     __syncwarp();
     if (lane == 0) mbar_arrive(&empty_bar[stage]);
     if (++stage == n_stages) { stage = 0; phase ^= 1u; }

@@ -253,3 +253,32 @@ def test_attention_on_a_pool_under_serving_churn(dev):
     ref = ol.paged_attention_decode(q_bits[sel], k_bits, v_bits, table[sel], ctx[sel].tolist(), scale)
     assert_close_to_oracle(got[sel], ref, "attention on a churned pool, sampled sequences")
     pool.close()
+
+
+def test_attention_repeated_launches_are_identical(dev):
+    """100 launches of configuration 2's attention give the same bits (ring stages are refilled
+    by bulk copies right after they are read)."""
+    from paper_2609_13592_b200.tiers import TieredKVCache, aligned_workspace
+    n_seq, hq, hkv, d, n_blocks = 8, 32, 8, 128, 2560
+    ctx = synth.ctx_lens_uniform(n_seq, 512, 4096, seed=2).tolist()
+    for modulus in (0, 8):
+        pool, ref_pool = B.KVPool(n_blocks, hkv, modulus), okp.KVPool(n_blocks, hkv, modulus)
+        table = build_tables(pool, ref_pool, ctx, churn=False)
+        cache = TieredKVCache(pool, hkv, n_blocks, d, dev)
+        cache.load(bf16_tensor(synth.normal_bf16((hkv, n_blocks, 16, d), 1.0, 80), dev),
+                   bf16_tensor(synth.normal_bf16((hkv, n_blocks, 16, d), 1.0, 81), dev))
+        q = bf16_tensor(synth.normal_bf16((n_seq, hq, d), 1.0, 82), dev)
+        max_blocks = table.shape[1]
+        ws_bytes = B.boost_paged_attn_workspace_bytes(n_seq, hq, d, max_blocks)
+        ws_t, ws = aligned_workspace(ws_bytes, dev)
+        table_d = torch.from_numpy(table).to(dev)
+        ctx_d = torch.tensor(ctx, dtype=torch.int32, device=dev)
+        outs = []
+        for _ in range(101):
+            out = torch.empty((n_seq, hq, d), dtype=torch.bfloat16, device=dev)
+            B.boost_paged_attn_decode_tiered(q, cache.k.page_ptr, cache.v.page_ptr, cache.tier, cache.n_pages, n_blocks,
+                                             table_d, max_blocks, ctx_d, n_seq, hq, hkv, d, 1.0 / math.sqrt(d), ws, ws_bytes, out)
+            torch.cuda.synchronize()
+            outs.append(out)
+        assert all(torch.equal(o, outs[0]) for o in outs[1:])
+        pool.close()

@@ -225,3 +225,26 @@ def test_gemv_full_size_batch128(dev, ratio):
     assert w.buf.n_host == (0 if ratio == 0 else w.buf.n_pages // 64)
     assert_close_to_oracle(y, ref, f"28672 x 4096, batch 128, host ratio {ratio}", floor_rms=2e-3)
     assert w.status_words() == [0]
+
+
+@pytest.mark.parametrize("n,k,m_b,ratio", [(4096, 14336, 32, 0.125), (4096, 14336, 32, 0.0), (6144, 4096, 8, 1 / 16)])
+def test_gemv_repeated_launches_are_identical(dev, n, k, m_b, ratio):
+    """150 launches on the same inputs give the same bits.  With host pages the grid is 224
+    threadblocks on 148 SMs, so some have an SM to themselves and their producer refills a ring
+    stage the moment it is released: this is the case that showed torn weight rows before the
+    consumers fenced their generic-proxy reads against the async-proxy refill."""
+    from paper_2609_13592_b200.tiers import TieredWeight
+    w_bits = synth.normal_bf16((n, k), 0.02, 70)
+    x_bits = synth.normal_bf16((m_b, k), 1.0, 71)
+    w = TieredWeight(bf16_tensor(w_bits, dev), ratio, device=dev)
+    x = bf16_tensor(x_bits, dev)
+    first = w.gemv(x).clone()
+    torch.cuda.synchronize()
+    assert_close_to_oracle(first.float().cpu().numpy(), ol.gemm(x_bits, w_bits), f"gemv {n}x{k} m_b={m_b}")
+    differing = 0
+    for _ in range(150):
+        y = w.gemv(x)
+        torch.cuda.synchronize()
+        differing += int(not torch.equal(y, first))
+    assert differing == 0
+    assert w.status_words() == [0]
