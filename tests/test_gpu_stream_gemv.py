@@ -227,7 +227,8 @@ def test_gemv_full_size_batch128(dev, ratio):
     assert w.status_words() == [0]
 
 
-@pytest.mark.parametrize("n,k,m_b,ratio", [(4096, 14336, 32, 0.125), (4096, 14336, 32, 0.0), (6144, 4096, 8, 1 / 16)])
+@pytest.mark.parametrize("n,k,m_b,ratio", [(4096, 14336, 32, 0.125), (4096, 14336, 32, 0.0), (6144, 4096, 8, 1 / 16),
+                                           (4096, 14336, 2, 0.125), (4096, 14336, 64, 0.125), (4096, 14336, 128, 0.0)])
 def test_gemv_repeated_launches_are_identical(dev, n, k, m_b, ratio):
     """150 launches on the same inputs give the same bits.  With host pages the grid is 224
     threadblocks on 148 SMs, so some have an SM to themselves and their producer refills a ring
