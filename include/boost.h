@@ -410,7 +410,10 @@ int boost_kv_gather(void* dst /*device*/, uint32_t n_kv_heads, uint32_t n_pool_b
  *                just before it on the stream when that kernel is one of this library's
  *                (which write neither); the newest K / V rows and q are read after it;
  *   out          device bf16 [B, Hq, D];
- *   workspace    device, >= boost_paged_attn_workspace_bytes(B, Hq, D, max_blocks). */
+ *   workspace    device, >= boost_paged_attn_workspace_bytes(B, Hq, D, max_blocks); its first
+ *                word collects error bits (1 = a bounded wait gave up, 2 = a block index
+ *                outside the pool or a context length outside [0, 16 * max_blocks]: such a
+ *                block is read as block 0, such a length is clamped) and is 0 after a clean run. */
 size_t boost_paged_attn_workspace_bytes(uint32_t B, uint32_t Hq, uint32_t D, uint32_t max_blocks);
 int boost_paged_attn_decode_tiered(const void* q /*device*/, const void* const* k_page_ptr /*device*/,
                                    const void* const* v_page_ptr /*device*/,

@@ -71,6 +71,12 @@ struct AttnParams {
   __nv_bfloat16* out;
 };
 
+// Cached tokens of sequence b, kept inside what its row of the block table can describe (a
+// length outside it is recorded in the status word where the sequence's items are processed).
+__device__ __forceinline__ uint32_t seq_len(const AttnParams& p, uint32_t b) {
+  return min((uint32_t)max(p.ctx_lens[b], 0), p.max_blocks * kTok);
+}
+
 __device__ __forceinline__ uint32_t movmatrix_trans(uint32_t a) {
   uint32_t d;
   asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(d) : "r"(a));
@@ -121,7 +127,7 @@ __global__ void __launch_bounds__(kAttnThreads, (NH == 1 ? 3 : 2)) paged_attn_ke
   // and runs of at most u give every slot a few items to even out through the queue.
   uint32_t my_blocks = 0, my_max = 0;
   for (uint32_t b = tid; b < p.B; b += kAttnThreads) {
-    const uint32_t n = ((uint32_t)max(p.ctx_lens[b], 0) + kTok - 1) / kTok;
+    const uint32_t n = (seq_len(p, b) + kTok - 1) / kTok;
     my_blocks += n;
     my_max = max(my_max, n);
   }
@@ -151,7 +157,7 @@ __global__ void __launch_bounds__(kAttnThreads, (NH == 1 ? 3 : 2)) paged_attn_ke
     uint32_t carry = 0;
     for (uint32_t b0 = 0; b0 < p.B; b0 += kAttnThreads) {
       const uint32_t b = b0 + tid;
-      const uint32_t n_blk = b < p.B ? ((uint32_t)max(p.ctx_lens[b], 0) + kTok - 1) / kTok : 0;
+      const uint32_t n_blk = b < p.B ? (seq_len(p, b) + kTok - 1) / kTok : 0;
       const uint32_t mine = b < p.B ? (n_blk ? (n_blk + cta_max - 1) / cta_max : 1u) : 0u;
       uint32_t incl = mine;
 #pragma unroll
@@ -204,7 +210,8 @@ __global__ void __launch_bounds__(kAttnThreads, (NH == 1 ? 3 : 2)) paged_attn_ke
       b = in_head / max_splits;
       split = in_head % max_splits;
     }
-    const uint32_t ctx = (uint32_t)max(p.ctx_lens[b], 0);
+    if (tid == 0 && (p.ctx_lens[b] < 0 || (uint32_t)p.ctx_lens[b] > p.max_blocks * kTok)) atomicOr(status, kErrBadIndex);
+    const uint32_t ctx = seq_len(p, b);
     const uint32_t n_blk = (ctx + kTok - 1) / kTok;
     const uint32_t n_splits = n_blk ? (n_blk + cta_max - 1) / cta_max : 1;
     if (split < n_splits) {

@@ -282,3 +282,31 @@ def test_attention_repeated_launches_are_identical(dev):
             outs.append(out)
         assert all(torch.equal(o, outs[0]) for o in outs[1:])
         pool.close()
+
+
+def test_attention_context_length_outside_the_table_is_clamped_and_flagged(dev):
+    """A context length beyond what the block table's row describes does not read past the row:
+    the sequence is processed up to 16 * max_blocks tokens and bit 2 of the status word is set."""
+    from paper_2609_13592_b200.tiers import TieredKVCache, aligned_workspace
+    n_seq, hq, hkv, d, n_blocks, max_blocks = 2, 8, 2, 128, 512, 8
+    pool = B.KVPool(n_blocks, hkv, 0)
+    table = np.stack([pool.alloc(b, max_blocks) for b in range(n_seq)]).astype(np.int32)
+    k_bits = synth.normal_bf16((hkv, n_blocks, 16, d), 1.0, 90)
+    v_bits = synth.normal_bf16((hkv, n_blocks, 16, d), 1.0, 91)
+    q_bits = synth.normal_bf16((n_seq, hq, d), 1.0, 92)
+    cache = TieredKVCache(pool, hkv, n_blocks, d, dev)
+    cache.load(bf16_tensor(k_bits, dev), bf16_tensor(v_bits, dev))
+    ws_bytes = B.boost_paged_attn_workspace_bytes(n_seq, hq, d, max_blocks)
+    ws_t, ws = aligned_workspace(ws_bytes, dev)
+    out = torch.empty((n_seq, hq, d), dtype=torch.bfloat16, device=dev)
+    ctx = np.array([100, 5000], dtype=np.int32)          # the second one is far beyond 8 blocks
+    scale = 1.0 / math.sqrt(d)
+    B.boost_paged_attn_decode_tiered(bf16_tensor(q_bits, dev), cache.k.page_ptr, cache.v.page_ptr, cache.tier, cache.n_pages,
+                                     n_blocks, torch.from_numpy(table).to(dev), max_blocks, torch.from_numpy(ctx).to(dev),
+                                     n_seq, hq, hkv, d, scale, ws, ws_bytes, out)
+    torch.cuda.synchronize()
+    off = ws - ws_t.data_ptr()
+    assert int(ws_t[off:off + 4].cpu().numpy().view(np.uint32)[0]) == 2
+    ref = ol.paged_attention_decode(q_bits, k_bits, v_bits, table, [100, 16 * max_blocks], scale)
+    assert_close_to_oracle(out.float().cpu().numpy(), ref, "attention with a clamped context length")
+    pool.close()
