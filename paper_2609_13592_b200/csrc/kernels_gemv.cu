@@ -92,6 +92,17 @@ struct GemvParams {
   uint32_t tiles_per_unit;   // tcgen05 kernel, even partition: 1, or 2 = adjacent row tiles share an activation tile
 };
 
+// Counter updates that publish this threadblock's earlier writes (release) and, where the old
+// value decides who reads the others' writes, also order those reads after it (acquire).
+__device__ __forceinline__ uint32_t atom_add_acq_rel(uint32_t* p, uint32_t v) {
+  uint32_t old;
+  asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], %2;" : "=r"(old) : "l"(p), "r"(v) : "memory");
+  return old;
+}
+__device__ __forceinline__ void red_add_release(uint32_t* p, uint32_t v) {
+  asm volatile("red.release.gpu.global.add.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+
 // First / last threadblock of the even partition that holds a block of row tile `t`.
 __device__ __forceinline__ uint32_t part_owner(uint64_t block, uint32_t G, uint32_t T) {
   return (uint32_t)(((block + 1) * G - 1) / T);
@@ -532,10 +543,10 @@ __global__ void __launch_bounds__(kGemvThreads, (NT >= 8 ? 1 : 2)) gemv_tiered_k
         // them and tell the grid (the x warps of all threadblocks wait for the count)
         named_barrier_sync(1, kConsumerThreads);
         if (tid == 0) {
-          __threadfence();
           if (mt.z & kFlagPhaseEnd) {
-            atomicAdd(cp.bar + mt.w, 1u);
+            red_add_release(cp.bar + mt.w, 1u);
           } else {
+            __threadfence();
             // last threadblock out puts the counters back to zero for the next launch; by then
             // every x warp has passed every phase boundary (its stop stage came after them)
             const uint32_t old = atomicAdd(cp.bar + kMaxPhases, 1u);
@@ -679,8 +690,9 @@ __global__ void __launch_bounds__(kGemvThreads, (NT >= 8 ? 1 : 2)) gemv_tiered_k
         // split order (fixed order: deterministic) and writes the output
         named_barrier_sync(1, kConsumerThreads);
         if (tid == 0) {
-          __threadfence();   // cumulative: publishes the partials of all consumer threads (ordered by the barrier)
-          s_old = atomicAdd(tile_cnt + row_tile, 1u);
+          // release: publishes the partials of all consumer threads (ordered by the barrier);
+          // acquire: the last to arrive reads the others' partials after this
+          s_old = atom_add_acq_rel(tile_cnt + row_tile, 1u);
         }
         named_barrier_sync(1, kConsumerThreads);
         if (s_old == n_seg - 1) {
@@ -978,10 +990,10 @@ __global__ void __launch_bounds__(kTcThreads, 1) gemv_tc_kernel(const __grid_con
       if (n_phases > 1) {
         named_barrier_sync(1, kTcEpiThreads);
         if (tid == 0) {
-          __threadfence();
           if (mt.z & kFlagPhaseEnd) {
-            atomicAdd(cp.bar + mt.w, 1u);
+            red_add_release(cp.bar + mt.w, 1u);
           } else {
+            __threadfence();
             const uint32_t old = atomicAdd(cp.bar + kMaxPhases, 1u);
             if (old == gridDim.x - 1) {
               for (uint32_t i = 0; i <= kMaxPhases; ++i) cp.bar[i] = 0u;
@@ -1042,10 +1054,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) gemv_tc_kernel(const __grid_con
       for (uint32_t ti = 0; ti < n_tiles; ++ti) {
         const uint32_t row_tile = mt.x + ti;
         named_barrier_sync(1, kTcEpiThreads);
-        if (tid == 0) {
-          __threadfence();
-          s_old = atomicAdd(tile_cnt + row_tile, 1u);
-        }
+        if (tid == 0) s_old = atom_add_acq_rel(tile_cnt + row_tile, 1u);   // release the partial sums, acquire the others'
         named_barrier_sync(1, kTcEpiThreads);
         if (s_old == n_seg - 1) {
           __threadfence();
