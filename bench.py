@@ -867,7 +867,7 @@ def main():
                          "configurations 1 - 3")
     ap.add_argument("--churn-steps", type=int, default=12000, help="pool_churn: decode steps replayed")
     ap.add_argument("--sweep-gib", default="1,4,16")
-    ap.add_argument("--sweep-seeds", type=int, default=5)
+    ap.add_argument("--sweep-seeds", type=int, default=20)
     ap.add_argument("--sweep-ratios", default="", help="stream_sweep: comma-separated host shares (default: the full list)")
     ap.add_argument("--sweep-policies", default="", help="stream_sweep: subset of modulo,contiguous,random")
     args = ap.parse_args()
