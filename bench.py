@@ -173,7 +173,8 @@ def run_reference(args, rank, world):
 
 
 def run_reference_configs(args):
-    """The CPU oracle, as it stands, timed on configurations 1 - 3 on this machine's host cores: with
+    """The CPU oracle, as it stands, timed on configurations 1 - 3 and on a sample of configuration 5
+    (one layer's attention for 8 of its 128 sequences) on this machine's host cores: with
     one thread and with all of them (the BLAS calls inside numpy are what threads).  One JSON
     document; the decode-step sample of configuration 4 is the default `--impl reference` line."""
     from oracle import kv_pool as okp
@@ -203,7 +204,20 @@ def run_reference_configs(args):
         fn()
         return time.perf_counter() - t0
 
+    # configuration 5, sampled: the attention of one layer for 8 of the 128 sequences (context lengths
+    # uniform in [2048, 4096], seed 5) through a pool with one page in five on the host
+    ctx5 = synth.ctx_lens_uniform(128, 2048, 4096, seed=5)[:8].tolist()
+    pool5 = okp.KVPool(2560, 8, 5, 16 * 128 * 2)
+    table5 = np.zeros((8, 256), np.int64)
+    for j in range(256):
+        for b, c in enumerate(ctx5):
+            if j < (c + 15) // 16:
+                table5[b, j] = pool5.alloc(b, 1)[0]
+    k5, v5 = synth.normal_bf16((8, 2560, 16, 128), 1.0, 50), synth.normal_bf16((8, 2560, 16, 128), 1.0, 51)
+    q5 = synth.normal_bf16((8, 32, 128), 1.0, 52)
     cases = {
+        "c5_sample_attention_of_one_layer_8_of_128_sequences_ctx2048_4096": lambda: ol.paged_attention_decode(
+            q5, k5, v5, table5, ctx5, 1.0 / np.sqrt(128.0)),
         "c1_place_pages_and_gemv_4096x4096_batch1": lambda: (op.place_pages(4096 * 4096 * 2, 1 / 16), ol.gemm(x1, w1)),
         "c2_attention_batch8_ctx512_4096": lambda: ol.paged_attention_decode(q2, k2, v2, table, ctx2, 1.0 / np.sqrt(128.0)),
         "c3_stream_sum_1gib": lambda: ol.stream_sum(buf3, page_elems),
@@ -215,7 +229,7 @@ def run_reference_configs(args):
             with threadpool_limits(limits=1):
                 row["one_thread_s"] = timed(fn)
         out[name] = row
-    print(json.dumps({"impl": "reference", "workload": "oracle_on_configs_1_to_3", "cores": os.cpu_count(),
+    print(json.dumps({"impl": "reference", "workload": "oracle_on_configs_1_to_3_and_a_sample_of_5", "cores": os.cpu_count(),
                       "seconds": out}), flush=True)
 
 
