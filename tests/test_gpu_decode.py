@@ -132,8 +132,9 @@ def dump_cache(dev, dec, li, name):
     return bits_of(t)
 
 
-@pytest.mark.parametrize("n_seq,kv_modulus,weight_ratio", [(3, 4, 0.5), (1, 0, 0.0), (20, 2, 0.25), (40, 4, 0.25)])
-def test_decode_steps_match_oracle(dev, n_seq, kv_modulus, weight_ratio):
+@pytest.mark.parametrize("n_seq,kv_modulus,weight_ratio,recycle", [(3, 4, 0.5, False), (1, 0, 0.0, False), (20, 2, 0.25, False),
+                                                                    (40, 4, 0.25, False), (6, 4, 0.5, True)])
+def test_decode_steps_match_oracle(dev, n_seq, kv_modulus, weight_ratio, recycle):
     from tests.helpers import chain_error
     cfg = dict(synth.TINY_LLAMA)
     w = synth.llama_weights(cfg, seed=n_seq, std=0.02)
@@ -160,6 +161,16 @@ def test_decode_steps_match_oracle(dev, n_seq, kv_modulus, weight_ratio):
         # both sides start every step from the same cache, so that a bf16 rounding that fell
         # differently in an earlier step does not carry over
         load_caches(dev, dec, k_host, v_host)
+        if recycle and step in (5, 9, 12):
+            # a sequence ends and a new one takes its place in the batch: its blocks go back to the
+            # pool (both sides) and the newcomer starts from an empty context on whatever the pool
+            # hands out next
+            gone = step % n_seq
+            dec.pool.free(gone)
+            ref_pool.free_request(gone)
+            ctx[gone], n_have[gone] = 0, 0
+            table[gone, :] = 0
+            tokens[gone] = (37 * step) % cfg["vocab"]
         ctx += 1                                           # the new token joins the context
         for b in range(n_seq):                             # blocks through the pool, both sides
             while n_have[b] * 16 < ctx[b]:
