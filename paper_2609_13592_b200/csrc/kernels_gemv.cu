@@ -733,6 +733,7 @@ template <uint32_t NPAD>
 __global__ void __launch_bounds__(kTcThreads, 1) gemv_tc_kernel(const __grid_constant__ ChainParams cp) {
   constexpr uint32_t kStageBytes = tc_stage_bytes(NPAD);
   constexpr uint32_t kTmemCols = 4 * NPAD < 32 ? 32 : 4 * NPAD;   // two accumulators (a pair of row tiles), double-buffered
+  if (threadIdx.x == 0) TRACE(0);
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   __shared__ uint64_t full_bar[kMaxStages];
@@ -794,6 +795,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) gemv_tc_kernel(const __grid_con
         if (lane == 0) grid_counter_wait(cp.bar + (ph - 1), gridDim.x, status);
         __syncwarp();
       }
+      if (warp == kTcEpiWarps + 2) TRACE(8 + 8 * ph + 2);
       // one block: the weight warp copies it, the activation warp stages x[:, 64 kb .. 64 kb + 64)
       // as NPAD rows of 128 bytes in the 128-byte swizzle (rows >= M_b are zero)
       // one stage: the weight warp copies the weight block (two blocks in pair mode), the
@@ -944,6 +946,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) gemv_tc_kernel(const __grid_con
           if (!mbar_wait(&acc_empty[buf], buf_phase ^ 1u, status)) { s_abort = 1; break; }   // the epilogue has read this accumulator
           accumulate = 0;
         }
+        TRACE_ONCE(8 + 8 * mt.w + 3);
         fence_proxy_async_smem();   // x (and host-tier weight blocks) were written through the load/store path
         tc_fence_after_sync();
         const uint32_t wbase = smem_u32(smem + (size_t)stage * kStageBytes);
@@ -987,6 +990,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) gemv_tc_kernel(const __grid_con
     if (!s_go[buf]) break;
     const uint4 mt = acc_meta[buf];
     if (mt.z & (kFlagStop | kFlagPhaseEnd)) {
+      if (warp == 0) TRACE(8 + 8 * mt.w + 4);
       if (n_phases > 1) {
         named_barrier_sync(1, kTcEpiThreads);
         if (tid == 0) {
@@ -1009,6 +1013,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) gemv_tc_kernel(const __grid_con
       continue;
     }
     tc_fence_after_sync();
+    if (warp == 0) TRACE(8 + 8 * mt.w + 6);
     const GemvParams& p = cp.ph[mt.w];
     const uint32_t split = mt.y;
     const uint32_t n_tiles = (mt.z & kFlagSecond) ? 2u : 1u;   // row tiles in this accumulator
@@ -1060,6 +1065,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) gemv_tc_kernel(const __grid_con
           __threadfence();
           combine_tile<NPAD, kTcEpiThreads>(p, row_tile, n_seg, tid, status);
           if (tid == 0) tile_cnt[row_tile] = 0;
+          if (warp == 0) TRACE(8 + 8 * mt.w + 5);
         }
         named_barrier_sync(1, kTcEpiThreads);
       }
