@@ -141,6 +141,128 @@ __device__ __forceinline__ uint2 pack4_bf16(float a, float b, float c, float d) 
 }
 __device__ __forceinline__ float round_bf16(float v) { return __bfloat162float(__float2bfloat16_rn(v)); }
 
+// Second half of a combine pass for one thread: its sums (lo = columns [4 v, 4 v + 4) of batch row m,
+// hi = their partners 64 columns on) are scaled by the row statistics, paired up and stored as the
+// epilogue of the product says (see combine_tile).  Called by whole warps: it shuffles.
+template <uint32_t kXRows>
+__device__ __forceinline__ void finish_pair(const GemvParams& p, uint32_t row_tile, uint32_t m, uint32_t v, bool valid,
+                                            float4 lo, float4 hi, float ss, float ss0, float ss1, const uint2 (&res)[2],
+                                            bool vec_out, uint32_t* status) {
+  if (p.ssq_in) {
+    ss += ss0 + ss1;
+    ss += __shfl_xor_sync(0xFFFFFFFFu, ss, 1);
+    ss += __shfl_xor_sync(0xFFFFFFFFu, ss, 2);
+    ss += __shfl_xor_sync(0xFFFFFFFFu, ss, 4);
+    ss += __shfl_xor_sync(0xFFFFFFFFu, ss, 8);
+    const float rs = rsqrtf(ss / (float)p.x_cols + p.rms_eps);
+    lo.x *= rs; lo.y *= rs; lo.z *= rs; lo.w *= rs;
+    hi.x *= rs; hi.y *= rs; hi.z *= rs; hi.w *= rs;
+  }
+  if (p.epi == kEpiPlain) {
+    float sq = 0.f;
+    if (valid) {
+      const float4 val[2] = {lo, hi};
+#pragma unroll
+      for (int half = 0; half < 2; ++half) {
+        const uint32_t n = row_tile * kBlockRows + half * 64 + v * 4;
+        float e[4] = {val[half].x, val[half].y, val[half].z, val[half].w};
+        if (n + 3 < p.N && vec_out) {
+          const size_t idx = (size_t)m * p.N + n;
+          if (p.residual) {
+            const uint2 r = res[half];
+            e[0] += bf16_lo(r.x); e[1] += bf16_hi(r.x); e[2] += bf16_lo(r.y); e[3] += bf16_hi(r.y);
+          }
+          if (p.y_dtype == 0) {
+            *reinterpret_cast<float4*>(static_cast<float*>(p.y) + idx) = make_float4(e[0], e[1], e[2], e[3]);
+          } else {
+            *reinterpret_cast<uint2*>(static_cast<__nv_bfloat16*>(p.y) + idx) = pack4_bf16(e[0], e[1], e[2], e[3]);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) { const float b = round_bf16(e[j]); sq = fmaf(b, b, sq); }
+          }
+        } else {
+#pragma unroll
+          for (int j = 0; j < 4; ++j)
+            if (n + j < p.N) {
+              float x = e[j];
+              if (p.residual) x += bf16_lo((uint32_t)__ldcg(reinterpret_cast<const unsigned short*>(p.residual) + (size_t)m * p.N + n + j));
+              if (p.y_dtype == 0) static_cast<float*>(p.y)[(size_t)m * p.N + n + j] = x;
+              else {
+                static_cast<__nv_bfloat16*>(p.y)[(size_t)m * p.N + n + j] = __float2bfloat16_rn(x);
+                const float b = round_bf16(x);
+                sq = fmaf(b, b, sq);
+              }
+            }
+        }
+      }
+    }
+    if (p.ssq_out) {   // sum over the 16 threads that share row m (a fixed butterfly order)
+      sq += __shfl_xor_sync(0xFFFFFFFFu, sq, 1);
+      sq += __shfl_xor_sync(0xFFFFFFFFu, sq, 2);
+      sq += __shfl_xor_sync(0xFFFFFFFFu, sq, 4);
+      sq += __shfl_xor_sync(0xFFFFFFFFu, sq, 8);
+      if (valid && v == 0) p.ssq_out[(size_t)row_tile * p.ssq_stride + m] = sq;
+    }
+  } else if (p.epi == kEpiSwiglu) {
+    if (valid) {
+      const float g[4] = {round_bf16(lo.x), round_bf16(lo.y), round_bf16(lo.z), round_bf16(lo.w)};
+      const float u[4] = {round_bf16(hi.x), round_bf16(hi.y), round_bf16(hi.z), round_bf16(hi.w)};
+      float a[4];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) a[j] = g[j] / (1.f + expf(-g[j])) * u[j];
+      const size_t idx = (size_t)m * (p.N / 2) + row_tile * 64 + v * 4;
+      *reinterpret_cast<uint2*>(static_cast<__nv_bfloat16*>(p.y) + idx) = pack4_bf16(a[0], a[1], a[2], a[3]);
+    }
+  } else {   // kEpiRope
+    const int32_t ctx = valid ? p.ctx_lens[m] : 0;
+    if (valid && ctx > 0) {
+      const uint32_t pos = (uint32_t)ctx - 1u;
+      const uint32_t head = row_tile;
+      float x1[4] = {round_bf16(lo.x), round_bf16(lo.y), round_bf16(lo.z), round_bf16(lo.w)};
+      float x2[4] = {round_bf16(hi.x), round_bf16(hi.y), round_bf16(hi.z), round_bf16(hi.w)};
+      if (head < p.Hq + p.Hkv) {
+        // cos / sin of position * base^(-2i/128) for i = 4v .. 4v+3, from the step's table
+        const float4 cs01 = __ldg(reinterpret_cast<const float4*>(p.rope_table + ((size_t)m * 64 + v * 4) * 2));
+        const float4 cs23 = __ldg(reinterpret_cast<const float4*>(p.rope_table + ((size_t)m * 64 + v * 4 + 2) * 2));
+        const float cs[4] = {cs01.x, cs01.z, cs23.x, cs23.z}, sn[4] = {cs01.y, cs01.w, cs23.y, cs23.w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const float y1 = x1[j] * cs[j] - x2[j] * sn[j];
+          const float y2 = x2[j] * cs[j] + x1[j] * sn[j];
+          x1[j] = y1; x2[j] = y2;
+        }
+      }
+      const uint2 o1 = pack4_bf16(x1[0], x1[1], x1[2], x1[3]), o2 = pack4_bf16(x2[0], x2[1], x2[2], x2[3]);
+      const uint32_t d = v * 4;
+      if (head < p.Hq) {
+        __nv_bfloat16* dst = p.q_out + ((size_t)m * p.Hq + head) * kBlockRows;
+        *reinterpret_cast<uint2*>(dst + d) = o1;
+        *reinterpret_cast<uint2*>(dst + d + 64) = o2;
+      } else {
+        const bool is_k = head < p.Hq + p.Hkv;
+        const uint32_t kvh = is_k ? head - p.Hq : head - p.Hq - p.Hkv;
+        const uint32_t bi = pos / BOOST_KV_BLOCK_TOKENS, slot = pos % BOOST_KV_BLOCK_TOKENS;
+        const int32_t blk = bi < p.max_blocks ? p.block_table[(size_t)m * p.max_blocks + bi] : -1;
+        if (blk < 0 || (uint32_t)blk >= p.n_pool_blocks) {
+          atomicOr(status, kErrBadIndex);
+        } else {
+          const void* const* pages = is_k ? p.k_page_ptr : p.v_page_ptr;
+          // chunk (kvh, blk): token `slot` at slot*256, 16-byte piece c at position c ^ (slot & 7)
+          const size_t chunk = ((size_t)kvh * p.n_pool_blocks + (uint32_t)blk) * 4096u + slot * 256u;
+          const size_t off1 = chunk + ((((d >> 3) ^ (slot & 7u))) << 4) + (d & 7u) * 2u;
+          const size_t off2 = chunk + (((((d + 64) >> 3) ^ (slot & 7u))) << 4) + (d & 7u) * 2u;
+          *reinterpret_cast<uint2*>(static_cast<uint8_t*>(const_cast<void*>(pages[off1 / kPageBytes])) + off1 % kPageBytes) = o1;
+          *reinterpret_cast<uint2*>(static_cast<uint8_t*>(const_cast<void*>(pages[off2 / kPageBytes])) + off2 % kPageBytes) = o2;
+          const void* const* pages2 = is_k ? p.k_page_ptr2 : p.v_page_ptr2;
+          if (pages2) {
+            *reinterpret_cast<uint2*>(static_cast<uint8_t*>(const_cast<void*>(pages2[off1 / kPageBytes])) + off1 % kPageBytes) = o1;
+            *reinterpret_cast<uint2*>(static_cast<uint8_t*>(const_cast<void*>(pages2[off2 / kPageBytes])) + off2 % kPageBytes) = o2;
+          }
+        }
+      }
+    }
+  }
+}
+
 // Sum the split-K partial sums of one row tile in split order and finish the outputs.
 // Thread -> (batch row m, columns [4 v, 4 v + 4) and their partners 64 columns on): the
 // partners are what SwiGLU (gate / up) and the rotary embedding (d / d + 64) pair up.
@@ -204,119 +326,96 @@ __device__ __forceinline__ void combine_tile(const GemvParams& p, uint32_t row_t
         }
       }
     }
+    finish_pair<kXRows>(p, row_tile, m, v, valid, lo, hi, ss, ss0, ss1, res, vec_out, status);
+  }
+}
+
+// The same combine with its passes overlapped, for kernels with registers to spare and many
+// passes per tile (the tcgen05 kernel at 64 and 128 batch rows: 4 and 8 passes of its 256
+// epilogue threads).  What a pass starts with - row statistics, residual, the first four partial
+// sums - is requested one pass ahead, so that its L2 round trip runs under the arithmetic and the
+// stores of the pass before.  Same sums in the same order as combine_tile.
+template <uint32_t kXRows, uint32_t kThreads>
+__device__ __forceinline__ void combine_tile_overlapped(const GemvParams& p, uint32_t row_tile, uint32_t n_seg,
+                                                        uint32_t tid, uint32_t* status) {
+  const float4* base = reinterpret_cast<const float4*>(p.partials + (size_t)row_tile * p.max_seg * kXRows * kBlockRows);
+  constexpr uint32_t kVecRow = kBlockRows / 4;   // float4 per batch row
+  const uint32_t n_pairs = p.M_b * 16;
+  const bool vec_out = (p.N & 3u) == 0;
+  float n_ss0 = 0.f, n_ss1 = 0.f;
+  uint2 n_res[2] = {make_uint2(0u, 0u), make_uint2(0u, 0u)};
+  float4 n0[4], n1[4];
+  auto request = [&](uint32_t pidx0) {
+    const uint32_t pidx = pidx0 + tid;
+    const bool valid = pidx < n_pairs;
+    const uint32_t m = valid ? (pidx >> 4) : 0u, v = pidx & 15u;
+    n_ss0 = n_ss1 = 0.f;
+    n_res[0] = n_res[1] = make_uint2(0u, 0u);
+    if (!valid) return;
     if (p.ssq_in) {
-      ss += ss0 + ss1;
-      ss += __shfl_xor_sync(0xFFFFFFFFu, ss, 1);
-      ss += __shfl_xor_sync(0xFFFFFFFFu, ss, 2);
-      ss += __shfl_xor_sync(0xFFFFFFFFu, ss, 4);
-      ss += __shfl_xor_sync(0xFFFFFFFFu, ss, 8);
-      const float rs = rsqrtf(ss / (float)p.x_cols + p.rms_eps);
-      lo.x *= rs; lo.y *= rs; lo.z *= rs; lo.w *= rs;
-      hi.x *= rs; hi.y *= rs; hi.z *= rs; hi.w *= rs;
+      if (v < p.ssq_in_tiles) n_ss0 = __ldcg(p.ssq_in + (size_t)v * p.ssq_stride + m);
+      if (v + 16 < p.ssq_in_tiles) n_ss1 = __ldcg(p.ssq_in + (size_t)(v + 16) * p.ssq_stride + m);
     }
-    if (p.epi == kEpiPlain) {
-      float sq = 0.f;
-      if (valid) {
-        const float4 val[2] = {lo, hi};
+    if (p.epi == kEpiPlain && p.residual && vec_out) {
 #pragma unroll
-        for (int half = 0; half < 2; ++half) {
-          const uint32_t n = row_tile * kBlockRows + half * 64 + v * 4;
-          float e[4] = {val[half].x, val[half].y, val[half].z, val[half].w};
-          if (n + 3 < p.N && vec_out) {
-            const size_t idx = (size_t)m * p.N + n;
-            if (p.residual) {
-              const uint2 r = res[half];
-              e[0] += bf16_lo(r.x); e[1] += bf16_hi(r.x); e[2] += bf16_lo(r.y); e[3] += bf16_hi(r.y);
-            }
-            if (p.y_dtype == 0) {
-              *reinterpret_cast<float4*>(static_cast<float*>(p.y) + idx) = make_float4(e[0], e[1], e[2], e[3]);
-            } else {
-              *reinterpret_cast<uint2*>(static_cast<__nv_bfloat16*>(p.y) + idx) = pack4_bf16(e[0], e[1], e[2], e[3]);
+      for (int half = 0; half < 2; ++half) {
+        const uint32_t n = row_tile * kBlockRows + half * 64 + v * 4;
+        if (n < p.N) n_res[half] = __ldcg(reinterpret_cast<const uint2*>(p.residual + (size_t)m * p.N + n));
+      }
+    }
+    const float4* src = base + m * kVecRow + v;
 #pragma unroll
-              for (int j = 0; j < 4; ++j) { const float b = round_bf16(e[j]); sq = fmaf(b, b, sq); }
-            }
-          } else {
+    for (uint32_t u = 0; u < 4; ++u) {
+      if (u < n_seg) {
+        n0[u] = __ldcg(src + (size_t)u * kXRows * kVecRow);
+        n1[u] = __ldcg(src + (size_t)u * kXRows * kVecRow + 16);
+      }
+    }
+  };
+  request(0);
+  for (uint32_t pidx0 = 0; pidx0 < n_pairs; pidx0 += kThreads) {
+    const uint32_t pidx = pidx0 + tid;
+    const bool valid = pidx < n_pairs;
+    const uint32_t m = valid ? (pidx >> 4) : 0u, v = pidx & 15u;
+    const uint32_t off = m * kVecRow + v;
+    // this pass's opening loads, then the next pass's go out
+    const float ss0 = n_ss0, ss1 = n_ss1;
+    const uint2 res[2] = {n_res[0], n_res[1]};
+    float4 lo = make_float4(0.f, 0.f, 0.f, 0.f), hi = lo;
+    if (valid) {
 #pragma unroll
-            for (int j = 0; j < 4; ++j)
-              if (n + j < p.N) {
-                float x = e[j];
-                if (p.residual) x += bf16_lo((uint32_t)__ldcg(reinterpret_cast<const unsigned short*>(p.residual) + (size_t)m * p.N + n + j));
-                if (p.y_dtype == 0) static_cast<float*>(p.y)[(size_t)m * p.N + n + j] = x;
-                else {
-                  static_cast<__nv_bfloat16*>(p.y)[(size_t)m * p.N + n + j] = __float2bfloat16_rn(x);
-                  const float b = round_bf16(x);
-                  sq = fmaf(b, b, sq);
-                }
-              }
-          }
+      for (uint32_t u = 0; u < 4; ++u) {
+        if (u < n_seg) {
+          lo.x += n0[u].x; lo.y += n0[u].y; lo.z += n0[u].z; lo.w += n0[u].w;
+          hi.x += n1[u].x; hi.y += n1[u].y; hi.z += n1[u].z; hi.w += n1[u].w;
         }
       }
-      if (p.ssq_out) {   // sum over the 16 threads that share row m (a fixed butterfly order)
-        sq += __shfl_xor_sync(0xFFFFFFFFu, sq, 1);
-        sq += __shfl_xor_sync(0xFFFFFFFFu, sq, 2);
-        sq += __shfl_xor_sync(0xFFFFFFFFu, sq, 4);
-        sq += __shfl_xor_sync(0xFFFFFFFFu, sq, 8);
-        if (valid && v == 0) p.ssq_out[(size_t)row_tile * p.ssq_stride + m] = sq;
-      }
-    } else if (p.epi == kEpiSwiglu) {
-      if (valid) {
-        const float g[4] = {round_bf16(lo.x), round_bf16(lo.y), round_bf16(lo.z), round_bf16(lo.w)};
-        const float u[4] = {round_bf16(hi.x), round_bf16(hi.y), round_bf16(hi.z), round_bf16(hi.w)};
-        float a[4];
+    }
+    if (pidx0 + kThreads < n_pairs) request(pidx0 + kThreads);
+    float ss = 0.f;
+    if (valid) {
+      if (p.ssq_in)
+        for (uint32_t t0 = v + 32; t0 < p.ssq_in_tiles; t0 += 16) ss += __ldcg(p.ssq_in + (size_t)t0 * p.ssq_stride + m);
+      for (uint32_t sp0 = 4; sp0 < n_seg; sp0 += 4) {
+        float4 t0[4], t1[4];
 #pragma unroll
-        for (int j = 0; j < 4; ++j) a[j] = g[j] / (1.f + expf(-g[j])) * u[j];
-        const size_t idx = (size_t)m * (p.N / 2) + row_tile * 64 + v * 4;
-        *reinterpret_cast<uint2*>(static_cast<__nv_bfloat16*>(p.y) + idx) = pack4_bf16(a[0], a[1], a[2], a[3]);
-      }
-    } else {   // kEpiRope
-      const int32_t ctx = valid ? p.ctx_lens[m] : 0;
-      if (valid && ctx > 0) {
-        const uint32_t pos = (uint32_t)ctx - 1u;
-        const uint32_t head = row_tile;
-        float x1[4] = {round_bf16(lo.x), round_bf16(lo.y), round_bf16(lo.z), round_bf16(lo.w)};
-        float x2[4] = {round_bf16(hi.x), round_bf16(hi.y), round_bf16(hi.z), round_bf16(hi.w)};
-        if (head < p.Hq + p.Hkv) {
-          // cos / sin of position * base^(-2i/128) for i = 4v .. 4v+3, from the step's table
-          const float4 cs01 = __ldg(reinterpret_cast<const float4*>(p.rope_table + ((size_t)m * 64 + v * 4) * 2));
-          const float4 cs23 = __ldg(reinterpret_cast<const float4*>(p.rope_table + ((size_t)m * 64 + v * 4 + 2) * 2));
-          const float cs[4] = {cs01.x, cs01.z, cs23.x, cs23.z}, sn[4] = {cs01.y, cs01.w, cs23.y, cs23.w};
-#pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            const float y1 = x1[j] * cs[j] - x2[j] * sn[j];
-            const float y2 = x2[j] * cs[j] + x1[j] * sn[j];
-            x1[j] = y1; x2[j] = y2;
+        for (uint32_t u = 0; u < 4; ++u) {
+          if (sp0 + u < n_seg) {
+            const float4* src = base + (size_t)(sp0 + u) * kXRows * kVecRow + off;
+            t0[u] = __ldcg(src);
+            t1[u] = __ldcg(src + 16);
           }
         }
-        const uint2 o1 = pack4_bf16(x1[0], x1[1], x1[2], x1[3]), o2 = pack4_bf16(x2[0], x2[1], x2[2], x2[3]);
-        const uint32_t d = v * 4;
-        if (head < p.Hq) {
-          __nv_bfloat16* dst = p.q_out + ((size_t)m * p.Hq + head) * kBlockRows;
-          *reinterpret_cast<uint2*>(dst + d) = o1;
-          *reinterpret_cast<uint2*>(dst + d + 64) = o2;
-        } else {
-          const bool is_k = head < p.Hq + p.Hkv;
-          const uint32_t kvh = is_k ? head - p.Hq : head - p.Hq - p.Hkv;
-          const uint32_t bi = pos / BOOST_KV_BLOCK_TOKENS, slot = pos % BOOST_KV_BLOCK_TOKENS;
-          const int32_t blk = bi < p.max_blocks ? p.block_table[(size_t)m * p.max_blocks + bi] : -1;
-          if (blk < 0 || (uint32_t)blk >= p.n_pool_blocks) {
-            atomicOr(status, kErrBadIndex);
-          } else {
-            const void* const* pages = is_k ? p.k_page_ptr : p.v_page_ptr;
-            // chunk (kvh, blk): token `slot` at slot*256, 16-byte piece c at position c ^ (slot & 7)
-            const size_t chunk = ((size_t)kvh * p.n_pool_blocks + (uint32_t)blk) * 4096u + slot * 256u;
-            const size_t off1 = chunk + ((((d >> 3) ^ (slot & 7u))) << 4) + (d & 7u) * 2u;
-            const size_t off2 = chunk + (((((d + 64) >> 3) ^ (slot & 7u))) << 4) + (d & 7u) * 2u;
-            *reinterpret_cast<uint2*>(static_cast<uint8_t*>(const_cast<void*>(pages[off1 / kPageBytes])) + off1 % kPageBytes) = o1;
-            *reinterpret_cast<uint2*>(static_cast<uint8_t*>(const_cast<void*>(pages[off2 / kPageBytes])) + off2 % kPageBytes) = o2;
-            const void* const* pages2 = is_k ? p.k_page_ptr2 : p.v_page_ptr2;
-            if (pages2) {
-              *reinterpret_cast<uint2*>(static_cast<uint8_t*>(const_cast<void*>(pages2[off1 / kPageBytes])) + off1 % kPageBytes) = o1;
-              *reinterpret_cast<uint2*>(static_cast<uint8_t*>(const_cast<void*>(pages2[off2 / kPageBytes])) + off2 % kPageBytes) = o2;
-            }
+#pragma unroll
+        for (uint32_t u = 0; u < 4; ++u) {
+          if (sp0 + u < n_seg) {
+            lo.x += t0[u].x; lo.y += t0[u].y; lo.z += t0[u].z; lo.w += t0[u].w;
+            hi.x += t1[u].x; hi.y += t1[u].y; hi.z += t1[u].z; hi.w += t1[u].w;
           }
         }
       }
     }
+    finish_pair<kXRows>(p, row_tile, m, v, valid, lo, hi, ss, ss0, ss1, res, vec_out, status);
   }
 }
 
@@ -1063,7 +1162,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) gemv_tc_kernel(const __grid_con
         named_barrier_sync(1, kTcEpiThreads);
         if (s_old == n_seg - 1) {
           __threadfence();
-          combine_tile<NPAD, kTcEpiThreads>(p, row_tile, n_seg, tid, status);
+          if constexpr (NPAD >= 64) combine_tile_overlapped<NPAD, kTcEpiThreads>(p, row_tile, n_seg, tid, status);
+          else combine_tile<NPAD, kTcEpiThreads>(p, row_tile, n_seg, tid, status);
           if (tid == 0) tile_cnt[row_tile] = 0;
           if (warp == 0) TRACE(8 + 8 * mt.w + 5);
         }
