@@ -7,8 +7,11 @@ attention kernels (Sec. 2.1; weights about 70 % and attention about 30 % of the
 time, Sec. 5.4) and says nothing about the small operators between them.  The
 layer structure below is the public Llama-3 architecture; its constants -
 RMSNorm epsilon 1e-5, RoPE base 500000 with the "rotate-half" pairing
-(element i pairs with i + D/2) - are choices of this repository: parity
-unpinned by the paper, pinned only by textbook special cases in the tests.
+(element i pairs with i + D/2) - are choices of this repository: the three
+constants are parity unpinned by the paper.  The structure of the step itself
+(row ranges, pairing, append position, head mapping, residual adds, both row
+scales, gate/up order, argmax ties) is pinned from outside by a restatement
+with plain loops over scalars on a tiny model, and by textbook special cases.
 
 All arithmetic is fp64.  Tensors that the device path stores as bf16 between
 kernels are rounded to bf16 here at the same places (marked "-> bf16"), so that
