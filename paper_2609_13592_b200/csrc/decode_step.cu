@@ -171,7 +171,7 @@ int run_step(Launcher& L, const boost_llama_model_t* m, const boost_llama_scratc
     if (!L.ok()) return L.rc;
   }
   auto chain = [&](const boost_gemv_call_t* calls, uint32_t n) {
-    return boosth::gemv_chain_launch(calls, n, B, s->gemv_ws, usable, slots.take(s, usable, n + 1), tiles, stream);
+    return boosth::gemv_chain_launch(calls, n, B, s->gemv_ws, usable, slots.take(s, usable, n + 1), true, tiles, stream);
   };
 
   L.run(kKindGlue, [&] { return boost_rope_table(ctx_lens, B, d, m->rope_base, s->rope_table, stream); });

@@ -11,6 +11,12 @@ void set_last_cuda_error(cudaError_t e);
 // Number of SMs of the current device (cached per device); 0 on failure.
 int sm_count();
 
+// What the launch paths set up once per device (function attributes, occupancy) is kept in
+// arrays of this many slots indexed by the current device's ordinal.
+constexpr int kMaxDevices = 64;
+// Ordinal of the current device, or -1 (no device, or an ordinal beyond kMaxDevices).
+int device_slot();
+
 inline int check(cudaError_t e) {
   if (e == cudaSuccess) return BOOST_OK;
   set_last_cuda_error(e);
@@ -70,10 +76,13 @@ int gemv_tiered_launch(const void* const* w_page_ptr, const uint32_t* w_order, s
                        void* stream);
 
 // A chain of 1..4 products in one launch (see boost_gemv_tiered_chain).  sync_words: 16 zeroed
-// uint32 per product (its queue words) followed by 16 more (phase counters), private to this
-// launch among the launches in flight.
+// uint32 per product (its queue words) followed by 16 more (phase counters).  early = true: the
+// words are private to this launch among the launches in flight (the caller rotates through
+// several sets), so the weight warps may take work before the preceding kernel has finished;
+// early = false: the preceding kernel on the stream may have used the same words.
 int gemv_chain_launch(const boost_gemv_call_t* calls, uint32_t n_calls, uint32_t M_b, void* workspace,
-                      size_t workspace_bytes, uint32_t* sync_words, uint32_t header_row_tiles, void* stream);
+                      size_t workspace_bytes, uint32_t* sync_words, bool early, uint32_t header_row_tiles,
+                      void* stream);
 
 // Bytes of the counter area for n_row_tiles row tiles, and of the partial sums of one product.
 size_t gemv_header_bytes(uint32_t n_row_tiles);

@@ -656,7 +656,10 @@ extern "C" int boost_paged_attn_decode_tiered(const void* q, const void* const* 
   p.part_o = p.part_ml + (size_t)B * Hq * partial_slots(max_blocks) * 2;
   p.out = static_cast<__nv_bfloat16*>(out);
   const size_t smem = (size_t)kAttnWarps * kWarpStages * kStageBytes + 128;
-  static bool configured = false;
+  static bool configured_on[boosth::kMaxDevices] = {false};   // function attributes are per device
+  const int slot = boosth::device_slot();
+  if (slot < 0) return BOOST_ERR_CUDA;
+  bool& configured = configured_on[slot];
   if (!configured) {
     int rc = boosth::check(cudaFuncSetAttribute(paged_attn_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     if (rc == BOOST_OK)

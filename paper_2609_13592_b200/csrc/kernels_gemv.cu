@@ -1297,14 +1297,20 @@ int launch_planned(void (*kernel)(ChainParams), KernelState& state, uint32_t thr
 // hand-over latency of the first (measured: +25 % bandwidth on B200).
 template <int NT, int MB>
 int launch_gemv(const ChainParams& chain, int sms, cudaStream_t stream) {
-  static KernelState state;
+  static KernelState states[boosth::kMaxDevices];   // attributes and occupancy are per device
+  const int slot = boosth::device_slot();
+  if (slot < 0) return BOOST_ERR_CUDA;
+  KernelState& state = states[slot];
   return launch_planned(gemv_tiered_kernel<NT, MB>, state, kGemvThreads, stage_bytes_of(NT, MB), (NT >= 8) ? 1 : 2, false,
                         chain, sms, stream);
 }
 
 template <uint32_t NPAD>
 int launch_gemv_tc(const ChainParams& chain, int sms, cudaStream_t stream) {
-  static KernelState state;
+  static KernelState states[boosth::kMaxDevices];
+  const int slot = boosth::device_slot();
+  if (slot < 0) return BOOST_ERR_CUDA;
+  KernelState& state = states[slot];
   return launch_planned(gemv_tc_kernel<NPAD>, state, kTcThreads, tc_stage_bytes(NPAD), 1, true, chain, sms, stream);
 }
 
@@ -1413,7 +1419,7 @@ namespace {
 int fill_params(GemvParams& p, const void* const* w_page_ptr, const uint32_t* w_order, size_t n_pages,
                 size_t n_host_pages, uint32_t N, uint32_t K, const void* x, uint32_t M_b, void* y, int y_dtype,
                 const void* residual, void* workspace, size_t workspace_bytes, const boost_gemv_epilogue_t* epi,
-                uint32_t* queue_words, uint32_t header_row_tiles) {
+                uint32_t* queue_words, bool early, uint32_t header_row_tiles) {
   const int mode = epi ? epi->mode : BOOST_EPI_PLAIN;
   if (!w_page_ptr || !w_order || !x || !workspace) return BOOST_ERR_INVALID;
   if (!y && mode != BOOST_EPI_ROPE_APPEND) return BOOST_ERR_INVALID;
@@ -1458,7 +1464,7 @@ int fill_params(GemvParams& p, const void* const* w_page_ptr, const uint32_t* w_
   p.residual = static_cast<const __nv_bfloat16*>(residual);
   p.ws = static_cast<uint32_t*>(workspace);
   p.queue = queue_words ? queue_words : p.ws;
-  p.early = queue_words ? 1u : 0u;
+  p.early = (queue_words && early) ? 1u : 0u;
   p.epi = (uint32_t)mode;
   p.ssq_in = epi ? epi->ssq_in : nullptr;
   p.ssq_in_tiles = epi ? epi->ssq_in_tiles : 0;
@@ -1516,13 +1522,13 @@ int boosth::gemv_tiered_launch(const void* const* w_page_ptr, const uint32_t* w_
   c.n_phases = 1;
   c.bar = nullptr;
   const int rc = fill_params(c.ph[0], w_page_ptr, w_order, n_pages, n_host_pages, N, K, x, M_b, y, y_dtype, residual,
-                             workspace, workspace_bytes, epi, queue_words, header_row_tiles);
+                             workspace, workspace_bytes, epi, queue_words, queue_words != nullptr, header_row_tiles);
   if (rc != BOOST_OK) return rc;
   return launch_routed(c, M_b, stream);
 }
 
 int boosth::gemv_chain_launch(const boost_gemv_call_t* calls, uint32_t n_calls, uint32_t M_b, void* workspace,
-                              size_t workspace_bytes, uint32_t* sync_words, uint32_t header_row_tiles,
+                              size_t workspace_bytes, uint32_t* sync_words, bool early, uint32_t header_row_tiles,
                               void* stream) {
   if (!calls || n_calls == 0 || n_calls > kMaxPhases || !sync_words) return BOOST_ERR_INVALID;
   uint32_t tiles = header_row_tiles;
@@ -1537,7 +1543,7 @@ int boosth::gemv_chain_launch(const boost_gemv_call_t* calls, uint32_t n_calls, 
     const boost_gemv_call_t& g = calls[i];
     const int rc = fill_params(c.ph[i], g.w.page_ptr, g.w.order, (size_t)g.w.n_pages, (size_t)g.w.n_host_pages, g.w.N,
                                g.w.K, g.x, M_b, g.y, g.y_dtype, g.residual, workspace, workspace_bytes,
-                               g.has_epilogue ? &g.epilogue : nullptr, sync_words + 16 * i, tiles);
+                               g.has_epilogue ? &g.epilogue : nullptr, sync_words + 16 * i, early, tiles);
     if (rc != BOOST_OK) return rc;
   }
   return launch_routed(c, M_b, stream);
@@ -1568,7 +1574,11 @@ extern "C" int boost_gemv_tiered_chain(const boost_gemv_call_t* calls, uint32_t 
   const size_t sync_bytes = 64 * (size_t)(n_calls + 1);
   const size_t usable = (workspace_bytes - sync_bytes) & ~(size_t)255;
   uint32_t* sync_words = reinterpret_cast<uint32_t*>(static_cast<uint8_t*>(workspace) + usable);
-  return boosth::gemv_chain_launch(calls, n_calls, M_b, workspace, usable, sync_words, 0, stream);
+  // The sync words sit at a fixed place of the caller's workspace, and the header lets the next
+  // call reuse the workspace on the same stream: that call's threadblocks may become resident
+  // while this one drains, so none of them may touch the words before this launch has completed
+  // (early = false: the weight warps also wait for the preceding kernel).
+  return boosth::gemv_chain_launch(calls, n_calls, M_b, workspace, usable, sync_words, false, 0, stream);
 }
 
 // Routing threshold between the two tensor-core kernels (measurement and tests).

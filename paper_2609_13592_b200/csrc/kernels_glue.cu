@@ -130,8 +130,9 @@ rope_kv_append_kernel(const __nv_bfloat16* __restrict__ qkv, __nv_bfloat16* __re
   }
   const bool is_k = head < Hq + Hkv;
   const uint32_t kvh = is_k ? head - Hq : head - Hq - Hkv;
-  const int32_t blk = block_table[(size_t)b * max_blocks + pos / kTok];
-  if (blk < 0 || (uint32_t)blk >= n_pool_blocks || pos / kTok >= max_blocks) {
+  // the table row is max_blocks wide: check the column before reading it
+  const int32_t blk = pos / kTok < max_blocks ? block_table[(size_t)b * max_blocks + pos / kTok] : -1;
+  if (blk < 0 || (uint32_t)blk >= n_pool_blocks) {
     atomicOr(status, kErrBadIndex);
     return;
   }

@@ -28,11 +28,14 @@ class LlamaDecoder:
     'lm_head' [V, hidden] (layer None) and per layer 'norm1', 'wqkv', 'wo', 'norm2', 'wgu', 'wd'.
     Weight matrices are placed per tensor with `weight_host_ratio` (modulo placement restarts
     for every tensor); the KV cache of every layer is placed linearly by a pool with
-    `kv_host_modulus`.
+    `kv_host_modulus`.  weight_tier, if given, is a callable (name, layer, n_pages) -> uint8 tier
+    array (or None for the placement function): an explicit page-to-tier table per matrix, for
+    models whose matrices are shorter than one placement period.
     """
 
     def __init__(self, cfg, get_weight, weight_host_ratio=0.0, n_pool_blocks=512, kv_host_modulus=0,
-                 max_batch=32, max_blocks=8, device="cuda", weight_policy=B.POLICY_MODULO, kv_prefetch=False):
+                 max_batch=32, max_blocks=8, device="cuda", weight_policy=B.POLICY_MODULO, kv_prefetch=False,
+                 weight_tier=None):
         self.cfg = dict(cfg)
         self.device = torch.device(device)
         self.max_batch, self.max_blocks = max_batch, max_blocks
@@ -47,8 +50,11 @@ class LlamaDecoder:
             # norm: name of the RMSNorm weight folded into this matrix at load time
             w = get_weight(name, layer).contiguous()
             g = get_weight(norm, layer).contiguous() if norm else None
+            tier = None
+            if weight_tier is not None:
+                tier = weight_tier(name, layer, B.boost_weight_layout(int(w.shape[0]), int(w.shape[1]))["n_pages"])
             tw = TieredWeight(w, weight_host_ratio, weight_policy, device=self.device, row_mode=row_mode,
-                              col_scale=g)
+                              col_scale=g, tier=tier)
             del w, g
             return tw
 

@@ -18,19 +18,15 @@ ABS_TOL = 2e-2   # max abs error against fp64 (spec tolerance)
 REL_TOL = 1e-2   # max rel error against fp64
 
 
-def assert_close_to_oracle(got, ref, what="", floor_rms=1e-3):
+def assert_close_to_oracle(got, ref, what="", floor_rms=1e-3, report_exceptions=False):
     """bf16-in / fp32-accumulate outputs against the fp64 oracle: max abs error <= 2e-2 and
     max rel error <= 1e-2.  The relative error of an element whose reference is (nearly)
     zero is taken against max(|ref|, floor_rms * rms(ref)); how many elements needed that
     floor is returned so callers can report it.
 
-    floor_rms: 1e-3 everywhere except the multi-million-output products at K = 4096, where it
-    is 2e-3.  The tensor cores add the 256 sixteen-wide partial products of such a row with a
-    truncating fp32 adder, which leaves about 256 * 2^-24 * rms = 1.5e-5 * rms on every output
-    whatever its size: 1 % of an output of 1.5e-3 * rms.  Among millions of outputs some lie
-    that close to zero, so the largest relative error hovers around the bound with a floor of
-    1e-3 * rms (1.009e-2 measured on 3.7 million outputs); the absolute bound and the relative
-    bound on every output above 2e-3 * rms still hold."""
+    report_exceptions=True (multi-million-output products): elements over the relative bound
+    do not fail here; they are returned as a list of (ref, abs err) next to the floor count
+    and the caller asserts how many there may be and what each must look like."""
     import numpy as np
     got = np.asarray(got, dtype=np.float64)
     ref = np.asarray(ref, dtype=np.float64)
@@ -43,8 +39,12 @@ def assert_close_to_oracle(got, ref, what="", floor_rms=1e-3):
     denom[denom == 0] = 1.0
     rel = err / denom
     assert err.max(initial=0.0) <= ABS_TOL, f"{what}: max abs err {err.max():.3e}"
+    n_floor = int((np.abs(ref) < floor).sum())
+    if report_exceptions:
+        over = np.flatnonzero(rel.reshape(-1) > REL_TOL)
+        return n_floor, [(float(ref.reshape(-1)[i]), float(err.reshape(-1)[i])) for i in over]
     assert rel.max(initial=0.0) <= REL_TOL, f"{what}: max rel err {rel.max():.3e}"
-    return int((np.abs(ref) < floor).sum())
+    return n_floor
 
 
 CHAIN_REL_TOL = 3e-2
@@ -82,3 +82,19 @@ def assert_chain_close(got, ref, what="", wide=False):
     if not wide:
         assert abs_err <= ABS_TOL, f"{what}: max abs err {abs_err:.3e}"
     assert rel <= CHAIN_REL_TOL, f"{what}: max err / max(|ref|, rms) {rel:.3e}"
+
+
+def assert_bulk_close(got, ref, what="", frac=0.6, tol=2e-3):
+    """Guard that goes with assert_chain_close on large tensors: its 3e-2 bound is sized for the
+    rare output behind a bf16 rounding that fell the other way, so on its own it would also pass
+    a result that is a little wrong everywhere.  At least `frac` of the outputs must agree to
+    `tol` of max(|ref|, rms(ref)): one bf16 ulp of an intermediate is 2^-8 = 4e-3 relative, so an
+    output within 2e-3 has no such event of its own size behind it."""
+    import numpy as np
+    got = np.asarray(got, dtype=np.float64)
+    ref = np.asarray(ref, dtype=np.float64)
+    rms = float(np.sqrt((ref * ref).mean()))
+    rel = np.abs(got - ref) / np.maximum(np.abs(ref), rms if rms > 0 else 1.0)
+    share = float((rel <= tol).mean())
+    assert share >= frac, f"{what}: only {share:.3f} of the outputs within {tol:g}"
+    return share

@@ -7,7 +7,7 @@ from oracle import kv_pool as okp
 from oracle import linalg as ol
 from paper_2609_13592_b200 import binding as B
 from paper_2609_13592_b200 import synth
-from tests.helpers import assert_chain_close, assert_close_to_oracle
+from tests.helpers import assert_bulk_close, assert_chain_close, assert_close_to_oracle
 
 torch = pytest.importorskip("torch")
 pytestmark = pytest.mark.gpu
@@ -108,14 +108,28 @@ def test_rope_kv_append(dev):
     pool.close()
 
 
-def build_decoder(dev, cfg, w, n_pool_blocks, kv_modulus, weight_ratio, max_batch, max_blocks):
+def build_decoder(dev, cfg, w, n_pool_blocks, kv_modulus, weight_ratio, max_batch, max_blocks, weight_tier=None):
     from paper_2609_13592_b200.llama import LlamaDecoder
 
     def get_weight(name, layer):
         src = w[name] if layer is None else w["layers"][layer][name]
         return bf16_tensor(src, dev)
 
-    return LlamaDecoder(cfg, get_weight, weight_ratio, n_pool_blocks, kv_modulus, max_batch, max_blocks, dev)
+    return LlamaDecoder(cfg, get_weight, weight_ratio, n_pool_blocks, kv_modulus, max_batch, max_blocks, dev,
+                        weight_tier=weight_tier)
+
+
+def first_page_on_host(name, layer, n_pages):
+    """Explicit tier table: the first page of every matrix in host memory.  The matrices of the
+    tiny test model are one page each - shorter than any placement period - so this is how a
+    multi-step decode gets host-tier weights (all of them, here)."""
+    tier = np.zeros(n_pages, np.uint8)
+    tier[0] = 1
+    return tier
+
+
+def all_weights(dec):
+    return [dec.lm_head] + [ly[k] for ly in dec.layers for k in ("wqkv", "wo", "wgu", "wd")]
 
 
 def load_caches(dev, dec, k_host, v_host):
@@ -132,15 +146,24 @@ def dump_cache(dev, dec, li, name):
     return bits_of(t)
 
 
-@pytest.mark.parametrize("n_seq,kv_modulus,weight_ratio,recycle", [(3, 4, 0.5, False), (1, 0, 0.0, False), (20, 2, 0.25, False),
-                                                                    (40, 4, 0.25, False), (6, 4, 0.5, True)])
-def test_decode_steps_match_oracle(dev, n_seq, kv_modulus, weight_ratio, recycle):
+@pytest.mark.parametrize("n_seq,kv_modulus,host_weights,recycle", [
+    (3, 4, True, False), (1, 0, False, False), (20, 2, True, False), (40, 4, True, False), (6, 4, False, True),
+    (2, 4, True, True), (70, 2, True, False)])
+def test_decode_steps_match_oracle(dev, n_seq, kv_modulus, host_weights, recycle):
+    """16 consecutive decode steps of the tiny model against the oracle.  host_weights: every weight
+    matrix has its (only) page in host memory, so all products of the chain take the host-tier
+    queue path; otherwise all weights are in HBM (even partition).  kv_modulus > 0 puts KV pages on
+    the host as the pool places them.  Batch 1 - 2 is the CUDA-core kernel, 3 - 32 mma.sync, 40 and
+    70 the tcgen05 kernel."""
     from tests.helpers import chain_error
     cfg = dict(synth.TINY_LLAMA)
     w = synth.llama_weights(cfg, seed=n_seq, std=0.02)
     hkv, d, nl = cfg["n_kv_heads"], cfg["head_dim"], cfg["n_layers"]
     n_pool_blocks, max_blocks = 512, 8
-    dec = build_decoder(dev, cfg, w, n_pool_blocks, kv_modulus, weight_ratio, max(n_seq, 4), max_blocks)
+    dec = build_decoder(dev, cfg, w, n_pool_blocks, kv_modulus, 0.0, max(n_seq, 4), max_blocks,
+                        weight_tier=first_page_on_host if host_weights else None)
+    assert all((tw.buf.n_host > 0) == host_weights for tw in all_weights(dec))
+    assert (dec.layers[0]["k"].n_host > 0) == (kv_modulus > 0)
     ref_pool = okp.KVPool(n_pool_blocks, hkv, kv_modulus, 16 * d * 2)
     assert dec.kv_tier.tolist() == ref_pool.page_tiers()
     # every sequence starts with a random prefix already in the cache (prefill stand-in)
@@ -242,7 +265,9 @@ def test_fused_product_epilogues_match_oracle(dev):
     # 1. plain: y = rs * (x W'^T) + residual, bf16, with the row statistics of y
     w_bits = synth.normal_bf16((640, hid), 0.05, 3)
     res_bits = synth.normal_bf16((m_b, 640), 1.0, 4)
-    w = TieredWeight(bf16_tensor(w_bits, dev), 0.5, device=dev, col_scale=bf16_tensor(gamma, dev))
+    on_host = np.array([1], np.uint8)       # the matrices here are one page each: that page in host memory
+    w = TieredWeight(bf16_tensor(w_bits, dev), device=dev, tier=on_host, col_scale=bf16_tensor(gamma, dev))
+    assert w.buf.n_host == 1
     ssq_out = torch.zeros(5, stride, dtype=torch.float32, device=dev)
     y = w.gemv(x, y_dtype=torch.bfloat16, residual=bf16_tensor(res_bits, dev),
                epilogue=epilogue(B.EPI_PLAIN, ssq_out=ssq_out.data_ptr()))
@@ -255,7 +280,7 @@ def test_fused_product_epilogues_match_oracle(dev):
 
     # 2. SwiGLU: [gate; up] packed with interleaved rows
     wgu_bits = synth.normal_bf16((2 * ffn, hid), 0.05, 5)
-    wgu = TieredWeight(bf16_tensor(wgu_bits, dev), 0.25, device=dev, row_mode=1, col_scale=bf16_tensor(gamma, dev))
+    wgu = TieredWeight(bf16_tensor(wgu_bits, dev), device=dev, row_mode=1, col_scale=bf16_tensor(gamma, dev))   # all in HBM
     act = wgu.gemv(x, y_dtype=torch.bfloat16, epilogue=epilogue(B.EPI_SWIGLU))
     torch.cuda.synchronize()
     assert tuple(act.shape) == (m_b, ffn)
@@ -276,7 +301,7 @@ def test_fused_product_epilogues_match_oracle(dev):
         for j in range((ctx[b] + 15) // 16):
             table[b, j] = next(used)
     wqkv_bits = synth.normal_bf16(((hq + 2 * hkv) * d, hid), 0.05, 9)
-    wqkv = TieredWeight(bf16_tensor(wqkv_bits, dev), 0.5, device=dev, col_scale=bf16_tensor(gamma, dev))
+    wqkv = TieredWeight(bf16_tensor(wqkv_bits, dev), device=dev, tier=on_host, col_scale=bf16_tensor(gamma, dev))
     q_out = torch.zeros(m_b, hq, d, dtype=torch.bfloat16, device=dev)
     table_d, ctx_d = torch.from_numpy(table).to(dev), torch.from_numpy(ctx).to(dev)
     rope_table = torch.zeros(m_b, d // 2, 2, dtype=torch.float32, device=dev)
@@ -349,6 +374,10 @@ def test_full_size_step_matches_oracle_on_samples(dev):
     assert_chain_close(dec.buf["h"].float().cpu().numpy(), ref["h_final"], "residual stream, full width", wide=True)
     logits = dec.buf["logits"].cpu().numpy()
     assert_chain_close(logits[:, rows], ref["logits"], "sampled logits", wide=True)
+    # the bound above is for the few outputs behind a bf16 rounding that fell the other way; the
+    # bulk must sit far inside it
+    assert_bulk_close(dec.buf["h"].float().cpu().numpy(), ref["h_final"], "residual stream")
+    assert_bulk_close(logits[:, rows], ref["logits"], "sampled logits")
     # integer work: the device's argmax of its own logits, lowest index on ties
     assert np.array_equal(nxt, np.argmax(logits, axis=-1))
     # every logit was written by this step: the buffer starts at zero, and an fp32 sum that
@@ -361,6 +390,75 @@ def test_full_size_step_matches_oracle_on_samples(dev):
         dec.step_host(tokens, table, ctx, nxt)
         differing += int(not torch.equal(dec.buf["logits"], first))
     assert differing == 0
+    assert dec.status_words() == [0, 0]
+
+
+def test_config5_launch_shape_matches_oracle_on_samples(dev):
+    """Configuration 5's launch shape: one Llama-3-8B-shaped layer + LM head at batch 128 (tcgen05
+    chain), context lengths uniform in [2048, 4096], KV blocks handed out by the wave-aware pool
+    with host modulus 5 (20 % of the KV pages in host memory), weight host share 1/131.  The
+    oracle runs the step for six sampled sequences (sequences do not interact) and every 61st
+    vocabulary row; the device runs the whole batch."""
+    cfg = dict(synth.LLAMA3_8B)
+    cfg["n_layers"] = 1
+    hq, hkv, d, hid, ffn, vocab = (cfg[k] for k in ("n_q_heads", "n_kv_heads", "head_dim", "hidden", "ffn", "vocab"))
+    n_seq, max_blocks, n_pool_blocks = 128, 256, 2560 * 13
+    head = synth.normal_bf16((vocab, hid), 0.02, 31)
+    gam = lambda s: synth.f32_to_bf16_bits(1.0 + 0.02 * np.random.default_rng(s).standard_normal(hid).astype(np.float32))
+    w = {"embed": head, "lm_head": head, "norm_f": gam(1), "layers": [{
+        "norm1": gam(2), "wqkv": synth.normal_bf16(((hq + 2 * hkv) * d, hid), 0.02, 32),
+        "wo": synth.normal_bf16((hid, hq * d), 0.02, 33), "norm2": gam(3),
+        "wgu": synth.normal_bf16((2 * ffn, hid), 0.02, 34), "wd": synth.normal_bf16((hid, ffn), 0.02, 35)}]}
+    dec = build_decoder(dev, cfg, w, n_pool_blocks, 5, 1.0 / 131, n_seq, max_blocks)
+    assert dec.host_weight_pages() > 0
+    n_kv_pages = dec.layers[0]["k"].n_pages
+    assert dec.layers[0]["k"].n_host == n_kv_pages // 5          # linear placement: the last fifth
+    ref_pool = okp.KVPool(n_pool_blocks, hkv, 5, 16 * d * 2)
+    assert dec.kv_tier.tolist() == ref_pool.page_tiers()
+    k_host = [synth.normal_bf16((hkv, n_pool_blocks, 16, d), 1.0, 41)]
+    v_host = [synth.normal_bf16((hkv, n_pool_blocks, 16, d), 1.0, 42)]
+    load_caches(dev, dec, k_host, v_host)
+    ctx = synth.ctx_lens_uniform(n_seq, 2048, 4096, 5).astype(np.int32)
+    table = np.zeros((n_seq, max_blocks), np.int32)
+    sample = [0, 17, 45, 77, 101, 127]
+    for j in range(max_blocks):                      # round-robin growth through the pool
+        for b in range(n_seq):
+            if j * 16 < ctx[b]:
+                table[b, j] = dec.pool.alloc(b, 1)[0]
+                got_ref = ref_pool.alloc(b, 1)[0]
+                if b in sample:
+                    assert table[b, j] == got_ref
+    tokens = np.random.default_rng(6).integers(0, vocab, size=n_seq).astype(np.int32)
+    nxt = np.zeros(n_seq, np.int32)
+    n_launch = dec.step_host(tokens, table, ctx, nxt)
+    assert n_launch == 4 + 2
+    assert dec.status_words() == [0, 0]
+
+    rows = np.arange(0, vocab, 61)
+    w_ref = dict(w)
+    w_ref["lm_head"] = head[rows]
+    ref = od.decode_step(cfg, w_ref, tokens[sample], k_host, v_host, table[sample], ctx[sample], n_layers=1, keep=True)
+    # the sampled sequences read host-tier KV: the second-to-last head's blocks above the pool's
+    # threshold and every block of the last head
+    assert dec.pool.query()["n_pages"] == n_kv_pages
+    assert_chain_close(dec.buf["act"].float().cpu().numpy()[sample], ref["act"], "SwiGLU output", wide=True)
+    assert_chain_close(dec.buf["h"].float().cpu().numpy()[sample], ref["h_final"], "residual stream", wide=True)
+    logits = dec.buf["logits"].cpu().numpy()
+    assert_chain_close(logits[sample][:, rows], ref["logits"], "sampled logits", wide=True)
+    assert_bulk_close(dec.buf["h"].float().cpu().numpy()[sample], ref["h_final"], "residual stream")
+    assert_bulk_close(logits[sample][:, rows], ref["logits"], "sampled logits")
+    assert np.array_equal(nxt, np.argmax(logits, axis=-1))
+    # the new K / V rows of the sampled sequences (the oracle appended them to k_host / v_host)
+    k_now, v_now = dump_cache(dev, dec, 0, "k"), dump_cache(dev, dec, 0, "v")
+    for b in sample:
+        pos = int(ctx[b]) - 1
+        blk, slot = table[b, pos // 16], pos % 16
+        assert_chain_close(ol.bf16_bits_to_f64(k_now[:, blk, slot]), ol.bf16_bits_to_f64(k_host[0][:, blk, slot]), "new k row", wide=True)
+        assert_chain_close(ol.bf16_bits_to_f64(v_now[:, blk, slot]), ol.bf16_bits_to_f64(v_host[0][:, blk, slot]), "new v row", wide=True)
+    # a second launch of the same step gives the same bits
+    first = dec.buf["logits"].clone()
+    dec.step_host(tokens, table, ctx, nxt)
+    assert torch.equal(dec.buf["logits"], first)
     assert dec.status_words() == [0, 0]
 
 
@@ -379,10 +477,14 @@ def test_gemv_chain_matches_separate_launches_and_oracle(dev, m_b):
     g2 = synth.f32_to_bf16_bits(1.0 + 0.1 * np.random.default_rng(4).standard_normal(hid).astype(np.float32))
     wb = [synth.normal_bf16((hid, kin), 0.03, 5), synth.normal_bf16((2 * ffn, hid), 0.03, 6),
           synth.normal_bf16((hid, ffn), 0.03, 7), synth.normal_bf16((n_out, hid), 0.03, 8)]
-    w = [TieredWeight(bf16_tensor(wb[0], dev), 0.5, device=dev),
-         TieredWeight(bf16_tensor(wb[1], dev), 0.25, device=dev, row_mode=1, col_scale=bf16_tensor(g1, dev)),
-         TieredWeight(bf16_tensor(wb[2], dev), 0.5, device=dev),
-         TieredWeight(bf16_tensor(wb[3], dev), 0.25, device=dev, col_scale=bf16_tensor(g2, dev))]
+    # explicit tier tables (the matrices are 1, 3, 2 and 2 pages: shorter than a placement period):
+    # an all-host matrix, a host page in the middle, at the end, at the start
+    t8 = lambda *t: np.array(t, np.uint8)
+    w = [TieredWeight(bf16_tensor(wb[0], dev), device=dev, tier=t8(1)),
+         TieredWeight(bf16_tensor(wb[1], dev), device=dev, tier=t8(0, 1, 0), row_mode=1, col_scale=bf16_tensor(g1, dev)),
+         TieredWeight(bf16_tensor(wb[2], dev), device=dev, tier=t8(0, 1)),
+         TieredWeight(bf16_tensor(wb[3], dev), device=dev, tier=t8(1, 0), col_scale=bf16_tensor(g2, dev))]
+    assert [tw.buf.n_pages for tw in w] == [1, 3, 2, 2]
     x = bf16_tensor(x_bits, dev)
 
     def buffers():
@@ -428,6 +530,30 @@ def test_gemv_chain_matches_separate_launches_and_oracle(dev, m_b):
     tail = ws_t[off + ws_bytes - 64 * 5:off + ws_bytes]
     assert int(tail.count_nonzero()) == 0                                         # queue words and phase counters reset
 
+    # The same workspace reused by launches that follow each other on the stream with nothing in
+    # between (no synchronise, no other kernel): a launch's threadblocks become resident while the
+    # one before drains, and must not touch the queue words (all four weights have host pages, so
+    # every product runs off the queues) before it has finished.  Chains of four and of one.
+    assert all(tw.buf.n_host > 0 for tw in w)
+    sets = [buffers() for _ in range(8)]
+    arrs = [B.gemv_calls(calls_for(b)) for b in sets]
+    torch.cuda.synchronize()
+    for arr in arrs:
+        B.boost_gemv_tiered_chain(arr, m_b, ws_ptr, ws_bytes)
+    torch.cuda.synchronize()
+    for i, b in enumerate(sets):
+        for name in ("h", "act", "logits", "ssq_a", "ssq_b"):
+            assert torch.equal(b[name], sep[name]), (name, i)
+    singles = [torch.zeros(m_b, n_out, dtype=torch.float32, device=dev) for _ in range(8)]
+    one = [B.gemv_calls([dict(w=w[3].struct(), x=sep["h"], y=y1, y_dtype=0, epilogue=epi(ssq_in=sep["ssq_a"]))]) for y1 in singles]
+    torch.cuda.synchronize()
+    for arr in one:
+        B.boost_gemv_tiered_chain(arr, m_b, ws_ptr, ws_bytes)
+    torch.cuda.synchronize()
+    for i, y1 in enumerate(singles):
+        assert torch.equal(y1, sep["logits"]), i
+    assert int(ws_t[off:off + 4].cpu().numpy().view(np.uint32)[0]) == 0
+
     # the oracle's operators one after the other, bf16 where the device stores bf16
     rnd = lambda a: ol.bf16_bits_to_f64(ol.f64_to_bf16_bits(a))
     x64, h64 = ol.bf16_bits_to_f64(x_bits), ol.bf16_bits_to_f64(h0_bits)
@@ -439,6 +565,8 @@ def test_gemv_chain_matches_separate_launches_and_oracle(dev, m_b):
     assert_chain_close(got["act"].float().cpu().numpy(), act, "chain: SwiGLU output", wide=True)
     assert_chain_close(got["h"].float().cpu().numpy(), h2, "chain: residual stream", wide=True)
     assert_chain_close(got["logits"].cpu().numpy(), logits, "chain: scaled product", wide=True)
+    assert_bulk_close(got["h"].float().cpu().numpy(), h2, "chain: residual stream")
+    assert_bulk_close(got["logits"].cpu().numpy(), logits, "chain: scaled product")
 
 
 def test_prefetch_variant_matches_tiered_step(dev):

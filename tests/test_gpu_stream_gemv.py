@@ -125,9 +125,19 @@ def test_gemv_config1(dev):
 
 @pytest.mark.parametrize("m_b", [1, 2, 3, 4, 5, 8, 9, 16, 17, 32, 33, 64, 100, 128])
 def test_gemv_batches(dev, m_b):
-    # several row tiles with a ragged last one, ragged K (5 k-blocks of 64, last one partial)
-    _, y, ref, _ = run_gemv(dev, 328, 296, m_b, 0.5, seed=10 + m_b)
-    assert_close_to_oracle(y, ref, f"gemv m_b={m_b}")
+    # several row tiles with a ragged last one, ragged K (5 k-blocks of 64, last one partial): one
+    # page, all in HBM (the even static partition) ...
+    w, y, ref, _ = run_gemv(dev, 328, 296, m_b, 0.0, seed=10 + m_b)
+    assert w.buf.n_pages == 1 and w.buf.n_host == 0
+    assert_close_to_oracle(y, ref, f"gemv m_b={m_b}, HBM only")
+    # ... and a tiered one: 8 row tiles (ragged last) x 20 k-blocks (ragged last) = 160 blocks over
+    # two pages, one of them in host memory (the work queues, host items first); which one
+    # alternates with the batch size
+    tier = np.array([1, 0] if m_b % 2 else [0, 1], np.uint8)
+    w, y, ref, _ = run_gemv(dev, 1000, 1256, m_b, 0.0, seed=40 + m_b, tier=tier)
+    assert w.buf.n_pages == 2 and w.buf.n_host == 1
+    assert_close_to_oracle(y, ref, f"gemv m_b={m_b}, one of two pages on the host")
+    assert w.status_words() == [0]
 
 
 @pytest.mark.parametrize("n,k,m_b,ratio", [
@@ -140,38 +150,52 @@ def test_gemv_shapes(dev, n, k, m_b, ratio):
     w, y, ref, _ = run_gemv(dev, n, k, m_b, ratio, seed=n + k + m_b)
     assert_close_to_oracle(y, ref, f"gemv {n}x{k} m_b={m_b}")
     assert w.buf.tier.tolist() == op.place_pages(w.layout["bytes"], ratio)
+    assert (w.buf.n_host > 0) == (ratio > 0)
 
 
 def test_gemv_bf16_output_with_residual(dev):
-    _, y, ref, _ = run_gemv(dev, 640, 1024, 32, 1 / 2, seed=5, y_dtype=torch.bfloat16, residual=True)
-    assert_close_to_oracle(y, ref, "bf16 out + residual")
-    _, y, ref, _ = run_gemv(dev, 640, 1024, 4, 1 / 2, seed=6, y_dtype=torch.bfloat16, residual=True)
-    assert_close_to_oracle(y, ref, "bf16 out + residual, small batch")
+    # 10 row tiles x 32 k-blocks = 320 blocks = three pages, the middle one on the host
+    tier = np.array([0, 1, 0], np.uint8)
+    for m_b, seed in ((32, 5), (4, 6), (100, 7)):
+        w, y, ref, _ = run_gemv(dev, 1280, 2048, m_b, 0.0, seed=seed, y_dtype=torch.bfloat16, residual=True, tier=tier)
+        assert w.buf.n_host == 1
+        assert_close_to_oracle(y, ref, f"bf16 out + residual, batch {m_b}, tiered")
+    _, y, ref, _ = run_gemv(dev, 640, 1024, 32, 0.0, seed=5, y_dtype=torch.bfloat16, residual=True)
+    assert_close_to_oracle(y, ref, "bf16 out + residual, HBM only")
 
 
 @pytest.mark.parametrize("m_b", [1, 32])
 def test_gemv_integer_inputs_are_exact_and_deterministic(dev, m_b):
     from paper_2609_13592_b200.tiers import TieredWeight
-    n, k = 512, 2048
+    n, k = 1024, 2048          # 8 row tiles x 32 k-blocks = two pages
     w_int = (synth.small_int_values(0, n * k).reshape(n, k)).astype(np.float32)
     x_int = (synth.small_int_values(12345, m_b * k).reshape(m_b, k)).astype(np.float32)
     w_bits, x_bits = synth.f32_to_bf16_bits(w_int), synth.f32_to_bf16_bits(x_int)
-    w = TieredWeight(bf16_tensor(w_bits, dev), 1 / 4, device=dev)
-    x = bf16_tensor(x_bits, dev)
-    y1 = w.gemv(x).clone()
-    y2 = w.gemv(x).clone()
-    torch.cuda.synchronize()
     ref = ol.gemm(x_bits, w_bits)
-    assert np.array_equal(y1.cpu().numpy().astype(np.float64), ref)   # integers: exact in fp32
-    assert torch.equal(y1, y2)
+    x = bf16_tensor(x_bits, dev)
+    for tier in ([0, 0], [0, 1], [1, 1]):       # HBM only, tiered, all on the host
+        w = TieredWeight(bf16_tensor(w_bits, dev), device=dev, tier=np.array(tier, np.uint8))
+        assert w.buf.n_host == sum(tier)
+        y1 = w.gemv(x).clone()
+        y2 = w.gemv(x).clone()
+        torch.cuda.synchronize()
+        assert np.array_equal(y1.cpu().numpy().astype(np.float64), ref), tier   # integers: exact in fp32
+        assert torch.equal(y1, y2)
 
 
 def test_gemv_result_independent_of_placement(dev):
     outs = []
+    tiers = []
     for ratio, policy in ((0.0, B.POLICY_MODULO), (1 / 4, B.POLICY_MODULO), (1 / 4, B.POLICY_RANDOM),
                           (1 / 4, B.POLICY_CONTIGUOUS)):
-        _, y, ref, _ = run_gemv(dev, 1024, 2048, 16, ratio, seed=3, policy=policy)
+        # 32 row tiles x 32 k-blocks = 8 pages: modulo puts pages 3 and 7 on the host, contiguous 6 and 7
+        w, y, ref, _ = run_gemv(dev, 4096, 2048, 16, ratio, seed=3, policy=policy)
+        assert w.buf.n_pages == 8 and (w.buf.n_host > 0) == (ratio > 0)
+        assert_close_to_oracle(y, ref, f"policy {policy} ratio {ratio}")
         outs.append(y)
+        tiers.append(w.buf.tier.tolist())
+    assert tiers[1] == [0, 0, 0, 1, 0, 0, 0, 1] and tiers[3] == [0, 0, 0, 0, 0, 0, 1, 1]
+    assert tiers[2] not in (tiers[0], tiers[1], tiers[3])
     # placement changes which threadblock adds up which blocks of a row tile (a weight with no
     # host page is cut evenly over the threadblocks, one with host pages into queue items), so
     # fp32 sums agree to rounding, not bit for bit
@@ -196,7 +220,7 @@ def test_gemv_argument_errors(dev):
     assert e.value.code == B.ERR_INVALID
 
 
-@pytest.mark.parametrize("m_b", [5, 24, 100])
+@pytest.mark.parametrize("m_b", [5, 24, 50, 100])
 def test_gemv_tcgen05_and_mma_sync_kernels_agree(dev, m_b):
     """The same product on the tcgen05 kernel (operands through shared-memory descriptors,
     accumulator in tensor memory) and on the mma.sync kernel: both against the oracle, and
@@ -206,14 +230,17 @@ def test_gemv_tcgen05_and_mma_sync_kernels_agree(dev, m_b):
     try:
         for name, threshold in (("tcgen05", 3), ("mma_sync", 1000)):
             B.boost_gemv_set_tc_min_batch(threshold)
-            for ratio in (0.0, 1 / 4):
-                _, y, ref, _ = run_gemv(dev, 1000, 2048 + 64, m_b, ratio, seed=11)
-                assert_close_to_oracle(y, ref, f"{name} M_b={m_b} host ratio {ratio}")
-                outs[(name, ratio)] = y
+            # 8 row tiles x 33 k-blocks = 264 blocks = three pages; tiered: the middle page on the host
+            for n_host, tier in ((0, [0, 0, 0]), (1, [0, 1, 0])):
+                w, y, ref, _ = run_gemv(dev, 1000, 2048 + 64, m_b, 0.0, seed=11, tier=np.array(tier, np.uint8))
+                assert w.buf.n_pages == 3 and w.buf.n_host == n_host
+                assert_close_to_oracle(y, ref, f"{name} M_b={m_b}, {n_host} host pages")
+                assert w.status_words() == [0]
+                outs[(name, n_host)] = y
     finally:
         B.boost_gemv_set_tc_min_batch(33)
-    for ratio in (0.0, 1 / 4):
-        assert np.allclose(outs[("tcgen05", ratio)], outs[("mma_sync", ratio)], rtol=2e-5, atol=2e-6)
+    for n_host in (0, 1):
+        assert np.allclose(outs[("tcgen05", n_host)], outs[("mma_sync", n_host)], rtol=2e-5, atol=2e-6)
 
 
 @pytest.mark.parametrize("ratio", [0.0, 1 / 64])
@@ -223,7 +250,17 @@ def test_gemv_full_size_batch128(dev, ratio):
     (even partition) and with one page in 64 on the host (queue items, host pages first)."""
     w, y, ref, _ = run_gemv(dev, 28672, 4096, 128, ratio, seed=21)
     assert w.buf.n_host == (0 if ratio == 0 else w.buf.n_pages // 64)
-    assert_close_to_oracle(y, ref, f"28672 x 4096, batch 128, host ratio {ratio}", floor_rms=2e-3)
+    # The strict tolerance with the 1e-3 * rms floor, the outputs that miss it counted and held to
+    # account one by one: each must be an output within 2e-3 * rms of zero whose absolute error is
+    # what the tensor cores' truncating fp32 adder leaves on every output of a K = 4096 row
+    # (256 sixteen-wide partial products: about 256 * 2^-24 * rms).  A handful among 3.7 million.
+    n_floor, exceptions = assert_close_to_oracle(y, ref, f"28672 x 4096, batch 128, host ratio {ratio}",
+                                                 report_exceptions=True)
+    rms = float(np.sqrt((ref * ref).mean()))
+    print(f"outputs below the 1e-3 rms floor: {n_floor}; outputs over 1e-2 relative: {len(exceptions)}")
+    assert len(exceptions) <= 16
+    for ref_v, err_v in exceptions:
+        assert abs(ref_v) < 2e-3 * rms and err_v <= 4 * 256 * 2.0 ** -24 * rms, (ref_v, err_v, rms)
     assert w.status_words() == [0]
 
 
