@@ -341,6 +341,17 @@ typedef struct {
  * (its matrix products are library kernels, Sec. 4.1). */
 int boost_gemv_set_tc_min_batch(uint32_t m_b);
 
+/* Where the split-K partial sums of a product are combined.  on = 1 (default): a product cut so
+ * finely that a row tile has four or more partial sums (the short products of a decode layer
+ * spread over the whole machine) combines all its tiles when its last block has been consumed,
+ * every threadblock taking a share of the (row tile, batch row) units and requesting all partial
+ * sums of a unit at once; other products, and every product with on = 0, combine each row tile in
+ * the threadblock that delivers its last partial sum.  Both orders of summation are fixed, so
+ * either setting is deterministic; they differ from each other in fp32 rounding.  Process-wide;
+ * for measurement and tests.  The paper has no counterpart (its products are library kernels,
+ * Sec. 4.1). */
+int boost_gemv_set_end_combine(uint32_t on);
+
 /* boost_gemv_tiered with an epilogue descriptor (NULL = plain). */
 int boost_gemv_tiered_fused(const void* const* w_page_ptr /*device*/, const uint32_t* w_order /*device*/,
                             size_t n_pages, size_t n_host_pages, uint32_t N, uint32_t K,

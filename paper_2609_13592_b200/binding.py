@@ -148,6 +148,7 @@ SIGNATURES = {
     "boost_swiglu": (_int, [_vp, _u32, _u32, _vp, _vp]),
     "boost_argmax": (_int, [_vp, _u32, _u32, _vp, _vp]),
     "boost_gemv_set_tc_min_batch": (_int, [_u32]),
+    "boost_gemv_set_end_combine": (_int, [_u32]),
     "boost_gemv_chain_workspace_bytes": (C.c_size_t, [_vp, _u32, _u32]),
     "boost_gemv_tiered_chain": (_int, [_vp, _u32, _u32, _vp, _sz, _vp]),
     "boost_llama_gemv_workspace_bytes": (C.c_size_t, [_vp, _u32]),
@@ -405,6 +406,10 @@ def gemv_calls(calls):
 
 def boost_gemv_set_tc_min_batch(m_b):
     _check(lib().boost_gemv_set_tc_min_batch(m_b), "boost_gemv_set_tc_min_batch")
+
+
+def boost_gemv_set_end_combine(on):
+    _check(lib().boost_gemv_set_end_combine(1 if on else 0), "boost_gemv_set_end_combine")
 
 
 def boost_gemv_chain_workspace_bytes(calls, m_b):

@@ -15,7 +15,8 @@ enum Kind { kKindGemv = 0, kKindAttn = 1, kKindGlue = 2, kNumKinds = 3 };
 struct Launcher {
   void* stream;
   bool timed = false;
-  uint32_t count = 0;
+  uint32_t count = 0;   // launches issued through run()
+  uint32_t extra = 0;   // kernels those launches added on their own
   int rc = BOOST_OK;
   cudaEvent_t ev[2 * 512];
   int kind_of[512];
@@ -171,7 +172,11 @@ int run_step(Launcher& L, const boost_llama_model_t* m, const boost_llama_scratc
     if (!L.ok()) return L.rc;
   }
   auto chain = [&](const boost_gemv_call_t* calls, uint32_t n) {
-    return boosth::gemv_chain_launch(calls, n, B, s->gemv_ws, usable, slots.take(s, usable, n + 1), true, tiles, stream);
+    uint32_t extra = 0;
+    const int rc = boosth::gemv_chain_launch(calls, n, B, s->gemv_ws, usable, slots.take(s, usable, n + 1), true, tiles,
+                                             stream, &extra);
+    L.extra += extra;   // (a product's combine may be a kernel of its own)
+    return rc;
   };
 
   L.run(kKindGlue, [&] { return boost_rope_table(ctx_lens, B, d, m->rope_base, s->rope_table, stream); });
@@ -242,9 +247,9 @@ extern "C" int boost_llama_decode_step(const boost_llama_model_t* m, const boost
                                        uint32_t max_blocks, const int32_t* ctx_lens, uint32_t B,
                                        int32_t* next_tokens, uint32_t* n_launches_out, void* stream) {
   static thread_local Launcher L;
-  L.stream = stream; L.timed = false; L.count = 0; L.rc = BOOST_OK;
+  L.stream = stream; L.timed = false; L.count = 0; L.extra = 0; L.rc = BOOST_OK;
   const int rc = run_step(L, m, s, tokens, block_table, max_blocks, ctx_lens, B, next_tokens);
-  if (n_launches_out) *n_launches_out = L.count;
+  if (n_launches_out) *n_launches_out = L.count + L.extra;
   return rc;
 }
 
@@ -293,9 +298,9 @@ extern "C" int boost_llama_decode_step_prefetch(const boost_llama_model_t* m, co
   if (prefetch->host_bytes && (!prefetch->k_stage[0] || !prefetch->k_stage[1] || !prefetch->v_stage[0] || !prefetch->v_stage[1]))
     return BOOST_ERR_INVALID;
   static thread_local Launcher L;
-  L.stream = stream; L.timed = false; L.count = 0; L.rc = BOOST_OK;
+  L.stream = stream; L.timed = false; L.count = 0; L.extra = 0; L.rc = BOOST_OK;
   const int rc = run_step(L, m, s, tokens, block_table, max_blocks, ctx_lens, B, next_tokens, prefetch, ctx);
-  if (n_launches_out) *n_launches_out = L.count;
+  if (n_launches_out) *n_launches_out = L.count + L.extra;
   return rc;
 }
 
@@ -307,7 +312,7 @@ extern "C" int boost_llama_decode_step_profile(const boost_llama_model_t* m, con
   if (!kind_ms_out || !kind_launches_out || !m) return BOOST_ERR_INVALID;
   if (4 + 2 * (uint64_t)m->n_layers > 512) return BOOST_ERR_UNSUPPORTED;
   static thread_local Launcher L;
-  L.stream = stream; L.timed = true; L.count = 0; L.rc = BOOST_OK;
+  L.stream = stream; L.timed = true; L.count = 0; L.extra = 0; L.rc = BOOST_OK;
   const uint32_t n_events = 2 * (4 + 2 * m->n_layers);
   uint32_t made = 0;
   int rc = BOOST_OK;

@@ -17,6 +17,11 @@ enum : uint32_t {
   kWsHostNext = 1,  // next item of the host-tier queue
   kWsHbmNext = 2,   // next item of the HBM queue
   kWsDone = 3,      // threadblocks that have finished (self-reset of the words above)
+  // Host-written, read-only for the kernels (both 0 in normal use):
+  kWsWaitLimit = 4,     // bounded waits give up after this many cycles instead of kWaitLimitCycles
+  kWsSkipArrivals = 5,  // honoured only with a non-zero kWsWaitLimit: threadblocks [0, n) leave out their
+                        // phase-boundary arrival, so that the others' waits run out (test of the wind-down)
+  kWsBar = 8,       // a weight product launched alone keeps its two grid-wide counters here
   kWsHeaderWords = 16
 };
 enum : uint32_t { kErrWaitTimeout = 1u, kErrBadIndex = 2u };
@@ -56,11 +61,19 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
 // caller simply carries on (its data is wrong, the host sees the status word), so that no
 // thread is left behind waiting for an arrival that never comes.
 // Returns false when it gave up.
+// `status` is the first word of the kernel's workspace header: the limit is read from the
+// header (kWsWaitLimit; 0 = kWaitLimitCycles) only once the barrier has not completed at the
+// first try, so callers carry no limit around.
+__device__ __forceinline__ long long wait_limit_of(const uint32_t* ws) {
+  const uint32_t v = __ldg(ws + kWsWaitLimit);
+  return v ? (long long)v : kWaitLimitCycles;
+}
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, uint32_t* status) {
   if (mbar_try_wait(bar, parity)) return true;
+  const long long limit = wait_limit_of(status);
   const long long t0 = clock64();
   while (!mbar_try_wait(bar, parity)) {
-    if (clock64() - t0 > kWaitLimitCycles) {
+    if (clock64() - t0 > limit) {
       atomicOr(status, kErrWaitTimeout);
       return false;
     }
@@ -106,18 +119,40 @@ __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;"
 // `target`: the grid barrier between two phases of one persistent kernel.  All threadblocks of
 // such a kernel are resident at once (the host sizes the grid from the occupancy), so the
 // counter always gets there; the wait is bounded all the same and records a timeout.
-__device__ __forceinline__ void grid_counter_wait(const uint32_t* ctr, uint32_t target, uint32_t* status) {
+// Returns false when it gave up.  `status`: first word of the workspace header (see mbar_wait).
+__device__ __forceinline__ bool grid_counter_wait(const uint32_t* ctr, uint32_t target, uint32_t* status) {
+  const long long limit = wait_limit_of(status);
   const long long t0 = clock64();
   for (;;) {
     uint32_t v;
     asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(ctr) : "memory");
-    if (v >= target) return;
-    if (clock64() - t0 > kWaitLimitCycles) {
+    if (v >= target) return true;
+    if (clock64() - t0 > limit) {
       atomicOr(status, kErrWaitTimeout);
-      return;
+      return false;
     }
     __nanosleep(32);
   }
+}
+
+// Named barrier among n_threads threads that also ORs a predicate over them: every participant
+// gets the same answer.
+__device__ __forceinline__ bool named_barrier_or(uint32_t id, uint32_t n_threads, bool pred) {
+  uint32_t r;
+  asm volatile(
+      "{\n\t.reg .pred p, q;\n\t"
+      "setp.ne.b32 p, %3, 0;\n\t"
+      "bar.red.or.pred q, %1, %2, p;\n\t"
+      "selp.u32 %0, 1, 0, q;\n\t}"
+      : "=r"(r)
+      : "r"(id), "r"(n_threads), "r"((uint32_t)pred)
+      : "memory");
+  return r != 0u;
+}
+
+// Test hook (see kWsSkipArrivals): how many threadblocks leave out their phase-boundary arrival.
+__device__ __forceinline__ uint32_t skip_arrivals_of(const uint32_t* ws) {
+  return __ldg(ws + kWsWaitLimit) ? __ldg(ws + kWsSkipArrivals) : 0u;
 }
 
 __device__ __forceinline__ void named_barrier_sync(uint32_t id, uint32_t n_threads) {

@@ -73,16 +73,18 @@ int gemv_tiered_launch(const void* const* w_page_ptr, const uint32_t* w_order, s
                        size_t n_host_pages, uint32_t N, uint32_t K, const void* x, uint32_t M_b, void* y,
                        int y_dtype, const void* residual, void* workspace, size_t workspace_bytes,
                        const boost_gemv_epilogue_t* epilogue, uint32_t* queue_words, uint32_t header_row_tiles,
-                       void* stream);
+                       void* stream, uint32_t* extra_launches = nullptr);
 
 // A chain of 1..4 products in one launch (see boost_gemv_tiered_chain).  sync_words: 16 zeroed
 // uint32 per product (its queue words) followed by 16 more (phase counters).  early = true: the
 // words are private to this launch among the launches in flight (the caller rotates through
 // several sets), so the weight warps may take work before the preceding kernel has finished;
 // early = false: the preceding kernel on the stream may have used the same words.
+// extra_launches (both calls, optional): incremented for every kernel launched beyond the first
+// (the combine of the last product when it has a kernel of its own).
 int gemv_chain_launch(const boost_gemv_call_t* calls, uint32_t n_calls, uint32_t M_b, void* workspace,
                       size_t workspace_bytes, uint32_t* sync_words, bool early, uint32_t header_row_tiles,
-                      void* stream);
+                      void* stream, uint32_t* extra_launches = nullptr);
 
 // Bytes of the counter area for n_row_tiles row tiles, and of the partial sums of one product.
 size_t gemv_header_bytes(uint32_t n_row_tiles);

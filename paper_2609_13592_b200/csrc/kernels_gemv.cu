@@ -1,14 +1,16 @@
 // Tiered weight-streaming product y = x W^T (GEMV at batch 1, skinny GEMM above) and the
 // kernel that packs a row-major weight into its paged 16 KiB-block form.
 //
-// One persistent threadblock per SM.  Two producer warps walk the work queue (host-tier
-// items first, Sec. 3.2) and fill a ring of shared-memory stages: a 16 KiB weight block
-// arrives by one bulk copy through the TMA unit when its page is in HBM, or by a deep fan of
-// 16-byte cp.async loads when the page is host memory behind the CPU-GPU link; the matching
-// 64-column slice of x rides along by cp.async.  Eight consumer warps multiply from shared
-// memory: on CUDA cores with warp-shuffle reductions for batches up to 8, with bf16
-// tensor-core MMAs above.  A work item is a run of blocks of one row tile inside one page,
-// so a threadblock reads one tier at a time.
+// Persistent threadblocks (two per SM for the mma.sync kernel, one for the tcgen05 kernel).  A
+// weight producer warp fills a ring of shared-memory stages: a 16 KiB weight block arrives by one
+// bulk copy through the TMA unit when its page is in HBM, or by a deep fan of 16-byte cp.async
+// loads when the page is host memory behind the CPU-GPU link; an activation producer warp adds
+// the matching 64-column slice of x.  Consumer warps multiply from shared memory: on CUDA cores
+// with warp-shuffle reductions for batches of 1 and 2, with mma.sync bf16 tensor-core MMAs up to
+// 32 rows, with tcgen05 MMAs into tensor memory above.  A weight with host pages is cut into work
+// items (runs of blocks of one row tile inside one page, host-tier items first, Sec. 3.2), so a
+// threadblock reads one tier at a time; a weight entirely in HBM is cut evenly over the
+// threadblocks.  Split-K partial sums meet in L2 and are combined in a fixed order.
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdlib.h>
@@ -33,6 +35,12 @@ constexpr uint32_t kXRowStride = 144;  // 128 data bytes + 16: 8 consecutive row
 
 enum : uint32_t { kFlagFirst = 1u, kFlagLast = 2u, kFlagStop = 4u, kFlagPhaseEnd = 8u, kFlagPair = 16u, kFlagSecond = 32u, kFlagHost = 64u };
 constexpr uint32_t kMaxPhases = 4;
+// Grid-wide counters of a launch, zero at rest: threadblocks that have left; per phase the
+// threadblocks whose partial sums are in memory, and the threadblocks that have finished the phase.
+enum : uint32_t { kBarExit = 0u, kBarPartials = 1u, kBarPhase = 1u + kMaxPhases, kBarWords = 1u + 2u * kMaxPhases };
+// From this many partial sums per row tile on, a phase combines all its tiles at its end, spread
+// over all threadblocks, instead of tile by tile in the threadblock that delivers the last one.
+constexpr uint32_t kEndCombineMinSegments = 4;
 enum : uint32_t { kEpiPlain = 0u, kEpiSwiglu = 1u, kEpiRope = 2u };
 
 #ifdef BOOST_TRACE
@@ -90,6 +98,13 @@ struct GemvParams {
   uint32_t even_part, total_blocks;
   uint32_t max_seg;       // partial-sum slots per row tile (= splits with the queues)
   uint32_t tiles_per_unit;   // tcgen05 kernel, even partition: 1, or 2 = adjacent row tiles share an activation tile
+  // 1: the partial sums of all row tiles are combined when the phase ends, every warp of the grid
+  // taking (row tile, batch row) units in turn (combine_units); 0: tile by tile as they complete
+  uint32_t end_combine;
+  // end_combine phases only.  1: this launch leaves the combine to a small kernel that follows it
+  // on the stream (gemv_combine_kernel) - the last phase of a launch, whose threadblocks then leave
+  // as soon as their partial sums are stored and make room for the next kernel's threadblocks
+  uint32_t defer_combine;
 };
 
 // Counter updates that publish this threadblock's earlier writes (release) and, where the old
@@ -108,6 +123,15 @@ __device__ __forceinline__ uint32_t part_owner(uint64_t block, uint32_t G, uint3
   return (uint32_t)(((block + 1) * G - 1) / T);
 }
 
+// Partial sums of row tile `row_tile` under the even partition: one per threadblock (of the G that
+// share the product) whose range holds some of the tile's blocks.
+__device__ __forceinline__ uint32_t even_part_segments(const GemvParams& p, uint32_t row_tile) {
+  const uint32_t tpu = p.tiles_per_unit;
+  const uint32_t T2 = ((p.n_row_tiles + tpu - 1) / tpu) * p.k_blocks;
+  const uint64_t u0 = (uint64_t)(row_tile / tpu) * p.k_blocks;
+  return part_owner(u0 + p.k_blocks - 1, p.active_ctas, T2) - part_owner(u0, p.active_ctas, T2) + 1;
+}
+
 // A launch runs one product, or a chain of up to kMaxPhases products in which each takes the
 // previous one's output (as its x, its residual or its row statistics).  The threadblocks stay
 // resident; between two phases they meet at a grid-wide counter, and because weights do not
@@ -116,6 +140,7 @@ __device__ __forceinline__ uint32_t part_owner(uint64_t block, uint32_t G, uint3
 // M_b, ws, n_stages and early are those of phase 0.
 struct ChainParams {
   uint32_t n_phases;
+
   uint32_t* bar;   // n_phases > 1: counters [kMaxPhases + 1], zero at rest (one per phase boundary, one for the exit)
   GemvParams ph[kMaxPhases];
 };
@@ -144,10 +169,33 @@ __device__ __forceinline__ float round_bf16(float v) { return __bfloat162float(_
 // Second half of a combine pass for one thread: its sums (lo = columns [4 v, 4 v + 4) of batch row m,
 // hi = their partners 64 columns on) are scaled by the row statistics, paired up and stored as the
 // epilogue of the product says (see combine_tile).  Called by whole warps: it shuffles.
+// What the RoPE epilogue reads besides the sums, requested ahead of them by callers that have the
+// registers for it (have = true): the context length, the block-table entry of the new token, the
+// cos / sin pairs.  Otherwise finish_pair loads them itself, after the sums.
+struct RopeOperands {
+  bool have = false;
+  int32_t ctx = 0, blk = -1;
+  float4 cs01 = make_float4(0.f, 0.f, 0.f, 0.f), cs23 = make_float4(0.f, 0.f, 0.f, 0.f);
+};
+__device__ __forceinline__ RopeOperands load_rope_operands(const GemvParams& p, uint32_t row_tile, uint32_t m, uint32_t v) {
+  RopeOperands r;
+  r.have = true;
+  r.ctx = p.ctx_lens[m];
+  if (row_tile < p.Hq + p.Hkv) {
+    r.cs01 = __ldg(reinterpret_cast<const float4*>(p.rope_table + ((size_t)m * 64 + v * 4) * 2));
+    r.cs23 = __ldg(reinterpret_cast<const float4*>(p.rope_table + ((size_t)m * 64 + v * 4 + 2) * 2));
+  }
+  if (row_tile >= p.Hq && r.ctx > 0) {
+    const uint32_t bi = ((uint32_t)r.ctx - 1u) / BOOST_KV_BLOCK_TOKENS;
+    r.blk = bi < p.max_blocks ? p.block_table[(size_t)m * p.max_blocks + bi] : -1;
+  }
+  return r;
+}
+
 template <uint32_t kXRows>
 __device__ __forceinline__ void finish_pair(const GemvParams& p, uint32_t row_tile, uint32_t m, uint32_t v, bool valid,
                                             float4 lo, float4 hi, float ss, float ss0, float ss1, const uint2 (&res)[2],
-                                            bool vec_out, uint32_t* status) {
+                                            bool vec_out, uint32_t* status, const RopeOperands& pre = RopeOperands()) {
   if (p.ssq_in) {
     ss += ss0 + ss1;
     ss += __shfl_xor_sync(0xFFFFFFFFu, ss, 1);
@@ -213,7 +261,7 @@ __device__ __forceinline__ void finish_pair(const GemvParams& p, uint32_t row_ti
       *reinterpret_cast<uint2*>(static_cast<__nv_bfloat16*>(p.y) + idx) = pack4_bf16(a[0], a[1], a[2], a[3]);
     }
   } else {   // kEpiRope
-    const int32_t ctx = valid ? p.ctx_lens[m] : 0;
+    const int32_t ctx = valid ? (pre.have ? pre.ctx : p.ctx_lens[m]) : 0;
     if (valid && ctx > 0) {
       const uint32_t pos = (uint32_t)ctx - 1u;
       const uint32_t head = row_tile;
@@ -221,8 +269,8 @@ __device__ __forceinline__ void finish_pair(const GemvParams& p, uint32_t row_ti
       float x2[4] = {round_bf16(hi.x), round_bf16(hi.y), round_bf16(hi.z), round_bf16(hi.w)};
       if (head < p.Hq + p.Hkv) {
         // cos / sin of position * base^(-2i/128) for i = 4v .. 4v+3, from the step's table
-        const float4 cs01 = __ldg(reinterpret_cast<const float4*>(p.rope_table + ((size_t)m * 64 + v * 4) * 2));
-        const float4 cs23 = __ldg(reinterpret_cast<const float4*>(p.rope_table + ((size_t)m * 64 + v * 4 + 2) * 2));
+        const float4 cs01 = pre.have ? pre.cs01 : __ldg(reinterpret_cast<const float4*>(p.rope_table + ((size_t)m * 64 + v * 4) * 2));
+        const float4 cs23 = pre.have ? pre.cs23 : __ldg(reinterpret_cast<const float4*>(p.rope_table + ((size_t)m * 64 + v * 4 + 2) * 2));
         const float cs[4] = {cs01.x, cs01.z, cs23.x, cs23.z}, sn[4] = {cs01.y, cs01.w, cs23.y, cs23.w};
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
@@ -241,7 +289,7 @@ __device__ __forceinline__ void finish_pair(const GemvParams& p, uint32_t row_ti
         const bool is_k = head < p.Hq + p.Hkv;
         const uint32_t kvh = is_k ? head - p.Hq : head - p.Hq - p.Hkv;
         const uint32_t bi = pos / BOOST_KV_BLOCK_TOKENS, slot = pos % BOOST_KV_BLOCK_TOKENS;
-        const int32_t blk = bi < p.max_blocks ? p.block_table[(size_t)m * p.max_blocks + bi] : -1;
+        const int32_t blk = pre.have ? pre.blk : (bi < p.max_blocks ? p.block_table[(size_t)m * p.max_blocks + bi] : -1);
         if (blk < 0 || (uint32_t)blk >= p.n_pool_blocks) {
           atomicOr(status, kErrBadIndex);
         } else {
@@ -419,6 +467,97 @@ __device__ __forceinline__ void combine_tile_overlapped(const GemvParams& p, uin
   }
 }
 
+// The combine as the mma.sync kernel runs it, warp by warp: one row tile (the threadblock that
+// delivered its last partial sum: first / step = warp index / warps of the threadblock), or all
+// row tiles of a product once every threadblock's partial sums are in memory (the caller has
+// waited for that: first / step = warp index / warps of the whole grid).  A warp takes one slot
+// per pass.  With few partial sums per tile (at most kPer) a slot is two batch rows, one per
+// half-warp, each lane summing all segments of its columns; with many, a slot is one batch row,
+// the half-warps take the even and the odd segments and the sums meet through a shuffle - eight
+// segments per round trip to L2 where the thread-per-row form above takes four.  Lane -> v = lane
+// % 16: columns [4 v, 4 v + 4) and their partners 64 on.  Sum order (fixed): ascending within a
+// lane, even segments + odd segments.  Short products (output, down, next qkv) have ten or so
+// partial sums per tile and all their tiles complete together at the end of the phase anyway:
+// combining them there, spread over all warps of the grid, replaces six dependent round trips in
+// 32 threadblocks by two in all of them.
+constexpr uint32_t kAllTiles = 0xFFFFFFFFu;
+template <uint32_t kXRows>
+__device__ __forceinline__ constexpr uint32_t combine_per_round() { return kXRows == 32 ? 6u : 5u; }
+// Slots of one row tile (see combine_units): pairs of batch rows, or single batch rows.
+template <uint32_t kXRows>
+__device__ __forceinline__ uint32_t combine_slots_per_tile(const GemvParams& p) {
+  return p.max_seg <= combine_per_round<kXRows>() ? (p.M_b + 1) / 2 : p.M_b;
+}
+template <uint32_t kXRows, bool kRopeAhead = false>
+__device__ __forceinline__ void combine_units(const GemvParams& p, uint32_t first, uint32_t step, uint32_t tile_or_all,
+                                              uint32_t lane, uint32_t* status) {
+  constexpr uint32_t kVecRow = kBlockRows / 4;   // float4 per batch row
+  // partial sums per lane and round: what the register budget of the instantiation leaves room for
+  constexpr uint32_t kPer = combine_per_round<kXRows>();
+  const uint32_t v = lane & 15u, half = lane >> 4;
+  const bool pair_mode = p.max_seg <= kPer;      // no tile of the product has more partial sums than that
+  const uint32_t slots_per_tile = combine_slots_per_tile<kXRows>(p);
+  const uint32_t n_slots = tile_or_all == kAllTiles ? p.n_row_tiles * slots_per_tile : slots_per_tile;
+  const bool vec_out = (p.N & 3u) == 0;
+  for (uint32_t s = first; s < n_slots; s += step) {
+    const uint32_t row_tile = tile_or_all == kAllTiles ? s / slots_per_tile : tile_or_all;
+    const uint32_t i = tile_or_all == kAllTiles ? s - row_tile * slots_per_tile : s;
+    const uint32_t m = pair_mode ? 2 * i + half : i;
+    const bool live = m < p.M_b;                       // (the second batch row of the last pair may not exist)
+    const bool valid = pair_mode ? live : half == 0;   // these lanes finish outputs
+    const uint32_t n_seg = p.even_part ? even_part_segments(p, row_tile) : p.splits;
+    const float4* base = reinterpret_cast<const float4*>(p.partials + (size_t)row_tile * p.max_seg * kXRows * kBlockRows) +
+                         (live ? m : 0u) * kVecRow + v;
+    // everything a lane needs from memory is requested before the first use
+    float ss = 0.f, ss0 = 0.f, ss1 = 0.f;
+    if (p.ssq_in && valid) {
+      if (v < p.ssq_in_tiles) ss0 = __ldcg(p.ssq_in + (size_t)v * p.ssq_stride + m);
+      if (v + 16 < p.ssq_in_tiles) ss1 = __ldcg(p.ssq_in + (size_t)(v + 16) * p.ssq_stride + m);
+      for (uint32_t t0 = v + 32; t0 < p.ssq_in_tiles; t0 += 16) ss += __ldcg(p.ssq_in + (size_t)t0 * p.ssq_stride + m);
+    }
+    uint2 res[2] = {make_uint2(0u, 0u), make_uint2(0u, 0u)};
+    if (valid && p.epi == kEpiPlain && p.residual && vec_out) {
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        const uint32_t n = row_tile * kBlockRows + h * 64 + v * 4;
+        if (n < p.N) res[h] = __ldcg(reinterpret_cast<const uint2*>(p.residual + (size_t)m * p.N + n));   // L2: an earlier phase may have rewritten it
+      }
+    }
+    RopeOperands pre;
+    if constexpr (kRopeAhead) {
+      if (p.epi == kEpiRope && valid) pre = load_rope_operands(p, row_tile, m, v);
+    }
+    float4 lo = make_float4(0.f, 0.f, 0.f, 0.f), hi = lo;
+    const uint32_t seg_first = pair_mode ? 0u : half, seg_step = pair_mode ? 1u : 2u;
+    for (uint32_t s0 = seg_first; s0 < n_seg; s0 += kPer * seg_step) {
+      float4 t0[kPer], t1[kPer];
+#pragma unroll
+      for (uint32_t j = 0; j < kPer; ++j) {
+        const uint32_t seg = s0 + j * seg_step;
+        if (seg < n_seg && live) {
+          const float4* src = base + (size_t)seg * kXRows * kVecRow;
+          t0[j] = __ldcg(src);
+          t1[j] = __ldcg(src + 16);
+        }
+      }
+#pragma unroll
+      for (uint32_t j = 0; j < kPer; ++j) {
+        if (s0 + j * seg_step < n_seg && live) {
+          lo.x += t0[j].x; lo.y += t0[j].y; lo.z += t0[j].z; lo.w += t0[j].w;
+          hi.x += t1[j].x; hi.y += t1[j].y; hi.z += t1[j].z; hi.w += t1[j].w;
+        }
+      }
+    }
+    if (!pair_mode) {   // lanes 0..15 take the odd segments' sums from lanes 16..31
+      lo.x += __shfl_down_sync(0xFFFFFFFFu, lo.x, 16); lo.y += __shfl_down_sync(0xFFFFFFFFu, lo.y, 16);
+      lo.z += __shfl_down_sync(0xFFFFFFFFu, lo.z, 16); lo.w += __shfl_down_sync(0xFFFFFFFFu, lo.w, 16);
+      hi.x += __shfl_down_sync(0xFFFFFFFFu, hi.x, 16); hi.y += __shfl_down_sync(0xFFFFFFFFu, hi.y, 16);
+      hi.z += __shfl_down_sync(0xFFFFFFFFu, hi.z, 16); hi.w += __shfl_down_sync(0xFFFFFFFFu, hi.w, 16);
+    }
+    finish_pair<kXRows>(p, row_tile, live ? m : 0u, v, valid, lo, hi, ss, ss0, ss1, res, vec_out, status, pre);
+  }
+}
+
 // NT > 0: tensor-core path with NT batch tiles of 8; NT == 0: CUDA-core path for MB rows.
 template <int NT, int MB>
 __global__ void __launch_bounds__(kGemvThreads, (NT >= 8 ? 1 : 2)) gemv_tiered_kernel(const __grid_constant__ ChainParams cp) {
@@ -433,6 +572,7 @@ __global__ void __launch_bounds__(kGemvThreads, (NT >= 8 ? 1 : 2)) gemv_tiered_k
   __shared__ uint64_t item_empty[4];
   __shared__ uint32_t item_ring[4];
   __shared__ uint32_t s_old;
+  __shared__ volatile uint32_t s_abort;    // a bounded wait ran out somewhere: every role leaves
 
   const uint32_t tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const uint32_t n_stages = cp.ph[0].n_stages;
@@ -445,14 +585,33 @@ __global__ void __launch_bounds__(kGemvThreads, (NT >= 8 ? 1 : 2)) gemv_tiered_k
     for (uint32_t s = 0; s < n_stages; ++s) {
       mbar_init(&full_bar[s], 65);              // 2 x 32 cp.async arrivals + the arrive.expect_tx
       mbar_init(&empty_bar[s], kConsumerWarps);
+      meta[s] = make_uint4(0u, 0u, 0u, 0u);     // a consumer whose wait ran out reads nothing wild
     }
     for (uint32_t s = 0; s < 4; ++s) {
       mbar_init(&item_full[s], 1);
       mbar_init(&item_empty[s], 1);
     }
+    s_abort = 0u;
     fence_barrier_init();
   }
   __syncthreads();
+
+  // Bounded waits.  On a timeout the status word gets kErrWaitTimeout, s_abort is raised and the
+  // warp leaves the kernel; the other roles see the flag (or run into their own limit) and leave
+  // too, so nothing is read or written on the strength of a wait that did not succeed.
+  auto lane0_wait = [&](uint64_t* bar, uint32_t parity) -> bool {   // lane 0 waits, the warp learns the outcome
+    uint32_t ok = 1u;
+    if (lane == 0) ok = (!s_abort && mbar_wait(bar, parity, status)) ? 1u : 0u;
+    ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
+    if (!ok) s_abort = 1u;
+    return ok != 0u;
+  };
+  auto warp_wait = [&](uint64_t* bar, uint32_t parity) -> bool {    // all lanes wait
+    const bool ok = !s_abort && mbar_wait(bar, parity, status);
+    const bool all_ok = __all_sync(0xFFFFFFFFu, ok);
+    if (!all_ok) s_abort = 1u;
+    return all_ok;
+  };
 
   if (warp >= kConsumerWarps) {
     // ------------------------------------------------------------------ producer warps
@@ -461,6 +620,17 @@ __global__ void __launch_bounds__(kGemvThreads, (NT >= 8 ? 1 : 2)) gemv_tiered_k
     // Two warps, because a lone warp's instruction latency would cap the fill rate.
     const bool leader = (warp == kConsumerWarps);
     uint32_t stage = 0, phase = 0, icount = 0;
+    // Leaving after a timeout: this warp's own copies must have landed first (a few microseconds
+    // for a block from the host tier; the wait is bounded all the same).
+    auto leave = [&]() {
+      cp_async_wait_all();
+      if (leader && lane == 0) {
+        const long long t0 = clock64();
+        for (uint32_t s = 0; s < n_stages; ++s)
+          while (!mbar_try_wait(&full_bar[s], 0u) && !mbar_try_wait(&full_bar[s], 1u) && clock64() - t0 < 200000) {}
+      }
+      __syncwarp();
+    };
     for (uint32_t ph = 0; ph < n_phases; ++ph) {
       const GemvParams& p = cp.ph[ph];
       const uint32_t n_host_items = p.n_host_pages * p.items_per_page;
@@ -475,8 +645,10 @@ __global__ void __launch_bounds__(kGemvThreads, (NT >= 8 ? 1 : 2)) gemv_tiered_k
       } else if (!leader) {
         // x of this phase is what the previous phase wrote: wait until every threadblock has
         // finished it.  The weight warp does not wait: it fills the ring meanwhile.
-        if (lane == 0) grid_counter_wait(cp.bar + (ph - 1), gridDim.x, status);
-        __syncwarp();
+        uint32_t ok = 1u;
+        if (lane == 0) ok = (!s_abort && grid_counter_wait(cp.bar + kBarPhase + (ph - 1), gridDim.x, status)) ? 1u : 0u;
+        ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
+        if (!ok) { s_abort = 1u; leave(); return; }
       }
       if (!leader) TRACE(8 + 8 * ph + 2);
       if (p.even_part) {
@@ -496,13 +668,13 @@ __global__ void __launch_bounds__(kGemvThreads, (NT >= 8 ? 1 : 2)) gemv_tiered_k
             const bool seg_first = (b == b0) || kb == 0, seg_last = (b + 1 == b1) || (kb + 1 == p.k_blocks);
             if (leader) {
               uint8_t* wdst = smem + (size_t)stage * kStageBytes;
+              if (!lane0_wait(&empty_bar[stage], phase ^ 1u)) { leave(); return; }
               if (lane == 0) {
                 if (b / kBlocksPerPage != page_of_base) {
                   page_of_base = b / kBlocksPerPage;
                   page_base = static_cast<const uint8_t*>(p.w_page_ptr[page_of_base]);
                 }
                 const uint8_t* src = page_base + (size_t)(b % kBlocksPerPage) * kBlockBytes;
-                mbar_wait(&empty_bar[stage], phase ^ 1u, status);
                 meta[stage] = make_uint4(row_tile, seg, (seg_first ? kFlagFirst : 0u) | (seg_last ? kFlagLast : 0u), ph);
                 mbar_arrive_expect_tx(&full_bar[stage], kBlockBytes);
                 bulk_copy_g2s(wdst, src, kBlockBytes, &full_bar[stage]);
@@ -510,7 +682,7 @@ __global__ void __launch_bounds__(kGemvThreads, (NT >= 8 ? 1 : 2)) gemv_tiered_k
               __syncwarp();
               cp_async_arrive_noinc(&full_bar[stage]);
             } else {
-              mbar_wait(&empty_bar[stage], phase ^ 1u, status);
+              if (!warp_wait(&empty_bar[stage], phase ^ 1u)) { leave(); return; }
               uint8_t* xdst = smem + (size_t)stage * kStageBytes + kBlockBytes + m0 * kXRowStride + c * 16;
               const uint32_t k = kb * kBlockK + c * 8;
               const bool k_ok = k < p.K;
@@ -538,13 +710,15 @@ __global__ void __launch_bounds__(kGemvThreads, (NT >= 8 ? 1 : 2)) gemv_tiered_k
               if (qi == 0xFFFFFFFFu) break;
               if (p.w_order[qi / p.items_per_page] * p.items_per_page + qi % p.items_per_page < p.n_items) break;
             }
-            mbar_wait(&item_empty[slot], iphase ^ 1u, status);
+          }
+          if (!lane0_wait(&item_empty[slot], iphase ^ 1u)) { leave(); return; }
+          if (lane == 0) {
             item_ring[slot] = qi;
             mbar_arrive(&item_full[slot]);
           }
           qi = __shfl_sync(0xFFFFFFFFu, qi, 0);
         } else {
-          mbar_wait(&item_full[slot], iphase, status);
+          if (!warp_wait(&item_full[slot], iphase)) { leave(); return; }
           qi = item_ring[slot];
           __syncwarp();
           if (lane == 0) mbar_arrive(&item_empty[slot]);
@@ -562,14 +736,15 @@ __global__ void __launch_bounds__(kGemvThreads, (NT >= 8 ? 1 : 2)) gemv_tiered_k
                                (size_t)(first_blk % kBlocksPerPage) * kBlockBytes;
           for (uint32_t j = 0; j < p.run; ++j, src += kBlockBytes) {
             uint8_t* wdst = smem + (size_t)stage * kStageBytes;
+            // (the other lanes must not run ahead of lane 0's wait on the stage)
+            if (!lane0_wait(&empty_bar[stage], phase ^ 1u)) { leave(); return; }
             if (lane == 0) {
-              mbar_wait(&empty_bar[stage], phase ^ 1u, status);
               meta[stage] = make_uint4(row_tile, kb0 / p.run,
                                        (j == 0 ? kFlagFirst : 0u) | (j + 1 == p.run ? kFlagLast : 0u), ph);
               mbar_arrive_expect_tx(&full_bar[stage], from_host ? 0u : kBlockBytes);
               if (!from_host) bulk_copy_g2s(wdst, src, kBlockBytes, &full_bar[stage]);
             }
-            __syncwarp();   // the other lanes must not run ahead of lane 0's wait on the stage
+            __syncwarp();
             if (from_host) {
               // host page: a fan of 16-byte loads through the load/store path keeps many
               // requests on the link at once (Sec. 3.2: this threadblock is a host-tier block)
@@ -584,7 +759,7 @@ __global__ void __launch_bounds__(kGemvThreads, (NT >= 8 ? 1 : 2)) gemv_tiered_k
           // lane -> (row m0 + 4 i, 16-byte chunk c); pointers advance by constants
           const uint32_t c = lane & 7, m0 = lane >> 3;
           for (uint32_t j = 0; j < p.run; ++j) {
-            mbar_wait(&empty_bar[stage], phase ^ 1u, status);
+            if (!warp_wait(&empty_bar[stage], phase ^ 1u)) { leave(); return; }
             uint8_t* xdst = smem + (size_t)stage * kStageBytes + kBlockBytes + m0 * kXRowStride + c * 16;
             const uint32_t k = (kb0 + j) * kBlockK + c * 8;
             const bool k_ok = k < p.K;
@@ -603,8 +778,8 @@ __global__ void __launch_bounds__(kGemvThreads, (NT >= 8 ? 1 : 2)) gemv_tiered_k
       // a stage without data tells the consumers that the phase (or the launch) is over
       if (leader) TRACE(8 + 8 * ph + 1);
       if (leader) {
+        if (!lane0_wait(&empty_bar[stage], phase ^ 1u)) { leave(); return; }
         if (lane == 0) {
-          mbar_wait(&empty_bar[stage], phase ^ 1u, status);
           meta[stage] = make_uint4(0u, 0u, ph + 1 == n_phases ? kFlagStop : kFlagPhaseEnd, ph);
           mbar_arrive(&full_bar[stage]);
         }
@@ -612,7 +787,7 @@ __global__ void __launch_bounds__(kGemvThreads, (NT >= 8 ? 1 : 2)) gemv_tiered_k
         cp_async_arrive_noinc(&full_bar[stage]);
         if (lane == 0 && active && !p.even_part) q.finish(p.active_ctas);
       } else {
-        mbar_wait(&empty_bar[stage], phase ^ 1u, status);
+        if (!warp_wait(&empty_bar[stage], phase ^ 1u)) { leave(); return; }
         cp_async_arrive_noinc(&full_bar[stage]);
       }
       if (++stage == n_stages) { stage = 0; phase ^= 1u; }
@@ -629,39 +804,33 @@ __global__ void __launch_bounds__(kGemvThreads, (NT >= 8 ? 1 : 2)) gemv_tiered_k
 #pragma unroll
     for (int j = 0; j < kAccM; ++j) acc[i][j] = 0.f;
 
+  // The consumer warps meet at named barrier 1, which also ORs their views of s_abort, so all of
+  // them take the same way out.  A hardware barrier has no time limit, so the wind-down after a
+  // failed wait must leave nobody in it: a warp whose (bounded) wait ran out arrives ONCE more,
+  // with "abort", before it leaves (end of this function).  Every other warp arrives once more too -
+  // at its next group_sync, or the same way after a failed wait of its own (once s_abort is up
+  // every wait fails at once) - so that barrier generation completes and tells everybody to leave.
+  // False: leave, without a further arrival.
+  auto group_sync = [&]() -> bool { return !named_barrier_or(1, kConsumerThreads, s_abort != 0u); };
   uint32_t* tile_cnt = cp.ph[0].ws + kWsHeaderWords;
   uint32_t stage = 0, phase = 0;
+  bool wait_failed = false;   // this warp's own wait ran out (as opposed to: it saw s_abort after a barrier)
   pdl_wait();
+  // Outer loop: one round per phase.  The inner loop consumes stages until the marker stage that
+  // ends the phase; what follows a phase (the combine of all tiles, the grid-wide counters) stays
+  // outside the inner loop, so that its register needs do not weigh on the streaming code.
   for (;;) {
-    mbar_wait(&full_bar[stage], phase, status);
+  uint4 mk = make_uint4(0u, 0u, 0u, 0u);
+  bool failed = false;
+  // Opaque copies of the warp and lane numbers, renewed for every phase: the shared-memory
+  // addresses the streaming loop derives from them are loop invariants that the compiler keeps in
+  // registers, and this keeps them from staying alive across the code that follows a phase.
+  uint32_t lw = warp, ll = lane;
+  asm volatile("" : "+r"(lw), "+r"(ll));
+  for (;;) {
+    if (!warp_wait(&full_bar[stage], phase)) { wait_failed = true; failed = true; break; }
     const uint4 mt = meta[stage];
-    if (mt.z & (kFlagStop | kFlagPhaseEnd)) {
-      if (warp == 0) TRACE(8 + 8 * mt.w + 4);
-      if (n_phases > 1) {
-        // every consumer thread has finished this phase's items, combines included: publish
-        // them and tell the grid (the x warps of all threadblocks wait for the count)
-        named_barrier_sync(1, kConsumerThreads);
-        if (tid == 0) {
-          if (mt.z & kFlagPhaseEnd) {
-            red_add_release(cp.bar + mt.w, 1u);
-          } else {
-            __threadfence();
-            // last threadblock out puts the counters back to zero for the next launch; by then
-            // every x warp has passed every phase boundary (its stop stage came after them)
-            const uint32_t old = atomicAdd(cp.bar + kMaxPhases, 1u);
-            if (old == gridDim.x - 1) {
-              for (uint32_t i = 0; i <= kMaxPhases; ++i) cp.bar[i] = 0u;
-              __threadfence();
-            }
-          }
-        }
-      }
-      if (mt.z & kFlagStop) break;
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&empty_bar[stage]);
-      if (++stage == n_stages) { stage = 0; phase ^= 1u; }
-      continue;
-    }
+    if (mt.z & (kFlagStop | kFlagPhaseEnd)) { mk = mt; break; }
     if (warp == 0 && (mt.z & kFlagFirst)) TRACE_ONCE(8 + 8 * mt.w + 3);
     if (mt.z & kFlagFirst) {
 #pragma unroll
@@ -673,14 +842,14 @@ __global__ void __launch_bounds__(kGemvThreads, (NT >= 8 ? 1 : 2)) gemv_tiered_k
     const uint8_t* xsm = wsm + kBlockBytes;
     if constexpr (NT > 0) {
       const uint32_t wbase = smem_u32(wsm), xbase = smem_u32(xsm);
-      const uint32_t a_row = warp * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
-      const uint32_t b_row0 = ((lane >> 4) << 3) + (lane & 7);
+      const uint32_t a_row = lw * 16 + (ll & 7) + ((ll >> 3) & 1) * 8;
+      const uint32_t b_row0 = ((ll >> 4) << 3) + (ll & 7);
 #pragma unroll
       for (uint32_t ks = 0; ks < 4; ++ks) {
         uint32_t a[4];
-        const uint32_t a_chunk = ks * 2 + (lane >> 4);
+        const uint32_t a_chunk = ks * 2 + (ll >> 4);
         ldmatrix_x4(a[0], a[1], a[2], a[3], wbase + a_row * 128 + ((a_chunk ^ (a_row & 7)) << 4));
-        const uint32_t b_chunk = ks * 2 + ((lane >> 3) & 1);
+        const uint32_t b_chunk = ks * 2 + ((ll >> 3) & 1);
 #pragma unroll
         for (int n2 = 0; n2 < NT / 2; ++n2) {
           const uint32_t b_row = n2 * 16 + b_row0;
@@ -691,12 +860,12 @@ __global__ void __launch_bounds__(kGemvThreads, (NT >= 8 ? 1 : 2)) gemv_tiered_k
         }
       }
     } else {
-      // lanes 8g..8g+7 share weight row (warp*16 + 4j + g) and split its 64 columns
-      const uint32_t c = lane & 7, g = lane >> 3;
+      // lanes 8g..8g+7 share weight row (lw*16 + 4j + g) and split its 64 columns
+      const uint32_t c = ll & 7, g = ll >> 3;
       float wf[4][8];
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
-        const uint32_t row = warp * 16 + 4 * j + g;
+        const uint32_t row = lw * 16 + 4 * j + g;
         const uint4 w = *reinterpret_cast<const uint4*>(wsm + row * 128 + ((c ^ (row & 7)) << 4));
         wf[j][0] = bf16_lo(w.x); wf[j][1] = bf16_hi(w.x); wf[j][2] = bf16_lo(w.y); wf[j][3] = bf16_hi(w.y);
         wf[j][4] = bf16_lo(w.z); wf[j][5] = bf16_hi(w.z); wf[j][6] = bf16_lo(w.w); wf[j][7] = bf16_hi(w.w);
@@ -744,15 +913,11 @@ __global__ void __launch_bounds__(kGemvThreads, (NT >= 8 ? 1 : 2)) gemv_tiered_k
             acc[j][m] = s;
           }
       }
-      // without splits (and without a row scale, pairing or row statistics) the sums go straight out
       // partial sums of this row tile: one per split of the queue items, or one per
       // threadblock of the even partition that holds some of its blocks
-      uint32_t n_seg = p.splits;
-      if (p.even_part) {
-        const uint64_t t0 = (uint64_t)row_tile * p.k_blocks;
-        n_seg = part_owner(t0 + p.k_blocks - 1, p.active_ctas, p.total_blocks) - part_owner(t0, p.active_ctas, p.total_blocks) + 1;
-      }
-      const bool direct = (n_seg == 1) && p.epi == kEpiPlain && !p.ssq_in && !p.ssq_out;
+      const uint32_t n_seg = p.even_part ? even_part_segments(p, row_tile) : p.splits;
+      // without splits (and without a row scale, pairing or row statistics) the sums go straight out
+      const bool direct = (n_seg == 1) && p.epi == kEpiPlain && !p.ssq_in && !p.ssq_out && !p.end_combine;
       float* part = p.partials + ((size_t)row_tile * p.max_seg + split) * kXRows * kBlockRows;
       if constexpr (NT > 0) {
 #pragma unroll
@@ -784,27 +949,102 @@ __global__ void __launch_bounds__(kGemvThreads, (NT >= 8 ? 1 : 2)) gemv_tiered_k
             }
         }
       }
-      if (!direct) {
-        // the threadblock that delivers the last partial sum of a row tile adds them up in
-        // split order (fixed order: deterministic) and writes the output
-        named_barrier_sync(1, kConsumerThreads);
+      if (!direct && !p.end_combine) {
+        // the threadblock that delivers the last partial sum of a row tile adds them up (in a
+        // fixed order: deterministic) and writes the output
+        if (!group_sync()) { failed = true; break; }
         if (tid == 0) {
           // release: publishes the partials of all consumer threads (ordered by the barrier);
           // acquire: the last to arrive reads the others' partials after this
           s_old = atom_add_acq_rel(tile_cnt + row_tile, 1u);
         }
-        named_barrier_sync(1, kConsumerThreads);
-        if (s_old == n_seg - 1) {
-          __threadfence();
-          combine_tile<kXRows>(p, row_tile, n_seg, tid, status);
-          if (tid == 0) tile_cnt[row_tile] = 0;
-          if (warp == 0) TRACE(8 + 8 * mt.w + 5);
+        if (!group_sync()) { failed = true; break; }
+        if (s_old == n_seg - 1) {   // ours was the last: leave the streaming loop for the combine
+          mk = make_uint4(row_tile, 0u, 0u, mt.w);
+          break;
         }
-        named_barrier_sync(1, kConsumerThreads);
       }
     }
   }
+  if (failed) break;
+  // ---- outside the streaming loop: a row tile to combine (mk.z == 0: tile mk.x of phase mk.w),
+  // or the marker that ends a phase or the launch.  One call of the combine serves both.
+  // (the accumulators hold nothing here: saying so frees their registers for the combine)
+#pragma unroll
+  for (int i = 0; i < kAccN; ++i)
+#pragma unroll
+    for (int j = 0; j < kAccM; ++j) acc[i][j] = 0.f;
+  {
+    const uint4 mt = mk;
+    const GemvParams& p = cp.ph[mt.w];
+    const bool phase_end = (mt.z & (kFlagStop | kFlagPhaseEnd)) != 0;
+    if (phase_end && warp == 0) TRACE(8 + 8 * mt.w + 4);
+    // Slots go to the warps of the grid in order, so only the first threadblocks have any; one
+    // without has nothing to wait for once its own partial sums are out (after the last phase it
+    // leaves at once and makes room for the next kernel's threadblocks).
+    bool combines = !phase_end;
+    const uint32_t combine_ctas = gridDim.x;
+    if (phase_end && p.end_combine && !p.defer_combine) {
+      // every threadblock's partial sums of this phase in memory -> all tiles combined, by all
+      if (!group_sync()) break;
+      combines = blockIdx.x < combine_ctas && blockIdx.x * kConsumerWarps < p.n_row_tiles * combine_slots_per_tile<kXRows>(p);
+      if (tid == 0) {
+        red_add_release(cp.bar + kBarPartials + mt.w, 1u);
+        if (combines && !grid_counter_wait(cp.bar + kBarPartials + mt.w, gridDim.x, status)) s_abort = 1u;
+      }
+      if (combines && !group_sync()) break;
+      if (warp == 0) TRACE(8 + 8 * mt.w + 7);
+    }
+    if (combines) {
+      __threadfence();
+      const bool all = phase_end;
+      combine_units<kXRows>(p, all ? blockIdx.x * kConsumerWarps + warp : warp, all ? combine_ctas * kConsumerWarps : kConsumerWarps,
+                            all ? kAllTiles : mt.x, lane, status);
+      if (warp == 0) TRACE(8 + 8 * mt.w + 5);
+    }
+    if (!phase_end) {
+      if (tid == 0) tile_cnt[mt.x] = 0;
+      if (!group_sync()) break;   // (s_old may be rewritten, the tile's slots reused)
+      continue;
+    }
+    // every consumer thread has finished this phase's items, combines included: publish
+    // them and tell the grid (the x warps of all threadblocks wait for the count)
+    if (!group_sync()) break;
+    if (tid == 0) {
+      if (mt.z & kFlagPhaseEnd) {
+        if (blockIdx.x >= skip_arrivals_of(cp.ph[0].ws)) red_add_release(cp.bar + kBarPhase + mt.w, 1u);
+      } else {
+        __threadfence();
+        // last threadblock out puts the counters back to zero for the next launch; by then
+        // every warp of every threadblock has passed every counter it waits for
+        const uint32_t old = atomicAdd(cp.bar + kBarExit, 1u);
+        if (old == gridDim.x - 1) {
+          for (uint32_t i = 0; i < (n_phases > 1 ? kBarWords : kBarPartials + 1); ++i) cp.bar[i] = 0u;
+          __threadfence();
+        }
+      }
+    }
+    if (mt.z & kFlagStop) break;
+    __syncwarp();
+    if (lane == 0) mbar_arrive(&empty_bar[stage]);
+    if (++stage == n_stages) { stage = 0; phase ^= 1u; }
+  }
+  }
+  if (wait_failed) named_barrier_or(1, kConsumerThreads, true);   // the arrival the others' next group_sync counts on
   if (warp == 0) TRACE(7);
+}
+
+// The combine of a product whose launch left it out (defer_combine): every row tile at once, the
+// warps of this small grid taking slots in turn.  It follows the product on the stream with
+// programmatic dependent launch, so its threadblocks are in place when the product's last
+// threadblock leaves, and the kernel after it (attention, in a decode step) finds the SMs free:
+// the product's threadblocks do not stay around for a combine that a handful of warps can do.
+template <uint32_t kXRows>
+__global__ void __launch_bounds__(kConsumerThreads) gemv_combine_kernel(const __grid_constant__ GemvParams p) {
+  pdl_launch_dependents();
+  pdl_wait();   // the product has completed: its partial sums are in memory
+  combine_units<kXRows, true>(p, blockIdx.x * kConsumerWarps + (threadIdx.x >> 5), gridDim.x * kConsumerWarps, kAllTiles,
+                              threadIdx.x & 31u, p.ws + kWsStatus);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -891,7 +1131,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) gemv_tc_kernel(const __grid_con
       if (ph == 0) {
         if (!leader || !p.early) pdl_wait();
       } else if (!leader) {
-        if (lane == 0) grid_counter_wait(cp.bar + (ph - 1), gridDim.x, status);
+        if (lane == 0 && !grid_counter_wait(cp.bar + kBarPhase + (ph - 1), gridDim.x, status)) s_abort = 1;
         __syncwarp();
       }
       if (warp == kTcEpiWarps + 2) TRACE(8 + 8 * ph + 2);
@@ -1090,16 +1330,16 @@ __global__ void __launch_bounds__(kTcThreads, 1) gemv_tc_kernel(const __grid_con
     const uint4 mt = acc_meta[buf];
     if (mt.z & (kFlagStop | kFlagPhaseEnd)) {
       if (warp == 0) TRACE(8 + 8 * mt.w + 4);
-      if (n_phases > 1) {
+      {
         named_barrier_sync(1, kTcEpiThreads);
         if (tid == 0) {
           if (mt.z & kFlagPhaseEnd) {
-            red_add_release(cp.bar + mt.w, 1u);
+            if (blockIdx.x >= skip_arrivals_of(cp.ph[0].ws)) red_add_release(cp.bar + kBarPhase + mt.w, 1u);
           } else {
             __threadfence();
-            const uint32_t old = atomicAdd(cp.bar + kMaxPhases, 1u);
+            const uint32_t old = atomicAdd(cp.bar + kBarExit, 1u);
             if (old == gridDim.x - 1) {
-              for (uint32_t i = 0; i <= kMaxPhases; ++i) cp.bar[i] = 0u;
+              for (uint32_t i = 0; i < (n_phases > 1 ? kBarWords : kBarPartials + 1); ++i) cp.bar[i] = 0u;
               __threadfence();
             }
           }
@@ -1228,6 +1468,11 @@ uint32_t pick_run(uint32_t n_row_tiles, uint32_t k_blocks) {
   return 1;
 }
 
+// Combine-at-phase-end on (1) or off (0: every tile by its last arriver), for measurements; and
+// whether the last phase's combine goes to a kernel of its own.
+uint32_t g_end_combine = 1;
+uint32_t g_defer_combine = 1;
+
 // Common launch path of the two kernels: ring depth from the shared-memory budget, grid and
 // per-phase threadblock counts, host-tier threadblocks.  `state` keeps what is set up once per
 // kernel instantiation.
@@ -1237,8 +1482,9 @@ struct KernelState {
 };
 
 // pairs: the even partition counts (pair of row tiles, k block) units instead of blocks.
-int launch_planned(void (*kernel)(ChainParams), KernelState& state, uint32_t threads, uint32_t stage_bytes,
-                   uint32_t ctas_per_sm, bool pairs, const ChainParams& chain, int sms, cudaStream_t stream) {
+int launch_planned(void (*kernel)(ChainParams), void (*combine_kernel)(GemvParams), uint32_t x_rows, KernelState& state,
+                   uint32_t threads, uint32_t stage_bytes, uint32_t ctas_per_sm, bool pairs, bool end_combine_allowed,
+                   const ChainParams& chain, int sms, cudaStream_t stream, uint32_t* extra_launches) {
   ChainParams c = chain;
   uint32_t n_stages = (kSmemBudget / ctas_per_sm - 1024) / stage_bytes;
   if (n_stages > kMaxStages) n_stages = kMaxStages;
@@ -1250,11 +1496,10 @@ int launch_planned(void (*kernel)(ChainParams), KernelState& state, uint32_t thr
     if (rc != BOOST_OK) return rc;
     state.configured = true;
   }
-  if (c.n_phases > 1) {
-    // the phases of a chain meet at grid-wide counters: every threadblock must be resident
-    if (state.resident < 1) return BOOST_ERR_UNSUPPORTED;
-    if ((uint32_t)state.resident < ctas_per_sm) ctas_per_sm = (uint32_t)state.resident;
-  }
+  // The phases of a chain, and the threadblocks of a product that combines its tiles at the end,
+  // meet at grid-wide counters: every threadblock must be resident.
+  if (state.resident < 1) return BOOST_ERR_UNSUPPORTED;
+  if ((uint32_t)state.resident < ctas_per_sm) ctas_per_sm = (uint32_t)state.resident;
   const uint32_t max_ctas = (uint32_t)sms * ctas_per_sm;
   uint32_t grid = 0;
   for (uint32_t i = 0; i < c.n_phases; ++i) {
@@ -1276,6 +1521,16 @@ int launch_planned(void (*kernel)(ChainParams), KernelState& state, uint32_t thr
     }
     q.active_ctas = g;
     if (g > grid) grid = g;
+    // Partial sums per row tile, typically: with ten or so (short products cut over the whole
+    // machine) all tiles complete together at the end of the phase, and they are combined then.
+    uint32_t typical_seg = q.splits;
+    if (q.even_part) {
+      const uint32_t units = ((q.n_row_tiles + q.tiles_per_unit - 1) / q.tiles_per_unit) * q.k_blocks;
+      const uint32_t per_cta2 = units / g ? units / g : 1;
+      typical_seg = (q.k_blocks + per_cta2 - 1) / per_cta2;
+    }
+    q.end_combine = (end_combine_allowed && typical_seg >= kEndCombineMinSegments) ? 1u : 0u;
+    q.defer_combine = (q.end_combine && i + 1 == c.n_phases && g_defer_combine) ? 1u : 0u;
   }
   // a chain keeps one grid for all phases: the full machine, so that threadblocks that run
   // out of items in one phase stream ahead in the next
@@ -1290,28 +1545,41 @@ int launch_planned(void (*kernel)(ChainParams), KernelState& state, uint32_t thr
     }
     q.n_host_ctas = n_host_ctas;
   }
-  return boosth::launch_chained(kernel, dim3(grid), dim3(threads), smem, stream, c);
+  int rc = boosth::launch_chained(kernel, dim3(grid), dim3(threads), smem, stream, c);
+  const GemvParams& last = c.ph[c.n_phases - 1];
+  if (rc == BOOST_OK && last.defer_combine) {
+    // one slot per warp where the machine has the warps for it (two small threadblocks per SM)
+    const uint32_t slots = last.n_row_tiles * (last.max_seg <= (x_rows == 32 ? 6u : 5u) ? (last.M_b + 1) / 2 : last.M_b);
+    uint32_t cgrid = (slots + kConsumerWarps - 1) / kConsumerWarps;
+    if (cgrid > 2u * (uint32_t)sms) cgrid = 2u * (uint32_t)sms;
+    if (cgrid == 0) cgrid = 1;
+    rc = boosth::launch_chained(combine_kernel, dim3(cgrid), dim3(kConsumerThreads), 0, stream, last);
+    if (rc == BOOST_OK && extra_launches) ++*extra_launches;
+  }
+  return rc;
 }
+
 
 // Two threadblocks per SM where registers allow: a second ring hides the producer / consumer
 // hand-over latency of the first (measured: +25 % bandwidth on B200).
 template <int NT, int MB>
-int launch_gemv(const ChainParams& chain, int sms, cudaStream_t stream) {
+int launch_gemv(const ChainParams& chain, int sms, cudaStream_t stream, uint32_t* extra_launches) {
   static KernelState states[boosth::kMaxDevices];   // attributes and occupancy are per device
   const int slot = boosth::device_slot();
   if (slot < 0) return BOOST_ERR_CUDA;
   KernelState& state = states[slot];
-  return launch_planned(gemv_tiered_kernel<NT, MB>, state, kGemvThreads, stage_bytes_of(NT, MB), (NT >= 8) ? 1 : 2, false,
-                        chain, sms, stream);
+  return launch_planned(gemv_tiered_kernel<NT, MB>, gemv_combine_kernel<x_rows_of(NT, MB)>, x_rows_of(NT, MB), state, kGemvThreads,
+                        stage_bytes_of(NT, MB), (NT >= 8) ? 1 : 2, false, g_end_combine != 0, chain, sms, stream, extra_launches);
 }
 
 template <uint32_t NPAD>
-int launch_gemv_tc(const ChainParams& chain, int sms, cudaStream_t stream) {
+int launch_gemv_tc(const ChainParams& chain, int sms, cudaStream_t stream, uint32_t* extra_launches) {
   static KernelState states[boosth::kMaxDevices];
   const int slot = boosth::device_slot();
   if (slot < 0) return BOOST_ERR_CUDA;
   KernelState& state = states[slot];
-  return launch_planned(gemv_tc_kernel<NPAD>, state, kTcThreads, tc_stage_bytes(NPAD), 1, true, chain, sms, stream);
+  return launch_planned(gemv_tc_kernel<NPAD>, nullptr, NPAD, state, kTcThreads, tc_stage_bytes(NPAD), 1, true, false, chain, sms, stream,
+                        extra_launches);
 }
 
 }  // namespace
@@ -1486,6 +1754,7 @@ int fill_params(GemvParams& p, const void* const* w_page_ptr, const uint32_t* w_
   p.rope_table = epi ? epi->rope_table : nullptr;
   p.partials = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + header);
   p.n_host_ctas = 0; p.n_stages = 0;
+  p.end_combine = 0;
   return BOOST_OK;
 }
 
@@ -1496,18 +1765,18 @@ int fill_params(GemvParams& p, const void* const* w_page_ptr, const uint32_t* w_
 // every warp.
 uint32_t g_tc_min_batch = 33;
 
-int launch_routed(const ChainParams& c, uint32_t M_b, void* stream) {
+int launch_routed(const ChainParams& c, uint32_t M_b, void* stream, uint32_t* extra_launches = nullptr) {
   const int sms = boosth::sm_count();
   if (sms <= 0) return BOOST_ERR_CUDA;
   cudaStream_t st = (cudaStream_t)stream;
   const bool tc = M_b >= g_tc_min_batch;
   switch (gemv_x_rows(M_b)) {
-    case 1: return launch_gemv<0, 1>(c, sms, st);
-    case 2: return launch_gemv<0, 2>(c, sms, st);
-    case 16: return tc ? launch_gemv_tc<16>(c, sms, st) : launch_gemv<2, 0>(c, sms, st);
-    case 32: return tc ? launch_gemv_tc<32>(c, sms, st) : launch_gemv<4, 0>(c, sms, st);
-    case 64: return tc ? launch_gemv_tc<64>(c, sms, st) : launch_gemv<8, 0>(c, sms, st);
-    default: return tc ? launch_gemv_tc<128>(c, sms, st) : launch_gemv<16, 0>(c, sms, st);
+    case 1: return launch_gemv<0, 1>(c, sms, st, extra_launches);
+    case 2: return launch_gemv<0, 2>(c, sms, st, extra_launches);
+    case 16: return tc ? launch_gemv_tc<16>(c, sms, st, extra_launches) : launch_gemv<2, 0>(c, sms, st, extra_launches);
+    case 32: return tc ? launch_gemv_tc<32>(c, sms, st, extra_launches) : launch_gemv<4, 0>(c, sms, st, extra_launches);
+    case 64: return tc ? launch_gemv_tc<64>(c, sms, st, extra_launches) : launch_gemv<8, 0>(c, sms, st, extra_launches);
+    default: return tc ? launch_gemv_tc<128>(c, sms, st, extra_launches) : launch_gemv<16, 0>(c, sms, st, extra_launches);
   }
 }
 
@@ -1517,19 +1786,19 @@ int boosth::gemv_tiered_launch(const void* const* w_page_ptr, const uint32_t* w_
                                size_t n_host_pages, uint32_t N, uint32_t K, const void* x, uint32_t M_b,
                                void* y, int y_dtype, const void* residual, void* workspace,
                                size_t workspace_bytes, const boost_gemv_epilogue_t* epi,
-                               uint32_t* queue_words, uint32_t header_row_tiles, void* stream) {
+                               uint32_t* queue_words, uint32_t header_row_tiles, void* stream, uint32_t* extra_launches) {
   ChainParams c;
   c.n_phases = 1;
-  c.bar = nullptr;
+  c.bar = static_cast<uint32_t*>(workspace) + kWsBar;   // a lone product's two counters live in the header
   const int rc = fill_params(c.ph[0], w_page_ptr, w_order, n_pages, n_host_pages, N, K, x, M_b, y, y_dtype, residual,
                              workspace, workspace_bytes, epi, queue_words, queue_words != nullptr, header_row_tiles);
   if (rc != BOOST_OK) return rc;
-  return launch_routed(c, M_b, stream);
+  return launch_routed(c, M_b, stream, extra_launches);
 }
 
 int boosth::gemv_chain_launch(const boost_gemv_call_t* calls, uint32_t n_calls, uint32_t M_b, void* workspace,
                               size_t workspace_bytes, uint32_t* sync_words, bool early, uint32_t header_row_tiles,
-                              void* stream) {
+                              void* stream, uint32_t* extra_launches) {
   if (!calls || n_calls == 0 || n_calls > kMaxPhases || !sync_words) return BOOST_ERR_INVALID;
   uint32_t tiles = header_row_tiles;
   for (uint32_t i = 0; i < n_calls; ++i) {
@@ -1538,7 +1807,7 @@ int boosth::gemv_chain_launch(const boost_gemv_call_t* calls, uint32_t n_calls, 
   }
   ChainParams c;
   c.n_phases = n_calls;
-  c.bar = n_calls > 1 ? sync_words + 16 * n_calls : nullptr;
+  c.bar = sync_words + 16 * n_calls;
   for (uint32_t i = 0; i < n_calls; ++i) {
     const boost_gemv_call_t& g = calls[i];
     const int rc = fill_params(c.ph[i], g.w.page_ptr, g.w.order, (size_t)g.w.n_pages, (size_t)g.w.n_host_pages, g.w.N,
@@ -1546,7 +1815,7 @@ int boosth::gemv_chain_launch(const boost_gemv_call_t* calls, uint32_t n_calls, 
                                g.has_epilogue ? &g.epilogue : nullptr, sync_words + 16 * i, early, tiles);
     if (rc != BOOST_OK) return rc;
   }
-  return launch_routed(c, M_b, stream);
+  return launch_routed(c, M_b, stream, extra_launches);
 }
 
 extern "C" size_t boost_gemv_chain_workspace_bytes(const boost_gemv_call_t* calls, uint32_t n_calls, uint32_t M_b) {
@@ -1584,6 +1853,13 @@ extern "C" int boost_gemv_tiered_chain(const boost_gemv_call_t* calls, uint32_t 
 // Routing threshold between the two tensor-core kernels (measurement and tests).
 extern "C" int boost_gemv_set_tc_min_batch(uint32_t m_b) {
   g_tc_min_batch = m_b;
+  return BOOST_OK;
+}
+
+// Where the partial sums of a product are combined (measurement and tests): 1 = at the end of
+// the phase by all threadblocks when a row tile has many (the default), 0 = always tile by tile.
+extern "C" int boost_gemv_set_end_combine(uint32_t on) {
+  g_end_combine = on ? 1u : 0u;
   return BOOST_OK;
 }
 

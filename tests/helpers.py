@@ -84,12 +84,15 @@ def assert_chain_close(got, ref, what="", wide=False):
     assert rel <= CHAIN_REL_TOL, f"{what}: max err / max(|ref|, rms) {rel:.3e}"
 
 
-def assert_bulk_close(got, ref, what="", frac=0.6, tol=2e-3):
+def assert_bulk_close(got, ref, what="", frac=0.6, tol=4e-3):
     """Guard that goes with assert_chain_close on large tensors: its 3e-2 bound is sized for the
     rare output behind a bf16 rounding that fell the other way, so on its own it would also pass
     a result that is a little wrong everywhere.  At least `frac` of the outputs must agree to
-    `tol` of max(|ref|, rms(ref)): one bf16 ulp of an intermediate is 2^-8 = 4e-3 relative, so an
-    output within 2e-3 has no such event of its own size behind it."""
+    `tol` of max(|ref|, rms(ref)).  tol = 4e-3 is one bf16 ulp (2^-8): in the full-size model
+    every output has thousands of bf16 intermediates behind it, a fraction of a percent of which
+    round the other way, and a bf16 output is itself either equal or one ulp off; measured on the
+    Llama-3-8B-shaped layer, 76 - 84 % of the outputs are within 4e-3, 97 - 99 % within 8e-3, all
+    within 1.6e-2 (the small chains of the tests: more than 99.9 % within 4e-3)."""
     import numpy as np
     got = np.asarray(got, dtype=np.float64)
     ref = np.asarray(ref, dtype=np.float64)

@@ -71,6 +71,7 @@ def run_attention(dev, n_seq, hq, hkv, ctx_lens, n_blocks, modulus, seed, churn=
     q_bits = synth.normal_bf16((n_seq, hq, d), 1.0, seed + 2)
     cache = TieredKVCache(pool, hkv, n_blocks, d, dev)
     assert cache.tier.tolist() == ref_pool.page_tiers()
+    assert (int((cache.tier == 1).sum()) > 0) == (modulus > 0)     # a tiered case really has host pages
     cache.load(bf16_tensor(k_bits, dev), bf16_tensor(v_bits, dev))
     back_k, back_v = cache.dump()
     assert np.array_equal(bits_of(back_k), k_bits) and np.array_equal(bits_of(back_v), v_bits)
@@ -118,7 +119,8 @@ def test_attention_config2_after_churn(dev):
 
 @pytest.mark.parametrize("ctx", [[1], [15], [16], [17], [127, 128, 129], [0, 5], [300, 1, 0, 2049]])
 def test_attention_edge_lengths(dev, ctx):
-    out, ref, _ = run_attention(dev, len(ctx), 8, 2, ctx, 512, 4, seed=40 + len(ctx) + ctx[0])
+    # 2048 blocks x 2 KV heads = 8 pages per tensor, modulus 4: the last two in host memory
+    out, ref, _ = run_attention(dev, len(ctx), 8, 2, ctx, 2048, 4, seed=40 + len(ctx) + ctx[0])
     assert_close_to_oracle(out, ref, f"attention ctx={ctx}")
     for b, c in enumerate(ctx):
         if c == 0:
@@ -127,7 +129,8 @@ def test_attention_edge_lengths(dev, ctx):
 
 @pytest.mark.parametrize("hq,hkv,modulus", [(8, 8, 0), (16, 1, 2), (4, 4, 12), (8, 8, 5), (32, 2, 3)])
 def test_attention_head_layouts(dev, hq, hkv, modulus):
-    n_blocks = {1: 512, 2: 512, 4: 1536, 8: 2560}[hkv] if modulus not in (0, 2, 3) else 512
+    # pool sizes that give every tiered case at least one host page (pages = heads * blocks / 512)
+    n_blocks = {(8, 0): 512, (1, 2): 1024, (4, 12): 1536, (8, 5): 2560, (2, 3): 1536}[(hkv, modulus)]
     ctx = [700, 33, 260]
     out, ref, _ = run_attention(dev, 3, hq, hkv, ctx, n_blocks, modulus, seed=hq * 100 + hkv)
     assert_close_to_oracle(out, ref, f"attention hq={hq} hkv={hkv} M={modulus}")
@@ -135,7 +138,8 @@ def test_attention_head_layouts(dev, hq, hkv, modulus):
 
 def test_attention_special_cases(dev):
     # ctx = 1: output is the V row itself (bf16 in, bf16 out: exact)
-    out, ref, _ = run_attention(dev, 4, 8, 2, [1, 1, 1, 1], 512, 4, seed=77)
+    # (2048 blocks x 2 heads = 8 pages, the last two in host memory)
+    out, ref, _ = run_attention(dev, 4, 8, 2, [1, 1, 1, 1], 2048, 4, seed=77)
     assert np.array_equal(out, ref)
 
 

@@ -65,9 +65,10 @@ def test_embed_rmsnorm_swiglu_argmax(dev):
 
 def test_rope_kv_append(dev):
     from paper_2609_13592_b200.tiers import TieredKVCache
-    hq, hkv, d, n_blocks = 8, 2, 128, 512
+    hq, hkv, d, n_blocks = 8, 2, 128, 2048     # 8 pages per tensor, the last two in host memory
     pool = B.KVPool(n_blocks, hkv, 4)
     cache = TieredKVCache(pool, hkv, n_blocks, d, dev)
+    assert int((cache.tier == 1).sum()) == 2
     k0 = synth.normal_bf16((hkv, n_blocks, 16, d), 1.0, 5)
     v0 = synth.normal_bf16((hkv, n_blocks, 16, d), 1.0, 6)
     cache.load(bf16_tensor(k0, dev), bf16_tensor(v0, dev))
@@ -159,7 +160,7 @@ def test_decode_steps_match_oracle(dev, n_seq, kv_modulus, host_weights, recycle
     cfg = dict(synth.TINY_LLAMA)
     w = synth.llama_weights(cfg, seed=n_seq, std=0.02)
     hkv, d, nl = cfg["n_kv_heads"], cfg["head_dim"], cfg["n_layers"]
-    n_pool_blocks, max_blocks = 512, 8
+    n_pool_blocks, max_blocks = 2048, 8      # a K or V tensor is 8 pages: modulus 4 puts 2 on the host, modulus 2 four
     dec = build_decoder(dev, cfg, w, n_pool_blocks, kv_modulus, 0.0, max(n_seq, 4), max_blocks,
                         weight_tier=first_page_on_host if host_weights else None)
     assert all((tw.buf.n_host > 0) == host_weights for tw in all_weights(dec))
@@ -205,7 +206,7 @@ def test_decode_steps_match_oracle(dev, n_seq, kv_modulus, host_weights, recycle
         ctx_pin.numpy()[:] = ctx
         tab_pin.numpy()[:] = table
         n_launch = dec.step_host(tok_pin.numpy(), tab_pin.numpy(), ctx_pin.numpy(), nxt_pin.numpy())
-        assert n_launch == 4 + 2 * nl
+        assert 4 + 2 * nl <= n_launch <= 4 + 3 * nl + 1       # + a combine kernel after a chain whose last product has many partial sums
         ref = od.decode_step(cfg, w, tokens, k_host, v_host, table, ctx)
         logits = dec.buf["logits"][:n_seq].cpu().numpy()
         assert_chain_close(logits, ref["logits"], f"logits step {step}")
@@ -233,6 +234,10 @@ def test_decode_steps_match_oracle(dev, n_seq, kv_modulus, host_weights, recycle
         tokens = ref["next_tokens"].astype(np.int32)       # both sides continue from the oracle's choice
     assert dec.status_words() == [0, 0]
     assert exact_rows >= 0.6 * total_rows, (exact_rows, total_rows)
+    if kv_modulus:
+        # the sequences really read host-tier KV: some of their blocks have a head in host memory
+        info = dec.pool.query()
+        assert info["live_host_chunks"] > 0, info
 
 
 def test_fused_product_epilogues_match_oracle(dev):
@@ -288,9 +293,10 @@ def test_fused_product_epilogues_match_oracle(dev):
     assert_chain_close(act.float().cpu().numpy(), od.silu(gu[:, :ffn]) * gu[:, ffn:], "fused swiglu")
 
     # 3. RoPE + KV append after the QKV product
-    n_blocks = 512
+    n_blocks = 2048                            # 8 pages per tensor, the last two in host memory
     pool = B.KVPool(n_blocks, hkv, 4)
     cache = TieredKVCache(pool, hkv, n_blocks, d, dev)
+    assert int((cache.tier == 1).sum()) == 2
     k0 = synth.normal_bf16((hkv, n_blocks, 16, d), 1.0, 6)
     v0 = synth.normal_bf16((hkv, n_blocks, 16, d), 1.0, 7)
     cache.load(bf16_tensor(k0, dev), bf16_tensor(v0, dev))
@@ -363,7 +369,7 @@ def test_full_size_step_matches_oracle_on_samples(dev):
     tokens = rng.integers(0, vocab, size=n_seq).astype(np.int32)
     nxt = np.zeros(n_seq, np.int32)
     n_launch = dec.step_host(tokens, table, ctx, nxt)
-    assert n_launch == 4 + 2
+    assert 4 + 2 <= n_launch <= 4 + 2 + 2
     assert dec.status_words() == [0, 0]
 
     rows = np.arange(0, vocab, 61)
@@ -431,7 +437,7 @@ def test_config5_launch_shape_matches_oracle_on_samples(dev):
     tokens = np.random.default_rng(6).integers(0, vocab, size=n_seq).astype(np.int32)
     nxt = np.zeros(n_seq, np.int32)
     n_launch = dec.step_host(tokens, table, ctx, nxt)
-    assert n_launch == 4 + 2
+    assert 4 + 2 <= n_launch <= 4 + 2 + 2
     assert dec.status_words() == [0, 0]
 
     rows = np.arange(0, vocab, 61)
@@ -608,7 +614,7 @@ def test_prefetch_variant_matches_tiered_step(dev):
         n0 = decs[0].step(tok[0], table_dev, ctx_dev, nxt[0])
         n1 = decs[1].step_prefetch(tok[1], table_dev, ctx_dev, nxt[1])
         torch.cuda.synchronize()
-        assert n0 == n1 == 4 + 2 * nl
+        assert n0 == n1 and 4 + 2 * nl <= n0 <= 4 + 3 * nl + 1
         assert torch.equal(decs[0].buf["logits"][:n_seq], decs[1].buf["logits"][:n_seq]), step
         assert torch.equal(nxt[0], nxt[1])
         tok = [nxt[0].clone(), nxt[1].clone()]
