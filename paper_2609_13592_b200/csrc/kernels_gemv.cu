@@ -168,7 +168,7 @@ __device__ __forceinline__ float round_bf16(float v) { return __bfloat162float(_
 
 // Second half of a combine pass for one thread: its sums (lo = columns [4 v, 4 v + 4) of batch row m,
 // hi = their partners 64 columns on) are scaled by the row statistics, paired up and stored as the
-// epilogue of the product says (see combine_tile).  Called by whole warps: it shuffles.
+// epilogue of the product says (see combine_units).  Called by whole warps: it shuffles.
 // What the RoPE epilogue reads besides the sums, requested ahead of them by callers that have the
 // registers for it (have = true): the context length, the block-table entry of the new token, the
 // cos / sin pairs.  Otherwise finish_pair loads them itself, after the sums.
@@ -311,9 +311,9 @@ __device__ __forceinline__ void finish_pair(const GemvParams& p, uint32_t row_ti
   }
 }
 
-// Sum the split-K partial sums of one row tile in split order and finish the outputs.
-// Thread -> (batch row m, columns [4 v, 4 v + 4) and their partners 64 columns on): the
-// partners are what SwiGLU (gate / up) and the rotary embedding (d / d + 64) pair up.
+// What a combine does with the sums of a (batch row m, columns [4 v, 4 v + 4) and their partners
+// 64 columns on) - the partners are what SwiGLU (gate / up) and the rotary embedding (d / d + 64)
+// pair up:
 //   plain   y = sum (* row scale) (+ residual); optionally the sum of squares of the bf16
 //           outputs per row, for the RMS scale of the next product;
 //   swiglu  rows 0..63 of the tile are gate rows, 64..127 the matching up rows:
@@ -323,158 +323,15 @@ __device__ __forceinline__ void finish_pair(const GemvParams& p, uint32_t row_ti
 //           into the paged cache at the position of the new token.
 // The row scale is rsqrt(mean(x^2) + eps) from per-tile sums of squares of the rows of x:
 // RMSNorm whose weight has been folded into the packed matrix.
-template <uint32_t kXRows, uint32_t kThreads = kConsumerThreads>
-__device__ __forceinline__ void combine_tile(const GemvParams& p, uint32_t row_tile, uint32_t n_seg, uint32_t tid,
-                                             uint32_t* status) {
-  const float4* base = reinterpret_cast<const float4*>(p.partials + (size_t)row_tile * p.max_seg * kXRows * kBlockRows);
-  constexpr uint32_t kVecRow = kBlockRows / 4;   // float4 per batch row
-  const uint32_t n_pairs = p.M_b * 16;
-  for (uint32_t pidx0 = 0; pidx0 < n_pairs; pidx0 += kThreads) {
-    const uint32_t pidx = pidx0 + tid;
-    const bool valid = pidx < n_pairs;
-    const uint32_t m = valid ? (pidx >> 4) : 0u, v = pidx & 15u;
-    const uint32_t off = m * kVecRow + v;
-    float4 lo = make_float4(0.f, 0.f, 0.f, 0.f), hi = lo;
-    // Everything this thread needs from memory is requested before the first use, so that the
-    // L2 round trips overlap: its share of the row statistics, the residual, the partial sums.
-    float ss = 0.f, ss0 = 0.f, ss1 = 0.f;
-    if (p.ssq_in && valid) {
-      // the 16 threads of row m take every 16th tile each; a butterfly adds the shares
-      if (v < p.ssq_in_tiles) ss0 = __ldcg(p.ssq_in + (size_t)v * p.ssq_stride + m);
-      if (v + 16 < p.ssq_in_tiles) ss1 = __ldcg(p.ssq_in + (size_t)(v + 16) * p.ssq_stride + m);
-      for (uint32_t t0 = v + 32; t0 < p.ssq_in_tiles; t0 += 16) ss += __ldcg(p.ssq_in + (size_t)t0 * p.ssq_stride + m);
-    }
-    const bool vec_out = (p.N & 3u) == 0;   // then n + 3 < N for every n = 4 v' < N
-    uint2 res[2] = {make_uint2(0u, 0u), make_uint2(0u, 0u)};
-    if (valid && p.epi == kEpiPlain && p.residual && vec_out) {
-#pragma unroll
-      for (int half = 0; half < 2; ++half) {
-        const uint32_t n = row_tile * kBlockRows + half * 64 + v * 4;
-        if (n < p.N) res[half] = __ldcg(reinterpret_cast<const uint2*>(p.residual + (size_t)m * p.N + n));   // L2: an earlier phase may have rewritten it
-      }
-    }
-    if (valid) {
-      // four splits (eight independent loads) per round: the L2 latency is paid per round
-      for (uint32_t sp0 = 0; sp0 < n_seg; sp0 += 4) {
-        float4 t0[4], t1[4];
-#pragma unroll
-        for (uint32_t u = 0; u < 4; ++u) {
-          if (sp0 + u < n_seg) {
-            const float4* src = base + (size_t)(sp0 + u) * kXRows * kVecRow + off;
-            t0[u] = __ldcg(src);
-            t1[u] = __ldcg(src + 16);
-          }
-        }
-#pragma unroll
-        for (uint32_t u = 0; u < 4; ++u) {
-          if (sp0 + u < n_seg) {
-            lo.x += t0[u].x; lo.y += t0[u].y; lo.z += t0[u].z; lo.w += t0[u].w;
-            hi.x += t1[u].x; hi.y += t1[u].y; hi.z += t1[u].z; hi.w += t1[u].w;
-          }
-        }
-      }
-    }
-    finish_pair<kXRows>(p, row_tile, m, v, valid, lo, hi, ss, ss0, ss1, res, vec_out, status);
-  }
-}
-
-// The same combine with its passes overlapped, for kernels with registers to spare and many
-// passes per tile (the tcgen05 kernel at 64 and 128 batch rows: 4 and 8 passes of its 256
-// epilogue threads).  What a pass starts with - row statistics, residual, the first four partial
-// sums - is requested one pass ahead, so that its L2 round trip runs under the arithmetic and the
-// stores of the pass before.  Same sums in the same order as combine_tile.
-template <uint32_t kXRows, uint32_t kThreads>
-__device__ __forceinline__ void combine_tile_overlapped(const GemvParams& p, uint32_t row_tile, uint32_t n_seg,
-                                                        uint32_t tid, uint32_t* status) {
-  const float4* base = reinterpret_cast<const float4*>(p.partials + (size_t)row_tile * p.max_seg * kXRows * kBlockRows);
-  constexpr uint32_t kVecRow = kBlockRows / 4;   // float4 per batch row
-  const uint32_t n_pairs = p.M_b * 16;
-  const bool vec_out = (p.N & 3u) == 0;
-  float n_ss0 = 0.f, n_ss1 = 0.f;
-  uint2 n_res[2] = {make_uint2(0u, 0u), make_uint2(0u, 0u)};
-  float4 n0[4], n1[4];
-  auto request = [&](uint32_t pidx0) {
-    const uint32_t pidx = pidx0 + tid;
-    const bool valid = pidx < n_pairs;
-    const uint32_t m = valid ? (pidx >> 4) : 0u, v = pidx & 15u;
-    n_ss0 = n_ss1 = 0.f;
-    n_res[0] = n_res[1] = make_uint2(0u, 0u);
-    if (!valid) return;
-    if (p.ssq_in) {
-      if (v < p.ssq_in_tiles) n_ss0 = __ldcg(p.ssq_in + (size_t)v * p.ssq_stride + m);
-      if (v + 16 < p.ssq_in_tiles) n_ss1 = __ldcg(p.ssq_in + (size_t)(v + 16) * p.ssq_stride + m);
-    }
-    if (p.epi == kEpiPlain && p.residual && vec_out) {
-#pragma unroll
-      for (int half = 0; half < 2; ++half) {
-        const uint32_t n = row_tile * kBlockRows + half * 64 + v * 4;
-        if (n < p.N) n_res[half] = __ldcg(reinterpret_cast<const uint2*>(p.residual + (size_t)m * p.N + n));
-      }
-    }
-    const float4* src = base + m * kVecRow + v;
-#pragma unroll
-    for (uint32_t u = 0; u < 4; ++u) {
-      if (u < n_seg) {
-        n0[u] = __ldcg(src + (size_t)u * kXRows * kVecRow);
-        n1[u] = __ldcg(src + (size_t)u * kXRows * kVecRow + 16);
-      }
-    }
-  };
-  request(0);
-  for (uint32_t pidx0 = 0; pidx0 < n_pairs; pidx0 += kThreads) {
-    const uint32_t pidx = pidx0 + tid;
-    const bool valid = pidx < n_pairs;
-    const uint32_t m = valid ? (pidx >> 4) : 0u, v = pidx & 15u;
-    const uint32_t off = m * kVecRow + v;
-    // this pass's opening loads, then the next pass's go out
-    const float ss0 = n_ss0, ss1 = n_ss1;
-    const uint2 res[2] = {n_res[0], n_res[1]};
-    float4 lo = make_float4(0.f, 0.f, 0.f, 0.f), hi = lo;
-    if (valid) {
-#pragma unroll
-      for (uint32_t u = 0; u < 4; ++u) {
-        if (u < n_seg) {
-          lo.x += n0[u].x; lo.y += n0[u].y; lo.z += n0[u].z; lo.w += n0[u].w;
-          hi.x += n1[u].x; hi.y += n1[u].y; hi.z += n1[u].z; hi.w += n1[u].w;
-        }
-      }
-    }
-    if (pidx0 + kThreads < n_pairs) request(pidx0 + kThreads);
-    float ss = 0.f;
-    if (valid) {
-      if (p.ssq_in)
-        for (uint32_t t0 = v + 32; t0 < p.ssq_in_tiles; t0 += 16) ss += __ldcg(p.ssq_in + (size_t)t0 * p.ssq_stride + m);
-      for (uint32_t sp0 = 4; sp0 < n_seg; sp0 += 4) {
-        float4 t0[4], t1[4];
-#pragma unroll
-        for (uint32_t u = 0; u < 4; ++u) {
-          if (sp0 + u < n_seg) {
-            const float4* src = base + (size_t)(sp0 + u) * kXRows * kVecRow + off;
-            t0[u] = __ldcg(src);
-            t1[u] = __ldcg(src + 16);
-          }
-        }
-#pragma unroll
-        for (uint32_t u = 0; u < 4; ++u) {
-          if (sp0 + u < n_seg) {
-            lo.x += t0[u].x; lo.y += t0[u].y; lo.z += t0[u].z; lo.w += t0[u].w;
-            hi.x += t1[u].x; hi.y += t1[u].y; hi.z += t1[u].z; hi.w += t1[u].w;
-          }
-        }
-      }
-    }
-    finish_pair<kXRows>(p, row_tile, m, v, valid, lo, hi, ss, ss0, ss1, res, vec_out, status);
-  }
-}
-
-// The combine as the mma.sync kernel runs it, warp by warp: one row tile (the threadblock that
+//
+// The combine, warp by warp: one row tile (the threadblock that
 // delivered its last partial sum: first / step = warp index / warps of the threadblock), or all
 // row tiles of a product once every threadblock's partial sums are in memory (the caller has
 // waited for that: first / step = warp index / warps of the whole grid).  A warp takes one slot
 // per pass.  With few partial sums per tile (at most kPer) a slot is two batch rows, one per
 // half-warp, each lane summing all segments of its columns; with many, a slot is one batch row,
 // the half-warps take the even and the odd segments and the sums meet through a shuffle - eight
-// segments per round trip to L2 where the thread-per-row form above takes four.  Lane -> v = lane
+// segments per round trip to L2.  Lane -> v = lane
 // % 16: columns [4 v, 4 v + 4) and their partners 64 on.  Sum order (fixed): ascending within a
 // lane, even segments + odd segments.  Short products (output, down, next qkv) have ten or so
 // partial sums per tile and all their tiles complete together at the end of the phase anyway:
@@ -1084,7 +941,6 @@ __global__ void __launch_bounds__(kTcThreads, 1) gemv_tc_kernel(const __grid_con
   __shared__ uint64_t acc_full[2];
   __shared__ uint64_t acc_empty[2];
   __shared__ uint4 acc_meta[2];
-  __shared__ uint32_t s_old;
   __shared__ uint32_t s_tmem;
   __shared__ uint32_t s_go[2];          // epilogue: thread 0's wait on an accumulator succeeded
   __shared__ volatile uint32_t s_abort; // a bounded wait ran out somewhere: everybody winds down
@@ -1314,11 +1170,16 @@ __global__ void __launch_bounds__(kTcThreads, 1) gemv_tc_kernel(const __grid_con
   }
 
   // -------------------------------------------------------------------- epilogue warps
+  // Each round of the loop takes one accumulator (or phase marker) from the MMA warp and ends
+  // with at most two combines - the row tiles of the accumulator whose last partial sum this
+  // threadblock delivered, or all tiles of a phase at its end - through ONE call of the combine,
+  // so that its code (and register needs) exist once in the kernel.
   uint32_t* tile_cnt = cp.ph[0].ws + kWsHeaderWords;
+  __shared__ uint32_t s_last[2];
   uint32_t buf = 0, buf_phase = 0;
   pdl_wait();
   for (;;) {
-    // thread 0 waits for the accumulator (or marker) and tells the others, so that all 128
+    // thread 0 waits for the accumulator (or marker) and tells the others, so that all 256
     // threads take the same way out if the wait runs out
     if (tid == 0) {
       const bool ok = mbar_wait(&acc_full[buf], buf_phase, status);
@@ -1328,20 +1189,91 @@ __global__ void __launch_bounds__(kTcThreads, 1) gemv_tc_kernel(const __grid_con
     named_barrier_sync(1, kTcEpiThreads);
     if (!s_go[buf]) break;
     const uint4 mt = acc_meta[buf];
-    if (mt.z & (kFlagStop | kFlagPhaseEnd)) {
+    const GemvParams& p = cp.ph[mt.w];
+    const bool phase_end = (mt.z & (kFlagStop | kFlagPhaseEnd)) != 0;
+    uint32_t n_jobs = 0, job[2] = {0u, 0u};   // row tiles to combine, or kAllTiles
+    if (phase_end) {
       if (warp == 0) TRACE(8 + 8 * mt.w + 4);
-      {
-        named_barrier_sync(1, kTcEpiThreads);
+      if (p.end_combine && !p.defer_combine) {
+        // every threadblock's partial sums of this phase in memory -> all tiles combined, by the
+        // epilogue warps of the whole grid (see combine_units)
+        const bool combines = blockIdx.x * kTcEpiWarps < p.n_row_tiles * combine_slots_per_tile<NPAD>(p);
         if (tid == 0) {
-          if (mt.z & kFlagPhaseEnd) {
-            if (blockIdx.x >= skip_arrivals_of(cp.ph[0].ws)) red_add_release(cp.bar + kBarPhase + mt.w, 1u);
-          } else {
-            __threadfence();
-            const uint32_t old = atomicAdd(cp.bar + kBarExit, 1u);
-            if (old == gridDim.x - 1) {
-              for (uint32_t i = 0; i < (n_phases > 1 ? kBarWords : kBarPartials + 1); ++i) cp.bar[i] = 0u;
-              __threadfence();
+          red_add_release(cp.bar + kBarPartials + mt.w, 1u);   // (the barrier above ordered everybody's stores before this)
+          bool ok = true;
+          if (combines && !grid_counter_wait(cp.bar + kBarPartials + mt.w, gridDim.x, status)) { s_abort = 1; ok = false; }
+          s_go[buf] = ok ? 1u : 0u;
+        }
+        named_barrier_sync(1, kTcEpiThreads);
+        if (!s_go[buf]) break;
+        if (combines) job[n_jobs++] = kAllTiles;
+      }
+    } else {
+      tc_fence_after_sync();
+      if (warp == 0) TRACE(8 + 8 * mt.w + 6);
+      const uint32_t split = mt.y;
+      const uint32_t n_tiles = (mt.z & kFlagSecond) ? 2u : 1u;   // row tiles in this accumulator
+      const uint32_t n_seg = p.even_part ? even_part_segments(p, mt.x) : p.splits;
+      const bool direct = (n_seg == 1) && p.epi == kEpiPlain && !p.ssq_in && !p.ssq_out && !p.end_combine;
+      const uint32_t quarter = warp & 3u, half = warp >> 2;
+      const uint32_t nl = quarter * 32 + lane;                                 // weight row of this thread = its TMEM lane
+      // warps 0-3 read the first half of the columns, warps 4-7 the second (16 columns: the first group reads all)
+      constexpr uint32_t kColsPerGroup = NPAD >= 32 ? NPAD / 2 : NPAD;
+      const uint32_t c_begin = half * kColsPerGroup;
+      const uint32_t c_end = (NPAD >= 32 || half == 0) ? c_begin + kColsPerGroup : c_begin;
+      for (uint32_t ti = 0; ti < n_tiles; ++ti) {
+        const uint32_t row_tile = mt.x + ti;
+        float* part = p.partials + ((size_t)row_tile * p.max_seg + split) * NPAD * kBlockRows;
+        const uint32_t taddr = tmem_base + ((quarter * 32u) << 16) + buf * 2 * NPAD + ti * NPAD;
+        for (uint32_t c0 = c_begin; c0 < c_end; c0 += 16) {
+          float v[16];
+          tmem_ld16(taddr + c0, v);
+#pragma unroll
+          for (uint32_t j = 0; j < 16; ++j) {
+            const uint32_t m = c0 + j;                                         // batch row = accumulator column
+            if (direct) {
+              const uint32_t n = row_tile * kBlockRows + nl;
+              if (m < p.M_b && n < p.N) store_out(p, m, n, v[j]);
+            } else {
+              __stcg(part + m * kBlockRows + nl, v[j]);
             }
+          }
+        }
+      }
+      // the accumulators may be overwritten
+      tc_fence_before_sync();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&acc_empty[buf]);
+      if (++buf == 2) { buf = 0; buf_phase ^= 1u; }
+      if (!direct && !p.end_combine) {
+        // the threadblock that delivers the last partial sum of a row tile combines it
+        named_barrier_sync(1, kTcEpiThreads);
+        if (tid < n_tiles) s_last[tid] = atom_add_acq_rel(tile_cnt + mt.x + tid, 1u) == n_seg - 1 ? 1u : 0u;   // release ours, acquire the others'
+        named_barrier_sync(1, kTcEpiThreads);
+        for (uint32_t ti = 0; ti < n_tiles; ++ti)
+          if (s_last[ti]) job[n_jobs++] = mt.x + ti;
+      }
+    }
+    for (uint32_t j = 0; j < n_jobs; ++j) {
+      const bool all = job[j] == kAllTiles;
+      __threadfence();
+      combine_units<NPAD>(p, all ? blockIdx.x * kTcEpiWarps + warp : warp, all ? gridDim.x * kTcEpiWarps : kTcEpiWarps, job[j], lane,
+                          status);
+      if (!all && tid == 0) tile_cnt[job[j]] = 0;
+      if (warp == 0) TRACE(8 + 8 * mt.w + 5);
+    }
+    if (n_jobs && !phase_end) named_barrier_sync(1, kTcEpiThreads);   // (s_last may be rewritten, the tiles' slots reused)
+    if (phase_end) {
+      named_barrier_sync(1, kTcEpiThreads);
+      if (tid == 0) {
+        if (mt.z & kFlagPhaseEnd) {
+          if (blockIdx.x >= skip_arrivals_of(cp.ph[0].ws)) red_add_release(cp.bar + kBarPhase + mt.w, 1u);
+        } else {
+          __threadfence();
+          const uint32_t old = atomicAdd(cp.bar + kBarExit, 1u);
+          if (old == gridDim.x - 1) {
+            for (uint32_t i = 0; i < (n_phases > 1 ? kBarWords : kBarPartials + 1); ++i) cp.bar[i] = 0u;
+            __threadfence();
           }
         }
       }
@@ -1349,66 +1281,6 @@ __global__ void __launch_bounds__(kTcThreads, 1) gemv_tc_kernel(const __grid_con
       if (lane == 0) mbar_arrive(&acc_empty[buf]);
       if (++buf == 2) { buf = 0; buf_phase ^= 1u; }
       if (mt.z & kFlagStop) break;
-      continue;
-    }
-    tc_fence_after_sync();
-    if (warp == 0) TRACE(8 + 8 * mt.w + 6);
-    const GemvParams& p = cp.ph[mt.w];
-    const uint32_t split = mt.y;
-    const uint32_t n_tiles = (mt.z & kFlagSecond) ? 2u : 1u;   // row tiles in this accumulator
-    uint32_t n_seg = p.splits;
-    if (p.even_part) {
-      const uint32_t tpu = p.tiles_per_unit;
-      const uint32_t T2 = ((p.n_row_tiles + tpu - 1) / tpu) * p.k_blocks;
-      const uint64_t u0 = (uint64_t)(mt.x / tpu) * p.k_blocks;
-      n_seg = part_owner(u0 + p.k_blocks - 1, p.active_ctas, T2) - part_owner(u0, p.active_ctas, T2) + 1;
-    }
-    const bool direct = (n_seg == 1) && p.epi == kEpiPlain && !p.ssq_in && !p.ssq_out;
-    const uint32_t quarter = warp & 3u, half = warp >> 2;
-    const uint32_t nl = quarter * 32 + lane;                                 // weight row of this thread = its TMEM lane
-    // warps 0-3 read the first half of the columns, warps 4-7 the second (16 columns: the first group reads all)
-    constexpr uint32_t kColsPerGroup = NPAD >= 32 ? NPAD / 2 : NPAD;
-    const uint32_t c_begin = half * kColsPerGroup;
-    const uint32_t c_end = (NPAD >= 32 || half == 0) ? c_begin + kColsPerGroup : c_begin;
-    for (uint32_t ti = 0; ti < n_tiles; ++ti) {
-      const uint32_t row_tile = mt.x + ti;
-      float* part = p.partials + ((size_t)row_tile * p.max_seg + split) * NPAD * kBlockRows;
-      const uint32_t taddr = tmem_base + ((quarter * 32u) << 16) + buf * 2 * NPAD + ti * NPAD;
-      for (uint32_t c0 = c_begin; c0 < c_end; c0 += 16) {
-        float v[16];
-        tmem_ld16(taddr + c0, v);
-#pragma unroll
-        for (uint32_t j = 0; j < 16; ++j) {
-          const uint32_t m = c0 + j;                                         // batch row = accumulator column
-          if (direct) {
-            const uint32_t n = row_tile * kBlockRows + nl;
-            if (m < p.M_b && n < p.N) store_out(p, m, n, v[j]);
-          } else {
-            __stcg(part + m * kBlockRows + nl, v[j]);
-          }
-        }
-      }
-    }
-    // the accumulators may be overwritten
-    tc_fence_before_sync();
-    __syncwarp();
-    if (lane == 0) mbar_arrive(&acc_empty[buf]);
-    if (++buf == 2) { buf = 0; buf_phase ^= 1u; }
-    if (!direct) {
-      for (uint32_t ti = 0; ti < n_tiles; ++ti) {
-        const uint32_t row_tile = mt.x + ti;
-        named_barrier_sync(1, kTcEpiThreads);
-        if (tid == 0) s_old = atom_add_acq_rel(tile_cnt + row_tile, 1u);   // release the partial sums, acquire the others'
-        named_barrier_sync(1, kTcEpiThreads);
-        if (s_old == n_seg - 1) {
-          __threadfence();
-          if constexpr (NPAD >= 64) combine_tile_overlapped<NPAD, kTcEpiThreads>(p, row_tile, n_seg, tid, status);
-          else combine_tile<NPAD, kTcEpiThreads>(p, row_tile, n_seg, tid, status);
-          if (tid == 0) tile_cnt[row_tile] = 0;
-          if (warp == 0) TRACE(8 + 8 * mt.w + 5);
-        }
-        named_barrier_sync(1, kTcEpiThreads);
-      }
     }
   }
   named_barrier_sync(2, kTcEpiThreads + 32);
@@ -1578,8 +1450,8 @@ int launch_gemv_tc(const ChainParams& chain, int sms, cudaStream_t stream, uint3
   const int slot = boosth::device_slot();
   if (slot < 0) return BOOST_ERR_CUDA;
   KernelState& state = states[slot];
-  return launch_planned(gemv_tc_kernel<NPAD>, nullptr, NPAD, state, kTcThreads, tc_stage_bytes(NPAD), 1, true, false, chain, sms, stream,
-                        extra_launches);
+  return launch_planned(gemv_tc_kernel<NPAD>, gemv_combine_kernel<NPAD>, NPAD, state, kTcThreads, tc_stage_bytes(NPAD), 1, true,
+                        g_end_combine != 0, chain, sms, stream, extra_launches);
 }
 
 }  // namespace
