@@ -477,14 +477,17 @@ __global__ void __launch_bounds__(kGemvThreads, (NT >= 8 ? 1 : 2)) gemv_tiered_k
     // Two warps, because a lone warp's instruction latency would cap the fill rate.
     const bool leader = (warp == kConsumerWarps);
     uint32_t stage = 0, phase = 0, icount = 0;
-    // Leaving after a timeout: this warp's own copies must have landed first (a few microseconds
-    // for a block from the host tier; the wait is bounded all the same).
+    // Leaving after a timeout: this warp's own copies into the ring must have landed before the
+    // threadblock's shared memory goes away.  The cp.async fans can be waited for; a bulk copy
+    // reports only to its stage's barrier, which in this situation may never complete, so the
+    // weight warp allows a grace period far longer than a copy takes (16 KiB from HBM: about a
+    // microsecond, over the host link: a few) - and in practice it got here through a wait that
+    // had already lasted the whole limit.
     auto leave = [&]() {
       cp_async_wait_all();
-      if (leader && lane == 0) {
+      if (leader) {
         const long long t0 = clock64();
-        for (uint32_t s = 0; s < n_stages; ++s)
-          while (!mbar_try_wait(&full_bar[s], 0u) && !mbar_try_wait(&full_bar[s], 1u) && clock64() - t0 < 200000) {}
+        while (clock64() - t0 < 100000) __nanosleep(1000);   // ~50 us
       }
       __syncwarp();
     };
