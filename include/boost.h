@@ -116,6 +116,45 @@ typedef struct {
 int boost_wave_stats(const uint8_t* tier /*host*/, size_t n_pages, size_t tile_bytes,
                      uint32_t ctas_per_wave, double host_ratio, boost_wave_stats_t* out /*host*/);
 
+/* ---- The schedule a kernel realised (Sec. 2.6, Sec. 3.1: the host share of every wave is what
+ * placement is about; Sec. 3.2: with threadblocks specialised by tier it is the hand-out order,
+ * not the address order, that decides it).  The tier-aware kernels hand out host-tier work first
+ * from queues of their own, so what each wave of work, and each stretch of time, really read from
+ * which tier is a property of the run.  Opt-in: put the device address of a log buffer into words
+ * 6 and 7 (one 64-bit value) of a kernel's zero-filled workspace header before the launch; every
+ * work item then appends one record.  Log buffer: boost_schedule_log_bytes(capacity) bytes of
+ * device memory, zero-filled, with the capacity stored in its second 64-bit word (the first
+ * counts the records claimed; more than the capacity means records were dropped).  The decode
+ * step's products share one workspace, its attention kernels another. */
+#define BOOST_SCHED_KIND_STREAM 1u /* stream reduce: a 128 KiB tile */
+#define BOOST_SCHED_KIND_GEMV 2u   /* weight product: a queue item, or a threadblock's segment of a row tile */
+#define BOOST_SCHED_KIND_ATTN 3u   /* attention: one warp's quarter of a run of KV blocks */
+typedef struct {
+  uint32_t kind_phase;  /* BOOST_SCHED_KIND_* | (phase of a chain << 8) */
+  uint32_t cta_warp;    /* threadblock | (warp << 24) */
+  uint32_t bytes;       /* bytes the item streams */
+  uint32_t host_bytes;  /* of which from host-tier pages */
+  uint64_t t_request;   /* GPU global timer (ns) when the item's first byte was requested */
+  uint64_t t_consumed;  /* ... when its last byte had been consumed; 0 = never finished */
+} boost_schedule_record_t;
+size_t boost_schedule_log_bytes(size_t capacity);
+/* Statistics of a log copied to host memory (log = the whole buffer, header included).
+ *   kind             only records of this BOOST_SCHED_KIND_* (0 = all);
+ *   items_per_wave   records are ordered by t_request (ties: cta_warp, then kind_phase) and cut
+ *                    into waves of this many consecutive starts; a wave's host share is its
+ *                    host_bytes / bytes -> wave_out (n_over_waves counts shares above host_ratio);
+ *   window_ns        the time from the first request to the last consumption is cut into windows
+ *                    of this length; a record's bytes are spread evenly over [t_request,
+ *                    t_consumed] (at least 1 ns) and a window's host share is host / all bytes
+ *                    that fall into it; windows without traffic are left out -> window_out;
+ *   n_records_out    records that passed the filter (unfinished ones are skipped).
+ * n_host_pages of the outputs holds the number of records with host_bytes > 0.
+ * Errors: INVALID (null pointers, zero items_per_wave or window_ns, a log shorter than its
+ * header says). */
+int boost_schedule_stats(const void* log /*host*/, size_t log_bytes, uint32_t kind, uint32_t items_per_wave,
+                         uint64_t window_ns, double host_ratio, boost_wave_stats_t* wave_out /*host*/,
+                         boost_wave_stats_t* window_out /*host*/, uint64_t* n_records_out /*host*/);
+
 /* Visit order for tier-specialised kernels: host pages first (ascending), then HBM pages
  * (ascending).  Each threadblock works on one tier at a time (Sec. 3.2); handing out the
  * slow tier's pages first keeps both tiers busy for the whole kernel.

@@ -168,3 +168,63 @@ def wave_stats(tier, tile_bytes, ctas_per_wave, host_ratio):
         out.update(mean=float(mean), var=float(var),
                    min=float(min(fractions)), max=float(max(fractions)))
     return out
+
+
+def schedule_stats(records, items_per_wave, window_ns, host_ratio, kind=0):
+    """Host share per wave of work and per stretch of time, of a schedule a kernel realised.
+
+    Sec. 2.6 and Sec. 3.1 judge a placement by the host share of every wave; with threadblocks
+    specialised by tier (Sec. 3.2) the order in which work is handed out, not the address order,
+    decides that share, so it is computed from a log of the run: `records` is a sequence of
+    (kind_phase, cta_warp, bytes, host_bytes, t_request, t_consumed) tuples of integers.
+
+    Waves: records ordered by (t_request, cta_warp, kind_phase) and cut into groups of
+    items_per_wave consecutive starts; share = host bytes / bytes of the group.
+    Windows: the time from the first request to the last consumption in windows of window_ns; a
+    record's bytes are spread evenly over [t_request, max(t_consumed, t_request + 1)); share =
+    host bytes / bytes that fall into the window; windows without traffic are left out.
+    Unfinished (t_consumed == 0) and empty records are skipped; kind != 0 keeps only records
+    whose kind_phase & 0xFF equals it.  Exact rational arithmetic.  Returns (waves, windows,
+    n_records), the first two shaped like wave_stats()."""
+    if items_per_wave <= 0 or window_ns <= 0:
+        raise ValueError("items_per_wave and window_ns must be positive")
+    recs = [r for r in records if (not kind or (r[0] & 0xFF) == kind) and r[5] != 0 and r[2] != 0]
+    recs.sort(key=lambda r: (r[4], r[1], r[0]))
+    n_host_items = sum(1 for r in recs if r[3] > 0)
+    target = Fraction(host_ratio) * (1 + _RATIO_SLACK)
+
+    def summary(shares):
+        n = len(shares)
+        out = {"n_waves": n, "n_host_pages": n_host_items,
+               "n_zero_waves": sum(1 for f in shares if f == 0),
+               "n_over_waves": sum(1 for f in shares if f > target),
+               "mean": 0.0, "var": 0.0, "min": 0.0, "max": 0.0}
+        if n:
+            mean = sum(shares, Fraction(0)) / n
+            var = sum(((f - mean) ** 2 for f in shares), Fraction(0)) / n
+            out.update(mean=float(mean), var=float(var), min=float(min(shares)), max=float(max(shares)))
+        return out
+
+    waves = []
+    for i in range(0, len(recs), items_per_wave):
+        group = recs[i:i + items_per_wave]
+        waves.append(Fraction(sum(r[3] for r in group), sum(r[2] for r in group)))
+    windows = []
+    if recs:
+        t0 = recs[0][4]
+        ends = [max(r[5], r[4] + 1) for r in recs]
+        n_win = -(-(max(ends) - t0) // window_ns)
+        host = [Fraction(0)] * n_win
+        total = [Fraction(0)] * n_win
+        for r, end in zip(recs, ends):
+            a, e = r[4] - t0, end - t0
+            w = a // window_ns
+            while w * window_ns < e:
+                lo, hi = max(w * window_ns, a), min((w + 1) * window_ns, e)
+                part = Fraction(hi - lo, e - a)
+                host[w] += part * r[3]
+                total[w] += part * r[2]
+                w += 1
+        windows = [h / t for h, t in zip(host, total) if t > 0]
+    return summary(waves), summary(windows), len(recs)
+

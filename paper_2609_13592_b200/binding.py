@@ -147,6 +147,8 @@ SIGNATURES = {
     "boost_rope_table": (_int, [_vp, _u32, _u32, _flt, _vp, _vp]),
     "boost_swiglu": (_int, [_vp, _u32, _u32, _vp, _vp]),
     "boost_argmax": (_int, [_vp, _u32, _u32, _vp, _vp]),
+    "boost_schedule_log_bytes": (C.c_size_t, [C.c_size_t]),
+    "boost_schedule_stats": (_int, [_vp, C.c_size_t, _u32, _u32, C.c_uint64, C.c_double, _vp, _vp, _vp]),
     "boost_gemv_set_tc_min_batch": (_int, [_u32]),
     "boost_gemv_set_end_combine": (_int, [_u32]),
     "boost_gemv_chain_workspace_bytes": (C.c_size_t, [_vp, _u32, _u32]),
@@ -406,6 +408,35 @@ def gemv_calls(calls):
 
 def boost_gemv_set_tc_min_batch(m_b):
     _check(lib().boost_gemv_set_tc_min_batch(m_b), "boost_gemv_set_tc_min_batch")
+
+
+SCHED_KIND_STREAM, SCHED_KIND_GEMV, SCHED_KIND_ATTN = 1, 2, 3
+WS_WAIT_LIMIT_WORD, WS_SKIP_ARRIVALS_WORD, WS_LOG_WORD = 4, 5, 6
+SCHED_RECORD_DTYPE = np.dtype([("kind_phase", "<u4"), ("cta_warp", "<u4"), ("bytes", "<u4"), ("host_bytes", "<u4"),
+                               ("t_request", "<u8"), ("t_consumed", "<u8")])
+
+
+def boost_schedule_log_bytes(capacity):
+    return int(lib().boost_schedule_log_bytes(capacity))
+
+
+def schedule_records(log_host):
+    """Records of a schedule log copied to the host (numpy uint8 array of the whole buffer) as a
+    structured array, and the number of records the kernels tried to write."""
+    head = log_host[:32].view("<u8")
+    claimed, capacity = int(head[0]), int(head[1])
+    n = min(claimed, capacity)
+    return log_host[32:32 + n * SCHED_RECORD_DTYPE.itemsize].view(SCHED_RECORD_DTYPE), claimed
+
+
+def boost_schedule_stats(log_host, kind, items_per_wave, window_ns, host_ratio):
+    """log_host: numpy uint8 array holding the whole log buffer -> (waves, windows, n_records)."""
+    log_host = np.ascontiguousarray(log_host, dtype=np.uint8)
+    waves, windows, n = WaveStats(), WaveStats(), C.c_uint64(0)
+    _check(lib().boost_schedule_stats(log_host.ctypes.data, log_host.size, kind, items_per_wave, window_ns, host_ratio,
+                                      C.addressof(waves), C.addressof(windows), C.addressof(n)), "boost_schedule_stats")
+    as_dict = lambda st: {f: getattr(st, f) for f, _ in WaveStats._fields_}
+    return as_dict(waves), as_dict(windows), int(n.value)
 
 
 def boost_gemv_set_end_combine(on):

@@ -21,6 +21,7 @@ enum : uint32_t {
   kWsWaitLimit = 4,     // bounded waits give up after this many cycles instead of kWaitLimitCycles
   kWsSkipArrivals = 5,  // honoured only with a non-zero kWsWaitLimit: threadblocks [0, n) leave out their
                         // phase-boundary arrival, so that the others' waits run out (test of the wind-down)
+  kWsLog = 6,           // two words: device address of a schedule log (boost_schedule_log_*), 0 = none
   kWsBar = 8,       // a weight product launched alone keeps its two grid-wide counters here
   kWsHeaderWords = 16
 };
@@ -254,6 +255,47 @@ __device__ __forceinline__ void mma_bf16_16816(float (&d)[4], const uint32_t (&a
       "{%0,%1,%2,%3};"
       : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
       : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+
+// ---- Schedule log (opt-in; see boost_schedule_stats).  The host puts the device address of a
+// log buffer into words kWsLog, kWsLog + 1 of a kernel's workspace header; the kernel then
+// appends one record per work item: who streamed how many bytes of which tier, from the moment
+// its first byte was requested to the moment its last byte had been consumed.  Buffer layout:
+// uint64 count (records claimed so far, may exceed the capacity), uint64 capacity, two unused
+// uint64, then the records.
+struct SchedRecord {
+  uint32_t kind_phase;   // BOOST_SCHED_KIND_* | phase of a chain << 8
+  uint32_t cta_warp;     // threadblock | warp << 24
+  uint32_t bytes;        // bytes of the item
+  uint32_t host_bytes;   // of which from host-tier pages
+  unsigned long long t_request;    // global timer, ns
+  unsigned long long t_consumed;   // global timer, ns; 0 while the item is in flight
+};
+constexpr uint32_t kNoRecord = 0xFFFFFFu;   // record indices travel in 24 bits
+
+__device__ __forceinline__ unsigned long long global_time_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+__device__ __forceinline__ unsigned long long* sched_log_of(const uint32_t* ws) {
+  return reinterpret_cast<unsigned long long*>(*reinterpret_cast<const unsigned long long*>(ws + kWsLog));
+}
+// Claim a record and fill in everything but the end time.  One thread.  Returns kNoRecord when
+// there is no log or it is full.
+__device__ __forceinline__ uint32_t sched_log_begin(unsigned long long* log, uint32_t kind_phase, uint32_t cta_warp,
+                                                    uint32_t bytes, uint32_t host_bytes) {
+  if (!log) return kNoRecord;
+  const unsigned long long idx = atomicAdd(log, 1ull);
+  if (idx >= log[1] || idx >= kNoRecord) return kNoRecord;
+  SchedRecord* r = reinterpret_cast<SchedRecord*>(log + 4) + idx;
+  r->kind_phase = kind_phase; r->cta_warp = cta_warp; r->bytes = bytes; r->host_bytes = host_bytes;
+  r->t_consumed = 0ull;
+  r->t_request = global_time_ns();
+  return (uint32_t)idx;
+}
+__device__ __forceinline__ void sched_log_end(unsigned long long* log, uint32_t idx) {
+  if (log && idx != kNoRecord) (reinterpret_cast<SchedRecord*>(log + 4) + idx)->t_consumed = global_time_ns();
 }
 
 // Two work queues: threadblocks with `host_first` take items of the host-tier queue

@@ -2,7 +2,9 @@
 // page-pointer tables.  Integer logic only; no CUDA calls in this file.
 #include <cmath>
 #include <cstdint>
+#include <algorithm>
 #include <cstring>
+#include <vector>
 #include <limits>
 
 #include "../../include/boost.h"
@@ -203,3 +205,102 @@ extern "C" int boost_page_table(const uint8_t* tier, size_t n_pages, void* hbm_s
   }
   return BOOST_OK;
 }
+
+// ---- statistics of a schedule log (see boost.h)
+
+extern "C" size_t boost_schedule_log_bytes(size_t capacity) {
+  return 32 + capacity * sizeof(boost_schedule_record_t);
+}
+
+namespace {
+
+struct ShareStats {
+  uint64_t n = 0, n_zero = 0, n_over = 0;
+  std::vector<double> f;
+  void add(double host, double all, double slack) {
+    const double v = host / all;
+    f.push_back(v);
+    ++n;
+    if (host == 0.0) ++n_zero;
+    if (v > slack) ++n_over;
+  }
+  void fill(boost_wave_stats_t* out, uint64_t n_host_items) const {
+    std::memset(out, 0, sizeof(*out));
+    out->n_waves = n;
+    out->n_host_pages = n_host_items;
+    out->n_zero_waves = n_zero;
+    out->n_over_waves = n_over;
+    if (!n) return;
+    double sum = 0.0, mn = f[0], mx = f[0];
+    for (double v : f) { sum += v; mn = v < mn ? v : mn; mx = v > mx ? v : mx; }
+    const double mean = sum / (double)n;
+    double dev = 0.0;
+    for (double v : f) dev += (v - mean) * (v - mean);
+    out->mean = mean; out->var = dev / (double)n; out->min = mn; out->max = mx;
+  }
+};
+
+}  // namespace
+
+extern "C" int boost_schedule_stats(const void* log, size_t log_bytes, uint32_t kind, uint32_t items_per_wave,
+                                    uint64_t window_ns, double host_ratio, boost_wave_stats_t* wave_out,
+                                    boost_wave_stats_t* window_out, uint64_t* n_records_out) {
+  if (!log || !wave_out || !window_out || !n_records_out || items_per_wave == 0 || window_ns == 0) return BOOST_ERR_INVALID;
+  if (log_bytes < 32 || !(host_ratio >= 0.0)) return BOOST_ERR_INVALID;
+  const uint64_t* head = static_cast<const uint64_t*>(log);
+  const uint64_t claimed = head[0], capacity = head[1];
+  const uint64_t n_all = claimed < capacity ? claimed : capacity;
+  if (log_bytes < 32 + n_all * sizeof(boost_schedule_record_t)) return BOOST_ERR_INVALID;
+  const boost_schedule_record_t* rec = reinterpret_cast<const boost_schedule_record_t*>(head + 4);
+  std::vector<const boost_schedule_record_t*> r;
+  for (uint64_t i = 0; i < n_all; ++i) {
+    if (kind && (rec[i].kind_phase & 0xFFu) != kind) continue;
+    if (rec[i].t_consumed == 0 || rec[i].bytes == 0) continue;
+    r.push_back(rec + i);
+  }
+  std::sort(r.begin(), r.end(), [](const boost_schedule_record_t* a, const boost_schedule_record_t* b) {
+    if (a->t_request != b->t_request) return a->t_request < b->t_request;
+    if (a->cta_warp != b->cta_warp) return a->cta_warp < b->cta_warp;
+    return a->kind_phase < b->kind_phase;
+  });
+  *n_records_out = r.size();
+  uint64_t n_host_items = 0;
+  for (const auto* x : r) n_host_items += x->host_bytes > 0;
+  const double slack = host_ratio * (1.0 + std::ldexp(1.0, -40));
+  // waves of consecutive starts
+  ShareStats waves;
+  for (size_t i = 0; i < r.size(); i += items_per_wave) {
+    uint64_t host = 0, all = 0;
+    for (size_t j = i; j < r.size() && j < i + items_per_wave; ++j) { host += r[j]->host_bytes; all += r[j]->bytes; }
+    waves.add((double)host, (double)all, slack);
+  }
+  waves.fill(wave_out, n_host_items);
+  // time windows: a record's bytes spread evenly over its interval
+  ShareStats windows;
+  if (!r.empty()) {
+    uint64_t t0 = r[0]->t_request, t1 = 0;
+    for (const auto* x : r) {
+      const uint64_t e = x->t_consumed > x->t_request ? x->t_consumed : x->t_request + 1;
+      t1 = e > t1 ? e : t1;
+    }
+    const uint64_t n_win = (t1 - t0 + window_ns - 1) / window_ns;
+    std::vector<double> host(n_win, 0.0), all(n_win, 0.0);
+    for (const auto* x : r) {
+      const uint64_t a = x->t_request - t0;
+      const uint64_t e = (x->t_consumed > x->t_request ? x->t_consumed : x->t_request + 1) - t0;
+      const double dur = (double)(e - a);
+      for (uint64_t w = a / window_ns; w * window_ns < e; ++w) {
+        const uint64_t lo = w * window_ns > a ? w * window_ns : a;
+        const uint64_t hi = (w + 1) * window_ns < e ? (w + 1) * window_ns : e;
+        const double part = (double)(hi - lo) / dur;
+        host[w] += part * (double)x->host_bytes;
+        all[w] += part * (double)x->bytes;
+      }
+    }
+    for (uint64_t w = 0; w < n_win; ++w)
+      if (all[w] > 0.0) windows.add(host[w], all[w], slack);
+  }
+  windows.fill(window_out, n_host_items);
+  return BOOST_OK;
+}
+

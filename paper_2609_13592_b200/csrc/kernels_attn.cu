@@ -275,6 +275,15 @@ __global__ void __launch_bounds__(kAttnThreads, (NH == 1 ? 3 : 2)) paged_attn_ke
         }
         cp_async_arrive_noinc(&full_bar[warp][st]);
       };
+      // schedule log (opt-in): one record per warp and item, the warp's quarter of the run
+      uint32_t rec = kNoRecord;
+      if (nb) {
+        const uint32_t host_blocks = __popc(__ballot_sync(0xFFFFFFFFu, (host_bits & 1u) != 0)) +
+                                     __popc(__ballot_sync(0xFFFFFFFFu, (host_bits & 2u) != 0));
+        if (lane == 0)
+          rec = sched_log_begin(sched_log_of(p.ws), BOOST_SCHED_KIND_ATTN, blockIdx.x | (warp << 24), nb * kStageBytes,
+                                host_blocks * kStageBytes);
+      }
       const uint32_t n_first = min(nb, kWarpStages);
       const bool early = !waited && blk0 + n_first + 1 <= n_blk;   // none of them is the last block
       if (early)
@@ -397,6 +406,7 @@ __global__ void __launch_bounds__(kAttnThreads, (NH == 1 ? 3 : 2)) paged_attn_ke
         __syncwarp();
         if (i + kWarpStages < nb) request(i + kWarpStages);
       }
+      if (lane == 0 && rec != kNoRecord) sched_log_end(sched_log_of(p.ws), rec);
 
       ATRACE(3);
       // ---- end of the run: the four warps' (m, l, O) meet in shared memory.  Each warp parks

@@ -477,6 +477,8 @@ __global__ void __launch_bounds__(kGemvThreads, (NT >= 8 ? 1 : 2)) gemv_tiered_k
     // Two warps, because a lone warp's instruction latency would cap the fill rate.
     const bool leader = (warp == kConsumerWarps);
     uint32_t stage = 0, phase = 0, icount = 0;
+    unsigned long long* const sched_log = (leader && lane == 0) ? sched_log_of(cp.ph[0].ws) : nullptr;
+    uint32_t rec = kNoRecord;   // schedule-log record of the item in production (weight warp, lane 0)
     // Leaving after a timeout: this warp's own copies into the ring must have landed before the
     // threadblock's shared memory goes away.  The cp.async fans can be waited for; a bulk copy
     // reports only to its stage's barrier, which in this situation may never complete, so the
@@ -535,7 +537,10 @@ __global__ void __launch_bounds__(kGemvThreads, (NT >= 8 ? 1 : 2)) gemv_tiered_k
                   page_base = static_cast<const uint8_t*>(p.w_page_ptr[page_of_base]);
                 }
                 const uint8_t* src = page_base + (size_t)(b % kBlocksPerPage) * kBlockBytes;
-                meta[stage] = make_uint4(row_tile, seg, (seg_first ? kFlagFirst : 0u) | (seg_last ? kFlagLast : 0u), ph);
+                if (seg_first)   // the segment: blocks up to the end of the row tile or of this threadblock's range
+                  rec = sched_log_begin(sched_log, BOOST_SCHED_KIND_GEMV | (ph << 8), blockIdx.x | (warp << 24),
+                                        min(b1 - b, p.k_blocks - kb) * kBlockBytes, 0u);
+                meta[stage] = make_uint4(row_tile, seg, (seg_first ? kFlagFirst : 0u) | (seg_last ? kFlagLast : 0u) | (rec << 8), ph);
                 mbar_arrive_expect_tx(&full_bar[stage], kBlockBytes);
                 bulk_copy_g2s(wdst, src, kBlockBytes, &full_bar[stage]);
               }
@@ -599,8 +604,11 @@ __global__ void __launch_bounds__(kGemvThreads, (NT >= 8 ? 1 : 2)) gemv_tiered_k
             // (the other lanes must not run ahead of lane 0's wait on the stage)
             if (!lane0_wait(&empty_bar[stage], phase ^ 1u)) { leave(); return; }
             if (lane == 0) {
+              if (j == 0)
+                rec = sched_log_begin(sched_log, BOOST_SCHED_KIND_GEMV | (ph << 8), blockIdx.x | (warp << 24),
+                                      p.run * kBlockBytes, from_host ? p.run * kBlockBytes : 0u);
               meta[stage] = make_uint4(row_tile, kb0 / p.run,
-                                       (j == 0 ? kFlagFirst : 0u) | (j + 1 == p.run ? kFlagLast : 0u), ph);
+                                       (j == 0 ? kFlagFirst : 0u) | (j + 1 == p.run ? kFlagLast : 0u) | (rec << 8), ph);
               mbar_arrive_expect_tx(&full_bar[stage], from_host ? 0u : kBlockBytes);
               if (!from_host) bulk_copy_g2s(wdst, src, kBlockBytes, &full_bar[stage]);
             }
@@ -758,6 +766,7 @@ __global__ void __launch_bounds__(kGemvThreads, (NT >= 8 ? 1 : 2)) gemv_tiered_k
 
     if (mt.z & kFlagLast) {
       if (warp == 0) TRACE(8 + 8 * mt.w + 6);
+      if (warp == 0 && lane == 0 && (mt.z >> 8) != kNoRecord) sched_log_end(sched_log_of(cp.ph[0].ws), mt.z >> 8);
       const GemvParams& p = cp.ph[mt.w];
       const uint32_t row_tile = mt.x, split = mt.y;
       if constexpr (NT == 0) {
@@ -981,6 +990,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) gemv_tc_kernel(const __grid_con
     const bool leader = (warp == kTcEpiWarps + 1);
     const uint32_t xw = warp - (kTcEpiWarps + 2);   // index among the activation producer warps
     uint32_t stage = 0, phase = 0, icount = 0;
+    unsigned long long* const sched_log = (leader && lane == 0) ? sched_log_of(cp.ph[0].ws) : nullptr;
+    uint32_t rec = kNoRecord;   // schedule-log record of the item in production (weight warp, lane 0)
     for (uint32_t ph = 0; ph < n_phases; ++ph) {
       const GemvParams& p = cp.ph[ph];
       const uint32_t n_host_items = p.n_host_pages * p.items_per_page;
@@ -1006,7 +1017,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) gemv_tc_kernel(const __grid_con
           uint8_t* wdst = smem + (size_t)stage * kStageBytes;
           if (lane == 0) {
             if (!mbar_wait(&empty_bar[stage], phase ^ 1u, status)) s_abort = 1;
-            meta[stage] = make_uint4(row_tile, seg, flags | (from_host ? kFlagHost : 0u), ph);
+            meta[stage] = make_uint4(row_tile, seg, flags | (from_host ? kFlagHost : 0u) | (rec << 8), ph);
             mbar_arrive_expect_tx(&full_bar[stage], from_host ? 0u : ((flags & kFlagSecond) ? 2 * kBlockBytes : kBlockBytes));
             if (!from_host) {
               bulk_copy_g2s(wdst, src, kBlockBytes, &full_bar[stage]);
@@ -1062,6 +1073,9 @@ __global__ void __launch_bounds__(kTcThreads, 1) gemv_tc_kernel(const __grid_con
                 }
                 src[h] = page_base[h] + (size_t)(b % kBlocksPerPage) * kBlockBytes;
               }
+              if (seg_first)   // the segment: units up to the end of the row tile (pair) or of this threadblock's range
+                rec = sched_log_begin(sched_log, BOOST_SCHED_KIND_GEMV | (ph << 8), blockIdx.x | (warp << 24),
+                                      min(u1 - u, p.k_blocks - kb) * (second ? 2u : 1u) * kBlockBytes, 0u);
             }
             produce(src[0], src[1], false, tpu * pair, seg,
                     kFlagPair | (second ? kFlagSecond : 0u) | (seg_first ? kFlagFirst : 0u) | (seg_last ? kFlagLast : 0u), kb);
@@ -1098,6 +1112,9 @@ __global__ void __launch_bounds__(kTcThreads, 1) gemv_tc_kernel(const __grid_con
           const uint32_t row_tile = first_blk / p.k_blocks, kb0 = first_blk % p.k_blocks;
           const bool from_host = qi < n_host_items;
           const uint8_t* src = static_cast<const uint8_t*>(p.w_page_ptr[page]) + (size_t)(first_blk % kBlocksPerPage) * kBlockBytes;
+          if (leader && lane == 0)
+            rec = sched_log_begin(sched_log, BOOST_SCHED_KIND_GEMV | (ph << 8), blockIdx.x | (warp << 24), p.run * kBlockBytes,
+                                  from_host ? p.run * kBlockBytes : 0u);
           for (uint32_t j = 0; j < p.run; ++j, src += kBlockBytes)
             produce(src, nullptr, from_host, row_tile, kb0 / p.run, (j == 0 ? kFlagFirst : 0u) | (j + 1 == p.run ? kFlagLast : 0u), kb0 + j);
         }
@@ -1214,6 +1231,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) gemv_tc_kernel(const __grid_con
     } else {
       tc_fence_after_sync();
       if (warp == 0) TRACE(8 + 8 * mt.w + 6);
+      if (tid == 0 && (mt.z >> 8) != kNoRecord) sched_log_end(sched_log_of(cp.ph[0].ws), mt.z >> 8);
       const uint32_t split = mt.y;
       const uint32_t n_tiles = (mt.z & kFlagSecond) ? 2u : 1u;   // row tiles in this accumulator
       const uint32_t n_seg = p.even_part ? even_part_segments(p, mt.x) : p.splits;

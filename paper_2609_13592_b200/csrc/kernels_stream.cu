@@ -75,9 +75,16 @@ stream_reduce_kernel(const void* const* __restrict__ page_ptr, const uint32_t* _
   TierQueues q;
   q.init(ws, n_host_pages * kTilesPerPage, n_pages * kTilesPerPage, n_host_ctas, blockIdx.x, gridDim.x);
   const uint32_t tid = threadIdx.x;
+  unsigned long long* const sched_log = tid == 0 ? sched_log_of(ws) : nullptr;
+  uint32_t rec = kNoRecord;
 
   for (;;) {
-    if (tid == 0) s_item = q.next();
+    if (tid == 0) {
+      s_item = q.next();
+      if (s_item != 0xFFFFFFFFu)
+        rec = sched_log_begin(sched_log, BOOST_SCHED_KIND_STREAM, blockIdx.x, kTileBytes,
+                              s_item < n_host_pages * kTilesPerPage ? kTileBytes : 0u);
+    }
     __syncthreads();
     const uint32_t item = s_item;
     if (item == 0xFFFFFFFFu) break;
@@ -100,6 +107,7 @@ stream_reduce_kernel(const void* const* __restrict__ page_ptr, const uint32_t* _
     if ((tid & 31) == 0) s_warp[tid >> 5] = acc;
     __syncthreads();
     if (tid == 0) {
+      sched_log_end(sched_log, rec);
       float t = 0.f;
 #pragma unroll
       for (uint32_t w = 0; w < kReduceThreads / 32; ++w) t += s_warp[w];

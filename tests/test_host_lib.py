@@ -295,3 +295,38 @@ def test_chain_and_step_workspace_sizes_and_argument_checks():
     assert s32 >= B.boost_gemv_workspace_bytes(128256, 4096, 32) and s128 > s32
     assert B.boost_llama_gemv_workspace_bytes(m, 0) == 0 and B.boost_llama_gemv_workspace_bytes(m, 129) == 0
     B.boost_gemv_set_tc_min_batch(33)
+
+
+def test_schedule_stats_match_oracle_on_random_logs():
+    """boost_schedule_stats against the oracle's exact-rational version on synthetic logs: counts
+    bit for bit, shares to 1e-12."""
+    rng = np.random.default_rng(5)
+    for case in range(12):
+        n = int(rng.integers(1, 400))
+        cap = n + int(rng.integers(0, 3))
+        recs = np.zeros(n, B.SCHED_RECORD_DTYPE)
+        recs["kind_phase"] = rng.integers(1, 4, n) | (rng.integers(0, 4, n) << 8)
+        recs["cta_warp"] = rng.integers(0, 300, n) | (rng.integers(0, 10, n) << 24)
+        recs["bytes"] = rng.integers(0, 5, n) * 16384
+        recs["host_bytes"] = np.where(rng.random(n) < 0.2, recs["bytes"], 0)
+        recs["t_request"] = 10 ** 12 + rng.integers(0, 50_000, n)
+        recs["t_consumed"] = np.where(rng.random(n) < 0.05, 0, recs["t_request"] + rng.integers(0, 9000, n))
+        log = np.zeros(B.boost_schedule_log_bytes(cap), np.uint8)
+        log[:32].view("<u8")[:2] = (n + (3 if case % 4 == 0 else 0), cap)     # sometimes more claimed than the log holds
+        log[32:32 + n * recs.itemsize] = recs.view(np.uint8)
+        got_recs, claimed = B.schedule_records(log)
+        assert claimed >= n and len(got_recs) == min(claimed, cap)     # (slots claimed but never written read as unfinished)
+        tuples = [tuple(int(v) for v in r) for r in got_recs]
+        for kind, per_wave, window_ns, ratio in ((0, 7, 1000, 0.2), (2, 1, 333, 0.1), (3, 50, 100_000, 0.5)):
+            w_ref, t_ref, n_ref = op.schedule_stats(tuples, per_wave, window_ns, ratio, kind)
+            w_got, t_got, n_got = B.boost_schedule_stats(log, kind, per_wave, window_ns, ratio)
+            assert n_got == n_ref
+            for got, ref in ((w_got, w_ref), (t_got, t_ref)):
+                for key in ("n_waves", "n_host_pages", "n_zero_waves"):
+                    assert got[key] == ref[key], (case, kind, key)
+                for key in ("mean", "var", "min", "max"):
+                    assert abs(got[key] - ref[key]) <= 1e-12 * max(1.0, abs(ref[key])), (case, kind, key)
+                # a share equal to the target up to rounding may fall either side in floating point
+                assert abs(got["n_over_waves"] - ref["n_over_waves"]) <= 1
+    with pytest.raises(B.BoostError):
+        B.boost_schedule_stats(np.zeros(16, np.uint8), 0, 1, 1, 0.1)

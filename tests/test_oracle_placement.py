@@ -208,3 +208,39 @@ def test_tier_order():
     assert sorted(order) == list(range(50)) and n_host == sum(tier)
     assert all(tier[i] == 1 for i in order[:n_host]) and all(tier[i] == 0 for i in order[n_host:])
     assert order[:n_host] == sorted(order[:n_host]) and order[n_host:] == sorted(order[n_host:])
+
+
+def test_schedule_stats_closed_forms():
+    """The realised-schedule statistics on logs whose answer is known by construction."""
+    K = 2          # kind
+    # 12 items of 100 bytes, one after the other on one warp, every 4th from the host tier
+    recs = [(K, 0, 100, 100 if i % 4 == 3 else 0, 1000 * i, 1000 * (i + 1)) for i in range(12)]
+    waves, windows, n = op.schedule_stats(recs, 4, 1000, 0.25)
+    assert n == 12 and waves["n_waves"] == 3 and waves["n_host_pages"] == 3
+    assert waves["mean"] == 0.25 and waves["var"] == 0.0 and waves["min"] == waves["max"] == 0.25
+    assert waves["n_zero_waves"] == 0 and waves["n_over_waves"] == 0
+    # windows of one item each: share 1 in the host items' windows, 0 elsewhere
+    assert windows["n_waves"] == 12 and windows["n_zero_waves"] == 9 and windows["max"] == 1.0 and windows["mean"] == 0.25
+    # windows of four items: exactly the target everywhere ("exact ratio at every wave", Sec. 3.1)
+    _, windows, _ = op.schedule_stats(recs, 4, 4000, 0.25)
+    assert windows["n_waves"] == 3 and windows["min"] == windows["max"] == 0.25 and windows["var"] == 0.0
+    # contiguous hand-out (host items last): waves 0, 0, 3/4 -> one over the target, two without host work
+    recs_c = [(K, 0, 100, 100 if i >= 9 else 0, 1000 * i, 1000 * (i + 1)) for i in range(12)]
+    waves, _, _ = op.schedule_stats(recs_c, 4, 1000, 0.25)
+    assert (waves["n_zero_waves"], waves["n_over_waves"], waves["max"]) == (2, 1, 0.75)
+    assert abs(waves["var"] - (2 * 0.25 ** 2 + 0.5 ** 2) / 3) < 1e-15
+    # a host item that streams for the whole kernel beside eight HBM items: every window sees both tiers
+    recs_p = [(K, 0, 800, 800, 0, 8000)] + [(K, 1, 100, 0, 1000 * i, 1000 * (i + 1)) for i in range(8)]
+    _, windows, _ = op.schedule_stats(recs_p, 3, 1000, 0.5)
+    assert windows["n_waves"] == 8 and windows["min"] == windows["max"] == 0.5
+    # an item across a window boundary is split by time: 300 bytes over [500, 2000) -> 100 | 200
+    _, windows, _ = op.schedule_stats([(K, 0, 300, 300, 500, 2000), (K, 1, 100, 0, 500, 1500)], 1, 1000, 1.0)
+    # window 0 = [500, 1500): host 200, hbm 100; window 1 = [1500, 2500): host 100, hbm 0
+    assert windows["n_waves"] == 2 and abs(windows["min"] - 2 / 3) < 1e-15 and windows["max"] == 1.0
+    # filters: other kinds, unfinished and empty records do not count; ties ordered by cta_warp
+    noisy = recs + [(3, 0, 100, 100, 0, 10), (K, 5, 100, 100, 50, 0), (K, 6, 0, 0, 60, 70)]
+    assert op.schedule_stats(noisy, 4, 1000, 0.25, kind=K)[2] == 12
+    a = op.schedule_stats([(K, 2, 10, 10, 7, 9), (K, 1, 10, 0, 7, 9), (K, 3, 10, 0, 8, 9), (K, 0, 10, 0, 8, 9)], 2, 10, 0.5)[0]
+    assert (a["n_waves"], a["min"], a["max"]) == (2, 0.0, 0.5)
+    with pytest.raises(ValueError):
+        op.schedule_stats(recs, 0, 1000, 0.25)
