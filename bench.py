@@ -621,7 +621,7 @@ def run_kv_spill(args):
 
 
 def run_pool_churn(args):
-    """KV pool under serving-like churn (Sec. 5.9, Sec. 5.10): Poisson arrivals with a
+    """KV pool under serving-like churn (Sec. 5.8, Sec. 5.11): Poisson arrivals with a
     long-generation length mix are replayed on the wave-aware pool at about 80 % utilisation for
     12 000 decode steps; the host share of the live KV chunks is recorded after every step
     (rolling median and min - max band over 500 steps, against the configured 1/M and the 1/H

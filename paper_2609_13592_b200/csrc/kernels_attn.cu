@@ -45,13 +45,6 @@ constexpr uint32_t kParkStride = kD + 4;                 // floats per parked he
 constexpr uint32_t kMaxListedSeqs = 1024;                // batches up to this size get a dense item list
 constexpr uint32_t kTailPieces = 4;                      // the runs of the last KV head are cut in this many items
 
-#ifdef BOOST_TRACE
-// Debug build only: per-warp time stamps (global timer, ns), 8 slots per warp.
-__device__ unsigned long long* g_attn_trace = nullptr;
-#define ATRACE(slot) do { if (g_attn_trace && (threadIdx.x & 31) == 0) { unsigned long long t_; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_)); g_attn_trace[((size_t)blockIdx.x * 4 + (threadIdx.x >> 5)) * 8 + (slot)] = t_; } } while (0)
-#else
-#define ATRACE(slot) do { } while (0)
-#endif
 
 struct AttnParams {
   const __nv_bfloat16* q;
@@ -99,7 +92,6 @@ __global__ void __launch_bounds__(kAttnThreads, (NH == 1 ? 3 : 2)) paged_attn_ke
     fence_barrier_init();
   }
   __syncwarp();
-  ATRACE(0);
   // The kernels just before this one produce q and the newest K / V row of every sequence
   // (in its last block).  Context lengths, block tables and all older blocks are not theirs:
   // the first item's look-ups, and its first blocks unless one of them is the sequence's
@@ -187,7 +179,6 @@ __global__ void __launch_bounds__(kAttnThreads, (NH == 1 ? 3 : 2)) paged_attn_ke
   const uint32_t n_long = (p.Hkv - 1) * per_head;
   const uint32_t n_items = n_long + per_head * tail_k;
   const uint32_t slots_per = max_splits * tail_k;      // partial results of one (sequence, query head)
-  ATRACE(7);
   uint32_t id = blockIdx.x;
 
   while (id < n_items) {
@@ -291,7 +282,6 @@ __global__ void __launch_bounds__(kAttnThreads, (NH == 1 ? 3 : 2)) paged_attn_ke
       if (!waited) {
         pdl_wait();
         waited = true;
-        ATRACE(1);
       }
       if (!early)
         for (uint32_t i = 0; i < n_first; ++i) request(i);
@@ -318,7 +308,6 @@ __global__ void __launch_bounds__(kAttnThreads, (NH == 1 ? 3 : 2)) paged_attn_ke
       for (uint32_t i = 0; i < nb; ++i) {
         const uint32_t st = i % kWarpStages;
         mbar_wait(&full_bar[warp][st], (phase_mask >> st) & 1u, status);
-        if (i == 0) ATRACE(2);
         phase_mask ^= 1u << st;
         const uint32_t kbase = smem_u32(ring + (size_t)st * kStageBytes);
         const uint32_t vbase = kbase + kChunkBytes;
@@ -408,7 +397,6 @@ __global__ void __launch_bounds__(kAttnThreads, (NH == 1 ? 3 : 2)) paged_attn_ke
       }
       if (lane == 0 && rec != kNoRecord) sched_log_end(sched_log_of(p.ws), rec);
 
-      ATRACE(3);
       // ---- end of the run: the four warps' (m, l, O) meet in shared memory.  Each warp parks
       // its result in its own (now idle) ring space: per head 128 outputs, then m and l.
       float* park = reinterpret_cast<float*>(ring);
@@ -473,7 +461,6 @@ __global__ void __launch_bounds__(kAttnThreads, (NH == 1 ? 3 : 2)) paged_attn_ke
           s_old = atomicAdd(cnt, 1u);
         }
         __syncthreads();
-        ATRACE(4);
         if (s_old == n_parts - 1) {
           __threadfence();
           for (uint32_t r = warp; r < p.group; r += kAttnWarps) {
@@ -519,7 +506,6 @@ __global__ void __launch_bounds__(kAttnThreads, (NH == 1 ? 3 : 2)) paged_attn_ke
             *reinterpret_cast<uint2*>(p.out + ((size_t)b * p.Hq + hq) * kD + lane * 4) = ov;
           }
           if (tid == 0) *cnt = 0;
-          ATRACE(5);
         }
       }
       // the ring is written by bulk copies again: every thread orders its reads and writes of the
@@ -535,7 +521,6 @@ __global__ void __launch_bounds__(kAttnThreads, (NH == 1 ? 3 : 2)) paged_attn_ke
     id = s_next;
     __syncthreads();
   }
-  ATRACE(6);
   // the last threadblock out resets the counters for the next launch
   if (tid == 0) {
     __threadfence();
@@ -591,11 +576,6 @@ size_t attn_header_bytes(uint32_t B, uint32_t Hkv_upper) {
 
 }  // namespace
 
-#ifdef BOOST_TRACE
-extern "C" int boost_debug_set_attn_trace(void* ptr) {
-  return boosth::check(cudaMemcpyToSymbol(g_attn_trace, &ptr, sizeof(ptr)));
-}
-#endif
 
 extern "C" int boost_kv_scatter(const void* src, uint32_t n_kv_heads, uint32_t n_pool_blocks,
                                 uint32_t D, const void* const* page_ptr, size_t n_pages, void* stream) {

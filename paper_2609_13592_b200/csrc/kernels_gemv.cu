@@ -43,21 +43,6 @@ enum : uint32_t { kBarExit = 0u, kBarPartials = 1u, kBarPhase = 1u + kMaxPhases,
 constexpr uint32_t kEndCombineMinSegments = 4;
 enum : uint32_t { kEpiPlain = 0u, kEpiSwiglu = 1u, kEpiRope = 2u };
 
-#ifdef BOOST_TRACE
-// Debug build only: per-threadblock time stamps (global timer, ns) for timeline analysis.
-// 64 slots per threadblock: 0 start, 7 exit, 8 + 8 * phase + k for the events of a phase.
-__device__ unsigned long long* g_trace = nullptr;
-__device__ __forceinline__ unsigned long long gtime() {
-  unsigned long long t;
-  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
-  return t;
-}
-#define TRACE(slot) do { if (g_trace && (threadIdx.x & 31) == 0) g_trace[(size_t)blockIdx.x * 64 + (slot)] = gtime(); } while (0)
-#define TRACE_ONCE(slot) do { if (g_trace && (threadIdx.x & 31) == 0 && g_trace[(size_t)blockIdx.x * 64 + (slot)] == 0) g_trace[(size_t)blockIdx.x * 64 + (slot)] = gtime(); } while (0)
-#else
-#define TRACE(slot) do { } while (0)
-#define TRACE_ONCE(slot) do { } while (0)
-#endif
 
 struct GemvParams {
   const void* const* w_page_ptr;
@@ -436,7 +421,6 @@ __global__ void __launch_bounds__(kGemvThreads, (NT >= 8 ? 1 : 2)) gemv_tiered_k
   const uint32_t n_phases = cp.n_phases;
   uint32_t* status = cp.ph[0].ws + kWsStatus;
 
-  if (tid == 0) TRACE(0);
   pdl_launch_dependents();
   if (tid == 0) {
     for (uint32_t s = 0; s < n_stages; ++s) {
@@ -512,7 +496,6 @@ __global__ void __launch_bounds__(kGemvThreads, (NT >= 8 ? 1 : 2)) gemv_tiered_k
         ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
         if (!ok) { s_abort = 1u; leave(); return; }
       }
-      if (!leader) TRACE(8 + 8 * ph + 2);
       if (p.even_part) {
         // Even partition: both warps walk the same static block range, no queue.
         const uint32_t G = p.active_ctas, T = p.total_blocks;
@@ -520,7 +503,6 @@ __global__ void __launch_bounds__(kGemvThreads, (NT >= 8 ? 1 : 2)) gemv_tiered_k
           const uint32_t b0 = (uint32_t)((uint64_t)blockIdx.x * T / G), b1 = (uint32_t)((uint64_t)(blockIdx.x + 1) * T / G);
           uint32_t row_tile = b0 / p.k_blocks, kb = b0 % p.k_blocks;
           uint32_t seg = blockIdx.x - part_owner((uint64_t)row_tile * p.k_blocks, G, T);
-          if (leader && b0 < b1) TRACE_ONCE(8 + 8 * ph + 0);
           const uint32_t c = lane & 7, m0 = lane >> 3;
           // the page address is looked up once per page, not once per block: a table look-up per
           // block would put an L2 round trip between any two copies of this warp
@@ -589,7 +571,6 @@ __global__ void __launch_bounds__(kGemvThreads, (NT >= 8 ? 1 : 2)) gemv_tiered_k
           if (lane == 0) mbar_arrive(&item_empty[slot]);
         }
         ++icount;
-        if (leader && qi != 0xFFFFFFFFu) TRACE_ONCE(8 + 8 * ph + 0);
         if (qi == 0xFFFFFFFFu) break;
         const uint32_t page = p.w_order[qi / p.items_per_page];
         const uint32_t first_blk = (page * p.items_per_page + qi % p.items_per_page) * p.run;
@@ -644,7 +625,6 @@ __global__ void __launch_bounds__(kGemvThreads, (NT >= 8 ? 1 : 2)) gemv_tiered_k
         }
       }
       // a stage without data tells the consumers that the phase (or the launch) is over
-      if (leader) TRACE(8 + 8 * ph + 1);
       if (leader) {
         if (!lane0_wait(&empty_bar[stage], phase ^ 1u)) { leave(); return; }
         if (lane == 0) {
@@ -699,7 +679,6 @@ __global__ void __launch_bounds__(kGemvThreads, (NT >= 8 ? 1 : 2)) gemv_tiered_k
     if (!warp_wait(&full_bar[stage], phase)) { wait_failed = true; failed = true; break; }
     const uint4 mt = meta[stage];
     if (mt.z & (kFlagStop | kFlagPhaseEnd)) { mk = mt; break; }
-    if (warp == 0 && (mt.z & kFlagFirst)) TRACE_ONCE(8 + 8 * mt.w + 3);
     if (mt.z & kFlagFirst) {
 #pragma unroll
       for (int i = 0; i < kAccN; ++i)
@@ -765,7 +744,6 @@ __global__ void __launch_bounds__(kGemvThreads, (NT >= 8 ? 1 : 2)) gemv_tiered_k
     if (++stage == n_stages) { stage = 0; phase ^= 1u; }
 
     if (mt.z & kFlagLast) {
-      if (warp == 0) TRACE(8 + 8 * mt.w + 6);
       if (warp == 0 && lane == 0 && (mt.z >> 8) != kNoRecord) sched_log_end(sched_log_of(cp.ph[0].ws), mt.z >> 8);
       const GemvParams& p = cp.ph[mt.w];
       const uint32_t row_tile = mt.x, split = mt.y;
@@ -847,7 +825,6 @@ __global__ void __launch_bounds__(kGemvThreads, (NT >= 8 ? 1 : 2)) gemv_tiered_k
     const uint4 mt = mk;
     const GemvParams& p = cp.ph[mt.w];
     const bool phase_end = (mt.z & (kFlagStop | kFlagPhaseEnd)) != 0;
-    if (phase_end && warp == 0) TRACE(8 + 8 * mt.w + 4);
     // Slots go to the warps of the grid in order, so only the first threadblocks have any; one
     // without has nothing to wait for once its own partial sums are out (after the last phase it
     // leaves at once and makes room for the next kernel's threadblocks).
@@ -862,14 +839,12 @@ __global__ void __launch_bounds__(kGemvThreads, (NT >= 8 ? 1 : 2)) gemv_tiered_k
         if (combines && !grid_counter_wait(cp.bar + kBarPartials + mt.w, gridDim.x, status)) s_abort = 1u;
       }
       if (combines && !group_sync()) break;
-      if (warp == 0) TRACE(8 + 8 * mt.w + 7);
     }
     if (combines) {
       __threadfence();
       const bool all = phase_end;
       combine_units<kXRows>(p, all ? blockIdx.x * kConsumerWarps + warp : warp, all ? combine_ctas * kConsumerWarps : kConsumerWarps,
                             all ? kAllTiles : mt.x, lane, status);
-      if (warp == 0) TRACE(8 + 8 * mt.w + 5);
     }
     if (!phase_end) {
       if (tid == 0) tile_cnt[mt.x] = 0;
@@ -900,7 +875,6 @@ __global__ void __launch_bounds__(kGemvThreads, (NT >= 8 ? 1 : 2)) gemv_tiered_k
   }
   }
   if (wait_failed) named_barrier_or(1, kConsumerThreads, true);   // the arrival the others' next group_sync counts on
-  if (warp == 0) TRACE(7);
 }
 
 // The combine of a product whose launch left it out (defer_combine): every row tile at once, the
@@ -941,7 +915,6 @@ template <uint32_t NPAD>
 __global__ void __launch_bounds__(kTcThreads, 1) gemv_tc_kernel(const __grid_constant__ ChainParams cp) {
   constexpr uint32_t kStageBytes = tc_stage_bytes(NPAD);
   constexpr uint32_t kTmemCols = 4 * NPAD < 32 ? 32 : 4 * NPAD;   // two accumulators (a pair of row tiles), double-buffered
-  if (threadIdx.x == 0) TRACE(0);
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   __shared__ uint64_t full_bar[kMaxStages];
@@ -1004,7 +977,6 @@ __global__ void __launch_bounds__(kTcThreads, 1) gemv_tc_kernel(const __grid_con
         if (lane == 0 && !grid_counter_wait(cp.bar + kBarPhase + (ph - 1), gridDim.x, status)) s_abort = 1;
         __syncwarp();
       }
-      if (warp == kTcEpiWarps + 2) TRACE(8 + 8 * ph + 2);
       // one block: the weight warp copies it, the activation warp stages x[:, 64 kb .. 64 kb + 64)
       // as NPAD rows of 128 bytes in the 128-byte swizzle (rows >= M_b are zero)
       // one stage: the weight warp copies the weight block (two blocks in pair mode), the
@@ -1161,7 +1133,6 @@ __global__ void __launch_bounds__(kTcThreads, 1) gemv_tc_kernel(const __grid_con
           if (!mbar_wait(&acc_empty[buf], buf_phase ^ 1u, status)) { s_abort = 1; break; }   // the epilogue has read this accumulator
           accumulate = 0;
         }
-        TRACE_ONCE(8 + 8 * mt.w + 3);
         fence_proxy_async_smem();   // x (and host-tier weight blocks) were written through the load/store path
         tc_fence_after_sync();
         const uint32_t wbase = smem_u32(smem + (size_t)stage * kStageBytes);
@@ -1213,7 +1184,6 @@ __global__ void __launch_bounds__(kTcThreads, 1) gemv_tc_kernel(const __grid_con
     const bool phase_end = (mt.z & (kFlagStop | kFlagPhaseEnd)) != 0;
     uint32_t n_jobs = 0, job[2] = {0u, 0u};   // row tiles to combine, or kAllTiles
     if (phase_end) {
-      if (warp == 0) TRACE(8 + 8 * mt.w + 4);
       if (p.end_combine && !p.defer_combine) {
         // every threadblock's partial sums of this phase in memory -> all tiles combined, by the
         // epilogue warps of the whole grid (see combine_units)
@@ -1230,7 +1200,6 @@ __global__ void __launch_bounds__(kTcThreads, 1) gemv_tc_kernel(const __grid_con
       }
     } else {
       tc_fence_after_sync();
-      if (warp == 0) TRACE(8 + 8 * mt.w + 6);
       if (tid == 0 && (mt.z >> 8) != kNoRecord) sched_log_end(sched_log_of(cp.ph[0].ws), mt.z >> 8);
       const uint32_t split = mt.y;
       const uint32_t n_tiles = (mt.z & kFlagSecond) ? 2u : 1u;   // row tiles in this accumulator
@@ -1281,7 +1250,6 @@ __global__ void __launch_bounds__(kTcThreads, 1) gemv_tc_kernel(const __grid_con
       combine_units<NPAD>(p, all ? blockIdx.x * kTcEpiWarps + warp : warp, all ? gridDim.x * kTcEpiWarps : kTcEpiWarps, job[j], lane,
                           status);
       if (!all && tid == 0) tile_cnt[job[j]] = 0;
-      if (warp == 0) TRACE(8 + 8 * mt.w + 5);
     }
     if (n_jobs && !phase_end) named_barrier_sync(1, kTcEpiThreads);   // (s_last may be rewritten, the tiles' slots reused)
     if (phase_end) {
@@ -1756,8 +1724,3 @@ extern "C" int boost_gemv_set_end_combine(uint32_t on) {
   return BOOST_OK;
 }
 
-#ifdef BOOST_TRACE
-extern "C" int boost_debug_set_trace(void* ptr) {
-  return boosth::check(cudaMemcpyToSymbol(g_trace, &ptr, sizeof(ptr)));
-}
-#endif

@@ -97,7 +97,7 @@ def serving_churn_trace(n_blocks, n_steps, arrivals_per_step, max_batch, seed, p
                         out_median=1500.0, out_sigma=0.8, out_cap=8192, block_tokens=16):
     """Allocation trace of a continuously batched decode server, one decode step at a time
     (a stand-in for the paper's serving runs with Poisson arrivals and a long-generation
-    length mix, Sec. 5.9, Sec. 5.10; shapes only, no dataset items).
+    length mix, Sec. 5.8 and Sec. 5.11; shapes only, no dataset items).
 
     Arrivals per step are Poisson; a request has a prompt of U[prompt_lo, prompt_hi] tokens
     and generates a log-normal number of tokens (median out_median, log-sigma out_sigma,

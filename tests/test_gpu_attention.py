@@ -207,7 +207,7 @@ def test_attention_config5_shape_on_sampled_sequences(dev):
 def test_attention_on_a_pool_under_serving_churn(dev):
     """Four KV heads (eight query heads each), one KV page in twelve on the host, the batch as a
     pool leaves it after 7000 decode steps of Poisson arrivals with a long-generation length
-    mix at about 80 % utilisation (Sec. 5.10): about 95 sequences of up to 6000 tokens whose
+    mix at about 80 % utilisation (Sec. 5.11): about 95 sequences of up to 6000 tokens whose
     blocks are scattered over the pool, so a sequence takes several work items and its
     partial results meet in global memory.  The library and the oracle pool replay the trace
     side by side; the oracle computes the longest, the shortest and three more sequences."""

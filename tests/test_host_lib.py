@@ -200,7 +200,7 @@ def test_pool_traces_bit_exact(geom):
 
 
 def test_pool_under_serving_churn_bit_exact_and_near_target():
-    # Sec. 5.10: four KV heads, one page in twelve on the host, Poisson arrivals with a
+    # Sec. 5.11: four KV heads, one page in twelve on the host, Poisson arrivals with a
     # long-generation length mix at about 80 % pool utilisation.  The library hands out the
     # same blocks as the oracle throughout, and the realised host share of the live KV
     # chunks stays within a point of the target, far below the 1/H granularity bound.

@@ -196,7 +196,7 @@ def test_exhaustive_short_traces_keep_invariants():
 
 
 def test_churn_keeps_live_host_share_near_target():
-    # Sec. 5.10: four KV heads, target one page in twelve (8.3 %): the realised share of
+    # Sec. 5.11: four KV heads, target one page in twelve (8.3 %): the realised share of
     # live KV chunks on the host stays within about a point of the target and far below 1/H.
     pool = kp.KVPool(12 * 1024, 4, 12)
     rng = random.Random(2024)
