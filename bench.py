@@ -38,6 +38,7 @@ FALLBACK_HBM_GBS = 6650.0
 # capture of two full-size chain launches of this workload (profiles/
 # gemv_tiered_kernel_chain_llama8b_m32.md): 1955.5 MB moved for 1872.8 MB of packed weights.
 GEMV_TRAFFIC_PER_ALGORITHMIC_BYTE = 1.044
+GEMV_TRAFFIC_PROFILE = "profiles/gemv_tiered_kernel_chain_llama8b_m32.md"
 
 
 def load_peaks():
@@ -349,6 +350,7 @@ def timed_device_steps(dec, dev, batch, ctx0, warmup, steps, max_blocks, dist_ct
     dist_ctx.barrier()
     ms = e0.elapsed_time(e1)
     kv_tokens = int(ctx_all[warmup:].sum())
+    dec.last_tokens = tok[(warmup + steps) % 2].cpu().numpy().copy()   # what the last timed step produced
     if not profile:
         drv.release()
         return ms, launches, kv_tokens, None, None
@@ -494,6 +496,7 @@ def run_ours(args, rank, world, local_rank):
         gemv_ms, gemv_n = t["kind_ms"][0], t["kind_n"][0]
         gemv_gbs = t["weight_bytes"] / (gemv_ms / 1e3) / 1e9
         gemv_bytes_per_launch = t["weight_bytes"] / max(gemv_n, 1)
+        gemv_step_bytes = t["weight_bytes"]
         # tier-wise bound: the slower of the two tiers if each streamed its own bytes at its own peak
         host_bytes = t["host_pages"] * (2 << 20)
         t_min_ms = 1e3 * max((bytes_step - host_bytes) / (hbm_peak * 1e9), host_bytes / (link_gbs * 1e9))
@@ -530,7 +533,13 @@ def run_ours(args, rank, world, local_rank):
                          "traffic": GEMV_TRAFFIC_PER_ALGORITHMIC_BYTE * gemv_bytes_per_launch,
                          "traffic_source": "ncu dram bytes of this workload's launches, ratio 1.044 to algorithmic",
                          "launches_per_step": gemv_n, "avg_launch_us": 1e3 * gemv_ms / max(gemv_n, 1),
-                         "peak_source": peak_src},
+                         "peak_source": peak_src,
+                         # events around every launch serialise the step: no launch overlaps its neighbours
+                         "serialised": True,
+                         # the same bytes over the weight products' share of the overlapped step
+                         # (step time minus the serialised time of the other kinds): an upper estimate
+                         "achieved_in_step": gemv_step_bytes / (max(ms_step - t["kind_ms"][1] - t["kind_ms"][2], 1e-6) / 1e3) / 1e9,
+                         "traffic_profile": GEMV_TRAFFIC_PROFILE},
             "roofline_attention": {"bound": "hbm", "kernel": "paged_attn_kernel", "achieved": attn_gbs,
                                    "peak": hbm_peak, "unit": "GB/s", "frac": attn_gbs / hbm_peak,
                                    "launches_per_step": attn_n, "avg_launch_us": 1e3 * attn_ms / max(attn_n, 1)},
@@ -584,6 +593,7 @@ def run_kv_spill(args):
     small = int(np.searchsorted(np.cumsum(blocks), budget, side="right"))
     null = DistCtx(0, 1, dev)
     out = {}
+    last_tokens = {}
     for label, b_run, pool_blocks, modulus, prefetch in (("tiered", batch, n_pool_blocks, 5, False),
                                                          ("prefetch", batch, n_pool_blocks, 5, True),
                                                          ("hbm_only", small, budget, 0, False)):
@@ -599,6 +609,7 @@ def run_kv_spill(args):
                       "weight_bytes": dec.weight_bytes(), "launches_per_step": launches // steps,
                       "pool_blocks": pool_blocks, "kv_host_pages_per_tensor": host_pages,
                       "status": dec.status_words()}
+        last_tokens[label] = dec.last_tokens
         del dec
         torch.cuda.empty_cache()
     t = out["tiered"]
@@ -616,8 +627,15 @@ def run_kv_spill(args):
             "combined_roofline_gbs": hbm_peak + link_gbs,
             "tier_bound": {"t_min_ms": t_min_ms, "frac_of_t_min": t_min_ms / t["ms_per_step"],
                            "note": "the host share (20 %) is far above the link share of this box, so the step is link-bound"},
-            "runs": out}
+            "runs": out,
+            # the same seeded model, cache and inputs: reading host pages in place and reading their
+            # staged copies must produce the same tokens after the same steps, sequence by sequence
+            "verified": {"tiered_vs_prefetch_next_tokens_equal": bool(np.array_equal(last_tokens["tiered"], last_tokens["prefetch"])),
+                         "sequences_compared": int(last_tokens["tiered"].size),
+                         "all_status_words_zero": all(v == 0 for r in out.values() for v in r["status"])}}
     print(json.dumps(line), flush=True)
+    if not (line["verified"]["tiered_vs_prefetch_next_tokens_equal"] and line["verified"]["all_status_words_zero"]):
+        raise SystemExit("kv_spill: the tiered and the prefetch run disagree, or a kernel recorded an error")
 
 
 def run_pool_churn(args):
@@ -824,17 +842,30 @@ def run_stream_sweep(args):
         policies = [pp for pp in policies if pp[0] in args.sweep_policies.split(",")]
     sizes = [int(x) for x in args.sweep_gib.split(",")]
     points = []
+    checked_points = 0
+    from paper_2609_13592_b200 import synth
+    page_elems = B.PAGE_BYTES // 2
     for gib in sizes:
         n_pages = gib * 512
         slabs = Slabs(n_pages, n_pages // 8 + n_pages // 32 + 8, dev)
         ws_bytes = B.boost_stream_reduce_workspace_bytes(n_pages)
         ws = torch.zeros(ws_bytes, dtype=torch.uint8, device=dev)
         sums = torch.zeros(n_pages, dtype=torch.float32, device=dev)
+        # The 1 GiB points are checked: the buffer holds the integer fill of the synthetic generator
+        # (values in [-4, 4], so fp32 page sums are exact) and every page sum must equal the integer
+        # sum of the generator's values for that page, bit for bit, under every placement.
+        check = gib == 1
+        if check:
+            flat = synth.small_int_bf16_torch(0, n_pages * page_elems, dev)
+            want = torch.from_numpy(synth.small_int_values(0, n_pages * page_elems).reshape(n_pages, page_elems)
+                                    .sum(axis=1).astype(np.float32)).to(dev)
+        log = torch.zeros(B.boost_schedule_log_bytes(16 * n_pages), dtype=torch.uint8, device=dev) if gib <= 16 else None
         for ratio in ratios:
             for name, pol in policies:
                 seeds = range(args.sweep_seeds) if (pol == B.POLICY_RANDOM and ratio > 0) else [0]
                 gbs, var = [], []
                 n_host = 0
+                realised = None
                 for seed in seeds:
                     buf = TieredBuffer(n_pages * B.PAGE_BYTES, ratio, pol, seed=seed, device=dev, slabs=slabs)
                     n_host = buf.n_host
@@ -850,16 +881,35 @@ def run_stream_sweep(args):
                             best = min(best, e0.elapsed_time(e1))
                     gbs.append(n_pages * B.PAGE_BYTES / best / 1e6)
                     var.append(st["var"])
+                    if check and seed == 0:
+                        buf.scatter_from(flat)
+                        B.boost_stream_reduce_tiered(buf.page_ptr, buf.order, n_pages, buf.n_host, sums, ws, ws_bytes)
+                        torch.cuda.synchronize(dev)
+                        if not torch.equal(sums, want):
+                            raise SystemExit(f"stream_sweep: page sums differ at ratio {ratio}, placement {name}")
+                        checked_points += 1
+                    if log is not None and seed == 0 and ratio > 0:
+                        # one more launch with the schedule log attached: the host share the queues realise,
+                        # per wave of tile starts and per 10 us of the run (address order: st above)
+                        log.zero_()
+                        log[:32].view(torch.int64)[1] = 16 * n_pages
+                        ws[:64].view(torch.int64)[B.WS_LOG_WORD // 2] = log.data_ptr()
+                        B.boost_stream_reduce_tiered(buf.page_ptr, buf.order, n_pages, buf.n_host, sums, ws, ws_bytes)
+                        torch.cuda.synchronize(dev)
+                        ws[:64].view(torch.int64)[B.WS_LOG_WORD // 2] = 0
+                        w_st, t_st, n_rec = B.boost_schedule_stats(log.cpu().numpy(), B.SCHED_KIND_STREAM, sms * 4, 10_000, ratio)
+                        realised = {"records": n_rec, "per_wave_of_starts": w_st, "per_10us_window": t_st}
                     del buf
                 bound = min(hbm_peak + link, link / ratio * 1.0) if ratio > 0 else hbm_peak
                 points.append({"gib": gib, "host_ratio": ratio, "placement": name, "host_pages": n_host,
                                "combined_gbs": float(np.mean(gbs)), "gbs_min": float(min(gbs)),
                                "gbs_max": float(max(gbs)), "wave_host_share_var": float(np.mean(var)),
-                               "tier_bound_gbs": bound, "seeds": len(list(seeds))})
+                               "tier_bound_gbs": bound, "seeds": len(list(seeds)), "realised_schedule": realised})
         del slabs, ws, sums
         torch.cuda.empty_cache()
     print(json.dumps({"workload": "c3_tiered_stream_sweep", "hbm_peak_gbs": hbm_peak, "hbm_peak_source": peak_src,
-                      "host_link_gbs": link, "combined_roofline_gbs": hbm_peak + link, "points": points}))
+                      "host_link_gbs": link, "combined_roofline_gbs": hbm_peak + link,
+                      "points_with_page_sums_verified": checked_points, "points": points}))
 
 
 def main():
