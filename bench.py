@@ -775,7 +775,7 @@ def run_gemv_sweep(args):
     shapes = {"qkv": (6144, 4096), "o": (4096, 4096), "gate_up": (28672, 4096), "down": (4096, 14336),
               "lm_head": (128256, 4096)}
     ratios = [("hbm_only", 0.0), (f"link_share_1/{modulus}", 1.0 / modulus), ("1/16", 1.0 / 16)]
-    batches = [1, 2, 4, 8, 16, 32, 64, 128]
+    batches = [1, 2, 4, 8, 16, 32, 64, 128, 256]
     points = []
     g = torch.Generator(device=dev)
     g.manual_seed(3)

@@ -314,7 +314,7 @@ int boost_pack_weights_ex(const void* w_row_major /*device*/, uint32_t N, uint32
  * handwritten matmul of Sec. 3.1 is the closest thing the paper describes).
  *   w_page_ptr, w_order  device arrays for the packed weight (n_pages entries; order from
  *                        boost_tier_order, host pages first);
- *   x          device, bf16 row-major [M_b, K];  1 <= M_b <= 128;
+ *   x          device, bf16 row-major [M_b, K];  1 <= M_b <= 256;
  *   y          device, row-major [M_b, N]; y_dtype 0 = fp32, 1 = bf16;
  *   residual   device bf16 [M_b, N] added before the final rounding, or NULL;
  *   workspace  device, >= boost_gemv_workspace_bytes(N, K, M_b).

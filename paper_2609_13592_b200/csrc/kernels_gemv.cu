@@ -909,12 +909,16 @@ constexpr uint32_t kTcXWarps = 4;   // activation producer warps: rows m with (m
 constexpr uint32_t kTcThreads = kTcEpiThreads + 64 + 32 * kTcXWarps;
 
 // a stage: two weight blocks (the same 64 columns of two adjacent row tiles) and one activation tile
-__host__ __device__ constexpr uint32_t tc_stage_bytes(uint32_t npad) { return 2 * kBlockBytes + npad * 128u; }
+// (at 256 batch rows the activation tile alone is 32 KiB and tensor memory holds two accumulators
+// of that width, not four: one weight block per stage, no pairs)
+__host__ __device__ constexpr uint32_t tc_weight_slots(uint32_t npad) { return npad <= 128 ? 2u : 1u; }
+__host__ __device__ constexpr uint32_t tc_stage_bytes(uint32_t npad) { return tc_weight_slots(npad) * kBlockBytes + npad * 128u; }
 
 template <uint32_t NPAD>
 __global__ void __launch_bounds__(kTcThreads, 1) gemv_tc_kernel(const __grid_constant__ ChainParams cp) {
   constexpr uint32_t kStageBytes = tc_stage_bytes(NPAD);
-  constexpr uint32_t kTmemCols = 4 * NPAD < 32 ? 32 : 4 * NPAD;   // two accumulators (a pair of row tiles), double-buffered
+  constexpr uint32_t kSlots = tc_weight_slots(NPAD);
+  constexpr uint32_t kTmemCols = 2 * kSlots * NPAD < 32 ? 32 : 2 * kSlots * NPAD;   // one accumulator per weight slot, double-buffered
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   __shared__ uint64_t full_bar[kMaxStages];
@@ -1005,7 +1009,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) gemv_tc_kernel(const __grid_con
         } else {
           if (!mbar_wait(&empty_bar[stage], phase ^ 1u, status)) s_abort = 1;
           const uint32_t c = lane & 7, m0 = (lane >> 3) + 4 * xw;
-          uint8_t* xbase = smem + (size_t)stage * kStageBytes + 2 * kBlockBytes;
+          uint8_t* xbase = smem + (size_t)stage * kStageBytes + kSlots * kBlockBytes;
           const uint32_t k = kb * kBlockK + c * 8;
           const bool k_ok = k < p.K;
 #pragma unroll 4
@@ -1136,8 +1140,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) gemv_tc_kernel(const __grid_con
         fence_proxy_async_smem();   // x (and host-tier weight blocks) were written through the load/store path
         tc_fence_after_sync();
         const uint32_t wbase = smem_u32(smem + (size_t)stage * kStageBytes);
-        const uint32_t xbase = wbase + 2 * kBlockBytes;
-        const uint32_t d0 = tmem_base + buf * 2 * NPAD;   // accumulator of the first row tile; the second follows it
+        const uint32_t xbase = wbase + kSlots * kBlockBytes;
+        const uint32_t d0 = tmem_base + buf * kSlots * NPAD;   // accumulator of the first row tile; the second follows it
 #pragma unroll
         for (uint32_t ks = 0; ks < kBlockK / 16; ++ks) {
           const uint64_t xdesc = umma_desc_k_sw128(xbase + ks * 32);
@@ -1214,7 +1218,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) gemv_tc_kernel(const __grid_con
       for (uint32_t ti = 0; ti < n_tiles; ++ti) {
         const uint32_t row_tile = mt.x + ti;
         float* part = p.partials + ((size_t)row_tile * p.max_seg + split) * NPAD * kBlockRows;
-        const uint32_t taddr = tmem_base + ((quarter * 32u) << 16) + buf * 2 * NPAD + ti * NPAD;
+        const uint32_t taddr = tmem_base + ((quarter * 32u) << 16) + buf * kSlots * NPAD + ti * NPAD;
         for (uint32_t c0 = c_begin; c0 < c_end; c0 += 16) {
           float v[16];
           tmem_ld16(taddr + c0, v);
@@ -1439,7 +1443,8 @@ int launch_gemv_tc(const ChainParams& chain, int sms, cudaStream_t stream, uint3
   const int slot = boosth::device_slot();
   if (slot < 0) return BOOST_ERR_CUDA;
   KernelState& state = states[slot];
-  return launch_planned(gemv_tc_kernel<NPAD>, gemv_combine_kernel<NPAD>, NPAD, state, kTcThreads, tc_stage_bytes(NPAD), 1, true,
+  return launch_planned(gemv_tc_kernel<NPAD>, gemv_combine_kernel<NPAD>, NPAD, state, kTcThreads, tc_stage_bytes(NPAD), 1,
+                        tc_weight_slots(NPAD) == 2,
                         g_end_combine != 0, chain, sms, stream, extra_launches);
 }
 
@@ -1491,7 +1496,8 @@ static uint32_t gemv_x_rows(uint32_t M_b) {
   if (M_b <= 16) return 16;
   if (M_b <= 32) return 32;
   if (M_b <= 64) return 64;
-  return 128;
+  if (M_b <= 128) return 128;
+  return 256;
 }
 
 size_t boosth::gemv_header_bytes(uint32_t n_row_tiles) {
@@ -1513,13 +1519,13 @@ static uint32_t partial_slots(const boost_weight_layout_t& lay, uint32_t M_b) {
 
 size_t boosth::gemv_partial_bytes(uint32_t N, uint32_t K, uint32_t M_b) {
   boost_weight_layout_t lay;
-  if (boost_weight_layout(N, K, &lay) != BOOST_OK || M_b == 0 || M_b > 128) return 0;
+  if (boost_weight_layout(N, K, &lay) != BOOST_OK || M_b == 0 || M_b > 256) return 0;
   return (size_t)lay.n_row_tiles * partial_slots(lay, M_b) * gemv_x_rows(M_b) * kBlockRows * 4;
 }
 
 extern "C" size_t boost_gemv_workspace_bytes(uint32_t N, uint32_t K, uint32_t M_b) {
   boost_weight_layout_t lay;
-  if (boost_weight_layout(N, K, &lay) != BOOST_OK || M_b == 0 || M_b > 128) return 0;
+  if (boost_weight_layout(N, K, &lay) != BOOST_OK || M_b == 0 || M_b > 256) return 0;
   return boosth::gemv_header_bytes(lay.n_row_tiles) + boosth::gemv_partial_bytes(N, K, M_b);
 }
 
@@ -1562,7 +1568,7 @@ int fill_params(GemvParams& p, const void* const* w_page_ptr, const uint32_t* w_
   }
   if (epi && epi->ssq_in && (epi->ssq_in_tiles == 0 || epi->ssq_stride < M_b)) return BOOST_ERR_INVALID;
   if (epi && epi->ssq_out && (mode != BOOST_EPI_PLAIN || y_dtype != 1 || epi->ssq_stride < M_b)) return BOOST_ERR_INVALID;
-  if (M_b == 0 || M_b > 128 || (y_dtype != 0 && y_dtype != 1)) return BOOST_ERR_INVALID;
+  if (M_b == 0 || M_b > 256 || (y_dtype != 0 && y_dtype != 1)) return BOOST_ERR_INVALID;
   boost_weight_layout_t lay;
   const int rc = boost_weight_layout(N, K, &lay);
   if (rc != BOOST_OK) return rc;
@@ -1637,7 +1643,8 @@ int launch_routed(const ChainParams& c, uint32_t M_b, void* stream, uint32_t* ex
     case 16: return tc ? launch_gemv_tc<16>(c, sms, st, extra_launches) : launch_gemv<2, 0>(c, sms, st, extra_launches);
     case 32: return tc ? launch_gemv_tc<32>(c, sms, st, extra_launches) : launch_gemv<4, 0>(c, sms, st, extra_launches);
     case 64: return tc ? launch_gemv_tc<64>(c, sms, st, extra_launches) : launch_gemv<8, 0>(c, sms, st, extra_launches);
-    default: return tc ? launch_gemv_tc<128>(c, sms, st, extra_launches) : launch_gemv<16, 0>(c, sms, st, extra_launches);
+    case 128: return tc ? launch_gemv_tc<128>(c, sms, st, extra_launches) : launch_gemv<16, 0>(c, sms, st, extra_launches);
+    default: return launch_gemv_tc<256>(c, sms, st, extra_launches);   // 129 - 256 rows: the tcgen05 kernel only
   }
 }
 

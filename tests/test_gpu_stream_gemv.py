@@ -79,6 +79,30 @@ def test_stream_reduce_bit_exact(dev, n_pages, ratio, policy):
         assert not ws[:(16 + n_pages) * 4].cpu().numpy().any()
 
 
+@pytest.mark.parametrize("n_pages,superpage,ratio", [(70, 7, 1 / 4), (64, 4, 1 / 8), (23, 7, 1 / 3)])
+def test_stream_reduce_over_superpage_placement(dev, n_pages, superpage, ratio):
+    """Superpages (Sec. 3.2, Sec. 4.4: groups of S pages that share a tier, S = 7 for the paper's
+    14 MB example) reach a kernel as a tier table like any other: placed by the library, checked
+    against the oracle's table, streamed host groups first, page sums bit for bit."""
+    from paper_2609_13592_b200.tiers import TieredBuffer
+    n_elems = n_pages * PAGE_ELEMS
+    buf = TieredBuffer(n_elems * 2, ratio, B.POLICY_MODULO, superpage_pages=superpage, device=dev)
+    want_tier = op.place_pages(n_elems * 2, ratio, op.POLICY_MODULO, 0, superpage)
+    assert buf.tier.tolist() == want_tier and buf.n_host > 0
+    # whole groups share a tier, and the host pages come in runs of S (the last group may be short)
+    for g0 in range(0, n_pages, superpage):
+        assert len(set(want_tier[g0:g0 + superpage])) == 1
+    buf.scatter_from(synth.small_int_bf16_torch(7, n_elems, dev))
+    ws_bytes = B.boost_stream_reduce_workspace_bytes(n_pages)
+    ws = torch.zeros(ws_bytes, dtype=torch.uint8, device=dev)
+    sums = torch.zeros(n_pages, dtype=torch.float32, device=dev)
+    B.boost_stream_reduce_tiered(buf.page_ptr, buf.order, n_pages, buf.n_host, sums, ws, ws_bytes)
+    torch.cuda.synchronize()
+    want, _ = ol.stream_sum(synth.small_int_bf16(7, n_elems), PAGE_ELEMS)
+    assert np.array_equal(sums.cpu().numpy().astype(np.float64), want)
+    assert status_word(ws) == 0
+
+
 def test_stream_reduce_all_host(dev):
     from paper_2609_13592_b200.tiers import TieredBuffer
     n_pages = 4
@@ -123,7 +147,7 @@ def test_gemv_config1(dev):
     assert w.status_words() == [0]   # no bounded wait gave up
 
 
-@pytest.mark.parametrize("m_b", [1, 2, 3, 4, 5, 8, 9, 16, 17, 32, 33, 64, 100, 128])
+@pytest.mark.parametrize("m_b", [1, 2, 3, 4, 5, 8, 9, 16, 17, 32, 33, 64, 100, 128, 129, 200, 256])
 def test_gemv_batches(dev, m_b):
     # several row tiles with a ragged last one, ragged K (5 k-blocks of 64, last one partial): one
     # page, all in HBM (the even static partition) ...
@@ -145,6 +169,7 @@ def test_gemv_batches(dev, m_b):
     (4096, 14336, 32, 1 / 8),     # down-projection shape: rows of 28 KiB, 57344-byte ... 1.75 pages per row tile
     (6144, 4096, 7, 1 / 3),
     (256, 512, 128, 0.0),
+    (4096, 4096, 256, 1 / 8),     # 256 batch rows: the widest accumulator the tcgen05 kernel takes
 ])
 def test_gemv_shapes(dev, n, k, m_b, ratio):
     w, y, ref, _ = run_gemv(dev, n, k, m_b, ratio, seed=n + k + m_b)
@@ -216,7 +241,7 @@ def test_gemv_argument_errors(dev):
         B.boost_gemv_tiered(w.buf.page_ptr, w.buf.order, 1, 0, 128, 64, x, 1, y, 0, None, ws_ptr, 16)
     assert e.value.code == B.ERR_CAPACITY
     with pytest.raises(B.BoostError) as e:
-        B.boost_gemv_tiered(w.buf.page_ptr, w.buf.order, 1, 0, 128, 64, x, 200, y, 0, None, ws_ptr, ws_bytes)
+        B.boost_gemv_tiered(w.buf.page_ptr, w.buf.order, 1, 0, 128, 64, x, 257, y, 0, None, ws_ptr, ws_bytes)
     assert e.value.code == B.ERR_INVALID
 
 
