@@ -22,7 +22,24 @@
  *     the counters in it at zero when they finish, so the same workspace can be
  *     reused by later calls on the same stream.  Calls that may overlap on the
  *     GPU need separate workspaces;
- *   - handles (boost_kv_pool_t) are not thread safe.
+ *   - the first 16 32-bit words of every workspace are its header.  Word 0 is the status
+ *     word: kernels OR error bits into it and never clear it (bit 0: a bounded wait ran out
+ *     and the kernel wound down early - its outputs are not valid; bit 1: a table index out
+ *     of range was skipped).  A non-zero status word means: zero-fill the whole workspace
+ *     before it is used again (counters may have been left mid-count).  Words 4 - 7 are the
+ *     caller's, read by the kernels and 0 in normal use: word 4 replaces the limit of every
+ *     bounded wait (GPU clock cycles; the default is about a second), word 5 - honoured only
+ *     with a non-zero word 4 - makes that many threadblocks withhold their arrival at the end
+ *     of a product of a chain (a test hook: it makes the others' waits run out), words 6 - 7
+ *     hold the device address of a schedule log (see boost_schedule_stats).  The other
+ *     header words belong to the kernels;
+ *   - every wait inside a kernel is bounded: none can hang the GPU;
+ *   - what the launch paths set up once (function attributes, occupancy) is kept per device,
+ *     indexed by the device that is current at the call, so one process may drive several
+ *     GPUs; handles (boost_kv_pool_t) are not thread safe;
+ *   - limits: head dimension 128; at most 16 query heads per KV head; the KV range of a
+ *     tensor must be placed linearly (host pages at its tail, as the pool places it);
+ *     weight products take 1 - 256 batch rows, the whole decode step 1 - 128 sequences.
  */
 #ifndef BOOST_H_
 #define BOOST_H_
@@ -322,12 +339,17 @@ int boost_pack_weights_ex(const void* w_row_major /*device*/, uint32_t N, uint32
  * cores (mma.sync up to 32 rows, tcgen05 with accumulators in tensor memory above; see
  * boost_gemv_set_tc_min_batch).  A weight with host pages is cut into work items handed out
  * host pages first; a weight entirely in HBM is cut evenly over the threadblocks.  Split-K
- * partial sums are combined in a fixed order by the last threadblock to finish a row tile, so
- * the result is deterministic (to the bit for a given placement, device and batch; across
- * placements the order of the fp32 sums, hence the last bits, may differ).
+ * partial sums meet in L2 and are combined in a fixed order - tile by tile in the threadblock
+ * that delivers a tile's last partial sum, or, for a product cut so finely that a tile has four
+ * or more, all tiles at the end of the product spread over the warps of the grid (see
+ * boost_gemv_set_end_combine; after the last product of a launch that combine runs as a small
+ * kernel of its own right behind it on the stream) - so the result is deterministic (to the bit
+ * for a given placement, device and batch; across placements the order of the fp32 sums, hence
+ * the last bits, may differ).
  * Errors: INVALID, ALIGN (x not 16-byte, workspace not 256-byte aligned, K % 8 != 0), CAPACITY,
- * CUDA.  Word 0 of the workspace collects error bits of the kernel (bit 0: a bounded wait ran
- * out; bit 1: a block index out of range in the RoPE / KV-append epilogue). */
+ * UNSUPPORTED (the device cannot hold one threadblock of the kernel), CUDA.  Status bits in
+ * word 0 of the workspace: see the conventions at the top (bit 1 here: a block index out of
+ * range in the RoPE / KV-append epilogue). */
 size_t boost_gemv_workspace_bytes(uint32_t N, uint32_t K, uint32_t M_b);
 int boost_gemv_tiered(const void* const* w_page_ptr /*device*/, const uint32_t* w_order /*device*/,
                       size_t n_pages, size_t n_host_pages, uint32_t N, uint32_t K,
@@ -426,8 +448,9 @@ typedef struct {
  * first, as in boost_gemv_tiered) while the tail of the current product drains, and meet at
  * a grid-wide counter between products.  All calls share M_b and the workspace.
  *   workspace  device, 256-byte aligned, >= boost_gemv_chain_workspace_bytes, zero-filled
- *              once (the kernel leaves its counters at zero); word 0 collects error bits
- *              (bit 0: a bounded wait ran out, including the wait between products).
+ *              once (the kernel leaves its counters at zero, so calls that follow one another
+ *              on a stream may reuse it with nothing in between); word 0 collects error bits
+ *              (bit 0: a bounded wait ran out, including the waits between products).
  * Errors: INVALID (n_calls outside 1..4, a call that boost_gemv_tiered_fused would reject),
  * ALIGN, CAPACITY, UNSUPPORTED (the device cannot hold one threadblock), CUDA. */
 size_t boost_gemv_chain_workspace_bytes(const boost_gemv_call_t* calls /*host*/, uint32_t n_calls, uint32_t M_b);
