@@ -181,6 +181,28 @@ int boost_tier_order(const uint8_t* tier /*host*/, size_t n_pages, uint32_t* ord
 
 /* ------------------------------------------------------------ materialisation */
 
+/* One virtual address range over both tiers.  The paper's kernels are unmodified library
+ * kernels: they read an ordinary address range whose 2 MiB pages have been placed on one tier
+ * or the other underneath them (Sec. 2.3: the GPU and the host memory share one address space;
+ * Sec. 4.4: the allocator binds each page of a tensor to its tier).  boost_va_buffer_create
+ * builds that on this machine with the CUDA virtual-memory API: it reserves n_pages * 2 MiB of
+ * device-visible address space and maps page i to a fresh HBM page (tier[i] = BOOST_TIER_HBM)
+ * or to a pinned page of host memory on NUMA node host_numa_node (BOOST_TIER_HOST).  The range
+ * is then one flat buffer for anything on the current device - cudaMemcpy, kernels of other
+ * libraries, this library's kernels through boost_va_buffer_page_table (page i at base +
+ * i * 2 MiB) - while every page lives where the tier table says.
+ *   tier   host array of n_pages entries (from boost_place_pages*); ownership stays with the caller;
+ *   out    receives the handle; release with boost_va_buffer_destroy (unmaps and frees all).
+ * Errors: INVALID, CAPACITY (out of HBM), UNSUPPORTED (the driver or the platform has no
+ * virtual-memory management for the tier, e.g. no host-NUMA allocations). Not thread safe. */
+typedef struct boost_va_buffer boost_va_buffer_t;
+int boost_va_buffer_create(const uint8_t* tier /*host*/, size_t n_pages, int host_numa_node,
+                           boost_va_buffer_t** out /*host*/);
+void* boost_va_buffer_base(const boost_va_buffer_t* buffer);   /* device address of page 0 */
+int boost_va_buffer_page_table(const boost_va_buffer_t* buffer, void** page_ptr_out /*host*/, size_t cap);
+int boost_va_buffer_destroy(boost_va_buffer_t* buffer);
+
+
 /* Device-visible address of a pinned (page-locked) host allocation; INVALID when the
  * pointer is not pinned host memory that the current device can address. */
 int boost_host_device_pointer(void* pinned_host, void** device_ptr_out /*host*/);

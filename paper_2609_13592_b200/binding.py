@@ -147,6 +147,10 @@ SIGNATURES = {
     "boost_rope_table": (_int, [_vp, _u32, _u32, _flt, _vp, _vp]),
     "boost_swiglu": (_int, [_vp, _u32, _u32, _vp, _vp]),
     "boost_argmax": (_int, [_vp, _u32, _u32, _vp, _vp]),
+    "boost_va_buffer_create": (_int, [_vp, C.c_size_t, _int, _vp]),
+    "boost_va_buffer_base": (C.c_void_p, [_vp]),
+    "boost_va_buffer_page_table": (_int, [_vp, _vp, C.c_size_t]),
+    "boost_va_buffer_destroy": (_int, [_vp]),
     "boost_schedule_log_bytes": (C.c_size_t, [C.c_size_t]),
     "boost_schedule_stats": (_int, [_vp, C.c_size_t, _u32, _u32, C.c_uint64, C.c_double, _vp, _vp, _vp]),
     "boost_gemv_set_tc_min_batch": (_int, [_u32]),
@@ -408,6 +412,34 @@ def gemv_calls(calls):
 
 def boost_gemv_set_tc_min_batch(m_b):
     _check(lib().boost_gemv_set_tc_min_batch(m_b), "boost_gemv_set_tc_min_batch")
+
+
+class VABuffer:
+    """Owner of a boost_va_buffer_t: one virtual range whose pages live on the tiers of `tier`."""
+
+    def __init__(self, tier, host_numa_node=0):
+        tier = np.ascontiguousarray(tier, dtype=np.uint8)
+        self.tier, self.n_pages = tier, int(tier.size)
+        self._h = C.c_void_p(0)
+        _check(lib().boost_va_buffer_create(tier.ctypes.data, tier.size, host_numa_node, C.addressof(self._h)),
+               "boost_va_buffer_create")
+        self.base = int(lib().boost_va_buffer_base(self._h))
+
+    def page_table(self):
+        out = np.zeros(self.n_pages, dtype=np.uint64)
+        _check(lib().boost_va_buffer_page_table(self._h, out.ctypes.data, out.size), "boost_va_buffer_page_table")
+        return out
+
+    def close(self):
+        if self._h:
+            lib().boost_va_buffer_destroy(self._h)
+            self._h = C.c_void_p(0)
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
 
 
 SCHED_KIND_STREAM, SCHED_KIND_GEMV, SCHED_KIND_ATTN = 1, 2, 3

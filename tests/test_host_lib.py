@@ -276,7 +276,7 @@ def test_chain_and_step_workspace_sizes_and_argument_checks():
     assert B.boost_gemv_chain_workspace_bytes(four, 128) > w4          # partial sums grow with the batch
     assert lib.boost_gemv_chain_workspace_bytes(C.addressof(four), 5, 32) == 0   # more than four products
     assert lib.boost_gemv_chain_workspace_bytes(C.addressof(four), 0, 32) == 0
-    assert B.boost_gemv_chain_workspace_bytes(four, 0) == 0 and B.boost_gemv_chain_workspace_bytes(four, 129) == 0
+    assert B.boost_gemv_chain_workspace_bytes(four, 0) == 0 and B.boost_gemv_chain_workspace_bytes(four, 257) == 0
     for n_calls in (0, 5):
         rc = lib.boost_gemv_tiered_chain(C.addressof(four), n_calls, 32, None, 1 << 30, None)
         assert rc == B.ERR_INVALID
