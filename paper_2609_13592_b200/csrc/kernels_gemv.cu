@@ -1379,8 +1379,10 @@ int launch_planned(void (*kernel)(ChainParams), void (*combine_kernel)(GemvParam
     if (g > queue_len) g = queue_len;
     if (q.even_part) {
       // at least one unit per threadblock: the partial-sum slots of a row tile are sized for that
-      // pairs of row tiles where every threadblock still gets a long run (32 units or more)
-      q.tiles_per_unit = (pairs && (uint64_t)((q.n_row_tiles + 1) / 2) * q.k_blocks >= 32ull * max_ctas) ? 2u : 1u;
+      // pairs of row tiles wherever every threadblock still gets two units or more: a stage then
+      // carries two weight blocks, and a single tile would leave half of the ring empty
+      // (measured, batch 64, down product 4096 x 14336: 61 -> 46 us inside a chain)
+      q.tiles_per_unit = (pairs && (uint64_t)((q.n_row_tiles + 1) / 2) * q.k_blocks >= 2ull * max_ctas) ? 2u : 1u;
       const uint32_t units = ((q.n_row_tiles + q.tiles_per_unit - 1) / q.tiles_per_unit) * q.k_blocks;
       g = units < max_ctas ? units : max_ctas;
     }
@@ -1394,7 +1396,15 @@ int launch_planned(void (*kernel)(ChainParams), void (*combine_kernel)(GemvParam
       const uint32_t per_cta2 = units / g ? units / g : 1;
       typical_seg = (q.k_blocks + per_cta2 - 1) / per_cta2;
     }
-    q.end_combine = (end_combine_allowed && typical_seg >= kEndCombineMinSegments) ? 1u : 0u;
+    // From 64 batch rows on (tcgen05 kernel) a tile's combine takes a threadblock's eight warps
+    // ten microseconds and more; where a threadblock holds under two units, every tile's combine
+    // would wait at the end of the phase behind its last partial sum anyway: all at once, then.
+    bool few_units = false;
+    if (q.even_part && x_rows >= 64) {
+      const uint32_t units = ((q.n_row_tiles + q.tiles_per_unit - 1) / q.tiles_per_unit) * q.k_blocks;
+      few_units = units < 2u * g * q.k_blocks;   // (a unit = one k block of a tile or pair)
+    }
+    q.end_combine = (end_combine_allowed && (typical_seg >= kEndCombineMinSegments || few_units)) ? 1u : 0u;
     q.defer_combine = (q.end_combine && i + 1 == c.n_phases && g_defer_combine) ? 1u : 0u;
   }
   // a chain keeps one grid for all phases: the full machine, so that threadblocks that run
@@ -1730,4 +1740,3 @@ extern "C" int boost_gemv_set_end_combine(uint32_t on) {
   g_end_combine = on ? 1u : 0u;
   return BOOST_OK;
 }
-
