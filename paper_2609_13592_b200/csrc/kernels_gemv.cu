@@ -907,12 +907,101 @@ constexpr uint32_t kTcEpiWarps = 8;
 constexpr uint32_t kTcEpiThreads = kTcEpiWarps * 32;
 constexpr uint32_t kTcXWarps = 4;   // activation producer warps: rows m with (m / 4) % 4 == their index
 constexpr uint32_t kTcThreads = kTcEpiThreads + 64 + 32 * kTcXWarps;
+// ring memory: what the epilogue's static arrays (row scales, the gate / up exchange buffer) leave
+constexpr uint32_t kTcSmemBudget = kSmemBudget - 10u * 1024u;
 
 // a stage: two weight blocks (the same 64 columns of two adjacent row tiles) and one activation tile
 // (at 256 batch rows the activation tile alone is 32 KiB and tensor memory holds two accumulators
 // of that width, not four: one weight block per stage, no pairs)
 __host__ __device__ constexpr uint32_t tc_weight_slots(uint32_t npad) { return npad <= 128 ? 2u : 1u; }
 __host__ __device__ constexpr uint32_t tc_stage_bytes(uint32_t npad) { return tc_weight_slots(npad) * kBlockBytes + npad * 128u; }
+
+// A row tile finished from tensor memory by the threadblock that delivered its last partial sum:
+// its own accumulator never goes to memory, the other segments' partial sums are added to it
+// in the order the combine above uses (ascending segments; even + odd where a product has more
+// than a lane's worth per round), and the epilogue runs in the accumulator's own layout -
+// thread = weight row (TMEM lane), a chunk of 16 batch rows at a time.  For the epilogues that
+// need nothing across weight rows but the gate / up partner 64 rows on, which changes hands
+// through shared memory: SwiGLU, and plain without sums of squares of the output.
+// s_rs: row scales of the phase (filled by the caller when the product has row statistics);
+// s_exch: 2 x 16 x 64 floats.  Called by all epilogue warps.
+template <uint32_t NPAD>
+__device__ __forceinline__ void tc_finish_tile(const GemvParams& p, uint32_t row_tile, uint32_t my_seg, uint32_t n_seg,
+                                               uint32_t taddr, uint32_t warp, uint32_t lane, const float* s_rs,
+                                               float* s_exch) {
+  const uint32_t quarter = warp & 3u, half = warp >> 2;
+  const uint32_t nl = quarter * 32u + lane;
+  constexpr uint32_t kColsPerGroup = NPAD >= 32 ? NPAD / 2 : NPAD;
+  const uint32_t c_begin = half * kColsPerGroup;
+  const uint32_t c_end = (NPAD >= 32 || half == 0) ? c_begin + kColsPerGroup : c_begin;
+  const bool split_mode = p.max_seg > combine_per_round<NPAD>();
+  const float* part0 = p.partials + (size_t)row_tile * p.max_seg * NPAD * kBlockRows + nl;
+  for (uint32_t c0 = c_begin; c0 < c_end; c0 += 16) {
+    float even[16], odd[16];
+#pragma unroll
+    for (uint32_t j = 0; j < 16; ++j) { even[j] = 0.f; odd[j] = 0.f; }
+    for (uint32_t s0 = 0; s0 < n_seg; s0 += 2) {
+      // segments s0 and s0 + 1: from memory, or (this threadblock's own) from tensor memory
+      float a[16], b[16];
+      const bool load_a = s0 != my_seg, has_b = s0 + 1 < n_seg, load_b = has_b && s0 + 1 != my_seg;
+      const float* pa = part0 + ((size_t)s0 * NPAD + c0) * kBlockRows;
+      const float* pb = pa + (size_t)NPAD * kBlockRows;
+      if (load_a) {
+#pragma unroll
+        for (uint32_t j = 0; j < 16; ++j) a[j] = __ldcg(pa + j * kBlockRows);
+      }
+      if (load_b) {
+#pragma unroll
+        for (uint32_t j = 0; j < 16; ++j) b[j] = __ldcg(pb + j * kBlockRows);
+      }
+      if (!load_a) tmem_ld16(taddr + c0, a);
+      else if (has_b && !load_b) tmem_ld16(taddr + c0, b);
+#pragma unroll
+      for (uint32_t j = 0; j < 16; ++j) even[j] += a[j];
+      if (has_b) {
+#pragma unroll
+        for (uint32_t j = 0; j < 16; ++j) {
+          if (split_mode) odd[j] += b[j];
+          else even[j] += b[j];
+        }
+      }
+    }
+#pragma unroll
+    for (uint32_t j = 0; j < 16; ++j) {
+      if (split_mode) even[j] += odd[j];
+      if (p.ssq_in) even[j] *= s_rs[c0 + j];
+    }
+    if (p.epi == kEpiSwiglu) {
+      // rows 64 .. 127 of the tile are the up rows of the gate rows 0 .. 63
+      float* ex = s_exch + half * (16u * 64u);
+      if (quarter >= 2) {
+#pragma unroll
+        for (uint32_t j = 0; j < 16; ++j) ex[j * 64u + (nl - 64u)] = even[j];
+      }
+      named_barrier_sync(3 + half, kTcEpiThreads / 2);
+      if (quarter < 2) {
+        __nv_bfloat16* out = static_cast<__nv_bfloat16*>(p.y) + (size_t)row_tile * 64u + nl;
+#pragma unroll
+        for (uint32_t j = 0; j < 16; ++j) {
+          const uint32_t m = c0 + j;
+          if (m < p.M_b) {
+            const float g = round_bf16(even[j]), u = round_bf16(ex[j * 64u + nl]);
+            out[(size_t)m * (p.N / 2)] = __float2bfloat16_rn(g / (1.f + expf(-g)) * u);
+          }
+        }
+      }
+      named_barrier_sync(3 + half, kTcEpiThreads / 2);   // (the next chunk overwrites the exchange buffer)
+    } else {
+      const uint32_t n = row_tile * kBlockRows + nl;
+#pragma unroll
+      for (uint32_t j = 0; j < 16; ++j) {
+        const uint32_t m = c0 + j;
+        if (m < p.M_b && n < p.N) store_out(p, m, n, even[j]);
+      }
+    }
+  }
+}
+
 
 template <uint32_t NPAD>
 __global__ void __launch_bounds__(kTcThreads, 1) gemv_tc_kernel(const __grid_constant__ ChainParams cp) {
@@ -933,6 +1022,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) gemv_tc_kernel(const __grid_con
   __shared__ uint32_t s_tmem;
   __shared__ uint32_t s_go[2];          // epilogue: thread 0's wait on an accumulator succeeded
   __shared__ volatile uint32_t s_abort; // a bounded wait ran out somewhere: everybody winds down
+  __shared__ uint32_t s_rs_phase;
 
   const uint32_t tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const uint32_t n_stages = cp.ph[0].n_stages;
@@ -954,6 +1044,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) gemv_tc_kernel(const __grid_con
       mbar_init(&acc_empty[s], kTcEpiWarps);
     }
     s_abort = 0;
+    s_rs_phase = 0xFFFFFFFFu;
     fence_barrier_init();
   }
   if (warp == kTcEpiWarps) tmem_alloc(&s_tmem, kTmemCols);
@@ -1171,6 +1262,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) gemv_tc_kernel(const __grid_con
   // so that its code (and register needs) exist once in the kernel.
   uint32_t* tile_cnt = cp.ph[0].ws + kWsHeaderWords;
   __shared__ uint32_t s_last[2];
+  __shared__ float s_rs[NPAD];           // row scales of phase s_rs_phase (tc_finish_tile)
+  __shared__ float s_exch[2 * 16 * 64];
   uint32_t buf = 0, buf_phase = 0;
   pdl_wait();
   for (;;) {
@@ -1207,15 +1300,26 @@ __global__ void __launch_bounds__(kTcThreads, 1) gemv_tc_kernel(const __grid_con
       if (tid == 0 && (mt.z >> 8) != kNoRecord) sched_log_end(sched_log_of(cp.ph[0].ws), mt.z >> 8);
       const uint32_t split = mt.y;
       const uint32_t n_tiles = (mt.z & kFlagSecond) ? 2u : 1u;   // row tiles in this accumulator
-      const uint32_t n_seg = p.even_part ? even_part_segments(p, mt.x) : p.splits;
-      const bool direct = (n_seg == 1) && p.epi == kEpiPlain && !p.ssq_in && !p.ssq_out && !p.end_combine;
+      const uint32_t n_seg = p.even_part ? even_part_segments(p, mt.x) : p.splits;   // (the same for both tiles of a pair)
       const uint32_t quarter = warp & 3u, half = warp >> 2;
       const uint32_t nl = quarter * 32 + lane;                                 // weight row of this thread = its TMEM lane
       // warps 0-3 read the first half of the columns, warps 4-7 the second (16 columns: the first group reads all)
       constexpr uint32_t kColsPerGroup = NPAD >= 32 ? NPAD / 2 : NPAD;
       const uint32_t c_begin = half * kColsPerGroup;
       const uint32_t c_end = (NPAD >= 32 || half == 0) ? c_begin + kColsPerGroup : c_begin;
+      // Tile by tile, with an epilogue that works in the accumulator's layout: whoever holds
+      // the last partial sum of a tile keeps it in tensor memory and finishes the tile from
+      // there (tc_finish_tile); the others write theirs out.  A tile's counter holds the
+      // arrivals in its low half and the partial sums in memory in its high half.
+      const bool native = !p.end_combine && (p.epi == kEpiSwiglu || (p.epi == kEpiPlain && !p.ssq_out));
+      if (native && n_seg > 1) {
+        if (tid < n_tiles) s_last[tid] = ((atomicAdd(tile_cnt + mt.x + tid, 1u) & 0xFFFFu) == n_seg - 1) ? 1u : 0u;
+        named_barrier_sync(1, kTcEpiThreads);
+      }
+      bool stored = false;
       for (uint32_t ti = 0; ti < n_tiles; ++ti) {
+        if (native && (n_seg == 1 || s_last[ti])) continue;
+        stored = true;
         const uint32_t row_tile = mt.x + ti;
         float* part = p.partials + ((size_t)row_tile * p.max_seg + split) * NPAD * kBlockRows;
         const uint32_t taddr = tmem_base + ((quarter * 32u) << 16) + buf * kSlots * NPAD + ti * NPAD;
@@ -1223,23 +1327,65 @@ __global__ void __launch_bounds__(kTcThreads, 1) gemv_tc_kernel(const __grid_con
           float v[16];
           tmem_ld16(taddr + c0, v);
 #pragma unroll
-          for (uint32_t j = 0; j < 16; ++j) {
-            const uint32_t m = c0 + j;                                         // batch row = accumulator column
-            if (direct) {
-              const uint32_t n = row_tile * kBlockRows + nl;
-              if (m < p.M_b && n < p.N) store_out(p, m, n, v[j]);
-            } else {
-              __stcg(part + m * kBlockRows + nl, v[j]);
+          for (uint32_t j = 0; j < 16; ++j) __stcg(part + (c0 + j) * kBlockRows + nl, v[j]);   // batch row = accumulator column
+        }
+      }
+      if (native) {
+        if (stored) {
+          named_barrier_sync(1, kTcEpiThreads);   // everybody's stores come before the release
+          if (tid < n_tiles && !s_last[tid]) red_add_release(tile_cnt + mt.x + tid, 0x10000u);
+        }
+        bool gave_up = false;
+        for (uint32_t ti = 0; ti < n_tiles; ++ti) {
+          if (n_seg > 1 && !s_last[ti]) continue;
+          const uint32_t row_tile = mt.x + ti;
+          if (n_seg > 1) {
+            // the other segments' partial sums: all in memory?  (their threadblocks are past
+            // their arrival and wait for nothing on the way to the release)
+            if (tid == 0) {
+              const bool ok = grid_counter_wait(tile_cnt + row_tile, (n_seg - 1) << 16, status);
+              if (!ok) s_abort = 1;
+              s_go[buf] = ok ? 1u : 0u;
+            }
+            named_barrier_sync(1, kTcEpiThreads);
+            if (!s_go[buf]) { gave_up = true; break; }
+            __threadfence();
+          }
+          if (p.ssq_in) {
+            // row scales of this phase's activations, once per phase (in the combine's order of sums)
+            named_barrier_sync(1, kTcEpiThreads);
+            if (s_rs_phase != mt.w) {
+              const uint32_t v = tid & 15u;
+              for (uint32_t m = tid >> 4; m < NPAD; m += kTcEpiThreads / 16) {
+                float ss = 0.f, ss0 = 0.f, ss1 = 0.f;
+                if (m < p.M_b) {
+                  if (v < p.ssq_in_tiles) ss0 = __ldcg(p.ssq_in + (size_t)v * p.ssq_stride + m);
+                  if (v + 16 < p.ssq_in_tiles) ss1 = __ldcg(p.ssq_in + (size_t)(v + 16) * p.ssq_stride + m);
+                  for (uint32_t t0 = v + 32; t0 < p.ssq_in_tiles; t0 += 16) ss += __ldcg(p.ssq_in + (size_t)t0 * p.ssq_stride + m);
+                }
+                ss += ss0 + ss1;
+                ss += __shfl_xor_sync(0xFFFFFFFFu, ss, 1);
+                ss += __shfl_xor_sync(0xFFFFFFFFu, ss, 2);
+                ss += __shfl_xor_sync(0xFFFFFFFFu, ss, 4);
+                ss += __shfl_xor_sync(0xFFFFFFFFu, ss, 8);
+                if (v == 0) s_rs[m] = rsqrtf(ss / (float)p.x_cols + p.rms_eps);
+              }
+              named_barrier_sync(1, kTcEpiThreads);
+              if (tid == 0) s_rs_phase = mt.w;
             }
           }
+          tc_finish_tile<NPAD>(p, row_tile, split, n_seg, tmem_base + ((quarter * 32u) << 16) + buf * kSlots * NPAD + ti * NPAD, warp,
+                               lane, s_rs, s_exch);
+          if (n_seg > 1 && tid == 0) tile_cnt[row_tile] = 0;
         }
+        if (gave_up) break;
       }
       // the accumulators may be overwritten
       tc_fence_before_sync();
       __syncwarp();
       if (lane == 0) mbar_arrive(&acc_empty[buf]);
       if (++buf == 2) { buf = 0; buf_phase ^= 1u; }
-      if (!direct && !p.end_combine) {
+      if (!native && !p.end_combine) {
         // the threadblock that delivers the last partial sum of a row tile combines it
         named_barrier_sync(1, kTcEpiThreads);
         if (tid < n_tiles) s_last[tid] = atom_add_acq_rel(tile_cnt + mt.x + tid, 1u) == n_seg - 1 ? 1u : 0u;   // release ours, acquire the others'
@@ -1348,14 +1494,14 @@ struct KernelState {
 
 // pairs: the even partition counts (pair of row tiles, k block) units instead of blocks.
 int launch_planned(void (*kernel)(ChainParams), void (*combine_kernel)(GemvParams), uint32_t x_rows, KernelState& state,
-                   uint32_t threads, uint32_t stage_bytes, uint32_t ctas_per_sm, bool pairs, bool end_combine_allowed,
+                   uint32_t threads, uint32_t stage_bytes, uint32_t smem_budget, uint32_t ctas_per_sm, bool pairs, bool end_combine_allowed,
                    const ChainParams& chain, int sms, cudaStream_t stream, uint32_t* extra_launches) {
   ChainParams c = chain;
-  uint32_t n_stages = (kSmemBudget / ctas_per_sm - 1024) / stage_bytes;
+  uint32_t n_stages = (smem_budget / ctas_per_sm - 1024) / stage_bytes;
   if (n_stages > kMaxStages) n_stages = kMaxStages;
   const size_t smem = (size_t)n_stages * stage_bytes + 1024;
   if (!state.configured) {
-    int rc = boosth::check(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(kSmemBudget + 1024)));
+    int rc = boosth::check(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(smem_budget + 1024)));
     if (rc != BOOST_OK) return rc;
     rc = boosth::check(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&state.resident, kernel, (int)threads, smem));
     if (rc != BOOST_OK) return rc;
@@ -1444,7 +1590,7 @@ int launch_gemv(const ChainParams& chain, int sms, cudaStream_t stream, uint32_t
   if (slot < 0) return BOOST_ERR_CUDA;
   KernelState& state = states[slot];
   return launch_planned(gemv_tiered_kernel<NT, MB>, gemv_combine_kernel<x_rows_of(NT, MB)>, x_rows_of(NT, MB), state, kGemvThreads,
-                        stage_bytes_of(NT, MB), (NT >= 8) ? 1 : 2, false, g_end_combine != 0, chain, sms, stream, extra_launches);
+                        stage_bytes_of(NT, MB), kSmemBudget, (NT >= 8) ? 1 : 2, false, g_end_combine != 0, chain, sms, stream, extra_launches);
 }
 
 template <uint32_t NPAD>
@@ -1453,7 +1599,7 @@ int launch_gemv_tc(const ChainParams& chain, int sms, cudaStream_t stream, uint3
   const int slot = boosth::device_slot();
   if (slot < 0) return BOOST_ERR_CUDA;
   KernelState& state = states[slot];
-  return launch_planned(gemv_tc_kernel<NPAD>, gemv_combine_kernel<NPAD>, NPAD, state, kTcThreads, tc_stage_bytes(NPAD), 1,
+  return launch_planned(gemv_tc_kernel<NPAD>, gemv_combine_kernel<NPAD>, NPAD, state, kTcThreads, tc_stage_bytes(NPAD), kTcSmemBudget, 1,
                         tc_weight_slots(NPAD) == 2,
                         g_end_combine != 0, chain, sms, stream, extra_launches);
 }
