@@ -93,6 +93,21 @@ __device__ __forceinline__ void bulk_copy_g2s(void* dst_smem, const void* src, u
       : "memory");
 }
 
+// Tiled (tensor-map) copy global -> shared through the TMA unit: the box of the map at
+// coordinates (c0 = innermost, in elements; c1 = row); completion is counted in bytes on `bar`.
+// c0 x element size must be a multiple of 16 bytes; elements outside the tensor arrive as zeros.
+__device__ __forceinline__ void tma_load_2d(void* dst_smem, const void* tensor_map, int32_t c0, int32_t c1, uint64_t* bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];" ::"r"(
+          smem_u32(dst_smem)),
+      "l"(tensor_map), "r"(smem_u32(bar)), "r"(c0), "r"(c1)
+      : "memory");
+}
+
+// Orders this thread's earlier generic-proxy view of memory (what it has acquired from other
+// threads' ordinary stores) before its later copies through the asynchronous proxy (TMA).
+__device__ __forceinline__ void fence_proxy_async_all() { asm volatile("fence.proxy.async;" ::: "memory"); }
+
 // 16-byte asynchronous copy through the load/store path (works on any mapped address,
 // host-pinned pages included); src_bytes = 0 writes zeros.
 __device__ __forceinline__ void cp_async_16(void* dst_smem, const void* src, uint32_t src_bytes) {

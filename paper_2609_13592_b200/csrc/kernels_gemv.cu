@@ -11,6 +11,7 @@
 // items (runs of blocks of one row tile inside one page, host-tier items first, Sec. 3.2), so a
 // threadblock reads one tier at a time; a weight entirely in HBM is cut evenly over the
 // threadblocks.  Split-K partial sums meet in L2 and are combined in a fixed order.
+#include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdlib.h>
@@ -128,6 +129,9 @@ struct ChainParams {
 
   uint32_t* bar;   // n_phases > 1: counters [kMaxPhases + 1], zero at rest (one per phase boundary, one for the exit)
   GemvParams ph[kMaxPhases];
+  // tcgen05 kernel: the activations of each phase as a tiled tensor map (box = 64 columns x the
+  // padded batch, 128-byte swizzle: the B operand's shared-memory layout as the copy lands)
+  alignas(64) CUtensorMap x_map[kMaxPhases];
 };
 
 __host__ __device__ constexpr uint32_t x_rows_of(int NT, int MB) { return NT > 0 ? NT * 8 : MB; }
@@ -899,14 +903,17 @@ __global__ void __launch_bounds__(kConsumerThreads) gemv_combine_kernel(const __
 // next segment accumulates while four epilogue warps read the finished one back
 // (tcgen05.ld), write the partial sums and run the same combine as the kernel above.
 // Warps: 0-7 epilogue (warp w reads TMEM lanes 32 (w % 4) .. + 31 = weight rows, and the half
-// w / 4 of the accumulator's columns), 8 MMA issue and TMEM allocation, 9 weight producer,
-// 10-13 activation producers.  One threadblock per SM (the driver keeps kernels that allocate
-// tensor memory at one per SM at this shared-memory size) with the whole shared memory as its
-// ring: no warp reads an operand back, so the ring's bandwidth is all HBM's.
+// w / 4 of the accumulator's columns), 8 MMA issue and TMEM allocation, 9 weight producer
+// (bulk copies; 16-byte copies of all its lanes for host-tier blocks), 10 activation producer
+// (one thread: a tiled TMA copy per stage lands x[:, 64 kb .. + 64) in the B operand's swizzled
+// layout, rows beyond the batch as zeros).  Eleven warps, three to an SM sub-partition at most,
+// leave each thread 168 registers: the epilogue's sums in flight.  One threadblock per SM (the
+// driver keeps kernels that allocate tensor memory at one per SM at this shared-memory size)
+// with nearly all shared memory as its ring: no warp reads an operand back, so the ring's
+// bandwidth is all HBM's.
 constexpr uint32_t kTcEpiWarps = 8;
 constexpr uint32_t kTcEpiThreads = kTcEpiWarps * 32;
-constexpr uint32_t kTcXWarps = 4;   // activation producer warps: rows m with (m / 4) % 4 == their index
-constexpr uint32_t kTcThreads = kTcEpiThreads + 64 + 32 * kTcXWarps;
+constexpr uint32_t kTcThreads = kTcEpiThreads + 96;   // + MMA warp, weight producer, activation producer
 // ring memory: what the epilogue's static arrays (row scales, the gate / up exchange buffer) leave
 constexpr uint32_t kTcSmemBudget = kSmemBudget - 10u * 1024u;
 
@@ -1032,12 +1039,12 @@ __global__ void __launch_bounds__(kTcThreads, 1) gemv_tc_kernel(const __grid_con
   pdl_launch_dependents();
   if (tid == 0) {
     for (uint32_t s = 0; s < n_stages; ++s) {
-      mbar_init(&full_bar[s], 33 + 32 * kTcXWarps);   // cp.async arrivals of the producer warps + the arrive.expect_tx
+      mbar_init(&full_bar[s], 34);   // the two producers' arrive.expect_tx + the cp.async arrivals of the weight warp
       mbar_init(&empty_bar[s], 1);   // the commit of the MMAs that read the stage
     }
     for (uint32_t s = 0; s < 4; ++s) {
       mbar_init(&item_full[s], 1);
-      mbar_init(&item_empty[s], kTcXWarps);
+      mbar_init(&item_empty[s], 1);
     }
     for (uint32_t s = 0; s < 2; ++s) {
       mbar_init(&acc_full[s], 1);
@@ -1056,7 +1063,6 @@ __global__ void __launch_bounds__(kTcThreads, 1) gemv_tc_kernel(const __grid_con
   if (warp > kTcEpiWarps) {
     // ------------------------------------------------------------------ producer warps (as above)
     const bool leader = (warp == kTcEpiWarps + 1);
-    const uint32_t xw = warp - (kTcEpiWarps + 2);   // index among the activation producer warps
     uint32_t stage = 0, phase = 0, icount = 0;
     unsigned long long* const sched_log = (leader && lane == 0) ? sched_log_of(cp.ph[0].ws) : nullptr;
     uint32_t rec = kNoRecord;   // schedule-log record of the item in production (weight warp, lane 0)
@@ -1072,10 +1078,11 @@ __global__ void __launch_bounds__(kTcThreads, 1) gemv_tc_kernel(const __grid_con
         if (lane == 0 && !grid_counter_wait(cp.bar + kBarPhase + (ph - 1), gridDim.x, status)) s_abort = 1;
         __syncwarp();
       }
-      // one block: the weight warp copies it, the activation warp stages x[:, 64 kb .. 64 kb + 64)
-      // as NPAD rows of 128 bytes in the 128-byte swizzle (rows >= M_b are zero)
+      // (the activations were written with ordinary stores, by this launch or the one before,
+      // and are read through the TMA unit)
+      if (!leader) fence_proxy_async_all();
       // one stage: the weight warp copies the weight block (two blocks in pair mode), the
-      // activation warps stage x[:, 64 kb .. 64 kb + 64) as NPAD rows of 128 bytes in the
+      // activation producer requests x[:, 64 kb .. 64 kb + 64) as NPAD rows of 128 bytes in the
       // 128-byte swizzle (rows >= M_b are zero)
       auto produce = [&](const uint8_t* src, const uint8_t* src1, bool from_host, uint32_t row_tile, uint32_t seg,
                          uint32_t flags, uint32_t kb) {
@@ -1098,17 +1105,13 @@ __global__ void __launch_bounds__(kTcThreads, 1) gemv_tc_kernel(const __grid_con
           }
           cp_async_arrive_noinc(&full_bar[stage]);
         } else {
-          if (!mbar_wait(&empty_bar[stage], phase ^ 1u, status)) s_abort = 1;
-          const uint32_t c = lane & 7, m0 = (lane >> 3) + 4 * xw;
-          uint8_t* xbase = smem + (size_t)stage * kStageBytes + kSlots * kBlockBytes;
-          const uint32_t k = kb * kBlockK + c * 8;
-          const bool k_ok = k < p.K;
-#pragma unroll 4
-          for (uint32_t m = m0; m < NPAD; m += 4 * kTcXWarps) {
-            const bool live = k_ok && m < p.M_b;
-            cp_async_16(xbase + m * 128 + ((c ^ (m & 7)) << 4), p.x + (live ? (size_t)m * p.K + k : 0u), live ? 16u : 0u);
+          if (lane == 0) {
+            if (!mbar_wait(&empty_bar[stage], phase ^ 1u, status)) s_abort = 1;
+            mbar_arrive_expect_tx(&full_bar[stage], NPAD * 128u);
+            tma_load_2d(smem + (size_t)stage * kStageBytes + kSlots * kBlockBytes, &cp.x_map[ph], (int32_t)(kb * kBlockK), 0,
+                        &full_bar[stage]);
           }
-          cp_async_arrive_noinc(&full_bar[stage]);
+          __syncwarp();
         }
         if (++stage == n_stages) { stage = 0; phase ^= 1u; }
       };
@@ -1197,8 +1200,11 @@ __global__ void __launch_bounds__(kTcThreads, 1) gemv_tc_kernel(const __grid_con
         cp_async_arrive_noinc(&full_bar[stage]);
         if (lane == 0 && active && !p.even_part) q.finish(p.active_ctas);
       } else {
-        mbar_wait(&empty_bar[stage], phase ^ 1u, status);
-        cp_async_arrive_noinc(&full_bar[stage]);
+        if (lane == 0) {
+          mbar_wait(&empty_bar[stage], phase ^ 1u, status);
+          mbar_arrive(&full_bar[stage]);
+        }
+        __syncwarp();
       }
       if (++stage == n_stages) { stage = 0; phase ^= 1u; }
     }
@@ -1593,12 +1599,44 @@ int launch_gemv(const ChainParams& chain, int sms, cudaStream_t stream, uint32_t
                         stage_bytes_of(NT, MB), kSmemBudget, (NT >= 8) ? 1 : 2, false, g_end_combine != 0, chain, sms, stream, extra_launches);
 }
 
+// Tensor map of a phase's activations x [M_b, K] (bf16, row-major) for the tcgen05 kernel: boxes of
+// 64 columns x npad rows in the 128-byte swizzle; rows and columns beyond the tensor read as zero.
+// The driver's encoder is looked up at run time (no link-time dependency on the driver library).
+int encode_x_map(CUtensorMap* map, const void* x, uint32_t M_b, uint32_t K, uint32_t npad) {
+  using Encode = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                              const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                              CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+  static Encode encode = [] {
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult st;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &st) != cudaSuccess ||
+        st != cudaDriverEntryPointSuccess)
+      fn = nullptr;
+    return reinterpret_cast<Encode>(fn);
+  }();
+  if (!encode) return BOOST_ERR_UNSUPPORTED;
+  const cuuint64_t dims[2] = {K, M_b};
+  const cuuint64_t strides[1] = {(cuuint64_t)K * 2};
+  const cuuint32_t box[2] = {kBlockK, npad};
+  const cuuint32_t elem[2] = {1, 1};
+  const CUresult r = encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(x), dims, strides, box, elem,
+                            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? BOOST_OK : BOOST_ERR_ALIGN;
+}
+
 template <uint32_t NPAD>
-int launch_gemv_tc(const ChainParams& chain, int sms, cudaStream_t stream, uint32_t* extra_launches) {
+int launch_gemv_tc(const ChainParams& chain_in, int sms, cudaStream_t stream, uint32_t* extra_launches) {
   static KernelState states[boosth::kMaxDevices];
   const int slot = boosth::device_slot();
   if (slot < 0) return BOOST_ERR_CUDA;
   KernelState& state = states[slot];
+  ChainParams chain = chain_in;
+  for (uint32_t i = 0; i < chain.n_phases; ++i) {
+    const GemvParams& q = chain.ph[i];
+    const int rc = encode_x_map(&chain.x_map[i], q.x, q.M_b, q.K, NPAD);
+    if (rc != BOOST_OK) return rc;
+  }
   return launch_planned(gemv_tc_kernel<NPAD>, gemv_combine_kernel<NPAD>, NPAD, state, kTcThreads, tc_stage_bytes(NPAD), kTcSmemBudget, 1,
                         tc_weight_slots(NPAD) == 2,
                         g_end_combine != 0, chain, sms, stream, extra_launches);
