@@ -135,9 +135,41 @@ __global__ void __launch_bounds__(kAttnThreads, (NH == 1 ? 3 : 2)) paged_attn_ke
 #pragma unroll
   for (uint32_t w = 0; w < kAttnWarps; ++w) { total_blocks += s_warp_sum[w]; longest = max(longest, s_warp_max[w]); }
   const bool mixed = (uint64_t)longest * p.B * 4 > total_blocks * 5;
-  const uint64_t quarters = mixed ? 4 : 7;   // run cap in quarters of u
-  const uint64_t run_cap = (total_blocks * p.Hkv * quarters + (uint64_t)p.cta_slots * 4 - 1) / ((uint64_t)p.cta_slots * 4);
-  const uint32_t item_blocks = (uint32_t)min((uint64_t)kMaxItemBlocks, max((uint64_t)kMinItemBlocks, (run_cap + kAttnWarps - 1) / kAttnWarps));
+  uint32_t item_blocks;
+  if (mixed) {
+    const uint64_t run_cap = (total_blocks * p.Hkv + (uint64_t)p.cta_slots - 1) / (uint64_t)p.cta_slots;   // u
+    item_blocks = (uint32_t)min((uint64_t)kMaxItemBlocks, max((uint64_t)kMinItemBlocks, (run_cap + kAttnWarps - 1) / kAttnWarps));
+  } else {
+    // Sequences about equally long, each cut into s runs: the slots take the items in rounds; a
+    // full round streams at the HBM rate, the last one at the rate its items can draw (a
+    // threadblock alone gets 1 / (55 % of the slots) of it), and every round costs a hand-over
+    // (table look-up, query load, merge: about 5 us = 4000 block times).  In units of the time
+    // HBM takes for one KV block: cost(s) = run x (full rounds x slots + max(55 % of slots,
+    // items of the last round)) + 4000 x rounds.  The s with the least cost wins.
+    // (single precision and 32-bit integers: every thread of every threadblock runs this)
+    const uint32_t slots = p.cta_slots;
+    const float sat = 0.55f * (float)slots, inv_slots = 1.f / (float)slots;
+    const uint32_t mean = ((uint32_t)total_blocks + p.B - 1) / p.B;
+    float best = 3.0e38f;
+    item_blocks = kMaxItemBlocks;
+    // candidates: 1 .. 4 runs per sequence, and one run per slot over 4 / 7 of the slots (runs of
+    // 1.75 times the blocks a slot gets on average: what long sequences in small batches need)
+    const uint32_t per_slot = ((uint32_t)total_blocks * p.Hkv * 7u + slots * 4u - 1u) / (slots * 4u);
+    // (one run per sequence that fills one round well needs no search)
+    const uint32_t whole = p.B * p.Hkv;
+    const bool one_round = longest <= kAttnWarps * kMaxItemBlocks && whole <= slots && (float)whole >= sat;
+    if (one_round) item_blocks = max(kMinItemBlocks, (longest + kAttnWarps - 1) / kAttnWarps);
+    for (uint32_t s = 0; s <= 4 && !one_round; ++s) {
+      const uint32_t run = s ? (longest + s - 1) / s : per_slot;
+      const uint32_t ib = min(kMaxItemBlocks, max(kMinItemBlocks, (run + kAttnWarps - 1) / kAttnWarps));
+      const uint32_t n_spl = mean ? (mean + kAttnWarps * ib - 1) / (kAttnWarps * ib) : 1u;
+      const float len = mean ? (float)((mean + n_spl - 1) / n_spl) : 0.f;
+      const float items = (float)(p.B * p.Hkv * n_spl);
+      const float full = floorf(items * inv_slots + 1e-4f), tail = items - full * (float)slots;
+      const float cost = len * (full * (float)slots + (tail > 0.5f ? fmaxf(sat, tail) : 0.f)) + 4000.f * (full + (tail > 0.5f ? 1.f : 0.f));
+      if (cost < best) { best = cost; item_blocks = ib; }
+    }
+  }
   const uint32_t cta_max = kAttnWarps * item_blocks;
   const uint32_t max_splits = (p.max_blocks + cta_max - 1) / cta_max;
   // ---- item list.  Up to kMaxListedSeqs sequences: items are numbered densely, sequence by

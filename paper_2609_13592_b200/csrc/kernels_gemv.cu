@@ -129,8 +129,12 @@ struct ChainParams {
 
   uint32_t* bar;   // n_phases > 1: counters [kMaxPhases + 1], zero at rest (one per phase boundary, one for the exit)
   GemvParams ph[kMaxPhases];
-  // tcgen05 kernel: the activations of each phase as a tiled tensor map (box = 64 columns x the
-  // padded batch, 128-byte swizzle: the B operand's shared-memory layout as the copy lands)
+};
+
+// tcgen05 kernel: the chain, and the activations of each phase as a tiled tensor map (box = 64
+// columns x the padded batch, 128-byte swizzle: the B operand's shared-memory layout as the copy lands)
+struct TcChainParams {
+  ChainParams chain;
   alignas(64) CUtensorMap x_map[kMaxPhases];
 };
 
@@ -1011,7 +1015,8 @@ __device__ __forceinline__ void tc_finish_tile(const GemvParams& p, uint32_t row
 
 
 template <uint32_t NPAD>
-__global__ void __launch_bounds__(kTcThreads, 1) gemv_tc_kernel(const __grid_constant__ ChainParams cp) {
+__global__ void __launch_bounds__(kTcThreads, 1) gemv_tc_kernel(const __grid_constant__ TcChainParams tp) {
+  const ChainParams& cp = tp.chain;
   constexpr uint32_t kStageBytes = tc_stage_bytes(NPAD);
   constexpr uint32_t kSlots = tc_weight_slots(NPAD);
   constexpr uint32_t kTmemCols = 2 * kSlots * NPAD < 32 ? 32 : 2 * kSlots * NPAD;   // one accumulator per weight slot, double-buffered
@@ -1108,7 +1113,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) gemv_tc_kernel(const __grid_con
           if (lane == 0) {
             if (!mbar_wait(&empty_bar[stage], phase ^ 1u, status)) s_abort = 1;
             mbar_arrive_expect_tx(&full_bar[stage], NPAD * 128u);
-            tma_load_2d(smem + (size_t)stage * kStageBytes + kSlots * kBlockBytes, &cp.x_map[ph], (int32_t)(kb * kBlockK), 0,
+            tma_load_2d(smem + (size_t)stage * kStageBytes + kSlots * kBlockBytes, &tp.x_map[ph], (int32_t)(kb * kBlockK), 0,
                         &full_bar[stage]);
           }
           __syncwarp();
@@ -1499,7 +1504,8 @@ struct KernelState {
 };
 
 // pairs: the even partition counts (pair of row tiles, k block) units instead of blocks.
-int launch_planned(void (*kernel)(ChainParams), void (*combine_kernel)(GemvParams), uint32_t x_rows, KernelState& state,
+template <typename KernelParams, typename Wrap>
+int launch_planned(void (*kernel)(KernelParams), Wrap wrap, void (*combine_kernel)(GemvParams), uint32_t x_rows, KernelState& state,
                    uint32_t threads, uint32_t stage_bytes, uint32_t smem_budget, uint32_t ctas_per_sm, bool pairs, bool end_combine_allowed,
                    const ChainParams& chain, int sms, cudaStream_t stream, uint32_t* extra_launches) {
   ChainParams c = chain;
@@ -1572,7 +1578,7 @@ int launch_planned(void (*kernel)(ChainParams), void (*combine_kernel)(GemvParam
     }
     q.n_host_ctas = n_host_ctas;
   }
-  int rc = boosth::launch_chained(kernel, dim3(grid), dim3(threads), smem, stream, c);
+  int rc = boosth::launch_chained(kernel, dim3(grid), dim3(threads), smem, stream, wrap(c));
   const GemvParams& last = c.ph[c.n_phases - 1];
   if (rc == BOOST_OK && last.defer_combine) {
     // one slot per warp where the machine has the warps for it (two small threadblocks per SM)
@@ -1595,7 +1601,8 @@ int launch_gemv(const ChainParams& chain, int sms, cudaStream_t stream, uint32_t
   const int slot = boosth::device_slot();
   if (slot < 0) return BOOST_ERR_CUDA;
   KernelState& state = states[slot];
-  return launch_planned(gemv_tiered_kernel<NT, MB>, gemv_combine_kernel<x_rows_of(NT, MB)>, x_rows_of(NT, MB), state, kGemvThreads,
+  return launch_planned(gemv_tiered_kernel<NT, MB>, [](const ChainParams& c) -> const ChainParams& { return c; },
+                        gemv_combine_kernel<x_rows_of(NT, MB)>, x_rows_of(NT, MB), state, kGemvThreads,
                         stage_bytes_of(NT, MB), kSmemBudget, (NT >= 8) ? 1 : 2, false, g_end_combine != 0, chain, sms, stream, extra_launches);
 }
 
@@ -1626,18 +1633,22 @@ int encode_x_map(CUtensorMap* map, const void* x, uint32_t M_b, uint32_t K, uint
 }
 
 template <uint32_t NPAD>
-int launch_gemv_tc(const ChainParams& chain_in, int sms, cudaStream_t stream, uint32_t* extra_launches) {
+int launch_gemv_tc(const ChainParams& chain, int sms, cudaStream_t stream, uint32_t* extra_launches) {
   static KernelState states[boosth::kMaxDevices];
   const int slot = boosth::device_slot();
   if (slot < 0) return BOOST_ERR_CUDA;
   KernelState& state = states[slot];
-  ChainParams chain = chain_in;
+  TcChainParams tp;
   for (uint32_t i = 0; i < chain.n_phases; ++i) {
     const GemvParams& q = chain.ph[i];
-    const int rc = encode_x_map(&chain.x_map[i], q.x, q.M_b, q.K, NPAD);
+    const int rc = encode_x_map(&tp.x_map[i], q.x, q.M_b, q.K, NPAD);
     if (rc != BOOST_OK) return rc;
   }
-  return launch_planned(gemv_tc_kernel<NPAD>, gemv_combine_kernel<NPAD>, NPAD, state, kTcThreads, tc_stage_bytes(NPAD), kTcSmemBudget, 1,
+  auto wrap = [&tp](const ChainParams& c) -> const TcChainParams& {
+    tp.chain = c;
+    return tp;
+  };
+  return launch_planned(gemv_tc_kernel<NPAD>, wrap, gemv_combine_kernel<NPAD>, NPAD, state, kTcThreads, tc_stage_bytes(NPAD), kTcSmemBudget, 1,
                         tc_weight_slots(NPAD) == 2,
                         g_end_combine != 0, chain, sms, stream, extra_launches);
 }
