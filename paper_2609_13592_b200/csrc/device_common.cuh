@@ -246,6 +246,26 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, float (&v)[16]) {
   for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
 }
 
+// kN = 16 or 32 consecutive columns of this warp's 32 TMEM lanes.
+template <uint32_t kN>
+__device__ __forceinline__ void tmem_ld(uint32_t taddr, float (&v)[kN]) {
+  static_assert(kN == 16 || kN == 32, "16 or 32 columns");
+  uint32_t r[kN];
+#pragma unroll
+  for (uint32_t h = 0; h < kN / 16; ++h)
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+        : "=r"(r[16 * h + 0]), "=r"(r[16 * h + 1]), "=r"(r[16 * h + 2]), "=r"(r[16 * h + 3]), "=r"(r[16 * h + 4]),
+          "=r"(r[16 * h + 5]), "=r"(r[16 * h + 6]), "=r"(r[16 * h + 7]), "=r"(r[16 * h + 8]), "=r"(r[16 * h + 9]),
+          "=r"(r[16 * h + 10]), "=r"(r[16 * h + 11]), "=r"(r[16 * h + 12]), "=r"(r[16 * h + 13]), "=r"(r[16 * h + 14]),
+          "=r"(r[16 * h + 15])
+        : "r"(taddr + 16 * h)
+        : "memory");
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+  for (uint32_t i = 0; i < kN; ++i) v[i] = __uint_as_float(r[i]);
+}
+
 // Two bf16 packed in a 32-bit word -> two floats (bf16 is the top half of an fp32).
 __device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
 __device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xFFFF0000u); }

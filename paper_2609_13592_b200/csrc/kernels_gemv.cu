@@ -919,7 +919,7 @@ constexpr uint32_t kTcEpiWarps = 8;
 constexpr uint32_t kTcEpiThreads = kTcEpiWarps * 32;
 constexpr uint32_t kTcThreads = kTcEpiThreads + 96;   // + MMA warp, weight producer, activation producer
 // ring memory: what the epilogue's static arrays (row scales, the gate / up exchange buffer) leave
-constexpr uint32_t kTcSmemBudget = kSmemBudget - 10u * 1024u;
+constexpr uint32_t kTcSmemBudget = kSmemBudget - 18u * 1024u;
 
 // a stage: two weight blocks (the same 64 columns of two adjacent row tiles) and one activation tile
 // (at 256 batch rows the activation tile alone is 32 KiB and tensor memory holds two accumulators
@@ -929,90 +929,79 @@ __host__ __device__ constexpr uint32_t tc_stage_bytes(uint32_t npad) { return tc
 
 // A row tile finished from tensor memory by the threadblock that delivered its last partial sum:
 // its own accumulator never goes to memory, the other segments' partial sums are added to it
-// in the order the combine above uses (ascending segments; even + odd where a product has more
-// than a lane's worth per round), and the epilogue runs in the accumulator's own layout -
-// thread = weight row (TMEM lane), a chunk of 16 batch rows at a time.  For the epilogues that
+// in the order the combine above uses for products with few partial sums per tile (ascending
+// segments), and the epilogue runs in the accumulator's own layout - thread = weight row (TMEM
+// lane), 32 batch rows at a time (16 for small batches).  For the epilogues that
 // need nothing across weight rows but the gate / up partner 64 rows on, which changes hands
 // through shared memory: SwiGLU, and plain without sums of squares of the output.
 // s_rs: row scales of the phase (filled by the caller when the product has row statistics);
-// s_exch: 2 x 16 x 64 floats.  Called by all epilogue warps.
+// s_exch: 2 x tc_finish_cols x 64 floats.  Called by all epilogue warps.
+// columns (batch rows) per pass of tc_finish_tile
+template <uint32_t NPAD>
+__host__ __device__ constexpr uint32_t tc_finish_cols() { return NPAD >= 64 ? 32u : 16u; }
+
 template <uint32_t NPAD>
 __device__ __forceinline__ void tc_finish_tile(const GemvParams& p, uint32_t row_tile, uint32_t my_seg, uint32_t n_seg,
                                                uint32_t taddr, uint32_t warp, uint32_t lane, const float* s_rs,
                                                float* s_exch) {
+  constexpr uint32_t kC = tc_finish_cols<NPAD>();
   const uint32_t quarter = warp & 3u, half = warp >> 2;
   const uint32_t nl = quarter * 32u + lane;
   constexpr uint32_t kColsPerGroup = NPAD >= 32 ? NPAD / 2 : NPAD;
   const uint32_t c_begin = half * kColsPerGroup;
   const uint32_t c_end = (NPAD >= 32 || half == 0) ? c_begin + kColsPerGroup : c_begin;
-  const bool split_mode = p.max_seg > combine_per_round<NPAD>();
   const float* part0 = p.partials + (size_t)row_tile * p.max_seg * NPAD * kBlockRows + nl;
-  for (uint32_t c0 = c_begin; c0 < c_end; c0 += 16) {
-    float even[16], odd[16];
+  for (uint32_t c0 = c_begin; c0 < c_end; c0 += kC) {
+    float acc[kC];
 #pragma unroll
-    for (uint32_t j = 0; j < 16; ++j) { even[j] = 0.f; odd[j] = 0.f; }
-    for (uint32_t s0 = 0; s0 < n_seg; s0 += 2) {
-      // segments s0 and s0 + 1: from memory, or (this threadblock's own) from tensor memory
-      float a[16], b[16];
-      const bool load_a = s0 != my_seg, has_b = s0 + 1 < n_seg, load_b = has_b && s0 + 1 != my_seg;
-      const float* pa = part0 + ((size_t)s0 * NPAD + c0) * kBlockRows;
-      const float* pb = pa + (size_t)NPAD * kBlockRows;
-      if (load_a) {
+    for (uint32_t j = 0; j < kC; ++j) acc[j] = 0.f;
+    for (uint32_t seg = 0; seg < n_seg; ++seg) {
+      // from memory, or (this threadblock's own) from tensor memory
+      float v[kC];
+      if (seg != my_seg) {
+        const float* ps = part0 + ((size_t)seg * NPAD + c0) * kBlockRows;
 #pragma unroll
-        for (uint32_t j = 0; j < 16; ++j) a[j] = __ldcg(pa + j * kBlockRows);
+        for (uint32_t j = 0; j < kC; ++j) v[j] = __ldcg(ps + j * kBlockRows);
+      } else {
+        tmem_ld<kC>(taddr + c0, v);
       }
-      if (load_b) {
 #pragma unroll
-        for (uint32_t j = 0; j < 16; ++j) b[j] = __ldcg(pb + j * kBlockRows);
-      }
-      if (!load_a) tmem_ld16(taddr + c0, a);
-      else if (has_b && !load_b) tmem_ld16(taddr + c0, b);
-#pragma unroll
-      for (uint32_t j = 0; j < 16; ++j) even[j] += a[j];
-      if (has_b) {
-#pragma unroll
-        for (uint32_t j = 0; j < 16; ++j) {
-          if (split_mode) odd[j] += b[j];
-          else even[j] += b[j];
-        }
-      }
+      for (uint32_t j = 0; j < kC; ++j) acc[j] += v[j];
     }
+    if (p.ssq_in) {
 #pragma unroll
-    for (uint32_t j = 0; j < 16; ++j) {
-      if (split_mode) even[j] += odd[j];
-      if (p.ssq_in) even[j] *= s_rs[c0 + j];
+      for (uint32_t j = 0; j < kC; ++j) acc[j] *= s_rs[c0 + j];
     }
     if (p.epi == kEpiSwiglu) {
       // rows 64 .. 127 of the tile are the up rows of the gate rows 0 .. 63
-      float* ex = s_exch + half * (16u * 64u);
+      float* ex = s_exch + half * (kC * 64u);
       if (quarter >= 2) {
 #pragma unroll
-        for (uint32_t j = 0; j < 16; ++j) ex[j * 64u + (nl - 64u)] = even[j];
+        for (uint32_t j = 0; j < kC; ++j) ex[j * 64u + (nl - 64u)] = acc[j];
       }
       named_barrier_sync(3 + half, kTcEpiThreads / 2);
       if (quarter < 2) {
         __nv_bfloat16* out = static_cast<__nv_bfloat16*>(p.y) + (size_t)row_tile * 64u + nl;
 #pragma unroll
-        for (uint32_t j = 0; j < 16; ++j) {
+        for (uint32_t j = 0; j < kC; ++j) {
           const uint32_t m = c0 + j;
           if (m < p.M_b) {
-            const float g = round_bf16(even[j]), u = round_bf16(ex[j * 64u + nl]);
+            const float g = round_bf16(acc[j]), u = round_bf16(ex[j * 64u + nl]);
             out[(size_t)m * (p.N / 2)] = __float2bfloat16_rn(g / (1.f + expf(-g)) * u);
           }
         }
       }
-      named_barrier_sync(3 + half, kTcEpiThreads / 2);   // (the next chunk overwrites the exchange buffer)
+      named_barrier_sync(3 + half, kTcEpiThreads / 2);   // (the next pass overwrites the exchange buffer)
     } else {
       const uint32_t n = row_tile * kBlockRows + nl;
 #pragma unroll
-      for (uint32_t j = 0; j < 16; ++j) {
+      for (uint32_t j = 0; j < kC; ++j) {
         const uint32_t m = c0 + j;
-        if (m < p.M_b && n < p.N) store_out(p, m, n, even[j]);
+        if (m < p.M_b && n < p.N) store_out(p, m, n, acc[j]);
       }
     }
   }
 }
-
 
 template <uint32_t NPAD>
 __global__ void __launch_bounds__(kTcThreads, 1) gemv_tc_kernel(const __grid_constant__ TcChainParams tp) {
@@ -1274,7 +1263,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) gemv_tc_kernel(const __grid_con
   uint32_t* tile_cnt = cp.ph[0].ws + kWsHeaderWords;
   __shared__ uint32_t s_last[2];
   __shared__ float s_rs[NPAD];           // row scales of phase s_rs_phase (tc_finish_tile)
-  __shared__ float s_exch[2 * 16 * 64];
+  __shared__ float s_exch[2 * tc_finish_cols<NPAD>() * 64];
   uint32_t buf = 0, buf_phase = 0;
   pdl_wait();
   for (;;) {
@@ -1322,7 +1311,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) gemv_tc_kernel(const __grid_con
       // the last partial sum of a tile keeps it in tensor memory and finishes the tile from
       // there (tc_finish_tile); the others write theirs out.  A tile's counter holds the
       // arrivals in its low half and the partial sums in memory in its high half.
-      const bool native = !p.end_combine && (p.epi == kEpiSwiglu || (p.epi == kEpiPlain && !p.ssq_out));
+      const bool native = !p.end_combine && p.max_seg <= combine_per_round<NPAD>() &&
+                          (p.epi == kEpiSwiglu || (p.epi == kEpiPlain && !p.ssq_out));
       if (native && n_seg > 1) {
         if (tid < n_tiles) s_last[tid] = ((atomicAdd(tile_cnt + mt.x + tid, 1u) & 0xFFFFu) == n_seg - 1) ? 1u : 0u;
         named_barrier_sync(1, kTcEpiThreads);
