@@ -30,7 +30,8 @@
  *     caller's, read by the kernels and 0 in normal use: word 4 replaces the limit of every
  *     bounded wait (GPU clock cycles; the default is about a second), word 5 - honoured only
  *     with a non-zero word 4 - makes that many threadblocks withhold their arrival at the end
- *     of a product of a chain (a test hook: it makes the others' waits run out), words 6 - 7
+ *     of a product of a chain, and their announcement that a row tile's partial sum is in
+ *     memory (a test hook: it makes the others' waits run out), words 6 - 7
  *     hold the device address of a schedule log (see boost_schedule_stats).  The other
  *     header words belong to the kernels;
  *   - every wait inside a kernel is bounded: none can hang the GPU;

@@ -1334,7 +1334,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) gemv_tc_kernel(const __grid_con
       if (native) {
         if (stored) {
           named_barrier_sync(1, kTcEpiThreads);   // everybody's stores come before the release
-          if (tid < n_tiles && !s_last[tid]) red_add_release(tile_cnt + mt.x + tid, 0x10000u);
+          if (tid < n_tiles && !s_last[tid] && blockIdx.x >= skip_arrivals_of(cp.ph[0].ws)) red_add_release(tile_cnt + mt.x + tid, 0x10000u);
         }
         bool gave_up = false;
         for (uint32_t ti = 0; ti < n_tiles; ++ti) {

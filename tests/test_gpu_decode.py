@@ -339,6 +339,49 @@ def test_fused_product_epilogues_match_oracle(dev):
     pool.close()
 
 
+@pytest.mark.parametrize("m_b", [48, 128, 200])
+def test_tile_finish_from_tensor_memory(dev, m_b):
+    """tcgen05 kernel, tile-by-tile mode: products wide enough that every threadblock holds several
+    row tiles (so their partial sums are not combined at the end of the phase), cut so that most
+    tiles have two or three partial sums.  The threadblock that delivers a tile's last one keeps
+    its accumulator in tensor memory and finishes the tile from there: SwiGLU with row scales
+    (gate / up partners exchanged through shared memory) and a plain product with a residual,
+    every output against the oracle."""
+    from paper_2609_13592_b200.tiers import TieredWeight
+    hid, ffn, n_plain = 192, 39040, 77952          # 3 k-blocks; 610 and 609 row tiles on 148 threadblocks
+    x_bits = synth.normal_bf16((m_b, hid), 1.0, 31)
+    gamma = synth.f32_to_bf16_bits(1.0 + 0.1 * np.random.default_rng(32).standard_normal(hid).astype(np.float32))
+    x = bf16_tensor(x_bits, dev)
+    x64 = ol.bf16_bits_to_f64(x_bits)
+    rs = od.rms_scale(x64)
+    stride = 256
+    ssq = torch.zeros(2, stride, dtype=torch.float32, device=dev)       # row statistics of x, two tiles of columns
+    ssq[0, :m_b] = torch.from_numpy((x64[:, :128] ** 2).sum(-1).astype(np.float32)).to(dev)
+    ssq[1, :m_b] = torch.from_numpy((x64[:, 128:] ** 2).sum(-1).astype(np.float32)).to(dev)
+    e = B.GemvEpilogue()
+    e.mode, e.ssq_in, e.ssq_in_tiles, e.ssq_stride, e.rms_eps = B.EPI_SWIGLU, ssq.data_ptr(), 2, stride, od.RMS_EPS
+    wgu_bits = synth.normal_bf16((2 * ffn, hid), 0.05, 33)
+    wgu = TieredWeight(bf16_tensor(wgu_bits, dev), device=dev, row_mode=1, col_scale=bf16_tensor(gamma, dev))
+    act = wgu.gemv(x, y_dtype=torch.bfloat16, epilogue=e)
+    torch.cuda.synchronize()
+    assert wgu.status_words() == [0]
+    gu = ol.bf16_bits_to_f64(ol.f64_to_bf16_bits(rs * (x64 @ ol.bf16_bits_to_f64(od.fold_norm_weight(wgu_bits, gamma)).T)))
+    assert_chain_close(act.float().cpu().numpy(), od.silu(gu[:, :ffn]) * gu[:, ffn:], f"swiglu finished from tensor memory, M_b={m_b}")
+    # plain, fp32 output with a residual, ragged last row tile (77952 = 609 x 128)
+    w_bits = synth.normal_bf16((n_plain - 40, hid), 0.05, 34)
+    res_bits = synth.normal_bf16((m_b, n_plain - 40), 1.0, 35)
+    w = TieredWeight(bf16_tensor(w_bits, dev), device=dev)
+    y = w.gemv(x, y_dtype=torch.float32, residual=bf16_tensor(res_bits, dev))
+    torch.cuda.synchronize()
+    assert w.status_words() == [0]
+    ref = x64 @ ol.bf16_bits_to_f64(w_bits).T + ol.bf16_bits_to_f64(res_bits)
+    assert_close_to_oracle(y.cpu().numpy(), ref, f"plain product finished from tensor memory, M_b={m_b}")
+    # the same launch again: the tile counters were left at zero, the result is the same bits
+    y2 = w.gemv(x, y_dtype=torch.float32, residual=bf16_tensor(res_bits, dev))
+    torch.cuda.synchronize()
+    assert torch.equal(y, y2)
+
+
 def test_full_size_step_matches_oracle_on_samples(dev):
     """One layer + LM head at the bench's shapes (hidden 4096, FFN 14336, 32 / 8 heads, vocab
     128256, batch 32, context about 2048, weight host share 1/131, block tables 133 wide): the

@@ -86,3 +86,36 @@ def test_missing_arrival_times_out_and_kernel_returns(dev, m_b):
     again_h, again_act = run(ws_ptr, ws_bytes)
     assert int(header[0]) == 0
     assert torch.equal(again_h, good_h) and torch.equal(again_act, good_act)
+
+
+def test_missing_partial_sum_times_out_in_tile_finish(dev):
+    """tcgen05 kernel, tile-by-tile mode: the threadblock that holds a row tile's last partial sum
+    waits until the others' are in memory before it finishes the tile from tensor memory.  Every
+    threadblock here keeps that announcement to itself, the waits give up after the shortened limit,
+    the kernel returns with the time-out on record, and after a zero-fill the next launch is bit
+    for bit what it was."""
+    from paper_2609_13592_b200.tiers import TieredWeight, aligned_workspace
+    m_b, hid, n = 96, 192, 77824                    # 608 row tiles on 148 threadblocks: most tiles in two or three pieces
+    x = bf16_tensor(synth.normal_bf16((m_b, hid), 1.0, 1), dev)
+    w = TieredWeight(bf16_tensor(synth.normal_bf16((n, hid), 0.05, 2), dev), device=dev)
+    ws_bytes = B.boost_gemv_workspace_bytes(n, hid, m_b)
+    ws_t, ws_ptr = aligned_workspace(ws_bytes, dev)
+    off = ws_ptr - ws_t.data_ptr()
+    header = ws_t[off:off + 64].view(torch.int32)
+
+    def run():
+        y = w.gemv(x, y_dtype=torch.float32, workspace=(ws_ptr, ws_bytes))
+        torch.cuda.synchronize()
+        return y
+
+    good = run()
+    assert int(header[0]) == 0 and float(good.abs().sum()) > 0
+    header[WS_WAIT_LIMIT_WORD] = 2_000_000
+    header[WS_SKIP_ARRIVALS_WORD] = 1 << 20         # every threadblock
+    torch.cuda.synchronize()
+    run()
+    assert int(header[0]) & 1 == 1
+    ws_t.zero_()
+    torch.cuda.synchronize()
+    again = run()
+    assert int(header[0]) == 0 and torch.equal(again, good)
