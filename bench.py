@@ -39,6 +39,10 @@ FALLBACK_HBM_GBS = 6650.0
 # gemv_tiered_kernel_chain_llama8b_m32.md): 1955.5 MB moved for 1872.8 MB of packed weights.
 GEMV_TRAFFIC_PER_ALGORITHMIC_BYTE = 1.044
 GEMV_TRAFFIC_PROFILE = "profiles/gemv_tiered_kernel_chain_llama8b_m32.md"
+# the tcgen05 kernel (batches above 32), same kind of capture at batch 128: (511.0 + 1609.5) MB moved for
+# (436.2 + 1436.6) MB of packed weights
+GEMV_TC_TRAFFIC_PER_ALGORITHMIC_BYTE = 1.132
+GEMV_TC_TRAFFIC_PROFILE = "profiles/gemv_tc_kernel_llama8b_m128.md"
 
 
 def load_peaks():
@@ -527,11 +531,14 @@ def run_ours(args, rank, world, local_rank):
             "host_weight_pages": t["host_pages"],
             "hbm_only": {"ms_per_step": hb_ms, "value": world * batch / (hb_ms / 1e3),
                          "tiered_over_hbm_only_time": ms_step / hb_ms},
-            "roofline": {"bound": "hbm", "kernel": "gemv_tiered_kernel (weight products, M_b = 32)",
+            "tiered_over_hbm_only_time": ms_step / hb_ms,
+            "roofline": {"bound": "hbm", "kernel": (f"gemv_tiered_kernel (weight products, M_b = {batch})" if batch <= 32 else
+                                                    f"gemv_tc_kernel (weight products on tcgen05, M_b = {batch})"),
                          "achieved": gemv_gbs, "peak": hbm_peak, "unit": "GB/s", "frac": gemv_gbs / hbm_peak,
                          "algorithmic_bytes_per_launch": gemv_bytes_per_launch,
-                         "traffic": GEMV_TRAFFIC_PER_ALGORITHMIC_BYTE * gemv_bytes_per_launch,
-                         "traffic_source": "ncu dram bytes of this workload's launches, ratio 1.044 to algorithmic",
+                         "traffic": (GEMV_TRAFFIC_PER_ALGORITHMIC_BYTE if batch <= 32 else GEMV_TC_TRAFFIC_PER_ALGORITHMIC_BYTE) * gemv_bytes_per_launch,
+                         "traffic_source": ("ncu dram bytes of this workload's launches, ratio 1.044 to algorithmic" if batch <= 32 else
+                                            "ncu dram bytes of the same chains at batch 128, ratio 1.132 to algorithmic"),
                          "launches_per_step": gemv_n, "avg_launch_us": 1e3 * gemv_ms / max(gemv_n, 1),
                          "peak_source": peak_src,
                          # events around every launch serialise the step: no launch overlaps its neighbours
@@ -539,7 +546,7 @@ def run_ours(args, rank, world, local_rank):
                          # the same bytes over the weight products' share of the overlapped step
                          # (step time minus the serialised time of the other kinds): an upper estimate
                          "achieved_in_step": gemv_step_bytes / (max(ms_step - t["kind_ms"][1] - t["kind_ms"][2], 1e-6) / 1e3) / 1e9,
-                         "traffic_profile": GEMV_TRAFFIC_PROFILE},
+                         "traffic_profile": GEMV_TRAFFIC_PROFILE if batch <= 32 else GEMV_TC_TRAFFIC_PROFILE},
             "roofline_attention": {"bound": "hbm", "kernel": "paged_attn_kernel", "achieved": attn_gbs,
                                    "peak": hbm_peak, "unit": "GB/s", "frac": attn_gbs / hbm_peak,
                                    "launches_per_step": attn_n, "avg_launch_us": 1e3 * attn_ms / max(attn_n, 1)},
