@@ -38,11 +38,11 @@ FALLBACK_HBM_GBS = 6650.0
 # capture of two full-size chain launches of this workload (profiles/
 # gemv_tiered_kernel_chain_llama8b_m32.md): 1955.5 MB moved for 1872.8 MB of packed weights.
 GEMV_TRAFFIC_PER_ALGORITHMIC_BYTE = 1.044
-GEMV_TRAFFIC_PROFILE = "profiles/gemv_tiered_kernel_chain_llama8b_m32.md"
+GEMV_TRAFFIC_PROFILE = "profiles/gemv_tiered_kernel_chain_llama8b_m32.md (captured at commit 7ba48f1; the kernel on this path is unchanged since)"
 # the tcgen05 kernel (batches above 32), same kind of capture at batch 128: (511.0 + 1609.5) MB moved for
 # (436.2 + 1436.6) MB of packed weights
 GEMV_TC_TRAFFIC_PER_ALGORITHMIC_BYTE = 1.132
-GEMV_TC_TRAFFIC_PROFILE = "profiles/gemv_tc_kernel_llama8b_m128.md"
+GEMV_TC_TRAFFIC_PROFILE = "profiles/gemv_tc_kernel_llama8b_m128.md (captured at commit d1a76e6)"
 
 
 def load_peaks():
