@@ -904,22 +904,25 @@ __global__ void __launch_bounds__(kConsumerThreads) gemv_combine_kernel(const __
 // K-major, 128-byte swizzle); the activations of the block's 64 columns are staged as the B
 // operand (NPAD rows, same layout); one thread issues four tcgen05.mma (K = 16 each) per block
 // and the 128 x NPAD fp32 accumulator lives in tensor memory, double-buffered so that the
-// next segment accumulates while four epilogue warps read the finished one back
+// next segment accumulates while the epilogue warps read the finished one back
 // (tcgen05.ld), write the partial sums and run the same combine as the kernel above.
-// Warps: 0-7 epilogue (warp w reads TMEM lanes 32 (w % 4) .. + 31 = weight rows, and the half
-// w / 4 of the accumulator's columns), 8 MMA issue and TMEM allocation, 9 weight producer
-// (bulk copies; 16-byte copies of all its lanes for host-tier blocks), 10 activation producer
-// (one thread: a tiled TMA copy per stage lands x[:, 64 kb .. + 64) in the B operand's swizzled
-// layout, rows beyond the batch as zeros).  Eleven warps, three to an SM sub-partition at most,
-// leave each thread 168 registers: the epilogue's sums in flight.  One threadblock per SM (the
-// driver keeps kernels that allocate tensor memory at one per SM at this shared-memory size)
+// Warps: 0-11 epilogue (warp w reads TMEM lanes 32 (w % 4) .. + 31 = weight rows, and the third
+// w / 4 of the accumulator's 16-column chunks), 12 MMA issue and TMEM allocation, 13 weight
+// producer (bulk copies; 16-byte copies of all its lanes for host-tier blocks), 14 activation
+// producer (one thread: a tiled TMA copy per stage lands x[:, 64 kb .. + 64) in the B operand's
+// swizzled layout, rows beyond the batch as zeros).  Twelve epilogue warps because the combine of
+// the partial sums is bound by what the warps of an SM can pull from L2 (eight: 163 us per chain
+// of four products at batch 128, twelve: 154, sixteen - 96 registers per thread - 155).  Fifteen
+// warps, four to an SM sub-partition at most: 128 registers per thread.  One threadblock per SM
+// (the driver keeps kernels that allocate tensor memory at one per SM at this shared-memory size)
 // with nearly all shared memory as its ring: no warp reads an operand back, so the ring's
 // bandwidth is all HBM's.
-constexpr uint32_t kTcEpiWarps = 8;
+constexpr uint32_t kTcEpiWarps = 12;
+constexpr uint32_t kTcGroups = kTcEpiWarps / 4;   // warps w, w + 4, w + 8 share TMEM lanes 32 (w % 4) .. + 31 and split the columns
 constexpr uint32_t kTcEpiThreads = kTcEpiWarps * 32;
 constexpr uint32_t kTcThreads = kTcEpiThreads + 96;   // + MMA warp, weight producer, activation producer
 // ring memory: what the epilogue's static arrays (row scales, the gate / up exchange buffer) leave
-constexpr uint32_t kTcSmemBudget = kSmemBudget - 18u * 1024u;
+constexpr uint32_t kTcSmemBudget = kSmemBudget - 14u * 1024u;
 
 // a stage: two weight blocks (the same 64 columns of two adjacent row tiles) and one activation tile
 // (at 256 batch rows the activation tile alone is 32 KiB and tensor memory holds two accumulators
@@ -935,21 +938,21 @@ __host__ __device__ constexpr uint32_t tc_stage_bytes(uint32_t npad) { return tc
 // need nothing across weight rows but the gate / up partner 64 rows on, which changes hands
 // through shared memory: SwiGLU, and plain without sums of squares of the output.
 // s_rs: row scales of the phase (filled by the caller when the product has row statistics);
-// s_exch: 2 x tc_finish_cols x 64 floats.  Called by all epilogue warps.
+// s_exch: kTcGroups x tc_finish_cols x 64 floats.  Called by all epilogue warps.
 // columns (batch rows) per pass of tc_finish_tile
 template <uint32_t NPAD>
-__host__ __device__ constexpr uint32_t tc_finish_cols() { return NPAD >= 64 ? 32u : 16u; }
+__host__ __device__ constexpr uint32_t tc_finish_cols() { return 16u; }
 
 template <uint32_t NPAD>
 __device__ __forceinline__ void tc_finish_tile(const GemvParams& p, uint32_t row_tile, uint32_t my_seg, uint32_t n_seg,
                                                uint32_t taddr, uint32_t warp, uint32_t lane, const float* s_rs,
                                                float* s_exch) {
   constexpr uint32_t kC = tc_finish_cols<NPAD>();
-  const uint32_t quarter = warp & 3u, half = warp >> 2;
+  const uint32_t quarter = warp & 3u, group = warp >> 2;
   const uint32_t nl = quarter * 32u + lane;
-  constexpr uint32_t kColsPerGroup = NPAD >= 32 ? NPAD / 2 : NPAD;
-  const uint32_t c_begin = half * kColsPerGroup;
-  const uint32_t c_end = (NPAD >= 32 || half == 0) ? c_begin + kColsPerGroup : c_begin;
+  // the column chunks of the accumulator, shared out between the groups of four warps
+  constexpr uint32_t kChunks = NPAD / kC;
+  const uint32_t c_begin = kChunks * group / kTcGroups * kC, c_end = kChunks * (group + 1) / kTcGroups * kC;
   const float* part0 = p.partials + (size_t)row_tile * p.max_seg * NPAD * kBlockRows + nl;
   for (uint32_t c0 = c_begin; c0 < c_end; c0 += kC) {
     float acc[kC];
@@ -974,12 +977,12 @@ __device__ __forceinline__ void tc_finish_tile(const GemvParams& p, uint32_t row
     }
     if (p.epi == kEpiSwiglu) {
       // rows 64 .. 127 of the tile are the up rows of the gate rows 0 .. 63
-      float* ex = s_exch + half * (kC * 64u);
+      float* ex = s_exch + group * (kC * 64u);
       if (quarter >= 2) {
 #pragma unroll
         for (uint32_t j = 0; j < kC; ++j) ex[j * 64u + (nl - 64u)] = acc[j];
       }
-      named_barrier_sync(3 + half, kTcEpiThreads / 2);
+      named_barrier_sync(3 + group, 128);
       if (quarter < 2) {
         __nv_bfloat16* out = static_cast<__nv_bfloat16*>(p.y) + (size_t)row_tile * 64u + nl;
 #pragma unroll
@@ -991,7 +994,7 @@ __device__ __forceinline__ void tc_finish_tile(const GemvParams& p, uint32_t row
           }
         }
       }
-      named_barrier_sync(3 + half, kTcEpiThreads / 2);   // (the next pass overwrites the exchange buffer)
+      named_barrier_sync(3 + group, 128);   // (the next pass overwrites the exchange buffer)
     } else {
       const uint32_t n = row_tile * kBlockRows + nl;
 #pragma unroll
@@ -1263,7 +1266,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) gemv_tc_kernel(const __grid_con
   uint32_t* tile_cnt = cp.ph[0].ws + kWsHeaderWords;
   __shared__ uint32_t s_last[2];
   __shared__ float s_rs[NPAD];           // row scales of phase s_rs_phase (tc_finish_tile)
-  __shared__ float s_exch[2 * tc_finish_cols<NPAD>() * 64];
+  __shared__ float s_exch[kTcGroups * tc_finish_cols<NPAD>() * 64];
   uint32_t buf = 0, buf_phase = 0;
   pdl_wait();
   for (;;) {
@@ -1301,12 +1304,11 @@ __global__ void __launch_bounds__(kTcThreads, 1) gemv_tc_kernel(const __grid_con
       const uint32_t split = mt.y;
       const uint32_t n_tiles = (mt.z & kFlagSecond) ? 2u : 1u;   // row tiles in this accumulator
       const uint32_t n_seg = p.even_part ? even_part_segments(p, mt.x) : p.splits;   // (the same for both tiles of a pair)
-      const uint32_t quarter = warp & 3u, half = warp >> 2;
+      const uint32_t quarter = warp & 3u, group = warp >> 2;
       const uint32_t nl = quarter * 32 + lane;                                 // weight row of this thread = its TMEM lane
-      // warps 0-3 read the first half of the columns, warps 4-7 the second (16 columns: the first group reads all)
-      constexpr uint32_t kColsPerGroup = NPAD >= 32 ? NPAD / 2 : NPAD;
-      const uint32_t c_begin = half * kColsPerGroup;
-      const uint32_t c_end = (NPAD >= 32 || half == 0) ? c_begin + kColsPerGroup : c_begin;
+      // the accumulator's columns in chunks of 16, shared out between the groups of four warps
+      constexpr uint32_t kChunks = NPAD / 16;
+      const uint32_t c_begin = kChunks * group / kTcGroups * 16, c_end = kChunks * (group + 1) / kTcGroups * 16;
       // Tile by tile, with an epilogue that works in the accumulator's layout: whoever holds
       // the last partial sum of a tile keeps it in tensor memory and finishes the tile from
       // there (tc_finish_tile); the others write theirs out.  A tile's counter holds the
@@ -1357,9 +1359,10 @@ __global__ void __launch_bounds__(kTcThreads, 1) gemv_tc_kernel(const __grid_con
             named_barrier_sync(1, kTcEpiThreads);
             if (s_rs_phase != mt.w) {
               const uint32_t v = tid & 15u;
-              for (uint32_t m = tid >> 4; m < NPAD; m += kTcEpiThreads / 16) {
+              for (uint32_t m_base = 0; m_base < NPAD; m_base += kTcEpiThreads / 16) {   // (every warp the same number of passes: it shuffles)
+                const uint32_t m = m_base + (tid >> 4);
                 float ss = 0.f, ss0 = 0.f, ss1 = 0.f;
-                if (m < p.M_b) {
+                if (m < p.M_b && m < NPAD) {
                   if (v < p.ssq_in_tiles) ss0 = __ldcg(p.ssq_in + (size_t)v * p.ssq_stride + m);
                   if (v + 16 < p.ssq_in_tiles) ss1 = __ldcg(p.ssq_in + (size_t)(v + 16) * p.ssq_stride + m);
                   for (uint32_t t0 = v + 32; t0 < p.ssq_in_tiles; t0 += 16) ss += __ldcg(p.ssq_in + (size_t)t0 * p.ssq_stride + m);
@@ -1369,7 +1372,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) gemv_tc_kernel(const __grid_con
                 ss += __shfl_xor_sync(0xFFFFFFFFu, ss, 2);
                 ss += __shfl_xor_sync(0xFFFFFFFFu, ss, 4);
                 ss += __shfl_xor_sync(0xFFFFFFFFu, ss, 8);
-                if (v == 0) s_rs[m] = rsqrtf(ss / (float)p.x_cols + p.rms_eps);
+                if (v == 0 && m < NPAD) s_rs[m] = rsqrtf(ss / (float)p.x_cols + p.rms_eps);
               }
               named_barrier_sync(1, kTcEpiThreads);
               if (tid == 0) s_rs_phase = mt.w;
