@@ -40,7 +40,7 @@
  *     GPUs; handles (boost_kv_pool_t) are not thread safe;
  *   - limits: head dimension 128; at most 16 query heads per KV head; the KV range of a
  *     tensor must be placed linearly (host pages at its tail, as the pool places it);
- *     weight products take 1 - 256 batch rows, the whole decode step 1 - 128 sequences.
+ *     weight products and the whole decode step take 1 - 256 batch rows (sequences).
  */
 #ifndef BOOST_H_
 #define BOOST_H_

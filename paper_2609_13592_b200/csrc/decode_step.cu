@@ -94,7 +94,7 @@ int run_step(Launcher& L, const boost_llama_model_t* m, const boost_llama_scratc
              const int32_t* block_table, uint32_t max_blocks, const int32_t* ctx_lens, uint32_t B,
              int32_t* next_tokens, const boost_kv_prefetch_t* pf = nullptr, boost_prefetch_ctx* pc = nullptr) {
   if (!m || !s || !tokens || !block_table || !ctx_lens || !next_tokens) return BOOST_ERR_INVALID;
-  if (B == 0 || B > 128 || !m->layers || m->n_layers == 0) return BOOST_ERR_INVALID;
+  if (B == 0 || B > 256 || !m->layers || m->n_layers == 0) return BOOST_ERR_INVALID;
   if (!s->h || !s->q_rot || !s->attn || !s->act || !s->logits || !s->ssq_a || !s->ssq_b || !s->rope_table || !s->gemv_ws ||
       !s->attn_ws || s->ssq_stride < B)
     return BOOST_ERR_INVALID;
@@ -229,7 +229,7 @@ int run_step(Launcher& L, const boost_llama_model_t* m, const boost_llama_scratc
 }  // namespace
 
 extern "C" size_t boost_llama_gemv_workspace_bytes(const boost_llama_model_t* m, uint32_t B) {
-  if (!m || !m->layers || B == 0 || B > 128) return 0;
+  if (!m || !m->layers || B == 0 || B > 256) return 0;
   size_t partial = boosth::gemv_partial_bytes(m->lm_head.N, m->lm_head.K, B);
   for (uint32_t li = 0; li < m->n_layers; ++li) {
     const boost_llama_layer_t& ly = m->layers[li];

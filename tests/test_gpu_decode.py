@@ -149,13 +149,13 @@ def dump_cache(dev, dec, li, name):
 
 @pytest.mark.parametrize("n_seq,kv_modulus,host_weights,recycle", [
     (3, 4, True, False), (1, 0, False, False), (20, 2, True, False), (40, 4, True, False), (6, 4, False, True),
-    (2, 4, True, True), (70, 2, True, False)])
+    (2, 4, True, True), (70, 2, True, False), (150, 2, False, False), (256, 4, True, False)])
 def test_decode_steps_match_oracle(dev, n_seq, kv_modulus, host_weights, recycle):
     """16 consecutive decode steps of the tiny model against the oracle.  host_weights: every weight
     matrix has its (only) page in host memory, so all products of the chain take the host-tier
     queue path; otherwise all weights are in HBM (even partition).  kv_modulus > 0 puts KV pages on
     the host as the pool places them.  Batch 1 - 2 is the CUDA-core kernel, 3 - 32 mma.sync, 40 and
-    70 the tcgen05 kernel."""
+    70 the tcgen05 kernel, 150 and 256 (the largest batch a step takes) its 256-column form."""
     from tests.helpers import chain_error
     cfg = dict(synth.TINY_LLAMA)
     w = synth.llama_weights(cfg, seed=n_seq, std=0.02)

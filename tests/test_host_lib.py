@@ -293,7 +293,7 @@ def test_chain_and_step_workspace_sizes_and_argument_checks():
     m.layers = C.cast(layers, C.POINTER(B.LlamaLayer))
     s32, s128 = B.boost_llama_gemv_workspace_bytes(m, 32), B.boost_llama_gemv_workspace_bytes(m, 128)
     assert s32 >= B.boost_gemv_workspace_bytes(128256, 4096, 32) and s128 > s32
-    assert B.boost_llama_gemv_workspace_bytes(m, 0) == 0 and B.boost_llama_gemv_workspace_bytes(m, 129) == 0
+    assert B.boost_llama_gemv_workspace_bytes(m, 0) == 0 and B.boost_llama_gemv_workspace_bytes(m, 257) == 0
     B.boost_gemv_set_tc_min_batch(33)
 
 
