@@ -179,6 +179,14 @@ int run_step(Launcher& L, const boost_llama_model_t* m, const boost_llama_scratc
     return rc;
   };
 
+  // The run length of the attention kernels' work items is a function of the context lengths:
+  // decided once, by a one-threadblock kernel, for all the layers' launches of this step.
+  L.run(kKindGlue, [&] {
+    const boost_llama_layer_t& l0 = m->layers[0];
+    return boosth::paged_attn_launch(s->q_rot, l0.k_page_ptr, l0.v_page_ptr, pf ? nullptr : m->kv_tier, (size_t)m->n_kv_pages,
+                                     m->n_pool_blocks, block_table, max_blocks, ctx_lens, B, hq, hkv, d, scale, s->attn_ws,
+                                     s->attn_ws_bytes, s->attn, stream, boosth::kAttnPlanOnly);
+  });
   L.run(kKindGlue, [&] { return boost_rope_table(ctx_lens, B, d, m->rope_base, s->rope_table, stream); });
   L.run(kKindGlue, [&] {
     return boost_embed_gather_ssq(m->embed, m->vocab, m->hidden, tokens, B, s->h, s->ssq_a, s->ssq_stride, stream);
@@ -191,11 +199,12 @@ int run_step(Launcher& L, const boost_llama_model_t* m, const boost_llama_scratc
     const boost_llama_layer_t& ly = m->layers[li];
     L.run(kKindAttn, [&] {
       // prefetch variant: every page is read from HBM (host pages from their staged copy)
-      return boost_paged_attn_decode_tiered(s->q_rot, pf ? pf->layers[li].k_page_ptr_staged : ly.k_page_ptr,
-                                            pf ? pf->layers[li].v_page_ptr_staged : ly.v_page_ptr,
-                                            pf ? nullptr : m->kv_tier, (size_t)m->n_kv_pages, m->n_pool_blocks,
-                                            block_table, max_blocks, ctx_lens, B, hq, hkv, d, scale, s->attn_ws,
-                                            s->attn_ws_bytes, s->attn, stream);
+      // (with the plan of the step's attention launches - see the top of the step)
+      return boosth::paged_attn_launch(s->q_rot, pf ? pf->layers[li].k_page_ptr_staged : ly.k_page_ptr,
+                                       pf ? pf->layers[li].v_page_ptr_staged : ly.v_page_ptr,
+                                       pf ? nullptr : m->kv_tier, (size_t)m->n_kv_pages, m->n_pool_blocks, block_table,
+                                       max_blocks, ctx_lens, B, hq, hkv, d, scale, s->attn_ws, s->attn_ws_bytes, s->attn,
+                                       stream, boosth::kAttnPlanReuse);
     });
     if (pf && L.ok()) {
       L.rc = boosth::check(cudaEventRecord(pc->attn_done[li], (cudaStream_t)stream));
@@ -310,10 +319,10 @@ extern "C" int boost_llama_decode_step_profile(const boost_llama_model_t* m, con
                                                int32_t* next_tokens, float* kind_ms_out,
                                                uint32_t* kind_launches_out, void* stream) {
   if (!kind_ms_out || !kind_launches_out || !m) return BOOST_ERR_INVALID;
-  if (4 + 2 * (uint64_t)m->n_layers > 512) return BOOST_ERR_UNSUPPORTED;
+  if (5 + 2 * (uint64_t)m->n_layers > 512) return BOOST_ERR_UNSUPPORTED;
   static thread_local Launcher L;
   L.stream = stream; L.timed = true; L.count = 0; L.extra = 0; L.rc = BOOST_OK;
-  const uint32_t n_events = 2 * (4 + 2 * m->n_layers);
+  const uint32_t n_events = 2 * (5 + 2 * m->n_layers);   // attention plan, rope table, embedding, first qkv, attention + chain per layer, argmax
   uint32_t made = 0;
   int rc = BOOST_OK;
   for (; made < n_events && rc == BOOST_OK; ++made) rc = boosth::check(cudaEventCreate(&L.ev[made]));

@@ -93,4 +93,11 @@ size_t gemv_partial_bytes(uint32_t N, uint32_t K, uint32_t M_b);
 // Launch check: picks up configuration errors of the launch just made.
 inline int check_launch() { return check(cudaGetLastError()); }
 
+// boost_paged_attn_decode_tiered with the choice of who plans the launch (see kernels_attn.cu).
+enum { kAttnPlanOwn = 0, kAttnPlanOnly = 1, kAttnPlanReuse = 2 };
+int paged_attn_launch(const void* q, const void* const* k_page_ptr, const void* const* v_page_ptr, const uint8_t* kv_tier,
+                      size_t n_kv_pages, uint32_t n_pool_blocks, const int32_t* block_table, uint32_t max_blocks,
+                      const int32_t* ctx_lens, uint32_t B, uint32_t Hq, uint32_t Hkv, uint32_t D, float scale, void* workspace,
+                      size_t workspace_bytes, void* out, void* stream, int plan);
+
 }  // namespace boosth

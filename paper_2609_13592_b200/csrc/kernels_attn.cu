@@ -43,6 +43,7 @@ constexpr uint32_t kWarpStages = 2;                      // ring depth of one wa
 constexpr uint32_t kMaxGroup = 16;
 constexpr uint32_t kParkStride = kD + 4;                 // floats per parked head: 128 outputs, m, l, padding
 constexpr uint32_t kMaxListedSeqs = 1024;                // batches up to this size get a dense item list
+constexpr uint32_t kWsPlan = 12;                         // workspace header word: the plan of attn_plan_kernel (0: none yet)
 constexpr uint32_t kTailPieces = 4;                      // the runs of the last KV head are cut in this many items
 
 
@@ -76,8 +77,97 @@ __device__ __forceinline__ uint32_t movmatrix_trans(uint32_t a) {
   return d;
 }
 
-// NH = number of 8-head tiles of a KV group (1: up to 8 query heads per KV head, 2: up to 16)
-template <int NH>
+// Run length for sequences about equally long, each cut into s runs: the slots take the items in
+// rounds; a full round streams at the HBM rate, the last one at the rate its items can draw (a
+// threadblock alone gets 1 / (55 % of the slots) of it), and every round costs a hand-over (table
+// look-up, query load, merge: about 5 us = 4000 block times).  In units of the time HBM takes for
+// one KV block: cost = run x (full rounds x slots + max(55 % of slots, items of the last round))
+// + 4000 x rounds.  Candidates: 1 .. 4 runs per sequence, and one run per slot over 4 / 7 of the
+// slots (runs of 1.75 times the blocks a slot gets on average: what long sequences in small
+// batches need).  Returns the blocks per warp of the cheapest.
+__device__ __forceinline__ uint32_t item_blocks_by_cost(uint32_t total_blocks, uint32_t longest, uint32_t B, uint32_t Hkv,
+                                                     uint32_t slots) {
+  const float sat = 0.55f * (float)slots, inv_slots = 1.f / (float)slots;
+  const uint32_t mean = (total_blocks + B - 1) / B;
+  const uint32_t per_slot = (total_blocks * Hkv * 7u + slots * 4u - 1u) / (slots * 4u);
+  float best = 3.0e38f;
+  uint32_t item_blocks = kMaxItemBlocks;
+#pragma unroll 1
+  for (uint32_t s = 0; s <= 4; ++s) {
+    const uint32_t run = s ? (longest + s - 1) / s : per_slot;
+    const uint32_t ib = min(kMaxItemBlocks, max(kMinItemBlocks, (run + kAttnWarps - 1) / kAttnWarps));
+    const uint32_t n_spl = mean ? (mean + kAttnWarps * ib - 1) / (kAttnWarps * ib) : 1u;
+    const float len = mean ? (float)((mean + n_spl - 1) / n_spl) : 0.f;
+    const float items = (float)(B * Hkv * n_spl);
+    const float full = floorf(items * inv_slots + 1e-4f), tail = items - full * (float)slots;
+    const float cost = len * (full * (float)slots + (tail > 0.5f ? fmaxf(sat, tail) : 0.f)) + 4000.f * (full + (tail > 0.5f ? 1.f : 0.f));
+    if (cost < best) { best = cost; item_blocks = ib; }
+  }
+  return item_blocks;
+}
+
+// The plan of a launch - blocks per warp and work item in the low half, bit 31: a mix of lengths -
+// from the sum and the maximum of the sequences' block counts.  An item costs a table look-up,
+// a query load and, when a sequence needs several items, a partial result in global memory,
+// so long runs are better; but the kernel ends with its longest item, and about 55 % of the
+// threadblocks the device holds saturate HBM (measured on B200: about a thousand warps with
+// 16 KiB in flight each).  With u KV blocks per threadblock slot on average: a mix of lengths
+// (longest above 1.25 times the mean) -> runs of at most u, a few items per slot to even out
+// through the queue; sequences about equally long -> runs of at most 1.75 u where one run per
+// sequence fills one round of the slots well (between 55 % of them and all), else what the cost
+// model picks.
+constexpr uint32_t kPlanMixed = 0x80000000u;
+__device__ __forceinline__ uint32_t attn_plan_word(uint64_t total_blocks, uint32_t longest, uint32_t B, uint32_t Hkv, uint32_t slots) {
+  const bool mixed = (uint64_t)longest * B * 4 > total_blocks * 5;
+  const uint64_t quarters = mixed ? 4 : 7;   // run cap in quarters of u
+  const uint64_t run_cap = (total_blocks * Hkv * quarters + (uint64_t)slots * 4 - 1) / ((uint64_t)slots * 4);
+  uint32_t item_blocks = (uint32_t)min((uint64_t)kMaxItemBlocks, max((uint64_t)kMinItemBlocks, (run_cap + kAttnWarps - 1) / kAttnWarps));
+  const uint32_t whole = B * Hkv;
+  if (!mixed && !(longest <= kAttnWarps * kMaxItemBlocks && whole <= slots && whole * 20u >= slots * 11u))
+    item_blocks = item_blocks_by_cost((uint32_t)total_blocks, longest, B, Hkv, slots);
+  return item_blocks | (mixed ? kPlanMixed : 0u);
+}
+
+// Sum and maximum of the sequences' block counts over a threadblock of kAttnThreads threads
+// (scratch: two arrays of kAttnWarps words).  Every thread gets the result.
+__device__ __forceinline__ void attn_block_counts(const AttnParams& p, uint32_t* s_sum, uint32_t* s_max, uint64_t& total_blocks,
+                                                  uint32_t& longest) {
+  const uint32_t tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  uint32_t my_blocks = 0, my_max = 0;
+  for (uint32_t b = tid; b < p.B; b += kAttnThreads) {
+    const uint32_t n = (seq_len(p, b) + kTok - 1) / kTok;
+    my_blocks += n;
+    my_max = max(my_max, n);
+  }
+#pragma unroll
+  for (int sh = 16; sh >= 1; sh >>= 1) {
+    my_blocks += __shfl_xor_sync(0xFFFFFFFFu, my_blocks, sh);
+    my_max = max(my_max, __shfl_xor_sync(0xFFFFFFFFu, my_max, sh));
+  }
+  if (lane == 0) { s_sum[warp] = my_blocks; s_max[warp] = my_max; }
+  __syncthreads();
+  total_blocks = 0;
+  longest = 0;
+#pragma unroll
+  for (uint32_t w = 0; w < kAttnWarps; ++w) { total_blocks += s_sum[w]; longest = max(longest, s_max[w]); }
+}
+
+// The plan as a kernel of its own (one threadblock): a decode step runs it once, ahead of its
+// attention launches, which then read the word instead of each deriving it (kOwnPlan = false).
+// It does not release its dependents early: whatever is launched behind it starts after it.
+__global__ void __launch_bounds__(kAttnThreads) attn_plan_kernel(const AttnParams p) {
+  __shared__ uint32_t s_sum[kAttnWarps], s_max[kAttnWarps];
+  pdl_wait();
+  uint64_t total_blocks;
+  uint32_t longest;
+  attn_block_counts(p, s_sum, s_max, total_blocks, longest);
+  if (threadIdx.x == 0) p.ws[kWsPlan] = attn_plan_word(total_blocks, longest, p.B, p.Hkv, p.cta_slots);
+}
+
+// NH = number of 8-head tiles of a KV group (1: up to 8 query heads per KV head, 2: up to 16);
+// kOwnPlan: the kernel derives its plan itself (every threadblock sums the context lengths), or
+// reads the word attn_plan_kernel left in the workspace.
+template <int NH, bool kOwnPlan>
 __global__ void __launch_bounds__(kAttnThreads, (NH == 1 ? 3 : 2)) paged_attn_kernel(const AttnParams p) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~uintptr_t(127));
@@ -108,68 +198,19 @@ __global__ void __launch_bounds__(kAttnThreads, (NH == 1 ? 3 : 2)) paged_attn_ke
   __shared__ uint32_t s_warp_sum[kAttnWarps], s_warp_max[kAttnWarps];
   __shared__ uint32_t s_first_item[kMaxListedSeqs + 1];   // first item of every sequence within a head
 
-  // ---- run length.  Every threadblock derives the same decomposition from the context
-  // lengths.  An item costs a table look-up, a query load and, when a sequence needs several
-  // items, a partial result in global memory, so long runs are better; but the kernel ends with
-  // its longest item, and about 55 % of the threadblocks the device holds saturate HBM
-  // (measured on B200: about a thousand warps with 16 KiB in flight each).  With u KV blocks
-  // per threadblock slot on average: when the sequences are about equally long, a run is at
-  // most 1.75 u blocks, so that share of the slots gets one item each and all end together;
-  // with a mix of lengths (longest above 1.25 times the mean) items differ in length anyway,
-  // and runs of at most u give every slot a few items to even out through the queue.
-  uint32_t my_blocks = 0, my_max = 0;
-  for (uint32_t b = tid; b < p.B; b += kAttnThreads) {
-    const uint32_t n = (seq_len(p, b) + kTok - 1) / kTok;
-    my_blocks += n;
-    my_max = max(my_max, n);
-  }
-#pragma unroll
-  for (int sh = 16; sh >= 1; sh >>= 1) {
-    my_blocks += __shfl_xor_sync(0xFFFFFFFFu, my_blocks, sh);
-    my_max = max(my_max, __shfl_xor_sync(0xFFFFFFFFu, my_max, sh));
-  }
-  if (lane == 0) { s_warp_sum[warp] = my_blocks; s_warp_max[warp] = my_max; }
-  __syncthreads();
-  uint64_t total_blocks = 0;
-  uint32_t longest = 0;
-#pragma unroll
-  for (uint32_t w = 0; w < kAttnWarps; ++w) { total_blocks += s_warp_sum[w]; longest = max(longest, s_warp_max[w]); }
-  const bool mixed = (uint64_t)longest * p.B * 4 > total_blocks * 5;
-  uint32_t item_blocks;
-  if (mixed) {
-    const uint64_t run_cap = (total_blocks * p.Hkv + (uint64_t)p.cta_slots - 1) / (uint64_t)p.cta_slots;   // u
-    item_blocks = (uint32_t)min((uint64_t)kMaxItemBlocks, max((uint64_t)kMinItemBlocks, (run_cap + kAttnWarps - 1) / kAttnWarps));
+  // ---- run length.  Every threadblock works with the same decomposition of the sequences into
+  // items (see attn_plan_word).
+  uint32_t plan;
+  if constexpr (kOwnPlan) {
+    uint64_t total_blocks;
+    uint32_t longest;
+    attn_block_counts(p, s_warp_sum, s_warp_max, total_blocks, longest);
+    plan = attn_plan_word(total_blocks, longest, p.B, p.Hkv, p.cta_slots);
   } else {
-    // Sequences about equally long, each cut into s runs: the slots take the items in rounds; a
-    // full round streams at the HBM rate, the last one at the rate its items can draw (a
-    // threadblock alone gets 1 / (55 % of the slots) of it), and every round costs a hand-over
-    // (table look-up, query load, merge: about 5 us = 4000 block times).  In units of the time
-    // HBM takes for one KV block: cost(s) = run x (full rounds x slots + max(55 % of slots,
-    // items of the last round)) + 4000 x rounds.  The s with the least cost wins.
-    // (single precision and 32-bit integers: every thread of every threadblock runs this)
-    const uint32_t slots = p.cta_slots;
-    const float sat = 0.55f * (float)slots, inv_slots = 1.f / (float)slots;
-    const uint32_t mean = ((uint32_t)total_blocks + p.B - 1) / p.B;
-    float best = 3.0e38f;
-    item_blocks = kMaxItemBlocks;
-    // candidates: 1 .. 4 runs per sequence, and one run per slot over 4 / 7 of the slots (runs of
-    // 1.75 times the blocks a slot gets on average: what long sequences in small batches need)
-    const uint32_t per_slot = ((uint32_t)total_blocks * p.Hkv * 7u + slots * 4u - 1u) / (slots * 4u);
-    // (one run per sequence that fills one round well needs no search)
-    const uint32_t whole = p.B * p.Hkv;
-    const bool one_round = longest <= kAttnWarps * kMaxItemBlocks && whole <= slots && (float)whole >= sat;
-    if (one_round) item_blocks = max(kMinItemBlocks, (longest + kAttnWarps - 1) / kAttnWarps);
-    for (uint32_t s = 0; s <= 4 && !one_round; ++s) {
-      const uint32_t run = s ? (longest + s - 1) / s : per_slot;
-      const uint32_t ib = min(kMaxItemBlocks, max(kMinItemBlocks, (run + kAttnWarps - 1) / kAttnWarps));
-      const uint32_t n_spl = mean ? (mean + kAttnWarps * ib - 1) / (kAttnWarps * ib) : 1u;
-      const float len = mean ? (float)((mean + n_spl - 1) / n_spl) : 0.f;
-      const float items = (float)(p.B * p.Hkv * n_spl);
-      const float full = floorf(items * inv_slots + 1e-4f), tail = items - full * (float)slots;
-      const float cost = len * (full * (float)slots + (tail > 0.5f ? fmaxf(sat, tail) : 0.f)) + 4000.f * (full + (tail > 0.5f ? 1.f : 0.f));
-      if (cost < best) { best = cost; item_blocks = ib; }
-    }
+    plan = __ldcg(p.ws + kWsPlan);
   }
+  const bool mixed = (plan & kPlanMixed) != 0;
+  const uint32_t item_blocks = min(kMaxItemBlocks, max(kMinItemBlocks, plan & 0xFFFFu));
   const uint32_t cta_max = kAttnWarps * item_blocks;
   const uint32_t max_splits = (p.max_blocks + cta_max - 1) / cta_max;
   // ---- item list.  Up to kMaxListedSeqs sequences: items are numbered densely, sequence by
@@ -627,13 +668,17 @@ extern "C" size_t boost_paged_attn_workspace_bytes(uint32_t B, uint32_t Hq, uint
   return attn_header_bytes(B, Hq) + (size_t)B * Hq * max_splits * (2 + kD) * 4;
 }
 
-extern "C" int boost_paged_attn_decode_tiered(const void* q, const void* const* k_page_ptr,
-                                              const void* const* v_page_ptr, const uint8_t* kv_tier,
-                                              size_t n_kv_pages, uint32_t n_pool_blocks,
-                                              const int32_t* block_table, uint32_t max_blocks,
-                                              const int32_t* ctx_lens, uint32_t B, uint32_t Hq,
-                                              uint32_t Hkv, uint32_t D, float scale, void* workspace,
-                                              size_t workspace_bytes, void* out, void* stream) {
+// plan: who decides the run length of the items.  kAttnPlanOwn: the attention kernel itself, every
+// threadblock from the context lengths (a call on its own); kAttnPlanOnly: no attention, only the
+// one-threadblock kernel that leaves the plan in the workspace (a decode step runs it first of
+// all, several launches ahead of the first attention kernel, which reads the word before its
+// dependency wait); kAttnPlanReuse: attention with the plan such a call left there for the same
+// batch and context lengths.
+int boosth::paged_attn_launch(const void* q, const void* const* k_page_ptr, const void* const* v_page_ptr,
+                              const uint8_t* kv_tier, size_t n_kv_pages, uint32_t n_pool_blocks,
+                              const int32_t* block_table, uint32_t max_blocks, const int32_t* ctx_lens, uint32_t B,
+                              uint32_t Hq, uint32_t Hkv, uint32_t D, float scale, void* workspace, size_t workspace_bytes,
+                              void* out, void* stream, int plan) {
   if (B == 0) return BOOST_OK;
   if (!q || !k_page_ptr || !v_page_ptr || !block_table || !ctx_lens || !workspace || !out)
     return BOOST_ERR_INVALID;
@@ -683,15 +728,35 @@ extern "C" int boost_paged_attn_decode_tiered(const void* q, const void* const* 
   if (slot < 0) return BOOST_ERR_CUDA;
   bool& configured = configured_on[slot];
   if (!configured) {
-    int rc = boosth::check(cudaFuncSetAttribute(paged_attn_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    int rc = boosth::check(cudaFuncSetAttribute(paged_attn_kernel<1, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     if (rc == BOOST_OK)
-      rc = boosth::check(cudaFuncSetAttribute(paged_attn_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+      rc = boosth::check(cudaFuncSetAttribute(paged_attn_kernel<2, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    if (rc == BOOST_OK)
+      rc = boosth::check(cudaFuncSetAttribute(paged_attn_kernel<1, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    if (rc == BOOST_OK)
+      rc = boosth::check(cudaFuncSetAttribute(paged_attn_kernel<2, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     if (rc != BOOST_OK) return rc;
     configured = true;
   }
   uint32_t grid = p.cta_slots;
   if (grid > max_items) grid = (uint32_t)max_items;
+  if (plan == boosth::kAttnPlanOnly)
+    return boosth::launch_chained(attn_plan_kernel, dim3(1), dim3(kAttnThreads), 0, (cudaStream_t)stream, p);
+  const bool own = plan == boosth::kAttnPlanOwn;
   if (p.group <= 8)
-    return boosth::launch_chained(paged_attn_kernel<1>, dim3(grid), dim3(kAttnThreads), smem, (cudaStream_t)stream, p);
-  return boosth::launch_chained(paged_attn_kernel<2>, dim3(grid), dim3(kAttnThreads), smem, (cudaStream_t)stream, p);
+    return own ? boosth::launch_chained(paged_attn_kernel<1, true>, dim3(grid), dim3(kAttnThreads), smem, (cudaStream_t)stream, p)
+               : boosth::launch_chained(paged_attn_kernel<1, false>, dim3(grid), dim3(kAttnThreads), smem, (cudaStream_t)stream, p);
+  return own ? boosth::launch_chained(paged_attn_kernel<2, true>, dim3(grid), dim3(kAttnThreads), smem, (cudaStream_t)stream, p)
+             : boosth::launch_chained(paged_attn_kernel<2, false>, dim3(grid), dim3(kAttnThreads), smem, (cudaStream_t)stream, p);
+}
+
+extern "C" int boost_paged_attn_decode_tiered(const void* q, const void* const* k_page_ptr,
+                                              const void* const* v_page_ptr, const uint8_t* kv_tier,
+                                              size_t n_kv_pages, uint32_t n_pool_blocks,
+                                              const int32_t* block_table, uint32_t max_blocks,
+                                              const int32_t* ctx_lens, uint32_t B, uint32_t Hq,
+                                              uint32_t Hkv, uint32_t D, float scale, void* workspace,
+                                              size_t workspace_bytes, void* out, void* stream) {
+  return boosth::paged_attn_launch(q, k_page_ptr, v_page_ptr, kv_tier, n_kv_pages, n_pool_blocks, block_table, max_blocks,
+                                   ctx_lens, B, Hq, Hkv, D, scale, workspace, workspace_bytes, out, stream, boosth::kAttnPlanOwn);
 }
