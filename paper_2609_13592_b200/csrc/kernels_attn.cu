@@ -43,6 +43,7 @@ constexpr uint32_t kWarpStages = 2;                      // ring depth of one wa
 constexpr uint32_t kMaxGroup = 16;
 constexpr uint32_t kParkStride = kD + 4;                 // floats per parked head: 128 outputs, m, l, padding
 constexpr uint32_t kMaxListedSeqs = 1024;                // batches up to this size get a dense item list
+constexpr uint32_t kMaxSmemPages = 256;                   // page tables up to this size are staged in shared memory
 constexpr uint32_t kWsPlan = 12;                         // workspace header word: the plan of attn_plan_kernel (0: none yet)
 constexpr uint32_t kTailPieces = 4;                      // the runs of the last KV head are cut in this many items
 
@@ -58,6 +59,7 @@ struct AttnParams {
   const int32_t* ctx_lens;
   uint32_t B, Hq, Hkv, group;
   uint32_t cta_slots;         // threadblocks the device holds at once (the balance target)
+  uint32_t smem_pages;        // > 0: the K and V page tables (this many entries each) are staged in shared memory
   float scale_log2e;
   uint32_t* ws;        // header (status, item counter, done counter) + one counter per (b, g)
   float* part_ml;      // [B][Hq][max_splits][2], max_splits from the run length chosen on the device
@@ -175,6 +177,13 @@ __global__ void __launch_bounds__(kAttnThreads, (NH == 1 ? 3 : 2)) paged_attn_ke
 
   const uint32_t tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   uint8_t* ring = smem + (size_t)warp * kWarpStages * kStageBytes;   // this warp's stages
+  // Small page tables are copied into shared memory once: a block's address is then one
+  // dependent global load (its table entry) away instead of two.
+  unsigned long long* s_pages = reinterpret_cast<unsigned long long*>(smem + (size_t)kAttnWarps * kWarpStages * kStageBytes);
+  for (uint32_t i = tid; i < p.smem_pages; i += kAttnThreads) {
+    s_pages[i] = reinterpret_cast<unsigned long long>(p.k_page_ptr[i]);
+    s_pages[p.smem_pages + i] = reinterpret_cast<unsigned long long>(p.v_page_ptr[i]);
+  }
   uint32_t* status = p.ws + kWsStatus;
   pdl_launch_dependents();
   if (lane == 0) {
@@ -217,6 +226,7 @@ __global__ void __launch_bounds__(kAttnThreads, (NH == 1 ? 3 : 2)) paged_attn_ke
   // sequence (s_first_item = running count of runs), so no threadblock draws an empty item.
   // Larger batches: every sequence has max_splits numbers and the unused ones are skipped.
   const bool listed = p.B <= kMaxListedSeqs;
+  if (!listed && p.smem_pages) __syncthreads();   // (the listed path below has barriers of its own)
   uint32_t per_head = p.B * max_splits;
   if (listed) {
     uint32_t carry = 0;
@@ -306,8 +316,11 @@ __global__ void __launch_bounds__(kAttnThreads, (NH == 1 ? 3 : 2)) paged_attn_ke
           const uint32_t lin = g * p.n_pool_blocks + (uint32_t)blk;
           const uint32_t page = lin / kChunksPerPage;
           const size_t in_page = (size_t)(lin % kChunksPerPage) * kChunkBytes;
-          ksrc[h] = static_cast<const uint8_t*>(p.k_page_ptr[page]) + in_page;
-          v_minus_k[h] = (size_t)(static_cast<const uint8_t*>(p.v_page_ptr[page]) + in_page - ksrc[h]);
+          const uint8_t* kpage = p.smem_pages ? reinterpret_cast<const uint8_t*>(s_pages[page]) : static_cast<const uint8_t*>(p.k_page_ptr[page]);
+          const uint8_t* vpage = p.smem_pages ? reinterpret_cast<const uint8_t*>(s_pages[p.smem_pages + page])
+                                              : static_cast<const uint8_t*>(p.v_page_ptr[page]);
+          ksrc[h] = kpage + in_page;
+          v_minus_k[h] = (size_t)(vpage + in_page - ksrc[h]);
           host_bits |= (page >= p.first_host_page ? 1u : 0u) << h;
         }
       }
@@ -722,19 +735,22 @@ int boosth::paged_attn_launch(const void* q, const void* const* k_page_ptr, cons
   // room for the shortest runs; the kernel indexes with the max_splits of the run length it picks
   p.part_o = p.part_ml + (size_t)B * Hq * partial_slots(max_blocks) * 2;
   p.out = static_cast<__nv_bfloat16*>(out);
-  const size_t smem = (size_t)kAttnWarps * kWarpStages * kStageBytes + 128;
+  // page tables of up to 256 entries ride in shared memory (three threadblocks per SM still fit)
+  p.smem_pages = n_kv_pages <= kMaxSmemPages ? (uint32_t)n_kv_pages : 0u;
+  const size_t smem_max = (size_t)kAttnWarps * kWarpStages * kStageBytes + 128 + (size_t)kMaxSmemPages * 16;
+  const size_t smem = (size_t)kAttnWarps * kWarpStages * kStageBytes + 128 + (size_t)p.smem_pages * 16;
   static bool configured_on[boosth::kMaxDevices] = {false};   // function attributes are per device
   const int slot = boosth::device_slot();
   if (slot < 0) return BOOST_ERR_CUDA;
   bool& configured = configured_on[slot];
   if (!configured) {
-    int rc = boosth::check(cudaFuncSetAttribute(paged_attn_kernel<1, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    int rc = boosth::check(cudaFuncSetAttribute(paged_attn_kernel<1, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_max));
     if (rc == BOOST_OK)
-      rc = boosth::check(cudaFuncSetAttribute(paged_attn_kernel<2, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+      rc = boosth::check(cudaFuncSetAttribute(paged_attn_kernel<2, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_max));
     if (rc == BOOST_OK)
-      rc = boosth::check(cudaFuncSetAttribute(paged_attn_kernel<1, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+      rc = boosth::check(cudaFuncSetAttribute(paged_attn_kernel<1, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_max));
     if (rc == BOOST_OK)
-      rc = boosth::check(cudaFuncSetAttribute(paged_attn_kernel<2, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+      rc = boosth::check(cudaFuncSetAttribute(paged_attn_kernel<2, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_max));
     if (rc != BOOST_OK) return rc;
     configured = true;
   }
