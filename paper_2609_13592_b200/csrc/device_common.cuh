@@ -104,6 +104,11 @@ __device__ __forceinline__ void tma_load_2d(void* dst_smem, const void* tensor_m
       : "memory");
 }
 
+// Brings a tensor map into the descriptor cache ahead of its first use.
+__device__ __forceinline__ void tma_prefetch_map(const void* tensor_map) {
+  asm volatile("prefetch.tensormap [%0];" ::"l"(tensor_map) : "memory");
+}
+
 // Orders this thread's earlier generic-proxy view of memory (what it has acquired from other
 // threads' ordinary stores) before its later copies through the asynchronous proxy (TMA).
 __device__ __forceinline__ void fence_proxy_async_all() { asm volatile("fence.proxy.async;" ::: "memory"); }

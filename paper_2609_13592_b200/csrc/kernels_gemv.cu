@@ -1060,6 +1060,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) gemv_tc_kernel(const __grid_con
   if (warp > kTcEpiWarps) {
     // ------------------------------------------------------------------ producer warps (as above)
     const bool leader = (warp == kTcEpiWarps + 1);
+    if (!leader && lane == 0)   // the phases' tensor maps: fetched now, not at each phase's first copy
+      for (uint32_t ph = 0; ph < n_phases; ++ph) tma_prefetch_map(&tp.x_map[ph]);
     uint32_t stage = 0, phase = 0, icount = 0;
     unsigned long long* const sched_log = (leader && lane == 0) ? sched_log_of(cp.ph[0].ws) : nullptr;
     uint32_t rec = kNoRecord;   // schedule-log record of the item in production (weight warp, lane 0)
