@@ -360,8 +360,10 @@ int boost_pack_weights_ex(const void* w_row_major /*device*/, uint32_t N, uint32
  *   workspace  device, >= boost_gemv_workspace_bytes(N, K, M_b).
  * M_b <= 2 runs on CUDA cores with warp-shuffle reductions; larger batches use the tensor
  * cores (mma.sync up to 32 rows, tcgen05 with accumulators in tensor memory above; see
- * boost_gemv_set_tc_min_batch).  A weight with host pages is cut into work items handed out
- * host pages first; a weight entirely in HBM is cut evenly over the threadblocks.  Split-K
+ * boost_gemv_set_tc_min_batch).  The blocks of a weight are cut evenly over the threadblocks;
+ * host pages are read in place, by the same bulk copies, by the threadblocks whose share holds
+ * them (boost_gemv_set_tier_schedule selects the two-queue schedule that hands host pages out
+ * first instead).  Split-K
  * partial sums meet in L2 and are combined in a fixed order - tile by tile in the threadblock
  * that delivers a tile's last partial sum, or, for a product cut so finely that a tile has four
  * or more, all tiles at the end of the product spread over the warps of the grid (see
@@ -435,6 +437,18 @@ int boost_gemv_set_tc_min_batch(uint32_t m_b);
  * for measurement and tests.  The paper has no counterpart (its products are library kernels,
  * Sec. 4.1). */
 int boost_gemv_set_end_combine(uint32_t on);
+
+/* How a weight with host pages is scheduled.  0 (the default): the even partition of a weight
+ * that is entirely in HBM, with every host-tier block read in place by the threadblock whose
+ * contiguous share holds it - both tiers stream for as long as such shares last, no queue, no
+ * specialised threadblocks.  1: the schedule of Sec. 3.2 and Sec. 3.1 - work items of one page
+ * each in two queues, host-tier items handed out first to a few threadblocks that stay on that
+ * tier while it has items (16-byte copies through the load/store path), the others on the HBM
+ * queue.  Measured on a B200 whose host link carries 0.8 % of the HBM bandwidth, the in-place
+ * form is as fast or faster for every Llama-3-8B matrix, batch size and host share tried, which
+ * is why it is the default.  Results differ between the two in fp32 rounding (other partial
+ * sums).  Process-wide; for measurement, tests and the comparison with the paper's schedule. */
+int boost_gemv_set_tier_schedule(uint32_t two_queues);
 
 /* boost_gemv_tiered with an epilogue descriptor (NULL = plain). */
 int boost_gemv_tiered_fused(const void* const* w_page_ptr /*device*/, const uint32_t* w_order /*device*/,

@@ -154,6 +154,7 @@ SIGNATURES = {
     "boost_schedule_log_bytes": (C.c_size_t, [C.c_size_t]),
     "boost_schedule_stats": (_int, [_vp, C.c_size_t, _u32, _u32, C.c_uint64, C.c_double, _vp, _vp, _vp]),
     "boost_gemv_set_tc_min_batch": (_int, [_u32]),
+    "boost_gemv_set_tier_schedule": (_int, [_u32]),
     "boost_gemv_set_end_combine": (_int, [_u32]),
     "boost_gemv_chain_workspace_bytes": (C.c_size_t, [_vp, _u32, _u32]),
     "boost_gemv_tiered_chain": (_int, [_vp, _u32, _u32, _vp, _sz, _vp]),
@@ -412,6 +413,10 @@ def gemv_calls(calls):
 
 def boost_gemv_set_tc_min_batch(m_b):
     _check(lib().boost_gemv_set_tc_min_batch(m_b), "boost_gemv_set_tc_min_batch")
+
+
+def boost_gemv_set_tier_schedule(two_queues):
+    _check(lib().boost_gemv_set_tier_schedule(1 if two_queues else 0), "boost_gemv_set_tier_schedule")
 
 
 class VABuffer:

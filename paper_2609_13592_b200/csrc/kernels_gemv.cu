@@ -118,6 +118,22 @@ __device__ __forceinline__ uint32_t even_part_segments(const GemvParams& p, uint
   return part_owner(u0 + p.k_blocks - 1, p.active_ctas, T2) - part_owner(u0, p.active_ctas, T2) + 1;
 }
 
+// Schedule log only: bytes of blocks [b, b + n) (one row tile's consecutive blocks) that lie in
+// host-tier pages.  The host pages of a weight are the first n_host_pages entries of w_order.
+__device__ __noinline__ uint32_t host_bytes_of_blocks(const GemvParams& p, uint32_t b, uint32_t n) {
+  uint32_t bytes = 0;
+  while (n) {
+    const uint32_t page = b / kBlocksPerPage;
+    const uint32_t here = min(n, kBlocksPerPage - b % kBlocksPerPage);
+    bool host = false;
+    for (uint32_t i = 0; i < p.n_host_pages && !host; ++i) host = p.w_order[i] == page;
+    if (host) bytes += here * kBlockBytes;
+    b += here;
+    n -= here;
+  }
+  return bytes;
+}
+
 // A launch runs one product, or a chain of up to kMaxPhases products in which each takes the
 // previous one's output (as its x, its residual or its row statistics).  The threadblocks stay
 // resident; between two phases they meet at a grid-wide counter, and because weights do not
@@ -527,9 +543,11 @@ __global__ void __launch_bounds__(kGemvThreads, (NT >= 8 ? 1 : 2)) gemv_tiered_k
                   page_base = static_cast<const uint8_t*>(p.w_page_ptr[page_of_base]);
                 }
                 const uint8_t* src = page_base + (size_t)(b % kBlocksPerPage) * kBlockBytes;
-                if (seg_first)   // the segment: blocks up to the end of the row tile or of this threadblock's range
+                if (seg_first && sched_log) {   // the segment: blocks up to the end of the row tile or of this threadblock's range
+                  const uint32_t n_seg_blocks = min(b1 - b, p.k_blocks - kb);
                   rec = sched_log_begin(sched_log, BOOST_SCHED_KIND_GEMV | (ph << 8), blockIdx.x | (warp << 24),
-                                        min(b1 - b, p.k_blocks - kb) * kBlockBytes, 0u);
+                                        n_seg_blocks * kBlockBytes, p.n_host_pages ? host_bytes_of_blocks(p, b, n_seg_blocks) : 0u);
+                }
                 meta[stage] = make_uint4(row_tile, seg, (seg_first ? kFlagFirst : 0u) | (seg_last ? kFlagLast : 0u) | (rec << 8), ph);
                 mbar_arrive_expect_tx(&full_bar[stage], kBlockBytes);
                 bulk_copy_g2s(wdst, src, kBlockBytes, &full_bar[stage]);
@@ -1142,9 +1160,16 @@ __global__ void __launch_bounds__(kTcThreads, 1) gemv_tc_kernel(const __grid_con
                 }
                 src[h] = page_base[h] + (size_t)(b % kBlocksPerPage) * kBlockBytes;
               }
-              if (seg_first)   // the segment: units up to the end of the row tile (pair) or of this threadblock's range
+              if (seg_first && sched_log) {   // the segment: units up to the end of the row tile (pair) or of this threadblock's range
+                const uint32_t n_seg_units = min(u1 - u, p.k_blocks - kb);
+                uint32_t host_bytes = 0;
+                if (p.n_host_pages) {
+                  host_bytes = host_bytes_of_blocks(p, tpu * pair * p.k_blocks + kb, n_seg_units);
+                  if (second) host_bytes += host_bytes_of_blocks(p, (tpu * pair + 1) * p.k_blocks + kb, n_seg_units);
+                }
                 rec = sched_log_begin(sched_log, BOOST_SCHED_KIND_GEMV | (ph << 8), blockIdx.x | (warp << 24),
-                                      min(u1 - u, p.k_blocks - kb) * (second ? 2u : 1u) * kBlockBytes, 0u);
+                                      n_seg_units * (second ? 2u : 1u) * kBlockBytes, host_bytes);
+              }
             }
             produce(src[0], src[1], false, tpu * pair, seg,
                     kFlagPair | (second ? kFlagSecond : 0u) | (seg_first ? kFlagFirst : 0u) | (seg_last ? kFlagLast : 0u), kb);
@@ -1487,6 +1512,8 @@ uint32_t pick_run(uint32_t n_row_tiles, uint32_t k_blocks) {
 
 // Combine-at-phase-end on (1) or off (0: every tile by its last arriver), for measurements; and
 // whether the last phase's combine goes to a kernel of its own.
+// 0: host pages are read in place under the even partition; 1: two queues of work items, host pages first
+uint32_t g_tier_schedule = 0;
 uint32_t g_end_combine = 1;
 uint32_t g_defer_combine = 1;
 
@@ -1787,7 +1814,7 @@ int fill_params(GemvParams& p, const void* const* w_page_ptr, const uint32_t* w_
   p.k_blocks = lay.k_blocks;
   p.run = lay.blocks_per_item;
   p.splits = lay.splits;
-  p.even_part = n_host_pages == 0 ? 1u : 0u;
+  p.even_part = (n_host_pages == 0 || g_tier_schedule == 0) ? 1u : 0u;
   p.total_blocks = lay.n_row_tiles * lay.k_blocks;
   p.max_seg = partial_slots(lay, M_b);
   p.tiles_per_unit = 1;
@@ -1928,5 +1955,13 @@ extern "C" int boost_gemv_set_tc_min_batch(uint32_t m_b) {
 // the phase by all threadblocks when a row tile has many (the default), 0 = always tile by tile.
 extern "C" int boost_gemv_set_end_combine(uint32_t on) {
   g_end_combine = on ? 1u : 0u;
+  return BOOST_OK;
+}
+
+// How a weight with host pages is scheduled (measurement and tests): 0 = its host pages are read
+// in place by the threadblocks whose share of the even partition holds them (the default), 1 = two
+// queues of work items, host pages first.
+extern "C" int boost_gemv_set_tier_schedule(uint32_t two_queues) {
+  g_tier_schedule = two_queues ? 1u : 0u;
   return BOOST_OK;
 }

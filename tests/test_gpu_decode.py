@@ -149,14 +149,18 @@ def dump_cache(dev, dec, li, name):
 
 @pytest.mark.parametrize("n_seq,kv_modulus,host_weights,recycle", [
     (3, 4, True, False), (1, 0, False, False), (20, 2, True, False), (40, 4, True, False), (6, 4, False, True),
-    (2, 4, True, True), (70, 2, True, False), (150, 2, False, False), (256, 4, True, False)])
+    (2, 4, True, True), (70, 2, True, False), (150, 2, False, False), (256, 4, True, False),
+    (3, 4, "two_queues", False), (24, 2, "two_queues", False), (70, 2, "two_queues", False)])
 def test_decode_steps_match_oracle(dev, n_seq, kv_modulus, host_weights, recycle):
     """16 consecutive decode steps of the tiny model against the oracle.  host_weights: every weight
     matrix has its (only) page in host memory, so all products of the chain take the host-tier
-    queue path; otherwise all weights are in HBM (even partition).  kv_modulus > 0 puts KV pages on
+    path (read in place under the even partition; "two_queues": the two-queue schedule, host pages
+    first); otherwise all weights are in HBM (even partition).  kv_modulus > 0 puts KV pages on
     the host as the pool places them.  Batch 1 - 2 is the CUDA-core kernel, 3 - 32 mma.sync, 40 and
     70 the tcgen05 kernel, 150 and 256 (the largest batch a step takes) its 256-column form."""
     from tests.helpers import chain_error
+    B.boost_gemv_set_tier_schedule(host_weights == "two_queues")   # (reset at the end of the test)
+    host_weights = bool(host_weights)
     cfg = dict(synth.TINY_LLAMA)
     w = synth.llama_weights(cfg, seed=n_seq, std=0.02)
     hkv, d, nl = cfg["n_kv_heads"], cfg["head_dim"], cfg["n_layers"]
@@ -234,6 +238,7 @@ def test_decode_steps_match_oracle(dev, n_seq, kv_modulus, host_weights, recycle
                     now[:, blk, slot] = host[li][:, blk, slot]
                 assert np.array_equal(now, host[li])       # nothing else was written
         tokens = ref["next_tokens"].astype(np.int32)       # both sides continue from the oracle's choice
+    B.boost_gemv_set_tier_schedule(False)
     assert dec.status_words() == [0, 0]
     assert exact_rows >= 0.6 * total_rows, (exact_rows, total_rows)
     if kv_modulus:
@@ -513,8 +518,18 @@ def test_config5_launch_shape_matches_oracle_on_samples(dev):
     assert dec.status_words() == [0, 0]
 
 
+@pytest.fixture
+def two_queue_schedule(request):
+    """The weight products of the test run under the schedule the parameter names (True: two queues,
+    host pages first; False: host pages read in place); the default comes back afterwards."""
+    B.boost_gemv_set_tier_schedule(bool(request.param))
+    yield bool(request.param)
+    B.boost_gemv_set_tier_schedule(False)
+
+
+@pytest.mark.parametrize("two_queue_schedule", [False, True], indirect=True)
 @pytest.mark.parametrize("m_b", [1, 24, 70])
-def test_gemv_chain_matches_separate_launches_and_oracle(dev, m_b):
+def test_gemv_chain_matches_separate_launches_and_oracle(dev, m_b, two_queue_schedule):
     """boost_gemv_tiered_chain: four dependent products in one launch (output product with
     residual and row statistics -> gate/up with row scale and SwiGLU -> down product with
     residual and statistics -> a scaled product with fp32 output and a ragged row count) give
@@ -583,8 +598,9 @@ def test_gemv_chain_matches_separate_launches_and_oracle(dev, m_b):
 
     # The same workspace reused by launches that follow each other on the stream with nothing in
     # between (no synchronise, no other kernel): a launch's threadblocks become resident while the
-    # one before drains, and must not touch the queue words (all four weights have host pages, so
-    # every product runs off the queues) before it has finished.  Chains of four and of one.
+    # one before drains, and must not touch the queue words (all four weights have host pages: under
+    # the two-queue schedule every product runs off the queues) before it has finished.  Chains of
+    # four and of one.
     assert all(tw.buf.n_host > 0 for tw in w)
     sets = [buffers() for _ in range(8)]
     arrs = [B.gemv_calls(calls_for(b)) for b in sets]

@@ -92,10 +92,13 @@ def test_stream_reduce_schedule(dev):
     attach(ws, ws_ptr, None)
 
 
-def test_gemv_chain_and_attention_schedule(dev):
+@pytest.mark.parametrize("two_queues", [False, True])
+def test_gemv_chain_and_attention_schedule(dev, two_queues):
     from paper_2609_13592_b200.tiers import TieredKVCache, TieredWeight, aligned_workspace
-    # a two-product chain: the first weight has a host page (queue items), the second is all HBM
-    # (even partition: one record per threadblock and row tile it touches)
+    # a two-product chain: the first weight has a host page (read in place under the even
+    # partition, or cut into queue items handed out host first), the second is all HBM (even
+    # partition: one record per threadblock and row tile it touches)
+    B.boost_gemv_set_tier_schedule(two_queues)
     m_b, kin, hid, ffn, stride = 32, 2048, 2048, 2048, 128
     t8 = lambda *t: np.array(t, np.uint8)
     w0 = TieredWeight(bf16_tensor(synth.normal_bf16((hid, kin), 0.03, 5), dev), device=dev, tier=t8(0, 1, 0, 0))
@@ -136,6 +139,7 @@ def test_gemv_chain_and_attention_schedule(dev):
     # the second product's weights start streaming before the first product's last item is consumed
     assert recs[phase == 1]["t_request"].min() < recs[phase == 0]["t_consumed"].max()
     attach(ws_t, ws_ptr, None)
+    B.boost_gemv_set_tier_schedule(False)
 
     # attention over a pool with a quarter of its pages on the host: records per warp and item
     n_seq, hq, hkv, d, n_blocks, modulus = 6, 8, 2, 128, 2048, 4

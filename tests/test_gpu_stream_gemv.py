@@ -26,6 +26,15 @@ def dev():
     return torch.device("cuda:0")
 
 
+@pytest.fixture(autouse=True, params=["in_place", "two_queues"])
+def tier_schedule(request, dev):
+    """Every test of this file runs under both schedules of a weight with host pages: read in
+    place under the even partition (the default), and the two queues with host pages first."""
+    B.boost_gemv_set_tier_schedule(request.param == "two_queues")
+    yield request.param
+    B.boost_gemv_set_tier_schedule(False)
+
+
 def bf16_tensor(bits, dev):
     return torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).to(dev).view(torch.bfloat16)
 
