@@ -37,8 +37,8 @@ FALLBACK_HBM_GBS = 6650.0
 # DRAM bytes (read + write) per algorithmic byte of the weight-product kernel, from one ncu
 # capture of two full-size chain launches of this workload (profiles/
 # gemv_tiered_kernel_chain_llama8b_m32.md): 1955.5 MB moved for 1872.8 MB of packed weights.
-GEMV_TRAFFIC_PER_ALGORITHMIC_BYTE = 1.044
-GEMV_TRAFFIC_PROFILE = "profiles/gemv_tiered_kernel_chain_llama8b_m32.md (captured at commit 7ba48f1; the kernel on this path is unchanged since)"
+GEMV_TRAFFIC_PER_ALGORITHMIC_BYTE = 1.046
+GEMV_TRAFFIC_PROFILE = "profiles/gemv_tiered_kernel_chain_llama8b_m32.md (captured at commit 9e981ac)"
 # the tcgen05 kernel (batches above 32), same kind of capture at batch 128: (511.7 + 1610.7) MB moved for
 # (436.2 + 1436.6) MB of packed weights
 GEMV_TC_TRAFFIC_PER_ALGORITHMIC_BYTE = 1.133
@@ -550,7 +550,7 @@ def run_ours(args, rank, world, local_rank):
                          "achieved": gemv_gbs, "peak": hbm_peak, "unit": "GB/s", "frac": gemv_gbs / hbm_peak,
                          "algorithmic_bytes_per_launch": gemv_bytes_per_launch,
                          "traffic": (GEMV_TRAFFIC_PER_ALGORITHMIC_BYTE if batch <= 32 else GEMV_TC_TRAFFIC_PER_ALGORITHMIC_BYTE) * gemv_bytes_per_launch,
-                         "traffic_source": ("ncu dram bytes of this workload's launches, ratio 1.044 to algorithmic" if batch <= 32 else
+                         "traffic_source": ("ncu dram bytes of this workload's launches, ratio 1.046 to algorithmic" if batch <= 32 else
                                             "ncu dram bytes of the same chains at batch 128, ratio 1.133 to algorithmic"),
                          "launches_per_step": gemv_n, "avg_launch_us": 1e3 * gemv_ms / max(gemv_n, 1),
                          "peak_source": peak_src,
