@@ -243,13 +243,14 @@ def run_reference_configs(args):
 
 # ------------------------------------------------------------------------------ device leg
 
-def measure_stream(dev, n_pages, tier_value, reps=5):
-    """GB/s of the tiered stream-reduce kernel over n_pages pages all in one tier."""
+def measure_stream(dev, n_pages, tier_value, reps=5, peer_device=None):
+    """GB/s of the tiered stream-reduce kernel over n_pages pages all in one tier (the second
+    tier: pinned host memory, or a peer GPU's memory when peer_device is given)."""
     import torch
     from paper_2609_13592_b200 import binding as B
     from paper_2609_13592_b200.tiers import TieredBuffer
     tier = np.full(n_pages, tier_value, np.uint8)
-    buf = TieredBuffer(n_pages * B.PAGE_BYTES, device=dev, tier=tier)
+    buf = TieredBuffer(n_pages * B.PAGE_BYTES, device=dev, tier=tier, peer_device=peer_device)
     ws_bytes = B.boost_stream_reduce_workspace_bytes(n_pages)
     ws = torch.zeros(ws_bytes, dtype=torch.uint8, device=dev)
     sums = torch.zeros(n_pages, dtype=torch.float32, device=dev)
@@ -839,6 +840,82 @@ def run_gemv_sweep(args):
                       "host_link_gbs": link, "points": points}))
 
 
+def run_peer_tier(args):
+    """The second tier in a peer GPU's HBM, read over NVLink (the paper's bandwidth-ratio
+    ablation): one process, GPU 0 computes, GPU 1 only holds pages.  Measures the peer-read
+    bandwidth with the stream-reduce kernel, derives the modulus from it, and compares tiered
+    with HBM-only runs of the stream reduce and of two weight products.  Needs two GPUs with peer
+    access; prints an `unavailable` line otherwise.  Prints one JSON document."""
+    import torch
+    from paper_2609_13592_b200 import binding as B
+    from paper_2609_13592_b200 import build as libbuild
+    from paper_2609_13592_b200.tiers import TieredBuffer, TieredWeight
+    if torch.cuda.device_count() < 2:
+        print(json.dumps({"workload": "peer_gpu_second_tier", "unavailable": "needs two GPUs in one process; this box shows %d" % torch.cuda.device_count()}))
+        return
+    libbuild.build_library()
+    B.lib()
+    dev = torch.device("cuda:0")
+    torch.cuda.set_device(dev)
+    torch.zeros(1, device=dev)
+    try:
+        B.boost_peer_tier_open(1)
+    except B.BoostError as e:
+        print(json.dumps({"workload": "peer_gpu_second_tier", "unavailable": "no peer access from GPU 0 to GPU 1: %s" % e}))
+        return
+    hbm_peak, peak_src = load_peaks()
+    link = measure_stream(dev, 512, 1, peer_device=1)
+    modulus = B.boost_modulus_from_bandwidths(hbm_peak, link)
+    out = {"workload": "peer_gpu_second_tier", "hbm_peak_gbs": hbm_peak, "hbm_peak_source": peak_src, "peer_read_gbs": link,
+           "alpha": link / (hbm_peak + link), "modulus": modulus, "stream": [], "weight_products": []}
+
+    def time_us(fn, reps):
+        for _ in range(3):
+            fn()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            fn()
+        e1.record()
+        torch.cuda.synchronize(dev)
+        return e0.elapsed_time(e1) * 1e3 / reps
+
+    n_pages = 2048   # 4 GiB: larger than L2 many times over
+    for label, ratio in (("hbm_only", 0.0), ("1/%d" % modulus, 1.0 / modulus), ("1/%d" % max(2, modulus // 2), 1.0 / max(2, modulus // 2))):
+        buf = TieredBuffer(n_pages * B.PAGE_BYTES, ratio, B.POLICY_MODULO, device=dev, peer_device=1)
+        ws_bytes = B.boost_stream_reduce_workspace_bytes(n_pages)
+        ws = torch.zeros(ws_bytes, dtype=torch.uint8, device=dev)
+        sums = torch.zeros(n_pages, dtype=torch.float32, device=dev)
+        us = time_us(lambda: B.boost_stream_reduce_tiered(buf.page_ptr, buf.order, n_pages, buf.n_host, sums, ws, ws_bytes), 5)
+        out["stream"].append({"placement": label, "peer_pages": buf.n_host, "us": us, "gbs": n_pages * B.PAGE_BYTES / us / 1e3,
+                              "status": int(ws[:4].cpu().numpy().view(np.uint32)[0])})
+        del buf
+    g = torch.Generator(device=dev)
+    g.manual_seed(5)
+    for name, (n, k) in {"gate_up": (28672, 4096), "lm_head": (128256, 4096)}.items():
+        n_copies = max(2, int(np.ceil(2 * 126e6 / (n * k * 2))))
+        for label, ratio in (("hbm_only", 0.0), ("1/%d" % modulus, 1.0 / modulus)):
+            ws_ = [TieredWeight((0.02 * torch.randn(n, k, generator=g, device=dev)).to(torch.bfloat16), ratio, device=dev, peer_device=1)
+                   for _ in range(n_copies)]
+            for mb in (1, 32, 128):
+                x = torch.randn(mb, k, generator=g, device=dev).to(torch.bfloat16)
+                y = torch.empty(mb, n, dtype=torch.bfloat16, device=dev)
+                for sched in ((0, 1) if ratio else (0,)):
+                    B.boost_gemv_set_tier_schedule(sched)
+
+                    def all_copies():
+                        for w in ws_:
+                            w.gemv(x, y=y)
+                    us = time_us(all_copies, 5) / n_copies
+                    out["weight_products"].append({"matrix": name, "batch": mb, "placement": label, "peer_pages": ws_[0].buf.n_host,
+                                                   "schedule": "two queues" if sched else "in place", "us": us,
+                                                   "gbs": ws_[0].layout["bytes"] / us / 1e3, "status": ws_[0].status_words()})
+                B.boost_gemv_set_tier_schedule(0)
+            del ws_
+            torch.cuda.empty_cache()
+    print(json.dumps(out))
+
+
 def run_stream_sweep(args):
     """Configuration 3: tiered streaming-read sweep.  A bf16 buffer of 1 / 4 / 16 (/ 64) GiB is
     reduced by the stream-reduce kernel (full waves of 4 threadblocks per SM) with the host
@@ -942,12 +1019,13 @@ def main():
     ap.add_argument("--ctx", type=int, default=2048)
     ap.add_argument("--layers", type=int, default=0, help="override the layer count (0 = 32)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--workload", default="decode", choices=["decode", "stream_sweep", "kv_spill", "gemv_sweep", "pool_churn", "oracle_configs"],
+    ap.add_argument("--workload", default="decode", choices=["decode", "stream_sweep", "kv_spill", "gemv_sweep", "pool_churn", "peer_tier", "oracle_configs"],
                     help="decode: the benchmark line; stream_sweep: the placement sweep of configuration 3; "
                          "kv_spill: configuration 5 (batch 128, one KV page in five on the host) with its "
                          "HBM-only and prefetch-to-HBM comparison runs; gemv_sweep: weight products over shapes, "
                          "batch sizes and host shares; pool_churn: the KV pool under serving-like arrivals, realised host "
-                         "share over time and attention timed on churned against fresh layouts; oracle_configs (with --impl reference): the CPU oracle timed on "
+                         "share over time and attention timed on churned against fresh layouts; peer_tier: the second tier in a peer GPU's HBM "
+                         "over NVLink (needs two GPUs in one process); oracle_configs (with --impl reference): the CPU oracle timed on "
                          "configurations 1 - 3")
     ap.add_argument("--churn-steps", type=int, default=12000, help="pool_churn: decode steps replayed")
     ap.add_argument("--sweep-gib", default="1,4,16")
@@ -971,6 +1049,9 @@ def main():
     elif args.workload == "stream_sweep":
         if rank == 0:
             run_stream_sweep(args)
+    elif args.workload == "peer_tier":
+        if rank == 0:
+            run_peer_tier(args)
     elif args.impl == "reference" and args.workload == "oracle_configs":
         if rank == 0:
             run_reference_configs(args)

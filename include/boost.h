@@ -208,6 +208,27 @@ int boost_va_buffer_destroy(boost_va_buffer_t* buffer);
  * pointer is not pinned host memory that the current device can address. */
 int boost_host_device_pointer(void* pinned_host, void** device_ptr_out /*host*/);
 
+/* A peer GPU's HBM as the second tier ("Bandwidth Ratio Ablation with NVLinks": the same
+ * placement with the second tier behind NVLink instead of the CPU link, where the bandwidth
+ * ratio is around 10 % instead of 1 %).  Pages of the second tier then live in a slab on
+ * peer_device; their addresses go into the page table through boost_page_table's host_slab
+ * argument and every kernel of this library reads them as it reads pinned host memory: each
+ * threadblock with its own copies into its own shared memory.  The modulus for such a tier is
+ * boost_modulus_from_bandwidths(hbm, link) with the measured peer-read bandwidth.
+ *   boost_peer_tier_open   lets kernels of the current device read peer_device's memory
+ *                          (idempotent);
+ *   boost_peer_tier_alloc  allocates `bytes` in peer_device's HBM; slab_out receives the
+ *                          address (valid on both devices once opened; the caller aligns it to
+ *                          2 MiB as for any slab); the caller's current device is unchanged;
+ *   boost_peer_tier_free   releases such a slab (NULL is accepted).
+ * Errors: INVALID (peer_device out of range or the current device itself, NULL / zero
+ * arguments), UNSUPPORTED (no peer access between the two devices), CAPACITY (out of memory
+ * on the peer), CUDA.  One process per GPU: the peer's slab is owned by the process that
+ * allocated it. */
+int boost_peer_tier_open(int peer_device);
+int boost_peer_tier_alloc(int peer_device, size_t bytes, void** slab_out /*host*/);
+int boost_peer_tier_free(int peer_device, void* slab /*device*/);
+
 /* Page base addresses for a placed tensor (the analogue of binding each 2 MiB region to a
  * memory node, Sec. 4.4).  HBM pages take consecutive 2 MiB slots of hbm_slab, host pages
  * consecutive slots of host_slab, both in page order.

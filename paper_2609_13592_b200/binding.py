@@ -114,6 +114,9 @@ SIGNATURES = {
     "boost_wave_stats": (_int, [_vp, _sz, _sz, _u32, _dbl, _vp]),
     "boost_tier_order": (_int, [_vp, _sz, _vp, _vp]),
     "boost_host_device_pointer": (_int, [_vp, _vp]),
+    "boost_peer_tier_open": (_int, [C.c_int]),
+    "boost_peer_tier_alloc": (_int, [C.c_int, C.c_size_t, _vp]),
+    "boost_peer_tier_free": (_int, [C.c_int, _vp]),
     "boost_page_table": (_int, [_vp, _sz, _vp, _sz, _vp, _sz, _vp]),
     "boost_scatter_pages": (_int, [_vp, _sz, _vp, _sz, _vp]),
     "boost_gather_pages": (_int, [_vp, _sz, _vp, _sz, _vp]),
@@ -276,6 +279,21 @@ def boost_host_device_pointer(pinned):
     out = C.c_void_p(0)
     _check(lib().boost_host_device_pointer(_ptr(pinned), C.addressof(out)), "boost_host_device_pointer")
     return out.value or 0
+
+
+def boost_peer_tier_open(peer_device):
+    _check(lib().boost_peer_tier_open(int(peer_device)), "boost_peer_tier_open")
+
+
+def boost_peer_tier_alloc(peer_device, n_bytes):
+    """-> address of a slab of n_bytes in peer_device's memory."""
+    out = C.c_void_p(0)
+    _check(lib().boost_peer_tier_alloc(int(peer_device), int(n_bytes), C.addressof(out)), "boost_peer_tier_alloc")
+    return out.value or 0
+
+
+def boost_peer_tier_free(peer_device, slab):
+    _check(lib().boost_peer_tier_free(int(peer_device), slab or None), "boost_peer_tier_free")
 
 
 def boost_page_table(tier, hbm_slab, hbm_slab_bytes, host_slab, host_slab_bytes):

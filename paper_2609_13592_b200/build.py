@@ -8,7 +8,7 @@ CSRC = os.path.join(PKG_DIR, "csrc")
 LIB_PATH = os.path.join(PKG_DIR, "libboost_b200.so")
 
 SOURCES = ["host_placement.cpp", "host_pool.cpp", "kernels_stream.cu", "kernels_gemv.cu",
-           "kernels_attn.cu", "kernels_glue.cu", "decode_step.cu", "va_buffer.cu"]
+           "kernels_attn.cu", "kernels_glue.cu", "decode_step.cu", "va_buffer.cu", "peer_tier.cu"]
 
 
 def sources():

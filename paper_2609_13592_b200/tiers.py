@@ -23,21 +23,46 @@ class Slabs:
     """An HBM slab and a pinned host slab that several TieredBuffers may map their pages onto
     (for placement sweeps, where only the page table changes between runs)."""
 
-    def __init__(self, hbm_pages, host_pages, device="cuda"):
+    def __init__(self, hbm_pages, host_pages, device="cuda", peer_device=None):
         self.device = torch.device(device)
         self.hbm_pages, self.host_pages = hbm_pages, host_pages
         self._hbm = torch.empty(hbm_pages * PAGE + PAGE, dtype=torch.uint8, device=self.device)
         self.hbm_base = _aligned(self._hbm)
-        self._host = torch.empty(max(host_pages, 1) * PAGE + PAGE, dtype=torch.uint8, pin_memory=True)
-        self.host_base_cpu = _aligned(self._host)
-        self.host_base = B.boost_host_device_pointer(self.host_base_cpu)
+        if peer_device is None:
+            self._host = torch.empty(max(host_pages, 1) * PAGE + PAGE, dtype=torch.uint8, pin_memory=True)
+            self.host_base_cpu = _aligned(self._host)
+            self.host_base = B.boost_host_device_pointer(self.host_base_cpu)
+        else:
+            self._host = PeerSlab(peer_device, max(host_pages, 1) * PAGE + PAGE)
+            self.host_base_cpu, self.host_base = 0, self._host.base
+
+
+class PeerSlab:
+    """Second-tier pages in a peer GPU's HBM (read over NVLink): a slab on peer_device that the
+    kernels of the current device may read.  Freed with the object."""
+
+    def __init__(self, peer_device, n_bytes):
+        self.peer_device = int(peer_device)
+        B.boost_peer_tier_open(self.peer_device)
+        self.ptr = B.boost_peer_tier_alloc(self.peer_device, n_bytes)
+        self.base = (self.ptr + PAGE - 1) // PAGE * PAGE
+
+    def __del__(self):
+        ptr, self.ptr = getattr(self, "ptr", 0), 0
+        if ptr:
+            try:
+                B.boost_peer_tier_free(self.peer_device, ptr)
+            except Exception:
+                pass
 
 
 class TieredBuffer:
     """A buffer of n_bytes cut into 2 MiB pages placed over HBM and pinned host memory."""
 
     def __init__(self, n_bytes, host_ratio=0.0, policy=B.POLICY_MODULO, seed=0, superpage_pages=1,
-                 device="cuda", tier=None, wave_size=0, slabs=None):
+                 device="cuda", tier=None, wave_size=0, slabs=None, peer_device=None):
+        """peer_device: ordinal of a second GPU whose HBM holds the second-tier pages instead of
+        pinned host memory (scatter_from / gather_to and the kernels work unchanged)."""
         self.n_bytes = int(n_bytes)
         self.device = torch.device(device)
         if tier is None:
@@ -58,6 +83,9 @@ class TieredBuffer:
             self.hbm_base = _aligned(self._hbm)
         if slabs is not None:
             pass
+        elif self.n_host and peer_device is not None:
+            self._host = PeerSlab(peer_device, self.n_host * PAGE + PAGE)
+            self.host_base_cpu, self.host_base = 0, self._host.base
         elif self.n_host:
             self._host = torch.empty(self.n_host * PAGE + PAGE, dtype=torch.uint8, pin_memory=True)
             self.host_base_cpu = _aligned(self._host)
@@ -94,13 +122,14 @@ class TieredWeight:
     """A row-major bf16 weight [N, K] packed into tiered pages for boost_gemv_tiered."""
 
     def __init__(self, w, host_ratio=0.0, policy=B.POLICY_MODULO, seed=0, device="cuda", tier=None,
-                 superpage_pages=1, row_mode=0, col_scale=None):
+                 superpage_pages=1, row_mode=0, col_scale=None, peer_device=None):
         """row_mode 1 interleaves the two halves of the rows (gate / up) per 64 rows; col_scale
         (bf16 [K]) is an RMSNorm weight folded into the matrix (see boost_pack_weights_ex)."""
         assert w.dtype == torch.bfloat16 and w.dim() == 2 and w.is_cuda and w.is_contiguous()
         self.N, self.K = int(w.shape[0]), int(w.shape[1])
         self.layout = B.boost_weight_layout(self.N, self.K)
-        self.buf = TieredBuffer(self.layout["bytes"], host_ratio, policy, seed, superpage_pages, device, tier)
+        self.buf = TieredBuffer(self.layout["bytes"], host_ratio, policy, seed, superpage_pages, device, tier,
+                                peer_device=peer_device)
         B.boost_pack_weights_ex(w, self.N, self.K, self.buf.page_ptr, self.buf.n_pages, row_mode, col_scale)
         torch.cuda.current_stream().synchronize()
         self._ws = {}
