@@ -2,15 +2,19 @@
 // kernel that packs a row-major weight into its paged 16 KiB-block form.
 //
 // Persistent threadblocks (two per SM for the mma.sync kernel, one for the tcgen05 kernel).  A
-// weight producer warp fills a ring of shared-memory stages: a 16 KiB weight block arrives by one
-// bulk copy through the TMA unit when its page is in HBM, or by a deep fan of 16-byte cp.async
-// loads when the page is host memory behind the CPU-GPU link; an activation producer warp adds
-// the matching 64-column slice of x.  Consumer warps multiply from shared memory: on CUDA cores
-// with warp-shuffle reductions for batches of 1 and 2, with mma.sync bf16 tensor-core MMAs up to
-// 32 rows, with tcgen05 MMAs into tensor memory above.  A weight with host pages is cut into work
-// items (runs of blocks of one row tile inside one page, host-tier items first, Sec. 3.2), so a
-// threadblock reads one tier at a time; a weight entirely in HBM is cut evenly over the
-// threadblocks.  Split-K partial sums meet in L2 and are combined in a fixed order.
+// weight producer warp fills a ring of shared-memory stages, one 16 KiB weight block per bulk copy
+// through the TMA unit; an activation producer warp adds the matching 64-column slice of x.
+// Consumer warps multiply from shared memory: on CUDA cores with warp-shuffle reductions for
+// batches of 1 and 2, with mma.sync bf16 tensor-core MMAs up to 32 rows, with tcgen05 MMAs into
+// tensor memory above.  Two schedules.  The default cuts every weight evenly over the
+// threadblocks, a contiguous share of the packed matrix each; blocks that lie in host pages are
+// read in place by the same bulk copies (they read pinned host memory as they read HBM), more
+// slowly, by whichever threadblock's share holds them - modulo placement spreads the host pages
+// over the matrix, so the link works from the start of the launch.  The other is the paper's
+// (Sec. 3.2; boost_gemv_set_tier_schedule): a weight with host pages is cut into work items (runs
+// of blocks of one row tile inside one page) in two queues, host-tier items first and fetched by
+// deep fans of 16-byte cp.async loads, so a threadblock reads one tier at a time.  Split-K partial
+// sums meet in L2 and are combined in a fixed order.
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
