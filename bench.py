@@ -486,7 +486,8 @@ def run_ours(args, rank, world, local_rank):
             clocks = sampler.stop()
         r = {"ms": dist_ctx.max(ms), "launches": launches, "kv_tokens": kv_tokens, "kind_ms": kind_ms,
              "kind_n": kind_n, "weight_bytes": dec.weight_bytes(), "kv_bytes_per_token": dec.kv_bytes_per_token(),
-             "host_pages": dec.host_weight_pages(), "status": dec.status_words()}
+             "host_pages": dec.host_weight_pages(), "status": dec.status_words(),
+             "last_tokens": dec.last_tokens}
         if label == "tiered":
             e_ms, h2d, d2h = timed_host_steps(dec, dev, batch, ctx0, args.warmup, args.steps, max_blocks, dist_ctx)
             r.update(e2e_ms=dist_ctx.max(e_ms), h2d=h2d, d2h=d2h)
@@ -544,6 +545,9 @@ def run_ours(args, rank, world, local_rank):
             "hbm_only": {"ms_per_step": hb_ms, "value": world * batch / (hb_ms / 1e3),
                          "tiered_over_hbm_only_time": ms_step / hb_ms},
             "tiered_over_hbm_only_time": ms_step / hb_ms,
+            # same model, inputs and steps: with host pages read in place the work partition does not
+            # depend on the placement, so the tiered run must reproduce the HBM-only run's tokens
+            "tiered_tokens_equal_hbm_only": bool(np.array_equal(t["last_tokens"], results["hbm_only"]["last_tokens"])),
             "weight_tier_schedule": {"this_line": "host pages read in place under the even partition",
                                      "two_queues_host_first_ms_per_step": t["two_queue_ms"] / args.steps},
             "roofline": {"bound": "hbm", "kernel": (f"gemv_tiered_kernel (weight products, M_b = {batch})" if batch <= 32 else
