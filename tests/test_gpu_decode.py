@@ -247,6 +247,42 @@ def test_decode_steps_match_oracle(dev, n_seq, kv_modulus, host_weights, recycle
         assert info["live_host_chunks"] > 0, info
 
 
+@pytest.mark.parametrize("n_seq", [2, 12, 48, 150])
+def test_step_bits_do_not_depend_on_weight_placement(dev, n_seq):
+    """With host pages read in place the work partition of a product is the same wherever its
+    pages live, so a decode step whose weights all sit in host memory gives the same logits, bit
+    for bit, as the step with all weights in HBM (CUDA-core, mma.sync and both tcgen05 forms)."""
+    cfg = dict(synth.TINY_LLAMA)
+    w = synth.llama_weights(cfg, seed=77, std=0.02)
+    hkv, d, nl = cfg["n_kv_heads"], cfg["head_dim"], cfg["n_layers"]
+    n_pool_blocks, max_blocks = 2048, 8
+    rng = np.random.default_rng(5)
+    ctx = rng.integers(1, 60, size=n_seq).astype(np.int32)
+    table = np.zeros((n_seq, max_blocks), np.int32)
+    perm = rng.permutation(n_pool_blocks)[:n_seq * 4].reshape(n_seq, 4)
+    table[:, :4] = perm
+    tokens = rng.integers(0, cfg["vocab"], size=n_seq).astype(np.int32)
+    k_host = [synth.normal_bf16((hkv, n_pool_blocks, 16, d), 1.0, 300 + li) for li in range(nl)]
+    v_host = [synth.normal_bf16((hkv, n_pool_blocks, 16, d), 1.0, 400 + li) for li in range(nl)]
+    logits = []
+    for tier_fn in (None, first_page_on_host):
+        dec = build_decoder(dev, cfg, w, n_pool_blocks, 0, 0.0, max(n_seq, 4), max_blocks, weight_tier=tier_fn)
+        assert all((tw.buf.n_host > 0) == (tier_fn is not None) for tw in all_weights(dec))
+        load_caches(dev, dec, k_host, v_host)
+        nxt = np.zeros(n_seq, np.int32)
+        per_step = []
+        tok, c = tokens.copy(), ctx.copy()
+        for step in range(3):
+            dec.step_host(tok, table, c, nxt)
+            per_step.append(dec.buf["logits"][:n_seq].cpu().numpy().copy())
+            tok, c = nxt.copy(), c + 1
+        assert dec.status_words() == [0, 0]
+        logits.append(per_step)
+        del dec
+    for a_, b_ in zip(*logits):
+        assert np.isfinite(a_).all() and np.array_equal(a_, b_)
+
+
 def test_fused_product_epilogues_match_oracle(dev):
     """boost_gemv_tiered_fused: RMS row scale with folded norm weight + row statistics, SwiGLU,
     RoPE + KV append - each against the oracle's operators applied one after the other."""
