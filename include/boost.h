@@ -467,8 +467,9 @@ int boost_gemv_set_end_combine(uint32_t on);
  * tier while it has items (16-byte copies through the load/store path), the others on the HBM
  * queue.  Measured on a B200 whose host link carries 0.8 % of the HBM bandwidth, the in-place
  * form is as fast or faster for every Llama-3-8B matrix, batch size and host share tried, which
- * is why it is the default.  Results differ between the two in fp32 rounding (other partial
- * sums).  Process-wide; for measurement, tests and the comparison with the paper's schedule. */
+ * is why it is the default.  Under 0 the result of a product does not depend on where its pages
+ * live (the same bits for every tier table); results differ between the two settings in fp32
+ * rounding (other partial sums).  Process-wide; for measurement, tests and the comparison with the paper's schedule. */
 int boost_gemv_set_tier_schedule(uint32_t two_queues);
 
 /* boost_gemv_tiered with an epilogue descriptor (NULL = plain). */

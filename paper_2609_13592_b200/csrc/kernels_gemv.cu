@@ -930,7 +930,8 @@ __global__ void __launch_bounds__(kConsumerThreads) gemv_combine_kernel(const __
 // (tcgen05.ld), write the partial sums and run the same combine as the kernel above.
 // Warps: 0-11 epilogue (warp w reads TMEM lanes 32 (w % 4) .. + 31 = weight rows, and the third
 // w / 4 of the accumulator's 16-column chunks), 12 MMA issue and TMEM allocation, 13 weight
-// producer (bulk copies; 16-byte copies of all its lanes for host-tier blocks), 14 activation
+// producer (bulk copies; under the two-queue schedule 16-byte copies of all its lanes for
+// host-tier blocks), 14 activation
 // producer (one thread: a tiled TMA copy per stage lands x[:, 64 kb .. + 64) in the B operand's
 // swizzled layout, rows beyond the batch as zeros).  Twelve epilogue warps because the combine of
 // the partial sums is bound by what the warps of an SM can pull from L2 (eight: 163 us per chain
