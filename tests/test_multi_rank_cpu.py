@@ -42,3 +42,18 @@ def test_two_gloo_ranks_report_max_time_and_whole_job_value(tmp_path):
     assert out["world"] == 2 and out["ms"] == 15.0
     # two replicas of 32 sequences each, one token per sequence per step, at the slowest rank's pace
     assert abs(out["value"] - 2 * 32 / 0.015) < 1e-6
+
+
+def test_peer_tier_workload_says_unavailable_without_two_gpus():
+    """The peer-GPU second tier needs two GPUs in one process; anywhere else the workload must say
+    so in one JSON line and exit 0 instead of touching a device."""
+    import json
+    import pytest
+    torch = pytest.importorskip("torch")
+    if torch.cuda.is_available() and torch.cuda.device_count() >= 2:
+        pytest.skip("this box has two GPUs: the workload would run")
+    res = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--workload", "peer_tier"],
+                         capture_output=True, text=True, timeout=240)
+    assert res.returncode == 0, res.stdout + res.stderr
+    out = json.loads([l for l in res.stdout.splitlines() if l.startswith("{")][-1])
+    assert out["workload"] == "peer_gpu_second_tier" and "two GPUs" in out["unavailable"]
