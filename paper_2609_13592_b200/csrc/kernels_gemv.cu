@@ -189,18 +189,50 @@ struct RopeOperands {
   bool have = false;
   int32_t ctx = 0, blk = -1;
   float4 cs01 = make_float4(0.f, 0.f, 0.f, 0.f), cs23 = make_float4(0.f, 0.f, 0.f, 0.f);
+  // K / V heads with a valid block: where the two halves of the new row go (second pair: the
+  // optional second copy of the cache), looked up through the page tables
+  uint8_t* dst[4] = {nullptr, nullptr, nullptr, nullptr};
 };
-__device__ __forceinline__ RopeOperands load_rope_operands(const GemvParams& p, uint32_t row_tile, uint32_t m, uint32_t v) {
-  RopeOperands r;
-  r.have = true;
-  r.ctx = p.ctx_lens[m];
+// Byte offsets, inside the K (or V) tensor, of the two 8-byte pieces a lane writes for the new
+// token of a sequence: chunk (kvh, blk), token `slot` at slot * 256, 16-byte piece c at position
+// c ^ (slot & 7); the lane holds d = 4 v .. 4 v + 3 and d + 64.
+__device__ __forceinline__ void kv_append_offsets(const GemvParams& p, uint32_t kvh, uint32_t blk, uint32_t pos, uint32_t v,
+                                                  size_t& off1, size_t& off2) {
+  const uint32_t slot = pos % BOOST_KV_BLOCK_TOKENS, d = v * 4;
+  const size_t chunk = ((size_t)kvh * p.n_pool_blocks + blk) * 4096u + slot * 256u;
+  off1 = chunk + ((((d >> 3) ^ (slot & 7u))) << 4) + (d & 7u) * 2u;
+  off2 = chunk + (((((d + 64) >> 3) ^ (slot & 7u))) << 4) + (d & 7u) * 2u;
+}
+// Two parts.  Where the new row goes (context length -> block-table entry -> page addresses:
+// three dependent look-ups) depends only on the caller's inputs and the page tables, which no
+// kernel of this library writes: it may be fetched before the wait on the product.  The cos / sin
+// pairs come from a table that an earlier kernel of the same step writes: after the wait.
+__device__ __forceinline__ void load_rope_table(const GemvParams& p, uint32_t row_tile, uint32_t m, uint32_t v, RopeOperands& r) {
   if (row_tile < p.Hq + p.Hkv) {
     r.cs01 = __ldg(reinterpret_cast<const float4*>(p.rope_table + ((size_t)m * 64 + v * 4) * 2));
     r.cs23 = __ldg(reinterpret_cast<const float4*>(p.rope_table + ((size_t)m * 64 + v * 4 + 2) * 2));
   }
+}
+__device__ __forceinline__ RopeOperands load_rope_operands(const GemvParams& p, uint32_t row_tile, uint32_t m, uint32_t v) {
+  RopeOperands r;
+  r.have = true;
+  r.ctx = p.ctx_lens[m];
   if (row_tile >= p.Hq && r.ctx > 0) {
     const uint32_t bi = ((uint32_t)r.ctx - 1u) / BOOST_KV_BLOCK_TOKENS;
     r.blk = bi < p.max_blocks ? p.block_table[(size_t)m * p.max_blocks + bi] : -1;
+    if (r.blk >= 0 && (uint32_t)r.blk < p.n_pool_blocks) {
+      const bool is_k = row_tile < p.Hq + p.Hkv;
+      size_t off1, off2;
+      kv_append_offsets(p, is_k ? row_tile - p.Hq : row_tile - p.Hq - p.Hkv, (uint32_t)r.blk, (uint32_t)r.ctx - 1u, v, off1, off2);
+      const void* const* pages = is_k ? p.k_page_ptr : p.v_page_ptr;
+      r.dst[0] = static_cast<uint8_t*>(const_cast<void*>(pages[off1 / kPageBytes])) + off1 % kPageBytes;
+      r.dst[1] = static_cast<uint8_t*>(const_cast<void*>(pages[off2 / kPageBytes])) + off2 % kPageBytes;
+      const void* const* pages2 = is_k ? p.k_page_ptr2 : p.v_page_ptr2;
+      if (pages2) {
+        r.dst[2] = static_cast<uint8_t*>(const_cast<void*>(pages2[off1 / kPageBytes])) + off1 % kPageBytes;
+        r.dst[3] = static_cast<uint8_t*>(const_cast<void*>(pages2[off2 / kPageBytes])) + off2 % kPageBytes;
+      }
+    }
   }
   return r;
 }
@@ -301,16 +333,21 @@ __device__ __forceinline__ void finish_pair(const GemvParams& p, uint32_t row_ti
       } else {
         const bool is_k = head < p.Hq + p.Hkv;
         const uint32_t kvh = is_k ? head - p.Hq : head - p.Hq - p.Hkv;
-        const uint32_t bi = pos / BOOST_KV_BLOCK_TOKENS, slot = pos % BOOST_KV_BLOCK_TOKENS;
+        const uint32_t bi = pos / BOOST_KV_BLOCK_TOKENS;
         const int32_t blk = pre.have ? pre.blk : (bi < p.max_blocks ? p.block_table[(size_t)m * p.max_blocks + bi] : -1);
         if (blk < 0 || (uint32_t)blk >= p.n_pool_blocks) {
           atomicOr(status, kErrBadIndex);
+        } else if (pre.have) {
+          *reinterpret_cast<uint2*>(pre.dst[0]) = o1;
+          *reinterpret_cast<uint2*>(pre.dst[1]) = o2;
+          if (pre.dst[2]) {
+            *reinterpret_cast<uint2*>(pre.dst[2]) = o1;
+            *reinterpret_cast<uint2*>(pre.dst[3]) = o2;
+          }
         } else {
           const void* const* pages = is_k ? p.k_page_ptr : p.v_page_ptr;
-          // chunk (kvh, blk): token `slot` at slot*256, 16-byte piece c at position c ^ (slot & 7)
-          const size_t chunk = ((size_t)kvh * p.n_pool_blocks + (uint32_t)blk) * 4096u + slot * 256u;
-          const size_t off1 = chunk + ((((d >> 3) ^ (slot & 7u))) << 4) + (d & 7u) * 2u;
-          const size_t off2 = chunk + (((((d + 64) >> 3) ^ (slot & 7u))) << 4) + (d & 7u) * 2u;
+          size_t off1, off2;
+          kv_append_offsets(p, kvh, (uint32_t)blk, pos, v, off1, off2);
           *reinterpret_cast<uint2*>(static_cast<uint8_t*>(const_cast<void*>(pages[off1 / kPageBytes])) + off1 % kPageBytes) = o1;
           *reinterpret_cast<uint2*>(static_cast<uint8_t*>(const_cast<void*>(pages[off2 / kPageBytes])) + off2 % kPageBytes) = o2;
           const void* const* pages2 = is_k ? p.k_page_ptr2 : p.v_page_ptr2;
@@ -369,6 +406,7 @@ __device__ __forceinline__ void combine_units(const GemvParams& p, uint32_t firs
   const uint32_t slots_per_tile = combine_slots_per_tile<kXRows>(p);
   const uint32_t n_slots = tile_or_all == kAllTiles ? p.n_row_tiles * slots_per_tile : slots_per_tile;
   const bool vec_out = (p.N & 3u) == 0;
+  bool waited = false;   // (kRopeAhead: the caller has not waited for the product yet)
   for (uint32_t s = first; s < n_slots; s += step) {
     const uint32_t row_tile = tile_or_all == kAllTiles ? s / slots_per_tile : tile_or_all;
     const uint32_t i = tile_or_all == kAllTiles ? s - row_tile * slots_per_tile : s;
@@ -379,6 +417,19 @@ __device__ __forceinline__ void combine_units(const GemvParams& p, uint32_t firs
     const float4* base = reinterpret_cast<const float4*>(p.partials + (size_t)row_tile * p.max_seg * kXRows * kBlockRows) +
                          (live ? m : 0u) * kVecRow + v;
     // everything a lane needs from memory is requested before the first use
+    RopeOperands pre;
+    if constexpr (kRopeAhead) {
+      // Where the RoPE epilogue puts the new K / V row - context length, block-table entry, page
+      // addresses - is not written by the product or anything before it on the stream's chain of
+      // kernels: it is fetched (three dependent look-ups) while the product is still running, and
+      // only then does the warp wait for the product (once: later slots find it complete).
+      if (p.epi == kEpiRope && valid) pre = load_rope_operands(p, row_tile, m, v);
+      if (!waited) {
+        pdl_wait();
+        waited = true;
+      }
+      if (p.epi == kEpiRope && valid) load_rope_table(p, row_tile, m, v, pre);
+    }
     float ss = 0.f, ss0 = 0.f, ss1 = 0.f;
     if (p.ssq_in && valid) {
       if (v < p.ssq_in_tiles) ss0 = __ldcg(p.ssq_in + (size_t)v * p.ssq_stride + m);
@@ -392,10 +443,6 @@ __device__ __forceinline__ void combine_units(const GemvParams& p, uint32_t firs
         const uint32_t n = row_tile * kBlockRows + h * 64 + v * 4;
         if (n < p.N) res[h] = __ldcg(reinterpret_cast<const uint2*>(p.residual + (size_t)m * p.N + n));   // L2: an earlier phase may have rewritten it
       }
-    }
-    RopeOperands pre;
-    if constexpr (kRopeAhead) {
-      if (p.epi == kEpiRope && valid) pre = load_rope_operands(p, row_tile, m, v);
     }
     float4 lo = make_float4(0.f, 0.f, 0.f, 0.f), hi = lo;
     const uint32_t seg_first = pair_mode ? 0u : half, seg_step = pair_mode ? 1u : 2u;
@@ -915,7 +962,8 @@ __global__ void __launch_bounds__(kGemvThreads, (NT >= 8 ? 1 : 2)) gemv_tiered_k
 template <uint32_t kXRows>
 __global__ void __launch_bounds__(kConsumerThreads) gemv_combine_kernel(const __grid_constant__ GemvParams p) {
   pdl_launch_dependents();
-  pdl_wait();   // the product has completed: its partial sums are in memory
+  // (combine_units waits for the product - its partial sums in memory - after it has requested
+  // what does not depend on it)
   combine_units<kXRows, true>(p, blockIdx.x * kConsumerWarps + (threadIdx.x >> 5), gridDim.x * kConsumerWarps, kAllTiles,
                               threadIdx.x & 31u, p.ws + kWsStatus);
 }
