@@ -379,6 +379,28 @@ def test_fused_product_epilogues_match_oracle(dev):
         k_want[:, blk, slot] = k_now[:, blk, slot]
         v_want[:, blk, slot] = v_now[:, blk, slot]
     assert np.array_equal(k_now, k_want) and np.array_equal(v_now, v_want)   # nothing else was touched
+    # block-table entries that point outside the pool: recorded in the status word (bit 1), the row
+    # is not written anywhere, every other sequence's row is
+    bad = table.copy()
+    bad[2, pos[2] // 16] = n_blocks + 5
+    bad[3, pos[3] // 16] = -1
+    cache.load(bf16_tensor(k0, dev), bf16_tensor(v0, dev))
+    bad_d = torch.from_numpy(bad).to(dev)
+    wqkv.gemv(x, epilogue=epilogue(B.EPI_ROPE_APPEND, q_out=q_out.data_ptr(), k_page_ptr=cache.k.page_ptr.data_ptr(),
+                                   v_page_ptr=cache.v.page_ptr.data_ptr(), n_pool_blocks=n_blocks,
+                                   block_table=bad_d.data_ptr(), max_blocks=8, ctx_lens=ctx_d.data_ptr(),
+                                   n_q_heads=hq, n_kv_heads=hkv, rope_table=rope_table.data_ptr()))
+    torch.cuda.synchronize()
+    assert wqkv.status_words() == [2]
+    k_bad, v_bad = (bits_of(t) for t in cache.dump())
+    k_want2, v_want2 = k0.copy(), v0.copy()
+    for b in range(m_b):
+        if ctx[b] == 0 or b in (2, 3):
+            continue
+        blk, slot = table[b, pos[b] // 16], pos[b] % 16
+        k_want2[:, blk, slot] = k_now[:, blk, slot]
+        v_want2[:, blk, slot] = v_now[:, blk, slot]
+    assert np.array_equal(k_bad, k_want2) and np.array_equal(v_bad, v_want2)
     pool.close()
 
 
